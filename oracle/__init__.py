@@ -1,0 +1,197 @@
+"""CPU oracle for the MRP drafting step -- TEST INFRASTRUCTURE ONLY.
+
+Thin ctypes access to ``mrp_oracle.c`` (plain C, fp64 arithmetic, OpenMP over independent
+outputs).  Only tests, the smoke check and the benchmark's ``cpu_baseline`` / reference arm
+may import this package; the product path never does.  Nothing here touches CUDA.
+
+The functions mirror the paper's steps (Algorithms 2-4): ``draft`` runs the head chain and
+the shared LM head and returns per-step softmax statistics, ``select`` applies the static /
+dynamic reveal rules and the remask rule, ``verify`` computes accepted draft prefixes.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from dataclasses import dataclass
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "mrp_oracle.c")
+_LIB = os.path.join(_HERE, "libmrp_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile ``mrp_oracle.c`` into ``libmrp_oracle.so`` next to it (gcc, OpenMP)."""
+    if (not force and os.path.exists(_LIB)
+            and os.path.getmtime(_LIB) >= os.path.getmtime(_SRC)):
+        return _LIB
+    tmp = _LIB + ".tmp.%d" % os.getpid()
+    cmd = ["gcc", "-O2", "-std=c99", "-fopenmp", "-fPIC", "-shared", "-o", tmp, _SRC, "-lm"]
+    subprocess.run(cmd, check=True)
+    os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build())
+        _lib.mrp_oracle_num_threads.restype = ctypes.c_int
+        _lib.mrp_oracle_cap.restype = ctypes.c_int
+        _lib.mrp_oracle_cap.argtypes = [ctypes.c_int, ctypes.c_int]
+        _lib.mrp_oracle_draft.restype = ctypes.c_int
+        _lib.mrp_oracle_select.restype = ctypes.c_int
+        _lib.mrp_oracle_verify.restype = ctypes.c_int
+    return _lib
+
+
+def num_threads() -> int:
+    return int(_load().mrp_oracle_num_threads())
+
+
+def cap(n_masked: int, L: int) -> int:
+    """Max-accept cap m = min(max(floor(0.7 n), 5), L) (Sec. 4.4)."""
+    return int(_load().mrp_oracle_cap(int(n_masked), int(L)))
+
+
+def _f32(a):
+    return np.ascontiguousarray(np.asarray(a, dtype=np.float32))
+
+
+def _i32(a):
+    return np.ascontiguousarray(np.asarray(a, dtype=np.int32))
+
+
+def _p(a, ct):
+    return a.ctypes.data_as(ctypes.POINTER(ct)) if a is not None else None
+
+
+@dataclass
+class DraftResult:
+    conf: np.ndarray      # [(K+1), M] float64
+    lse: np.ndarray       # [(K+1), M] float64
+    token: np.ndarray     # [(K+1), M] int32
+    margin: np.ndarray    # [(K+1), M] float64, top-1 minus top-2 logit
+    logits: np.ndarray | None   # [K, M, V] float64
+    hidden: np.ndarray | None   # [M, d] float64
+
+
+def draft(hidden, logits0, heads, w_lm, K=None, row_index=None, eps=1e-6,
+          want_logits=False, want_hidden=False) -> DraftResult:
+    """Head chain + shared LM head + softmax statistics (Algorithm 2, inner loop).
+
+    ``heads`` is a sequence of dicts with float32-representable arrays ``gamma`` [d],
+    ``w_gate`` [F,d], ``w_up`` [F,d], ``w_down`` [d,F]; ``hidden`` [rows,d]; ``logits0``
+    [rows,V]; ``w_lm`` [V,d]; ``row_index`` selects the masked rows (None = all rows).
+    """
+    lib = _load()
+    hidden = _f32(hidden)
+    logits0 = _f32(logits0)
+    w_lm = _f32(w_lm)
+    n_rows, d = hidden.shape
+    V = w_lm.shape[0]
+    assert w_lm.shape[1] == d and logits0.shape == (n_rows, V)
+    K = len(heads) if K is None else int(K)
+    assert 0 <= K <= len(heads)
+    ri = None
+    M = n_rows
+    if row_index is not None:
+        ri = _i32(row_index)
+        M = ri.shape[0]
+        assert M == 0 or (ri.min() >= 0 and ri.max() < n_rows)
+    keep = []
+    F = heads[0]["w_gate"].shape[0] if len(heads) else 1
+    PtrArr = ctypes.POINTER(ctypes.c_float) * max(K, 1)
+    arrs = {}
+    for name, shape in (("gamma", (d,)), ("w_gate", (F, d)), ("w_up", (F, d)), ("w_down", (d, F))):
+        lst = []
+        for k in range(K):
+            a = _f32(heads[k][name])
+            assert a.shape == shape, (name, a.shape, shape)
+            keep.append(a)
+            lst.append(_p(a, ctypes.c_float))
+        arrs[name] = PtrArr(*lst) if K else PtrArr()
+    conf = np.zeros((K + 1, M), np.float64)
+    lse = np.zeros((K + 1, M), np.float64)
+    margin = np.zeros((K + 1, M), np.float64)
+    token = np.zeros((K + 1, M), np.int32)
+    logits = np.zeros((K, M, V), np.float64) if want_logits else None
+    hid = np.zeros((M, d), np.float64) if want_hidden else None
+    rc = lib.mrp_oracle_draft(
+        ctypes.c_int(d), ctypes.c_int(F), ctypes.c_int(V), ctypes.c_int(K), ctypes.c_int(M),
+        ctypes.c_double(eps), _p(hidden, ctypes.c_float), _p(logits0, ctypes.c_float),
+        _p(ri, ctypes.c_int32), arrs["gamma"], arrs["w_gate"], arrs["w_up"], arrs["w_down"],
+        _p(w_lm, ctypes.c_float), _p(conf, ctypes.c_double), _p(lse, ctypes.c_double),
+        _p(token, ctypes.c_int32), _p(margin, ctypes.c_double), _p(logits, ctypes.c_double),
+        _p(hid, ctypes.c_double))
+    if rc != 0:
+        raise RuntimeError("mrp_oracle_draft failed (%d)" % rc)
+    return DraftResult(conf, lse, token, margin, logits, hid)
+
+
+@dataclass
+class SelectResult:
+    reveal_mask: np.ndarray   # [B*L] int8
+    remask_mask: np.ndarray   # [B*L] int8
+    out_token: np.ndarray     # [B*L] int32
+    step_of: np.ndarray       # [B*L] int8
+    draft_pos: np.ndarray     # [B, Kd] int32
+    draft_tok: np.ndarray     # [B, Kd] int32
+    draft_len: np.ndarray     # [B] int32
+
+
+STATIC = 0
+DYNAMIC_REMASK = 1
+
+
+def select(conf, token, row_index, B, L, mode, tau=0.9, r_reveal=1, r_draft=1,
+           use_cap=False, remask_policy=0, ensure_progress=True) -> SelectResult:
+    """Static top-r reveal/draft or dynamic threshold reveal + remask (Algorithms 2-4)."""
+    lib = _load()
+    conf = _f32(conf)
+    token = _i32(token)
+    Kp1, M = conf.shape
+    assert token.shape == conf.shape
+    K = Kp1 - 1
+    ri = _i32(row_index) if row_index is not None else None
+    Kd = K * max(int(r_draft), 0)
+    out = SelectResult(
+        np.zeros(B * L, np.int8), np.zeros(B * L, np.int8), np.zeros(B * L, np.int32),
+        np.zeros(B * L, np.int8), np.zeros((B, Kd), np.int32), np.zeros((B, Kd), np.int32),
+        np.zeros(B, np.int32))
+    rc = lib.mrp_oracle_select(
+        _p(conf, ctypes.c_float), _p(token, ctypes.c_int32), _p(ri, ctypes.c_int32),
+        ctypes.c_int(M), ctypes.c_int(K), ctypes.c_int(B), ctypes.c_int(L), ctypes.c_int(mode),
+        ctypes.c_float(tau), ctypes.c_int(r_reveal), ctypes.c_int(r_draft),
+        ctypes.c_int(int(use_cap)), ctypes.c_int(int(remask_policy)),
+        ctypes.c_int(int(ensure_progress)),
+        _p(out.reveal_mask, ctypes.c_int8), _p(out.remask_mask, ctypes.c_int8),
+        _p(out.out_token, ctypes.c_int32), _p(out.step_of, ctypes.c_int8),
+        _p(out.draft_pos, ctypes.c_int32), _p(out.draft_tok, ctypes.c_int32),
+        _p(out.draft_len, ctypes.c_int32))
+    if rc != 0:
+        raise RuntimeError("mrp_oracle_select failed (%d)" % rc)
+    return out
+
+
+def verify(draft_tok, verify_tok, draft_len, positionwise=False):
+    """Accepted-prefix length of drafted tokens against backbone tokens (Algorithm 3)."""
+    lib = _load()
+    draft_tok = _i32(draft_tok)
+    verify_tok = _i32(verify_tok)
+    draft_len = _i32(draft_len)
+    B, Kd = draft_tok.shape
+    assert verify_tok.shape == (B, Kd) and draft_len.shape == (B,)
+    accept_len = np.zeros(B, np.int32)
+    accept_mask = np.zeros((B, Kd), np.int8)
+    rc = lib.mrp_oracle_verify(
+        _p(draft_tok, ctypes.c_int32), _p(verify_tok, ctypes.c_int32),
+        _p(draft_len, ctypes.c_int32), ctypes.c_int(B), ctypes.c_int(Kd),
+        ctypes.c_int(int(positionwise)), _p(accept_len, ctypes.c_int32),
+        _p(accept_mask, ctypes.c_int8))
+    if rc != 0:
+        raise RuntimeError("mrp_oracle_verify failed (%d)" % rc)
+    return accept_len, accept_mask

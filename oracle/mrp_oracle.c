@@ -1,0 +1,335 @@
+/*
+ * MRP drafting step -- CPU oracle (TEST INFRASTRUCTURE, not a product path).
+ *
+ * A plain, slow, fp64 restatement of what one Multi-token Residual Prediction
+ * drafting step computes, written from the paper's definitions:
+ *   - confidence = top-1 softmax probability of a position (Sec. 2, "Denoising Loop");
+ *   - the chain  Delta,delta <- g(x_t,h);  h <- h+Delta;  l <- l+delta  repeated K times
+ *     (Algorithm 2, inner loop; Algorithm 3, "MRP drafting"; Algorithm 4, "MRP forward");
+ *   - delta is produced by the backbone's own LM head applied to the module output (Sec. 3.2);
+ *   - static reveal = the r most confident still-masked positions of the block,
+ *     dynamic reveal = every masked position whose confidence clears tau, at least one
+ *     per step (Sec. 4.1, "Denoising Mode");
+ *   - remask = revoke positions of the reveal set whose updated confidence is below the
+ *     same tau (Algorithm 4; Sec. 3.4 "Remasking decoding");
+ *   - max-accept cap m = min(max(floor(0.7 n), 5), L) (Sec. 4.4);
+ *   - verification = a drafted token is accepted iff it equals the backbone's argmax
+ *     (Algorithm 3), with the prefix semantics of Figure 1(d).
+ * The head g is the reduced module this build is specified on: RMSNorm followed by a
+ * SwiGLU MLP (no biases), whose output r is both the hidden residual Delta and the
+ * vector sent through the LM head (delta = W_lm r).
+ *
+ * Only tests, the smoke check and the benchmark's cpu_baseline leg may call this file.
+ * It shares no code, header, table or constant with the CUDA path.  Inputs are float32
+ * arrays holding exactly the values the GPU sees (bf16 values are exact in float32);
+ * every arithmetic step is done in double.  There is no blocking, fusion or reordering
+ * beyond the loops written here; OpenMP only spreads independent output elements over
+ * cores.
+ *
+ * Parity pins live in tests/ (zero-residual heads, softmax normalisation, linearity of the
+ * chain in the residual, brute force on tiny vocabularies, a second implementation on
+ * library routines, closed forms for the cap and the accepted-prefix length).
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+int mrp_oracle_num_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+/* Softmax statistics of one logit row (Sec. 2): maximum, lowest-index argmax,
+ * log-sum-exp, confidence = exp(max - lse), and the gap between the two largest logits. */
+static void softmax_stats(const double *l, int V, double *conf, double *lse, int32_t *tok,
+                          double *margin)
+{
+    double mx = l[0];
+    int32_t arg = 0;
+    for (int v = 1; v < V; ++v)
+        if (l[v] > mx) { mx = l[v]; arg = v; }
+    double second = -INFINITY;
+    for (int v = 0; v < V; ++v)
+        if (v != arg && l[v] > second) second = l[v];
+    double S = 0.0;
+    for (int v = 0; v < V; ++v) S += exp(l[v] - mx);
+    double L = mx + log(S);
+    *conf = exp(mx - L);
+    *lse = L;
+    *tok = arg;
+    *margin = (V > 1) ? (mx - second) : INFINITY;
+}
+
+/*
+ * One drafting pass over M masked rows (Algorithm 2, lines "for k = 1..K").
+ *   hidden  [n_rows, d]   backbone hidden states h
+ *   logits0 [n_rows, V]   backbone logits l
+ *   row_index [M] or NULL rows of the dense arrays that are masked (NULL = 0..M-1)
+ *   gamma/w_gate/w_up/w_down: K pointers each, head k (1-based) = entry k-1;
+ *       gamma [d], w_gate [F,d], w_up [F,d], w_down [d,F], row-major [out,in]
+ *   w_lm [V, d]
+ * Outputs, step-major, k = 0 is the backbone's own logits:
+ *   conf, lse, margin [(K+1), M] double; token [(K+1), M] int32
+ *   logits_out  optional [K, M, V]  (l after step k = 1..K)
+ *   hidden_out  optional [M, d]     (h after step K)
+ * Returns 0, or -1 on allocation failure / bad arguments.
+ */
+int mrp_oracle_draft(int d, int F, int V, int K, int M, double eps,
+                     const float *hidden, const float *logits0, const int32_t *row_index,
+                     const float *const *gamma, const float *const *w_gate,
+                     const float *const *w_up, const float *const *w_down,
+                     const float *w_lm,
+                     double *conf, double *lse, int32_t *token, double *margin,
+                     double *logits_out, double *hidden_out)
+{
+    if (d <= 0 || F <= 0 || V <= 0 || K < 0 || M < 0) return -1;
+    double *h = (double *)malloc(sizeof(double) * (size_t)d);
+    double *xh = (double *)malloc(sizeof(double) * (size_t)d);
+    double *a = (double *)malloc(sizeof(double) * (size_t)F);
+    double *r = (double *)malloc(sizeof(double) * (size_t)d);
+    double *l = (double *)malloc(sizeof(double) * (size_t)V);
+    if (!h || !xh || !a || !r || !l) { free(h); free(xh); free(a); free(r); free(l); return -1; }
+
+    for (int m = 0; m < M; ++m) {
+        const size_t row = row_index ? (size_t)row_index[m] : (size_t)m;
+        for (int j = 0; j < d; ++j) h[j] = (double)hidden[row * (size_t)d + j];
+        for (int v = 0; v < V; ++v) l[v] = (double)logits0[row * (size_t)V + v];
+        softmax_stats(l, V, &conf[m], &lse[m], &token[m], &margin[m]);
+
+        for (int k = 1; k <= K; ++k) {
+            const float *g_k = gamma[k - 1];
+            const float *wg = w_gate[k - 1], *wu = w_up[k - 1], *wd = w_down[k - 1];
+            /* RMSNorm: xh = h / sqrt(mean(h^2) + eps) * gamma */
+            double ss = 0.0;
+            for (int j = 0; j < d; ++j) ss += h[j] * h[j];
+            const double rstd = 1.0 / sqrt(ss / (double)d + eps);
+            for (int j = 0; j < d; ++j) xh[j] = h[j] * rstd * (double)g_k[j];
+            /* SwiGLU: a = silu(W_g xh) * (W_u xh), silu(x) = x / (1 + exp(-x)) */
+#pragma omp parallel for schedule(static)
+            for (int f = 0; f < F; ++f) {
+                double g = 0.0, u = 0.0;
+                const float *wgr = wg + (size_t)f * d, *wur = wu + (size_t)f * d;
+                for (int j = 0; j < d; ++j) g += (double)wgr[j] * xh[j];
+                for (int j = 0; j < d; ++j) u += (double)wur[j] * xh[j];
+                a[f] = g / (1.0 + exp(-g)) * u;
+            }
+            /* r = W_d a : the hidden residual Delta */
+#pragma omp parallel for schedule(static)
+            for (int j = 0; j < d; ++j) {
+                double s = 0.0;
+                const float *wdr = wd + (size_t)j * F;
+                for (int f = 0; f < F; ++f) s += (double)wdr[f] * a[f];
+                r[j] = s;
+            }
+            /* h <- h + Delta */
+            for (int j = 0; j < d; ++j) h[j] += r[j];
+            /* l <- l + delta, delta = W_lm Delta (shared LM head) */
+#pragma omp parallel for schedule(static)
+            for (int v = 0; v < V; ++v) {
+                double s = 0.0;
+                const float *wr = w_lm + (size_t)v * d;
+                for (int j = 0; j < d; ++j) s += (double)wr[j] * r[j];
+                l[v] += s;
+            }
+            const size_t o = (size_t)k * M + m;
+            softmax_stats(l, V, &conf[o], &lse[o], &token[o], &margin[o]);
+            if (logits_out)
+                memcpy(logits_out + ((size_t)(k - 1) * M + m) * V, l, sizeof(double) * (size_t)V);
+        }
+        if (hidden_out) memcpy(hidden_out + (size_t)m * d, h, sizeof(double) * (size_t)d);
+    }
+    free(h); free(xh); free(a); free(r); free(l);
+    return 0;
+}
+
+/* Max-accept cap (Sec. 4.4): m = min(max(floor(0.7 n), 5), L). */
+int mrp_oracle_cap(int n_masked, int L)
+{
+    int m = (int)floor(0.7 * (double)n_masked + 1e-9);
+    if (m < 5) m = 5;
+    if (m > L) m = L;
+    return m;
+}
+
+/* Among candidate rows cand[0..n) pick the one with the largest confidence,
+ * ties to the lower block position.  Returns its index into cand, or -1. */
+static int best_candidate(const int *cand, int n, const uint8_t *taken, const float *c,
+                          const int32_t *pos)
+{
+    int best = -1;
+    for (int i = 0; i < n; ++i) {
+        if (taken[i]) continue;
+        if (best < 0) { best = i; continue; }
+        const float ci = c[cand[i]], cb = c[cand[best]];
+        if (ci > cb || (ci == cb && pos[cand[i]] < pos[cand[best]])) best = i;
+    }
+    return best;
+}
+
+/*
+ * Reveal selection, remasking (Algorithms 2-4; Sec. 4.1 "Denoising Mode"; Sec. 4.4).
+ *   conf  [(K+1), M] float32, token [(K+1), M] int32  -- per-step statistics of the masked rows
+ *   row_index [M] or NULL: dense position b*L+i of each masked row (NULL = 0..M-1)
+ *   mode 0 = STATIC: for k = 0..K take the r (k=0: r_reveal, k>=1: r_draft) most confident
+ *            still-masked positions of each block under step k's logits; k=0 picks are
+ *            reveals, k>=1 picks are drafts (listed in draft order).
+ *   mode 1 = DYNAMIC + REMASK: R = {masked i : conf[0,i] >= tau}; if empty and
+ *            ensure_progress, R = {most confident}; if use_cap and |R| > m keep the m most
+ *            confident; remask i in R whose updated confidence c'(i) < tau, where
+ *            c'(i) = min_{k=1..K} conf[k,i] (remask_policy 0) or conf[K,i] (policy 1);
+ *            if everything was revoked and ensure_progress, the most confident of R stays.
+ * Outputs (all written for every dense position / block):
+ *   reveal_mask, remask_mask [B*L] int8; out_token [B*L] int32 (-1 = nothing committed
+ *   or drafted); step_of [B*L] int8 (-1 = untouched); draft_pos, draft_tok [B, Kd] int32
+ *   (-1 pad) with Kd = K*r_draft; draft_len [B].
+ * All confidence comparisons are float32 comparisons.
+ */
+int mrp_oracle_select(const float *conf, const int32_t *token, const int32_t *row_index,
+                      int M, int K, int B, int L, int mode, float tau, int r_reveal,
+                      int r_draft, int use_cap, int remask_policy, int ensure_progress,
+                      int8_t *reveal_mask, int8_t *remask_mask, int32_t *out_token,
+                      int8_t *step_of, int32_t *draft_pos, int32_t *draft_tok,
+                      int32_t *draft_len)
+{
+    if (M < 0 || K < 0 || B <= 0 || L <= 0) return -1;
+    const int Kd = K * (r_draft > 0 ? r_draft : 0);
+    for (int i = 0; i < B * L; ++i) {
+        reveal_mask[i] = 0; remask_mask[i] = 0; out_token[i] = -1; step_of[i] = -1;
+    }
+    for (int i = 0; i < B * Kd; ++i) { draft_pos[i] = -1; draft_tok[i] = -1; }
+    for (int b = 0; b < B; ++b) draft_len[b] = 0;
+
+    int *cand = (int *)malloc(sizeof(int) * (size_t)(M > 0 ? M : 1));
+    int32_t *pos = (int32_t *)malloc(sizeof(int32_t) * (size_t)(M > 0 ? M : 1));
+    uint8_t *taken = (uint8_t *)malloc((size_t)(M > 0 ? M : 1));
+    uint8_t *inR = (uint8_t *)malloc((size_t)(M > 0 ? M : 1));
+    if (!cand || !pos || !taken || !inR) { free(cand); free(pos); free(taken); free(inR); return -1; }
+    for (int m = 0; m < M; ++m) {
+        const int idx = row_index ? row_index[m] : m;
+        if (idx < 0 || idx >= B * L) { free(cand); free(pos); free(taken); free(inR); return -1; }
+        pos[m] = idx % L;
+    }
+
+    for (int b = 0; b < B; ++b) {
+        /* masked rows of this block */
+        int n = 0;
+        for (int m = 0; m < M; ++m) {
+            const int idx = row_index ? row_index[m] : m;
+            if (idx / L == b) cand[n++] = m;
+        }
+        if (n == 0) continue;
+        memset(taken, 0, (size_t)n);
+
+        if (mode == 0) {
+            for (int k = 0; k <= K; ++k) {
+                const int r = (k == 0) ? r_reveal : r_draft;
+                const float *ck = conf + (size_t)k * M;
+                for (int t = 0; t < r; ++t) {
+                    const int bi = best_candidate(cand, n, taken, ck, pos);
+                    if (bi < 0) break;
+                    taken[bi] = 1;
+                    const int m = cand[bi];
+                    const int dense = b * L + pos[m];
+                    out_token[dense] = token[(size_t)k * M + m];
+                    step_of[dense] = (int8_t)k;
+                    if (k == 0) {
+                        reveal_mask[dense] = 1;
+                    } else {
+                        const int q = draft_len[b]++;
+                        draft_pos[b * Kd + q] = pos[m];
+                        draft_tok[b * Kd + q] = token[(size_t)k * M + m];
+                    }
+                }
+            }
+        } else {
+            int nR = 0;
+            for (int i = 0; i < n; ++i) { inR[i] = (conf[cand[i]] >= tau); nR += inR[i]; }
+            if (nR == 0 && ensure_progress) {
+                const int bi = best_candidate(cand, n, taken, conf, pos);
+                inR[bi] = 1; nR = 1;
+            }
+            if (use_cap) {
+                const int cap = mrp_oracle_cap(n, L);
+                if (nR > cap) {
+                    /* keep the cap most confident members of R */
+                    for (int i = 0; i < n; ++i) taken[i] = !inR[i];
+                    memset(inR, 0, (size_t)n);
+                    for (int t = 0; t < cap; ++t) {
+                        const int bi = best_candidate(cand, n, taken, conf, pos);
+                        taken[bi] = 1; inR[bi] = 1;
+                    }
+                    nR = cap;
+                    memset(taken, 0, (size_t)n);
+                }
+            }
+            int kept = 0;
+            for (int i = 0; i < n; ++i) {
+                if (!inR[i]) continue;
+                const int m = cand[i];
+                const int dense = b * L + pos[m];
+                reveal_mask[dense] = 1;
+                float c2;
+                if (K == 0) {
+                    c2 = conf[m];
+                } else if (remask_policy == 1) {
+                    c2 = conf[(size_t)K * M + m];
+                } else {
+                    c2 = conf[(size_t)1 * M + m];
+                    for (int k = 2; k <= K; ++k)
+                        if (conf[(size_t)k * M + m] < c2) c2 = conf[(size_t)k * M + m];
+                }
+                if (c2 < tau) remask_mask[dense] = 1; else ++kept;
+            }
+            if (kept == 0 && nR > 0 && ensure_progress) {
+                for (int i = 0; i < n; ++i) taken[i] = !inR[i];
+                const int bi = best_candidate(cand, n, taken, conf, pos);
+                remask_mask[b * L + pos[cand[bi]]] = 0;
+            }
+            for (int i = 0; i < n; ++i) {
+                if (!inR[i]) continue;
+                const int m = cand[i];
+                const int dense = b * L + pos[m];
+                if (!remask_mask[dense]) { out_token[dense] = token[m]; step_of[dense] = 0; }
+            }
+        }
+    }
+    free(cand); free(pos); free(taken); free(inR);
+    return 0;
+}
+
+/*
+ * Draft verification (Algorithm 3, "Reject drafted positions where argmax differ";
+ * Figure 1(d): candidate k embeds the first k draft tokens, hence prefix acceptance).
+ *   draft_tok, verify_tok [B, Kd]; draft_len [B] (entries j >= draft_len[b] are ignored)
+ *   positionwise = 0: accept_len = number of leading matches, accept_mask cleared after
+ *                     the first mismatch (those drafts are remasked);
+ *   positionwise = 1: accept_mask = per-slot match, accept_len = their count.
+ */
+int mrp_oracle_verify(const int32_t *draft_tok, const int32_t *verify_tok,
+                      const int32_t *draft_len, int B, int Kd, int positionwise,
+                      int32_t *accept_len, int8_t *accept_mask)
+{
+    if (B < 0 || Kd < 0) return -1;
+    for (int b = 0; b < B; ++b) {
+        int n = draft_len[b];
+        if (n > Kd) n = Kd;
+        if (n < 0) n = 0;
+        int acc = 0, alive = 1;
+        for (int j = 0; j < Kd; ++j) {
+            int ok = (j < n) && (draft_tok[b * Kd + j] == verify_tok[b * Kd + j]);
+            if (!positionwise) { if (!ok) alive = 0; ok = ok && alive; }
+            accept_mask[b * Kd + j] = (int8_t)ok;
+            acc += ok;
+        }
+        accept_len[b] = acc;
+    }
+    return 0;
+}
