@@ -1,0 +1,217 @@
+/*
+ * mrp.h -- C ABI of the B200-native MRP drafting step.
+ *
+ * One call of the library covers what happens between two backbone forwards of a
+ * block-diffusion language model that carries a Multi-token Residual Prediction (MRP)
+ * module: for every still-masked position of the active block, a chain of K lightweight
+ * heads turns the backbone hidden state into a residual, the residual goes through the
+ * backbone's own LM head and is added to the previous step's logits, and the new logits
+ * are reduced to confidence (top-1 softmax probability), log-sum-exp and argmax; these
+ * drive the reveal rules, the remask rule and draft verification.
+ *
+ * Conventions that hold for every entry point
+ *   - All tensor pointers are DEVICE pointers owned by the caller; the library borrows
+ *     them for the duration of the call (weights and workspace: for the lifetime of the
+ *     context; they are not copied).  Struct pointers (configs, parameter blocks, output
+ *     descriptors) are HOST pointers and are read before the call returns.
+ *   - Matrices are row-major.  Weight matrices are [out_features, in_features].
+ *   - Calls enqueue work on the given CUDA stream (a cudaStream_t passed as void*, NULL =
+ *     the default stream) and return without synchronising.  No entry point allocates
+ *     device memory; all scratch lives in the caller-provided workspace.
+ *   - The return value is an mrp_status.  Argument errors are detected on the host before
+ *     anything is launched.  Device-side anomalies (non-finite statistics, a bounded wait
+ *     that gave up) are OR-ed as MRP_DEV_* bits into an int32 device status word that the
+ *     caller may read after synchronising; kernels never trap or spin without a limit.
+ *   - A context is not thread-safe: use one context per stream.
+ */
+#ifndef MRP_H
+#define MRP_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct mrp_ctx mrp_ctx;
+
+typedef enum {
+    MRP_OK = 0,
+    MRP_ERR_INVALID_ARG = 1,   /* null pointer, size out of range, misaligned pointer   */
+    MRP_ERR_UNSUPPORTED = 2,   /* shape not supported by the requested kernel family    */
+    MRP_ERR_CUDA = 3,          /* a CUDA runtime / driver call failed                   */
+    MRP_ERR_NOMEM = 4,         /* workspace too small, or host allocation failed        */
+    MRP_ERR_NONFINITE = 5,
+    MRP_ERR_TIMEOUT = 6
+} mrp_status;
+
+/* Bits of the device status word. */
+#define MRP_DEV_NONFINITE 1    /* a log-sum-exp came out NaN or infinite                */
+#define MRP_DEV_TIMEOUT 2      /* a bounded barrier wait inside a kernel ran out        */
+
+typedef enum { MRP_F32 = 0, MRP_BF16 = 1 } mrp_dtype;
+
+/* mrp_config.flags */
+#define MRP_FLAG_FORCE_SIMT 1  /* bf16 context: use the CUDA-core kernels instead of the
+                                  tensor-core (tcgen05) kernels; a cross-check path      */
+
+typedef struct {
+    int32_t d;          /* hidden size                                                   */
+    int32_t d_ff;       /* SwiGLU inner size F                                           */
+    int32_t vocab;      /* vocabulary size V                                             */
+    int32_t n_heads;    /* number of head weight sets handed to mrp_create               */
+    int32_t max_rows;   /* largest M (masked rows per call)                              */
+    int32_t max_seqs;   /* largest B (sequences, i.e. active blocks, per call)           */
+    int32_t block_len;  /* largest L (positions per block)                               */
+    int32_t dtype;      /* mrp_dtype of weights and hidden states; logits are fp32       */
+    float rms_eps;      /* epsilon of the heads' RMSNorm                                 */
+    int32_t device;     /* CUDA device ordinal the context lives on                      */
+    int32_t flags;      /* MRP_FLAG_*                                                    */
+} mrp_config;
+
+/*
+ * One MRP head in the reduced form this library is specified on: RMSNorm followed by a
+ * SwiGLU MLP without biases,
+ *     x = h * rsqrt(mean(h^2) + eps) * gamma,   r = W_down ( silu(W_gate x) * (W_up x) ).
+ * r is the hidden residual (Algorithm 2: h <- h + Delta) and also the vector sent through
+ * the LM head (Sec. 3.2: the module reuses the backbone's LM head to produce delta).
+ * The same weight set may be listed several times (a module applied K times).
+ */
+typedef struct {
+    const void *rms_gamma;  /* [d]        */
+    const void *w_gate;     /* [d_ff, d]  */
+    const void *w_up;       /* [d_ff, d]  */
+    const void *w_down;     /* [d, d_ff]  */
+} mrp_head_weights;
+
+/* Bytes of device workspace a context of this configuration needs (0 on a bad config). */
+size_t mrp_workspace_bytes(const mrp_config *cfg);
+
+/*
+ * Create a context.  heads: HOST array of cfg->n_heads entries holding DEVICE pointers;
+ * w_lm: DEVICE [vocab, d]; workspace: DEVICE, 256-byte aligned, at least
+ * mrp_workspace_bytes(cfg) bytes, owned by the caller and kept alive until mrp_destroy.
+ * The bf16 tensor-core kernels need d % 64 == 0, d_ff % 64 == 0, vocab % 16 == 0 and
+ * 16-byte aligned weights; other bf16 shapes run on the CUDA-core kernels.
+ * On success *out receives the context.  Errors: INVALID_ARG, NOMEM, CUDA.
+ */
+int mrp_create(const mrp_config *cfg, const mrp_head_weights *heads, const void *w_lm,
+               void *workspace, size_t workspace_bytes, mrp_ctx **out);
+
+/* Release the host-side context (the workspace stays the caller's).  NULL is allowed. */
+void mrp_destroy(mrp_ctx *ctx);
+
+/*
+ * Outputs of mrp_draft.  conf/lse/token (and margin) are step-major [(K+1), M]: entry
+ * k*M + m is masked row m after k MRP steps; k = 0 is the backbone's own logits.
+ *   conf   = top-1 softmax probability (Sec. 2: the "confidence" of a position)
+ *   lse    = log-sum-exp of the logit row
+ *   token  = argmax, lowest token id on exact ties
+ *   margin = top-1 minus top-2 logit (optional, NULL = skip)
+ *   logits_out = optional [K, M, V] fp32: l_k for k = 1..K; NULL = the V-wide rows are
+ *                never written to memory
+ *   hidden_out = optional [M, d] fp32: h after step K; NULL = skip
+ *   status = optional device int32 that receives MRP_DEV_* bits (OR-ed, never cleared)
+ */
+typedef struct {
+    float *conf;
+    float *lse;
+    int32_t *token;
+    float *margin;
+    float *logits_out;
+    float *hidden_out;
+    int32_t *status;
+} mrp_draft_out;
+
+/*
+ * The drafting pass (Algorithm 2, lines "for k = 1..K": Delta,delta <- g(h); h <- h+Delta;
+ * l <- l+delta; likewise Algorithm 3 "MRP drafting" and Algorithm 4 "MRP forward").
+ *   hidden  [n_rows, d]   backbone hidden states, dtype of the context
+ *   logits0 [n_rows, V]   backbone logits, fp32
+ *   row_index [M] int32   rows of hidden/logits0 that are masked positions (dense position
+ *                         b*L+i of each masked row), or NULL for rows 0..M-1
+ *   M in [0, max_rows], K in [0, n_heads] (head k uses weight set k-1)
+ * Step k's logits are l_0 + W_lm (h_k - h_0), which equals the per-step accumulation
+ * l <- l + W_lm Delta by linearity of the LM head.  Errors: INVALID_ARG, CUDA.
+ */
+int mrp_draft(mrp_ctx *ctx, const void *hidden, const float *logits0, const int32_t *row_index,
+              int32_t M, int32_t K, const mrp_draft_out *out, void *cuda_stream);
+
+typedef enum { MRP_SELECT_STATIC = 0, MRP_SELECT_DYNAMIC_REMASK = 1 } mrp_select_mode;
+
+typedef struct {
+    int32_t mode;             /* mrp_select_mode                                         */
+    float tau;                /* confidence threshold (dynamic mode)                     */
+    int32_t r_reveal;         /* static: positions revealed from the backbone step k=0   */
+    int32_t r_draft;          /* static: positions drafted per MRP step k>=1             */
+    int32_t use_cap;          /* dynamic: cap |R| at min(max(floor(0.7 n),5),L), Sec.4.4 */
+    int32_t remask_policy;    /* 0 = min over steps 1..K must stay >= tau, 1 = step K    */
+    int32_t ensure_progress;  /* keep at least one reveal per block                      */
+} mrp_select_params;
+
+/*
+ * Outputs of mrp_reveal_remask; every element is written on every call.
+ *   reveal_mask [B*L] int8  static: positions picked at step 0; dynamic: the reveal set R
+ *   remask_mask [B*L] int8  dynamic: members of R revoked by the MRP-updated confidence
+ *   out_token   [B*L] int32 token committed or drafted at the position, -1 otherwise
+ *   step_of     [B*L] int8  step k at which the position was taken, -1 otherwise
+ *   draft_pos, draft_tok [B, Kd] int32, Kd = K * r_draft: block positions and tokens of the
+ *               drafts (steps k >= 1) in draft order, -1 padded
+ *   draft_len   [B] int32
+ */
+typedef struct {
+    int8_t *reveal_mask;
+    int8_t *remask_mask;
+    int32_t *out_token;
+    int8_t *step_of;
+    int32_t *draft_pos;
+    int32_t *draft_tok;
+    int32_t *draft_len;
+} mrp_select_out;
+
+/*
+ * Reveal selection and remasking from the per-step statistics of mrp_draft.
+ *   STATIC (Algorithm 2 "Reveal r tokens with highest confidence", Algorithm 3 "Draft
+ *   token with highest confidence"; Sec. 4.1 static denoising): for k = 0..K take the r
+ *   most confident still-masked positions of each block under step k (confidence
+ *   descending, position ascending on ties); k = 0 picks are reveals, k >= 1 are drafts.
+ *   DYNAMIC_REMASK (Algorithm 4; Sec. 4.1 dynamic denoising; Sec. 4.4 cap): R = masked
+ *   positions with conf_0 >= tau (the most confident one if none and ensure_progress;
+ *   the cap's most confident ones if use_cap and |R| exceeds it); remask members of R whose
+ *   updated confidence (policy) is < tau; if that revokes all of R and ensure_progress, the
+ *   most confident member stays.  Comparisons are fp32.
+ * conf, token: [(K+1), M]; row_index [M] (unique, < B*L) or NULL; 1 <= L <= block_len,
+ * 1 <= B <= max_seqs.  Errors: INVALID_ARG, CUDA.
+ */
+int mrp_reveal_remask(mrp_ctx *ctx, const float *conf, const int32_t *token,
+                      const int32_t *row_index, int32_t M, int32_t K, int32_t B, int32_t L,
+                      const mrp_select_params *params, const mrp_select_out *out,
+                      void *cuda_stream);
+
+/*
+ * Draft verification (Algorithm 3: a drafted position is rejected where the backbone's
+ * argmax differs from the draft; Figure 1(d): candidate k embeds the first k drafts, so a
+ * draft only counts while all earlier drafts were accepted).
+ *   draft_tok, verify_tok [B, Kd] int32; draft_len [B] int32 (slots >= draft_len ignored)
+ *   positionwise = 0: accept_len[b] = number of leading matches, accept_mask cleared from the
+ *                     first mismatch on;  1: per-slot matches and their count
+ *   accept_len [B] int32, accept_mask [B, Kd] int8.  Errors: INVALID_ARG, CUDA.
+ */
+int mrp_verify(mrp_ctx *ctx, const int32_t *draft_tok, const int32_t *verify_tok,
+               const int32_t *draft_len, int32_t B, int32_t Kd, int32_t positionwise,
+               int32_t *accept_len, int8_t *accept_mask, void *cuda_stream);
+
+/* Number of kernels the last mrp_draft / mrp_reveal_remask / mrp_verify call on this
+ * context launched (for accounting in benchmarks). */
+int32_t mrp_last_launch_count(const mrp_ctx *ctx);
+
+/* Name of the kernel family a bf16/fp32 context resolved to: "simt" or "tcgen05". */
+const char *mrp_kernel_family(const mrp_ctx *ctx);
+
+const char *mrp_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MRP_H */

@@ -1,0 +1,235 @@
+"""Thin ctypes binding of libmrp_b200.so: argument marshalling only.
+
+The functions carry the C ABI's names (``mrp_create``, ``mrp_draft``, ``mrp_reveal_remask``,
+``mrp_verify``, ``mrp_destroy``) and take torch CUDA tensors, which serve as device memory
+and supply the current stream; every step of the drafting pass runs in the library's own
+kernels.  Importing this module loads the shared library and raises if it is missing or
+cannot be loaded: there is no CPU or PyTorch fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libmrp_b200.so")
+
+MRP_F32, MRP_BF16 = 0, 1
+MRP_FLAG_FORCE_SIMT = 1
+MRP_SELECT_STATIC, MRP_SELECT_DYNAMIC_REMASK = 0, 1
+MRP_DEV_NONFINITE, MRP_DEV_TIMEOUT = 1, 2
+
+EXPORTS = ("mrp_workspace_bytes", "mrp_create", "mrp_destroy", "mrp_draft", "mrp_reveal_remask",
+           "mrp_verify", "mrp_last_launch_count", "mrp_kernel_family", "mrp_status_string")
+
+
+class mrp_config(ctypes.Structure):
+    _fields_ = [("d", ctypes.c_int32), ("d_ff", ctypes.c_int32), ("vocab", ctypes.c_int32),
+                ("n_heads", ctypes.c_int32), ("max_rows", ctypes.c_int32),
+                ("max_seqs", ctypes.c_int32), ("block_len", ctypes.c_int32),
+                ("dtype", ctypes.c_int32), ("rms_eps", ctypes.c_float),
+                ("device", ctypes.c_int32), ("flags", ctypes.c_int32)]
+
+
+class mrp_head_weights(ctypes.Structure):
+    _fields_ = [("rms_gamma", ctypes.c_void_p), ("w_gate", ctypes.c_void_p),
+                ("w_up", ctypes.c_void_p), ("w_down", ctypes.c_void_p)]
+
+
+class mrp_draft_out(ctypes.Structure):
+    _fields_ = [("conf", ctypes.c_void_p), ("lse", ctypes.c_void_p), ("token", ctypes.c_void_p),
+                ("margin", ctypes.c_void_p), ("logits_out", ctypes.c_void_p),
+                ("hidden_out", ctypes.c_void_p), ("status", ctypes.c_void_p)]
+
+
+class mrp_select_params(ctypes.Structure):
+    _fields_ = [("mode", ctypes.c_int32), ("tau", ctypes.c_float), ("r_reveal", ctypes.c_int32),
+                ("r_draft", ctypes.c_int32), ("use_cap", ctypes.c_int32),
+                ("remask_policy", ctypes.c_int32), ("ensure_progress", ctypes.c_int32)]
+
+
+class mrp_select_out(ctypes.Structure):
+    _fields_ = [("reveal_mask", ctypes.c_void_p), ("remask_mask", ctypes.c_void_p),
+                ("out_token", ctypes.c_void_p), ("step_of", ctypes.c_void_p),
+                ("draft_pos", ctypes.c_void_p), ("draft_tok", ctypes.c_void_p),
+                ("draft_len", ctypes.c_void_p)]
+
+
+def _load():
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            "libmrp_b200.so is not built (%s); run `python -m paper_2605_18817_b200.build` "
+            "-- there is no fallback path" % LIB_PATH)
+    lib = ctypes.CDLL(LIB_PATH)
+    for name in EXPORTS:
+        getattr(lib, name)
+    lib.mrp_workspace_bytes.restype = ctypes.c_size_t
+    lib.mrp_workspace_bytes.argtypes = [ctypes.POINTER(mrp_config)]
+    lib.mrp_create.restype = ctypes.c_int
+    lib.mrp_create.argtypes = [ctypes.POINTER(mrp_config), ctypes.POINTER(mrp_head_weights),
+                               ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t,
+                               ctypes.POINTER(ctypes.c_void_p)]
+    lib.mrp_destroy.restype = None
+    lib.mrp_destroy.argtypes = [ctypes.c_void_p]
+    lib.mrp_draft.restype = ctypes.c_int
+    lib.mrp_draft.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                              ctypes.c_int32, ctypes.c_int32, ctypes.POINTER(mrp_draft_out),
+                              ctypes.c_void_p]
+    lib.mrp_reveal_remask.restype = ctypes.c_int
+    lib.mrp_reveal_remask.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                                      ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32,
+                                      ctypes.c_int32, ctypes.c_int32,
+                                      ctypes.POINTER(mrp_select_params),
+                                      ctypes.POINTER(mrp_select_out), ctypes.c_void_p]
+    lib.mrp_verify.restype = ctypes.c_int
+    lib.mrp_verify.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                               ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p,
+                               ctypes.c_void_p, ctypes.c_void_p]
+    lib.mrp_last_launch_count.restype = ctypes.c_int32
+    lib.mrp_last_launch_count.argtypes = [ctypes.c_void_p]
+    lib.mrp_kernel_family.restype = ctypes.c_char_p
+    lib.mrp_kernel_family.argtypes = [ctypes.c_void_p]
+    lib.mrp_status_string.restype = ctypes.c_char_p
+    lib.mrp_status_string.argtypes = [ctypes.c_int]
+    return lib
+
+
+lib = _load()
+
+
+class MrpError(RuntimeError):
+    def __init__(self, where: str, status: int):
+        self.status = status
+        super().__init__("%s: %s (%d)" % (where, lib.mrp_status_string(status).decode(), status))
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream=None):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _check(t, dtype, what):
+    if t is None:
+        return
+    if not (t.is_cuda and t.is_contiguous() and t.dtype == dtype):
+        raise TypeError("%s must be a contiguous CUDA tensor of %s" % (what, dtype))
+
+
+@dataclass
+class Context:
+    handle: int
+    cfg: mrp_config
+    keep: tuple           # weights + workspace kept alive for the context's lifetime
+
+    @property
+    def family(self) -> str:
+        return lib.mrp_kernel_family(self.handle).decode()
+
+    @property
+    def last_launch_count(self) -> int:
+        return int(lib.mrp_last_launch_count(self.handle))
+
+
+def mrp_workspace_bytes(cfg: mrp_config) -> int:
+    return int(lib.mrp_workspace_bytes(ctypes.byref(cfg)))
+
+
+def mrp_create(d, d_ff, vocab, heads, w_lm, max_rows, max_seqs, block_len, rms_eps=1e-6,
+               flags=0) -> Context:
+    """heads: list of dicts of CUDA tensors gamma [d], w_gate [F,d], w_up [F,d], w_down [d,F];
+    w_lm: CUDA tensor [V,d]; dtype (float32 or bfloat16) is taken from w_lm."""
+    tdtype = w_lm.dtype
+    if tdtype not in (torch.float32, torch.bfloat16):
+        raise TypeError("weights must be float32 or bfloat16")
+    _check(w_lm, tdtype, "w_lm")
+    dev = w_lm.device.index if w_lm.device.index is not None else torch.cuda.current_device()
+    cfg = mrp_config(int(d), int(d_ff), int(vocab), len(heads), int(max_rows), int(max_seqs),
+                     int(block_len), MRP_F32 if tdtype == torch.float32 else MRP_BF16,
+                     float(rms_eps), int(dev), int(flags))
+    harr = (mrp_head_weights * max(len(heads), 1))()
+    keep = [w_lm]
+    for k, h in enumerate(heads):
+        for name in ("gamma", "w_gate", "w_up", "w_down"):
+            _check(h[name], tdtype, name)
+            keep.append(h[name])
+        harr[k] = mrp_head_weights(h["gamma"].data_ptr(), h["w_gate"].data_ptr(),
+                                   h["w_up"].data_ptr(), h["w_down"].data_ptr())
+    nbytes = mrp_workspace_bytes(cfg)
+    if nbytes == 0:
+        raise MrpError("mrp_workspace_bytes", 1)
+    ws = torch.empty(nbytes + 256, dtype=torch.uint8, device=w_lm.device)
+    off = (-ws.data_ptr()) % 256
+    keep.append(ws)
+    handle = ctypes.c_void_p()
+    rc = lib.mrp_create(ctypes.byref(cfg), harr, _ptr(w_lm), ctypes.c_void_p(ws.data_ptr() + off),
+                        ctypes.c_size_t(nbytes), ctypes.byref(handle))
+    if rc != 0:
+        raise MrpError("mrp_create", rc)
+    return Context(handle.value, cfg, tuple(keep))
+
+
+def mrp_destroy(ctx: Context) -> None:
+    if ctx.handle:
+        lib.mrp_destroy(ctx.handle)
+        ctx.handle = 0
+
+
+def mrp_draft(ctx: Context, hidden, logits0, row_index, M, K, conf, lse, token, margin=None,
+              logits_out=None, hidden_out=None, status=None, stream=None) -> None:
+    """Enqueue one drafting pass; outputs are written into the given CUDA tensors."""
+    _check(hidden, torch.float32 if ctx.cfg.dtype == MRP_F32 else torch.bfloat16, "hidden")
+    _check(logits0, torch.float32, "logits0")
+    _check(row_index, torch.int32, "row_index")
+    for t, dt, nm in ((conf, torch.float32, "conf"), (lse, torch.float32, "lse"),
+                      (token, torch.int32, "token"), (margin, torch.float32, "margin"),
+                      (logits_out, torch.float32, "logits_out"),
+                      (hidden_out, torch.float32, "hidden_out"), (status, torch.int32, "status")):
+        _check(t, dt, nm)
+    out = mrp_draft_out(_ptr(conf), _ptr(lse), _ptr(token), _ptr(margin), _ptr(logits_out),
+                        _ptr(hidden_out), _ptr(status))
+    rc = lib.mrp_draft(ctx.handle, _ptr(hidden), _ptr(logits0), _ptr(row_index), int(M), int(K),
+                       ctypes.byref(out), _stream(stream))
+    if rc != 0:
+        raise MrpError("mrp_draft", rc)
+
+
+def mrp_reveal_remask(ctx: Context, conf, token, row_index, M, K, B, L, mode, tau=0.9, r_reveal=1,
+                      r_draft=1, use_cap=False, remask_policy=0, ensure_progress=True, *,
+                      reveal_mask, remask_mask, out_token, step_of, draft_pos, draft_tok, draft_len,
+                      stream=None) -> None:
+    _check(conf, torch.float32, "conf")
+    _check(token, torch.int32, "token")
+    _check(row_index, torch.int32, "row_index")
+    for t, dt, nm in ((reveal_mask, torch.int8, "reveal_mask"), (remask_mask, torch.int8, "remask_mask"),
+                      (out_token, torch.int32, "out_token"), (step_of, torch.int8, "step_of"),
+                      (draft_pos, torch.int32, "draft_pos"), (draft_tok, torch.int32, "draft_tok"),
+                      (draft_len, torch.int32, "draft_len")):
+        _check(t, dt, nm)
+    p = mrp_select_params(int(mode), float(tau), int(r_reveal), int(r_draft), int(bool(use_cap)),
+                          int(remask_policy), int(bool(ensure_progress)))
+    o = mrp_select_out(_ptr(reveal_mask), _ptr(remask_mask), _ptr(out_token), _ptr(step_of),
+                       _ptr(draft_pos), _ptr(draft_tok), _ptr(draft_len))
+    rc = lib.mrp_reveal_remask(ctx.handle, _ptr(conf), _ptr(token), _ptr(row_index), int(M), int(K),
+                               int(B), int(L), ctypes.byref(p), ctypes.byref(o), _stream(stream))
+    if rc != 0:
+        raise MrpError("mrp_reveal_remask", rc)
+
+
+def mrp_verify(ctx: Context, draft_tok, verify_tok, draft_len, B, Kd, positionwise, accept_len,
+               accept_mask, stream=None) -> None:
+    for t, dt, nm in ((draft_tok, torch.int32, "draft_tok"), (verify_tok, torch.int32, "verify_tok"),
+                      (draft_len, torch.int32, "draft_len"), (accept_len, torch.int32, "accept_len"),
+                      (accept_mask, torch.int8, "accept_mask")):
+        _check(t, dt, nm)
+    rc = lib.mrp_verify(ctx.handle, _ptr(draft_tok), _ptr(verify_tok), _ptr(draft_len), int(B),
+                        int(Kd), int(bool(positionwise)), _ptr(accept_len), _ptr(accept_mask),
+                        _stream(stream))
+    if rc != 0:
+        raise MrpError("mrp_verify", rc)

@@ -1,0 +1,221 @@
+// C ABI of libmrp_b200.so: argument validation, workspace layout, launch sequencing.
+#include <stdlib.h>
+#include <string.h>
+
+#include <new>
+
+#include "mrp_internal.cuh"
+
+namespace mrp {
+
+WorkspaceLayout workspace_layout(const mrp_config &cfg)
+{
+    WorkspaceLayout l;
+    memset(&l, 0, sizeof(l));
+    const size_t rows = (size_t)cfg.max_rows, d = (size_t)cfg.d, F = (size_t)cfg.d_ff;
+    const size_t steps = (size_t)cfg.n_heads + 1;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { const size_t o = off; off = align_up(off + bytes, 256); return o; };
+    l.status = take(64 * sizeof(int32_t));
+    l.h0f = take(rows * d * 4);
+    l.hcur = take(rows * d * 4);
+    l.xg = take(rows * d * 4);
+    l.act = take(rows * F * 4);
+    l.xt = take(steps * rows * d * 4);
+    l.sumsq = take((size_t)kSumsqSlices * rows * 4);
+    const int v_slices = (cfg.vocab + kSimtSliceV - 1) / kSimtSliceV;
+    l.n_slices_max = v_slices < kSimtMaxBlocks ? v_slices : kSimtMaxBlocks;
+    l.partials = take((size_t)l.n_slices_max * steps * rows * sizeof(Partial));
+    l.dense_row = take((size_t)cfg.max_seqs * (size_t)cfg.block_len * 4);
+    l.total = off;
+    return l;
+}
+
+static bool config_ok(const mrp_config *c)
+{
+    if (!c) return false;
+    if (c->d <= 0 || c->d_ff <= 0 || c->vocab <= 0 || c->n_heads < 0 || c->max_rows <= 0 ||
+        c->max_seqs <= 0 || c->block_len <= 0 || c->block_len > 1024)
+        return false;
+    if (c->dtype != MRP_F32 && c->dtype != MRP_BF16) return false;
+    if (!(c->rms_eps >= 0.f)) return false;
+    if ((long long)c->max_seqs * c->block_len > (1ll << 30)) return false;
+    return true;
+}
+
+struct DeviceGuard {
+    int prev = -1;
+    bool switched = false;
+    cudaError_t err = cudaSuccess;
+    explicit DeviceGuard(int dev)
+    {
+        err = cudaGetDevice(&prev);
+        if (err == cudaSuccess && prev != dev) {
+            err = cudaSetDevice(dev);
+            switched = (err == cudaSuccess);
+        }
+    }
+    ~DeviceGuard()
+    {
+        if (switched) cudaSetDevice(prev);
+    }
+};
+
+}  // namespace mrp
+
+using namespace mrp;
+
+struct mrp_ctx {
+    Ctx c;
+};
+
+extern "C" {
+
+size_t mrp_workspace_bytes(const mrp_config *cfg)
+{
+    if (!config_ok(cfg)) return 0;
+    return workspace_layout(*cfg).total;
+}
+
+int mrp_create(const mrp_config *cfg, const mrp_head_weights *heads, const void *w_lm,
+               void *workspace, size_t workspace_bytes, mrp_ctx **out)
+{
+    if (!out) return MRP_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!config_ok(cfg) || !w_lm || !workspace) return MRP_ERR_INVALID_ARG;
+    if (cfg->n_heads > 0 && !heads) return MRP_ERR_INVALID_ARG;
+    for (int k = 0; k < cfg->n_heads; ++k)
+        if (!heads[k].rms_gamma || !heads[k].w_gate || !heads[k].w_up || !heads[k].w_down)
+            return MRP_ERR_INVALID_ARG;
+    if (((uintptr_t)workspace & 255u) != 0) return MRP_ERR_INVALID_ARG;
+    const WorkspaceLayout lay = workspace_layout(*cfg);
+    if (workspace_bytes < lay.total) return MRP_ERR_NOMEM;
+
+    DeviceGuard guard(cfg->device);
+    if (guard.err != cudaSuccess) return MRP_ERR_CUDA;
+    mrp_ctx *ctx = new (std::nothrow) mrp_ctx;
+    if (!ctx) return MRP_ERR_NOMEM;
+    Ctx &c = ctx->c;
+    memset(&c, 0, sizeof(c));
+    c.cfg = *cfg;
+    c.heads = nullptr;
+    if (cfg->n_heads > 0) {
+        c.heads = (mrp_head_weights *)malloc(sizeof(mrp_head_weights) * (size_t)cfg->n_heads);
+        if (!c.heads) { delete ctx; return MRP_ERR_NOMEM; }
+        memcpy(c.heads, heads, sizeof(mrp_head_weights) * (size_t)cfg->n_heads);
+    }
+    c.w_lm = w_lm;
+    c.ws = (char *)workspace;
+    c.lay = lay;
+    c.launches = 0;
+    c.tc_state = nullptr;
+    int sm = 0;
+    if (cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, cfg->device) != cudaSuccess || sm <= 0) {
+        free(c.heads); delete ctx; return MRP_ERR_CUDA;
+    }
+    c.sm_count = sm;
+    c.use_tc = (cfg->dtype == MRP_BF16) && !(cfg->flags & MRP_FLAG_FORCE_SIMT) &&
+               tc_supported(*cfg, c.heads, w_lm);
+    if (c.use_tc) {
+        if (tc_create(&c) != cudaSuccess) { free(c.heads); delete ctx; return MRP_ERR_CUDA; }
+    }
+    if (cudaMemset(c.ws + lay.status, 0, 64 * sizeof(int32_t)) != cudaSuccess) {
+        if (c.use_tc) tc_destroy(&c);
+        free(c.heads); delete ctx; return MRP_ERR_CUDA;
+    }
+    *out = ctx;
+    return MRP_OK;
+}
+
+void mrp_destroy(mrp_ctx *ctx)
+{
+    if (!ctx) return;
+    if (ctx->c.use_tc) tc_destroy(&ctx->c);
+    free(ctx->c.heads);
+    delete ctx;
+}
+
+int mrp_draft(mrp_ctx *ctx, const void *hidden, const float *logits0, const int32_t *row_index,
+              int32_t M, int32_t K, const mrp_draft_out *out, void *cuda_stream)
+{
+    if (!ctx || !out) return MRP_ERR_INVALID_ARG;
+    Ctx &c = ctx->c;
+    if (M < 0 || M > c.cfg.max_rows || K < 0 || K > c.cfg.n_heads) return MRP_ERR_INVALID_ARG;
+    c.launches = 0;
+    if (M == 0) return MRP_OK;
+    if (!hidden || !logits0 || !out->conf || !out->lse || !out->token) return MRP_ERR_INVALID_ARG;
+    if (((uintptr_t)hidden & 15u) || ((uintptr_t)logits0 & 15u)) return MRP_ERR_INVALID_ARG;
+    DeviceGuard guard(c.cfg.device);
+    if (guard.err != cudaSuccess) return MRP_ERR_CUDA;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    cudaError_t e = c.use_tc ? tc_draft(&c, hidden, logits0, row_index, M, K, *out, st)
+                             : simt_draft(&c, hidden, logits0, row_index, M, K, *out, st);
+    return e == cudaSuccess ? MRP_OK : MRP_ERR_CUDA;
+}
+
+int mrp_reveal_remask(mrp_ctx *ctx, const float *conf, const int32_t *token,
+                      const int32_t *row_index, int32_t M, int32_t K, int32_t B, int32_t L,
+                      const mrp_select_params *params, const mrp_select_out *out, void *cuda_stream)
+{
+    if (!ctx || !params || !out) return MRP_ERR_INVALID_ARG;
+    Ctx &c = ctx->c;
+    if (B < 1 || B > c.cfg.max_seqs || L < 1 || L > c.cfg.block_len) return MRP_ERR_INVALID_ARG;
+    if (M < 0 || (long long)M > (long long)B * L || K < 0) return MRP_ERR_INVALID_ARG;
+    if (M > 0 && (!conf || !token)) return MRP_ERR_INVALID_ARG;
+    if (params->mode != MRP_SELECT_STATIC && params->mode != MRP_SELECT_DYNAMIC_REMASK)
+        return MRP_ERR_INVALID_ARG;
+    if (params->r_reveal < 0 || params->r_draft < 0) return MRP_ERR_INVALID_ARG;
+    if (params->remask_policy != 0 && params->remask_policy != 1) return MRP_ERR_INVALID_ARG;
+    if (!out->reveal_mask || !out->remask_mask || !out->out_token || !out->step_of || !out->draft_len)
+        return MRP_ERR_INVALID_ARG;
+    const int Kd = K * params->r_draft;
+    if (Kd > 0 && (!out->draft_pos || !out->draft_tok)) return MRP_ERR_INVALID_ARG;
+    c.launches = 0;
+    DeviceGuard guard(c.cfg.device);
+    if (guard.err != cudaSuccess) return MRP_ERR_CUDA;
+    cudaError_t e = launch_select(&c, conf, token, row_index, M, K, B, L, *params, *out,
+                                  (cudaStream_t)cuda_stream);
+    return e == cudaSuccess ? MRP_OK : MRP_ERR_CUDA;
+}
+
+int mrp_verify(mrp_ctx *ctx, const int32_t *draft_tok, const int32_t *verify_tok,
+               const int32_t *draft_len, int32_t B, int32_t Kd, int32_t positionwise,
+               int32_t *accept_len, int8_t *accept_mask, void *cuda_stream)
+{
+    if (!ctx) return MRP_ERR_INVALID_ARG;
+    Ctx &c = ctx->c;
+    if (B < 0 || B > c.cfg.max_seqs || Kd < 0) return MRP_ERR_INVALID_ARG;
+    c.launches = 0;
+    if (B == 0) return MRP_OK;
+    if (!draft_len || !accept_len) return MRP_ERR_INVALID_ARG;
+    if (Kd > 0 && (!draft_tok || !verify_tok || !accept_mask)) return MRP_ERR_INVALID_ARG;
+    DeviceGuard guard(c.cfg.device);
+    if (guard.err != cudaSuccess) return MRP_ERR_CUDA;
+    cudaError_t e = launch_verify(&c, draft_tok, verify_tok, draft_len, B, Kd, positionwise ? 1 : 0,
+                                  accept_len, accept_mask, (cudaStream_t)cuda_stream);
+    return e == cudaSuccess ? MRP_OK : MRP_ERR_CUDA;
+}
+
+int32_t mrp_last_launch_count(const mrp_ctx *ctx) { return ctx ? ctx->c.launches : 0; }
+
+const char *mrp_kernel_family(const mrp_ctx *ctx)
+{
+    if (!ctx) return "none";
+    return ctx->c.use_tc ? "tcgen05" : "simt";
+}
+
+const char *mrp_status_string(int status)
+{
+    switch (status) {
+    case MRP_OK: return "ok";
+    case MRP_ERR_INVALID_ARG: return "invalid argument";
+    case MRP_ERR_UNSUPPORTED: return "unsupported shape";
+    case MRP_ERR_CUDA: return "CUDA error";
+    case MRP_ERR_NOMEM: return "workspace too small or out of host memory";
+    case MRP_ERR_NONFINITE: return "non-finite values";
+    case MRP_ERR_TIMEOUT: return "device wait timed out";
+    default: return "unknown status";
+    }
+}
+
+}  // extern "C"

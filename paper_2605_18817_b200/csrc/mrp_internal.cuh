@@ -1,0 +1,99 @@
+// Internal declarations shared by the translation units of libmrp_b200.so.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "mrp.h"
+
+namespace mrp {
+
+// Partial softmax statistics of one (step, row) over a slice of the vocabulary.
+struct __align__(16) Partial {
+    float mx;      // largest logit of the slice
+    float sum;     // sum of exp(logit - mx) over the slice
+    int32_t idx;   // lowest token id attaining mx
+    float second;  // second largest logit of the slice (-inf if none)
+};
+
+__host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Regions of the caller-provided workspace (byte offsets, each 256-byte aligned).
+struct WorkspaceLayout {
+    size_t status;      // int32[64]: device status word (first element)
+    size_t h0f;         // fp32 [max_rows, d]       gathered h_0
+    size_t hcur;        // fp32 [max_rows, d]       residual stream h_k
+    size_t xg;          // [max_rows, d]            head input operand (fp32 simt / bf16 tc)
+    size_t act;         // [max_rows, F]            SwiGLU activations (fp32 simt / bf16 tc)
+    size_t xt;          // [(n_heads+1)*max_rows, d] stacked LM-head operand rows h_k - h_0
+    size_t sumsq;       // fp32 [kSumsqSlices, max_rows] per-CTA partial sums of squares
+    size_t partials;    // Partial [n_slices_max, (n_heads+1)*max_rows]
+    size_t dense_row;   // int32 [max_seqs*block_len] dense position -> masked row or -1
+    size_t total;
+    int32_t n_slices_max;
+};
+
+constexpr int kSumsqSlices = 512;
+constexpr int kSimtSliceV = 128;      // vocabulary entries per SIMT LM-head slice
+constexpr int kSimtMaxBlocks = 592;   // SIMT LM-head grid cap (4 per SM)
+
+WorkspaceLayout workspace_layout(const mrp_config &cfg);
+
+struct Ctx {
+    mrp_config cfg;
+    mrp_head_weights *heads;   // host array [n_heads] of device pointers
+    const void *w_lm;
+    char *ws;
+    WorkspaceLayout lay;
+    bool use_tc;
+    int32_t launches;
+    int sm_count;
+    void *tc_state;            // tensor-core path state (tensor maps), owned by tc_*.cu
+};
+
+// ---- CUDA-core kernel family (simt_kernels.cu) -------------------------------------
+cudaError_t simt_draft(Ctx *c, const void *hidden, const float *logits0, const int32_t *row_index,
+                       int M, int K, const mrp_draft_out &out, cudaStream_t st);
+
+// Shared by both families: merge per-slice partials into conf/lse/token/margin.
+cudaError_t launch_combine(Ctx *c, const Partial *partials, int n_slices, int n_rowsteps,
+                           const mrp_draft_out &out, int32_t *status, cudaStream_t st);
+// Shared by both families: gather masked rows of `hidden` into fp32 h0f / hcur.
+cudaError_t launch_prep(Ctx *c, const void *hidden, const int32_t *row_index, int M,
+                        cudaStream_t st);
+
+// ---- selection / verification (select_verify.cu) ------------------------------------
+cudaError_t launch_select(Ctx *c, const float *conf, const int32_t *token, const int32_t *row_index,
+                          int M, int K, int B, int L, const mrp_select_params &p,
+                          const mrp_select_out &out, cudaStream_t st);
+cudaError_t launch_verify(Ctx *c, const int32_t *draft_tok, const int32_t *verify_tok,
+                          const int32_t *draft_len, int B, int Kd, int positionwise,
+                          int32_t *accept_len, int8_t *accept_mask, cudaStream_t st);
+
+// ---- tensor-core kernel family (tc_*.cu) ---------------------------------------------
+bool tc_supported(const mrp_config &cfg, const mrp_head_weights *heads, const void *w_lm);
+cudaError_t tc_create(Ctx *c);
+void tc_destroy(Ctx *c);
+cudaError_t tc_draft(Ctx *c, const void *hidden, const float *logits0, const int32_t *row_index,
+                     int M, int K, const mrp_draft_out &out, cudaStream_t st);
+
+// Merge of two partial statistics; ties on the maximum go to the lower token id.
+__device__ inline Partial merge_partial(const Partial &a, const Partial &b)
+{
+    Partial r;
+    const bool b_wins = (b.mx > a.mx) || (b.mx == a.mx && b.idx < a.idx);
+    const float hi = b_wins ? b.mx : a.mx;
+    const float lo = b_wins ? a.mx : b.mx;
+    r.mx = hi;
+    r.idx = b_wins ? b.idx : a.idx;
+    float sec = lo;
+    sec = a.second > sec ? a.second : sec;
+    sec = b.second > sec ? b.second : sec;
+    r.second = sec;
+    const float ea = (a.sum == 0.f) ? 0.f : a.sum * expf(a.mx - hi);
+    const float eb = (b.sum == 0.f) ? 0.f : b.sum * expf(b.mx - hi);
+    r.sum = ea + eb;
+    return r;
+}
+
+}  // namespace mrp

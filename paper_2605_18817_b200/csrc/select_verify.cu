@@ -1,0 +1,208 @@
+// Reveal selection, remasking and draft verification: one warp per (sequence, block).
+//
+// STATIC   (Algorithm 2 "Reveal r tokens with highest confidence"; Algorithm 3 "Draft token
+//           with highest confidence"): for k = 0..K the r most confident still-masked
+//           positions under step k, confidence descending then position ascending.
+// DYNAMIC  (Algorithm 4; Sec. 4.1 dynamic denoising; Sec. 4.4 cap): R = {conf_0 >= tau},
+//           at least one, optionally capped; remask members of R whose updated confidence
+//           is below the same tau.
+// VERIFY   (Algorithm 3 "Reject drafted positions where argmax differ"; Figure 1(d)).
+// Lane l owns block positions l, l+32, ... (up to 32 strides, i.e. L <= 1024); membership
+// sets are per-lane bit masks over the strides.
+#include <limits.h>
+
+#include "mrp_internal.cuh"
+
+namespace mrp {
+
+__global__ void scatter_rows_kernel(const int32_t *__restrict__ row_index, int M,
+                                    int32_t *__restrict__ dense_row)
+{
+    const int m = blockIdx.x * blockDim.x + threadIdx.x;
+    if (m < M) dense_row[row_index ? row_index[m] : m] = m;
+}
+
+// Most confident position among the lanes' candidate bit sets under confidences c[row]:
+// (confidence desc, position asc).  Returns the block position or INT_MAX if none.
+__device__ __forceinline__ int warp_best(uint32_t cand, const float *__restrict__ c,
+                                         const int32_t *__restrict__ rows, int lane)
+{
+    float bc = -INFINITY;
+    int bi = INT_MAX;
+    while (cand) {
+        const int s = __ffs(cand) - 1;
+        cand &= cand - 1;
+        const int i = lane + 32 * s;
+        const float v = c[rows[i]];
+        if (bi == INT_MAX || v > bc || (v == bc && i < bi)) { bc = v; bi = i; }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float oc = __shfl_xor_sync(0xffffffffu, bc, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+        if (oi != INT_MAX && (bi == INT_MAX || oc > bc || (oc == bc && oi < bi))) { bc = oc; bi = oi; }
+    }
+    return bi;
+}
+
+__device__ __forceinline__ int warp_popc(uint32_t bits)
+{
+    int n = __popc(bits);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) n += __shfl_xor_sync(0xffffffffu, n, o);
+    return n;
+}
+
+__global__ void __launch_bounds__(32)
+select_kernel(const float *__restrict__ conf, const int32_t *__restrict__ token,
+              const int32_t *__restrict__ dense_row, int M, int K, int L, mrp_select_params p,
+              mrp_select_out out, int Kd)
+{
+    const int b = blockIdx.x, lane = threadIdx.x;
+    const int32_t *rows = dense_row + (size_t)b * L;
+    int8_t *reveal = out.reveal_mask + (size_t)b * L, *remask = out.remask_mask + (size_t)b * L;
+    int32_t *otok = out.out_token + (size_t)b * L;
+    int8_t *step = out.step_of + (size_t)b * L;
+    for (int i = lane; i < L; i += 32) { reveal[i] = 0; remask[i] = 0; otok[i] = -1; step[i] = -1; }
+    for (int q = lane; q < Kd; q += 32) {
+        out.draft_pos[(size_t)b * Kd + q] = -1;
+        out.draft_tok[(size_t)b * Kd + q] = -1;
+    }
+    __syncwarp();
+    uint32_t avail = 0;
+    for (int s = 0; lane + 32 * s < L; ++s)
+        if (rows[lane + 32 * s] >= 0) avail |= 1u << s;
+    const int n = warp_popc(avail);
+    int dl = 0;
+    if (n > 0 && p.mode == MRP_SELECT_STATIC) {
+        for (int k = 0; k <= K; ++k) {
+            const int r = (k == 0) ? p.r_reveal : p.r_draft;
+            const float *ck = conf + (size_t)k * M;
+            for (int t = 0; t < r; ++t) {
+                const int bi = warp_best(avail, ck, rows, lane);
+                if (bi == INT_MAX) break;
+                if ((bi & 31) == lane) {
+                    avail &= ~(1u << (bi >> 5));
+                    const int32_t tk = token[(size_t)k * M + rows[bi]];
+                    otok[bi] = tk;
+                    step[bi] = (int8_t)k;
+                    if (k == 0) {
+                        reveal[bi] = 1;
+                    } else {
+                        out.draft_pos[(size_t)b * Kd + dl] = bi;
+                        out.draft_tok[(size_t)b * Kd + dl] = tk;
+                    }
+                }
+                if (k > 0) ++dl;
+            }
+        }
+    } else if (n > 0) {
+        uint32_t inR = 0;
+        for (uint32_t c = avail; c; c &= c - 1) {
+            const int s = __ffs(c) - 1;
+            if (conf[rows[lane + 32 * s]] >= p.tau) inR |= 1u << s;
+        }
+        int nR = warp_popc(inR);
+        if (nR == 0 && p.ensure_progress) {
+            const int bi = warp_best(avail, conf, rows, lane);
+            if ((bi & 31) == lane) inR |= 1u << (bi >> 5);
+            nR = 1;
+        }
+        if (p.use_cap) {
+            int cap = (7 * n) / 10;
+            cap = cap < 5 ? 5 : cap;
+            cap = cap > L ? L : cap;
+            if (nR > cap) {
+                uint32_t cand = inR, keep = 0;
+                for (int t = 0; t < cap; ++t) {
+                    const int bi = warp_best(cand, conf, rows, lane);
+                    if ((bi & 31) == lane) { cand &= ~(1u << (bi >> 5)); keep |= 1u << (bi >> 5); }
+                }
+                inR = keep;
+                nR = cap;
+            }
+        }
+        uint32_t rem = 0;
+        for (uint32_t c = inR; c; c &= c - 1) {
+            const int s = __ffs(c) - 1;
+            const int m = rows[lane + 32 * s];
+            float c2;
+            if (K == 0) {
+                c2 = conf[m];
+            } else if (p.remask_policy == 1) {
+                c2 = conf[(size_t)K * M + m];
+            } else {
+                c2 = conf[(size_t)M + m];
+                for (int k = 2; k <= K; ++k) c2 = fminf(c2, conf[(size_t)k * M + m]);
+            }
+            if (c2 < p.tau) rem |= 1u << s;
+        }
+        const int kept = warp_popc(inR & ~rem);
+        if (kept == 0 && nR > 0 && p.ensure_progress) {
+            const int bi = warp_best(inR, conf, rows, lane);
+            if ((bi & 31) == lane) rem &= ~(1u << (bi >> 5));
+        }
+        for (uint32_t c = inR; c; c &= c - 1) {
+            const int s = __ffs(c) - 1;
+            const int i = lane + 32 * s;
+            reveal[i] = 1;
+            if (rem & (1u << s)) {
+                remask[i] = 1;
+            } else {
+                otok[i] = token[rows[i]];
+                step[i] = 0;
+            }
+        }
+    }
+    if (lane == 0) out.draft_len[b] = dl;
+}
+
+__global__ void verify_kernel(const int32_t *__restrict__ draft_tok,
+                              const int32_t *__restrict__ verify_tok,
+                              const int32_t *__restrict__ draft_len, int B, int Kd, int positionwise,
+                              int32_t *__restrict__ accept_len, int8_t *__restrict__ accept_mask)
+{
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= B) return;
+    int n = draft_len[b];
+    n = n > Kd ? Kd : (n < 0 ? 0 : n);
+    int acc = 0;
+    bool alive = true;
+    for (int j = 0; j < Kd; ++j) {
+        bool ok = (j < n) && (draft_tok[(size_t)b * Kd + j] == verify_tok[(size_t)b * Kd + j]);
+        if (!positionwise) { alive = alive && ok; ok = alive; }
+        accept_mask[(size_t)b * Kd + j] = (int8_t)ok;
+        acc += ok;
+    }
+    accept_len[b] = acc;
+}
+
+cudaError_t launch_select(Ctx *c, const float *conf, const int32_t *token, const int32_t *row_index,
+                          int M, int K, int B, int L, const mrp_select_params &p,
+                          const mrp_select_out &out, cudaStream_t st)
+{
+    int32_t *dense_row = (int32_t *)(c->ws + c->lay.dense_row);
+    cudaError_t e = cudaMemsetAsync(dense_row, 0xFF, sizeof(int32_t) * (size_t)B * L, st);
+    if (e != cudaSuccess) return e;
+    if (M > 0) {
+        scatter_rows_kernel<<<(M + 255) / 256, 256, 0, st>>>(row_index, M, dense_row);
+        c->launches++;
+    }
+    const int Kd = K * (p.r_draft > 0 ? p.r_draft : 0);
+    select_kernel<<<B, 32, 0, st>>>(conf, token, dense_row, M, K, L, p, out, Kd);
+    c->launches++;
+    return cudaGetLastError();
+}
+
+cudaError_t launch_verify(Ctx *c, const int32_t *draft_tok, const int32_t *verify_tok,
+                          const int32_t *draft_len, int B, int Kd, int positionwise,
+                          int32_t *accept_len, int8_t *accept_mask, cudaStream_t st)
+{
+    if (B == 0) return cudaSuccess;
+    verify_kernel<<<(B + 127) / 128, 128, 0, st>>>(draft_tok, verify_tok, draft_len, B, Kd,
+                                                   positionwise, accept_len, accept_mask);
+    c->launches++;
+    return cudaGetLastError();
+}
+
+}  // namespace mrp

@@ -1,0 +1,343 @@
+// CUDA-core kernel family of the MRP drafting pass.
+//
+// This family computes everything in fp32 on the CUDA cores from fp32 or bf16 weights.  It is
+// the production path of fp32 contexts (the tiny configuration), the path of bf16 shapes the
+// tensor-core kernels do not cover, and an on-device cross-check of the tcgen05 family.
+// Steps (Algorithm 2, inner loop): gather masked rows -> per head: RMSNorm, gate/up + SwiGLU,
+// down projection and h <- h + Delta -> LM head on h_k - h_0 added to l_0 with per-slice
+// softmax statistics -> combine over slices.
+#include <float.h>
+#include <limits.h>
+
+#include "mrp_internal.cuh"
+
+namespace mrp {
+
+__device__ __forceinline__ float ld_f(const float *p, size_t i) { return p[i]; }
+__device__ __forceinline__ float ld_f(const __nv_bfloat16 *p, size_t i) { return __bfloat162float(p[i]); }
+
+__device__ __forceinline__ float warp_sum(float v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// ---- a0: gather masked rows into the fp32 residual stream --------------------------------
+template <typename T>
+__global__ void prep_kernel(const T *__restrict__ hidden, const int32_t *__restrict__ row_index,
+                            int d, float *__restrict__ h0f, float *__restrict__ hcur)
+{
+    const int m = blockIdx.x;
+    const size_t row = row_index ? (size_t)row_index[m] : (size_t)m;
+    for (int j = threadIdx.x; j < d; j += blockDim.x) {
+        const float v = ld_f(hidden, row * d + j);
+        h0f[(size_t)m * d + j] = v;
+        hcur[(size_t)m * d + j] = v;
+    }
+}
+
+cudaError_t launch_prep(Ctx *c, const void *hidden, const int32_t *row_index, int M, cudaStream_t st)
+{
+    if (M == 0) return cudaSuccess;
+    float *h0f = (float *)(c->ws + c->lay.h0f), *hcur = (float *)(c->ws + c->lay.hcur);
+    if (c->cfg.dtype == MRP_F32)
+        prep_kernel<float><<<M, 256, 0, st>>>((const float *)hidden, row_index, c->cfg.d, h0f, hcur);
+    else
+        prep_kernel<__nv_bfloat16><<<M, 256, 0, st>>>((const __nv_bfloat16 *)hidden, row_index,
+                                                      c->cfg.d, h0f, hcur);
+    c->launches++;
+    return cudaGetLastError();
+}
+
+// ---- a1: RMSNorm of the residual stream --------------------------------------------------
+template <typename T>
+__global__ void rmsnorm_kernel(const float *__restrict__ hcur, const T *__restrict__ gamma, int d,
+                               float eps, float *__restrict__ xg)
+{
+    __shared__ float red[32];
+    const int m = blockIdx.x;
+    const float *h = hcur + (size_t)m * d;
+    float ss = 0.f;
+    for (int j = threadIdx.x; j < d; j += blockDim.x) ss += h[j] * h[j];
+    ss = warp_sum(ss);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        float v = (threadIdx.x < (blockDim.x >> 5)) ? red[threadIdx.x] : 0.f;
+        v = warp_sum(v);
+        if (threadIdx.x == 0) red[0] = v;
+    }
+    __syncthreads();
+    const float rstd = rsqrtf(red[0] / (float)d + eps);
+    for (int j = threadIdx.x; j < d; j += blockDim.x)
+        xg[(size_t)m * d + j] = h[j] * rstd * ld_f(gamma, j);
+}
+
+// ---- a1: gate/up projections + SwiGLU; one warp per inner feature, 4 rows at a time -------
+constexpr int kRC = 4;
+
+template <typename T>
+__global__ void gateup_kernel(const T *__restrict__ w_gate, const T *__restrict__ w_up,
+                              const float *__restrict__ xg, int M, int d, int F,
+                              float *__restrict__ act)
+{
+    const int f = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (f >= F) return;
+    const T *wg = w_gate + (size_t)f * d, *wu = w_up + (size_t)f * d;
+    for (int m0 = 0; m0 < M; m0 += kRC) {
+        float g[kRC], u[kRC];
+#pragma unroll
+        for (int r = 0; r < kRC; ++r) g[r] = u[r] = 0.f;
+        for (int j = lane; j < d; j += 32) {
+            const float a = ld_f(wg, j), b = ld_f(wu, j);
+#pragma unroll
+            for (int r = 0; r < kRC; ++r) {
+                if (m0 + r < M) {
+                    const float x = xg[(size_t)(m0 + r) * d + j];
+                    g[r] = fmaf(a, x, g[r]);
+                    u[r] = fmaf(b, x, u[r]);
+                }
+            }
+        }
+#pragma unroll
+        for (int r = 0; r < kRC; ++r) {
+            const float gs = warp_sum(g[r]), us = warp_sum(u[r]);
+            if (lane == 0 && m0 + r < M)
+                act[(size_t)(m0 + r) * F + f] = gs / (1.f + expf(-gs)) * us;
+        }
+    }
+}
+
+// ---- a1: down projection, h <- h + Delta, LM-head operand h_k - h_0 ------------------------
+template <typename T>
+__global__ void down_kernel(const T *__restrict__ w_down, const float *__restrict__ act, int M,
+                            int d, int F, float *__restrict__ hcur, const float *__restrict__ h0f,
+                            float *__restrict__ xt_k, float *__restrict__ hidden_out)
+{
+    const int j = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (j >= d) return;
+    const T *wd = w_down + (size_t)j * F;
+    for (int m0 = 0; m0 < M; m0 += kRC) {
+        float s[kRC];
+#pragma unroll
+        for (int r = 0; r < kRC; ++r) s[r] = 0.f;
+        for (int f = lane; f < F; f += 32) {
+            const float a = ld_f(wd, f);
+#pragma unroll
+            for (int r = 0; r < kRC; ++r)
+                if (m0 + r < M) s[r] = fmaf(a, act[(size_t)(m0 + r) * F + f], s[r]);
+        }
+#pragma unroll
+        for (int r = 0; r < kRC; ++r) {
+            const float v = warp_sum(s[r]);
+            if (lane == 0 && m0 + r < M) {
+                const size_t o = (size_t)(m0 + r) * d + j;
+                const float hn = hcur[o] + v;
+                hcur[o] = hn;
+                xt_k[o] = hn - h0f[o];
+                if (hidden_out) hidden_out[o] = hn;
+            }
+        }
+    }
+}
+
+// ---- a2 + a3: LM head on the residual, added to l_0, per-slice softmax statistics ---------
+// A block owns vocabulary slices of kSimtSliceV entries (grid-stride over slices).  For each
+// chunk of kLR row-steps rs = k*M + m, the 8 warps compute delta for 16 entries each, the
+// tile l = l_0 + delta goes to shared memory, and warp w reduces row-step w of the chunk.
+constexpr int kLR = 8;
+
+template <typename T>
+__global__ void __launch_bounds__(256)
+lm_simt_kernel(const T *__restrict__ w_lm, const float *__restrict__ xt,
+               const float *__restrict__ logits0, const int32_t *__restrict__ row_index, int M,
+               int K, int d, int V, int n_slices, Partial *__restrict__ partials,
+               float *__restrict__ logits_out)
+{
+    __shared__ float tile[kLR][kSimtSliceV];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n_rs = (K + 1) * M;
+    bool first = true;
+    for (int slice = blockIdx.x; slice < n_slices; slice += gridDim.x, first = false) {
+        const int v0 = slice * kSimtSliceV;
+        for (int rs0 = 0; rs0 < n_rs; rs0 += kLR) {
+            // delta for entries v0 + warp*16 .. +16, row-steps rs0 .. rs0+kLR
+            for (int e = 0; e < kSimtSliceV / 8; ++e) {
+                const int vl = warp * (kSimtSliceV / 8) + e;
+                const int v = v0 + vl;
+                float acc[kLR];
+#pragma unroll
+                for (int r = 0; r < kLR; ++r) acc[r] = 0.f;
+                if (v < V) {
+                    const T *wr = w_lm + (size_t)v * d;
+                    for (int j = lane; j < d; j += 32) {
+                        const float a = ld_f(wr, j);
+#pragma unroll
+                        for (int r = 0; r < kLR; ++r) {
+                            const int rs = rs0 + r;
+                            if (rs < n_rs && rs >= M)   // step 0 has no residual
+                                acc[r] = fmaf(a, xt[(size_t)(rs - M) * d + j], acc[r]);
+                        }
+                    }
+                }
+#pragma unroll
+                for (int r = 0; r < kLR; ++r) {
+                    const float s = warp_sum(acc[r]);
+                    const int rs = rs0 + r;
+                    if (lane == 0) {
+                        float l = -INFINITY;
+                        if (v < V && rs < n_rs) {
+                            const int m = rs % M;
+                            const size_t row = row_index ? (size_t)row_index[m] : (size_t)m;
+                            l = logits0[row * (size_t)V + v] + s;
+                        }
+                        tile[r][vl] = l;
+                    }
+                }
+            }
+            __syncthreads();
+            const int rs = rs0 + warp;
+            if (rs < n_rs) {
+                float mx = -INFINITY, sec = -INFINITY;
+                int idx = INT_MAX;
+                float vals[kSimtSliceV / 32];
+#pragma unroll
+                for (int i = 0; i < kSimtSliceV / 32; ++i) {
+                    const int vl = lane + 32 * i;
+                    const float l = tile[warp][vl];
+                    vals[i] = l;
+                    if (l > mx) { sec = mx; mx = l; idx = v0 + vl; }
+                    else if (l > sec) sec = l;
+                }
+                if (mx == -INFINITY) idx = INT_MAX;
+                // warp merge of (mx, idx, second)
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+                    const float omx = __shfl_xor_sync(0xffffffffu, mx, o);
+                    const int oidx = __shfl_xor_sync(0xffffffffu, idx, o);
+                    const float osec = __shfl_xor_sync(0xffffffffu, sec, o);
+                    const bool ow = (omx > mx) || (omx == mx && oidx < idx);
+                    const float lo = ow ? mx : omx;
+                    float ns = lo > sec ? lo : sec;
+                    ns = osec > ns ? osec : ns;
+                    sec = ns;
+                    if (ow) { mx = omx; idx = oidx; }
+                }
+                float sum = 0.f;
+#pragma unroll
+                for (int i = 0; i < kSimtSliceV / 32; ++i)
+                    sum += (vals[i] == -INFINITY) ? 0.f : expf(vals[i] - mx);
+                sum = warp_sum(sum);
+                if (logits_out && rs >= M) {
+#pragma unroll
+                    for (int i = 0; i < kSimtSliceV / 32; ++i) {
+                        const int v = v0 + lane + 32 * i;
+                        if (v < V) logits_out[(size_t)(rs - M) * V + v] = vals[i];
+                    }
+                }
+                if (lane == 0) {
+                    Partial p;
+                    p.mx = mx; p.sum = sum; p.idx = idx; p.second = sec;
+                    Partial *dst = partials + (size_t)blockIdx.x * n_rs + rs;
+                    if (!first) p = merge_partial(*dst, p);
+                    *dst = p;
+                }
+            }
+            __syncthreads();
+        }
+    }
+}
+
+// ---- a4: combine per-slice partials -------------------------------------------------------
+__global__ void combine_kernel(const Partial *__restrict__ partials, int n_slices, int n_rs,
+                               float *__restrict__ conf, float *__restrict__ lse,
+                               int32_t *__restrict__ token, float *__restrict__ margin,
+                               int32_t *__restrict__ status, int32_t *__restrict__ user_status)
+{
+    const int rs = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (rs >= n_rs) return;
+    Partial p;
+    p.mx = -INFINITY; p.sum = 0.f; p.idx = INT_MAX; p.second = -INFINITY;
+    for (int s = lane; s < n_slices; s += 32) p = merge_partial(p, partials[(size_t)s * n_rs + rs]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        Partial q;
+        q.mx = __shfl_xor_sync(0xffffffffu, p.mx, o);
+        q.sum = __shfl_xor_sync(0xffffffffu, p.sum, o);
+        q.idx = __shfl_xor_sync(0xffffffffu, p.idx, o);
+        q.second = __shfl_xor_sync(0xffffffffu, p.second, o);
+        // fixed operand order (lower lane first) keeps the result identical on both sides
+        p = (lane & o) ? merge_partial(q, p) : merge_partial(p, q);
+    }
+    if (lane == 0) {
+        const float l = p.mx + logf(p.sum);
+        conf[rs] = 1.f / p.sum;
+        lse[rs] = l;
+        token[rs] = p.idx;
+        if (margin) margin[rs] = p.mx - p.second;
+        if (!isfinite(l)) {
+            atomicOr(status, MRP_DEV_NONFINITE);
+            if (user_status) atomicOr(user_status, MRP_DEV_NONFINITE);
+        }
+    }
+}
+
+cudaError_t launch_combine(Ctx *c, const Partial *partials, int n_slices, int n_rowsteps,
+                           const mrp_draft_out &out, int32_t *status, cudaStream_t st)
+{
+    if (n_rowsteps == 0) return cudaSuccess;
+    const int warps = 4;
+    combine_kernel<<<(n_rowsteps + warps - 1) / warps, warps * 32, 0, st>>>(
+        partials, n_slices, n_rowsteps, out.conf, out.lse, out.token, out.margin, status, out.status);
+    c->launches++;
+    return cudaGetLastError();
+}
+
+template <typename T>
+static cudaError_t simt_draft_t(Ctx *c, const void *hidden, const float *logits0,
+                                const int32_t *row_index, int M, int K, const mrp_draft_out &out,
+                                cudaStream_t st)
+{
+    const int d = c->cfg.d, F = c->cfg.d_ff, V = c->cfg.vocab;
+    float *h0f = (float *)(c->ws + c->lay.h0f), *hcur = (float *)(c->ws + c->lay.hcur);
+    float *xg = (float *)(c->ws + c->lay.xg), *act = (float *)(c->ws + c->lay.act);
+    float *xt = (float *)(c->ws + c->lay.xt);
+    Partial *partials = (Partial *)(c->ws + c->lay.partials);
+    int32_t *status = (int32_t *)(c->ws + c->lay.status);
+    cudaError_t e = launch_prep(c, hidden, row_index, M, st);
+    if (e != cudaSuccess) return e;
+    if (K == 0 && out.hidden_out)
+        cudaMemcpyAsync(out.hidden_out, h0f, sizeof(float) * (size_t)M * d, cudaMemcpyDeviceToDevice, st);
+    for (int k = 1; k <= K; ++k) {
+        const mrp_head_weights &hw = c->heads[k - 1];
+        rmsnorm_kernel<T><<<M, 256, 0, st>>>(hcur, (const T *)hw.rms_gamma, d, c->cfg.rms_eps, xg);
+        gateup_kernel<T><<<(F + 7) / 8, 256, 0, st>>>((const T *)hw.w_gate, (const T *)hw.w_up, xg, M, d, F, act);
+        down_kernel<T><<<(d + 7) / 8, 256, 0, st>>>((const T *)hw.w_down, act, M, d, F, hcur, h0f,
+                                                    xt + (size_t)(k - 1) * M * d,
+                                                    (k == K) ? out.hidden_out : nullptr);
+        c->launches += 3;
+    }
+    const int n_slices = (V + kSimtSliceV - 1) / kSimtSliceV;
+    const int grid = n_slices < kSimtMaxBlocks ? n_slices : kSimtMaxBlocks;
+    lm_simt_kernel<T><<<grid, 256, 0, st>>>((const T *)c->w_lm, xt, logits0, row_index, M, K, d, V,
+                                            n_slices, partials, out.logits_out);
+    c->launches++;
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    return launch_combine(c, partials, grid, (K + 1) * M, out, status, st);
+}
+
+cudaError_t simt_draft(Ctx *c, const void *hidden, const float *logits0, const int32_t *row_index,
+                       int M, int K, const mrp_draft_out &out, cudaStream_t st)
+{
+    if (M == 0) return cudaSuccess;
+    if (c->cfg.dtype == MRP_F32)
+        return simt_draft_t<float>(c, hidden, logits0, row_index, M, K, out, st);
+    return simt_draft_t<__nv_bfloat16>(c, hidden, logits0, row_index, M, K, out, st);
+}
+
+}  // namespace mrp

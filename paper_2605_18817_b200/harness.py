@@ -1,0 +1,97 @@
+"""Device-memory plumbing around the binding: upload synthetic weights/inputs, allocate
+output tensors, call the C ABI.  No arithmetic of the method happens here."""
+from __future__ import annotations
+
+from dataclasses import dataclass
+
+import numpy as np
+import torch
+
+from . import binding, synth
+
+
+def to_device(a: np.ndarray, dtype: str, device) -> torch.Tensor:
+    """float32 host array -> CUDA tensor in the storage dtype (bf16 values are exact)."""
+    if dtype == "bf16":
+        bits = synth.bf16_bits(a)
+        return torch.from_numpy(bits.view(np.int16)).to(device).view(torch.bfloat16)
+    return torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).to(device)
+
+
+def upload_weights(w: synth.Weights, device):
+    heads = [{k: to_device(v, w.dtype, device) for k, v in h.items()} for h in w.heads]
+    return heads, to_device(w.w_lm, w.dtype, device)
+
+
+@dataclass
+class DraftOut:
+    conf: torch.Tensor
+    lse: torch.Tensor
+    token: torch.Tensor
+    margin: torch.Tensor | None
+    logits: torch.Tensor | None
+    hidden: torch.Tensor | None
+    status: torch.Tensor
+
+
+def alloc_draft_out(M, K, V, d, device, margin=True, logits=False, hidden=False) -> DraftOut:
+    f = dict(device=device, dtype=torch.float32)
+    return DraftOut(
+        torch.empty((K + 1, M), **f), torch.empty((K + 1, M), **f),
+        torch.empty((K + 1, M), device=device, dtype=torch.int32),
+        torch.empty((K + 1, M), **f) if margin else None,
+        torch.empty((K, M, V), **f) if logits else None,
+        torch.empty((M, d), **f) if hidden else None,
+        torch.zeros(1, device=device, dtype=torch.int32))
+
+
+def draft(ctx, hidden, logits0, row_index, M, K, out: DraftOut, stream=None):
+    binding.mrp_draft(ctx, hidden, logits0, row_index, M, K, out.conf, out.lse, out.token,
+                      out.margin, out.logits, out.hidden, out.status, stream=stream)
+    return out
+
+
+@dataclass
+class SelectOut:
+    reveal_mask: torch.Tensor
+    remask_mask: torch.Tensor
+    out_token: torch.Tensor
+    step_of: torch.Tensor
+    draft_pos: torch.Tensor
+    draft_tok: torch.Tensor
+    draft_len: torch.Tensor
+
+
+def alloc_select_out(B, L, Kd, device) -> SelectOut:
+    i8 = dict(device=device, dtype=torch.int8)
+    i32 = dict(device=device, dtype=torch.int32)
+    return SelectOut(torch.empty(B * L, **i8), torch.empty(B * L, **i8), torch.empty(B * L, **i32),
+                     torch.empty(B * L, **i8), torch.empty((B, Kd), **i32),
+                     torch.empty((B, Kd), **i32), torch.empty(B, **i32))
+
+
+def select(ctx, conf, token, row_index, M, K, B, L, mode, out: SelectOut, **kw):
+    binding.mrp_reveal_remask(ctx, conf, token, row_index, M, K, B, L, mode,
+                              reveal_mask=out.reveal_mask, remask_mask=out.remask_mask,
+                              out_token=out.out_token, step_of=out.step_of,
+                              draft_pos=out.draft_pos, draft_tok=out.draft_tok,
+                              draft_len=out.draft_len, **kw)
+    return out
+
+
+def verify(ctx, draft_tok, verify_tok, draft_len, positionwise=False):
+    B, Kd = draft_tok.shape
+    accept_len = torch.empty(B, device=draft_tok.device, dtype=torch.int32)
+    accept_mask = torch.empty((B, Kd), device=draft_tok.device, dtype=torch.int8)
+    binding.mrp_verify(ctx, draft_tok, verify_tok, draft_len, B, Kd, positionwise, accept_len,
+                       accept_mask)
+    return accept_len, accept_mask
+
+
+def create_for(cfg: dict, w: synth.Weights, device, max_rows=None, flags=0):
+    """Context for a configuration dict plus the uploaded weights."""
+    heads, w_lm = upload_weights(w, device)
+    rows = cfg["B"] * cfg["L"] if max_rows is None else max_rows
+    ctx = binding.mrp_create(w.d, w.F, w.V, heads, w_lm, max_rows=rows, max_seqs=cfg["B"],
+                             block_len=cfg["L"], flags=flags)
+    return ctx

@@ -116,11 +116,13 @@ class Inputs:
 
 
 def make_inputs(w: Weights, B: int, L: int, seed: int, s_lo: float, s_hi: float,
-                mask_prob: float = 1.0, calibrated: bool = True) -> Inputs:
+                mask_prob: float = 1.0, calibrated: bool = True, logits_fn=None) -> Inputs:
     """Backbone outputs for one active block per sequence.
 
     ``mask_prob`` < 1 masks each position independently (at least one per block, by
-    resampling the block); 1.0 masks every position.
+    resampling the block); 1.0 masks every position.  ``logits_fn(hidden_rows)`` may replace
+    the host matrix product that produces the base logits (e.g. an fp32 product on another
+    device); whatever it returns is the input both sides then share.
     """
     n = B * L
     d, V = w.d, w.V
@@ -150,7 +152,7 @@ def make_inputs(w: Weights, B: int, L: int, seed: int, s_lo: float, s_hi: float,
     step = 256
     for i in range(0, row_index.size, step):                 # base logits = LM head on h
         idx = row_index[i:i + step]
-        logits0[idx] = hidden[idx] @ w.w_lm.T
+        logits0[idx] = logits_fn(hidden[idx]) if logits_fn else hidden[idx] @ w.w_lm.T
     return Inputs(B, L, hidden, logits0, row_index, planted, strength)
 
 
@@ -187,11 +189,11 @@ def sweep_config(M: int, K: int) -> dict:
                 mode="static", seed=4000 + p)
 
 
-def make_config(cfg: dict, weights: Weights | None = None):
+def make_config(cfg: dict, weights: Weights | None = None, logits_fn=None):
     """Weights (unless given) and inputs of a configuration dict."""
     if weights is None:
         weights = make_weights(cfg["d"], cfg["F"], cfg["V"], cfg["n_heads"], cfg["dtype"],
                                cfg["seed"])
     inp = make_inputs(weights, cfg["B"], cfg["L"], cfg["seed"], cfg["s_lo"], cfg["s_hi"],
-                      cfg["mask_prob"])
+                      cfg["mask_prob"], logits_fn=logits_fn)
     return weights, inp

@@ -1,0 +1,182 @@
+"""Full-size parity: the five benchmark configurations run through the C ABI at their real
+shapes; the oracle recomputes sampled rows (all V columns) or whole sampled blocks."""
+import gc
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2605_18817_b200 import binding, harness, synth
+from test_gpu_parity import DEV, _assert_select_equal, check_stats
+
+pytestmark = pytest.mark.gpu
+
+
+class Device:
+    """Weights uploaded once, contexts created per (rows, seqs, block) shape."""
+
+    def __init__(self, w):
+        self.w = w
+        self.heads, self.w_lm = harness.upload_weights(w, DEV)
+        self.w_lm_f32 = None
+
+    def logits_fn(self, rows):
+        # base logits of the synthetic backbone: fp32 product on the device (input data)
+        if self.w_lm_f32 is None:
+            torch.backends.cuda.matmul.allow_tf32 = False
+        x = torch.from_numpy(rows).to(DEV)
+        out = torch.empty((x.shape[0], self.w.V), device=DEV)
+        step = 16384
+        for v0 in range(0, self.w.V, step):
+            out[:, v0:v0 + step] = x @ self.w_lm[v0:v0 + step].float().T
+        return out.cpu().numpy()
+
+    def ctx(self, rows, seqs, block, n_heads=None, flags=0):
+        heads = self.heads if n_heads is None else self.heads[:n_heads]
+        return binding.mrp_create(self.w.d, self.w.F, self.w.V, heads, self.w_lm, max_rows=rows,
+                                  max_seqs=seqs, block_len=block, flags=flags)
+
+
+def gpu_draft(dev, ctx, inp, K, **kw):
+    M = len(inp.row_index)
+    hid = harness.to_device(inp.hidden, dev.w.dtype, DEV)
+    l0 = torch.from_numpy(inp.logits0).to(DEV)
+    ri = torch.from_numpy(inp.row_index).to(DEV)
+    out = harness.alloc_draft_out(M, K, dev.w.V, dev.w.d, DEV, **kw)
+    harness.draft(ctx, hid, l0, ri, M, K, out)
+    torch.cuda.synchronize()
+    return out, ri
+
+
+def test_config1_decode_shape_all_rows():
+    cfg = synth.CONFIGS[1]
+    w = synth.make_weights(cfg["d"], cfg["F"], cfg["V"], cfg["n_heads"], cfg["dtype"], cfg["seed"])
+    dev = Device(w)
+    _, inp = synth.make_config(cfg, w)
+    ctx = dev.ctx(4, 1, 4)
+    out, ri = gpu_draft(dev, ctx, inp, cfg["K"], logits=True, hidden=True)
+    ref = oracle.draft(inp.hidden, inp.logits0, w.heads, w.w_lm, K=cfg["K"], row_index=inp.row_index,
+                       want_logits=True, want_hidden=True)
+    check_stats(out, ref, "bf16")
+    lg = out.logits.cpu().numpy().astype(np.float64)
+    rms = np.sqrt((ref.logits ** 2).mean(axis=2, keepdims=True))
+    assert np.all(np.abs(lg - ref.logits) <= 2e-2 * np.maximum(np.abs(ref.logits), rms))
+    assert np.abs(out.hidden.cpu().numpy() - ref.hidden).max() <= 2e-2
+    # static reveal + drafts, then verification against synthetic backbone tokens
+    K, B, L, M = cfg["K"], 1, 4, 4
+    sel = harness.alloc_select_out(B, L, K, DEV)
+    harness.select(ctx, out.conf, out.token, ri, M, K, B, L, binding.MRP_SELECT_STATIC, sel)
+    torch.cuda.synchronize()
+    osel = oracle.select(out.conf.cpu().numpy(), out.token.cpu().numpy(), inp.row_index, B, L,
+                         oracle.STATIC)
+    _assert_select_equal(sel, osel)
+    binding.mrp_destroy(ctx)
+
+
+def test_config2_speculative_shape_sampled_rows_and_verify():
+    cfg = synth.CONFIGS[2]
+    w = synth.make_weights(cfg["d"], cfg["F"], cfg["V"], cfg["n_heads"], cfg["dtype"], cfg["seed"])
+    dev = Device(w)
+    _, inp = synth.make_config(cfg, w, logits_fn=dev.logits_fn)
+    K, B, L = cfg["K"], cfg["B"], cfg["L"]
+    M = len(inp.row_index)
+    assert M == 128
+    ctx = dev.ctx(M, B, L)
+    out, ri = gpu_draft(dev, ctx, inp, K)
+    sample = np.array([0, 37, 64, 101, 126, 127])
+    ref = oracle.draft(inp.hidden, inp.logits0, w.heads, w.w_lm, K=K, row_index=inp.row_index[sample])
+    check_stats(out, ref, "bf16", cols=sample)
+    # selection on the device's own statistics is bit-exact against the oracle's rules
+    sel = harness.alloc_select_out(B, L, K, DEV)
+    harness.select(ctx, out.conf, out.token, ri, M, K, B, L, binding.MRP_SELECT_STATIC, sel)
+    torch.cuda.synchronize()
+    osel = oracle.select(out.conf.cpu().numpy(), out.token.cpu().numpy(), inp.row_index, B, L,
+                         oracle.STATIC)
+    _assert_select_equal(sel, osel)
+    # verification: backbone tokens equal the draft with probability 0.7 per slot
+    dt = sel.draft_tok.cpu().numpy()
+    vt = synth.make_verify_tokens(dt, w.V, cfg["seed"], 0.7)
+    al, am = harness.verify(ctx, sel.draft_tok, torch.from_numpy(vt).to(DEV), sel.draft_len)
+    torch.cuda.synchronize()
+    ol, om = oracle.verify(dt, vt, sel.draft_len.cpu().numpy())
+    assert np.array_equal(al.cpu().numpy(), ol) and np.array_equal(am.cpu().numpy(), om)
+    assert 0 < ol.mean() < K
+    binding.mrp_destroy(ctx)
+    del dev, w
+    gc.collect()
+
+
+def test_config3_remask_shape_sampled_blocks():
+    cfg = synth.CONFIGS[3]
+    w = synth.make_weights(cfg["d"], cfg["F"], cfg["V"], cfg["n_heads"], cfg["dtype"], cfg["seed"])
+    dev = Device(w)
+    _, inp = synth.make_config(cfg, w, logits_fn=dev.logits_fn)
+    K, B, L, tau = cfg["K"], cfg["B"], cfg["L"], cfg["tau"]
+    M = len(inp.row_index)
+    assert 850 < M < 1200
+    ctx = dev.ctx(B * L, B, L)
+    out, ri = gpu_draft(dev, ctx, inp, K)
+    for policy in (0, 1):
+        sel = harness.alloc_select_out(B, L, K, DEV)
+        harness.select(ctx, out.conf, out.token, ri, M, K, B, L, binding.MRP_SELECT_DYNAMIC_REMASK,
+                       sel, tau=tau, remask_policy=policy)
+        torch.cuda.synchronize()
+        # (i) the rules, bit-exact, on the device's own statistics
+        osel = oracle.select(out.conf.cpu().numpy(), out.token.cpu().numpy(), inp.row_index, B, L,
+                             oracle.DYNAMIC_REMASK, tau=tau, remask_policy=policy)
+        _assert_select_equal(sel, osel)
+        assert 0 < osel.remask_mask.sum() < osel.reveal_mask.sum()
+    # (ii) end to end on three whole blocks, recomputed by the oracle
+    blocks = [0, 31, 63]
+    rows = np.flatnonzero(np.isin(inp.row_index // L, blocks))
+    ref = oracle.draft(inp.hidden, inp.logits0, w.heads, w.w_lm, K=K, row_index=inp.row_index[rows])
+    check_stats(out, ref, "bf16", cols=rows)
+    checked = 0
+    sel_np = {n: getattr(sel, n).cpu().numpy() for n in ("reveal_mask", "remask_mask", "out_token")}
+    for b in blocks:
+        r = np.flatnonzero(inp.row_index[rows] // L == b)
+        conf_b = ref.conf[:, r].astype(np.float32)
+        if np.abs(conf_b - tau).min() < 2e-3 or (ref.margin[:, r] <= 1e-2).any():
+            continue                      # a decision inside the tolerance band: not unique
+        ri_b = (inp.row_index[rows][r] % L).astype(np.int32)
+        o = oracle.select(conf_b, ref.token[:, r], ri_b, 1, L, oracle.DYNAMIC_REMASK, tau=tau,
+                          remask_policy=1)
+        sl = slice(b * L, (b + 1) * L)
+        assert np.array_equal(sel_np["reveal_mask"][sl], o.reveal_mask)
+        assert np.array_equal(sel_np["remask_mask"][sl], o.remask_mask)
+        assert np.array_equal(sel_np["out_token"][sl], o.out_token)
+        checked += 1
+    assert checked >= 1
+    binding.mrp_destroy(ctx)
+    del dev, w
+    gc.collect()
+
+
+@pytest.fixture(scope="module")
+def sweep_dev():
+    w = synth.make_weights(4096, 8192, 151936, 4, "bf16", 4000)
+    dev = Device(w)
+    yield dev
+
+
+@pytest.mark.parametrize("M,K", [(1, 1), (4, 2), (16, 4), (64, 2), (256, 4), (1024, 1), (4096, 4)])
+def test_sweep_points_sampled_rows(sweep_dev, M, K):
+    dev = sweep_dev
+    cfg = synth.sweep_config(M, K)
+    _, inp = synth.make_config(cfg, dev.w, logits_fn=dev.logits_fn)
+    ctx = dev.ctx(M, M, 1, n_heads=K)
+    out, _ = gpu_draft(dev, ctx, inp, K, margin=False)
+    sample = np.unique(np.array([0, M // 3, M // 2, M - 1]))
+    ref = oracle.draft(inp.hidden, inp.logits0, dev.w.heads, dev.w.w_lm, K=K,
+                       row_index=inp.row_index[sample])
+    check_stats(out, ref, "bf16", cols=sample)
+    # properties that hold at any size, checked on every row
+    conf = out.conf.cpu().numpy()
+    assert np.all(conf > 1.0 / dev.w.V) and np.all(conf <= 1.0 + 1e-6)
+    tok = out.token.cpu().numpy()
+    assert tok.min() >= 0 and tok.max() < dev.w.V
+    l0 = torch.from_numpy(inp.logits0).to(DEV)
+    assert torch.equal(l0.argmax(dim=1).int().cpu(), out.token[0].cpu())
+    assert torch.allclose(torch.logsumexp(l0, dim=1), out.lse[0], atol=2e-3)
+    binding.mrp_destroy(ctx)

@@ -1,0 +1,233 @@
+"""Parity of the CUDA path (through the C ABI) against the CPU oracle on the same seeded
+inputs.  Tolerances: integer outputs bit-exact wherever the oracle's top-2 logit margin
+exceeds 1e-2; confidence and log-sum-exp within 2e-3 absolute on bf16 contexts (1e-5 on
+fp32 contexts); materialised logits within 2e-2 relative to max(|logit|, row RMS)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2605_18817_b200 import binding, harness, synth
+
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda:0"
+TOL = {"f32": 1e-5, "bf16": 2e-3}
+
+
+def run_gpu_draft(w, inp, K, flags=0, margin=True, logits=False, hidden=False, row_index="inp",
+                  ctx=None):
+    heads, w_lm = (None, None)
+    own = ctx is None
+    if own:
+        heads, w_lm = harness.upload_weights(w, DEV)
+        ctx = binding.mrp_create(w.d, w.F, w.V, heads, w_lm, max_rows=max(inp.B * inp.L, 1),
+                                 max_seqs=inp.B, block_len=inp.L, flags=flags)
+    ri = inp.row_index if isinstance(row_index, str) else row_index
+    M = inp.hidden.shape[0] if ri is None else len(ri)
+    hid = harness.to_device(inp.hidden, w.dtype, DEV)
+    l0 = torch.from_numpy(inp.logits0).to(DEV)
+    ri_t = None if ri is None else torch.from_numpy(np.asarray(ri, np.int32)).to(DEV)
+    out = harness.alloc_draft_out(M, K, w.V, w.d, DEV, margin=margin, logits=logits, hidden=hidden)
+    harness.draft(ctx, hid, l0, ri_t, M, K, out)
+    torch.cuda.synchronize()
+    fam = ctx.family
+    if own:
+        binding.mrp_destroy(ctx)
+    return out, fam
+
+
+def check_stats(out, ref, dtype, cols=None):
+    """Compare conf/lse/token of the GPU (all rows, or the columns `cols`) with the oracle."""
+    tol = TOL[dtype]
+    conf = out.conf.cpu().numpy().astype(np.float64)
+    lse = out.lse.cpu().numpy().astype(np.float64)
+    tok = out.token.cpu().numpy()
+    if cols is not None:
+        conf, lse, tok = conf[:, cols], lse[:, cols], tok[:, cols]
+    assert conf.shape == ref.conf.shape
+    assert np.abs(conf - ref.conf).max() <= tol, np.abs(conf - ref.conf).max()
+    assert np.abs(lse - ref.lse).max() <= tol, np.abs(lse - ref.lse).max()
+    clear = ref.margin > 1e-2
+    assert clear.mean() > 0.5
+    assert np.array_equal(tok[clear], ref.token[clear])
+    if out.margin is not None:
+        mg = out.margin.cpu().numpy().astype(np.float64)
+        if cols is not None:
+            mg = mg[:, cols]
+        assert np.abs(mg - ref.margin).max() <= max(10 * tol, 2e-2)
+    assert int(out.status.item()) == 0
+
+
+def test_config0_fp32_all_outputs():
+    cfg = synth.CONFIGS[0]
+    w, inp = synth.make_config(cfg)
+    out, fam = run_gpu_draft(w, inp, cfg["K"], logits=True, hidden=True)
+    assert fam == "simt"
+    ref = oracle.draft(inp.hidden, inp.logits0, w.heads, w.w_lm, K=cfg["K"], row_index=inp.row_index,
+                       want_logits=True, want_hidden=True)
+    check_stats(out, ref, "f32")
+    lg = out.logits.cpu().numpy().astype(np.float64)
+    assert np.abs(lg - ref.logits).max() <= 1e-4
+    assert np.abs(out.hidden.cpu().numpy() - ref.hidden).max() <= 1e-4
+
+
+@pytest.mark.parametrize("dtype,flags", [("f32", 0), ("bf16", binding.MRP_FLAG_FORCE_SIMT)])
+def test_ragged_shapes_on_cuda_cores(dtype, flags):
+    # sizes that are not multiples of any tile: d, F, V ragged, odd row count, row subset
+    w = synth.make_weights(72, 136, 1000, 3, dtype, 31, head_std=0.1)
+    for k, h in enumerate(w.heads):
+        h["gamma"] = (1.0 + 0.25 * np.cos(np.arange(72) + k)).astype(np.float32)
+        if dtype == "bf16":
+            h["gamma"] = synth.bf16_round(h["gamma"])
+    inp = synth.make_inputs(w, 5, 3, 31, 1.0, 4.0, mask_prob=0.7)
+    out, fam = run_gpu_draft(w, inp, 3, flags=flags, logits=True, hidden=True)
+    assert fam == "simt"
+    ref = oracle.draft(inp.hidden, inp.logits0, w.heads, w.w_lm, row_index=inp.row_index,
+                       want_logits=True, want_hidden=True)
+    check_stats(out, ref, "f32")     # the CUDA-core family keeps fp32 intermediates
+    assert np.abs(out.logits.cpu().numpy() - ref.logits).max() <= 1e-4
+    assert np.abs(out.hidden.cpu().numpy() - ref.hidden).max() <= 1e-4
+    # chain truncated to K = 1 and K = 0
+    for K in (1, 0):
+        o, _ = run_gpu_draft(w, inp, K, flags=flags)
+        r = oracle.draft(inp.hidden, inp.logits0, w.heads, w.w_lm, K=K, row_index=inp.row_index)
+        check_stats(o, r, "f32")
+
+
+def test_empty_call_and_argument_errors():
+    cfg = synth.CONFIGS[0]
+    w, inp = synth.make_config(cfg)
+    ctx = harness.create_for(cfg, w, DEV)
+    out = harness.alloc_draft_out(4, 3, w.V, w.d, DEV)
+    hid = harness.to_device(inp.hidden, w.dtype, DEV)
+    l0 = torch.from_numpy(inp.logits0).to(DEV)
+    out.conf.fill_(-7.0)
+    harness.draft(ctx, hid, l0, None, 0, 3, out)          # M = 0: nothing is written
+    torch.cuda.synchronize()
+    assert float(out.conf.min()) == -7.0 and ctx.last_launch_count == 0
+    with pytest.raises(binding.MrpError):                  # M beyond max_rows
+        harness.draft(ctx, hid, l0, None, 5, 3, out)
+    with pytest.raises(binding.MrpError):                  # K beyond n_heads
+        harness.draft(ctx, hid, l0, None, 4, 4, out)
+    with pytest.raises(binding.MrpError):                  # missing required output
+        binding.mrp_draft(ctx, hid, l0, None, 4, 3, None, out.lse, out.token)
+    harness.draft(ctx, hid, l0, None, 4, 3, out)           # context still usable
+    torch.cuda.synchronize()
+    assert float(out.conf.min()) > 0
+    binding.mrp_destroy(ctx)
+
+
+def _rand_select_case(rng, K, B, L, mask_prob):
+    mask = rng.random((B, L)) < mask_prob
+    ri = np.flatnonzero(mask.reshape(-1)).astype(np.int32)
+    rng.shuffle(ri)                                        # row order need not be ascending
+    M = ri.size
+    conf = rng.random((K + 1, M)).astype(np.float32)
+    # plant exact ties and exact threshold hits
+    if M > 3:
+        conf[:, 1] = conf[:, 0]
+        conf[0, 2] = np.float32(0.5)
+    token = rng.integers(0, 1000, (K + 1, M)).astype(np.int32)
+    return ri, conf, token
+
+
+@pytest.fixture(scope="module")
+def select_ctx():
+    w = synth.make_weights(16, 16, 32, 0, "f32", 1)
+    heads, w_lm = harness.upload_weights(w, DEV)
+    ctx = binding.mrp_create(16, 16, 32, heads, w_lm, max_rows=64 * 100, max_seqs=64, block_len=100)
+    yield ctx
+    binding.mrp_destroy(ctx)
+
+
+def _gpu_select(ctx, conf, token, ri, B, L, mode, **kw):
+    K = conf.shape[0] - 1
+    M = conf.shape[1]
+    Kd = K * kw.get("r_draft", 1)
+    out = harness.alloc_select_out(B, L, Kd, DEV)
+    c = torch.from_numpy(conf).to(DEV)
+    t = torch.from_numpy(token).to(DEV)
+    r = torch.from_numpy(ri).to(DEV) if ri is not None else None
+    harness.select(ctx, c, t, r, M, K, B, L, mode, out, **kw)
+    torch.cuda.synchronize()
+    return out
+
+
+def _assert_select_equal(g, o):
+    for name in ("reveal_mask", "remask_mask", "out_token", "step_of", "draft_pos", "draft_tok",
+                 "draft_len"):
+        a = getattr(g, name).cpu().numpy()
+        b = getattr(o, name)
+        assert np.array_equal(a.reshape(b.shape), b), name
+
+
+@pytest.mark.parametrize("L", [1, 4, 16, 32, 33, 100])
+def test_select_bit_exact_on_shared_statistics(select_ctx, L):
+    rng = np.random.default_rng(L)
+    for case in range(6):
+        K = case % 4
+        B = 1 + (case * 7) % 23
+        ri, conf, token = _rand_select_case(rng, K, B, L, 0.3 + 0.1 * case)
+        if ri.size == 0:
+            continue
+        kw = dict(r_reveal=1 + case % 3, r_draft=case % 3)
+        g = _gpu_select(select_ctx, conf, token, ri, B, L, binding.MRP_SELECT_STATIC, **kw)
+        o = oracle.select(conf, token, ri, B, L, oracle.STATIC, **kw)
+        _assert_select_equal(g, o)
+        for tau in (0.0, 0.3, 0.5, 0.8, 1.5):
+            for cap in (False, True):
+                for policy in (0, 1):
+                    for prog in (True, False):
+                        kw = dict(tau=tau, use_cap=cap, remask_policy=policy, ensure_progress=prog)
+                        g = _gpu_select(select_ctx, conf, token, ri, B, L,
+                                        binding.MRP_SELECT_DYNAMIC_REMASK, **kw)
+                        o = oracle.select(conf, token, ri, B, L, oracle.DYNAMIC_REMASK, **kw)
+                        _assert_select_equal(g, o)
+
+
+def test_select_with_no_masked_rows_writes_defaults(select_ctx):
+    out = harness.alloc_select_out(3, 4, 2, DEV)
+    empty_f = torch.empty((3, 0), device=DEV)
+    empty_i = torch.empty((3, 0), device=DEV, dtype=torch.int32)
+    harness.select(select_ctx, empty_f, empty_i, None, 0, 2, 3, 4, binding.MRP_SELECT_STATIC, out)
+    torch.cuda.synchronize()
+    assert not out.reveal_mask.any() and bool((out.out_token == -1).all())
+    assert bool((out.draft_pos == -1).all()) and not out.draft_len.any()
+
+
+def test_verify_bit_exact(select_ctx):
+    rng = np.random.default_rng(5)
+    for B, Kd in ((1, 1), (32, 3), (64, 4), (7, 12)):
+        d = rng.integers(0, 50, (B, Kd)).astype(np.int32)
+        v = synth.make_verify_tokens(d, 50, seed=B, p_match=0.7)
+        n = rng.integers(0, Kd + 1, B).astype(np.int32)
+        for pw in (False, True):
+            al, am = harness.verify(select_ctx, torch.from_numpy(d).to(DEV), torch.from_numpy(v).to(DEV),
+                                    torch.from_numpy(n).to(DEV), positionwise=pw)
+            torch.cuda.synchronize()
+            ol, om = oracle.verify(d, v, n, positionwise=pw)
+            assert np.array_equal(al.cpu().numpy(), ol) and np.array_equal(am.cpu().numpy(), om)
+
+
+def test_config0_static_selection_end_to_end():
+    cfg = synth.CONFIGS[0]
+    w, inp = synth.make_config(cfg)
+    ctx = harness.create_for(cfg, w, DEV)
+    K, B, L = cfg["K"], cfg["B"], cfg["L"]
+    M = len(inp.row_index)
+    hid = harness.to_device(inp.hidden, w.dtype, DEV)
+    l0 = torch.from_numpy(inp.logits0).to(DEV)
+    ri = torch.from_numpy(inp.row_index).to(DEV)
+    out = harness.alloc_draft_out(M, K, w.V, w.d, DEV)
+    harness.draft(ctx, hid, l0, ri, M, K, out)
+    sel = harness.alloc_select_out(B, L, K, DEV)
+    harness.select(ctx, out.conf, out.token, ri, M, K, B, L, binding.MRP_SELECT_STATIC, sel)
+    torch.cuda.synchronize()
+    ref = oracle.draft(inp.hidden, inp.logits0, w.heads, w.w_lm, K=K, row_index=inp.row_index)
+    osel = oracle.select(ref.conf.astype(np.float32), ref.token, inp.row_index, B, L, oracle.STATIC)
+    # the four confidences of this instance are separated by far more than the tolerance
+    gaps = np.abs(ref.conf[:, :, None] - ref.conf[:, None, :])[:, ~np.eye(M, dtype=bool)]
+    assert gaps.min() > 1e-4
+    _assert_select_equal(sel, osel)
+    binding.mrp_destroy(ctx)
