@@ -206,6 +206,18 @@ int mrp_verify(mrp_ctx *ctx, const int32_t *draft_tok, const int32_t *verify_tok
  * context launched (for accounting in benchmarks). */
 int32_t mrp_last_launch_count(const mrp_ctx *ctx);
 
+/*
+ * Per-phase timing of mrp_draft for benchmarks (no counterpart in the paper).  While enabled,
+ * every mrp_draft call records CUDA events on its stream around three phases: 0 = row gather
+ * and head chain, 1 = fused LM-head kernel, 2 = combine.  mrp_profile_read must be called
+ * after the stream has been synchronised; it returns the summed milliseconds of each phase
+ * over the calls since the last read (the most recent 1024 at most) in ms_phase[3] (HOST),
+ * their number in *n_calls (HOST), and restarts the count.  Enabling creates CUDA events
+ * (no device memory); disabling destroys them.  Errors: INVALID_ARG, NOMEM, CUDA.
+ */
+int mrp_profile_enable(mrp_ctx *ctx, int32_t enable);
+int mrp_profile_read(mrp_ctx *ctx, float *ms_phase, int32_t *n_calls);
+
 /* Name of the kernel family a bf16/fp32 context resolved to: "simt" or "tcgen05". */
 const char *mrp_kernel_family(const mrp_ctx *ctx);
 

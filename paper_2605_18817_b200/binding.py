@@ -23,7 +23,8 @@ MRP_SELECT_STATIC, MRP_SELECT_DYNAMIC_REMASK = 0, 1
 MRP_DEV_NONFINITE, MRP_DEV_TIMEOUT = 1, 2
 
 EXPORTS = ("mrp_workspace_bytes", "mrp_create", "mrp_destroy", "mrp_draft", "mrp_reveal_remask",
-           "mrp_verify", "mrp_last_launch_count", "mrp_kernel_family", "mrp_status_string")
+           "mrp_verify", "mrp_last_launch_count", "mrp_kernel_family", "mrp_status_string",
+           "mrp_profile_enable", "mrp_profile_read")
 
 
 class mrp_config(ctypes.Structure):
@@ -88,6 +89,11 @@ def _load():
     lib.mrp_verify.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
                                ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p,
                                ctypes.c_void_p, ctypes.c_void_p]
+    lib.mrp_profile_enable.restype = ctypes.c_int
+    lib.mrp_profile_enable.argtypes = [ctypes.c_void_p, ctypes.c_int32]
+    lib.mrp_profile_read.restype = ctypes.c_int
+    lib.mrp_profile_read.argtypes = [ctypes.c_void_p, ctypes.POINTER(ctypes.c_float),
+                                     ctypes.POINTER(ctypes.c_int32)]
     lib.mrp_last_launch_count.restype = ctypes.c_int32
     lib.mrp_last_launch_count.argtypes = [ctypes.c_void_p]
     lib.mrp_kernel_family.restype = ctypes.c_char_p
@@ -179,6 +185,22 @@ def mrp_destroy(ctx: Context) -> None:
     if ctx.handle:
         lib.mrp_destroy(ctx.handle)
         ctx.handle = 0
+
+
+def mrp_profile_enable(ctx: Context, enable: bool) -> None:
+    rc = lib.mrp_profile_enable(ctx.handle, int(bool(enable)))
+    if rc != 0:
+        raise MrpError("mrp_profile_enable", rc)
+
+
+def mrp_profile_read(ctx: Context):
+    """(ms_heads, ms_lm_head, ms_combine) summed over n calls, and n; sync the stream first."""
+    ms = (ctypes.c_float * 3)()
+    n = ctypes.c_int32()
+    rc = lib.mrp_profile_read(ctx.handle, ms, ctypes.byref(n))
+    if rc != 0:
+        raise MrpError("mrp_profile_read", rc)
+    return (float(ms[0]), float(ms[1]), float(ms[2])), int(n.value)
 
 
 def mrp_draft(ctx: Context, hidden, logits0, row_index, M, K, conf, lse, token, margin=None,

@@ -127,9 +127,65 @@ int mrp_create(const mrp_config *cfg, const mrp_head_weights *heads, const void 
     return MRP_OK;
 }
 
+static void prof_release(Ctx &c)
+{
+    if (c.prof_events) {
+        for (int i = 0; i < kProfSlots * kProfMarks; ++i)
+            if (c.prof_events[i]) cudaEventDestroy(c.prof_events[i]);
+        free(c.prof_events);
+        c.prof_events = nullptr;
+    }
+    c.prof_enabled = false;
+    c.prof_calls = 0;
+}
+
+int mrp_profile_enable(mrp_ctx *ctx, int32_t enable)
+{
+    if (!ctx) return MRP_ERR_INVALID_ARG;
+    Ctx &c = ctx->c;
+    DeviceGuard guard(c.cfg.device);
+    if (guard.err != cudaSuccess) return MRP_ERR_CUDA;
+    if (!enable) { prof_release(c); return MRP_OK; }
+    if (!c.prof_events) {
+        c.prof_events = (cudaEvent_t *)calloc((size_t)kProfSlots * kProfMarks, sizeof(cudaEvent_t));
+        if (!c.prof_events) return MRP_ERR_NOMEM;
+        for (int i = 0; i < kProfSlots * kProfMarks; ++i)
+            if (cudaEventCreate(&c.prof_events[i]) != cudaSuccess) { prof_release(c); return MRP_ERR_CUDA; }
+    }
+    c.prof_calls = 0;
+    c.prof_enabled = true;
+    return MRP_OK;
+}
+
+int mrp_profile_read(mrp_ctx *ctx, float *ms_phase, int32_t *n_calls)
+{
+    if (!ctx || !ms_phase || !n_calls) return MRP_ERR_INVALID_ARG;
+    Ctx &c = ctx->c;
+    ms_phase[0] = ms_phase[1] = ms_phase[2] = 0.f;
+    *n_calls = 0;
+    if (!c.prof_enabled) return MRP_OK;
+    DeviceGuard guard(c.cfg.device);
+    if (guard.err != cudaSuccess) return MRP_ERR_CUDA;
+    const int n = (int)(c.prof_calls < kProfSlots ? c.prof_calls : kProfSlots);
+    double acc[3] = {0, 0, 0};
+    for (int i = 0; i < n; ++i) {
+        cudaEvent_t *ev = c.prof_events + (size_t)i * kProfMarks;
+        for (int ph = 0; ph < 3; ++ph) {
+            float ms = 0.f;
+            if (cudaEventElapsedTime(&ms, ev[ph], ev[ph + 1]) != cudaSuccess) return MRP_ERR_CUDA;
+            acc[ph] += ms;
+        }
+    }
+    for (int ph = 0; ph < 3; ++ph) ms_phase[ph] = (float)acc[ph];
+    *n_calls = n;
+    c.prof_calls = 0;
+    return MRP_OK;
+}
+
 void mrp_destroy(mrp_ctx *ctx)
 {
     if (!ctx) return;
+    prof_release(ctx->c);
     if (ctx->c.use_tc) tc_destroy(&ctx->c);
     free(ctx->c.heads);
     delete ctx;

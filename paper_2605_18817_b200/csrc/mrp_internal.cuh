@@ -49,7 +49,21 @@ struct Ctx {
     int32_t launches;
     int sm_count;
     void *tc_state;            // tensor-core path state (tensor maps), owned by tc_*.cu
+    // Optional per-phase timing of mrp_draft (CUDA events on the call's stream).
+    bool prof_enabled;
+    cudaEvent_t *prof_events;  // [kProfSlots][kProfMarks]
+    int64_t prof_calls;
 };
+
+constexpr int kProfSlots = 1024;
+constexpr int kProfMarks = 4;   // start, after head chain, after LM head, after combine
+
+inline void prof_mark(Ctx *c, int mark, cudaStream_t st)
+{
+    if (!c->prof_enabled) return;
+    cudaEventRecord(c->prof_events[(c->prof_calls % kProfSlots) * kProfMarks + mark], st);
+    if (mark == kProfMarks - 1) c->prof_calls++;
+}
 
 // ---- CUDA-core kernel family (simt_kernels.cu) -------------------------------------
 cudaError_t simt_draft(Ctx *c, const void *hidden, const float *logits0, const int32_t *row_index,

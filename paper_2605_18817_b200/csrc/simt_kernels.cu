@@ -308,6 +308,7 @@ static cudaError_t simt_draft_t(Ctx *c, const void *hidden, const float *logits0
     float *xt = (float *)(c->ws + c->lay.xt);
     Partial *partials = (Partial *)(c->ws + c->lay.partials);
     int32_t *status = (int32_t *)(c->ws + c->lay.status);
+    prof_mark(c, 0, st);
     cudaError_t e = launch_prep(c, hidden, row_index, M, st);
     if (e != cudaSuccess) return e;
     if (K == 0 && out.hidden_out)
@@ -321,6 +322,7 @@ static cudaError_t simt_draft_t(Ctx *c, const void *hidden, const float *logits0
                                                     (k == K) ? out.hidden_out : nullptr);
         c->launches += 3;
     }
+    prof_mark(c, 1, st);
     const int n_slices = (V + kSimtSliceV - 1) / kSimtSliceV;
     const int grid = n_slices < kSimtMaxBlocks ? n_slices : kSimtMaxBlocks;
     lm_simt_kernel<T><<<grid, 256, 0, st>>>((const T *)c->w_lm, xt, logits0, row_index, M, K, d, V,
@@ -328,7 +330,10 @@ static cudaError_t simt_draft_t(Ctx *c, const void *hidden, const float *logits0
     c->launches++;
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    return launch_combine(c, partials, grid, (K + 1) * M, out, status, st);
+    prof_mark(c, 2, st);
+    e = launch_combine(c, partials, grid, (K + 1) * M, out, status, st);
+    prof_mark(c, 3, st);
+    return e;
 }
 
 cudaError_t simt_draft(Ctx *c, const void *hidden, const float *logits0, const int32_t *row_index,
