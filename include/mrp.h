@@ -218,6 +218,10 @@ int32_t mrp_last_launch_count(const mrp_ctx *ctx);
 int mrp_profile_enable(mrp_ctx *ctx, int32_t enable);
 int mrp_profile_read(mrp_ctx *ctx, float *ms_phase, int32_t *n_calls);
 
+/* Detail of the last failed call on this context (which CUDA call, its error string); an
+ * empty string if the last mrp_draft succeeded.  The pointer stays valid until mrp_destroy. */
+const char *mrp_last_error(const mrp_ctx *ctx);
+
 /* Name of the kernel family a bf16/fp32 context resolved to: "simt" or "tcgen05". */
 const char *mrp_kernel_family(const mrp_ctx *ctx);
 

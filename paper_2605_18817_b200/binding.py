@@ -24,7 +24,7 @@ MRP_DEV_NONFINITE, MRP_DEV_TIMEOUT = 1, 2
 
 EXPORTS = ("mrp_workspace_bytes", "mrp_create", "mrp_destroy", "mrp_draft", "mrp_reveal_remask",
            "mrp_verify", "mrp_last_launch_count", "mrp_kernel_family", "mrp_status_string",
-           "mrp_profile_enable", "mrp_profile_read")
+           "mrp_profile_enable", "mrp_profile_read", "mrp_last_error")
 
 
 class mrp_config(ctypes.Structure):
@@ -96,6 +96,8 @@ def _load():
                                      ctypes.POINTER(ctypes.c_int32)]
     lib.mrp_last_launch_count.restype = ctypes.c_int32
     lib.mrp_last_launch_count.argtypes = [ctypes.c_void_p]
+    lib.mrp_last_error.restype = ctypes.c_char_p
+    lib.mrp_last_error.argtypes = [ctypes.c_void_p]
     lib.mrp_kernel_family.restype = ctypes.c_char_p
     lib.mrp_kernel_family.argtypes = [ctypes.c_void_p]
     lib.mrp_status_string.restype = ctypes.c_char_p
@@ -107,9 +109,10 @@ lib = _load()
 
 
 class MrpError(RuntimeError):
-    def __init__(self, where: str, status: int):
+    def __init__(self, where: str, status: int, detail: str = ""):
         self.status = status
-        super().__init__("%s: %s (%d)" % (where, lib.mrp_status_string(status).decode(), status))
+        super().__init__("%s: %s (%d)%s" % (where, lib.mrp_status_string(status).decode(), status,
+                                            " -- " + detail if detail else ""))
 
 
 def _ptr(t):
@@ -219,7 +222,7 @@ def mrp_draft(ctx: Context, hidden, logits0, row_index, M, K, conf, lse, token, 
     rc = lib.mrp_draft(ctx.handle, _ptr(hidden), _ptr(logits0), _ptr(row_index), int(M), int(K),
                        ctypes.byref(out), _stream(stream))
     if rc != 0:
-        raise MrpError("mrp_draft", rc)
+        raise MrpError("mrp_draft", rc, lib.mrp_last_error(ctx.handle).decode())
 
 
 def mrp_reveal_remask(ctx: Context, conf, token, row_index, M, K, B, L, mode, tau=0.9, r_reveal=1,

@@ -25,6 +25,7 @@ WorkspaceLayout workspace_layout(const mrp_config &cfg)
     l.sumsq = take((size_t)kSumsqSlices * rows * 4);
     const int v_slices = (cfg.vocab + kSimtSliceV - 1) / kSimtSliceV;
     l.n_slices_max = v_slices < kSimtMaxBlocks ? v_slices : kSimtMaxBlocks;
+    if (l.n_slices_max < kSumsqSlices) l.n_slices_max = kSumsqSlices;   // one slice per CTA (tc family)
     l.partials = take((size_t)l.n_slices_max * steps * rows * sizeof(Partial));
     l.dense_row = take((size_t)cfg.max_seqs * (size_t)cfg.block_len * 4);
     l.total = off;
@@ -204,8 +205,10 @@ int mrp_draft(mrp_ctx *ctx, const void *hidden, const float *logits0, const int3
     DeviceGuard guard(c.cfg.device);
     if (guard.err != cudaSuccess) return MRP_ERR_CUDA;
     cudaStream_t st = (cudaStream_t)cuda_stream;
+    c.err[0] = 0;
     cudaError_t e = c.use_tc ? tc_draft(&c, hidden, logits0, row_index, M, K, *out, st)
                              : simt_draft(&c, hidden, logits0, row_index, M, K, *out, st);
+    if (e != cudaSuccess && !c.err[0]) note_err(&c, e, "mrp_draft");
     return e == cudaSuccess ? MRP_OK : MRP_ERR_CUDA;
 }
 
@@ -253,6 +256,8 @@ int mrp_verify(mrp_ctx *ctx, const int32_t *draft_tok, const int32_t *verify_tok
 }
 
 int32_t mrp_last_launch_count(const mrp_ctx *ctx) { return ctx ? ctx->c.launches : 0; }
+
+const char *mrp_last_error(const mrp_ctx *ctx) { return ctx ? ctx->c.err : ""; }
 
 const char *mrp_kernel_family(const mrp_ctx *ctx)
 {

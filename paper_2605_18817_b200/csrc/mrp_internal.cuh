@@ -3,6 +3,7 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <stdio.h>
 
 #include "mrp.h"
 
@@ -50,10 +51,18 @@ struct Ctx {
     int sm_count;
     void *tc_state;            // tensor-core path state (tensor maps), owned by tc_*.cu
     // Optional per-phase timing of mrp_draft (CUDA events on the call's stream).
+    char err[192];             // detail of the last failure ("" if none)
     bool prof_enabled;
     cudaEvent_t *prof_events;  // [kProfSlots][kProfMarks]
     int64_t prof_calls;
 };
+
+// Records where a CUDA call failed; returns the error unchanged.
+inline cudaError_t note_err(Ctx *c, cudaError_t e, const char *where)
+{
+    if (e != cudaSuccess) snprintf(c->err, sizeof(c->err), "%s: %s", where, cudaGetErrorString(e));
+    return e;
+}
 
 constexpr int kProfSlots = 1024;
 constexpr int kProfMarks = 4;   // start, after head chain, after LM head, after combine

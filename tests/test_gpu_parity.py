@@ -231,3 +231,35 @@ def test_config0_static_selection_end_to_end():
     assert gaps.min() > 1e-4
     _assert_select_equal(sel, osel)
     binding.mrp_destroy(ctx)
+
+
+@pytest.mark.parametrize("d,F,V,B,L,K", [
+    (256, 512, 4096, 2, 4, 2),      # all row-steps stacked in one 128-row block
+    (128, 256, 2048, 10, 4, 3),     # 160 row-steps: one accumulator per step, M < 128
+    (192, 320, 4112, 150, 1, 2),    # two row blocks, vocabulary not a multiple of the tile
+    (64, 64, 1024, 128, 1, 1),      # exactly one full row block
+    (256, 512, 4096, 75, 4, 4),     # 300 rows, four accumulators
+    (64, 128, 160, 3, 1, 1),        # fewer vocabulary units than CTAs
+])
+def test_tensor_core_family_small_shapes(d, F, V, B, L, K):
+    w = synth.make_weights(d, F, V, K, "bf16", 77, head_std=0.05)
+    for k, h in enumerate(w.heads):
+        h["gamma"] = synth.bf16_round((1.0 + 0.25 * np.cos(np.arange(d) + k)).astype(np.float32))
+    inp = synth.make_inputs(w, B, L, 77, 1.0, 4.0)
+    out, fam = run_gpu_draft(w, inp, K, logits=True, hidden=True)
+    assert fam == "tcgen05"
+    ref = oracle.draft(inp.hidden, inp.logits0, w.heads, w.w_lm, K=K, row_index=inp.row_index,
+                       want_logits=True, want_hidden=True)
+    check_stats(out, ref, "bf16")
+    lg = out.logits.cpu().numpy().astype(np.float64)
+    rms = np.sqrt((ref.logits ** 2).mean(axis=2, keepdims=True))
+    assert np.all(np.abs(lg - ref.logits) <= 2e-2 * np.maximum(np.abs(ref.logits), rms))
+    assert np.abs(out.hidden.cpu().numpy() - ref.hidden).max() <= 2e-2
+    # without the optional outputs the statistics are identical
+    out2, _ = run_gpu_draft(w, inp, K, margin=False)
+    assert torch.equal(out2.conf, out.conf) and torch.equal(out2.token, out.token)
+    # a row subset through row_index, shorter chain
+    sub = inp.row_index[::3]
+    out3, _ = run_gpu_draft(w, inp, max(K - 1, 1), row_index=sub)
+    ref3 = oracle.draft(inp.hidden, inp.logits0, w.heads, w.w_lm, K=max(K - 1, 1), row_index=sub)
+    check_stats(out3, ref3, "bf16")
