@@ -43,7 +43,8 @@ typedef enum {
     MRP_ERR_CUDA = 3,          /* a CUDA runtime / driver call failed                   */
     MRP_ERR_NOMEM = 4,         /* workspace too small, or host allocation failed        */
     MRP_ERR_NONFINITE = 5,
-    MRP_ERR_TIMEOUT = 6
+    MRP_ERR_TIMEOUT = 6,
+    MRP_ERR_CAPACITY = 7       /* size beyond a fixed built-in capacity (mrp_reveal_remask_noalloc) */
 } mrp_status;
 
 /* Bits of the device status word. */
@@ -201,6 +202,34 @@ int mrp_reveal_remask(mrp_ctx *ctx, const float *conf, const int32_t *token,
 int mrp_verify(mrp_ctx *ctx, const int32_t *draft_tok, const int32_t *verify_tok,
                const int32_t *draft_len, int32_t B, int32_t Kd, int32_t positionwise,
                int32_t *accept_len, int8_t *accept_mask, void *cuda_stream);
+
+/*
+ * mrp_reveal_remask without a context and without any allocation (the paper has no
+ * counterpart: this is a packaging variant of the call above, same rules, same outputs).
+ *
+ * For callers that cannot allocate device memory and therefore cannot hand mrp_create a
+ * workspace: an engine whose own pool already owns the whole GPU, a plugin running inside a
+ * foreign CUDA context, a latency path on which cudaMalloc (which may synchronise the device)
+ * is off limits.  The one piece of scratch the selection needs, the map from dense block
+ * position to masked row, lives in a fixed array inside the library instead: 4 bytes x
+ * MRP_NOALLOC_MAX_POSITIONS = 256 KiB of device memory on every GPU that loads the library,
+ * held until the process exits.
+ *   - B * L must not exceed MRP_NOALLOC_MAX_POSITIONS, else MRP_ERR_CAPACITY (nothing is
+ *     launched); L <= 1024.  All other arguments, layouts and errors as mrp_reveal_remask;
+ *     the caller still owns every input and output buffer.
+ *   - Works on the CURRENT device, which must be the device of cuda_stream and of the buffers.
+ *   - The first call on each device looks up the array's device address
+ *     (cudaGetSymbolAddress); make that first call outside of any stream capture.  Later
+ *     calls only enqueue a memset and two kernels.  Never calls cudaMalloc / cudaFree.
+ *   - All calls on a device share the one array.  Each call re-initialises the part it uses,
+ *     so earlier calls leave nothing behind, but two calls that may overlap on the GPU
+ *     (different streams, no ordering between them) race on it: serialise them.
+ */
+#define MRP_NOALLOC_MAX_POSITIONS 65536
+int mrp_reveal_remask_noalloc(const float *conf, const int32_t *token, const int32_t *row_index,
+                              int32_t M, int32_t K, int32_t B, int32_t L,
+                              const mrp_select_params *params, const mrp_select_out *out,
+                              void *cuda_stream);
 
 /* Number of kernels the last mrp_draft / mrp_reveal_remask / mrp_verify call on this
  * context launched (for accounting in benchmarks). */

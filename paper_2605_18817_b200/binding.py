@@ -24,7 +24,10 @@ MRP_DEV_NONFINITE, MRP_DEV_TIMEOUT = 1, 2
 
 EXPORTS = ("mrp_workspace_bytes", "mrp_create", "mrp_destroy", "mrp_draft", "mrp_reveal_remask",
            "mrp_verify", "mrp_last_launch_count", "mrp_kernel_family", "mrp_status_string",
-           "mrp_profile_enable", "mrp_profile_read", "mrp_last_error")
+           "mrp_profile_enable", "mrp_profile_read", "mrp_last_error",
+           "mrp_reveal_remask_noalloc")
+MRP_NOALLOC_MAX_POSITIONS = 65536
+MRP_ERR_CAPACITY = 7
 
 
 class mrp_config(ctypes.Structure):
@@ -85,6 +88,8 @@ def _load():
                                       ctypes.c_int32, ctypes.c_int32,
                                       ctypes.POINTER(mrp_select_params),
                                       ctypes.POINTER(mrp_select_out), ctypes.c_void_p]
+    lib.mrp_reveal_remask_noalloc.restype = ctypes.c_int
+    lib.mrp_reveal_remask_noalloc.argtypes = lib.mrp_reveal_remask.argtypes[1:]
     lib.mrp_verify.restype = ctypes.c_int
     lib.mrp_verify.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
                                ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p,
@@ -245,6 +250,33 @@ def mrp_reveal_remask(ctx: Context, conf, token, row_index, M, K, B, L, mode, ta
                                int(B), int(L), ctypes.byref(p), ctypes.byref(o), _stream(stream))
     if rc != 0:
         raise MrpError("mrp_reveal_remask", rc)
+
+
+def mrp_reveal_remask_noalloc(conf, token, row_index, M, K, B, L, mode, tau=0.9, r_reveal=1,
+                              r_draft=1, use_cap=False, remask_policy=0, ensure_progress=True, *,
+                              reveal_mask, remask_mask, out_token, step_of, draft_pos, draft_tok,
+                              draft_len, stream=None) -> None:
+    """Reveal selection for callers that cannot allocate device memory: no context and no
+    workspace, the position map lives in a fixed array inside the library (B * L at most
+    MRP_NOALLOC_MAX_POSITIONS).  The tensors' device must be the current device.  Calls on
+    one device share that array, so calls that could overlap on the GPU must be serialised."""
+    _check(conf, torch.float32, "conf")
+    _check(token, torch.int32, "token")
+    _check(row_index, torch.int32, "row_index")
+    for t, dt, nm in ((reveal_mask, torch.int8, "reveal_mask"), (remask_mask, torch.int8, "remask_mask"),
+                      (out_token, torch.int32, "out_token"), (step_of, torch.int8, "step_of"),
+                      (draft_pos, torch.int32, "draft_pos"), (draft_tok, torch.int32, "draft_tok"),
+                      (draft_len, torch.int32, "draft_len")):
+        _check(t, dt, nm)
+    p = mrp_select_params(int(mode), float(tau), int(r_reveal), int(r_draft), int(bool(use_cap)),
+                          int(remask_policy), int(bool(ensure_progress)))
+    o = mrp_select_out(_ptr(reveal_mask), _ptr(remask_mask), _ptr(out_token), _ptr(step_of),
+                       _ptr(draft_pos), _ptr(draft_tok), _ptr(draft_len))
+    rc = lib.mrp_reveal_remask_noalloc(_ptr(conf), _ptr(token), _ptr(row_index), int(M), int(K),
+                                       int(B), int(L), ctypes.byref(p), ctypes.byref(o),
+                                       _stream(stream))
+    if rc != 0:
+        raise MrpError("mrp_reveal_remask_noalloc", rc)
 
 
 def mrp_verify(ctx: Context, draft_tok, verify_tok, draft_len, B, Kd, positionwise, accept_len,

@@ -275,6 +275,7 @@ const char *mrp_status_string(int status)
     case MRP_ERR_NOMEM: return "workspace too small or out of host memory";
     case MRP_ERR_NONFINITE: return "non-finite values";
     case MRP_ERR_TIMEOUT: return "device wait timed out";
+    case MRP_ERR_CAPACITY: return "size exceeds the fixed built-in scratch capacity";
     default: return "unknown status";
     }
 }

@@ -11,6 +11,8 @@
 // sets are per-lane bit masks over the strides.
 #include <limits.h>
 
+#include <mutex>
+
 #include "mrp_internal.cuh"
 
 namespace mrp {
@@ -206,3 +208,66 @@ cudaError_t launch_verify(Ctx *c, const int32_t *draft_tok, const int32_t *verif
 }
 
 }  // namespace mrp
+
+// ---------------------------------------------------------------------------------------
+// Allocation-free selection entry point
+// ---------------------------------------------------------------------------------------
+// Some hosts of this library may not allocate device memory at all once they are running: a
+// serving engine that handed the whole GPU to its own pool allocator, a plugin that lives
+// inside someone else's CUDA context, code on a path where cudaMalloc would synchronise the
+// device or is simply forbidden by policy.  Such a caller cannot provide the workspace a
+// context needs, so reveal selection is offered once more with its only scratch (the dense
+// position -> masked row map) in the fixed array below.  The array exists once per GPU that
+// loads the library and is held until the process exits.
+static __device__ __align__(256) int32_t mrp_noalloc_dense_row[MRP_NOALLOC_MAX_POSITIONS];
+
+namespace {
+constexpr int kNoAllocMaxDevices = 64;
+// Device address of mrp_noalloc_dense_row on each device, resolved on first use.  In host
+// code the array's name is only a handle for the runtime, never a device address.
+int32_t *g_noalloc_ptr[kNoAllocMaxDevices];
+std::mutex g_noalloc_mu;
+}  // namespace
+
+extern "C" int mrp_reveal_remask_noalloc(const float *conf, const int32_t *token,
+                                         const int32_t *row_index, int32_t M, int32_t K, int32_t B,
+                                         int32_t L, const mrp_select_params *params,
+                                         const mrp_select_out *out, void *cuda_stream)
+{
+    using namespace mrp;
+    if (!params || !out) return MRP_ERR_INVALID_ARG;
+    if (B < 1 || L < 1 || L > 1024 || K < 0) return MRP_ERR_INVALID_ARG;
+    if ((long long)B * L > (long long)MRP_NOALLOC_MAX_POSITIONS) return MRP_ERR_CAPACITY;
+    if (M < 0 || (long long)M > (long long)B * L) return MRP_ERR_INVALID_ARG;
+    if (M > 0 && (!conf || !token)) return MRP_ERR_INVALID_ARG;
+    if (params->mode != MRP_SELECT_STATIC && params->mode != MRP_SELECT_DYNAMIC_REMASK)
+        return MRP_ERR_INVALID_ARG;
+    if (params->r_reveal < 0 || params->r_draft < 0) return MRP_ERR_INVALID_ARG;
+    if (params->remask_policy != 0 && params->remask_policy != 1) return MRP_ERR_INVALID_ARG;
+    if (!out->reveal_mask || !out->remask_mask || !out->out_token || !out->step_of || !out->draft_len)
+        return MRP_ERR_INVALID_ARG;
+    const int Kd = K * params->r_draft;
+    if (Kd > 0 && (!out->draft_pos || !out->draft_tok)) return MRP_ERR_INVALID_ARG;
+
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return MRP_ERR_CUDA;
+    if (dev < 0 || dev >= kNoAllocMaxDevices) return MRP_ERR_UNSUPPORTED;
+    int32_t *dense_row = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_noalloc_mu);
+        if (!g_noalloc_ptr[dev]) {
+            // once per device, with that device current
+            void *p = nullptr;
+            if (cudaGetSymbolAddress(&p, mrp_noalloc_dense_row) != cudaSuccess || !p) return MRP_ERR_CUDA;
+            g_noalloc_ptr[dev] = (int32_t *)p;
+        }
+        dense_row = g_noalloc_ptr[dev];
+    }
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    // the array still holds the previous call's map: every position of this call starts at -1
+    if (cudaMemsetAsync(dense_row, 0xFF, sizeof(int32_t) * (size_t)B * L, st) != cudaSuccess)
+        return MRP_ERR_CUDA;
+    if (M > 0) scatter_rows_kernel<<<(M + 255) / 256, 256, 0, st>>>(row_index, M, dense_row);
+    select_kernel<<<B, 32, 0, st>>>(conf, token, dense_row, M, K, L, *params, *out, Kd);
+    return cudaGetLastError() == cudaSuccess ? MRP_OK : MRP_ERR_CUDA;
+}
