@@ -41,6 +41,7 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="1",
                     help="0..3 = benchmark configuration, or sweep:M:K for a roofline-sweep point")
+    ap.add_argument("--flags", type=int, default=0, help="mrp_config.flags (MRP_FLAG_* bits) for A/B timing")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     return ap.parse_args()
@@ -247,7 +248,7 @@ def main():
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
-    if rank == 0:
+    if rank == 0 and not os.environ.get("MRP_B200_LIB"):
         _build.build()
     dist = None
     if world > 1:
@@ -264,7 +265,7 @@ def main():
     K, B, L = cfg["K"], cfg["B"], cfg["L"]
     M = len(inp.row_index)
     static = cfg["mode"] == "static"
-    ctx = harness.create_for(cfg, w, dev)
+    ctx = harness.create_for(cfg, w, dev, flags=args.flags)
     hid = harness.to_device(inp.hidden, w.dtype, dev)
     l0 = torch.from_numpy(inp.logits0).to(dev)
     ri = torch.from_numpy(inp.row_index).to(dev)

@@ -57,6 +57,10 @@ typedef enum { MRP_F32 = 0, MRP_BF16 = 1 } mrp_dtype;
 #define MRP_FLAG_FORCE_SIMT 1  /* bf16 context: use the CUDA-core kernels instead of the
                                   tensor-core (tcgen05) kernels; a cross-check path      */
 
+#define MRP_FLAG_NO_PDL 2      /* launch every kernel fully serialised (no programmatic
+                                  dependent launch); for timing comparisons               */
+#define MRP_FLAG_ROW_MAJOR_ONLY 4   /* tensor-core family: never use the few-row kernels  */
+
 typedef struct {
     int32_t d;          /* hidden size                                                   */
     int32_t d_ff;       /* SwiGLU inner size F                                           */

@@ -15,10 +15,13 @@ from dataclasses import dataclass
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libmrp_b200.so")
+# MRP_B200_LIB names a library built elsewhere (e.g. an out-of-tree build of the same sources).
+LIB_PATH = os.environ.get("MRP_B200_LIB") or os.path.join(_HERE, "libmrp_b200.so")
 
 MRP_F32, MRP_BF16 = 0, 1
 MRP_FLAG_FORCE_SIMT = 1
+MRP_FLAG_NO_PDL = 2
+MRP_FLAG_ROW_MAJOR_ONLY = 4
 MRP_SELECT_STATIC, MRP_SELECT_DYNAMIC_REMASK = 0, 1
 MRP_DEV_NONFINITE, MRP_DEV_TIMEOUT = 1, 2
 

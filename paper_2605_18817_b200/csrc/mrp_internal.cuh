@@ -100,6 +100,13 @@ void tc_destroy(Ctx *c);
 cudaError_t tc_draft(Ctx *c, const void *hidden, const float *logits0, const int32_t *row_index,
                      int M, int K, const mrp_draft_out &out, cudaStream_t st);
 
+// Few-row variants (tc_skinny.cu): weight rows on the MMA M axis; rows <= 32.
+bool sk_rows_ok(int rows);
+cudaError_t sk_gateup(Ctx *c, int k, int M, int K, int n_ss, const mrp_draft_out &out, cudaStream_t st, bool pdl);
+cudaError_t sk_down(Ctx *c, int k, int M, int K, const mrp_draft_out &out, cudaStream_t st, bool pdl);
+cudaError_t sk_lm(Ctx *c, const float *logits0, const int32_t *row_index, int M, int K,
+                  const mrp_draft_out &out, cudaStream_t st, bool pdl);
+
 // Merge of two partial statistics; ties on the maximum go to the lower token id.
 __device__ inline Partial merge_partial(const Partial &a, const Partial &b)
 {

@@ -1,0 +1,263 @@
+// Pieces shared by the tensor-core kernel files: PTX wrappers (mbarrier, TMA, tcgen05), shared
+// memory / instruction descriptors, bf16 hi+lo splitting, tensor-map encoding.
+#pragma once
+#include <cuda.h>
+#include <limits.h>
+
+#include "mrp_internal.cuh"
+
+namespace mrp {
+namespace {
+
+constexpr int kBK = 64;                    // bf16 elements per k-chunk = one 128-byte swizzle row
+constexpr int kSmemBudget = 230000;        // dynamic shared memory we ask for at most
+constexpr long long kWaitCycles = 3000000000LL;   // bound on any barrier wait (about 1.5 s)
+
+// ---------------------------------------------------------------------------------------
+// PTX wrappers
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait: gives up after kWaitCycles or when another role already gave up.
+template <typename P>
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
+                                          const P &p)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    long long t0 = clock64();
+    uint32_t spins = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if ((++spins & 255u) == 0) {
+            if (*abort_flag) return false;
+            if (clock64() - t0 > kWaitCycles) {
+                *abort_flag = 1;
+                atomicOr(p.status, MRP_DEV_TIMEOUT);
+                if (p.user_status) atomicOr(p.user_status, MRP_DEV_TIMEOUT);
+                return false;
+            }
+        }
+    }
+    return true;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int c0, int c1, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void prefetch_tmap(const CUtensorMap *map)
+{
+    asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t da, uint64_t db, uint32_t idesc, uint32_t acc)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(da), "l"(db), "r"(idesc), "r"(acc) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float *v)
+{
+    uint32_t r[16];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, float *v)
+{
+    uint32_t r[8];
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                 : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ float ex2f(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ float4 ldg_nc4(const float *p)
+{
+    float4 v;
+    asm volatile("ld.global.nc.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p));
+    return v;
+}
+
+// Shared-memory matrix descriptor of a K-major bf16 tile whose rows are 128 bytes, stored with
+// the 128-byte swizzle in 8-row groups of 1024 bytes (what a SWIZZLE_128B TMA box writes).
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr)
+{
+    uint64_t desc = 0;
+    desc |= (uint64_t)((saddr & 0x3FFFFu) >> 4);        // start address, 16-byte units
+    desc |= (uint64_t)1 << 16;                          // leading byte offset (unused with swizzle)
+    desc |= (uint64_t)(1024 >> 4) << 32;                // stride byte offset: 8-row group pitch
+    desc |= (uint64_t)1 << 46;                          // descriptor version (Blackwell)
+    desc |= (uint64_t)2 << 61;                          // layout type: 128-byte swizzle
+    return desc;
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = bn.
+__device__ __forceinline__ uint32_t make_idesc(int bn)
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+}
+
+constexpr float kLog2e = 1.4426950408889634f;
+
+// Online softmax statistics of one logit row, updated 16 columns at a time.
+struct RowStat {
+    float mx, sum, second;
+    int idx;
+    __device__ __forceinline__ void init() { mx = -INFINITY; sum = 0.f; second = -INFINITY; idx = INT_MAX; }
+    template <bool MARGIN>
+    __device__ __forceinline__ void update(const float *l, int v_base)
+    {
+        float cmax = l[0];
+#pragma unroll
+        for (int j = 1; j < 16; ++j) cmax = fmaxf(cmax, l[j]);
+        if (cmax > mx) {
+            int jj = 15;
+#pragma unroll
+            for (int j = 14; j >= 0; --j) jj = (l[j] == cmax) ? j : jj;
+            if (MARGIN) {
+                float c2 = -INFINITY;
+#pragma unroll
+                for (int j = 0; j < 16; ++j) c2 = (j != jj) ? fmaxf(c2, l[j]) : c2;
+                second = fmaxf(mx, c2);
+            }
+            sum *= ex2f((mx - cmax) * kLog2e);
+            mx = cmax;
+            idx = v_base + jj;
+        } else if (MARGIN) {
+            second = fmaxf(second, cmax);
+        }
+        const float ms = mx * kLog2e;
+        float s = 0.f;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) s += ex2f(fmaf(l[j], kLog2e, -ms));
+        sum += s;
+    }
+    __device__ __forceinline__ Partial partial() const
+    {
+        Partial p;
+        p.mx = mx; p.sum = sum; p.idx = idx; p.second = second;
+        return p;
+    }
+};
+
+__device__ __forceinline__ void load16(const float *p, float *v)
+{
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float4 x = ldg_nc4(p + 4 * i);
+        v[4 * i] = x.x; v[4 * i + 1] = x.y; v[4 * i + 2] = x.z; v[4 * i + 3] = x.w;
+    }
+}
+__device__ __forceinline__ void load16_rw(const float *p, float *v)   // data this kernel also writes
+{
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float4 x = *reinterpret_cast<const float4 *>(p + 4 * i);
+        v[4 * i] = x.x; v[4 * i + 1] = x.y; v[4 * i + 2] = x.z; v[4 * i + 3] = x.w;
+    }
+}
+__device__ __forceinline__ void store16(float *p, const float *v)
+{
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+        *reinterpret_cast<float4 *>(p + 4 * i) = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+}
+__device__ __forceinline__ uint32_t pack_bf16(float a, float b)
+{
+    __nv_bfloat162 t = __floats2bfloat162_rn(a, b);
+    return *reinterpret_cast<uint32_t *>(&t);
+}
+// hi = bf16(a, b); lo = bf16 of the rounding remainders.
+__device__ __forceinline__ void split_bf16(float a, float b, uint32_t &hi, uint32_t &lo)
+{
+    const __nv_bfloat16 ha = __float2bfloat16_rn(a), hb = __float2bfloat16_rn(b);
+    __nv_bfloat162 h;
+    h.x = ha; h.y = hb;
+    hi = *reinterpret_cast<uint32_t *>(&h);
+    lo = pack_bf16(a - __bfloat162float(ha), b - __bfloat162float(hb));
+}
+// Stores n (8 or 16) values as bf16 hi at dst and bf16 lo at dst + lo_off.
+template <int N>
+__device__ __forceinline__ void store_split(__nv_bfloat16 *dst, size_t lo_off, const float *v)
+{
+    uint32_t hi[N / 2], lo[N / 2];
+#pragma unroll
+    for (int j = 0; j < N; j += 2) split_bf16(v[j], v[j + 1], hi[j >> 1], lo[j >> 1]);
+    uint4 *dh = reinterpret_cast<uint4 *>(dst), *dl = reinterpret_cast<uint4 *>(dst + lo_off);
+#pragma unroll
+    for (int i = 0; i < N / 8; ++i) {
+        dh[i] = make_uint4(hi[4 * i], hi[4 * i + 1], hi[4 * i + 2], hi[4 * i + 3]);
+        dl[i] = make_uint4(lo[4 * i], lo[4 * i + 1], lo[4 * i + 2], lo[4 * i + 3]);
+    }
+}
+
+}  // namespace
+
+// ---------------------------------------------------------------------------------------
+// Tensor maps
+// ---------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+struct TcState {
+    EncodeTiledFn encode;
+};
+
+// bf16 row-major [rows, inner] matrix, box = [box_rows, 64 elements], 128-byte swizzle,
+// out-of-range elements read as zero.
+inline bool make_map(const TcState *s, CUtensorMap *map, const void *ptr, uint64_t inner, uint64_t rows,
+                     uint32_t box_rows)
+{
+    cuuint64_t dims[2] = {inner, rows};
+    cuuint64_t strides[1] = {inner * 2};
+    cuuint32_t box[2] = {(cuuint32_t)kBK, box_rows};
+    cuuint32_t es[2] = {1, 1};
+    return s->encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(ptr), dims, strides, box, es,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace mrp

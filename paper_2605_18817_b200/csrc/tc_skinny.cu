@@ -1,0 +1,573 @@
+// Tensor-core kernels for few activation rows (sm_100a): the weight rows sit on the MMA M axis
+// (128 TMEM lanes, one weight row per epilogue thread) and the activation rows on the N axis,
+// so a k-chunk of a stage is 16 KB of weights next to a few KB of activations and the ring of
+// TMA stages holds almost nothing but weight bytes in flight.  Same three GEMMs, same operand
+// buffers and same results as the row-major family (tc_kernels.cu):
+//   GU  gate/up + SwiGLU (a tile = 64 gate rows on lanes 0-63, their 64 up rows on 64-127)
+//   DN  down projection, h <- h + Delta, operands of the next GEMMs, partial sums of squares
+//   LM  shared LM head on the stacked rows h_k - h_0, "+ l_0", online softmax statistics kept
+//       per (thread, row-step) in registers and merged once per CTA                  (a2, a3)
+// Each activation operand is a bf16 hi block followed by a bf16 lo block; a stage holds both as
+// one B tile of N = 2 * RP rows, so one MMA per k-step yields the products with hi in columns
+// [0, RP) and with lo in [RP, 2 RP) of the accumulator; the epilogue adds the two.
+// Every CTA owns a contiguous range of 16-row weight units: full 128-row tiles, then one
+// shorter tile fetched through a tensor map with a smaller box, so no weight byte is read twice.
+// A kernel launched with programmatic stream serialisation starts fetching its weights while
+// the previous kernel drains: only the activation fetches and the epilogue wait for it.
+#include <string.h>
+
+#include "tc_common.cuh"
+
+namespace mrp {
+namespace {
+
+constexpr int kSkThreads = 192;
+constexpr int kWTile = 128 * 128;          // bytes of a 128-row weight tile of one k-chunk
+constexpr int kAuxBytes = 12288;           // epilogue scratch after the barriers
+constexpr int kAuxRstd = 0;                // float[32]
+constexpr int kAuxRowOff = 128;            // long long[32]
+constexpr int kAuxVote = 384;              // int: an epilogue warp gave up on a wait
+constexpr int kAuxSsq = 2560;              // float[4][32]
+constexpr int kAuxExch = 4096;             // float[32][64]
+
+enum { SK_GU = 0, SK_DN = 1, SK_LM = 2 };
+
+struct SkMaps {
+    CUtensorMap x;      // activation operand, box = r_pad rows
+    CUtensorMap w[6];   // [part * 3 + kind]: part 0 = gate / the matrix, 1 = up;
+                        // kind 0 = full tile, 1 / 2 = the two short-tile box heights
+};
+
+struct SkParams {
+    int units_total;     // weight rows / 16 (GU: gate rows / 8, a unit = 8 gate + 8 up rows)
+    int k_chunks;        // contraction extent / 64
+    int n_stages;
+    int r_pad;           // activation rows per part (16 or 32); MMA N = 2 * r_pad
+    int tmem_cols;       // allocated TMEM columns (power of two >= 2 buffers * 2 * r_pad)
+    int x_row_hi, x_row_lo;
+    int tail_units[2];   // units of short-tile kinds 1 and 2
+    int M, K, V, d, F, n_rs;
+    // LM
+    const float *logits0;
+    const int32_t *row_index;
+    Partial *partials;
+    float *logits_out;
+    // GU
+    const float *sumsq;
+    int n_ss;
+    float eps;
+    __nv_bfloat16 *act;
+    // DN
+    float *hcur;
+    const float *h0f;
+    const __nv_bfloat16 *gamma_next;
+    __nv_bfloat16 *xg_next;
+    __nv_bfloat16 *xt_k;
+    float *sumsq_out;
+    float *hidden_out;
+    int32_t *status;
+    int32_t *user_status;
+};
+
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void griddep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
+__device__ __forceinline__ void store_hi_lo(__nv_bfloat16 *dst, size_t lo_off, float v)
+{
+    const __nv_bfloat16 hi = __float2bfloat16_rn(v);
+    dst[0] = hi;
+    dst[lo_off] = __float2bfloat16_rn(v - __bfloat162float(hi));
+}
+
+template <int KIND, int RP, bool MARGIN>
+__global__ void __launch_bounds__(kSkThreads, 1)
+sk_gemm_kernel(const __grid_constant__ SkMaps maps, const SkParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    constexpr int x_bytes = 2 * RP * 128;            // hi rows then lo rows of one k-chunk
+    constexpr int stage_bytes = kWTile + x_bytes;
+    const uint32_t bars = base + (uint32_t)p.n_stages * stage_bytes;
+    auto full_bar = [&](int s) { return bars + 8u * s; };
+    auto empty_bar = [&](int s) { return bars + 8u * (p.n_stages + s); };
+    auto tfull_bar = [&](int a) { return bars + 8u * (2 * p.n_stages + a); };
+    auto tempty_bar = [&](int a) { return bars + 8u * (2 * p.n_stages + 2 + a); };
+    uint8_t *gen_base = smem_raw + (base - smem_u32(smem_raw));
+    uint8_t *after_bars = gen_base + (size_t)p.n_stages * stage_bytes + 8 * (2 * p.n_stages + 4);
+    uint32_t *tmem_holder = reinterpret_cast<uint32_t *>(after_bars);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_holder + 1);
+    uint8_t *aux = after_bars + 16;        // 16-byte aligned: stages and barrier block are multiples of 16
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int cta = blockIdx.x, G = gridDim.x;
+    const int u_base = p.units_total / G, u_extra = p.units_total % G;
+    const int units = u_base + (cta < u_extra ? 1 : 0);
+    const int u0 = cta * u_base + min(cta, u_extra);
+    const int n_full = units >> 3, rem = units & 7;
+    const int n_tiles = n_full + (rem ? 1 : 0);
+    const int tail_kind = (rem == p.tail_units[0]) ? 1 : 2;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < p.n_stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        prefetch_tmap(&maps.x);
+        prefetch_tmap(&maps.w[0]);
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(tmem_holder)), "r"((uint32_t)p.tmem_cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_holder;
+    griddep_launch();
+
+    if (warp == 0) {
+        // ---------------- TMA producer ----------------
+        if (lane == 0) {
+            const int total_it = n_tiles * p.k_chunks;
+            const int pre = min(p.n_stages, total_it);
+            auto load_w = [&](int t, int kk, int s) {
+                const uint32_t sw = base + (uint32_t)s * stage_bytes;
+                const bool is_full = t < n_full;
+                const int kind = is_full ? 0 : tail_kind;
+                const uint32_t w_bytes = is_full ? (uint32_t)kWTile : (uint32_t)rem * 2048u;
+                mbar_expect_tx(full_bar(s), w_bytes + (uint32_t)x_bytes);
+                const int ut = u0 + 8 * t;
+                if (KIND == SK_GU) {
+                    tma_load_2d(sw, &maps.w[kind], kk * kBK, ut * 8, full_bar(s));
+                    tma_load_2d(sw + 64 * 128, &maps.w[3 + kind], kk * kBK, ut * 8, full_bar(s));
+                } else {
+                    tma_load_2d(sw, &maps.w[kind], kk * kBK, ut * 16, full_bar(s));
+                }
+            };
+            auto load_x = [&](int kk, int s) {
+                const uint32_t sx = base + (uint32_t)s * stage_bytes + kWTile;
+                tma_load_2d(sx, &maps.x, kk * kBK, p.x_row_hi, full_bar(s));
+                tma_load_2d(sx + RP * 128, &maps.x, kk * kBK, p.x_row_lo, full_bar(s));
+            };
+            // weights do not depend on the previous kernel: fill the ring with them first
+            int t = 0, kk = 0;
+            for (int it = 0; it < pre; ++it) {
+                load_w(t, kk, it);
+                if (++kk == p.k_chunks) { kk = 0; ++t; }
+            }
+            griddep_wait();
+            for (int it = 0, k2 = 0; it < pre; ++it) {
+                load_x(k2, it);
+                if (++k2 == p.k_chunks) k2 = 0;
+            }
+            int s = 0;
+            uint32_t ph = 1;              // the ring has been filled once
+            for (int it = pre; it < total_it; ++it) {
+                if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p)) break;
+                load_w(t, kk, s);
+                load_x(kk, s);
+                if (++kk == p.k_chunks) { kk = 0; ++t; }
+                if (++s == p.n_stages) { s = 0; ph ^= 1u; }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
+        if (lane == 0) {
+            const uint32_t idesc = make_idesc(2 * RP);
+            int s = 0, acc = 0;
+            uint32_t ph = 0, acc_ph = 0;
+            bool ok = true;
+            for (int t = 0; t < n_tiles && ok; ++t) {
+                if (!mbar_wait(tempty_bar(acc), acc_ph ^ 1u, abort_flag, p)) break;
+                tc_fence_after();
+                const uint32_t dt = tmem_base + (uint32_t)(acc * 2 * RP);
+                for (int kk = 0; kk < p.k_chunks; ++kk) {
+                    if (!mbar_wait(full_bar(s), ph, abort_flag, p)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t sw = base + (uint32_t)s * stage_bytes;
+                    const uint64_t dw = make_smem_desc(sw);
+                    const uint64_t dx = make_smem_desc(sw + kWTile);
+#pragma unroll
+                    for (int k4 = 0; k4 < kBK / 16; ++k4)
+                        umma_bf16(dt, dw + 2u * k4, dx + 2u * k4, idesc, (kk > 0 || k4 > 0) ? 1u : 0u);
+                    umma_commit(empty_bar(s));
+                    if (++s == p.n_stages) { s = 0; ph ^= 1u; }
+                }
+                if (!ok) break;
+                umma_commit(tfull_bar(acc));
+                acc ^= 1;
+                if (acc == 0) acc_ph ^= 1u;
+            }
+        }
+    } else {
+        // ---------------- epilogue warps: thread t owns TMEM lane t = weight row t of the tile ----
+        const int q = warp & 3;
+        const int t = q * 32 + lane;
+        const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
+        float *rstd_s = reinterpret_cast<float *>(aux + kAuxRstd);
+        long long *rowoff_s = reinterpret_cast<long long *>(aux + kAuxRowOff);
+        float *ssq_s = reinterpret_cast<float *>(aux + kAuxSsq);
+        float *exch_s = reinterpret_cast<float *>(aux + kAuxExch);
+        volatile int *vote_s = reinterpret_cast<volatile int *>(aux + kAuxVote);
+
+        if (t == 0) *vote_s = 0;
+        griddep_wait();
+        if (KIND == SK_LM) {
+            if (t < p.n_rs) {
+                const int m = t % p.M;
+                rowoff_s[t] = (long long)(p.row_index ? p.row_index[m] : m) * p.V;
+            }
+        } else if (KIND == SK_GU) {
+            if (t < p.M) {
+                float s = 0.f;
+                for (int i = 0; i < p.n_ss; ++i) s += p.sumsq[(size_t)i * p.M + t];
+                rstd_s[t] = rsqrtf(s / (float)p.d + p.eps);
+            }
+        }
+        epi_sync();
+
+        // per-thread running state
+        float st_mx[KIND == SK_LM ? RP : 1], st_sum[KIND == SK_LM ? RP : 1], st_sec[KIND == SK_LM ? RP : 1];
+        int st_idx[KIND == SK_LM ? RP : 1];
+        float ssq[KIND == SK_DN ? RP : 1];
+        if (KIND == SK_LM) {
+#pragma unroll
+            for (int s = 0; s < RP; ++s) { st_mx[s] = -INFINITY; st_sum[s] = 0.f; st_sec[s] = -INFINITY; st_idx[s] = INT_MAX; }
+        }
+        if (KIND == SK_DN) {
+#pragma unroll
+            for (int s = 0; s < RP; ++s) ssq[s] = 0.f;
+        }
+
+        int acc = 0;
+        uint32_t acc_ph = 0;
+        bool ok = true;
+        for (int ti = 0; ti < n_tiles && ok; ++ti) {
+            const int ut = u0 + 8 * ti;
+            const int units_here = ti < n_full ? 8 : rem;
+            // What the tile's outputs are added to does not depend on the accumulator: fetch it
+            // (independent loads, all in flight together) before waiting for the MMAs.
+            float a[RP];
+            float h0v[KIND == SK_DN ? RP : 1];
+            const bool valid = KIND == SK_GU ? (t < 64 && t < units_here * 8) : (t < units_here * 16);
+            const int wrow = KIND == SK_GU ? ut * 8 + t : ut * 16 + t;     // weight row = output feature
+#pragma unroll
+            for (int j = 0; j < RP; ++j) {
+                a[j] = 0.f;
+                if (KIND == SK_LM) {
+                    if (valid && j < p.n_rs) a[j] = __ldg(p.logits0 + rowoff_s[j] + wrow);
+                } else if (KIND == SK_DN) {
+                    h0v[j] = 0.f;
+                    if (valid && j < p.M) {
+                        a[j] = p.hcur[(size_t)j * p.d + wrow];
+                        h0v[j] = __ldg(p.h0f + (size_t)j * p.d + wrow);
+                    }
+                }
+            }
+            const float gm = (KIND == SK_DN && valid && p.xg_next) ? __bfloat162float(p.gamma_next[wrow]) : 0.f;
+
+            ok = __all_sync(0xffffffffu, mbar_wait(tfull_bar(acc), acc_ph, abort_flag, p));
+            if (KIND == SK_GU) {
+                // the four warps meet at barriers below: they must leave the loop together
+                if (!ok && lane == 0) *vote_s = 1;
+                epi_sync();
+                ok = (*vote_s == 0);
+            }
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t tacc = lane_addr + (uint32_t)(acc * 2 * RP);
+#pragma unroll
+            for (int c0 = 0; c0 < 2 * RP; c0 += 16) {          // products with the hi rows, then the lo rows
+                float part[16];
+                tmem_ld16(tacc + c0, part);
+#pragma unroll
+                for (int j = 0; j < 16; ++j) a[(c0 + j) % RP] += part[j];
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tempty_bar(acc));
+            acc ^= 1;
+            if (acc == 0) acc_ph ^= 1u;
+
+            if (KIND == SK_LM) {
+                const int v = wrow;
+                if (valid) {
+#pragma unroll
+                    for (int s = 0; s < RP; ++s) {
+                        if (s < p.n_rs) {
+                            const float l = a[s];
+                            const float nm = fmaxf(st_mx[s], l);
+                            st_sum[s] = st_sum[s] * ex2f((st_mx[s] - nm) * kLog2e) + ex2f((l - nm) * kLog2e);
+                            if (l > st_mx[s]) {
+                                if (MARGIN) st_sec[s] = st_mx[s];
+                                st_idx[s] = v;
+                            } else if (MARGIN) {
+                                st_sec[s] = fmaxf(st_sec[s], l);
+                            }
+                            st_mx[s] = nm;
+                            if (p.logits_out && s >= p.M) p.logits_out[(size_t)(s - p.M) * p.V + v] = l;
+                        }
+                    }
+                }
+            } else if (KIND == SK_GU) {
+                // lanes 0-63 hold gate rows, 64-127 the matching up rows: hand the up values over
+                if (t >= 64) {
+#pragma unroll
+                    for (int m = 0; m < RP; ++m)
+                        if (m < p.M) exch_s[m * 64 + (t - 64)] = a[m] * rstd_s[m];
+                }
+                epi_sync();
+                if (valid) {
+#pragma unroll
+                    for (int m = 0; m < RP; ++m) {
+                        if (m < p.M) {
+                            const float g = a[m] * rstd_s[m];
+                            const float av = g / (1.f + __expf(-g)) * exch_s[m * 64 + t];
+                            store_hi_lo(p.act + (size_t)m * p.F + wrow, (size_t)p.M * p.F, av);
+                        }
+                    }
+                }
+                epi_sync();
+            } else {
+                if (valid) {
+#pragma unroll
+                    for (int m = 0; m < RP; ++m) {
+                        if (m < p.M) {
+                            const size_t o = (size_t)m * p.d + wrow;
+                            const float hc = a[m];
+                            p.hcur[o] = hc;
+                            if (p.hidden_out) p.hidden_out[o] = hc;
+                            ssq[m] = fmaf(hc, hc, ssq[m]);
+                            store_hi_lo(p.xt_k + o, (size_t)p.n_rs * p.d, hc - h0v[m]);
+                            if (p.xg_next) store_hi_lo(p.xg_next + o, (size_t)p.M * p.d, hc * gm);
+                        }
+                    }
+                }
+            }
+        }
+
+        // ---- per-CTA results ----
+        if (KIND == SK_LM) {
+            // Every thread parks its row-step statistics in the (now idle) ring memory; the merge
+            // over the 128 threads is then a short loop instead of unrolled straight-line code,
+            // which would be fetched once, instruction line by line, from a saturated memory system.
+            Partial *park = reinterpret_cast<Partial *>(gen_base);
+            if (!ok && lane == 0) *vote_s = 1;
+            epi_sync();
+            ok = (*vote_s == 0);          // on a failed wait copies may still be landing in the ring
+            if (ok) {
+#pragma unroll
+                for (int s = 0; s < RP; ++s) {
+                    if (s < p.n_rs) {
+                        Partial pr;
+                        pr.mx = st_mx[s]; pr.sum = st_sum[s]; pr.idx = st_idx[s]; pr.second = st_sec[s];
+                        park[s * 128 + t] = pr;
+                    }
+                }
+            }
+            epi_sync();
+            if (ok) {
+#pragma unroll 1
+                for (int s = q; s < p.n_rs; s += 4) {
+                    // fixed order: lane quadrants first, then the butterfly over lanes
+                    Partial pr = park[s * 128 + lane];
+#pragma unroll 1
+                    for (int w = 1; w < 4; ++w) pr = merge_partial(pr, park[s * 128 + w * 32 + lane]);
+#pragma unroll 1
+                    for (int o = 16; o > 0; o >>= 1) {
+                        Partial other;
+                        other.mx = __shfl_xor_sync(0xffffffffu, pr.mx, o);
+                        other.sum = __shfl_xor_sync(0xffffffffu, pr.sum, o);
+                        other.idx = __shfl_xor_sync(0xffffffffu, pr.idx, o);
+                        other.second = __shfl_xor_sync(0xffffffffu, pr.second, o);
+                        pr = (lane & o) ? merge_partial(other, pr) : merge_partial(pr, other);
+                    }
+                    if (lane == 0) p.partials[(size_t)cta * p.n_rs + s] = pr;
+                }
+            }
+        } else if (KIND == SK_DN) {
+#pragma unroll
+            for (int m = 0; m < RP; ++m) {
+                if (m < p.M) {
+                    float v = ssq[m];
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+                    if (lane == 0) ssq_s[q * 32 + m] = v;
+                }
+            }
+            epi_sync();
+            if (ok && t < p.M)
+                p.sumsq_out[(size_t)cta * p.M + t] = (ssq_s[t] + ssq_s[32 + t]) + (ssq_s[64 + t] + ssq_s[96 + t]);
+        }
+    }
+
+    // ---------------- teardown ----------------
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        // a wait gave up: give copies still in flight time to land before the CTA leaves
+        const long long t0 = clock64();
+        while (clock64() - t0 < 200000) __nanosleep(1000);
+        __syncthreads();
+    }
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)p.tmem_cols) : "memory");
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// Host side
+// ---------------------------------------------------------------------------------------
+size_t sk_smem_bytes(const SkParams &p)
+{
+    const int stage = kWTile + 2 * p.r_pad * 128;
+    return (size_t)p.n_stages * stage + 1024 + 8 * (2 * p.n_stages + 4) + 16 + kAuxBytes;
+}
+
+void sk_finish_shape(SkParams &p, int grid)
+{
+    // the ring always takes all the shared memory there is: it also parks the LM statistics
+    const int stage = kWTile + 2 * p.r_pad * 128;
+    int ns = (kSmemBudget - 1024 - 256 - 16 - kAuxBytes) / stage;
+    if (ns > 12) ns = 12;
+    p.n_stages = ns;
+    int cols = 32;
+    while (cols < 2 * 2 * p.r_pad) cols <<= 1;
+    p.tmem_cols = cols;
+    const int u_base = p.units_total / grid;
+    p.tail_units[0] = u_base % 8;
+    p.tail_units[1] = (u_base + 1) % 8;
+}
+
+// Tensor maps of one weight matrix part: full tiles and the two short-tile heights.
+bool sk_weight_maps(const TcState *s, SkMaps &maps, int part, const void *w, uint64_t inner, uint64_t rows,
+                    int unit_rows, const SkParams &p)
+{
+    if (!make_map(s, &maps.w[part * 3], w, inner, rows, 8 * unit_rows)) return false;
+    for (int k = 0; k < 2; ++k)
+        if (p.tail_units[k] > 0 &&
+            !make_map(s, &maps.w[part * 3 + 1 + k], w, inner, rows, p.tail_units[k] * unit_rows))
+            return false;
+    return true;
+}
+
+template <int KIND, int RP, bool MARGIN>
+cudaError_t sk_launch(const SkMaps &maps, const SkParams &p, int grid, cudaStream_t st, bool pdl)
+{
+    auto kern = sk_gemm_kernel<KIND, RP, MARGIN>;
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kSkThreads);
+    cfg.dynamicSmemBytes = sk_smem_bytes(p);
+    cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kern, maps, p);
+}
+
+template <int KIND>
+cudaError_t sk_launch_rp(const SkMaps &maps, const SkParams &p, int grid, cudaStream_t st, bool pdl, bool margin)
+{
+    if constexpr (KIND != SK_LM) {
+        return p.r_pad == 16 ? sk_launch<KIND, 16, false>(maps, p, grid, st, pdl)
+                             : sk_launch<KIND, 32, false>(maps, p, grid, st, pdl);
+    } else {
+        if (p.r_pad == 16)
+            return margin ? sk_launch<KIND, 16, true>(maps, p, grid, st, pdl) : sk_launch<KIND, 16, false>(maps, p, grid, st, pdl);
+        return margin ? sk_launch<KIND, 32, true>(maps, p, grid, st, pdl) : sk_launch<KIND, 32, false>(maps, p, grid, st, pdl);
+    }
+}
+
+void sk_common(Ctx *c, SkParams &p, int M, int K, const mrp_draft_out &out)
+{
+    memset(&p, 0, sizeof(p));
+    p.M = M; p.K = K; p.V = c->cfg.vocab; p.d = c->cfg.d; p.F = c->cfg.d_ff; p.n_rs = (K + 1) * M;
+    p.status = (int32_t *)(c->ws + c->lay.status);
+    p.user_status = out.status;
+}
+
+}  // namespace
+
+bool sk_rows_ok(int rows) { return rows >= 1 && rows <= 32; }
+
+cudaError_t sk_gateup(Ctx *c, int k, int M, int K, int n_ss, const mrp_draft_out &out, cudaStream_t st, bool pdl)
+{
+    const TcState *s = (const TcState *)c->tc_state;
+    const mrp_head_weights &hw = c->heads[k - 1];
+    const int d = c->cfg.d, F = c->cfg.d_ff, G = c->sm_count;
+    SkParams p;
+    sk_common(c, p, M, K, out);
+    p.units_total = F / 8; p.k_chunks = d / kBK; p.r_pad = M <= 16 ? 16 : 32;
+    p.x_row_hi = 0; p.x_row_lo = M;
+    p.sumsq = (const float *)(c->ws + c->lay.sumsq); p.n_ss = n_ss; p.eps = c->cfg.rms_eps;
+    p.act = (__nv_bfloat16 *)(c->ws + c->lay.act);
+    sk_finish_shape(p, G);
+    SkMaps maps;
+    memset(&maps, 0, sizeof(maps));
+    if (!make_map(s, &maps.x, c->ws + c->lay.xg, d, 2 * (uint64_t)M, p.r_pad) ||
+        !sk_weight_maps(s, maps, 0, hw.w_gate, d, F, 8, p) || !sk_weight_maps(s, maps, 1, hw.w_up, d, F, 8, p))
+        return note_err(c, cudaErrorInvalidValue, "tensor map (gate/up, few rows)");
+    c->launches++;
+    return note_err(c, sk_launch_rp<SK_GU>(maps, p, G, st, pdl, false), "gate/up kernel (few rows)");
+}
+
+cudaError_t sk_down(Ctx *c, int k, int M, int K, const mrp_draft_out &out, cudaStream_t st, bool pdl)
+{
+    const TcState *s = (const TcState *)c->tc_state;
+    const mrp_head_weights &hw = c->heads[k - 1];
+    const int d = c->cfg.d, F = c->cfg.d_ff, G = c->sm_count;
+    SkParams p;
+    sk_common(c, p, M, K, out);
+    p.units_total = d / 16; p.k_chunks = F / kBK; p.r_pad = M <= 16 ? 16 : 32;
+    p.x_row_hi = 0; p.x_row_lo = M;
+    p.hcur = (float *)(c->ws + c->lay.hcur); p.h0f = (const float *)(c->ws + c->lay.h0f);
+    p.gamma_next = (k < K) ? (const __nv_bfloat16 *)c->heads[k].rms_gamma : nullptr;
+    p.xg_next = (k < K) ? (__nv_bfloat16 *)(c->ws + c->lay.xg) : nullptr;
+    p.xt_k = (__nv_bfloat16 *)(c->ws + c->lay.xt) + (size_t)k * M * d;
+    p.sumsq_out = (float *)(c->ws + c->lay.sumsq);
+    p.hidden_out = (k == K) ? out.hidden_out : nullptr;
+    sk_finish_shape(p, G);
+    SkMaps maps;
+    memset(&maps, 0, sizeof(maps));
+    if (!make_map(s, &maps.x, c->ws + c->lay.act, F, 2 * (uint64_t)M, p.r_pad) ||
+        !sk_weight_maps(s, maps, 0, hw.w_down, F, d, 16, p))
+        return note_err(c, cudaErrorInvalidValue, "tensor map (down, few rows)");
+    c->launches++;
+    return note_err(c, sk_launch_rp<SK_DN>(maps, p, G, st, pdl, false), "down kernel (few rows)");
+}
+
+cudaError_t sk_lm(Ctx *c, const float *logits0, const int32_t *row_index, int M, int K,
+                  const mrp_draft_out &out, cudaStream_t st, bool pdl)
+{
+    const TcState *s = (const TcState *)c->tc_state;
+    const int d = c->cfg.d, V = c->cfg.vocab, G = c->sm_count;
+    SkParams p;
+    sk_common(c, p, M, K, out);
+    p.units_total = V / 16; p.k_chunks = d / kBK; p.r_pad = p.n_rs <= 16 ? 16 : 32;
+    p.x_row_hi = 0; p.x_row_lo = p.n_rs;
+    p.logits0 = logits0; p.row_index = row_index;
+    p.partials = (Partial *)(c->ws + c->lay.partials); p.logits_out = out.logits_out;
+    sk_finish_shape(p, G);
+    SkMaps maps;
+    memset(&maps, 0, sizeof(maps));
+    if (!make_map(s, &maps.x, c->ws + c->lay.xt, d, 2 * (uint64_t)p.n_rs, p.r_pad) ||
+        !sk_weight_maps(s, maps, 0, c->w_lm, d, V, 16, p))
+        return note_err(c, cudaErrorInvalidValue, "tensor map (LM head, few rows)");
+    c->launches++;
+    return note_err(c, sk_launch_rp<SK_LM>(maps, p, G, st, pdl, out.margin != nullptr), "LM-head kernel (few rows)");
+}
+
+}  // namespace mrp

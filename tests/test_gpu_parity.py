@@ -240,9 +240,14 @@ def test_config0_static_selection_end_to_end():
     (64, 64, 1024, 128, 1, 1),      # exactly one full row block
     (256, 512, 4096, 75, 4, 4),     # 300 rows, four accumulators
     (64, 128, 160, 3, 1, 1),        # fewer vocabulary units than CTAs
+    (128, 256, 2048, 16, 1, 1),     # few-row kernels at their 32-row-step limit
+    (128, 256, 2048, 32, 1, 2),     # few-row head kernels at 32 rows, row-major LM head
+    (64, 12288, 2304, 5, 1, 2),     # gate/up: full 128-row weight tiles plus short tiles
+    (19008, 64, 512, 3, 1, 1),      # down projection: full weight tiles plus short tiles
 ])
 def test_tensor_core_family_small_shapes(d, F, V, B, L, K):
-    w = synth.make_weights(d, F, V, K, "bf16", 77, head_std=0.05)
+    # residuals of order one at every shape (the very long contraction gets smaller weights)
+    w = synth.make_weights(d, F, V, K, "bf16", 77, head_std=0.05 if d < 4096 else 0.03)
     for k, h in enumerate(w.heads):
         h["gamma"] = synth.bf16_round((1.0 + 0.25 * np.cos(np.arange(d) + k)).astype(np.float32))
     inp = synth.make_inputs(w, B, L, 77, 1.0, 4.0)
@@ -263,3 +268,6 @@ def test_tensor_core_family_small_shapes(d, F, V, B, L, K):
     out3, _ = run_gpu_draft(w, inp, max(K - 1, 1), row_index=sub)
     ref3 = oracle.draft(inp.hidden, inp.logits0, w.heads, w.w_lm, K=max(K - 1, 1), row_index=sub)
     check_stats(out3, ref3, "bf16")
+    # the row-major kernels alone, fully serialised launches: same results within tolerance
+    out4, _ = run_gpu_draft(w, inp, K, flags=binding.MRP_FLAG_ROW_MAJOR_ONLY | binding.MRP_FLAG_NO_PDL)
+    check_stats(out4, ref, "bf16")
