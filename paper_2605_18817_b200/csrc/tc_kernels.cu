@@ -38,13 +38,15 @@ struct TcParams {
     int n_boxes;         // TMA boxes per B tile (GU 2, else 1)
     int k_chunks;        // contraction extent / 64
     int n_stages;
-    int n_mb;            // 128-row activation blocks
-    int a_row_base;      // A row coordinate of accumulator 0, block 0 (hi part)
-    int a_row_step;      // A row offset between accumulators
+    // decomposition of the work over CTAs: CTA = (weight-row range, group of row blocks)
+    int n_vr;            // weight-row ranges
+    int n_groups;        // row-block groups; group g owns blocks g, g + n_groups, ...
+    int n_rb;            // 128-row activation blocks
+    int rows;            // valid activation rows (GU/DN: M; LM: K*M row-steps of steps 1..K)
+    int a_row_base;      // A row coordinate of row 0 (hi part)
     int a_part_rows;     // A row offset from the hi part to the lo part
     int M, K, V, d, F;
-    int stacked;         // LM: all (K+1)*M row-steps in one block
-    int n_rs;            // LM: (K+1)*M
+    int n_rs;            // (K+1)*M
     // LM
     const float *logits0;
     const int32_t *row_index;
@@ -70,21 +72,16 @@ struct TcParams {
 // ---------------------------------------------------------------------------------------
 // The kernel
 // ---------------------------------------------------------------------------------------
-template <int KIND, int NACC, bool MARGIN>
+template <int KIND, bool MARGIN>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
                const __grid_constant__ CUtensorMap tmB1, const TcParams p)
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    // With one accumulator a stage holds the hi and the lo A tile and one B tile; with several
-    // accumulators a stage holds one A tile per accumulator and the k-loop alternates hi / lo
-    // (the B chunk is then fetched twice in a row, the second time from L2).
-    constexpr bool SIS = (NACC == 1);
-    constexpr int NA = SIS ? 2 : NACC;
-    const int n_it = SIS ? p.k_chunks : 2 * p.k_chunks;
+    // a stage holds the hi and the lo A tile of a k-chunk and one B tile
     const int b_bytes = (p.bn * 128 + 1023) & ~1023;
-    const int stage_bytes = NA * kATile + b_bytes;
+    const int stage_bytes = 2 * kATile + b_bytes;
     const uint32_t bars = base + (uint32_t)p.n_stages * stage_bytes;   // 8-byte aligned
     // barrier slots: full[s], empty[s], tmem_full[2], tmem_empty[2]
     auto full_bar = [&](int s) { return bars + 8u * s; };
@@ -96,9 +93,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_holder + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int cta = blockIdx.x, G = gridDim.x;
-    const int u0 = (int)((long long)cta * p.units_total / G);
-    const int u1 = (int)((long long)(cta + 1) * p.units_total / G);
+    const int cta = blockIdx.x;
+    const int vr = cta % p.n_vr, grp = cta / p.n_vr;
+    const int u0 = (int)((long long)vr * p.units_total / p.n_vr);
+    const int u1 = (int)((long long)(vr + 1) * p.units_total / p.n_vr);
     const int n_t = (u1 - u0 + p.w_units - 1) / p.w_units;
 
     if (threadIdx.x == 0) {
@@ -123,31 +121,21 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     if (warp == 0) {
         // ---------------- TMA producer ----------------
         if (lane == 0) {
-            const uint32_t tx = (uint32_t)(NA * kATile + p.bn * 128);
+            const uint32_t tx = (uint32_t)(2 * kATile + p.bn * 128);
             const int box_rows = p.bn / p.n_boxes;
             int s = 0;
             uint32_t ph = 0;
             bool ok = true;
-            for (int mb = 0; mb < p.n_mb && ok; ++mb) {
+            for (int mb = grp; mb < p.n_rb && ok; mb += p.n_groups) {
                 for (int t = 0; t < n_t && ok; ++t) {
                     const int n0 = (u0 + t * p.w_units) * p.unit_rows;
-                    for (int it = 0; it < n_it; ++it) {
-                        const int kk = SIS ? it : (it >> 1);
+                    for (int kk = 0; kk < p.k_chunks; ++kk) {
                         if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p)) { ok = false; break; }
                         mbar_expect_tx(full_bar(s), tx);
                         const uint32_t sa = base + (uint32_t)s * stage_bytes;
-                        if (SIS) {
-                            tma_load_2d(sa, &tmA, kk * kBK, p.a_row_base + mb * 128, full_bar(s));
-                            tma_load_2d(sa + kATile, &tmA, kk * kBK, p.a_part_rows + p.a_row_base + mb * 128,
-                                        full_bar(s));
-                        } else {
-                            const int part_row = (it & 1) * p.a_part_rows;
-#pragma unroll
-                            for (int a = 0; a < NACC; ++a)
-                                tma_load_2d(sa + a * kATile, &tmA, kk * kBK,
-                                            part_row + p.a_row_base + a * p.a_row_step + mb * 128, full_bar(s));
-                        }
-                        const uint32_t sb = sa + NA * kATile;
+                        tma_load_2d(sa, &tmA, kk * kBK, p.a_row_base + mb * 128, full_bar(s));
+                        tma_load_2d(sa + kATile, &tmA, kk * kBK, p.a_part_rows + p.a_row_base + mb * 128, full_bar(s));
+                        const uint32_t sb = sa + 2 * kATile;
                         tma_load_2d(sb, &tmB0, kk * kBK, n0, full_bar(s));
                         if (KIND == KIND_GU)
                             tma_load_2d(sb + box_rows * 128, &tmB1, kk * kBK, n0, full_bar(s));
@@ -163,23 +151,22 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             int s = 0, acc = 0;
             uint32_t ph = 0, acc_ph = 0;
             bool ok = true;
-            for (int mb = 0; mb < p.n_mb && ok; ++mb) {
+            for (int mb = grp; mb < p.n_rb && ok; mb += p.n_groups) {
                 for (int t = 0; t < n_t && ok; ++t) {
                     if (!mbar_wait(tempty_bar(acc), acc_ph ^ 1u, abort_flag, p)) { ok = false; break; }
                     tc_fence_after();
-                    for (int it = 0; it < n_it; ++it) {
+                    const uint32_t dt = tmem_base + (uint32_t)(acc * kAccCols);
+                    for (int kk = 0; kk < p.k_chunks; ++kk) {
                         if (!mbar_wait(full_bar(s), ph, abort_flag, p)) { ok = false; break; }
                         tc_fence_after();
                         const uint32_t sa = base + (uint32_t)s * stage_bytes;
-                        const uint64_t db = make_smem_desc(sa + NA * kATile);
+                        const uint64_t db = make_smem_desc(sa + 2 * kATile);
 #pragma unroll
-                        for (int a = 0; a < NA; ++a) {
+                        for (int a = 0; a < 2; ++a) {
                             const uint64_t da = make_smem_desc(sa + a * kATile);
-                            const uint32_t dt = tmem_base + (uint32_t)(acc * kAccCols + (SIS ? 0 : a * p.bn));
 #pragma unroll
                             for (int k4 = 0; k4 < kBK / 16; ++k4)
-                                umma_bf16(dt, da + 2u * k4, db + 2u * k4, idesc,
-                                          (it > 0 || k4 > 0 || (SIS && a > 0)) ? 1u : 0u);
+                                umma_bf16(dt, da + 2u * k4, db + 2u * k4, idesc, (kk > 0 || k4 > 0 || a > 0) ? 1u : 0u);
                         }
                         umma_commit(empty_bar(s));
                         if (++s == p.n_stages) { s = 0; ph ^= 1u; }
@@ -194,41 +181,34 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     } else {
         // ---------------- epilogue warps (TMEM lane quadrant = warp % 4) ----------------
         const int q = warp & 3;
-        const int r = q * 32 + lane;
+        const int rl = q * 32 + lane;
         const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
         int acc = 0;
         uint32_t acc_ph = 0;
         bool ok = true;
-        for (int mb = 0; mb < p.n_mb && ok; ++mb) {
-            // ---- per-block state ----
-            const int m_or_rs = mb * 128 + r;
-            RowStat st[KIND == KIND_LM ? NACC + 1 : 1];
-            bool valid = false;
+        for (int mb = grp; mb < p.n_rb && ok; mb += p.n_groups) {
+            // ---- per-block state: this thread's activation row ----
+            const int r = mb * 128 + rl;
+            const bool valid = r < p.rows;
+            RowStat st, st0;       // LM: statistics of the row's own step, and of step 0 (rows of step 1 only)
+            bool first_step = false;
             const float *l0p = nullptr;
-            int k_of_row = 0, m_of_row = 0;
+            int k_of_row = 0, m_of_row = r;
             float rstd = 0.f, ssq = 0.f;
             if (KIND == KIND_LM) {
-#pragma unroll
-                for (int i = 0; i < NACC + 1; ++i) st[i].init();
-                if (p.stacked) {
-                    valid = m_or_rs < p.n_rs;
-                    if (valid) { k_of_row = m_or_rs / p.M; m_of_row = m_or_rs - k_of_row * p.M; }
-                } else {
-                    valid = m_or_rs < p.M;
-                    m_of_row = m_or_rs;
-                }
+                st.init();
+                st0.init();
                 if (valid) {
+                    k_of_row = r / p.M + 1;
+                    m_of_row = r - (k_of_row - 1) * p.M;
+                    first_step = (k_of_row == 1);
                     const size_t row = p.row_index ? (size_t)p.row_index[m_of_row] : (size_t)m_of_row;
                     l0p = p.logits0 + row * (size_t)p.V;
                 }
-            } else {
-                valid = m_or_rs < p.M;
-                m_of_row = m_or_rs;
-                if (KIND == KIND_GU && valid) {
-                    float s = 0.f;
-                    for (int i = 0; i < p.n_ss; ++i) s += p.sumsq[(size_t)i * p.M + m_of_row];
-                    rstd = rsqrtf(s / (float)p.d + p.eps);
-                }
+            } else if (KIND == KIND_GU && valid) {
+                float s = 0.f;
+                for (int i = 0; i < p.n_ss; ++i) s += p.sumsq[(size_t)i * p.M + m_of_row];
+                rstd = rsqrtf(s / (float)p.d + p.eps);
             }
             for (int t = 0; t < n_t && ok; ++t) {
                 ok = __all_sync(0xffffffffu, mbar_wait(tfull_bar(acc), acc_ph, abort_flag, p));
@@ -241,30 +221,15 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     const int v_tile = ut * 16;
                     for (int c = 0; c < units_here; ++c) {
                         const int v = v_tile + c * 16;
-                        float l0[16], a[16], l[16];
+                        float l0[16], a[16];
                         if (valid) load16(l0p + v, l0);
-                        if (p.stacked) {
-                            tmem_ld16(tacc + c * 16, a);
-                            if (valid) {
+                        tmem_ld16(tacc + c * 16, a);
+                        if (valid) {
+                            if (first_step) st0.template update<MARGIN>(l0, v);
 #pragma unroll
-                                for (int j = 0; j < 16; ++j) l[j] = (k_of_row > 0) ? l0[j] + a[j] : l0[j];
-                                st[0].template update<MARGIN>(l, v);
-                                if (p.logits_out && k_of_row > 0)
-                                    store16(p.logits_out + ((size_t)(m_or_rs - p.M)) * p.V + v, l);
-                            }
-                        } else {
-                            if (valid) st[0].template update<MARGIN>(l0, v);
-#pragma unroll
-                            for (int s = 0; s < NACC; ++s) {
-                                tmem_ld16(tacc + s * p.bn + c * 16, a);
-                                if (valid) {
-#pragma unroll
-                                    for (int j = 0; j < 16; ++j) l[j] = l0[j] + a[j];
-                                    st[s + 1].template update<MARGIN>(l, v);
-                                    if (p.logits_out)
-                                        store16(p.logits_out + ((size_t)s * p.M + m_of_row) * p.V + v, l);
-                                }
-                            }
+                            for (int j = 0; j < 16; ++j) a[j] += l0[j];
+                            st.template update<MARGIN>(a, v);
+                            if (p.logits_out) store16(p.logits_out + (size_t)r * p.V + v, a);
                         }
                     }
                 } else if (KIND == KIND_GU) {
@@ -319,15 +284,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             // ---- per-block results ----
             if (ok && valid) {
                 if (KIND == KIND_LM) {
-                    if (p.stacked) {
-                        p.partials[(size_t)cta * p.n_rs + m_or_rs] = st[0].partial();
-                    } else {
-#pragma unroll
-                        for (int s = 0; s < NACC + 1; ++s)
-                            p.partials[(size_t)cta * p.n_rs + (size_t)s * p.M + m_of_row] = st[s].partial();
-                    }
+                    p.partials[(size_t)vr * p.n_rs + (size_t)k_of_row * p.M + m_of_row] = st.partial();
+                    if (first_step) p.partials[(size_t)vr * p.n_rs + m_of_row] = st0.partial();
                 } else if (KIND == KIND_DN) {
-                    p.sumsq_out[(size_t)cta * p.M + m_of_row] = ssq;
+                    p.sumsq_out[(size_t)vr * p.M + m_of_row] = ssq;
                 }
             }
         }
@@ -388,23 +348,20 @@ __global__ void tc_prep_kernel(const __nv_bfloat16 *__restrict__ hidden, const i
 // ---------------------------------------------------------------------------------------
 // Host side
 // ---------------------------------------------------------------------------------------
-// Tile width (in units, at most w_max) for CTAs owning up to `maxunits` units: the width that
-// wastes the fewest rows beyond the range, the wider one on ties.
+// Tile width (in units, at most w_max) for CTAs owning up to `maxunits` units.  An MMA costs
+// about the same whatever its N, so the tile count is kept minimal first; among the widths that
+// reach it the narrowest wastes the fewest rows beyond the range.
 int choose_tile_units(int maxunits, int w_max)
 {
-    int best_w = 1, best_waste = INT_MAX;
-    for (int w = 1; w <= w_max; ++w) {
-        const int T = (maxunits + w - 1) / w;
-        const int waste = T * w - maxunits;
-        if (waste <= best_waste) { best_waste = waste; best_w = w; }
-    }
-    return best_w;
+    const int t_min = (maxunits + w_max - 1) / w_max;
+    return (maxunits + t_min - 1) / t_min;
 }
 
-void finish_shape(TcParams &p, int nacc, int grid)
+void finish_shape(TcParams &p, int n_vr)
 {
-    const int maxunits = (p.units_total + grid - 1) / grid;
-    const int bn_max = kAccCols / nacc;
+    p.n_vr = n_vr;
+    const int maxunits = (p.units_total + n_vr - 1) / n_vr;
+    const int bn_max = kAccCols;
     const int rows_per_unit = p.unit_rows * p.n_boxes;
     int w_max = bn_max / rows_per_unit;
     if (w_max > 256 / rows_per_unit) w_max = 256 / rows_per_unit;
@@ -412,24 +369,24 @@ void finish_shape(TcParams &p, int nacc, int grid)
     p.w_units = choose_tile_units(maxunits < 1 ? 1 : maxunits, w_max);
     p.bn = p.w_units * rows_per_unit;
     const int b_bytes = (p.bn * 128 + 1023) & ~1023;
-    const int stage = (nacc == 1 ? 2 : nacc) * kATile + b_bytes;
+    const int stage = 2 * kATile + b_bytes;
     int ns = (kSmemBudget - 1024 - 512) / stage;
     if (ns > 12) ns = 12;
     p.n_stages = ns;
 }
 
-size_t smem_bytes(const TcParams &p, int nacc)
+size_t smem_bytes(const TcParams &p)
 {
     const int b_bytes = (p.bn * 128 + 1023) & ~1023;
-    return (size_t)p.n_stages * ((nacc == 1 ? 2 : nacc) * kATile + b_bytes) + 1024 + 8 * (2 * p.n_stages + 4) + 16;
+    return (size_t)p.n_stages * (2 * kATile + b_bytes) + 1024 + 8 * (2 * p.n_stages + 4) + 16;
 }
 
-template <int KIND, int NACC, bool MARGIN>
+template <int KIND, bool MARGIN>
 cudaError_t launch_tc(const CUtensorMap &a, const CUtensorMap &b0, const CUtensorMap &b1, const TcParams &p,
                       int grid, cudaStream_t st)
 {
-    auto kern = tc_gemm_kernel<KIND, NACC, MARGIN>;
-    const size_t smem = smem_bytes(p, NACC);
+    auto kern = tc_gemm_kernel<KIND, MARGIN>;
+    const size_t smem = smem_bytes(p);
     static bool attr_set = false;
     if (!attr_set) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
@@ -438,18 +395,6 @@ cudaError_t launch_tc(const CUtensorMap &a, const CUtensorMap &b0, const CUtenso
     }
     kern<<<grid, kThreads, smem, st>>>(a, b0, b1, p);
     return cudaGetLastError();
-}
-
-template <bool MARGIN>
-cudaError_t launch_lm(int nacc, const CUtensorMap &a, const CUtensorMap &b, const TcParams &p, int grid, cudaStream_t st)
-{
-    switch (nacc) {
-    case 1: return launch_tc<KIND_LM, 1, MARGIN>(a, b, b, p, grid, st);
-    case 2: return launch_tc<KIND_LM, 2, MARGIN>(a, b, b, p, grid, st);
-    case 3: return launch_tc<KIND_LM, 3, MARGIN>(a, b, b, p, grid, st);
-    case 4: return launch_tc<KIND_LM, 4, MARGIN>(a, b, b, p, grid, st);
-    default: return cudaErrorInvalidValue;
-    }
 }
 
 }  // namespace
@@ -532,21 +477,22 @@ cudaError_t tc_draft(Ctx *c, const void *hidden, const float *logits0, const int
         // gate/up + SwiGLU
         TcParams p;
         memset(&p, 0, sizeof(p));
-        p.units_total = F / 8; p.unit_rows = 8; p.n_boxes = 2; p.k_chunks = d / kBK; p.n_mb = n_mb;
-        p.a_row_base = 0; p.a_row_step = 0; p.a_part_rows = M;
+        p.units_total = F / 8; p.unit_rows = 8; p.n_boxes = 2; p.k_chunks = d / kBK;
+        p.n_groups = 1; p.n_rb = n_mb; p.rows = M; p.a_row_base = 0; p.a_part_rows = M;
         p.M = M; p.K = K; p.V = V; p.d = d; p.F = F; p.n_rs = n_rs;
         p.sumsq = sumsq; p.n_ss = n_ss; p.eps = c->cfg.rms_eps; p.act = act;
         p.status = status; p.user_status = out.status;
-        finish_shape(p, 1, G);
+        finish_shape(p, G);
         if (!make_map(s, &mA, xg, d, 2 * (uint64_t)M, 128) || !make_map(s, &mB0, hw.w_gate, d, F, p.bn / 2) ||
             !make_map(s, &mB1, hw.w_up, d, F, p.bn / 2))
             return note_err(c, cudaErrorInvalidValue, "tensor map (gate/up)");
-        e = note_err(c, launch_tc<KIND_GU, 1, false>(mA, mB0, mB1, p, G, st), "gate/up kernel");
+        e = note_err(c, launch_tc<KIND_GU, false>(mA, mB0, mB1, p, G, st), "gate/up kernel");
         c->launches++;
         if (e != cudaSuccess) return e;
         // down projection, residual add, next operands
         memset(&p, 0, sizeof(p));
-        p.units_total = d / 16; p.unit_rows = 16; p.n_boxes = 1; p.k_chunks = F / kBK; p.n_mb = n_mb;
+        p.units_total = d / 16; p.unit_rows = 16; p.n_boxes = 1; p.k_chunks = F / kBK;
+        p.n_groups = 1; p.n_rb = n_mb; p.rows = M;
         p.M = M; p.K = K; p.V = V; p.d = d; p.F = F; p.n_rs = n_rs; p.a_part_rows = M;
         p.hcur = hcur; p.h0f = h0f;
         p.gamma_next = (k < K) ? (const __nv_bfloat16 *)c->heads[k].rms_gamma : nullptr;
@@ -555,15 +501,16 @@ cudaError_t tc_draft(Ctx *c, const void *hidden, const float *logits0, const int
         p.sumsq_out = sumsq;
         p.hidden_out = (k == K) ? out.hidden_out : nullptr;
         p.status = status; p.user_status = out.status;
-        finish_shape(p, 1, G);
+        finish_shape(p, G);
         if (!make_map(s, &mA, act, F, 2 * (uint64_t)M, 128) || !make_map(s, &mB0, hw.w_down, F, d, p.bn))
             return note_err(c, cudaErrorInvalidValue, "tensor map (down)");
-        e = note_err(c, launch_tc<KIND_DN, 1, false>(mA, mB0, mB0, p, G, st), "down kernel");
+        e = note_err(c, launch_tc<KIND_DN, false>(mA, mB0, mB0, p, G, st), "down kernel");
         c->launches++;
         if (e != cudaSuccess) return e;
         n_ss = G;
     }
     prof_mark(c, 1, st);
+    int n_slices = G;
     if (sk_rows_ok(n_rs) && !(c->cfg.flags & MRP_FLAG_ROW_MAJOR_ONLY)) {
         e = sk_lm(c, logits0, row_index, M, K, out, st, pdl);
         if (e != cudaSuccess) return e;
@@ -571,24 +518,37 @@ cudaError_t tc_draft(Ctx *c, const void *hidden, const float *logits0, const int
         CUtensorMap mA, mB;
         TcParams p;
         memset(&p, 0, sizeof(p));
-        const bool stacked = n_rs <= 128;
-        const int nacc = stacked ? 1 : K;
-        p.units_total = V / 16; p.unit_rows = 16; p.n_boxes = 1; p.k_chunks = d / kBK;
-        p.n_mb = stacked ? 1 : n_mb;
-        p.a_row_base = stacked ? 0 : M; p.a_row_step = stacked ? 0 : M; p.a_part_rows = n_rs;
-        p.M = M; p.K = K; p.V = V; p.d = d; p.F = F; p.stacked = stacked ? 1 : 0; p.n_rs = n_rs;
+        // Row-steps of steps 1..K in 128-row blocks; CTA = (vocabulary range, group of row blocks).
+        // Pick the split with the shortest longest CTA (in tiles), the fewest passes on ties.
+        const int rows = K * M, n_rb = (rows + 127) / 128, U = V / 16;
+        int best_g = 1;
+        long long best_cost = -1;
+        for (int g = 1; g <= n_rb && g <= G; ++g) {
+            const int nv = G / g;
+            const int passes = (n_rb + g - 1) / g;
+            const int units = (U + nv - 1) / nv;
+            const long long cost = (long long)passes * ((units + 15) / 16);
+            if (best_cost < 0 || cost <= best_cost) { best_cost = cost; best_g = g; }
+        }
+        p.n_groups = best_g;
+        n_slices = G / best_g;
+        p.n_rb = n_rb; p.rows = rows;
+        p.units_total = U; p.unit_rows = 16; p.n_boxes = 1; p.k_chunks = d / kBK;
+        p.a_row_base = M; p.a_part_rows = n_rs;
+        p.M = M; p.K = K; p.V = V; p.d = d; p.F = F; p.n_rs = n_rs;
         p.logits0 = logits0; p.row_index = row_index; p.partials = partials; p.logits_out = out.logits_out;
         p.status = status; p.user_status = out.status;
-        finish_shape(p, nacc, G);
+        finish_shape(p, n_slices);
         if (!make_map(s, &mA, xt, d, 2 * (uint64_t)n_rs, 128) || !make_map(s, &mB, c->w_lm, d, V, p.bn))
             return note_err(c, cudaErrorInvalidValue, "tensor map (LM head)");
-        e = note_err(c, out.margin ? launch_lm<true>(nacc, mA, mB, p, G, st)
-                                   : launch_lm<false>(nacc, mA, mB, p, G, st), "LM-head kernel");
+        const int grid = p.n_groups * p.n_vr;
+        e = note_err(c, out.margin ? launch_tc<KIND_LM, true>(mA, mB, mB, p, grid, st)
+                                   : launch_tc<KIND_LM, false>(mA, mB, mB, p, grid, st), "LM-head kernel");
         c->launches++;
         if (e != cudaSuccess) return e;
     }
     prof_mark(c, 2, st);
-    e = launch_combine(c, partials, G, (K + 1) * M, out, status, st);
+    e = launch_combine(c, partials, n_slices, (K + 1) * M, out, status, st);
     prof_mark(c, 3, st);
     return e;
 }
