@@ -357,6 +357,22 @@ int choose_tile_units(int maxunits, int w_max)
     return (maxunits + t_min - 1) / t_min;
 }
 
+// Split of the work over `G` CTAs: n_groups row-block groups times G / n_groups weight-row
+// ranges, chosen for the shortest longest CTA (in 16-unit tiles), the fewest passes on ties.
+int choose_groups(int n_rb, int units_total, int G)
+{
+    int best_g = 1;
+    long long best_cost = -1;
+    for (int g = 1; g <= n_rb && g <= G; ++g) {
+        const int nv = G / g;
+        const int passes = (n_rb + g - 1) / g;
+        const int units = (units_total + nv - 1) / nv;
+        const long long cost = (long long)passes * ((units + 15) / 16);
+        if (best_cost < 0 || cost <= best_cost) { best_cost = cost; best_g = g; }
+    }
+    return best_g;
+}
+
 void finish_shape(TcParams &p, int n_vr)
 {
     p.n_vr = n_vr;
@@ -478,21 +494,21 @@ cudaError_t tc_draft(Ctx *c, const void *hidden, const float *logits0, const int
         TcParams p;
         memset(&p, 0, sizeof(p));
         p.units_total = F / 8; p.unit_rows = 8; p.n_boxes = 2; p.k_chunks = d / kBK;
-        p.n_groups = 1; p.n_rb = n_mb; p.rows = M; p.a_row_base = 0; p.a_part_rows = M;
+        p.n_groups = choose_groups(n_mb, p.units_total, G); p.n_rb = n_mb; p.rows = M; p.a_row_base = 0; p.a_part_rows = M;
         p.M = M; p.K = K; p.V = V; p.d = d; p.F = F; p.n_rs = n_rs;
         p.sumsq = sumsq; p.n_ss = n_ss; p.eps = c->cfg.rms_eps; p.act = act;
         p.status = status; p.user_status = out.status;
-        finish_shape(p, G);
+        finish_shape(p, G / p.n_groups);
         if (!make_map(s, &mA, xg, d, 2 * (uint64_t)M, 128) || !make_map(s, &mB0, hw.w_gate, d, F, p.bn / 2) ||
             !make_map(s, &mB1, hw.w_up, d, F, p.bn / 2))
             return note_err(c, cudaErrorInvalidValue, "tensor map (gate/up)");
-        e = note_err(c, launch_tc<KIND_GU, false>(mA, mB0, mB1, p, G, st), "gate/up kernel");
+        e = note_err(c, launch_tc<KIND_GU, false>(mA, mB0, mB1, p, p.n_groups * p.n_vr, st), "gate/up kernel");
         c->launches++;
         if (e != cudaSuccess) return e;
         // down projection, residual add, next operands
         memset(&p, 0, sizeof(p));
         p.units_total = d / 16; p.unit_rows = 16; p.n_boxes = 1; p.k_chunks = F / kBK;
-        p.n_groups = 1; p.n_rb = n_mb; p.rows = M;
+        p.n_groups = choose_groups(n_mb, p.units_total, G); p.n_rb = n_mb; p.rows = M;
         p.M = M; p.K = K; p.V = V; p.d = d; p.F = F; p.n_rs = n_rs; p.a_part_rows = M;
         p.hcur = hcur; p.h0f = h0f;
         p.gamma_next = (k < K) ? (const __nv_bfloat16 *)c->heads[k].rms_gamma : nullptr;
@@ -501,13 +517,13 @@ cudaError_t tc_draft(Ctx *c, const void *hidden, const float *logits0, const int
         p.sumsq_out = sumsq;
         p.hidden_out = (k == K) ? out.hidden_out : nullptr;
         p.status = status; p.user_status = out.status;
-        finish_shape(p, G);
+        finish_shape(p, G / p.n_groups);
         if (!make_map(s, &mA, act, F, 2 * (uint64_t)M, 128) || !make_map(s, &mB0, hw.w_down, F, d, p.bn))
             return note_err(c, cudaErrorInvalidValue, "tensor map (down)");
-        e = note_err(c, launch_tc<KIND_DN, false>(mA, mB0, mB0, p, G, st), "down kernel");
+        e = note_err(c, launch_tc<KIND_DN, false>(mA, mB0, mB0, p, p.n_groups * p.n_vr, st), "down kernel");
         c->launches++;
         if (e != cudaSuccess) return e;
-        n_ss = G;
+        n_ss = p.n_vr;
     }
     prof_mark(c, 1, st);
     int n_slices = G;
@@ -521,15 +537,7 @@ cudaError_t tc_draft(Ctx *c, const void *hidden, const float *logits0, const int
         // Row-steps of steps 1..K in 128-row blocks; CTA = (vocabulary range, group of row blocks).
         // Pick the split with the shortest longest CTA (in tiles), the fewest passes on ties.
         const int rows = K * M, n_rb = (rows + 127) / 128, U = V / 16;
-        int best_g = 1;
-        long long best_cost = -1;
-        for (int g = 1; g <= n_rb && g <= G; ++g) {
-            const int nv = G / g;
-            const int passes = (n_rb + g - 1) / g;
-            const int units = (U + nv - 1) / nv;
-            const long long cost = (long long)passes * ((units + 15) / 16);
-            if (best_cost < 0 || cost <= best_cost) { best_cost = cost; best_g = g; }
-        }
+        const int best_g = choose_groups(n_rb, U, G);
         p.n_groups = best_g;
         n_slices = G / best_g;
         p.n_rb = n_rb; p.rows = rows;
