@@ -60,6 +60,15 @@ typedef enum { MRP_F32 = 0, MRP_BF16 = 1 } mrp_dtype;
 #define MRP_FLAG_NO_PDL 2      /* launch every kernel fully serialised (no programmatic
                                   dependent launch); for timing comparisons               */
 #define MRP_FLAG_ROW_MAJOR_ONLY 4   /* tensor-core family: never use the few-row kernels  */
+#define MRP_FLAG_EXACT_OPERANDS 8   /* tensor-core family: always carry the LM-head activation
+                                       operand as a bf16 hi + lo pair (products exact to 2^-17),
+                                       also where the contraction is tensor-core bound.  Without
+                                       it, calls with more than 128 row-steps (K * M) round that
+                                       operand once to fp16 (11 significant bits) against an fp16
+                                       copy of W_lm kept in the workspace: half the tensor work,
+                                       confidence / log-sum-exp still within 2e-3.  The copy is
+                                       exact except for |w| < 2^-17 (absolute error <= 2^-25);
+                                       a W_lm with |w| > 65504 switches the mode off by itself. */
 
 typedef struct {
     int32_t d;          /* hidden size                                                   */

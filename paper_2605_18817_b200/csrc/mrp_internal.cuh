@@ -30,6 +30,9 @@ struct WorkspaceLayout {
     size_t sumsq;       // fp32 [kSumsqSlices, max_rows] per-CTA partial sums of squares
     size_t partials;    // Partial [n_slices_max, (n_heads+1)*max_rows]
     size_t dense_row;   // int32 [max_seqs*block_len] dense position -> masked row or -1
+    size_t w16;         // fp16 [V, d] copy of the LM head (0 bytes unless the fp16 LM path can run)
+    size_t xt16;        // fp16 [n_heads*max_rows, d] rows h_k - h_0 for that path
+    bool has_f16;
     size_t total;
     int32_t n_slices_max;
 };
@@ -37,6 +40,7 @@ struct WorkspaceLayout {
 constexpr int kSumsqSlices = 512;
 constexpr int kSimtSliceV = 128;      // vocabulary entries per SIMT LM-head slice
 constexpr int kSimtMaxBlocks = 592;   // SIMT LM-head grid cap (4 per SM)
+constexpr int kF16MinRowSteps = 129;  // fp16 LM-head operands from this many row-steps K*M on
 
 WorkspaceLayout workspace_layout(const mrp_config &cfg);
 
@@ -47,6 +51,7 @@ struct Ctx {
     char *ws;
     WorkspaceLayout lay;
     bool use_tc;
+    bool use_f16_lm;           // the fp16 copy of W_lm exists and is usable
     int32_t launches;
     int sm_count;
     void *tc_state;            // tensor-core path state (tensor maps), owned by tc_*.cu
@@ -78,9 +83,22 @@ inline void prof_mark(Ctx *c, int mark, cudaStream_t st)
 cudaError_t simt_draft(Ctx *c, const void *hidden, const float *logits0, const int32_t *row_index,
                        int M, int K, const mrp_draft_out &out, cudaStream_t st);
 
+// Optional exact recomputation of each row-step's top logit during the combine (used when the
+// LM-head operands were rounded to fp16): l_top = l_0[row, tok] + W_lm[tok] . (h_k - h_0) in
+// fp32 from the bf16 hi + lo rows, which removes the dominant token's rounding error from
+// log-sum-exp and confidence.  w == nullptr: off.
+struct TopFix {
+    const __nv_bfloat16 *w;      // [V, d]
+    const __nv_bfloat16 *xt;     // [2 * n_rs, d]: hi rows then lo rows, row-step major
+    const float *logits0;
+    const int32_t *row_index;
+    int d, V, M, n_rs;
+};
+
 // Shared by both families: merge per-slice partials into conf/lse/token/margin.
 cudaError_t launch_combine(Ctx *c, const Partial *partials, int n_slices, int n_rowsteps,
-                           const mrp_draft_out &out, int32_t *status, cudaStream_t st);
+                           const mrp_draft_out &out, int32_t *status, cudaStream_t st,
+                           const TopFix *fix = nullptr);
 // Shared by both families: gather masked rows of `hidden` into fp32 h0f / hcur.
 cudaError_t launch_prep(Ctx *c, const void *hidden, const int32_t *row_index, int M,
                         cudaStream_t st);

@@ -8,6 +8,7 @@
 // softmax statistics -> combine over slices.
 #include <float.h>
 #include <limits.h>
+#include <string.h>
 
 #include "mrp_internal.cuh"
 
@@ -255,7 +256,8 @@ lm_simt_kernel(const T *__restrict__ w_lm, const float *__restrict__ xt,
 __global__ void combine_kernel(const Partial *__restrict__ partials, int n_slices, int n_rs,
                                float *__restrict__ conf, float *__restrict__ lse,
                                int32_t *__restrict__ token, float *__restrict__ margin,
-                               int32_t *__restrict__ status, int32_t *__restrict__ user_status)
+                               int32_t *__restrict__ status, int32_t *__restrict__ user_status,
+                               const TopFix fix)
 {
     const int rs = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
@@ -273,12 +275,33 @@ __global__ void combine_kernel(const Partial *__restrict__ partials, int n_slice
         // fixed operand order (lower lane first) keeps the result identical on both sides
         p = (lane & o) ? merge_partial(q, p) : merge_partial(p, q);
     }
+    float top = p.mx;      // the top logit as the sum of exponentials saw it
+    if (fix.w && rs >= fix.M) {
+        // exact top logit: l_0[row, tok] + W[tok] . (hi + lo), fp32, fixed summation order
+        const int tok = __shfl_sync(0xffffffffu, p.idx, 0);
+        const int m = rs % fix.M;
+        const size_t row = fix.row_index ? (size_t)fix.row_index[m] : (size_t)m;
+        const __nv_bfloat16 *wr = fix.w + (size_t)tok * fix.d;
+        const __nv_bfloat16 *xh = fix.xt + (size_t)rs * fix.d, *xl = xh + (size_t)fix.n_rs * fix.d;
+        float dot = 0.f;
+        for (int j = lane * 2; j < fix.d; j += 64) {
+            const float2 w2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(wr + j));
+            const float2 h2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(xh + j));
+            const float2 l2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(xl + j));
+            dot = fmaf(w2.x, h2.x + l2.x, dot);
+            dot = fmaf(w2.y, h2.y + l2.y, dot);
+        }
+        dot = warp_sum(dot);
+        top = fix.logits0[row * (size_t)fix.V + tok] + dot;
+    }
     if (lane == 0) {
-        const float l = p.mx + logf(p.sum);
-        conf[rs] = 1.f / p.sum;
+        // the term of the top token entered the sum as exp(0) = 1: swap in its exact value
+        const float sum = (top == p.mx) ? p.sum : (p.sum - 1.f) + expf(top - p.mx);
+        const float l = p.mx + logf(sum);
+        conf[rs] = (top == p.mx) ? 1.f / sum : expf(top - l);
         lse[rs] = l;
         token[rs] = p.idx;
-        if (margin) margin[rs] = p.mx - p.second;
+        if (margin) margin[rs] = top - p.second;
         if (!isfinite(l)) {
             atomicOr(status, MRP_DEV_NONFINITE);
             if (user_status) atomicOr(user_status, MRP_DEV_NONFINITE);
@@ -287,12 +310,15 @@ __global__ void combine_kernel(const Partial *__restrict__ partials, int n_slice
 }
 
 cudaError_t launch_combine(Ctx *c, const Partial *partials, int n_slices, int n_rowsteps,
-                           const mrp_draft_out &out, int32_t *status, cudaStream_t st)
+                           const mrp_draft_out &out, int32_t *status, cudaStream_t st, const TopFix *fix)
 {
     if (n_rowsteps == 0) return cudaSuccess;
     const int warps = 4;
+    TopFix f;
+    memset(&f, 0, sizeof(f));
+    if (fix) f = *fix;
     combine_kernel<<<(n_rowsteps + warps - 1) / warps, warps * 32, 0, st>>>(
-        partials, n_slices, n_rowsteps, out.conf, out.lse, out.token, out.margin, status, out.status);
+        partials, n_slices, n_rowsteps, out.conf, out.lse, out.token, out.margin, status, out.status, f);
     c->launches++;
     return cudaGetLastError();
 }

@@ -138,6 +138,12 @@ __device__ __forceinline__ uint32_t make_idesc(int bn)
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 }
 
+// Same, fp16 x fp16 -> fp32.
+__device__ __forceinline__ uint32_t make_idesc_f16(int bn)
+{
+    return (1u << 4) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+}
+
 constexpr float kLog2e = 1.4426950408889634f;
 
 // Online softmax statistics of one logit row, updated 16 columns at a time.

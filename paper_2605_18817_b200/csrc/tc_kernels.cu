@@ -14,6 +14,7 @@
 // Orientation: activation rows are the MMA M dimension (128 TMEM lanes, one row per epilogue
 // thread), weight rows are the MMA N dimension.  Every CTA owns a contiguous range of weight
 // rows, split into equal tiles, and streams it exactly once per 128-row activation block.
+#include <cuda_fp16.h>
 #include <string.h>
 
 #include <new>
@@ -63,6 +64,7 @@ struct TcParams {
     const __nv_bfloat16 *gamma_next;
     __nv_bfloat16 *xg_next;
     __nv_bfloat16 *xt_k;
+    __half *xt16_k;      // optional: the same rows rounded once to fp16
     float *sumsq_out;
     float *hidden_out;
     int32_t *status;
@@ -72,16 +74,19 @@ struct TcParams {
 // ---------------------------------------------------------------------------------------
 // The kernel
 // ---------------------------------------------------------------------------------------
-template <int KIND, bool MARGIN>
+// F16: one fp16 A tile per stage against fp16 weights (LM head only); otherwise the bf16 hi and lo
+// A tiles of a k-chunk against bf16 weights.
+template <int KIND, bool MARGIN, bool F16>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
                const __grid_constant__ CUtensorMap tmB1, const TcParams p)
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    // a stage holds the hi and the lo A tile of a k-chunk and one B tile
+    // a stage holds the A tile(s) of a k-chunk and one B tile
+    constexpr int PARTS = F16 ? 1 : 2;
     const int b_bytes = (p.bn * 128 + 1023) & ~1023;
-    const int stage_bytes = 2 * kATile + b_bytes;
+    const int stage_bytes = PARTS * kATile + b_bytes;
     const uint32_t bars = base + (uint32_t)p.n_stages * stage_bytes;   // 8-byte aligned
     // barrier slots: full[s], empty[s], tmem_full[2], tmem_empty[2]
     auto full_bar = [&](int s) { return bars + 8u * s; };
@@ -121,7 +126,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     if (warp == 0) {
         // ---------------- TMA producer ----------------
         if (lane == 0) {
-            const uint32_t tx = (uint32_t)(2 * kATile + p.bn * 128);
+            const uint32_t tx = (uint32_t)(PARTS * kATile + p.bn * 128);
             const int box_rows = p.bn / p.n_boxes;
             int s = 0;
             uint32_t ph = 0;
@@ -134,8 +139,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         mbar_expect_tx(full_bar(s), tx);
                         const uint32_t sa = base + (uint32_t)s * stage_bytes;
                         tma_load_2d(sa, &tmA, kk * kBK, p.a_row_base + mb * 128, full_bar(s));
-                        tma_load_2d(sa + kATile, &tmA, kk * kBK, p.a_part_rows + p.a_row_base + mb * 128, full_bar(s));
-                        const uint32_t sb = sa + 2 * kATile;
+                        if (!F16)
+                            tma_load_2d(sa + kATile, &tmA, kk * kBK, p.a_part_rows + p.a_row_base + mb * 128, full_bar(s));
+                        const uint32_t sb = sa + PARTS * kATile;
                         tma_load_2d(sb, &tmB0, kk * kBK, n0, full_bar(s));
                         if (KIND == KIND_GU)
                             tma_load_2d(sb + box_rows * 128, &tmB1, kk * kBK, n0, full_bar(s));
@@ -147,7 +153,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
         if (lane == 0) {
-            const uint32_t idesc = make_idesc(p.bn);
+            const uint32_t idesc = F16 ? make_idesc_f16(p.bn) : make_idesc(p.bn);
             int s = 0, acc = 0;
             uint32_t ph = 0, acc_ph = 0;
             bool ok = true;
@@ -160,9 +166,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         if (!mbar_wait(full_bar(s), ph, abort_flag, p)) { ok = false; break; }
                         tc_fence_after();
                         const uint32_t sa = base + (uint32_t)s * stage_bytes;
-                        const uint64_t db = make_smem_desc(sa + 2 * kATile);
+                        const uint64_t db = make_smem_desc(sa + PARTS * kATile);
 #pragma unroll
-                        for (int a = 0; a < 2; ++a) {
+                        for (int a = 0; a < PARTS; ++a) {
                             const uint64_t da = make_smem_desc(sa + a * kATile);
 #pragma unroll
                             for (int k4 = 0; k4 < kBK / 16; ++k4)
@@ -266,6 +272,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
                             for (int j = 0; j < 16; ++j) h0[j] = hc[j] - h0[j];
                             store_split<16>(p.xt_k + o, (size_t)p.n_rs * p.d, h0);
+                            if (p.xt16_k) {
+                                __half2 hh[8];
+#pragma unroll
+                                for (int j = 0; j < 8; ++j) hh[j] = __floats2half2_rn(h0[2 * j], h0[2 * j + 1]);
+                                uint4 *dst = reinterpret_cast<uint4 *>(p.xt16_k + o);
+                                dst[0] = *reinterpret_cast<uint4 *>(&hh[0]);
+                                dst[1] = *reinterpret_cast<uint4 *>(&hh[4]);
+                            }
                             if (p.xg_next) {
                                 const __nv_bfloat16 *gm = p.gamma_next + j_tile + c * 16;
 #pragma unroll
@@ -345,6 +359,22 @@ __global__ void tc_prep_kernel(const __nv_bfloat16 *__restrict__ hidden, const i
     }
 }
 
+// fp16 copy of a bf16 matrix.  bf16 values inside fp16's normal range convert exactly; smaller
+// ones round to fp16 subnormals (absolute error <= 2^-25); flag[0] is set if a finite value
+// overflows fp16 or a value is not finite, which rules the copy out.
+__global__ void to_half_kernel(const __nv_bfloat16 *__restrict__ src, __half *__restrict__ dst, size_t n,
+                               int32_t *__restrict__ flag)
+{
+    bool bad = false;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        const float v = __bfloat162float(src[i]);
+        const __half h = __float2half_rn(v);
+        bad |= !isfinite(__half2float(h));
+        dst[i] = h;
+    }
+    if (bad) atomicOr(flag, 1);
+}
+
 // ---------------------------------------------------------------------------------------
 // Host side
 // ---------------------------------------------------------------------------------------
@@ -373,7 +403,7 @@ int choose_groups(int n_rb, int units_total, int G)
     return best_g;
 }
 
-void finish_shape(TcParams &p, int n_vr)
+void finish_shape(TcParams &p, int n_vr, int parts = 2)
 {
     p.n_vr = n_vr;
     const int maxunits = (p.units_total + n_vr - 1) / n_vr;
@@ -385,24 +415,24 @@ void finish_shape(TcParams &p, int n_vr)
     p.w_units = choose_tile_units(maxunits < 1 ? 1 : maxunits, w_max);
     p.bn = p.w_units * rows_per_unit;
     const int b_bytes = (p.bn * 128 + 1023) & ~1023;
-    const int stage = 2 * kATile + b_bytes;
+    const int stage = parts * kATile + b_bytes;
     int ns = (kSmemBudget - 1024 - 512) / stage;
     if (ns > 12) ns = 12;
     p.n_stages = ns;
 }
 
-size_t smem_bytes(const TcParams &p)
+size_t smem_bytes(const TcParams &p, int parts)
 {
     const int b_bytes = (p.bn * 128 + 1023) & ~1023;
-    return (size_t)p.n_stages * (2 * kATile + b_bytes) + 1024 + 8 * (2 * p.n_stages + 4) + 16;
+    return (size_t)p.n_stages * (parts * kATile + b_bytes) + 1024 + 8 * (2 * p.n_stages + 4) + 16;
 }
 
-template <int KIND, bool MARGIN>
+template <int KIND, bool MARGIN, bool F16 = false>
 cudaError_t launch_tc(const CUtensorMap &a, const CUtensorMap &b0, const CUtensorMap &b1, const TcParams &p,
                       int grid, cudaStream_t st)
 {
-    auto kern = tc_gemm_kernel<KIND, MARGIN>;
-    const size_t smem = smem_bytes(p);
+    auto kern = tc_gemm_kernel<KIND, MARGIN, F16>;
+    const size_t smem = smem_bytes(p, F16 ? 1 : 2);
     static bool attr_set = false;
     if (!attr_set) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
@@ -441,6 +471,21 @@ cudaError_t tc_create(Ctx *c)
     }
     s->encode = (EncodeTiledFn)fn;
     c->tc_state = s;
+    c->use_f16_lm = false;
+    if (c->lay.has_f16) {
+        // one-time fp16 copy of the LM head for the tensor-core-bound regime
+        int32_t *flag = (int32_t *)(c->ws + c->lay.status) + 8;
+        e = cudaMemset(flag, 0, sizeof(int32_t));
+        if (e != cudaSuccess) return e;
+        to_half_kernel<<<c->sm_count * 8, 256>>>((const __nv_bfloat16 *)c->w_lm, (__half *)(c->ws + c->lay.w16),
+                                                 (size_t)c->cfg.vocab * c->cfg.d, flag);
+        e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+        int32_t bad = 1;
+        e = cudaMemcpy(&bad, flag, sizeof(bad), cudaMemcpyDeviceToHost);
+        if (e != cudaSuccess) return e;
+        c->use_f16_lm = (bad == 0);
+    }
     return cudaSuccess;
 }
 
@@ -477,6 +522,7 @@ cudaError_t tc_draft(Ctx *c, const void *hidden, const float *logits0, const int
     if (e != cudaSuccess) return e;
 
     const bool pdl = !(c->cfg.flags & MRP_FLAG_NO_PDL);
+    const bool f16_lm = c->use_f16_lm && K * M >= kF16MinRowSteps;
     const bool few_rows = sk_rows_ok(M) && !(c->cfg.flags & MRP_FLAG_ROW_MAJOR_ONLY);
     int n_ss = 1;
     for (int k = 1; k <= K; ++k) {
@@ -514,6 +560,7 @@ cudaError_t tc_draft(Ctx *c, const void *hidden, const float *logits0, const int
         p.gamma_next = (k < K) ? (const __nv_bfloat16 *)c->heads[k].rms_gamma : nullptr;
         p.xg_next = (k < K) ? xg : nullptr;
         p.xt_k = xt + (size_t)k * M * d;
+        p.xt16_k = f16_lm ? (__half *)(c->ws + c->lay.xt16) + (size_t)(k - 1) * M * d : nullptr;
         p.sumsq_out = sumsq;
         p.hidden_out = (k == K) ? out.hidden_out : nullptr;
         p.status = status; p.user_status = out.status;
@@ -546,17 +593,34 @@ cudaError_t tc_draft(Ctx *c, const void *hidden, const float *logits0, const int
         p.M = M; p.K = K; p.V = V; p.d = d; p.F = F; p.n_rs = n_rs;
         p.logits0 = logits0; p.row_index = row_index; p.partials = partials; p.logits_out = out.logits_out;
         p.status = status; p.user_status = out.status;
-        finish_shape(p, n_slices);
-        if (!make_map(s, &mA, xt, d, 2 * (uint64_t)n_rs, 128) || !make_map(s, &mB, c->w_lm, d, V, p.bn))
-            return note_err(c, cudaErrorInvalidValue, "tensor map (LM head)");
+        finish_shape(p, n_slices, f16_lm ? 1 : 2);
         const int grid = p.n_groups * p.n_vr;
-        e = note_err(c, out.margin ? launch_tc<KIND_LM, true>(mA, mB, mB, p, grid, st)
-                                   : launch_tc<KIND_LM, false>(mA, mB, mB, p, grid, st), "LM-head kernel");
+        if (f16_lm) {
+            // 16-bit elements either way: the bf16 tensor-map type only moves the bytes
+            p.a_row_base = 0;
+            if (!make_map(s, &mA, c->ws + c->lay.xt16, d, (uint64_t)rows, 128) ||
+                !make_map(s, &mB, c->ws + c->lay.w16, d, V, p.bn))
+                return note_err(c, cudaErrorInvalidValue, "tensor map (LM head, fp16)");
+            e = note_err(c, out.margin ? launch_tc<KIND_LM, true, true>(mA, mB, mB, p, grid, st)
+                                       : launch_tc<KIND_LM, false, true>(mA, mB, mB, p, grid, st),
+                         "LM-head kernel (fp16 operands)");
+        } else {
+            if (!make_map(s, &mA, xt, d, 2 * (uint64_t)n_rs, 128) || !make_map(s, &mB, c->w_lm, d, V, p.bn))
+                return note_err(c, cudaErrorInvalidValue, "tensor map (LM head)");
+            e = note_err(c, out.margin ? launch_tc<KIND_LM, true>(mA, mB, mB, p, grid, st)
+                                       : launch_tc<KIND_LM, false>(mA, mB, mB, p, grid, st), "LM-head kernel");
+        }
         c->launches++;
         if (e != cudaSuccess) return e;
     }
     prof_mark(c, 2, st);
-    e = launch_combine(c, partials, n_slices, (K + 1) * M, out, status, st);
+    TopFix fix;
+    memset(&fix, 0, sizeof(fix));
+    if (f16_lm) {
+        fix.w = (const __nv_bfloat16 *)c->w_lm; fix.xt = xt; fix.logits0 = logits0; fix.row_index = row_index;
+        fix.d = d; fix.V = V; fix.M = M; fix.n_rs = n_rs;
+    }
+    e = launch_combine(c, partials, n_slices, (K + 1) * M, out, status, st, f16_lm ? &fix : nullptr);
     prof_mark(c, 3, st);
     return e;
 }

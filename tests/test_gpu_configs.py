@@ -180,3 +180,29 @@ def test_sweep_points_sampled_rows(sweep_dev, M, K):
     assert torch.equal(l0.argmax(dim=1).int().cpu(), out.token[0].cpu())
     assert torch.allclose(torch.logsumexp(l0, dim=1), out.lse[0], atol=2e-3)
     binding.mrp_destroy(ctx)
+
+
+@pytest.mark.parametrize("M,K", [(256, 1), (1024, 2), (4096, 4)])
+def test_fp16_operand_mode_stays_close_to_exact_operands_on_every_row(sweep_dev, M, K):
+    """Above 128 row-steps the LM head rounds its activation operand once to fp16 instead of
+    carrying a bf16 hi + lo pair.  Every row-step of the call is compared with the same call
+    under MRP_FLAG_EXACT_OPERANDS (itself checked against the oracle on sampled rows above):
+    the two must agree well inside the 2e-3 tolerance, which leaves the exact path's own error
+    as margin."""
+    dev = sweep_dev
+    cfg = synth.sweep_config(M, K)
+    _, inp = synth.make_config(cfg, dev.w, logits_fn=dev.logits_fn)
+    outs = []
+    for flags in (0, binding.MRP_FLAG_EXACT_OPERANDS):
+        ctx = dev.ctx(M, M, 1, n_heads=K, flags=flags)
+        out, _ = gpu_draft(dev, ctx, inp, K, margin=True)
+        outs.append(out)
+        binding.mrp_destroy(ctx)
+    a, b = outs
+    dconf = (a.conf - b.conf).abs().max().item()
+    dlse = (a.lse - b.lse).abs().max().item()
+    print("M=%d K=%d max|dconf|=%.2e max|dlse|=%.2e" % (M, K, dconf, dlse))
+    assert dconf <= 1.5e-3 and dlse <= 1.5e-3
+    clear = b.margin > 1e-2
+    assert torch.equal(a.token[clear], b.token[clear])
+    assert torch.equal(a.conf[0], b.conf[0])          # step 0 never touches the operands
