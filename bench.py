@@ -40,7 +40,7 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="1",
-                    help="0..3 = benchmark configuration, or sweep:M:K for a roofline-sweep point")
+                    help="0..3 = benchmark configuration, sweep:M:K = one roofline-sweep point, sweep = all 21 points")
     ap.add_argument("--flags", type=int, default=0, help="mrp_config.flags (MRP_FLAG_* bits) for A/B timing")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -236,8 +236,76 @@ def run_reference(args, cfg):
     print(json.dumps(line), flush=True)
 
 
+def run_sweep(args):
+    """Roofline sweep (configuration 4): d = 4096, V = 151936, masked rows M in {1 .. 4096} times
+    chain length K in {1, 2, 4}, one weight set shared by all points.  Prints one JSON line per
+    point: time per drafting pass, draft tokens/s, the fused LM-head kernel's time and its
+    fraction of the roofline (slower of algorithmic bytes over HBM bandwidth and flops over the
+    bf16 tensor peak), and the same fraction for the whole mrp_draft call."""
+    import numpy as np
+    import torch
+    from paper_2605_18817_b200 import build as _build
+    if not os.environ.get("MRP_B200_LIB"):
+        _build.build()
+    from paper_2605_18817_b200 import binding, harness, synth
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    peaks, peaks_kind = load_peaks()
+    w = synth.make_weights(4096, 8192, 151936, 4, "bf16", 4000)
+    heads, w_lm = harness.upload_weights(w, dev)
+    logits_fn = harness.device_logits_fn(w_lm)
+    d, F, V = w.d, w.F, w.V
+    for M in synth.SWEEP_ROWS:
+        for K in synth.SWEEP_CHAIN:
+            cfg = synth.sweep_config(M, K)
+            _, inp = synth.make_config(cfg, w, logits_fn=logits_fn)
+            ctx = binding.mrp_create(d, F, V, heads[:K], w_lm, max_rows=M, max_seqs=M, block_len=1,
+                                     flags=args.flags)
+            hid = harness.to_device(inp.hidden, w.dtype, dev)
+            l0 = torch.from_numpy(inp.logits0).to(dev)
+            ri = torch.from_numpy(inp.row_index).to(dev)
+            out = harness.alloc_draft_out(M, K, V, d, dev, margin=False)
+            for _ in range(3):
+                harness.draft(ctx, hid, l0, ri, M, K, out)
+            torch.cuda.synchronize()
+            ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            ev0.record()
+            harness.draft(ctx, hid, l0, ri, M, K, out)
+            ev1.record()
+            torch.cuda.synchronize()
+            n = int(max(5, min(200, 300.0 / max(ev0.elapsed_time(ev1), 1e-3))))
+            ev0.record()
+            for _ in range(n):
+                harness.draft(ctx, hid, l0, ri, M, K, out)
+            ev1.record()
+            torch.cuda.synchronize()
+            ms = ev0.elapsed_time(ev1) / n
+            binding.mrp_profile_enable(ctx, True)
+            for _ in range(n):
+                harness.draft(ctx, hid, l0, ri, M, K, out)
+            torch.cuda.synchronize()
+            (ms_heads, ms_lm, ms_comb), nc = binding.mrp_profile_read(ctx)
+            binding.mrp_profile_enable(ctx, False)
+            roof = lm_head_roofline(cfg, M, ms_lm / nc, peaks, peaks_kind, None)
+            call_bytes = 2.0 * V * d + K * (6.0 * d * F + 2 * d) + 4.0 * M * V + 2.0 * M * d + 12.0 * (K + 1) * M
+            call_flops = 2.0 * K * M * V * d + 6.0 * K * M * d * F
+            t_roof = max(call_bytes / (peaks["hbm_gbs"] * 1e9), call_flops / (peaks["bf16_tflops_sustained"] * 1e12))
+            print(json.dumps({
+                "workload": cfg["name"], "rows": M, "chain": K, "ms_per_draft": ms,
+                "draft_tokens_per_s": K * M / (ms * 1e-3), "heads_ms": ms_heads / nc,
+                "lm_head_ms": ms_lm / nc, "combine_ms": ms_comb / nc,
+                "lm_head_roofline": {k: roof[k] for k in ("bound", "achieved", "peak", "unit", "frac")},
+                "draft_call_roofline_frac": t_roof / (ms * 1e-3), "family": ctx.family,
+                "peaks": peaks_kind}), flush=True)
+            binding.mrp_destroy(ctx)
+            del hid, l0, ri, out
+
+
 def main():
     args = parse_args()
+    if args.config == "sweep":
+        run_sweep(args)
+        return
     cfg = resolve_config(args.config)
     if args.impl == "reference":
         run_reference(args, cfg)

@@ -18,6 +18,19 @@ def to_device(a: np.ndarray, dtype: str, device) -> torch.Tensor:
     return torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).to(device)
 
 
+def device_logits_fn(w_lm: torch.Tensor, chunk: int = 16384):
+    """Input generation helper: base logits of the synthetic backbone as an fp32 product on
+    the device (TF32 off), returned to the host; plugs into ``synth.make_inputs(logits_fn=)``."""
+    def fn(rows: np.ndarray) -> np.ndarray:
+        torch.backends.cuda.matmul.allow_tf32 = False
+        x = torch.from_numpy(np.ascontiguousarray(rows, dtype=np.float32)).to(w_lm.device)
+        out = torch.empty((x.shape[0], w_lm.shape[0]), device=w_lm.device)
+        for v0 in range(0, w_lm.shape[0], chunk):
+            out[:, v0:v0 + chunk] = x @ w_lm[v0:v0 + chunk].float().T
+        return out.cpu().numpy()
+    return fn
+
+
 def upload_weights(w: synth.Weights, device):
     heads = [{k: to_device(v, w.dtype, device) for k, v in h.items()} for h in w.heads]
     return heads, to_device(w.w_lm, w.dtype, device)
