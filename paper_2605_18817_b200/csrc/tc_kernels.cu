@@ -327,8 +327,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 __global__ void tc_prep_kernel(const __nv_bfloat16 *__restrict__ hidden, const int32_t *__restrict__ row_index,
                                int d, int M, int n_rs, const __nv_bfloat16 *__restrict__ gamma1,
                                float *__restrict__ h0f, float *__restrict__ hcur, __nv_bfloat16 *__restrict__ xg,
-                               __nv_bfloat16 *__restrict__ xt0, float *__restrict__ sumsq)
+                               __nv_bfloat16 *__restrict__ xt0, float *__restrict__ sumsq,
+                               int32_t *__restrict__ counters, int n_counters)
 {
+    // arrival counters of the few-row head kernels start every pass at zero
+    if (blockIdx.x == 0)
+        for (int i = threadIdx.x; i < n_counters; i += blockDim.x) counters[i] = 0;
     __shared__ float red[8];
     const int m = blockIdx.x;
     const size_t row = row_index ? (size_t)row_index[m] : (size_t)m;
@@ -516,22 +520,23 @@ cudaError_t tc_draft(Ctx *c, const void *hidden, const float *logits0, const int
     prof_mark(c, 0, st);
     const int n_rs = (K + 1) * M;
     tc_prep_kernel<<<M, 256, 0, st>>>((const __nv_bfloat16 *)hidden, row_index, d, M, n_rs,
-                                      (const __nv_bfloat16 *)c->heads[0].rms_gamma, h0f, hcur, xg, xt, sumsq);
+                                      (const __nv_bfloat16 *)c->heads[0].rms_gamma, h0f, hcur, xg, xt, sumsq,
+                                      (int32_t *)(c->ws + c->lay.sk_counters), kSkMaxTiles);
     c->launches++;
     cudaError_t e = note_err(c, cudaGetLastError(), "tc_prep_kernel");
     if (e != cudaSuccess) return e;
 
     const bool pdl = !(c->cfg.flags & MRP_FLAG_NO_PDL);
     const bool f16_lm = c->use_f16_lm && K * M >= kF16MinRowSteps;
-    const bool few_rows = sk_rows_ok(M) && !(c->cfg.flags & MRP_FLAG_ROW_MAJOR_ONLY);
+    const bool few_rows = sk_rows_ok(M) && sk_heads_ok(c->cfg) && G <= kSkScratchCtas &&
+                          !(c->cfg.flags & MRP_FLAG_ROW_MAJOR_ONLY);
     int n_ss = 1;
     for (int k = 1; k <= K; ++k) {
         if (few_rows) {
             e = sk_gateup(c, k, M, K, n_ss, out, st, pdl);
             if (e != cudaSuccess) return e;
-            e = sk_down(c, k, M, K, out, st, pdl);
+            e = sk_down(c, k, M, K, out, st, pdl, &n_ss);
             if (e != cudaSuccess) return e;
-            n_ss = G;
             continue;
         }
         const mrp_head_weights &hw = c->heads[k - 1];

@@ -45,7 +45,11 @@ struct SkParams {
     int r_pad;           // activation rows per part (16 or 32); MMA N = 2 * r_pad
     int tmem_cols;       // allocated TMEM columns (power of two >= 2 buffers * 2 * r_pad)
     int x_row_hi, x_row_lo;
-    int tail_units[2];   // units of short-tile kinds 1 and 2
+    int tail_units[2];   // units of short-tile kinds 1 and 2 (LM)
+    int n_split;         // GU/DN: CTAs sharing one 128-row weight tile, each a slice of the contraction
+    int w_rows;          // GU/DN: weight rows (gate rows for GU)
+    float *scratch;      // GU/DN: partial accumulators [tile][split][RP][128]
+    int32_t *counters;   // GU/DN: arrivals per tile (zero between launches)
     int M, K, V, d, F, n_rs;
     // LM
     const float *logits0;
@@ -101,9 +105,22 @@ sk_gemm_kernel(const __grid_constant__ SkMaps maps, const SkParams p)
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int cta = blockIdx.x, G = gridDim.x;
-    const int u_base = p.units_total / G, u_extra = p.units_total % G;
-    const int units = u_base + (cta < u_extra ? 1 : 0);
-    const int u0 = cta * u_base + min(cta, u_extra);
+    // LM: a contiguous range of 16-row units per CTA, the whole contraction.
+    // GU/DN: one full 128-row tile per CTA and one of n_split slices of the contraction; the
+    // slices of a tile are summed, in slice order, by whichever of its CTAs finishes last.
+    int units, u0, kc0 = 0, kc1 = p.k_chunks;
+    if (KIND == SK_LM) {
+        const int u_base = p.units_total / G, u_extra = p.units_total % G;
+        units = u_base + (cta < u_extra ? 1 : 0);
+        u0 = cta * u_base + min(cta, u_extra);
+    } else {
+        const int cps = (p.k_chunks + p.n_split - 1) / p.n_split;
+        units = 8;
+        u0 = (cta / p.n_split) * 8;
+        kc0 = (cta % p.n_split) * cps;
+        kc1 = min(p.k_chunks, kc0 + cps);
+    }
+    const int nk = kc1 - kc0;
     const int n_full = units >> 3, rem = units & 7;
     const int n_tiles = n_full + (rem ? 1 : 0);
     const int tail_kind = (rem == p.tail_units[0]) ? 1 : 2;
@@ -130,7 +147,7 @@ sk_gemm_kernel(const __grid_constant__ SkMaps maps, const SkParams p)
     if (warp == 0) {
         // ---------------- TMA producer ----------------
         if (lane == 0) {
-            const int total_it = n_tiles * p.k_chunks;
+            const int total_it = n_tiles * nk;
             const int pre = min(p.n_stages, total_it);
             auto load_w = [&](int t, int kk, int s) {
                 const uint32_t sw = base + (uint32_t)s * stage_bytes;
@@ -140,27 +157,27 @@ sk_gemm_kernel(const __grid_constant__ SkMaps maps, const SkParams p)
                 mbar_expect_tx(full_bar(s), w_bytes + (uint32_t)x_bytes);
                 const int ut = u0 + 8 * t;
                 if (KIND == SK_GU) {
-                    tma_load_2d(sw, &maps.w[kind], kk * kBK, ut * 8, full_bar(s));
-                    tma_load_2d(sw + 64 * 128, &maps.w[3 + kind], kk * kBK, ut * 8, full_bar(s));
+                    tma_load_2d(sw, &maps.w[kind], (kc0 + kk) * kBK, ut * 8, full_bar(s));
+                    tma_load_2d(sw + 64 * 128, &maps.w[3 + kind], (kc0 + kk) * kBK, ut * 8, full_bar(s));
                 } else {
-                    tma_load_2d(sw, &maps.w[kind], kk * kBK, ut * 16, full_bar(s));
+                    tma_load_2d(sw, &maps.w[kind], (kc0 + kk) * kBK, ut * 16, full_bar(s));
                 }
             };
             auto load_x = [&](int kk, int s) {
                 const uint32_t sx = base + (uint32_t)s * stage_bytes + kWTile;
-                tma_load_2d(sx, &maps.x, kk * kBK, p.x_row_hi, full_bar(s));
-                tma_load_2d(sx + RP * 128, &maps.x, kk * kBK, p.x_row_lo, full_bar(s));
+                tma_load_2d(sx, &maps.x, (kc0 + kk) * kBK, p.x_row_hi, full_bar(s));
+                tma_load_2d(sx + RP * 128, &maps.x, (kc0 + kk) * kBK, p.x_row_lo, full_bar(s));
             };
             // weights do not depend on the previous kernel: fill the ring with them first
             int t = 0, kk = 0;
             for (int it = 0; it < pre; ++it) {
                 load_w(t, kk, it);
-                if (++kk == p.k_chunks) { kk = 0; ++t; }
+                if (++kk == nk) { kk = 0; ++t; }
             }
             griddep_wait();
             for (int it = 0, k2 = 0; it < pre; ++it) {
                 load_x(k2, it);
-                if (++k2 == p.k_chunks) k2 = 0;
+                if (++k2 == nk) k2 = 0;
             }
             int s = 0;
             uint32_t ph = 1;              // the ring has been filled once
@@ -168,7 +185,7 @@ sk_gemm_kernel(const __grid_constant__ SkMaps maps, const SkParams p)
                 if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p)) break;
                 load_w(t, kk, s);
                 load_x(kk, s);
-                if (++kk == p.k_chunks) { kk = 0; ++t; }
+                if (++kk == nk) { kk = 0; ++t; }
                 if (++s == p.n_stages) { s = 0; ph ^= 1u; }
             }
         }
@@ -183,7 +200,7 @@ sk_gemm_kernel(const __grid_constant__ SkMaps maps, const SkParams p)
                 if (!mbar_wait(tempty_bar(acc), acc_ph ^ 1u, abort_flag, p)) break;
                 tc_fence_after();
                 const uint32_t dt = tmem_base + (uint32_t)(acc * 2 * RP);
-                for (int kk = 0; kk < p.k_chunks; ++kk) {
+                for (int kk = 0; kk < nk; ++kk) {
                     if (!mbar_wait(full_bar(s), ph, abort_flag, p)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t sw = base + (uint32_t)s * stage_bytes;
@@ -247,29 +264,20 @@ sk_gemm_kernel(const __grid_constant__ SkMaps maps, const SkParams p)
         for (int ti = 0; ti < n_tiles && ok; ++ti) {
             const int ut = u0 + 8 * ti;
             const int units_here = ti < n_full ? 8 : rem;
-            // What the tile's outputs are added to does not depend on the accumulator: fetch it
-            // (independent loads, all in flight together) before waiting for the MMAs.
             float a[RP];
-            float h0v[KIND == SK_DN ? RP : 1];
-            const bool valid = KIND == SK_GU ? (t < 64 && t < units_here * 8) : (t < units_here * 16);
             const int wrow = KIND == SK_GU ? ut * 8 + t : ut * 16 + t;     // weight row = output feature
+            const bool valid = KIND == SK_LM ? (t < units_here * 16)
+                                             : (KIND == SK_GU ? (t < 64 && wrow < p.w_rows) : (wrow < p.w_rows));
+            // LM: what the tile's outputs are added to does not depend on the accumulator: fetch
+            // it (independent loads, all in flight together) before waiting for the MMAs.
 #pragma unroll
             for (int j = 0; j < RP; ++j) {
                 a[j] = 0.f;
-                if (KIND == SK_LM) {
-                    if (valid && j < p.n_rs) a[j] = __ldg(p.logits0 + rowoff_s[j] + wrow);
-                } else if (KIND == SK_DN) {
-                    h0v[j] = 0.f;
-                    if (valid && j < p.M) {
-                        a[j] = p.hcur[(size_t)j * p.d + wrow];
-                        h0v[j] = __ldg(p.h0f + (size_t)j * p.d + wrow);
-                    }
-                }
+                if (KIND == SK_LM && valid && j < p.n_rs) a[j] = __ldg(p.logits0 + rowoff_s[j] + wrow);
             }
-            const float gm = (KIND == SK_DN && valid && p.xg_next) ? __bfloat162float(p.gamma_next[wrow]) : 0.f;
 
             ok = __all_sync(0xffffffffu, mbar_wait(tfull_bar(acc), acc_ph, abort_flag, p));
-            if (KIND == SK_GU) {
+            if (KIND != SK_LM) {
                 // the four warps meet at barriers below: they must leave the loop together
                 if (!ok && lane == 0) *vote_s = 1;
                 epi_sync();
@@ -311,7 +319,36 @@ sk_gemm_kernel(const __grid_constant__ SkMaps maps, const SkParams p)
                         }
                     }
                 }
-            } else if (KIND == SK_GU) {
+                continue;
+            }
+
+            // ---- GU / DN: sum the slices of the contraction ----
+            if (p.n_split > 1) {
+                const int tile = cta / p.n_split, split = cta % p.n_split;
+                float *mine = p.scratch + ((size_t)cta * RP) * 128;
+#pragma unroll
+                for (int j = 0; j < RP; ++j)
+                    if (j < p.M) mine[j * 128 + t] = a[j];
+                __threadfence();
+                epi_sync();
+                if (t == 0) *vote_s = (atomicAdd(p.counters + tile, 1) == p.n_split - 1) ? 2 : 0;
+                epi_sync();
+                if (*vote_s != 2) break;          // another CTA of this tile finishes the job
+                __threadfence();
+                const float *first = p.scratch + ((size_t)tile * p.n_split * RP) * 128;
+#pragma unroll
+                for (int j = 0; j < RP; ++j) a[j] = 0.f;
+#pragma unroll 1
+                for (int sp = 0; sp < p.n_split; ++sp) {          // slice order: the sum does not depend on who is last
+#pragma unroll
+                    for (int j = 0; j < RP; ++j)
+                        if (j < p.M) a[j] += __ldcg(first + ((size_t)sp * RP + j) * 128 + t);
+                }
+                if (t == 0) p.counters[tile] = 0;
+                (void)split;
+            }
+
+            if (KIND == SK_GU) {
                 // lanes 0-63 hold gate rows, 64-127 the matching up rows: hand the up values over
                 if (t >= 64) {
 #pragma unroll
@@ -329,20 +366,27 @@ sk_gemm_kernel(const __grid_constant__ SkMaps maps, const SkParams p)
                         }
                     }
                 }
-                epi_sync();
-            } else {
-                if (valid) {
+            } else if (valid) {
+                float hc[RP], h0v[RP];
 #pragma unroll
-                    for (int m = 0; m < RP; ++m) {
-                        if (m < p.M) {
-                            const size_t o = (size_t)m * p.d + wrow;
-                            const float hc = a[m];
-                            p.hcur[o] = hc;
-                            if (p.hidden_out) p.hidden_out[o] = hc;
-                            ssq[m] = fmaf(hc, hc, ssq[m]);
-                            store_hi_lo(p.xt_k + o, (size_t)p.n_rs * p.d, hc - h0v[m]);
-                            if (p.xg_next) store_hi_lo(p.xg_next + o, (size_t)p.M * p.d, hc * gm);
-                        }
+                for (int m = 0; m < RP; ++m) {
+                    hc[m] = 0.f; h0v[m] = 0.f;
+                    if (m < p.M) {
+                        hc[m] = p.hcur[(size_t)m * p.d + wrow];
+                        h0v[m] = __ldg(p.h0f + (size_t)m * p.d + wrow);
+                    }
+                }
+                const float gm = p.xg_next ? __bfloat162float(p.gamma_next[wrow]) : 0.f;
+#pragma unroll
+                for (int m = 0; m < RP; ++m) {
+                    if (m < p.M) {
+                        const size_t o = (size_t)m * p.d + wrow;
+                        const float h = hc[m] + a[m];
+                        p.hcur[o] = h;
+                        if (p.hidden_out) p.hidden_out[o] = h;
+                        ssq[m] = fmaf(h, h, ssq[m]);
+                        store_hi_lo(p.xt_k + o, (size_t)p.n_rs * p.d, h - h0v[m]);
+                        if (p.xg_next) store_hi_lo(p.xg_next + o, (size_t)p.M * p.d, h * gm);
                     }
                 }
             }
@@ -398,8 +442,10 @@ sk_gemm_kernel(const __grid_constant__ SkMaps maps, const SkParams p)
                 }
             }
             epi_sync();
-            if (ok && t < p.M)
-                p.sumsq_out[(size_t)cta * p.M + t] = (ssq_s[t] + ssq_s[32 + t]) + (ssq_s[64 + t] + ssq_s[96 + t]);
+            // one slice of sums of squares per weight tile, written by the CTA that finished it
+            const bool finisher = p.n_split == 1 || *vote_s == 2;
+            if (ok && finisher && t < p.M)
+                p.sumsq_out[(size_t)(cta / p.n_split) * p.M + t] = (ssq_s[t] + ssq_s[32 + t]) + (ssq_s[64 + t] + ssq_s[96 + t]);
         }
     }
 
@@ -437,9 +483,27 @@ void sk_finish_shape(SkParams &p, int grid)
     int cols = 32;
     while (cols < 2 * 2 * p.r_pad) cols <<= 1;
     p.tmem_cols = cols;
-    const int u_base = p.units_total / grid;
-    p.tail_units[0] = u_base % 8;
-    p.tail_units[1] = (u_base + 1) % 8;
+    p.n_split = 1;
+    p.tail_units[0] = p.tail_units[1] = 0;
+    if (grid > 0) {           // LM: contiguous unit ranges, short tiles of two possible heights
+        const int u_base = p.units_total / grid;
+        p.tail_units[0] = u_base % 8;
+        p.tail_units[1] = (u_base + 1) % 8;
+    }
+}
+
+// GU/DN: n_tiles full weight tiles, each shared by n_split CTAs that take slices of the contraction.
+int sk_split(Ctx *c, SkParams &p, int n_tiles)
+{
+    int S = c->sm_count / n_tiles;
+    if (S < 1) S = 1;
+    if (S > p.k_chunks) S = p.k_chunks;
+    const int cps = (p.k_chunks + S - 1) / S;
+    S = (p.k_chunks + cps - 1) / cps;          // no empty slice
+    p.n_split = S;
+    p.scratch = (float *)(c->ws + c->lay.sk_scratch);
+    p.counters = (int32_t *)(c->ws + c->lay.sk_counters);
+    return n_tiles * S;
 }
 
 // Tensor maps of one weight matrix part: full tiles and the two short-tile heights.
@@ -503,6 +567,8 @@ void sk_common(Ctx *c, SkParams &p, int M, int K, const mrp_draft_out &out)
 
 bool sk_rows_ok(int rows) { return rows >= 1 && rows <= 32; }
 
+bool sk_heads_ok(const mrp_config &cfg) { return (cfg.d + 127) / 128 <= kSumsqSlices && cfg.d_ff / 64 <= kSkMaxTiles; }
+
 cudaError_t sk_gateup(Ctx *c, int k, int M, int K, int n_ss, const mrp_draft_out &out, cudaStream_t st, bool pdl)
 {
     const TcState *s = (const TcState *)c->tc_state;
@@ -510,28 +576,30 @@ cudaError_t sk_gateup(Ctx *c, int k, int M, int K, int n_ss, const mrp_draft_out
     const int d = c->cfg.d, F = c->cfg.d_ff, G = c->sm_count;
     SkParams p;
     sk_common(c, p, M, K, out);
-    p.units_total = F / 8; p.k_chunks = d / kBK; p.r_pad = M <= 16 ? 16 : 32;
+    p.units_total = F / 8; p.k_chunks = d / kBK; p.r_pad = M <= 16 ? 16 : 32; p.w_rows = F;
     p.x_row_hi = 0; p.x_row_lo = M;
     p.sumsq = (const float *)(c->ws + c->lay.sumsq); p.n_ss = n_ss; p.eps = c->cfg.rms_eps;
     p.act = (__nv_bfloat16 *)(c->ws + c->lay.act);
-    sk_finish_shape(p, G);
+    sk_finish_shape(p, 0);
+    const int grid = sk_split(c, p, F / 64);
+    (void)G;
     SkMaps maps;
     memset(&maps, 0, sizeof(maps));
     if (!make_map(s, &maps.x, c->ws + c->lay.xg, d, 2 * (uint64_t)M, p.r_pad) ||
         !sk_weight_maps(s, maps, 0, hw.w_gate, d, F, 8, p) || !sk_weight_maps(s, maps, 1, hw.w_up, d, F, 8, p))
         return note_err(c, cudaErrorInvalidValue, "tensor map (gate/up, few rows)");
     c->launches++;
-    return note_err(c, sk_launch_rp<SK_GU>(maps, p, G, st, pdl, false), "gate/up kernel (few rows)");
+    return note_err(c, sk_launch_rp<SK_GU>(maps, p, grid, st, pdl, false), "gate/up kernel (few rows)");
 }
 
-cudaError_t sk_down(Ctx *c, int k, int M, int K, const mrp_draft_out &out, cudaStream_t st, bool pdl)
+cudaError_t sk_down(Ctx *c, int k, int M, int K, const mrp_draft_out &out, cudaStream_t st, bool pdl, int *n_ss_out)
 {
     const TcState *s = (const TcState *)c->tc_state;
     const mrp_head_weights &hw = c->heads[k - 1];
     const int d = c->cfg.d, F = c->cfg.d_ff, G = c->sm_count;
     SkParams p;
     sk_common(c, p, M, K, out);
-    p.units_total = d / 16; p.k_chunks = F / kBK; p.r_pad = M <= 16 ? 16 : 32;
+    p.units_total = d / 16; p.k_chunks = F / kBK; p.r_pad = M <= 16 ? 16 : 32; p.w_rows = d;
     p.x_row_hi = 0; p.x_row_lo = M;
     p.hcur = (float *)(c->ws + c->lay.hcur); p.h0f = (const float *)(c->ws + c->lay.h0f);
     p.gamma_next = (k < K) ? (const __nv_bfloat16 *)c->heads[k].rms_gamma : nullptr;
@@ -539,14 +607,18 @@ cudaError_t sk_down(Ctx *c, int k, int M, int K, const mrp_draft_out &out, cudaS
     p.xt_k = (__nv_bfloat16 *)(c->ws + c->lay.xt) + (size_t)k * M * d;
     p.sumsq_out = (float *)(c->ws + c->lay.sumsq);
     p.hidden_out = (k == K) ? out.hidden_out : nullptr;
-    sk_finish_shape(p, G);
+    sk_finish_shape(p, 0);
+    const int n_tiles = (d + 127) / 128;
+    const int grid = sk_split(c, p, n_tiles);
+    *n_ss_out = n_tiles;
+    (void)G;
     SkMaps maps;
     memset(&maps, 0, sizeof(maps));
     if (!make_map(s, &maps.x, c->ws + c->lay.act, F, 2 * (uint64_t)M, p.r_pad) ||
         !sk_weight_maps(s, maps, 0, hw.w_down, F, d, 16, p))
         return note_err(c, cudaErrorInvalidValue, "tensor map (down, few rows)");
     c->launches++;
-    return note_err(c, sk_launch_rp<SK_DN>(maps, p, G, st, pdl, false), "down kernel (few rows)");
+    return note_err(c, sk_launch_rp<SK_DN>(maps, p, grid, st, pdl, false), "down kernel (few rows)");
 }
 
 cudaError_t sk_lm(Ctx *c, const float *logits0, const int32_t *row_index, int M, int K,
