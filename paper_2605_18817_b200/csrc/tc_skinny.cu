@@ -132,6 +132,7 @@ sk_gemm_kernel(const __grid_constant__ SkMaps maps, const SkParams p)
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         prefetch_tmap(&maps.x);
         prefetch_tmap(&maps.w[0]);
+        if (KIND == SK_GU) prefetch_tmap(&maps.w[3]);
     }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
@@ -338,7 +339,7 @@ sk_gemm_kernel(const __grid_constant__ SkMaps maps, const SkParams p)
                 const float *first = p.scratch + ((size_t)tile * p.n_split * RP) * 128;
 #pragma unroll
                 for (int j = 0; j < RP; ++j) a[j] = 0.f;
-#pragma unroll 1
+#pragma unroll 4
                 for (int sp = 0; sp < p.n_split; ++sp) {          // slice order: the sum does not depend on who is last
 #pragma unroll
                     for (int j = 0; j < RP; ++j)
