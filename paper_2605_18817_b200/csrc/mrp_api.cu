@@ -28,7 +28,7 @@ WorkspaceLayout workspace_layout(const mrp_config &cfg)
     if (l.n_slices_max < kSumsqSlices) l.n_slices_max = kSumsqSlices;   // one slice per CTA (tc family)
     l.partials = take((size_t)l.n_slices_max * steps * rows * sizeof(Partial));
     l.dense_row = take((size_t)cfg.max_seqs * (size_t)cfg.block_len * 4);
-    l.sk_scratch = take((size_t)kSkScratchCtas * 32 * 128 * 4);
+    l.sk_scratch = take((size_t)kSkScratchBytes);
     l.sk_counters = take((size_t)kSkMaxTiles * 4);
     l.has_f16 = cfg.dtype == MRP_BF16 && !(cfg.flags & (MRP_FLAG_FORCE_SIMT | MRP_FLAG_EXACT_OPERANDS)) &&
                 (long long)cfg.n_heads * cfg.max_rows >= kF16MinRowSteps && cfg.d % 64 == 0 &&

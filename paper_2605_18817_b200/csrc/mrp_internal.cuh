@@ -30,7 +30,7 @@ struct WorkspaceLayout {
     size_t sumsq;       // fp32 [kSumsqSlices, max_rows] per-CTA partial sums of squares
     size_t partials;    // Partial [n_slices_max, (n_heads+1)*max_rows]
     size_t dense_row;   // int32 [max_seqs*block_len] dense position -> masked row or -1
-    size_t sk_scratch;  // fp32 [CTAs][32][128] partial accumulators of the few-row head kernels
+    size_t sk_scratch;  // fp32 [CTAs][r_pad][128] partial accumulators of the few-row head kernels
     size_t sk_counters; // int32 [kSkMaxTiles] arrivals per weight tile (zero between launches)
     size_t w16;         // fp16 [V, d] copy of the LM head (0 bytes unless the fp16 LM path can run)
     size_t xt16;        // fp16 [n_heads*max_rows, d] rows h_k - h_0 for that path
@@ -41,7 +41,7 @@ struct WorkspaceLayout {
 
 constexpr int kSumsqSlices = 512;
 constexpr int kSkMaxTiles = 4096;     // weight tiles of a few-row head kernel
-constexpr int kSkScratchCtas = 1024;  // CTAs of a split few-row head kernel (>= SM count)
+constexpr int kSkScratchBytes = 192 * 128 * 128 * 4;   // partial accumulators of split few-row head kernels
 constexpr int kSimtSliceV = 128;      // vocabulary entries per SIMT LM-head slice
 constexpr int kSimtMaxBlocks = 592;   // SIMT LM-head grid cap (4 per SM)
 constexpr int kF16MinRowSteps = 129;  // fp16 LM-head operands from this many row-steps K*M on
@@ -123,10 +123,11 @@ cudaError_t tc_draft(Ctx *c, const void *hidden, const float *logits0, const int
                      int M, int K, const mrp_draft_out &out, cudaStream_t st);
 
 // Few-row variants (tc_skinny.cu): weight rows on the MMA M axis; rows <= 32.
-bool sk_rows_ok(int rows);
+bool sk_rows_ok(int rows);          // LM head: row-steps incl. step 0
+bool sk_head_rows_ok(int M);       // head chain: masked rows
 cudaError_t sk_gateup(Ctx *c, int k, int M, int K, int n_ss, const mrp_draft_out &out, cudaStream_t st, bool pdl);
 cudaError_t sk_down(Ctx *c, int k, int M, int K, const mrp_draft_out &out, cudaStream_t st, bool pdl,
-                    int *n_ss_out);
+                    int *n_ss_out, bool f16_lm);
 bool sk_heads_ok(const mrp_config &cfg);
 cudaError_t sk_lm(Ctx *c, const float *logits0, const int32_t *row_index, int M, int K,
                   const mrp_draft_out &out, cudaStream_t st, bool pdl);

@@ -528,14 +528,14 @@ cudaError_t tc_draft(Ctx *c, const void *hidden, const float *logits0, const int
 
     const bool pdl = !(c->cfg.flags & MRP_FLAG_NO_PDL);
     const bool f16_lm = c->use_f16_lm && K * M >= kF16MinRowSteps;
-    const bool few_rows = sk_rows_ok(M) && sk_heads_ok(c->cfg) && G <= kSkScratchCtas &&
+    const bool few_rows = sk_head_rows_ok(M) && sk_heads_ok(c->cfg) &&
                           !(c->cfg.flags & MRP_FLAG_ROW_MAJOR_ONLY);
     int n_ss = 1;
     for (int k = 1; k <= K; ++k) {
         if (few_rows) {
             e = sk_gateup(c, k, M, K, n_ss, out, st, pdl);
             if (e != cudaSuccess) return e;
-            e = sk_down(c, k, M, K, out, st, pdl, &n_ss);
+            e = sk_down(c, k, M, K, out, st, pdl, &n_ss, f16_lm);
             if (e != cudaSuccess) return e;
             continue;
         }

@@ -14,6 +14,7 @@
 // shorter tile fetched through a tensor map with a smaller box, so no weight byte is read twice.
 // A kernel launched with programmatic stream serialisation starts fetching its weights while
 // the previous kernel drains: only the activation fetches and the epilogue wait for it.
+#include <cuda_fp16.h>
 #include <string.h>
 
 #include "tc_common.cuh"
@@ -24,11 +25,11 @@ namespace {
 constexpr int kSkThreads = 192;
 constexpr int kWTile = 128 * 128;          // bytes of a 128-row weight tile of one k-chunk
 constexpr int kAuxBytes = 12288;           // epilogue scratch after the barriers
-constexpr int kAuxRstd = 0;                // float[32]
-constexpr int kAuxRowOff = 128;            // long long[32]
-constexpr int kAuxVote = 384;              // int: an epilogue warp gave up on a wait
-constexpr int kAuxSsq = 2560;              // float[4][32]
-constexpr int kAuxExch = 4096;             // float[32][64]
+constexpr int kAuxRstd = 0;                // float[128]
+constexpr int kAuxRowOff = 512;            // long long[32]
+constexpr int kAuxVote = 768;              // int: epilogue warps' common decision
+constexpr int kAuxSsq = 1024;              // float[4][128]
+constexpr int kAuxExch = 4096;             // float[16][64]
 
 enum { SK_GU = 0, SK_DN = 1, SK_LM = 2 };
 
@@ -67,6 +68,7 @@ struct SkParams {
     const __nv_bfloat16 *gamma_next;
     __nv_bfloat16 *xg_next;
     __nv_bfloat16 *xt_k;
+    __half *xt16_k;      // optional: the same rows rounded once to fp16 (fp16 LM-head mode)
     float *sumsq_out;
     float *hidden_out;
     int32_t *status;
@@ -246,62 +248,42 @@ sk_gemm_kernel(const __grid_constant__ SkMaps maps, const SkParams p)
         }
         epi_sync();
 
-        // per-thread running state
-        float st_mx[KIND == SK_LM ? RP : 1], st_sum[KIND == SK_LM ? RP : 1], st_sec[KIND == SK_LM ? RP : 1];
-        int st_idx[KIND == SK_LM ? RP : 1];
-        float ssq[KIND == SK_DN ? RP : 1];
-        if (KIND == SK_LM) {
+        if constexpr (KIND == SK_LM) {
+            // per-thread running statistics of every row-step
+            float st_mx[RP], st_sum[RP], st_sec[RP];
+            int st_idx[RP];
 #pragma unroll
             for (int s = 0; s < RP; ++s) { st_mx[s] = -INFINITY; st_sum[s] = 0.f; st_sec[s] = -INFINITY; st_idx[s] = INT_MAX; }
-        }
-        if (KIND == SK_DN) {
+            int acc = 0;
+            uint32_t acc_ph = 0;
+            bool ok = true;
+            for (int ti = 0; ti < n_tiles && ok; ++ti) {
+                const int ut = u0 + 8 * ti;
+                const int units_here = ti < n_full ? 8 : rem;
+                const int v = ut * 16 + t;
+                const bool valid = t < units_here * 16;
+                // What the tile's outputs are added to does not depend on the accumulator: fetch
+                // it (independent loads, all in flight together) before waiting for the MMAs.
+                float a[RP];
 #pragma unroll
-            for (int s = 0; s < RP; ++s) ssq[s] = 0.f;
-        }
-
-        int acc = 0;
-        uint32_t acc_ph = 0;
-        bool ok = true;
-        for (int ti = 0; ti < n_tiles && ok; ++ti) {
-            const int ut = u0 + 8 * ti;
-            const int units_here = ti < n_full ? 8 : rem;
-            float a[RP];
-            const int wrow = KIND == SK_GU ? ut * 8 + t : ut * 16 + t;     // weight row = output feature
-            const bool valid = KIND == SK_LM ? (t < units_here * 16)
-                                             : (KIND == SK_GU ? (t < 64 && wrow < p.w_rows) : (wrow < p.w_rows));
-            // LM: what the tile's outputs are added to does not depend on the accumulator: fetch
-            // it (independent loads, all in flight together) before waiting for the MMAs.
+                for (int j = 0; j < RP; ++j)
+                    a[j] = (valid && j < p.n_rs) ? __ldg(p.logits0 + rowoff_s[j] + v) : 0.f;
+                ok = __all_sync(0xffffffffu, mbar_wait(tfull_bar(acc), acc_ph, abort_flag, p));
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t tacc = lane_addr + (uint32_t)(acc * 2 * RP);
 #pragma unroll
-            for (int j = 0; j < RP; ++j) {
-                a[j] = 0.f;
-                if (KIND == SK_LM && valid && j < p.n_rs) a[j] = __ldg(p.logits0 + rowoff_s[j] + wrow);
-            }
-
-            ok = __all_sync(0xffffffffu, mbar_wait(tfull_bar(acc), acc_ph, abort_flag, p));
-            if (KIND != SK_LM) {
-                // the four warps meet at barriers below: they must leave the loop together
-                if (!ok && lane == 0) *vote_s = 1;
-                epi_sync();
-                ok = (*vote_s == 0);
-            }
-            if (!ok) break;
-            tc_fence_after();
-            const uint32_t tacc = lane_addr + (uint32_t)(acc * 2 * RP);
+                for (int c0 = 0; c0 < 2 * RP; c0 += 16) {          // products with the hi rows, then the lo rows
+                    float part[16];
+                    tmem_ld16(tacc + c0, part);
 #pragma unroll
-            for (int c0 = 0; c0 < 2 * RP; c0 += 16) {          // products with the hi rows, then the lo rows
-                float part[16];
-                tmem_ld16(tacc + c0, part);
-#pragma unroll
-                for (int j = 0; j < 16; ++j) a[(c0 + j) % RP] += part[j];
-            }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(tempty_bar(acc));
-            acc ^= 1;
-            if (acc == 0) acc_ph ^= 1u;
-
-            if (KIND == SK_LM) {
-                const int v = wrow;
+                    for (int j = 0; j < 16; ++j) a[(c0 + j) % RP] += part[j];
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(tempty_bar(acc));
+                acc ^= 1;
+                if (acc == 0) acc_ph ^= 1u;
                 if (valid) {
 #pragma unroll
                     for (int s = 0; s < RP; ++s) {
@@ -320,81 +302,7 @@ sk_gemm_kernel(const __grid_constant__ SkMaps maps, const SkParams p)
                         }
                     }
                 }
-                continue;
             }
-
-            // ---- GU / DN: sum the slices of the contraction ----
-            if (p.n_split > 1) {
-                const int tile = cta / p.n_split, split = cta % p.n_split;
-                float *mine = p.scratch + ((size_t)cta * RP) * 128;
-#pragma unroll
-                for (int j = 0; j < RP; ++j)
-                    if (j < p.M) mine[j * 128 + t] = a[j];
-                __threadfence();
-                epi_sync();
-                if (t == 0) *vote_s = (atomicAdd(p.counters + tile, 1) == p.n_split - 1) ? 2 : 0;
-                epi_sync();
-                if (*vote_s != 2) break;          // another CTA of this tile finishes the job
-                __threadfence();
-                const float *first = p.scratch + ((size_t)tile * p.n_split * RP) * 128;
-#pragma unroll
-                for (int j = 0; j < RP; ++j) a[j] = 0.f;
-#pragma unroll 4
-                for (int sp = 0; sp < p.n_split; ++sp) {          // slice order: the sum does not depend on who is last
-#pragma unroll
-                    for (int j = 0; j < RP; ++j)
-                        if (j < p.M) a[j] += __ldcg(first + ((size_t)sp * RP + j) * 128 + t);
-                }
-                if (t == 0) p.counters[tile] = 0;
-                (void)split;
-            }
-
-            if (KIND == SK_GU) {
-                // lanes 0-63 hold gate rows, 64-127 the matching up rows: hand the up values over
-                if (t >= 64) {
-#pragma unroll
-                    for (int m = 0; m < RP; ++m)
-                        if (m < p.M) exch_s[m * 64 + (t - 64)] = a[m] * rstd_s[m];
-                }
-                epi_sync();
-                if (valid) {
-#pragma unroll
-                    for (int m = 0; m < RP; ++m) {
-                        if (m < p.M) {
-                            const float g = a[m] * rstd_s[m];
-                            const float av = g / (1.f + __expf(-g)) * exch_s[m * 64 + t];
-                            store_hi_lo(p.act + (size_t)m * p.F + wrow, (size_t)p.M * p.F, av);
-                        }
-                    }
-                }
-            } else if (valid) {
-                float hc[RP], h0v[RP];
-#pragma unroll
-                for (int m = 0; m < RP; ++m) {
-                    hc[m] = 0.f; h0v[m] = 0.f;
-                    if (m < p.M) {
-                        hc[m] = p.hcur[(size_t)m * p.d + wrow];
-                        h0v[m] = __ldg(p.h0f + (size_t)m * p.d + wrow);
-                    }
-                }
-                const float gm = p.xg_next ? __bfloat162float(p.gamma_next[wrow]) : 0.f;
-#pragma unroll
-                for (int m = 0; m < RP; ++m) {
-                    if (m < p.M) {
-                        const size_t o = (size_t)m * p.d + wrow;
-                        const float h = hc[m] + a[m];
-                        p.hcur[o] = h;
-                        if (p.hidden_out) p.hidden_out[o] = h;
-                        ssq[m] = fmaf(h, h, ssq[m]);
-                        store_hi_lo(p.xt_k + o, (size_t)p.n_rs * p.d, h - h0v[m]);
-                        if (p.xg_next) store_hi_lo(p.xg_next + o, (size_t)p.M * p.d, h * gm);
-                    }
-                }
-            }
-        }
-
-        // ---- per-CTA results ----
-        if (KIND == SK_LM) {
             // Every thread parks its row-step statistics in the (now idle) ring memory; the merge
             // over the 128 threads is then a short loop instead of unrolled straight-line code,
             // which would be fetched once, instruction line by line, from a saturated memory system.
@@ -432,21 +340,132 @@ sk_gemm_kernel(const __grid_constant__ SkMaps maps, const SkParams p)
                     if (lane == 0) p.partials[(size_t)cta * p.n_rs + s] = pr;
                 }
             }
-        } else if (KIND == SK_DN) {
+        } else {
+            // GU / DN: one weight tile per CTA; activation columns are handled 16 at a time
+            const int wrow = KIND == SK_GU ? u0 * 8 + t : u0 * 16 + t;     // weight row = output feature
+            const bool valid = KIND == SK_GU ? (t < 64 && wrow < p.w_rows) : (wrow < p.w_rows);
+            const int n_ch = (p.M + 15) >> 4;
+            const int tile = cta / p.n_split;
+            bool ok = __all_sync(0xffffffffu, mbar_wait(tfull_bar(0), 0u, abort_flag, p));
+            // the four warps meet at barriers below: they must agree on going on
+            if (!ok && lane == 0) *vote_s = 1;
+            epi_sync();
+            ok = (*vote_s == 0);
+            bool finisher = ok;
+            if (ok) tc_fence_after();
+            if (ok && p.n_split > 1) {
+                // park this slice's partial sums; the last CTA of the tile to arrive adds the slices
+                float *mine = p.scratch + ((size_t)cta * RP) * 128;
+#pragma unroll 1
+                for (int ch = 0; ch < n_ch; ++ch) {
+                    float v[16], w[16];
+                    tmem_ld16(lane_addr + ch * 16, v);
+                    tmem_ld16(lane_addr + RP + ch * 16, w);
 #pragma unroll
-            for (int m = 0; m < RP; ++m) {
-                if (m < p.M) {
-                    float v = ssq[m];
-#pragma unroll
-                    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-                    if (lane == 0) ssq_s[q * 32 + m] = v;
+                    for (int j = 0; j < 16; ++j)
+                        if (ch * 16 + j < p.M) mine[(ch * 16 + j) * 128 + t] = v[j] + w[j];
+                }
+                __threadfence();
+                epi_sync();
+                if (t == 0) *vote_s = (atomicAdd(p.counters + tile, 1) == p.n_split - 1) ? 2 : 0;
+                epi_sync();
+                finisher = (*vote_s == 2);
+                if (finisher) {
+                    __threadfence();
+                    if (t == 0) p.counters[tile] = 0;
                 }
             }
-            epi_sync();
-            // one slice of sums of squares per weight tile, written by the CTA that finished it
-            const bool finisher = p.n_split == 1 || *vote_s == 2;
-            if (ok && finisher && t < p.M)
-                p.sumsq_out[(size_t)(cta / p.n_split) * p.M + t] = (ssq_s[t] + ssq_s[32 + t]) + (ssq_s[64 + t] + ssq_s[96 + t]);
+            if (finisher) {
+                const float *first = p.scratch + ((size_t)tile * p.n_split * RP) * 128;
+                const float gm = (KIND == SK_DN && valid && p.xg_next) ? __bfloat162float(p.gamma_next[wrow]) : 0.f;
+#pragma unroll 1
+                for (int ch = 0; ch < n_ch; ++ch) {
+                    const int c0 = ch * 16;
+                    float v[16];
+                    float hc[16], h0v[16];          // DN: what the outputs are added to, fetched first
+                    if (KIND == SK_DN) {
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            hc[j] = 0.f; h0v[j] = 0.f;
+                            if (valid && c0 + j < p.M) {
+                                hc[j] = p.hcur[(size_t)(c0 + j) * p.d + wrow];
+                                h0v[j] = __ldg(p.h0f + (size_t)(c0 + j) * p.d + wrow);
+                            }
+                        }
+                    }
+                    if (p.n_split > 1) {
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) v[j] = 0.f;
+#pragma unroll 4
+                        for (int sp = 0; sp < p.n_split; ++sp) {   // slice order: the sum does not depend on who is last
+#pragma unroll
+                            for (int j = 0; j < 16; ++j)
+                                if (c0 + j < p.M) v[j] += __ldcg(first + ((size_t)sp * RP + c0 + j) * 128 + t);
+                        }
+                    } else {
+                        float w[16];
+                        tmem_ld16(lane_addr + c0, v);
+                        tmem_ld16(lane_addr + RP + c0, w);
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) v[j] += w[j];
+                    }
+                    if (KIND == SK_GU) {
+                        // lanes 0-63 hold gate rows, 64-127 the matching up rows: hand the up values over
+                        if (t >= 64) {
+#pragma unroll
+                            for (int j = 0; j < 16; ++j)
+                                if (c0 + j < p.M) exch_s[j * 64 + (t - 64)] = v[j] * rstd_s[c0 + j];
+                        }
+                        epi_sync();
+                        if (valid) {
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) {
+                                if (c0 + j < p.M) {
+                                    const float g = v[j] * rstd_s[c0 + j];
+                                    const float av = g / (1.f + __expf(-g)) * exch_s[j * 64 + t];
+                                    store_hi_lo(p.act + (size_t)(c0 + j) * p.F + wrow, (size_t)p.M * p.F, av);
+                                }
+                            }
+                        }
+                        epi_sync();
+                    } else {
+                        float sq[16];
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) sq[j] = 0.f;
+                        if (valid) {
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) {
+                                if (c0 + j < p.M) {
+                                    const size_t o = (size_t)(c0 + j) * p.d + wrow;
+                                    const float h = hc[j] + v[j];
+                                    p.hcur[o] = h;
+                                    if (p.hidden_out) p.hidden_out[o] = h;
+                                    sq[j] = h * h;
+                                    store_hi_lo(p.xt_k + o, (size_t)p.n_rs * p.d, h - h0v[j]);
+                                    if (p.xt16_k) p.xt16_k[o] = __float2half_rn(h - h0v[j]);
+                                    if (p.xg_next) store_hi_lo(p.xg_next + o, (size_t)p.M * p.d, h * gm);
+                                }
+                            }
+                        }
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            float s = sq[j];
+#pragma unroll
+                            for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+                            if (lane == 0) ssq_s[q * 128 + c0 + j] = s;
+                        }
+                    }
+                }
+            }
+            if (KIND == SK_DN) {
+                epi_sync();
+                // one slice of sums of squares per weight tile, written by the CTA that finished it
+                if (finisher) {
+                    for (int m = t; m < p.M; m += 128)
+                        p.sumsq_out[(size_t)tile * p.M + m] =
+                            (ssq_s[m] + ssq_s[128 + m]) + (ssq_s[256 + m] + ssq_s[384 + m]);
+                }
+            }
         }
     }
 
@@ -501,6 +520,7 @@ int sk_split(Ctx *c, SkParams &p, int n_tiles)
     if (S > p.k_chunks) S = p.k_chunks;
     const int cps = (p.k_chunks + S - 1) / S;
     S = (p.k_chunks + cps - 1) / cps;          // no empty slice
+    if ((size_t)n_tiles * S * p.r_pad * 128 * 4 > (size_t)kSkScratchBytes) S = 1;
     p.n_split = S;
     p.scratch = (float *)(c->ws + c->lay.sk_scratch);
     p.counters = (int32_t *)(c->ws + c->lay.sk_counters);
@@ -547,14 +567,20 @@ template <int KIND>
 cudaError_t sk_launch_rp(const SkMaps &maps, const SkParams &p, int grid, cudaStream_t st, bool pdl, bool margin)
 {
     if constexpr (KIND != SK_LM) {
-        return p.r_pad == 16 ? sk_launch<KIND, 16, false>(maps, p, grid, st, pdl)
-                             : sk_launch<KIND, 32, false>(maps, p, grid, st, pdl);
+        switch (p.r_pad) {
+        case 16: return sk_launch<KIND, 16, false>(maps, p, grid, st, pdl);
+        case 32: return sk_launch<KIND, 32, false>(maps, p, grid, st, pdl);
+        case 64: return sk_launch<KIND, 64, false>(maps, p, grid, st, pdl);
+        default: return sk_launch<KIND, 128, false>(maps, p, grid, st, pdl);
+        }
     } else {
         if (p.r_pad == 16)
             return margin ? sk_launch<KIND, 16, true>(maps, p, grid, st, pdl) : sk_launch<KIND, 16, false>(maps, p, grid, st, pdl);
         return margin ? sk_launch<KIND, 32, true>(maps, p, grid, st, pdl) : sk_launch<KIND, 32, false>(maps, p, grid, st, pdl);
     }
 }
+
+int sk_head_pad(int M) { return M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : 128; }
 
 void sk_common(Ctx *c, SkParams &p, int M, int K, const mrp_draft_out &out)
 {
@@ -568,6 +594,10 @@ void sk_common(Ctx *c, SkParams &p, int M, int K, const mrp_draft_out &out)
 
 bool sk_rows_ok(int rows) { return rows >= 1 && rows <= 32; }
 
+// Above 64 rows the per-CTA re-read of the activation tile and the serial 16-column epilogue
+// cost more than the row-major kernels' narrow weight tiles (measured at M = 128).
+bool sk_head_rows_ok(int M) { return M >= 1 && M <= 64; }
+
 bool sk_heads_ok(const mrp_config &cfg) { return (cfg.d + 127) / 128 <= kSumsqSlices && cfg.d_ff / 64 <= kSkMaxTiles; }
 
 cudaError_t sk_gateup(Ctx *c, int k, int M, int K, int n_ss, const mrp_draft_out &out, cudaStream_t st, bool pdl)
@@ -577,7 +607,7 @@ cudaError_t sk_gateup(Ctx *c, int k, int M, int K, int n_ss, const mrp_draft_out
     const int d = c->cfg.d, F = c->cfg.d_ff, G = c->sm_count;
     SkParams p;
     sk_common(c, p, M, K, out);
-    p.units_total = F / 8; p.k_chunks = d / kBK; p.r_pad = M <= 16 ? 16 : 32; p.w_rows = F;
+    p.units_total = F / 8; p.k_chunks = d / kBK; p.r_pad = sk_head_pad(M); p.w_rows = F;
     p.x_row_hi = 0; p.x_row_lo = M;
     p.sumsq = (const float *)(c->ws + c->lay.sumsq); p.n_ss = n_ss; p.eps = c->cfg.rms_eps;
     p.act = (__nv_bfloat16 *)(c->ws + c->lay.act);
@@ -593,19 +623,21 @@ cudaError_t sk_gateup(Ctx *c, int k, int M, int K, int n_ss, const mrp_draft_out
     return note_err(c, sk_launch_rp<SK_GU>(maps, p, grid, st, pdl, false), "gate/up kernel (few rows)");
 }
 
-cudaError_t sk_down(Ctx *c, int k, int M, int K, const mrp_draft_out &out, cudaStream_t st, bool pdl, int *n_ss_out)
+cudaError_t sk_down(Ctx *c, int k, int M, int K, const mrp_draft_out &out, cudaStream_t st, bool pdl, int *n_ss_out,
+                    bool f16_lm)
 {
     const TcState *s = (const TcState *)c->tc_state;
     const mrp_head_weights &hw = c->heads[k - 1];
     const int d = c->cfg.d, F = c->cfg.d_ff, G = c->sm_count;
     SkParams p;
     sk_common(c, p, M, K, out);
-    p.units_total = d / 16; p.k_chunks = F / kBK; p.r_pad = M <= 16 ? 16 : 32; p.w_rows = d;
+    p.units_total = d / 16; p.k_chunks = F / kBK; p.r_pad = sk_head_pad(M); p.w_rows = d;
     p.x_row_hi = 0; p.x_row_lo = M;
     p.hcur = (float *)(c->ws + c->lay.hcur); p.h0f = (const float *)(c->ws + c->lay.h0f);
     p.gamma_next = (k < K) ? (const __nv_bfloat16 *)c->heads[k].rms_gamma : nullptr;
     p.xg_next = (k < K) ? (__nv_bfloat16 *)(c->ws + c->lay.xg) : nullptr;
     p.xt_k = (__nv_bfloat16 *)(c->ws + c->lay.xt) + (size_t)k * M * d;
+    p.xt16_k = f16_lm ? (__half *)(c->ws + c->lay.xt16) + (size_t)(k - 1) * M * d : nullptr;
     p.sumsq_out = (float *)(c->ws + c->lay.sumsq);
     p.hidden_out = (k == K) ? out.hidden_out : nullptr;
     sk_finish_shape(p, 0);
