@@ -46,7 +46,7 @@ struct SkParams {
     int r_pad;           // activation rows per part (16 or 32); MMA N = 2 * r_pad
     int tmem_cols;       // allocated TMEM columns (power of two >= 2 buffers * 2 * r_pad)
     int x_row_hi, x_row_lo;
-    int tail_units[2];   // units of short-tile kinds 1 and 2 (LM)
+    int lm_h[4];         // LM: tile heights (units) other than 8, fetched through maps w[1], w[2], w[4], w[5]
     int n_split;         // GU/DN: CTAs sharing one 128-row weight tile, each a slice of the contraction
     int w_rows;          // GU/DN: weight rows (gate rows for GU)
     float *scratch;      // GU/DN: partial accumulators [tile][split][RP][128]
@@ -123,9 +123,17 @@ sk_gemm_kernel(const __grid_constant__ SkMaps maps, const SkParams p)
         kc1 = min(p.k_chunks, kc0 + cps);
     }
     const int nk = kc1 - kc0;
-    const int n_full = units >> 3, rem = units & 7;
-    const int n_tiles = n_full + (rem ? 1 : 0);
-    const int tail_kind = (rem == p.tail_units[0]) ? 1 : 2;
+    // The range is cut into the fewest tiles of at most 8 units and the tiles are made equally
+    // high (an MMA costs the same at any height, so a short extra tile would cost a full one):
+    // the first t_extra tiles have t_base + 1 units, the others t_base.
+    const int n_tiles = (units + 7) >> 3;
+    const int t_base = n_tiles ? units / n_tiles : 0, t_extra = n_tiles ? units % n_tiles : 0;
+    auto tile_units = [&](int ti) { return t_base + (ti < t_extra ? 1 : 0); };
+    auto tile_start = [&](int ti) { return u0 + ti * t_base + min(ti, t_extra); };
+    auto tile_map = [&](int h) {
+        if (h == 8) return 0;
+        return h == p.lm_h[0] ? 1 : h == p.lm_h[1] ? 2 : h == p.lm_h[2] ? 4 : 5;
+    };
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.n_stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
@@ -154,16 +162,14 @@ sk_gemm_kernel(const __grid_constant__ SkMaps maps, const SkParams p)
             const int pre = min(p.n_stages, total_it);
             auto load_w = [&](int t, int kk, int s) {
                 const uint32_t sw = base + (uint32_t)s * stage_bytes;
-                const bool is_full = t < n_full;
-                const int kind = is_full ? 0 : tail_kind;
-                const uint32_t w_bytes = is_full ? (uint32_t)kWTile : (uint32_t)rem * 2048u;
-                mbar_expect_tx(full_bar(s), w_bytes + (uint32_t)x_bytes);
-                const int ut = u0 + 8 * t;
+                const int h = tile_units(t);
+                mbar_expect_tx(full_bar(s), (uint32_t)h * 2048u + (uint32_t)x_bytes);
+                const int ut = tile_start(t);
                 if (KIND == SK_GU) {
-                    tma_load_2d(sw, &maps.w[kind], (kc0 + kk) * kBK, ut * 8, full_bar(s));
-                    tma_load_2d(sw + 64 * 128, &maps.w[3 + kind], (kc0 + kk) * kBK, ut * 8, full_bar(s));
+                    tma_load_2d(sw, &maps.w[0], (kc0 + kk) * kBK, ut * 8, full_bar(s));
+                    tma_load_2d(sw + 64 * 128, &maps.w[3], (kc0 + kk) * kBK, ut * 8, full_bar(s));
                 } else {
-                    tma_load_2d(sw, &maps.w[kind], (kc0 + kk) * kBK, ut * 16, full_bar(s));
+                    tma_load_2d(sw, &maps.w[tile_map(h)], (kc0 + kk) * kBK, ut * 16, full_bar(s));
                 }
             };
             auto load_x = [&](int kk, int s) {
@@ -258,8 +264,8 @@ sk_gemm_kernel(const __grid_constant__ SkMaps maps, const SkParams p)
             uint32_t acc_ph = 0;
             bool ok = true;
             for (int ti = 0; ti < n_tiles && ok; ++ti) {
-                const int ut = u0 + 8 * ti;
-                const int units_here = ti < n_full ? 8 : rem;
+                const int ut = tile_start(ti);
+                const int units_here = tile_units(ti);
                 const int v = ut * 16 + t;
                 const bool valid = t < units_here * 16;
                 // What the tile's outputs are added to does not depend on the accumulator: fetch
@@ -504,11 +510,18 @@ void sk_finish_shape(SkParams &p, int grid)
     while (cols < 2 * 2 * p.r_pad) cols <<= 1;
     p.tmem_cols = cols;
     p.n_split = 1;
-    p.tail_units[0] = p.tail_units[1] = 0;
-    if (grid > 0) {           // LM: contiguous unit ranges, short tiles of two possible heights
-        const int u_base = p.units_total / grid;
-        p.tail_units[0] = u_base % 8;
-        p.tail_units[1] = (u_base + 1) % 8;
+    for (int i = 0; i < 4; ++i) p.lm_h[i] = 0;
+    if (grid > 0) {           // LM: contiguous unit ranges of u_base or u_base + 1 units, equal-height tiles
+        int n = 0;
+        for (int units = p.units_total / grid; units <= p.units_total / grid + 1; ++units) {
+            const int nt = (units + 7) / 8;
+            if (nt == 0) continue;
+            for (int h = units / nt; h <= units / nt + (units % nt ? 1 : 0); ++h) {
+                bool seen = (h == 8 || h == 0);
+                for (int i = 0; i < n; ++i) seen |= (p.lm_h[i] == h);
+                if (!seen) p.lm_h[n++] = h;
+            }
+        }
     }
 }
 
@@ -527,15 +540,14 @@ int sk_split(Ctx *c, SkParams &p, int n_tiles)
     return n_tiles * S;
 }
 
-// Tensor maps of one weight matrix part: full tiles and the two short-tile heights.
+// Tensor maps of one weight matrix part: full tiles, and for the LM head the other tile heights.
 bool sk_weight_maps(const TcState *s, SkMaps &maps, int part, const void *w, uint64_t inner, uint64_t rows,
                     int unit_rows, const SkParams &p)
 {
     if (!make_map(s, &maps.w[part * 3], w, inner, rows, 8 * unit_rows)) return false;
-    for (int k = 0; k < 2; ++k)
-        if (p.tail_units[k] > 0 &&
-            !make_map(s, &maps.w[part * 3 + 1 + k], w, inner, rows, p.tail_units[k] * unit_rows))
-            return false;
+    static const int slot[4] = {1, 2, 4, 5};
+    for (int k = 0; k < 4 && part == 0; ++k)
+        if (p.lm_h[k] > 0 && !make_map(s, &maps.w[slot[k]], w, inner, rows, p.lm_h[k] * unit_rows)) return false;
     return true;
 }
 
