@@ -136,7 +136,7 @@ def _rand_select_case(rng, K, B, L, mask_prob):
 def select_ctx():
     w = synth.make_weights(16, 16, 32, 0, "f32", 1)
     heads, w_lm = harness.upload_weights(w, DEV)
-    ctx = binding.mrp_create(16, 16, 32, heads, w_lm, max_rows=64 * 100, max_seqs=64, block_len=100)
+    ctx = binding.mrp_create(16, 16, 32, heads, w_lm, max_rows=4, max_seqs=64, block_len=1024)
     yield ctx
     binding.mrp_destroy(ctx)
 
@@ -162,7 +162,7 @@ def _assert_select_equal(g, o):
         assert np.array_equal(a.reshape(b.shape), b), name
 
 
-@pytest.mark.parametrize("L", [1, 4, 16, 32, 33, 100])
+@pytest.mark.parametrize("L", [1, 4, 16, 32, 33, 100, 1024])
 def test_select_bit_exact_on_shared_statistics(select_ctx, L):
     rng = np.random.default_rng(L)
     for case in range(6):
@@ -271,3 +271,26 @@ def test_tensor_core_family_small_shapes(d, F, V, B, L, K):
     # the row-major kernels alone, fully serialised launches: same results within tolerance
     out4, _ = run_gpu_draft(w, inp, K, flags=binding.MRP_FLAG_ROW_MAJOR_ONLY | binding.MRP_FLAG_NO_PDL)
     check_stats(out4, ref, "bf16")
+
+
+@pytest.mark.parametrize("flags", [0, binding.MRP_FLAG_FORCE_SIMT])
+def test_non_finite_logits_raise_the_status_bit_and_leave_the_context_usable(flags):
+    w = synth.make_weights(128, 256, 2048, 2, "bf16", 5, head_std=0.05)
+    inp = synth.make_inputs(w, 2, 4, 5, 1.0, 4.0)
+    heads, w_lm = harness.upload_weights(w, DEV)
+    ctx = binding.mrp_create(w.d, w.F, w.V, heads, w_lm, max_rows=8, max_seqs=2, block_len=4, flags=flags)
+    hid = harness.to_device(inp.hidden, w.dtype, DEV)
+    l0 = torch.from_numpy(inp.logits0).to(DEV)
+    bad = l0.clone()
+    bad[3, 100] = float("inf")
+    out = harness.alloc_draft_out(8, 2, w.V, w.d, DEV)
+    harness.draft(ctx, hid, bad, None, 8, 2, out)
+    torch.cuda.synchronize()
+    assert int(out.status.item()) & binding.MRP_DEV_NONFINITE
+    good = harness.alloc_draft_out(8, 2, w.V, w.d, DEV)
+    harness.draft(ctx, hid, l0, None, 8, 2, good)
+    torch.cuda.synchronize()
+    assert int(good.status.item()) == 0
+    ref = oracle.draft(inp.hidden, inp.logits0, w.heads, w.w_lm, K=2)
+    check_stats(good, ref, "bf16")
+    binding.mrp_destroy(ctx)
