@@ -226,8 +226,10 @@ def run_reference(args, cfg):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
-        "data": "synthetic", "config": {"workload": cfg["name"], "rows": M, "chain": K,
-                                         "d": cfg["d"], "vocab": cfg["V"]},
+        "data": "synthetic",
+        "config": {"workload": cfg["name"], "rows": M, "chain": K, "d": cfg["d"], "d_ff": cfg["F"],
+                   "vocab": cfg["V"], "seqs": cfg["B"], "block_len": L, "mode": cfg["mode"],
+                   "l2": "host cores (oracle)", "parallelism": "rank 0 only"},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(),
                          "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},

@@ -1,19 +1,23 @@
-// Tensor-core kernel family (sm_100a): tcgen05.mma with TMEM accumulators, operands staged in
-// shared memory by TMA (128-byte swizzle), warp-specialised: one TMA producer thread, one MMA
-// issuer thread, four epilogue warps that read the accumulators back with tcgen05.ld.
+// Tensor-core kernel family, row-major form (sm_100a): tcgen05.mma with TMEM accumulators, operands
+// staged in shared memory by TMA (128-byte swizzle), warp-specialised: one TMA producer thread,
+// one MMA issuer thread, four epilogue warps that read the accumulators back with tcgen05.ld.
+// Used where there are many activation rows; tc_skinny.cu holds the few-row form.
 //
 // All three GEMMs of the drafting pass share one main loop and differ in the epilogue:
 //   GU  gate/up projections of a head:  act = silu(rstd * Wg x) * (rstd * Wu x)          (a1)
-//   DN  down projection:  h <- h + Wd act, emits the bf16 operands of the next GEMMs      (a1)
-//   LM  shared LM head on the stacked residual rows h_k - h_0, fused with "+ l_0" and the
-//       online softmax statistics (max, sum of exponentials, argmax, runner-up)      (a2, a3)
-// Precision: weights are exact bf16; every activation operand (head input, SwiGLU output, stacked
-// residual rows) is carried as a pair of bf16 matrices hi + lo (lo = bf16 of what hi lost), and
-// each weight tile is multiplied by both, so the products are exact to about 2^-17 and the
-// fp32 accumulators stay within the 2e-3 tolerance on confidence / log-sum-exp.
+//   DN  down projection:  h <- h + Wd act, emits the operands of the next GEMMs           (a1)
+//   LM  shared LM head on the stacked residual rows h_k - h_0 of steps 1..K, fused with
+//       "+ l_0" and the online softmax statistics (max, sum of exponentials, argmax,
+//       runner-up); the statistics of step 0 ride on the rows of step 1               (a2, a3)
+// Precision: weights are exact bf16.  Activation operands are a pair of bf16 matrices hi + lo
+// (lo = bf16 of what hi lost), both multiplied by every weight tile into one accumulator, so the
+// products are exact to about 2^-17.  The LM head above 128 row-steps instead takes its operand
+// rounded once to fp16 against an fp16 copy of W_lm (one MMA pass; the combine then recomputes
+// each row-step's top logit exactly).
 // Orientation: activation rows are the MMA M dimension (128 TMEM lanes, one row per epilogue
-// thread), weight rows are the MMA N dimension.  Every CTA owns a contiguous range of weight
-// rows, split into equal tiles, and streams it exactly once per 128-row activation block.
+// thread), weight rows the MMA N dimension.  A CTA is a (weight-row range, group of 128-row
+// activation blocks) pair: it streams its range once per block of its group, and CTAs of the
+// same range share those reads through L2.
 #include <cuda_fp16.h>
 #include <string.h>
 

@@ -10,8 +10,10 @@
 // Each activation operand is a bf16 hi block followed by a bf16 lo block; a stage holds both as
 // one B tile of N = 2 * RP rows, so one MMA per k-step yields the products with hi in columns
 // [0, RP) and with lo in [RP, 2 RP) of the accumulator; the epilogue adds the two.
-// Every CTA owns a contiguous range of 16-row weight units: full 128-row tiles, then one
-// shorter tile fetched through a tensor map with a smaller box, so no weight byte is read twice.
+// LM: every CTA owns a contiguous range of 16-row vocabulary units, cut into the fewest tiles of
+// at most 128 rows, all (nearly) equally high; each height has its own tensor map (TMA box), so
+// no weight byte is read twice.  GU / DN: one full 128-row weight tile per CTA and a slice of the
+// contraction; the slices of a tile are added, in slice order, by the last of its CTAs to arrive.
 // A kernel launched with programmatic stream serialisation starts fetching its weights while
 // the previous kernel drains: only the activation fetches and the epilogue wait for it.
 #include <cuda_fp16.h>
