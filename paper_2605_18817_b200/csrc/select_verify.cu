@@ -58,10 +58,25 @@ __device__ __forceinline__ int warp_popc(uint32_t bits)
 __global__ void __launch_bounds__(32)
 select_kernel(const float *__restrict__ conf, const int32_t *__restrict__ token,
               const int32_t *__restrict__ dense_row, int M, int K, int L, mrp_select_params p,
-              mrp_select_out out, int Kd)
+              mrp_select_out out, int Kd, const int32_t *__restrict__ row_index)
 {
     const int b = blockIdx.x, lane = threadIdx.x;
-    const int32_t *rows = dense_row + (size_t)b * L;
+    // Position -> masked row of this block: from the prepared dense map, or (dense_row == NULL,
+    // few masked rows) built here in shared memory by one scan over the row list.
+    __shared__ int32_t rows_s[1024];
+    const int32_t *rows = rows_s;
+    if (dense_row) {
+        rows = dense_row + (size_t)b * L;
+    } else {
+        for (int i = lane; i < L; i += 32) rows_s[i] = -1;
+        __syncwarp();
+        const long long lo = (long long)b * L;
+        for (int m = lane; m < M; m += 32) {
+            const long long idx = row_index ? row_index[m] : m;
+            if (idx >= lo && idx < lo + L) rows_s[idx - lo] = m;
+        }
+        __syncwarp();
+    }
     int8_t *reveal = out.reveal_mask + (size_t)b * L, *remask = out.remask_mask + (size_t)b * L;
     int32_t *otok = out.out_token + (size_t)b * L;
     int8_t *step = out.step_of + (size_t)b * L;
@@ -183,6 +198,13 @@ cudaError_t launch_select(Ctx *c, const float *conf, const int32_t *token, const
                           int M, int K, int B, int L, const mrp_select_params &p,
                           const mrp_select_out &out, cudaStream_t st)
 {
+    const int Kd = K * (p.r_draft > 0 ? p.r_draft : 0);
+    if ((long long)B * M <= (1ll << 22)) {
+        // few rows: every block finds its rows itself, one launch instead of three
+        select_kernel<<<B, 32, 0, st>>>(conf, token, nullptr, M, K, L, p, out, Kd, row_index);
+        c->launches++;
+        return cudaGetLastError();
+    }
     int32_t *dense_row = (int32_t *)(c->ws + c->lay.dense_row);
     cudaError_t e = cudaMemsetAsync(dense_row, 0xFF, sizeof(int32_t) * (size_t)B * L, st);
     if (e != cudaSuccess) return e;
@@ -190,8 +212,7 @@ cudaError_t launch_select(Ctx *c, const float *conf, const int32_t *token, const
         scatter_rows_kernel<<<(M + 255) / 256, 256, 0, st>>>(row_index, M, dense_row);
         c->launches++;
     }
-    const int Kd = K * (p.r_draft > 0 ? p.r_draft : 0);
-    select_kernel<<<B, 32, 0, st>>>(conf, token, dense_row, M, K, L, p, out, Kd);
+    select_kernel<<<B, 32, 0, st>>>(conf, token, dense_row, M, K, L, p, out, Kd, nullptr);
     c->launches++;
     return cudaGetLastError();
 }
@@ -268,6 +289,6 @@ extern "C" int mrp_reveal_remask_noalloc(const float *conf, const int32_t *token
     if (cudaMemsetAsync(dense_row, 0xFF, sizeof(int32_t) * (size_t)B * L, st) != cudaSuccess)
         return MRP_ERR_CUDA;
     if (M > 0) scatter_rows_kernel<<<(M + 255) / 256, 256, 0, st>>>(row_index, M, dense_row);
-    select_kernel<<<B, 32, 0, st>>>(conf, token, dense_row, M, K, L, *params, *out, Kd);
+    select_kernel<<<B, 32, 0, st>>>(conf, token, dense_row, M, K, L, *params, *out, Kd, nullptr);
     return cudaGetLastError() == cudaSuccess ? MRP_OK : MRP_ERR_CUDA;
 }

@@ -612,7 +612,7 @@ bool sk_rows_ok(int rows) { return rows >= 1 && rows <= 32; }
 // cost more than the row-major kernels' narrow weight tiles (measured at M = 128).
 bool sk_head_rows_ok(int M) { return M >= 1 && M <= 64; }
 
-bool sk_heads_ok(const mrp_config &cfg) { return (cfg.d + 127) / 128 <= kSumsqSlices && cfg.d_ff / 64 <= kSkMaxTiles; }
+bool sk_heads_ok(const mrp_config &cfg) { return (cfg.d + 127) / 128 <= kSumsqSlices && cfg.d_ff / 64 < kSkMaxTiles; }
 
 cudaError_t sk_gateup(Ctx *c, int k, int M, int K, int n_ss, const mrp_draft_out &out, cudaStream_t st, bool pdl)
 {
