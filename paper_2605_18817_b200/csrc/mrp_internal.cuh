@@ -83,6 +83,30 @@ inline void prof_mark(Ctx *c, int mark, cudaStream_t st)
     if (mark == kProfMarks - 1) c->prof_calls++;
 }
 
+// Programmatic dependent launch.  A kernel that calls pdl_wait() before it touches anything an
+// earlier kernel of the stream wrote may be launched with launch_k(..., pdl = true): it is then
+// scheduled while its predecessor drains instead of after it.  pdl_trigger() lets the kernel's
+// own successor do the same.  Launched without the attribute both calls do nothing.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                            bool pdl, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 // ---- CUDA-core kernel family (simt_kernels.cu) -------------------------------------
 cudaError_t simt_draft(Ctx *c, const void *hidden, const float *logits0, const int32_t *row_index,
                        int M, int K, const mrp_draft_out &out, cudaStream_t st);

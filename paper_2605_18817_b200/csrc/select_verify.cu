@@ -60,6 +60,8 @@ select_kernel(const float *__restrict__ conf, const int32_t *__restrict__ token,
               const int32_t *__restrict__ dense_row, int M, int K, int L, mrp_select_params p,
               mrp_select_out out, int Kd, const int32_t *__restrict__ row_index)
 {
+    pdl_trigger();
+    pdl_wait();
     const int b = blockIdx.x, lane = threadIdx.x;
     // Position -> masked row of this block: from the prepared dense map, or (dense_row == NULL,
     // few masked rows) built here in shared memory by one scan over the row list.
@@ -179,6 +181,8 @@ __global__ void verify_kernel(const int32_t *__restrict__ draft_tok,
                               const int32_t *__restrict__ draft_len, int B, int Kd, int positionwise,
                               int32_t *__restrict__ accept_len, int8_t *__restrict__ accept_mask)
 {
+    pdl_trigger();
+    pdl_wait();
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
     if (b >= B) return;
     int n = draft_len[b];
@@ -201,9 +205,9 @@ cudaError_t launch_select(Ctx *c, const float *conf, const int32_t *token, const
     const int Kd = K * (p.r_draft > 0 ? p.r_draft : 0);
     if ((long long)B * M <= (1ll << 22)) {
         // few rows: every block finds its rows itself, one launch instead of three
-        select_kernel<<<B, 32, 0, st>>>(conf, token, nullptr, M, K, L, p, out, Kd, row_index);
         c->launches++;
-        return cudaGetLastError();
+        return launch_k(select_kernel, dim3(B), dim3(32), 0, st, !(c->cfg.flags & MRP_FLAG_NO_PDL), conf, token,
+                        (const int32_t *)nullptr, M, K, L, p, out, Kd, row_index);
     }
     int32_t *dense_row = (int32_t *)(c->ws + c->lay.dense_row);
     cudaError_t e = cudaMemsetAsync(dense_row, 0xFF, sizeof(int32_t) * (size_t)B * L, st);
@@ -222,10 +226,9 @@ cudaError_t launch_verify(Ctx *c, const int32_t *draft_tok, const int32_t *verif
                           int32_t *accept_len, int8_t *accept_mask, cudaStream_t st)
 {
     if (B == 0) return cudaSuccess;
-    verify_kernel<<<(B + 127) / 128, 128, 0, st>>>(draft_tok, verify_tok, draft_len, B, Kd,
-                                                   positionwise, accept_len, accept_mask);
     c->launches++;
-    return cudaGetLastError();
+    return launch_k(verify_kernel, dim3((B + 127) / 128), dim3(128), 0, st, !(c->cfg.flags & MRP_FLAG_NO_PDL),
+                    draft_tok, verify_tok, draft_len, B, Kd, positionwise, accept_len, accept_mask);
 }
 
 }  // namespace mrp

@@ -259,11 +259,14 @@ __global__ void combine_kernel(const Partial *__restrict__ partials, int n_slice
                                int32_t *__restrict__ status, int32_t *__restrict__ user_status,
                                const TopFix fix)
 {
+    pdl_trigger();
+    pdl_wait();
     const int rs = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (rs >= n_rs) return;
     Partial p;
     p.mx = -INFINITY; p.sum = 0.f; p.idx = INT_MAX; p.second = -INFINITY;
+#pragma unroll 8
     for (int s = lane; s < n_slices; s += 32) p = merge_partial(p, partials[(size_t)s * n_rs + rs]);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
@@ -317,10 +320,10 @@ cudaError_t launch_combine(Ctx *c, const Partial *partials, int n_slices, int n_
     TopFix f;
     memset(&f, 0, sizeof(f));
     if (fix) f = *fix;
-    combine_kernel<<<(n_rowsteps + warps - 1) / warps, warps * 32, 0, st>>>(
-        partials, n_slices, n_rowsteps, out.conf, out.lse, out.token, out.margin, status, out.status, f);
     c->launches++;
-    return cudaGetLastError();
+    return launch_k(combine_kernel, dim3((n_rowsteps + warps - 1) / warps), dim3(warps * 32), 0, st,
+                    !(c->cfg.flags & MRP_FLAG_NO_PDL), partials, n_slices, n_rowsteps, out.conf, out.lse,
+                    out.token, out.margin, status, out.status, f);
 }
 
 template <typename T>

@@ -334,6 +334,8 @@ __global__ void tc_prep_kernel(const __nv_bfloat16 *__restrict__ hidden, const i
                                __nv_bfloat16 *__restrict__ xt0, float *__restrict__ sumsq,
                                int32_t *__restrict__ counters, int n_counters)
 {
+    pdl_trigger();
+    pdl_wait();
     // arrival counters of the few-row head kernels start every pass at zero
     if (blockIdx.x == 0)
         for (int i = threadIdx.x; i < n_counters; i += blockDim.x) counters[i] = 0;
@@ -523,11 +525,11 @@ cudaError_t tc_draft(Ctx *c, const void *hidden, const float *logits0, const int
 
     prof_mark(c, 0, st);
     const int n_rs = (K + 1) * M;
-    tc_prep_kernel<<<M, 256, 0, st>>>((const __nv_bfloat16 *)hidden, row_index, d, M, n_rs,
+    cudaError_t e = note_err(c, launch_k(tc_prep_kernel, dim3(M), dim3(256), 0, st, !(c->cfg.flags & MRP_FLAG_NO_PDL),
+                                         (const __nv_bfloat16 *)hidden, row_index, d, M, n_rs,
                                       (const __nv_bfloat16 *)c->heads[0].rms_gamma, h0f, hcur, xg, xt, sumsq,
-                                      (int32_t *)(c->ws + c->lay.sk_counters), kSkMaxTiles);
+                                      (int32_t *)(c->ws + c->lay.sk_counters), kSkMaxTiles), "tc_prep_kernel");
     c->launches++;
-    cudaError_t e = note_err(c, cudaGetLastError(), "tc_prep_kernel");
     if (e != cudaSuccess) return e;
 
     const bool pdl = !(c->cfg.flags & MRP_FLAG_NO_PDL);

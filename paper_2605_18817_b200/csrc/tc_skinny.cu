@@ -162,22 +162,23 @@ sk_gemm_kernel(const __grid_constant__ SkMaps maps, const SkParams p)
         if (lane == 0) {
             const int total_it = n_tiles * nk;
             const int pre = min(p.n_stages, total_it);
+            const uint64_t pol_w = l2_policy_evict_first(), pol_x = l2_policy_evict_last();
             auto load_w = [&](int t, int kk, int s) {
                 const uint32_t sw = base + (uint32_t)s * stage_bytes;
                 const int h = tile_units(t);
                 mbar_expect_tx(full_bar(s), (uint32_t)h * 2048u + (uint32_t)x_bytes);
                 const int ut = tile_start(t);
                 if (KIND == SK_GU) {
-                    tma_load_2d(sw, &maps.w[0], (kc0 + kk) * kBK, ut * 8, full_bar(s));
-                    tma_load_2d(sw + 64 * 128, &maps.w[3], (kc0 + kk) * kBK, ut * 8, full_bar(s));
+                    tma_load_2d_hint(sw, &maps.w[0], (kc0 + kk) * kBK, ut * 8, full_bar(s), pol_w);
+                    tma_load_2d_hint(sw + 64 * 128, &maps.w[3], (kc0 + kk) * kBK, ut * 8, full_bar(s), pol_w);
                 } else {
-                    tma_load_2d(sw, &maps.w[tile_map(h)], (kc0 + kk) * kBK, ut * 16, full_bar(s));
+                    tma_load_2d_hint(sw, &maps.w[tile_map(h)], (kc0 + kk) * kBK, ut * 16, full_bar(s), pol_w);
                 }
             };
             auto load_x = [&](int kk, int s) {
                 const uint32_t sx = base + (uint32_t)s * stage_bytes + kWTile;
-                tma_load_2d(sx, &maps.x, (kc0 + kk) * kBK, p.x_row_hi, full_bar(s));
-                tma_load_2d(sx + RP * 128, &maps.x, (kc0 + kk) * kBK, p.x_row_lo, full_bar(s));
+                tma_load_2d_hint(sx, &maps.x, (kc0 + kk) * kBK, p.x_row_hi, full_bar(s), pol_x);
+                tma_load_2d_hint(sx + RP * 128, &maps.x, (kc0 + kk) * kBK, p.x_row_lo, full_bar(s), pol_x);
             };
             // weights do not depend on the previous kernel: fill the ring with them first
             int t = 0, kk = 0;
