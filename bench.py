@@ -123,6 +123,20 @@ class ClockSampler:
                 "samples": len(sm)}
 
 
+def replica_throughput(dist, device, units_per_rank, seconds):
+    """Whole-job throughput of independent replicas (the path has no collective): every rank
+    processed ``units_per_rank`` units; the job's time is the slowest rank's.  Returns
+    (units per second over all ranks, that time).  ``dist`` None = a single process."""
+    import torch
+    world = 1
+    if dist is not None:
+        t = torch.tensor([seconds], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        seconds = float(t.item())
+        world = dist.get_world_size()
+    return world * units_per_rank / seconds, seconds
+
+
 def lm_head_roofline(cfg, M, lm_ms, peaks, peaks_kind, traffic):
     """Roofline of the fused LM-head kernel: algorithmic bytes 2Vd + 4MV + 2KMd (one read of
     the LM head, one read of l_0, the stacked residual rows), flops 2KMVd."""
@@ -393,12 +407,9 @@ def main():
         t_wall1 = time.time()
     sampler.stop()
     clocks = sampler.summary(t_wall0, t_wall1)
-    if dist is not None:
-        t = torch.tensor([ms_total], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    value, sec_total = replica_throughput(dist, dev, K * M * args.steps, ms_total * 1e-3)
+    ms_total = sec_total * 1e3
     ms_step = ms_total / args.steps
-    value = world * K * M * args.steps / (ms_total * 1e-3)
 
     # per-phase kernel times, CUDA events on the launching stream, same number of steps
     binding.mrp_profile_enable(ctx, True)
@@ -471,11 +482,8 @@ def main():
             e2e_step()
         barrier()
         dt = time.perf_counter() - t0
-        if dist is not None:
-            t = torch.tensor([dt], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            dt = float(t.item())
-        e2e = {"value": world * K * M * n_e2e / dt, "unit": UNIT, "h2d_bytes_per_step": bi,
+        e2e_value, dt = replica_throughput(dist, dev, K * M * n_e2e, dt)
+        e2e = {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": bi,
                "d2h_bytes_per_step": bo, "steps": n_e2e, "ms_per_step": dt / n_e2e * 1e3, "mode": e2e_mode}
 
     cpu = None
