@@ -62,8 +62,8 @@ typedef enum { MRP_F32 = 0, MRP_BF16 = 1 } mrp_dtype;
 #define MRP_FLAG_ROW_MAJOR_ONLY 4   /* tensor-core family: never use the few-row kernels  */
 #define MRP_FLAG_EXACT_OPERANDS 8   /* tensor-core family: always carry the LM-head activation
                                        operand as a bf16 hi + lo pair (products exact to 2^-17),
-                                       also where the contraction is tensor-core bound.  Without
-                                       it, calls with more than 128 row-steps (K * M) round that
+                                       also where that doubles the tensor work for nothing.  Without
+                                       it, calls with more than 32 row-steps ((K+1) * M) round that
                                        operand once to fp16 (11 significant bits) against an fp16
                                        copy of W_lm kept in the workspace: half the tensor work,
                                        confidence / log-sum-exp still within 2e-3.  The copy is

@@ -44,7 +44,8 @@ constexpr int kSkMaxTiles = 4096;     // weight tiles of a few-row head kernel
 constexpr int kSkScratchBytes = 192 * 128 * 128 * 4;   // partial accumulators of split few-row head kernels
 constexpr int kSimtSliceV = 128;      // vocabulary entries per SIMT LM-head slice
 constexpr int kSimtMaxBlocks = 592;   // SIMT LM-head grid cap (4 per SM)
-constexpr int kF16MinRowSteps = 129;  // fp16 LM-head operands from this many row-steps K*M on
+constexpr int kF16MinRowSteps = 33;   // fp16 LM-head operands from this many row-steps (K+1)*M on,
+                                      // i.e. wherever the row-major LM-head kernel runs
 
 WorkspaceLayout workspace_layout(const mrp_config &cfg);
 

@@ -287,6 +287,7 @@ __global__ void combine_kernel(const Partial *__restrict__ partials, int n_slice
         const __nv_bfloat16 *wr = fix.w + (size_t)tok * fix.d;
         const __nv_bfloat16 *xh = fix.xt + (size_t)rs * fix.d, *xl = xh + (size_t)fix.n_rs * fix.d;
         float dot = 0.f;
+#pragma unroll 8
         for (int j = lane * 2; j < fix.d; j += 64) {
             const float2 w2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(wr + j));
             const float2 h2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(xh + j));

@@ -533,7 +533,8 @@ cudaError_t tc_draft(Ctx *c, const void *hidden, const float *logits0, const int
     if (e != cudaSuccess) return e;
 
     const bool pdl = !(c->cfg.flags & MRP_FLAG_NO_PDL);
-    const bool f16_lm = c->use_f16_lm && K * M >= kF16MinRowSteps;
+    const bool f16_lm = c->use_f16_lm && (K + 1) * M >= kF16MinRowSteps &&
+                        !(sk_rows_ok((K + 1) * M) && !(c->cfg.flags & MRP_FLAG_ROW_MAJOR_ONLY));
     const bool few_rows = sk_head_rows_ok(M) && sk_heads_ok(c->cfg) &&
                           !(c->cfg.flags & MRP_FLAG_ROW_MAJOR_ONLY);
     int n_ss = 1;

@@ -182,9 +182,9 @@ def test_sweep_points_sampled_rows(sweep_dev, M, K):
     binding.mrp_destroy(ctx)
 
 
-@pytest.mark.parametrize("M,K", [(256, 1), (1024, 2), (4096, 4)])
+@pytest.mark.parametrize("M,K", [(16, 2), (64, 4), (256, 1), (1024, 2), (4096, 4)])
 def test_fp16_operand_mode_stays_close_to_exact_operands_on_every_row(sweep_dev, M, K):
-    """Above 128 row-steps the LM head rounds its activation operand once to fp16 instead of
+    """Above 32 row-steps the LM head rounds its activation operand once to fp16 instead of
     carrying a bf16 hi + lo pair.  Every row-step of the call is compared with the same call
     under MRP_FLAG_EXACT_OPERANDS (itself checked against the oracle on sampled rows above):
     the two must agree well inside the 2e-3 tolerance, which leaves the exact path's own error
