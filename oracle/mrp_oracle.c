@@ -15,7 +15,7 @@
  *   - max-accept cap m = min(max(floor(0.7 n), 5), L) (Sec. 4.4);
  *   - verification = a drafted token is accepted iff it equals the backbone's argmax
  *     (Algorithm 3), with the prefix semantics of Figure 1(d).
- * The head g is the reduced module this build is specified on: RMSNorm followed by a
+ * The head g is the reduced module of the benchmark configurations: RMSNorm followed by a
  * SwiGLU MLP (no biases), whose output r is both the hidden residual Delta and the
  * vector sent through the LM head (delta = W_lm r).
  *
