@@ -60,6 +60,8 @@ typedef enum { MRP_F32 = 0, MRP_BF16 = 1 } mrp_dtype;
 #define MRP_FLAG_NO_PDL 2      /* launch every kernel fully serialised (no programmatic
                                   dependent launch); for timing comparisons               */
 #define MRP_FLAG_ROW_MAJOR_ONLY 4   /* tensor-core family: never use the few-row kernels  */
+#define MRP_FLAG_NO_CHAIN 16    /* tensor-core family: run the head chain of a few-row call as
+                                  one kernel per GEMM instead of one persistent kernel      */
 #define MRP_FLAG_EXACT_OPERANDS 8   /* tensor-core family: always carry the LM-head activation
                                        operand as a bf16 hi + lo pair (products exact to 2^-17),
                                        also where that doubles the tensor work for nothing.  Without

@@ -23,6 +23,7 @@ MRP_FLAG_FORCE_SIMT = 1
 MRP_FLAG_NO_PDL = 2
 MRP_FLAG_ROW_MAJOR_ONLY = 4
 MRP_FLAG_EXACT_OPERANDS = 8
+MRP_FLAG_NO_CHAIN = 16
 MRP_SELECT_STATIC, MRP_SELECT_DYNAMIC_REMASK = 0, 1
 MRP_DEV_NONFINITE, MRP_DEV_TIMEOUT = 1, 2
 

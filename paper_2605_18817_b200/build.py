@@ -9,7 +9,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(_HERE), "include")
 LIB = os.path.join(_HERE, "libmrp_b200.so")
-SOURCES = ["mrp_api.cu", "simt_kernels.cu", "select_verify.cu", "tc_kernels.cu", "tc_skinny.cu"]
+SOURCES = ["mrp_api.cu", "simt_kernels.cu", "select_verify.cu", "tc_kernels.cu", "tc_skinny.cu", "tc_chain.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17"]
 
 

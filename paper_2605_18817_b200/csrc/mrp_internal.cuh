@@ -154,6 +154,8 @@ cudaError_t sk_gateup(Ctx *c, int k, int M, int K, int n_ss, const mrp_draft_out
 cudaError_t sk_down(Ctx *c, int k, int M, int K, const mrp_draft_out &out, cudaStream_t st, bool pdl,
                     int *n_ss_out, bool f16_lm);
 bool sk_heads_ok(const mrp_config &cfg);
+// The whole head chain as one cooperative kernel (tc_chain.cu); cudaErrorNotSupported = use the others.
+cudaError_t sk_chain(Ctx *c, int M, int K, const mrp_draft_out &out, cudaStream_t st, bool f16_lm);
 cudaError_t sk_lm(Ctx *c, const float *logits0, const int32_t *row_index, int M, int K,
                   const mrp_draft_out &out, cudaStream_t st, bool pdl);
 

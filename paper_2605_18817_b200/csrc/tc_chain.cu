@@ -1,0 +1,519 @@
+// The head chain for few activation rows as ONE persistent kernel (sm_100a, cooperative launch).
+//
+// For a handful of masked rows each GEMM of the chain (gate/up and down projection of every
+// head, a1) moves 17-67 MB of weights and lasts a few microseconds; run as separate kernels
+// they spend more time on launch, ring fill, first-use code fetch and drain than on the weights.
+// Here the 2K GEMMs are phases of one kernel: every CTA walks the phases with the same TMA ring,
+// MMA issuer and epilogue warps as the few-row kernels (tc_skinny.cu: weight rows on the MMA M
+// axis, bf16 hi + lo activation rows stacked on N, one 128-row weight tile and one slice of the
+// contraction per CTA and phase).  A phase needs the previous phase's activations, so the
+// CTAs meet at a grid barrier between phases -- but the weights depend on nothing: the producer
+// fills the ring with the next phase's weight tiles before it waits, and only the activation
+// tiles are fetched after the barrier.
+// Every wait is bounded: a barrier or mbarrier wait that runs out sets MRP_DEV_TIMEOUT and the
+// CTA leaves; the others then run out as well.
+#include <cuda_fp16.h>
+#include <string.h>
+
+#include "tc_common.cuh"
+
+namespace mrp {
+namespace {
+
+constexpr int kChThreads = 192;
+constexpr int kChWTile = 128 * 128;
+constexpr int kChAuxBytes = 12288;
+constexpr int kChAuxRstd = 0;              // float[128]
+constexpr int kChAuxVote = 768;            // int
+constexpr int kChAuxReleased = 772;        // int: phases whose barrier this CTA has seen released
+constexpr int kChAuxSq = 4096;             // float[2048]: squares of a share's outputs
+constexpr int kChMaxShare = 2048;          // outputs a CTA finishes per down-projection phase, at most
+constexpr int kChTilesPerPhase = 448;      // arrival counters per phase
+constexpr int kChMaxPhases = 8;
+constexpr long long kBarrierCycles = 1000000000LL;   // bound on a grid-barrier wait (about 0.5 s)
+
+enum { CH_GU = 0, CH_DN = 1 };
+
+struct ChainMaps {
+    CUtensorMap m[2 + 3 * 4];   // 0: head input (xg), 1: SwiGLU output (act), 2+3h: gate, 3+3h: up, 4+3h: down of head h
+};
+
+struct ChainPhase {
+    int kind;
+    int k_chunks;        // contraction extent / 64
+    int n_tiles;         // 128-row weight tiles (GU: 64 gate + 64 up rows)
+    int n_split;         // CTAs per tile, each a slice of the contraction
+    int w_rows;          // weight rows (GU: gate rows)
+    int map_x, map_w0, map_w1;
+    int n_ss;            // GU: slices of sums of squares to add up
+    const __nv_bfloat16 *gamma_next;   // DN
+    __nv_bfloat16 *xg_next;
+    __nv_bfloat16 *xt_k;
+    __half *xt16_k;
+    float *hidden_out;
+};
+
+struct ChainParams {
+    int n_phases, n_stages, tmem_cols;
+    int M, d, F, n_rs;
+    float eps;
+    ChainPhase ph[kChMaxPhases];
+    __nv_bfloat16 *act;
+    float *hcur;
+    const float *h0f;
+    float *sumsq;            // [slices][M]: read by GU, written (one slice per CTA) by DN
+    float *scratch;          // partial accumulators [cta][RP][128]
+    int32_t *counters;       // arrivals per (phase, tile) (zero at launch)
+    unsigned int *grid_bar;  // CTAs that have finished a phase, summed over phases (zero at launch)
+    int32_t *status;
+    int32_t *user_status;
+};
+
+__device__ __forceinline__ void ch_epi_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+__device__ __forceinline__ void ch_store_hi_lo(__nv_bfloat16 *dst, size_t lo_off, float v)
+{
+    const __nv_bfloat16 hi = __float2bfloat16_rn(v);
+    dst[0] = hi;
+    dst[lo_off] = __float2bfloat16_rn(v - __bfloat162float(hi));
+}
+__device__ __forceinline__ unsigned int ld_acquire_u32(const unsigned int *p)
+{
+    unsigned int v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+// Waits until `target` arrivals have been counted; false if the wait ran out or another role gave up.
+__device__ __forceinline__ bool grid_bar_wait(const unsigned int *bar, unsigned int target, volatile int *abort_flag,
+                                              const ChainParams &p)
+{
+    if ((int)(ld_acquire_u32(bar) - target) >= 0) return true;
+    const long long t0 = clock64();
+    while ((int)(ld_acquire_u32(bar) - target) < 0) {
+        __nanosleep(128);
+        if (*abort_flag) return false;
+        if (clock64() - t0 > kBarrierCycles) {
+            *abort_flag = 1;
+            atomicOr(p.status, MRP_DEV_TIMEOUT);
+            if (p.user_status) atomicOr(p.user_status, MRP_DEV_TIMEOUT);
+            return false;
+        }
+    }
+    return true;
+}
+
+template <int RP>
+__global__ void __launch_bounds__(kChThreads, 1)
+sk_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    constexpr int x_bytes = 2 * RP * 128;            // hi rows then lo rows of one k-chunk
+    constexpr int stage_bytes = kChWTile + x_bytes;
+    const uint32_t bars = base + (uint32_t)p.n_stages * stage_bytes;
+    auto full_bar = [&](int s) { return bars + 8u * s; };
+    auto empty_bar = [&](int s) { return bars + 8u * (p.n_stages + s); };
+    auto tfull_bar = [&](int a) { return bars + 8u * (2 * p.n_stages + a); };
+    auto tempty_bar = [&](int a) { return bars + 8u * (2 * p.n_stages + 2 + a); };
+    uint8_t *gen_base = smem_raw + (base - smem_u32(smem_raw));
+    uint8_t *after_bars = gen_base + (size_t)p.n_stages * stage_bytes + 8 * (2 * p.n_stages + 4);
+    uint32_t *tmem_holder = reinterpret_cast<uint32_t *>(after_bars);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_holder + 1);
+    uint8_t *aux = after_bars + 16;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int cta = blockIdx.x, G = gridDim.x;
+
+    // this CTA's share of phase i: weight tile, chunk range; false if it has none
+    auto share = [&](int i, int &tile, int &kc0, int &nk) {
+        const ChainPhase &ph = p.ph[i];
+        if (cta >= ph.n_tiles * ph.n_split) return false;
+        const int cps = (ph.k_chunks + ph.n_split - 1) / ph.n_split;
+        tile = cta / ph.n_split;
+        kc0 = (cta % ph.n_split) * cps;
+        nk = min(ph.k_chunks, kc0 + cps) - kc0;
+        return true;
+    };
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < p.n_stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        prefetch_tmap(&maps.m[0]);
+        prefetch_tmap(&maps.m[2]);
+        prefetch_tmap(&maps.m[3]);
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(tmem_holder)), "r"((uint32_t)p.tmem_cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_holder;
+    pdl_trigger();
+
+    if (warp == 0) {
+        // ---------------- TMA producer ----------------
+        if (lane == 0) {
+            const uint64_t pol_w = l2_policy_evict_first(), pol_x = l2_policy_evict_last();
+            int it = 0;                       // chunks issued so far, over all phases
+            bool ok = true;
+            for (int i = 0; i < p.n_phases && ok; ++i) {
+                int tile, kc0, nk;
+                if (!share(i, tile, kc0, nk)) continue;
+                const ChainPhase &ph = p.ph[i];
+                auto stage_of = [&](int n) { return n % p.n_stages; };
+                auto claim = [&](int n) {     // wait until the stage of chunk n is free, arm its barrier
+                    const int s = stage_of(n), use = n / p.n_stages;
+                    if (use > 0 && !mbar_wait(empty_bar(s), (uint32_t)((use - 1) & 1), abort_flag, p)) return false;
+                    mbar_expect_tx(full_bar(s), (uint32_t)(kChWTile + x_bytes));
+                    return true;
+                };
+                auto load_w = [&](int n, int kk) {
+                    const uint32_t sw = base + (uint32_t)stage_of(n) * stage_bytes;
+                    if (ph.kind == CH_GU) {
+                        tma_load_2d_hint(sw, &maps.m[ph.map_w0], (kc0 + kk) * kBK, tile * 64, full_bar(stage_of(n)), pol_w);
+                        tma_load_2d_hint(sw + 64 * 128, &maps.m[ph.map_w1], (kc0 + kk) * kBK, tile * 64, full_bar(stage_of(n)), pol_w);
+                    } else {
+                        tma_load_2d_hint(sw, &maps.m[ph.map_w0], (kc0 + kk) * kBK, tile * 128, full_bar(stage_of(n)), pol_w);
+                    }
+                };
+                auto load_x = [&](int n, int kk) {
+                    const uint32_t sx = base + (uint32_t)stage_of(n) * stage_bytes + kChWTile;
+                    tma_load_2d_hint(sx, &maps.m[ph.map_x], (kc0 + kk) * kBK, 0, full_bar(stage_of(n)), pol_x);
+                    tma_load_2d_hint(sx + RP * 128, &maps.m[ph.map_x], (kc0 + kk) * kBK, p.M, full_bar(stage_of(n)), pol_x);
+                };
+                // weights depend on nothing: put as many chunks of them in flight as the ring holds
+                const int pre = min(p.n_stages, nk);
+                for (int kk = 0; kk < pre && ok; ++kk) {
+                    ok = claim(it + kk);
+                    if (ok) load_w(it + kk, kk);
+                }
+                if (!ok) break;
+                // the activations are the previous phase's (or the previous kernel's) output
+                if (i == 0) {
+                    pdl_wait();
+                } else {
+                    // one thread of the CTA (epilogue thread 0) polls the grid barrier; wait for its word
+                    volatile int *released_s = reinterpret_cast<volatile int *>(aux + kChAuxReleased);
+                    const long long t0 = clock64();
+                    bool passed = true;
+                    while (*released_s < i) {
+                        if (*abort_flag || clock64() - t0 > 2 * kBarrierCycles) { passed = false; break; }
+                    }
+                    if (!passed) break;
+                }
+                asm volatile("fence.proxy.async;" ::: "memory");
+                for (int kk = 0; kk < pre; ++kk) load_x(it + kk, kk);
+                for (int kk = pre; kk < nk && ok; ++kk) {
+                    ok = claim(it + kk);
+                    if (ok) { load_w(it + kk, kk); load_x(it + kk, kk); }
+                }
+                it += nk;
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
+        if (lane == 0) {
+            const uint32_t idesc = make_idesc(2 * RP);
+            int it = 0, n_acc = 0;
+            bool ok = true;
+            for (int i = 0; i < p.n_phases && ok; ++i) {
+                int tile, kc0, nk;
+                if (!share(i, tile, kc0, nk)) continue;
+                const int acc = n_acc & 1, use = n_acc >> 1;
+                if (use > 0 && !mbar_wait(tempty_bar(acc), (uint32_t)((use - 1) & 1), abort_flag, p)) break;
+                tc_fence_after();
+                const uint32_t dt = tmem_base + (uint32_t)(acc * 2 * RP);
+                for (int kk = 0; kk < nk; ++kk) {
+                    const int s = (it + kk) % p.n_stages;
+                    if (!mbar_wait(full_bar(s), (uint32_t)(((it + kk) / p.n_stages) & 1), abort_flag, p)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t sw = base + (uint32_t)s * stage_bytes;
+                    const uint64_t dw = make_smem_desc(sw);
+                    const uint64_t dx = make_smem_desc(sw + kChWTile);
+#pragma unroll
+                    for (int k4 = 0; k4 < kBK / 16; ++k4)
+                        umma_bf16(dt, dw + 2u * k4, dx + 2u * k4, idesc, (kk > 0 || k4 > 0) ? 1u : 0u);
+                    umma_commit(empty_bar(s));
+                }
+                if (!ok) break;
+                umma_commit(tfull_bar(acc));
+                it += nk;
+                ++n_acc;
+            }
+        }
+    } else {
+        // ---------------- epilogue warps ----------------
+        // Per phase: (1) thread t parks TMEM lane t (weight row t of the tile) of this slice's
+        // accumulator in global scratch; (2) the CTAs of the tile wait for one another; (3) every
+        // CTA finishes its own share of the tile's rows from the parked slices, added in slice
+        // order, so all SMs take part in the element-wise work and its memory round trips.
+        const int q = warp & 3;
+        const int t = q * 32 + lane;
+        const uint32_t lane_base = tmem_base + ((uint32_t)(q * 32) << 16);
+        float *rstd_s = reinterpret_cast<float *>(aux + kChAuxRstd);
+        float *sq_s = reinterpret_cast<float *>(aux + kChAuxSq);
+        volatile int *vote_s = reinterpret_cast<volatile int *>(aux + kChAuxVote);
+        volatile int *released_s = reinterpret_cast<volatile int *>(aux + kChAuxReleased);
+        const int n_ch = (p.M + 15) >> 4;
+        int n_acc = 0;
+        bool alive = true;
+        pdl_wait();
+        for (int i = 0; i < p.n_phases && alive; ++i) {
+            const ChainPhase &ph = p.ph[i];
+            // everything this phase reads was written before the previous phase's barrier
+            if (t == 0) {
+                if (i == 0) { *vote_s = 0; *released_s = 0; }
+                else if (grid_bar_wait(p.grid_bar, (unsigned int)i * G, abort_flag, p)) *released_s = i;
+                else *vote_s = 1;
+            }
+            ch_epi_sync();
+            if (*vote_s == 1) { alive = false; break; }
+            int tile, kc0, nk;
+            const bool active = share(i, tile, kc0, nk);
+            if (active) {
+                const int split = cta % ph.n_split;
+                if (ph.kind == CH_GU) {
+                    // rstd of row m from the slices of sums of squares: warp per row, lanes over slices
+                    for (int m = q; m < p.M; m += 4) {
+                        float s = 0.f;
+                        for (int j = lane; j < ph.n_ss; j += 32) s += __ldcg(p.sumsq + (size_t)j * p.M + m);
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+                        if (lane == 0) rstd_s[m] = rsqrtf(s / (float)p.d + p.eps);
+                    }
+                }
+                const int acc = n_acc & 1, use = n_acc >> 1;
+                ++n_acc;
+                const uint32_t lane_addr = lane_base + (uint32_t)(acc * 2 * RP);
+                bool ok = __all_sync(0xffffffffu, mbar_wait(tfull_bar(acc), (uint32_t)(use & 1), abort_flag, p));
+                if (!ok && lane == 0) *vote_s = 1;
+                ch_epi_sync();                      // also publishes rstd_s
+                if (*vote_s == 1) { alive = false; break; }
+                tc_fence_after();
+                // (1) park this slice: scratch[cta][column][lane]
+                float *mine = p.scratch + ((size_t)cta * RP) * 128;
+#pragma unroll 1
+                for (int ch = 0; ch < n_ch; ++ch) {
+                    float v[16], w[16];
+                    tmem_ld16(lane_addr + ch * 16, v);
+                    tmem_ld16(lane_addr + RP + ch * 16, w);
+#pragma unroll
+                    for (int j = 0; j < 16; ++j)
+                        if (ch * 16 + j < p.M) mine[(ch * 16 + j) * 128 + t] = v[j] + w[j];
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(tempty_bar(acc));     // the accumulator buffer is free again
+                // (2) meet the other CTAs of the tile
+                __threadfence();
+                ch_epi_sync();
+                if (t == 0) {
+                    unsigned int *cnt = reinterpret_cast<unsigned int *>(p.counters) + i * kChTilesPerPhase + tile;
+                    atomicAdd(cnt, 1u);
+                    if (!grid_bar_wait(cnt, (unsigned int)ph.n_split, abort_flag, p)) *vote_s = 1;
+                }
+                ch_epi_sync();
+                if (*vote_s == 1) { alive = false; break; }
+                __threadfence();
+                // (3) this CTA's share of the tile's output rows, element by element from the parked slices
+                const int rows_tile = ph.kind == CH_GU ? 64 : 128;
+                const int per = (rows_tile + ph.n_split - 1) / ph.n_split;
+                const int r0 = split * per;
+                const int n_r = max(0, min(rows_tile, r0 + per) - r0);
+                const int n_items = n_r * p.M;
+                const float *first = p.scratch + ((size_t)tile * ph.n_split * RP) * 128;
+                if (ph.kind == CH_GU) {
+#pragma unroll 2
+                    for (int e = t; e < n_items; e += 128) {
+                        const int m = e / n_r, row = r0 + (e - m * n_r);
+                        const int f = tile * 64 + row;
+                        if (f < ph.w_rows) {
+                            float g = 0.f, u = 0.f;
+                            for (int s0 = 0; s0 < ph.n_split; s0 += 8) {  // slice order; 8 slices' loads in flight
+                                float gs[8], us[8];
+#pragma unroll
+                                for (int k = 0; k < 8; ++k) {
+                                    const float *src = first + ((size_t)(s0 + k) * RP + m) * 128 + row;
+                                    gs[k] = (s0 + k < ph.n_split) ? __ldcg(src) : 0.f;
+                                    us[k] = (s0 + k < ph.n_split) ? __ldcg(src + 64) : 0.f;
+                                }
+#pragma unroll
+                                for (int k = 0; k < 8; ++k) { g += gs[k]; u += us[k]; }
+                            }
+                            g *= rstd_s[m];
+                            u *= rstd_s[m];
+                            ch_store_hi_lo(p.act + (size_t)m * p.F + f, (size_t)p.M * p.F, g / (1.f + __expf(-g)) * u);
+                        }
+                    }
+                } else {
+#pragma unroll 2
+                    for (int e = t; e < n_items; e += 128) {
+                        const int m = e / n_r, row = r0 + (e - m * n_r);
+                        const int j = tile * 128 + row;
+                        float sq = 0.f;
+                        if (j < ph.w_rows) {
+                            const size_t o = (size_t)m * p.d + j;
+                            const float hc = __ldcg(p.hcur + o), h0 = __ldg(p.h0f + o);
+                            float a = 0.f;
+                            for (int s0 = 0; s0 < ph.n_split; s0 += 8) {  // slice order; 8 slices' loads in flight
+                                float as[8];
+#pragma unroll
+                                for (int k = 0; k < 8; ++k)
+                                    as[k] = (s0 + k < ph.n_split) ? __ldcg(first + ((size_t)(s0 + k) * RP + m) * 128 + row) : 0.f;
+#pragma unroll
+                                for (int k = 0; k < 8; ++k) a += as[k];
+                            }
+                            const float h = hc + a;
+                            p.hcur[o] = h;
+                            if (ph.hidden_out) ph.hidden_out[o] = h;
+                            sq = h * h;
+                            ch_store_hi_lo(ph.xt_k + o, (size_t)p.n_rs * p.d, h - h0);
+                            if (ph.xt16_k) ph.xt16_k[o] = __float2half_rn(h - h0);
+                            if (ph.xg_next) ch_store_hi_lo(ph.xg_next + o, (size_t)p.M * p.d, h * __bfloat162float(ph.gamma_next[j]));
+                        }
+                        sq_s[e] = sq;
+                    }
+                    ch_epi_sync();
+                    // one slice of sums of squares per CTA: its rows, in row order
+                    for (int m = t; m < p.M; m += 128) {
+                        float s = 0.f;
+                        for (int r = 0; r < n_r; ++r) s += sq_s[m * n_r + r];
+                        p.sumsq[(size_t)cta * p.M + m] = s;
+                    }
+                }
+            }
+            // this CTA's part of the phase is in memory: arrive at the grid barrier
+            __threadfence();
+            ch_epi_sync();
+            if (t == 0) atomicAdd(p.grid_bar, 1u);
+        }
+    }
+
+    // ---------------- teardown ----------------
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        // a wait gave up: give copies still in flight time to land before the CTA leaves
+        const long long t0 = clock64();
+        while (clock64() - t0 < 200000) __nanosleep(1000);
+        __syncthreads();
+    }
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)p.tmem_cols) : "memory");
+    }
+}
+
+template <int RP>
+cudaError_t chain_launch(const ChainMaps &maps, const ChainParams &p, int grid, size_t smem, cudaStream_t st)
+{
+    auto kern = sk_chain_kernel<RP>;
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kChThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    // the CTAs wait for one another at the phase barriers: they must all be resident
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeCooperative;
+    at[0].val.cooperative = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, maps, p);
+}
+
+}  // namespace
+
+// The whole head chain (K heads) for M <= 64 rows as one kernel.  Returns cudaErrorNotSupported
+// (nothing launched) if the shape does not fit this form; the caller then runs the chain as
+// separate kernels.
+cudaError_t sk_chain(Ctx *c, int M, int K, const mrp_draft_out &out, cudaStream_t st, bool f16_lm)
+{
+    const TcState *s = (const TcState *)c->tc_state;
+    const int d = c->cfg.d, F = c->cfg.d_ff, G = c->sm_count;
+    if (K < 1 || K > 4 || 2 * K > kChMaxPhases || M < 1 || M > 64) return cudaErrorNotSupported;
+    // Worth it while a GEMM of the chain is latency-bound (a few tens of MB of weights): measured
+    // 71 vs 77 us at d = 2048, F = 4096, but 201 vs 183 us at d = 4096, F = 8192 (M = 4).
+    if ((long long)d * F > (12ll << 20)) return cudaErrorNotSupported;
+    const int r_pad = M <= 16 ? 16 : M <= 32 ? 32 : 64;
+    const int gu_tiles = F / 64, dn_tiles = (d + 127) / 128;
+    if (gu_tiles > G || dn_tiles > G || G > kSumsqSlices || gu_tiles > kChTilesPerPhase ||
+        kChMaxPhases * kChTilesPerPhase >= kSkMaxTiles)
+        return cudaErrorNotSupported;
+    if ((size_t)G * r_pad * 128 * 4 > (size_t)kSkScratchBytes) return cudaErrorNotSupported;
+
+    ChainParams p;
+    memset(&p, 0, sizeof(p));
+    ChainMaps maps;
+    memset(&maps, 0, sizeof(maps));
+    const int n_rs = (K + 1) * M;
+    p.n_phases = 2 * K; p.M = M; p.d = d; p.F = F; p.n_rs = n_rs; p.eps = c->cfg.rms_eps;
+    p.act = (__nv_bfloat16 *)(c->ws + c->lay.act);
+    p.hcur = (float *)(c->ws + c->lay.hcur); p.h0f = (const float *)(c->ws + c->lay.h0f);
+    p.sumsq = (float *)(c->ws + c->lay.sumsq);
+    p.scratch = (float *)(c->ws + c->lay.sk_scratch);
+    p.counters = (int32_t *)(c->ws + c->lay.sk_counters);
+    p.grid_bar = (unsigned int *)(c->ws + c->lay.sk_counters) + (kSkMaxTiles - 1);
+    p.status = (int32_t *)(c->ws + c->lay.status); p.user_status = out.status;
+    const int stage = kChWTile + 2 * r_pad * 128;
+    int ns = (kSmemBudget - 1024 - 256 - 16 - kChAuxBytes) / stage;
+    if (ns > 12) ns = 12;
+    p.n_stages = ns;
+    int cols = 32;
+    while (cols < 2 * 2 * r_pad) cols <<= 1;
+    p.tmem_cols = cols;
+    const size_t smem = (size_t)ns * stage + 1024 + 8 * (2 * ns + 4) + 16 + kChAuxBytes;
+
+    auto split = [&](int n_tiles, int k_chunks) {
+        int S = G / n_tiles;
+        if (S < 1) S = 1;
+        if (S > k_chunks) S = k_chunks;
+        const int cps = (k_chunks + S - 1) / S;
+        return (k_chunks + cps - 1) / cps;          // no empty slice
+    };
+    __nv_bfloat16 *xg = (__nv_bfloat16 *)(c->ws + c->lay.xg);
+    __nv_bfloat16 *xt = (__nv_bfloat16 *)(c->ws + c->lay.xt);
+    if (!make_map(s, &maps.m[0], xg, d, 2 * (uint64_t)M, r_pad) ||
+        !make_map(s, &maps.m[1], p.act, F, 2 * (uint64_t)M, r_pad))
+        return note_err(c, cudaErrorInvalidValue, "tensor map (head chain, activations)");
+    for (int k = 1; k <= K; ++k) {
+        const mrp_head_weights &hw = c->heads[k - 1];
+        const int b = 2 + 3 * (k - 1);
+        if (!make_map(s, &maps.m[b], hw.w_gate, d, F, 64) || !make_map(s, &maps.m[b + 1], hw.w_up, d, F, 64) ||
+            !make_map(s, &maps.m[b + 2], hw.w_down, F, d, 128))
+            return note_err(c, cudaErrorInvalidValue, "tensor map (head chain, weights)");
+        ChainPhase &gu = p.ph[2 * (k - 1)], &dn = p.ph[2 * (k - 1) + 1];
+        gu.kind = CH_GU; gu.k_chunks = d / kBK; gu.n_tiles = gu_tiles; gu.n_split = split(gu_tiles, gu.k_chunks);
+        gu.w_rows = F; gu.map_x = 0; gu.map_w0 = b; gu.map_w1 = b + 1;
+        gu.n_ss = (k == 1) ? 1 : dn_tiles * split(dn_tiles, F / kBK);
+        dn.kind = CH_DN; dn.k_chunks = F / kBK; dn.n_tiles = dn_tiles; dn.n_split = split(dn_tiles, dn.k_chunks);
+        if (M * ((128 + dn.n_split - 1) / dn.n_split) > kChMaxShare) return cudaErrorNotSupported;
+        dn.w_rows = d; dn.map_x = 1; dn.map_w0 = b + 2; dn.map_w1 = b + 2;
+        dn.gamma_next = (k < K) ? (const __nv_bfloat16 *)c->heads[k].rms_gamma : nullptr;
+        dn.xg_next = (k < K) ? xg : nullptr;
+        dn.xt_k = xt + (size_t)k * M * d;
+        dn.xt16_k = f16_lm ? (__half *)(c->ws + c->lay.xt16) + (size_t)(k - 1) * M * d : nullptr;
+        dn.hidden_out = (k == K) ? out.hidden_out : nullptr;
+    }
+    cudaError_t e;
+    switch (r_pad) {
+    case 16: e = chain_launch<16>(maps, p, G, smem, st); break;
+    case 32: e = chain_launch<32>(maps, p, G, smem, st); break;
+    default: e = chain_launch<64>(maps, p, G, smem, st); break;
+    }
+    c->launches++;
+    return note_err(c, e, "head-chain kernel");
+}
+
+}  // namespace mrp

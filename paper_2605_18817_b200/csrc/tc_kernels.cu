@@ -538,7 +538,13 @@ cudaError_t tc_draft(Ctx *c, const void *hidden, const float *logits0, const int
     const bool few_rows = sk_head_rows_ok(M) && sk_heads_ok(c->cfg) &&
                           !(c->cfg.flags & MRP_FLAG_ROW_MAJOR_ONLY);
     int n_ss = 1;
-    for (int k = 1; k <= K; ++k) {
+    bool chain_done = false;
+    if (few_rows && !(c->cfg.flags & MRP_FLAG_NO_CHAIN)) {
+        e = sk_chain(c, M, K, out, st, f16_lm);
+        if (e == cudaSuccess) chain_done = true;
+        else if (e != cudaErrorNotSupported) return e;
+    }
+    for (int k = 1; k <= K && !chain_done; ++k) {
         if (few_rows) {
             e = sk_gateup(c, k, M, K, n_ss, out, st, pdl);
             if (e != cudaSuccess) return e;

@@ -271,6 +271,9 @@ def test_tensor_core_family_small_shapes(d, F, V, B, L, K):
     # the row-major kernels alone, fully serialised launches: same results within tolerance
     out4, _ = run_gpu_draft(w, inp, K, flags=binding.MRP_FLAG_ROW_MAJOR_ONLY | binding.MRP_FLAG_NO_PDL)
     check_stats(out4, ref, "bf16")
+    # the head chain as one kernel per GEMM instead of one persistent kernel
+    out5, _ = run_gpu_draft(w, inp, K, flags=binding.MRP_FLAG_NO_CHAIN)
+    check_stats(out5, ref, "bf16")
 
 
 @pytest.mark.parametrize("flags", [0, binding.MRP_FLAG_FORCE_SIMT])
