@@ -19,9 +19,10 @@ WorkspaceLayout workspace_layout(const mrp_config &cfg)
     l.status = take(64 * sizeof(int32_t));
     l.h0f = take(rows * d * 4);
     l.hcur = take(rows * d * 4);
-    l.xg = take(rows * d * 4);
-    l.act = take(rows * F * 4);
-    l.xt = take(steps * rows * d * 4);
+    // bf16 hi block + lo block each; the few-row kernels put the lo block at a padded row offset
+    l.xg = take((rows + 64) * d * 4);
+    l.act = take((rows + 64) * F * 4);
+    l.xt = take((steps * rows + 32) * d * 4);
     l.sumsq = take((size_t)kSumsqSlices * rows * 4);
     const int v_slices = (cfg.vocab + kSimtSliceV - 1) / kSimtSliceV;
     l.n_slices_max = v_slices < kSimtMaxBlocks ? v_slices : kSimtMaxBlocks;

@@ -57,6 +57,10 @@ struct Ctx {
     WorkspaceLayout lay;
     bool use_tc;
     bool use_f16_lm;           // the fp16 copy of W_lm exists and is usable
+    // Row offset of the bf16 lo block behind the hi block in this call's operand buffers: M and
+    // (K+1)M for the row-major kernels, the padded row count for the few-row kernels (which then
+    // fetch hi and lo rows of a k-chunk with one TMA box).
+    int lo_x, lo_xt;
     int32_t launches;
     int sm_count;
     void *tc_state;            // tensor-core path state (tensor maps), owned by tc_*.cu
@@ -150,6 +154,8 @@ cudaError_t tc_draft(Ctx *c, const void *hidden, const float *logits0, const int
 // Few-row variants (tc_skinny.cu): weight rows on the MMA M axis; rows <= 32.
 bool sk_rows_ok(int rows);          // LM head: row-steps incl. step 0
 bool sk_head_rows_ok(int M);       // head chain: masked rows
+int sk_head_pad(int M);            // rows of an activation block as the few-row head kernels see it
+int sk_lm_pad(int n_rs);           // likewise for the few-row LM-head kernel
 cudaError_t sk_gateup(Ctx *c, int k, int M, int K, int n_ss, const mrp_draft_out &out, cudaStream_t st, bool pdl);
 cudaError_t sk_down(Ctx *c, int k, int M, int K, const mrp_draft_out &out, cudaStream_t st, bool pdl,
                     int *n_ss_out, bool f16_lm);

@@ -56,6 +56,7 @@ struct ChainPhase {
 struct ChainParams {
     int n_phases, n_stages, tmem_cols;
     int M, d, F, n_rs;
+    int lo_x, lo_xt;         // row offset of the lo block in the head operands / the LM-head operand
     float eps;
     ChainPhase ph[kChMaxPhases];
     __nv_bfloat16 *act;
@@ -182,8 +183,8 @@ sk_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant__ 
                 };
                 auto load_x = [&](int n, int kk) {
                     const uint32_t sx = base + (uint32_t)stage_of(n) * stage_bytes + kChWTile;
+                    // one box: RP hi rows, then (the lo block starts at row RP of the buffer) RP lo rows
                     tma_load_2d_hint(sx, &maps.m[ph.map_x], (kc0 + kk) * kBK, 0, full_bar(stage_of(n)), pol_x);
-                    tma_load_2d_hint(sx + RP * 128, &maps.m[ph.map_x], (kc0 + kk) * kBK, p.M, full_bar(stage_of(n)), pol_x);
                 };
                 // weights depend on nothing: put as many chunks of them in flight as the ring holds
                 const int pre = min(p.n_stages, nk);
@@ -346,7 +347,7 @@ sk_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant__ 
                             }
                             g *= rstd_s[m];
                             u *= rstd_s[m];
-                            ch_store_hi_lo(p.act + (size_t)m * p.F + f, (size_t)p.M * p.F, g / (1.f + __expf(-g)) * u);
+                            ch_store_hi_lo(p.act + (size_t)m * p.F + f, (size_t)p.lo_x * p.F, g / (1.f + __expf(-g)) * u);
                         }
                     }
                 } else {
@@ -371,9 +372,9 @@ sk_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant__ 
                             p.hcur[o] = h;
                             if (ph.hidden_out) ph.hidden_out[o] = h;
                             sq = h * h;
-                            ch_store_hi_lo(ph.xt_k + o, (size_t)p.n_rs * p.d, h - h0);
+                            ch_store_hi_lo(ph.xt_k + o, (size_t)p.lo_xt * p.d, h - h0);
                             if (ph.xt16_k) ph.xt16_k[o] = __float2half_rn(h - h0);
-                            if (ph.xg_next) ch_store_hi_lo(ph.xg_next + o, (size_t)p.M * p.d, h * __bfloat162float(ph.gamma_next[j]));
+                            if (ph.xg_next) ch_store_hi_lo(ph.xg_next + o, (size_t)p.lo_x * p.d, h * __bfloat162float(ph.gamma_next[j]));
                         }
                         sq_s[e] = sq;
                     }
@@ -459,6 +460,7 @@ cudaError_t sk_chain(Ctx *c, int M, int K, const mrp_draft_out &out, cudaStream_
     memset(&maps, 0, sizeof(maps));
     const int n_rs = (K + 1) * M;
     p.n_phases = 2 * K; p.M = M; p.d = d; p.F = F; p.n_rs = n_rs; p.eps = c->cfg.rms_eps;
+    p.lo_x = c->lo_x; p.lo_xt = c->lo_xt;
     p.act = (__nv_bfloat16 *)(c->ws + c->lay.act);
     p.hcur = (float *)(c->ws + c->lay.hcur); p.h0f = (const float *)(c->ws + c->lay.h0f);
     p.sumsq = (float *)(c->ws + c->lay.sumsq);
@@ -484,8 +486,8 @@ cudaError_t sk_chain(Ctx *c, int M, int K, const mrp_draft_out &out, cudaStream_
     };
     __nv_bfloat16 *xg = (__nv_bfloat16 *)(c->ws + c->lay.xg);
     __nv_bfloat16 *xt = (__nv_bfloat16 *)(c->ws + c->lay.xt);
-    if (!make_map(s, &maps.m[0], xg, d, 2 * (uint64_t)M, r_pad) ||
-        !make_map(s, &maps.m[1], p.act, F, 2 * (uint64_t)M, r_pad))
+    if (!make_map(s, &maps.m[0], xg, d, 2 * (uint64_t)r_pad, 2 * r_pad) ||
+        !make_map(s, &maps.m[1], p.act, F, 2 * (uint64_t)r_pad, 2 * r_pad))
         return note_err(c, cudaErrorInvalidValue, "tensor map (head chain, activations)");
     for (int k = 1; k <= K; ++k) {
         const mrp_head_weights &hw = c->heads[k - 1];

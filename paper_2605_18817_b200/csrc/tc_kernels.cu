@@ -329,7 +329,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 // Gather masked rows: fp32 copies of h_0, the first head's operand bf16(h_0 * gamma_1), the
 // row sums of squares, and the zero rows that stand for step 0 in the stacked LM-head operand.
 __global__ void tc_prep_kernel(const __nv_bfloat16 *__restrict__ hidden, const int32_t *__restrict__ row_index,
-                               int d, int M, int n_rs, const __nv_bfloat16 *__restrict__ gamma1,
+                               int d, int lo_x, int lo_xt, const __nv_bfloat16 *__restrict__ gamma1,
                                float *__restrict__ h0f, float *__restrict__ hcur, __nv_bfloat16 *__restrict__ xg,
                                __nv_bfloat16 *__restrict__ xt0, float *__restrict__ sumsq,
                                int32_t *__restrict__ counters, int n_counters)
@@ -352,10 +352,10 @@ __global__ void tc_prep_kernel(const __nv_bfloat16 *__restrict__ hidden, const i
             const float x = v * __bfloat162float(gamma1[j]);
             const __nv_bfloat16 hi = __float2bfloat16_rn(x);
             xg[o] = hi;
-            xg[(size_t)M * d + o] = __float2bfloat16_rn(x - __bfloat162float(hi));
+            xg[(size_t)lo_x * d + o] = __float2bfloat16_rn(x - __bfloat162float(hi));
         }
         xt0[o] = __float2bfloat16(0.f);
-        xt0[(size_t)n_rs * d + o] = __float2bfloat16(0.f);
+        xt0[(size_t)lo_xt * d + o] = __float2bfloat16(0.f);
         ss = fmaf(v, v, ss);
     }
 #pragma unroll
@@ -523,20 +523,24 @@ cudaError_t tc_draft(Ctx *c, const void *hidden, const float *logits0, const int
         return note_err(c, cudaErrorInvalidValue, "workspace slices");
     const int n_mb = (M + 127) / 128;
 
-    prof_mark(c, 0, st);
     const int n_rs = (K + 1) * M;
+    // which kernel family runs the head chain and the LM head of this call
+    const bool pdl = !(c->cfg.flags & MRP_FLAG_NO_PDL);
+    const bool few_rows = sk_head_rows_ok(M) && sk_heads_ok(c->cfg) &&
+                          !(c->cfg.flags & MRP_FLAG_ROW_MAJOR_ONLY);
+    const bool lm_few = sk_rows_ok(n_rs) && !(c->cfg.flags & MRP_FLAG_ROW_MAJOR_ONLY);
+    const bool f16_lm = c->use_f16_lm && n_rs >= kF16MinRowSteps && !lm_few;
+    c->lo_x = few_rows ? sk_head_pad(M) : M;
+    c->lo_xt = lm_few ? sk_lm_pad(n_rs) : n_rs;
+
+    prof_mark(c, 0, st);
     cudaError_t e = note_err(c, launch_k(tc_prep_kernel, dim3(M), dim3(256), 0, st, !(c->cfg.flags & MRP_FLAG_NO_PDL),
-                                         (const __nv_bfloat16 *)hidden, row_index, d, M, n_rs,
+                                         (const __nv_bfloat16 *)hidden, row_index, d, c->lo_x, c->lo_xt,
                                       (const __nv_bfloat16 *)c->heads[0].rms_gamma, h0f, hcur, xg, xt, sumsq,
                                       (int32_t *)(c->ws + c->lay.sk_counters), kSkMaxTiles), "tc_prep_kernel");
     c->launches++;
     if (e != cudaSuccess) return e;
 
-    const bool pdl = !(c->cfg.flags & MRP_FLAG_NO_PDL);
-    const bool f16_lm = c->use_f16_lm && (K + 1) * M >= kF16MinRowSteps &&
-                        !(sk_rows_ok((K + 1) * M) && !(c->cfg.flags & MRP_FLAG_ROW_MAJOR_ONLY));
-    const bool few_rows = sk_head_rows_ok(M) && sk_heads_ok(c->cfg) &&
-                          !(c->cfg.flags & MRP_FLAG_ROW_MAJOR_ONLY);
     int n_ss = 1;
     bool chain_done = false;
     if (few_rows && !(c->cfg.flags & MRP_FLAG_NO_CHAIN)) {
@@ -592,7 +596,7 @@ cudaError_t tc_draft(Ctx *c, const void *hidden, const float *logits0, const int
     }
     prof_mark(c, 1, st);
     int n_slices = G;
-    if (sk_rows_ok(n_rs) && !(c->cfg.flags & MRP_FLAG_ROW_MAJOR_ONLY)) {
+    if (lm_few) {
         e = sk_lm(c, logits0, row_index, M, K, out, st, pdl);
         if (e != cudaSuccess) return e;
     } else {

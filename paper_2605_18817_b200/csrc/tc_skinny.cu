@@ -47,7 +47,7 @@ struct SkParams {
     int n_stages;
     int r_pad;           // activation rows per part (16 or 32); MMA N = 2 * r_pad
     int tmem_cols;       // allocated TMEM columns (power of two >= 2 buffers * 2 * r_pad)
-    int x_row_hi, x_row_lo;
+    int lo_x, lo_xt;     // row offset of the lo block in the head operands / the LM-head operand
     int lm_h[4];         // LM: tile heights (units) other than 8, fetched through maps w[1], w[2], w[4], w[5]
     int n_split;         // GU/DN: CTAs sharing one 128-row weight tile, each a slice of the contraction
     int w_rows;          // GU/DN: weight rows (gate rows for GU)
@@ -177,8 +177,8 @@ sk_gemm_kernel(const __grid_constant__ SkMaps maps, const SkParams p)
             };
             auto load_x = [&](int kk, int s) {
                 const uint32_t sx = base + (uint32_t)s * stage_bytes + kWTile;
-                tma_load_2d_hint(sx, &maps.x, (kc0 + kk) * kBK, p.x_row_hi, full_bar(s), pol_x);
-                tma_load_2d_hint(sx + RP * 128, &maps.x, (kc0 + kk) * kBK, p.x_row_lo, full_bar(s), pol_x);
+                // one box: RP hi rows, then (the lo block starts at row RP of the buffer) RP lo rows
+                tma_load_2d_hint(sx, &maps.x, (kc0 + kk) * kBK, 0, full_bar(s), pol_x);
             };
             // weights do not depend on the previous kernel: fill the ring with them first
             int t = 0, kk = 0;
@@ -432,7 +432,7 @@ sk_gemm_kernel(const __grid_constant__ SkMaps maps, const SkParams p)
                                 if (c0 + j < p.M) {
                                     const float g = v[j] * rstd_s[c0 + j];
                                     const float av = g / (1.f + __expf(-g)) * exch_s[j * 64 + t];
-                                    store_hi_lo(p.act + (size_t)(c0 + j) * p.F + wrow, (size_t)p.M * p.F, av);
+                                    store_hi_lo(p.act + (size_t)(c0 + j) * p.F + wrow, (size_t)p.lo_x * p.F, av);
                                 }
                             }
                         }
@@ -450,9 +450,9 @@ sk_gemm_kernel(const __grid_constant__ SkMaps maps, const SkParams p)
                                     p.hcur[o] = h;
                                     if (p.hidden_out) p.hidden_out[o] = h;
                                     sq[j] = h * h;
-                                    store_hi_lo(p.xt_k + o, (size_t)p.n_rs * p.d, h - h0v[j]);
+                                    store_hi_lo(p.xt_k + o, (size_t)p.lo_xt * p.d, h - h0v[j]);
                                     if (p.xt16_k) p.xt16_k[o] = __float2half_rn(h - h0v[j]);
-                                    if (p.xg_next) store_hi_lo(p.xg_next + o, (size_t)p.M * p.d, h * gm);
+                                    if (p.xg_next) store_hi_lo(p.xg_next + o, (size_t)p.lo_x * p.d, h * gm);
                                 }
                             }
                         }
@@ -595,17 +595,20 @@ cudaError_t sk_launch_rp(const SkMaps &maps, const SkParams &p, int grid, cudaSt
     }
 }
 
-int sk_head_pad(int M) { return M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : 128; }
-
 void sk_common(Ctx *c, SkParams &p, int M, int K, const mrp_draft_out &out)
 {
     memset(&p, 0, sizeof(p));
     p.M = M; p.K = K; p.V = c->cfg.vocab; p.d = c->cfg.d; p.F = c->cfg.d_ff; p.n_rs = (K + 1) * M;
     p.status = (int32_t *)(c->ws + c->lay.status);
     p.user_status = out.status;
+    p.lo_x = c->lo_x; p.lo_xt = c->lo_xt;
 }
 
 }  // namespace
+
+int sk_head_pad(int M) { return M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : 128; }
+
+int sk_lm_pad(int n_rs) { return n_rs <= 16 ? 16 : 32; }
 
 bool sk_rows_ok(int rows) { return rows >= 1 && rows <= 32; }
 
@@ -623,7 +626,6 @@ cudaError_t sk_gateup(Ctx *c, int k, int M, int K, int n_ss, const mrp_draft_out
     SkParams p;
     sk_common(c, p, M, K, out);
     p.units_total = F / 8; p.k_chunks = d / kBK; p.r_pad = sk_head_pad(M); p.w_rows = F;
-    p.x_row_hi = 0; p.x_row_lo = M;
     p.sumsq = (const float *)(c->ws + c->lay.sumsq); p.n_ss = n_ss; p.eps = c->cfg.rms_eps;
     p.act = (__nv_bfloat16 *)(c->ws + c->lay.act);
     sk_finish_shape(p, 0);
@@ -631,7 +633,7 @@ cudaError_t sk_gateup(Ctx *c, int k, int M, int K, int n_ss, const mrp_draft_out
     (void)G;
     SkMaps maps;
     memset(&maps, 0, sizeof(maps));
-    if (!make_map(s, &maps.x, c->ws + c->lay.xg, d, 2 * (uint64_t)M, p.r_pad) ||
+    if (!make_map(s, &maps.x, c->ws + c->lay.xg, d, 2 * (uint64_t)p.r_pad, 2 * p.r_pad) ||
         !sk_weight_maps(s, maps, 0, hw.w_gate, d, F, 8, p) || !sk_weight_maps(s, maps, 1, hw.w_up, d, F, 8, p))
         return note_err(c, cudaErrorInvalidValue, "tensor map (gate/up, few rows)");
     c->launches++;
@@ -647,7 +649,6 @@ cudaError_t sk_down(Ctx *c, int k, int M, int K, const mrp_draft_out &out, cudaS
     SkParams p;
     sk_common(c, p, M, K, out);
     p.units_total = d / 16; p.k_chunks = F / kBK; p.r_pad = sk_head_pad(M); p.w_rows = d;
-    p.x_row_hi = 0; p.x_row_lo = M;
     p.hcur = (float *)(c->ws + c->lay.hcur); p.h0f = (const float *)(c->ws + c->lay.h0f);
     p.gamma_next = (k < K) ? (const __nv_bfloat16 *)c->heads[k].rms_gamma : nullptr;
     p.xg_next = (k < K) ? (__nv_bfloat16 *)(c->ws + c->lay.xg) : nullptr;
@@ -662,7 +663,7 @@ cudaError_t sk_down(Ctx *c, int k, int M, int K, const mrp_draft_out &out, cudaS
     (void)G;
     SkMaps maps;
     memset(&maps, 0, sizeof(maps));
-    if (!make_map(s, &maps.x, c->ws + c->lay.act, F, 2 * (uint64_t)M, p.r_pad) ||
+    if (!make_map(s, &maps.x, c->ws + c->lay.act, F, 2 * (uint64_t)p.r_pad, 2 * p.r_pad) ||
         !sk_weight_maps(s, maps, 0, hw.w_down, F, d, 16, p))
         return note_err(c, cudaErrorInvalidValue, "tensor map (down, few rows)");
     c->launches++;
@@ -676,14 +677,13 @@ cudaError_t sk_lm(Ctx *c, const float *logits0, const int32_t *row_index, int M,
     const int d = c->cfg.d, V = c->cfg.vocab, G = c->sm_count;
     SkParams p;
     sk_common(c, p, M, K, out);
-    p.units_total = V / 16; p.k_chunks = d / kBK; p.r_pad = p.n_rs <= 16 ? 16 : 32;
-    p.x_row_hi = 0; p.x_row_lo = p.n_rs;
+    p.units_total = V / 16; p.k_chunks = d / kBK; p.r_pad = sk_lm_pad(p.n_rs);
     p.logits0 = logits0; p.row_index = row_index;
     p.partials = (Partial *)(c->ws + c->lay.partials); p.logits_out = out.logits_out;
     sk_finish_shape(p, G);
     SkMaps maps;
     memset(&maps, 0, sizeof(maps));
-    if (!make_map(s, &maps.x, c->ws + c->lay.xt, d, 2 * (uint64_t)p.n_rs, p.r_pad) ||
+    if (!make_map(s, &maps.x, c->ws + c->lay.xt, d, 2 * (uint64_t)p.r_pad, 2 * p.r_pad) ||
         !sk_weight_maps(s, maps, 0, c->w_lm, d, V, 16, p))
         return note_err(c, cudaErrorInvalidValue, "tensor map (LM head, few rows)");
     c->launches++;
