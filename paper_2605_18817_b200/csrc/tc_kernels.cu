@@ -21,6 +21,8 @@
 #include <cuda_fp16.h>
 #include <string.h>
 
+#include <atomic>
+
 #include <new>
 
 #include "tc_common.cuh"
@@ -443,11 +445,16 @@ cudaError_t launch_tc(const CUtensorMap &a, const CUtensorMap &b0, const CUtenso
 {
     auto kern = tc_gemm_kernel<KIND, MARGIN, F16>;
     const size_t smem = smem_bytes(p, F16 ? 1 : 2);
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
-        if (e != cudaSuccess) return e;
-        attr_set = true;
+    // the shared-memory limit of a kernel is set once per device (the attribute is per device)
+    static std::atomic<unsigned long long> attr_devices{0};
+    int dev = 0;
+    cudaError_t ea = cudaGetDevice(&dev);
+    if (ea != cudaSuccess) return ea;
+    const unsigned long long bit = 1ull << (dev & 63);
+    if (!(attr_devices.load() & bit)) {
+        ea = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
+        if (ea != cudaSuccess) return ea;
+        attr_devices.fetch_or(bit);
     }
     kern<<<grid, kThreads, smem, st>>>(a, b0, b1, p);
     return cudaGetLastError();

@@ -19,6 +19,8 @@
 #include <cuda_fp16.h>
 #include <string.h>
 
+#include <atomic>
+
 #include "tc_common.cuh"
 
 namespace mrp {
@@ -558,11 +560,16 @@ template <int KIND, int RP, bool MARGIN>
 cudaError_t sk_launch(const SkMaps &maps, const SkParams &p, int grid, cudaStream_t st, bool pdl)
 {
     auto kern = sk_gemm_kernel<KIND, RP, MARGIN>;
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
-        if (e != cudaSuccess) return e;
-        attr_set = true;
+    // the shared-memory limit of a kernel is set once per device (the attribute is per device)
+    static std::atomic<unsigned long long> attr_devices{0};
+    int dev = 0;
+    cudaError_t ea = cudaGetDevice(&dev);
+    if (ea != cudaSuccess) return ea;
+    const unsigned long long bit = 1ull << (dev & 63);
+    if (!(attr_devices.load() & bit)) {
+        ea = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
+        if (ea != cudaSuccess) return ea;
+        attr_devices.fetch_or(bit);
     }
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));
