@@ -24,7 +24,7 @@ WorkspaceLayout workspace_layout(const mrp_config &cfg)
     l.act = take((rows + 64) * F * 4);
     l.xt = take((steps * rows + 32) * d * 4);
     l.sumsq = take((size_t)kSumsqSlices * rows * 4);
-    const int v_slices = (cfg.vocab + kSimtSliceV - 1) / kSimtSliceV;
+    const int v_slices = (cfg.vocab + 31) / 32;      // the narrowest slicing of the CUDA-core LM head
     l.n_slices_max = v_slices < kSimtMaxBlocks ? v_slices : kSimtMaxBlocks;
     if (l.n_slices_max < kSumsqSlices) l.n_slices_max = kSumsqSlices;   // one slice per CTA (tc family)
     l.partials = take((size_t)l.n_slices_max * steps * rows * sizeof(Partial));

@@ -29,6 +29,8 @@ template <typename T>
 __global__ void prep_kernel(const T *__restrict__ hidden, const int32_t *__restrict__ row_index,
                             int d, float *__restrict__ h0f, float *__restrict__ hcur)
 {
+    pdl_trigger();
+    pdl_wait();
     const int m = blockIdx.x;
     const size_t row = row_index ? (size_t)row_index[m] : (size_t)m;
     for (int j = threadIdx.x; j < d; j += blockDim.x) {
@@ -42,13 +44,15 @@ cudaError_t launch_prep(Ctx *c, const void *hidden, const int32_t *row_index, in
 {
     if (M == 0) return cudaSuccess;
     float *h0f = (float *)(c->ws + c->lay.h0f), *hcur = (float *)(c->ws + c->lay.hcur);
+    const bool pdl = !(c->cfg.flags & MRP_FLAG_NO_PDL);
+    cudaError_t e;
     if (c->cfg.dtype == MRP_F32)
-        prep_kernel<float><<<M, 256, 0, st>>>((const float *)hidden, row_index, c->cfg.d, h0f, hcur);
+        e = launch_k(prep_kernel<float>, dim3(M), dim3(256), 0, st, pdl, (const float *)hidden, row_index, c->cfg.d, h0f, hcur);
     else
-        prep_kernel<__nv_bfloat16><<<M, 256, 0, st>>>((const __nv_bfloat16 *)hidden, row_index,
-                                                      c->cfg.d, h0f, hcur);
+        e = launch_k(prep_kernel<__nv_bfloat16>, dim3(M), dim3(256), 0, st, pdl, (const __nv_bfloat16 *)hidden, row_index,
+                     c->cfg.d, h0f, hcur);
     c->launches++;
-    return cudaGetLastError();
+    return e;
 }
 
 // ---- a1: RMSNorm of the residual stream --------------------------------------------------
@@ -56,6 +60,8 @@ template <typename T>
 __global__ void rmsnorm_kernel(const float *__restrict__ hcur, const T *__restrict__ gamma, int d,
                                float eps, float *__restrict__ xg)
 {
+    pdl_trigger();
+    pdl_wait();
     __shared__ float red[32];
     const int m = blockIdx.x;
     const float *h = hcur + (size_t)m * d;
@@ -83,6 +89,8 @@ __global__ void gateup_kernel(const T *__restrict__ w_gate, const T *__restrict_
                               const float *__restrict__ xg, int M, int d, int F,
                               float *__restrict__ act)
 {
+    pdl_trigger();
+    pdl_wait();
     const int f = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (f >= F) return;
@@ -117,6 +125,8 @@ __global__ void down_kernel(const T *__restrict__ w_down, const float *__restric
                             int d, int F, float *__restrict__ hcur, const float *__restrict__ h0f,
                             float *__restrict__ xt_k, float *__restrict__ hidden_out)
 {
+    pdl_trigger();
+    pdl_wait();
     const int j = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (j >= d) return;
@@ -146,28 +156,30 @@ __global__ void down_kernel(const T *__restrict__ w_down, const float *__restric
 }
 
 // ---- a2 + a3: LM head on the residual, added to l_0, per-slice softmax statistics ---------
-// A block owns vocabulary slices of kSimtSliceV entries (grid-stride over slices).  For each
+// A block owns vocabulary slices of SLICE (128, or 32 for small vocabularies) entries (grid-stride over slices).  For each
 // chunk of kLR row-steps rs = k*M + m, the 8 warps compute delta for 16 entries each, the
 // tile l = l_0 + delta goes to shared memory, and warp w reduces row-step w of the chunk.
 constexpr int kLR = 8;
 
-template <typename T>
+template <typename T, int SLICE>
 __global__ void __launch_bounds__(256)
 lm_simt_kernel(const T *__restrict__ w_lm, const float *__restrict__ xt,
                const float *__restrict__ logits0, const int32_t *__restrict__ row_index, int M,
                int K, int d, int V, int n_slices, Partial *__restrict__ partials,
                float *__restrict__ logits_out)
 {
-    __shared__ float tile[kLR][kSimtSliceV];
+    pdl_trigger();
+    pdl_wait();
+    __shared__ float tile[kLR][SLICE];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n_rs = (K + 1) * M;
     bool first = true;
     for (int slice = blockIdx.x; slice < n_slices; slice += gridDim.x, first = false) {
-        const int v0 = slice * kSimtSliceV;
+        const int v0 = slice * SLICE;
         for (int rs0 = 0; rs0 < n_rs; rs0 += kLR) {
             // delta for entries v0 + warp*16 .. +16, row-steps rs0 .. rs0+kLR
-            for (int e = 0; e < kSimtSliceV / 8; ++e) {
-                const int vl = warp * (kSimtSliceV / 8) + e;
+            for (int e = 0; e < SLICE / 8; ++e) {
+                const int vl = warp * (SLICE / 8) + e;
                 const int v = v0 + vl;
                 float acc[kLR];
 #pragma unroll
@@ -204,9 +216,9 @@ lm_simt_kernel(const T *__restrict__ w_lm, const float *__restrict__ xt,
             if (rs < n_rs) {
                 float mx = -INFINITY, sec = -INFINITY;
                 int idx = INT_MAX;
-                float vals[kSimtSliceV / 32];
+                float vals[SLICE / 32];
 #pragma unroll
-                for (int i = 0; i < kSimtSliceV / 32; ++i) {
+                for (int i = 0; i < SLICE / 32; ++i) {
                     const int vl = lane + 32 * i;
                     const float l = tile[warp][vl];
                     vals[i] = l;
@@ -229,12 +241,12 @@ lm_simt_kernel(const T *__restrict__ w_lm, const float *__restrict__ xt,
                 }
                 float sum = 0.f;
 #pragma unroll
-                for (int i = 0; i < kSimtSliceV / 32; ++i)
+                for (int i = 0; i < SLICE / 32; ++i)
                     sum += (vals[i] == -INFINITY) ? 0.f : expf(vals[i] - mx);
                 sum = warp_sum(sum);
                 if (logits_out && rs >= M) {
 #pragma unroll
-                    for (int i = 0; i < kSimtSliceV / 32; ++i) {
+                    for (int i = 0; i < SLICE / 32; ++i) {
                         const int v = v0 + lane + 32 * i;
                         if (v < V) logits_out[(size_t)(rs - M) * V + v] = vals[i];
                     }
@@ -338,6 +350,7 @@ static cudaError_t simt_draft_t(Ctx *c, const void *hidden, const float *logits0
     float *xt = (float *)(c->ws + c->lay.xt);
     Partial *partials = (Partial *)(c->ws + c->lay.partials);
     int32_t *status = (int32_t *)(c->ws + c->lay.status);
+    const bool pdl = !(c->cfg.flags & MRP_FLAG_NO_PDL);
     prof_mark(c, 0, st);
     cudaError_t e = launch_prep(c, hidden, row_index, M, st);
     if (e != cudaSuccess) return e;
@@ -345,20 +358,31 @@ static cudaError_t simt_draft_t(Ctx *c, const void *hidden, const float *logits0
         cudaMemcpyAsync(out.hidden_out, h0f, sizeof(float) * (size_t)M * d, cudaMemcpyDeviceToDevice, st);
     for (int k = 1; k <= K; ++k) {
         const mrp_head_weights &hw = c->heads[k - 1];
-        rmsnorm_kernel<T><<<M, 256, 0, st>>>(hcur, (const T *)hw.rms_gamma, d, c->cfg.rms_eps, xg);
-        gateup_kernel<T><<<(F + 7) / 8, 256, 0, st>>>((const T *)hw.w_gate, (const T *)hw.w_up, xg, M, d, F, act);
-        down_kernel<T><<<(d + 7) / 8, 256, 0, st>>>((const T *)hw.w_down, act, M, d, F, hcur, h0f,
-                                                    xt + (size_t)(k - 1) * M * d,
-                                                    (k == K) ? out.hidden_out : nullptr);
+        e = launch_k(rmsnorm_kernel<T>, dim3(M), dim3(256), 0, st, pdl, (const float *)hcur, (const T *)hw.rms_gamma, d,
+                     c->cfg.rms_eps, xg);
+        if (e == cudaSuccess)
+            e = launch_k(gateup_kernel<T>, dim3((F + 7) / 8), dim3(256), 0, st, pdl, (const T *)hw.w_gate,
+                         (const T *)hw.w_up, (const float *)xg, M, d, F, act);
+        if (e == cudaSuccess)
+            e = launch_k(down_kernel<T>, dim3((d + 7) / 8), dim3(256), 0, st, pdl, (const T *)hw.w_down,
+                         (const float *)act, M, d, F, hcur, (const float *)h0f, xt + (size_t)(k - 1) * M * d,
+                         (k == K) ? out.hidden_out : (float *)nullptr);
+        if (e != cudaSuccess) return e;
         c->launches += 3;
     }
     prof_mark(c, 1, st);
-    const int n_slices = (V + kSimtSliceV - 1) / kSimtSliceV;
+    // small vocabularies: narrower slices so that every SM gets a block
+    const bool narrow = (V + kSimtSliceV - 1) / kSimtSliceV < 2 * c->sm_count;
+    const int slice_v = narrow ? 32 : kSimtSliceV;
+    const int n_slices = (V + slice_v - 1) / slice_v;
     const int grid = n_slices < kSimtMaxBlocks ? n_slices : kSimtMaxBlocks;
-    lm_simt_kernel<T><<<grid, 256, 0, st>>>((const T *)c->w_lm, xt, logits0, row_index, M, K, d, V,
-                                            n_slices, partials, out.logits_out);
+    if (narrow)
+        e = launch_k(lm_simt_kernel<T, 32>, dim3(grid), dim3(256), 0, st, pdl, (const T *)c->w_lm, (const float *)xt,
+                     logits0, row_index, M, K, d, V, n_slices, partials, out.logits_out);
+    else
+        e = launch_k(lm_simt_kernel<T, kSimtSliceV>, dim3(grid), dim3(256), 0, st, pdl, (const T *)c->w_lm,
+                     (const float *)xt, logits0, row_index, M, K, d, V, n_slices, partials, out.logits_out);
     c->launches++;
-    e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     prof_mark(c, 2, st);
     e = launch_combine(c, partials, grid, (K + 1) * M, out, status, st);
