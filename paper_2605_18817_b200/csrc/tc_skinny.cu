@@ -47,6 +47,7 @@ struct SkParams {
     int units_total;     // weight rows / 16 (GU: gate rows / 8, a unit = 8 gate + 8 up rows)
     int k_chunks;        // contraction extent / 64
     int n_stages;
+    int kc;              // 64-element k-chunks per ring stage
     int r_pad;           // activation rows per part (16 or 32); MMA N = 2 * r_pad
     int tmem_cols;       // allocated TMEM columns (power of two >= 2 buffers * 2 * r_pad)
     int lo_x, lo_xt;     // row offset of the lo block in the head operands / the LM-head operand
@@ -90,14 +91,16 @@ __device__ __forceinline__ void store_hi_lo(__nv_bfloat16 *dst, size_t lo_off, f
     dst[lo_off] = __float2bfloat16_rn(v - __bfloat162float(hi));
 }
 
-template <int KIND, int RP, bool MARGIN>
+// KC: 64-element k-chunks per ring stage (2 for the LM head: fewer, larger stages stream better).
+template <int KIND, int RP, bool MARGIN, int KC>
 __global__ void __launch_bounds__(kSkThreads, 1)
 sk_gemm_kernel(const __grid_constant__ SkMaps maps, const SkParams p)
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     constexpr int x_bytes = 2 * RP * 128;            // hi rows then lo rows of one k-chunk
-    constexpr int stage_bytes = kWTile + x_bytes;
+    constexpr int sub_bytes = kWTile + x_bytes;      // one k-chunk: weight tile, then activation rows
+    constexpr int stage_bytes = KC * sub_bytes;
     const uint32_t bars = base + (uint32_t)p.n_stages * stage_bytes;
     auto full_bar = [&](int s) { return bars + 8u * s; };
     auto empty_bar = [&](int s) { return bars + 8u * (p.n_stages + s); };
@@ -126,7 +129,7 @@ sk_gemm_kernel(const __grid_constant__ SkMaps maps, const SkParams p)
         kc0 = (cta % p.n_split) * cps;
         kc1 = min(p.k_chunks, kc0 + cps);
     }
-    const int nk = kc1 - kc0;
+    const int nk = (kc1 - kc0) / KC;                 // ring stages per tile
     // The range is cut into the fewest tiles of at most 8 units and the tiles are made equally
     // high (an MMA costs the same at any height, so a short extra tile would cost a full one):
     // the first t_extra tiles have t_base + 1 units, the others t_base.
@@ -168,19 +171,25 @@ sk_gemm_kernel(const __grid_constant__ SkMaps maps, const SkParams p)
             auto load_w = [&](int t, int kk, int s) {
                 const uint32_t sw = base + (uint32_t)s * stage_bytes;
                 const int h = tile_units(t);
-                mbar_expect_tx(full_bar(s), (uint32_t)h * 2048u + (uint32_t)x_bytes);
+                mbar_expect_tx(full_bar(s), (uint32_t)KC * ((uint32_t)h * 2048u + (uint32_t)x_bytes));
                 const int ut = tile_start(t);
-                if (KIND == SK_GU) {
-                    tma_load_2d_hint(sw, &maps.w[0], (kc0 + kk) * kBK, ut * 8, full_bar(s), pol_w);
-                    tma_load_2d_hint(sw + 64 * 128, &maps.w[3], (kc0 + kk) * kBK, ut * 8, full_bar(s), pol_w);
-                } else {
-                    tma_load_2d_hint(sw, &maps.w[tile_map(h)], (kc0 + kk) * kBK, ut * 16, full_bar(s), pol_w);
+#pragma unroll
+                for (int b = 0; b < KC; ++b) {
+                    const int kx = (kc0 + kk * KC + b) * kBK;
+                    if (KIND == SK_GU) {
+                        tma_load_2d_hint(sw + b * sub_bytes, &maps.w[0], kx, ut * 8, full_bar(s), pol_w);
+                        tma_load_2d_hint(sw + b * sub_bytes + 64 * 128, &maps.w[3], kx, ut * 8, full_bar(s), pol_w);
+                    } else {
+                        tma_load_2d_hint(sw + b * sub_bytes, &maps.w[tile_map(h)], kx, ut * 16, full_bar(s), pol_w);
+                    }
                 }
             };
             auto load_x = [&](int kk, int s) {
                 const uint32_t sx = base + (uint32_t)s * stage_bytes + kWTile;
-                // one box: RP hi rows, then (the lo block starts at row RP of the buffer) RP lo rows
-                tma_load_2d_hint(sx, &maps.x, (kc0 + kk) * kBK, 0, full_bar(s), pol_x);
+                // one box per k-chunk: RP hi rows, then (the lo block starts at row RP of the buffer) RP lo rows
+#pragma unroll
+                for (int b = 0; b < KC; ++b)
+                    tma_load_2d_hint(sx + b * sub_bytes, &maps.x, (kc0 + kk * KC + b) * kBK, 0, full_bar(s), pol_x);
             };
             // weights do not depend on the previous kernel: fill the ring with them first
             int t = 0, kk = 0;
@@ -218,11 +227,14 @@ sk_gemm_kernel(const __grid_constant__ SkMaps maps, const SkParams p)
                     if (!mbar_wait(full_bar(s), ph, abort_flag, p)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t sw = base + (uint32_t)s * stage_bytes;
-                    const uint64_t dw = make_smem_desc(sw);
-                    const uint64_t dx = make_smem_desc(sw + kWTile);
 #pragma unroll
-                    for (int k4 = 0; k4 < kBK / 16; ++k4)
-                        umma_bf16(dt, dw + 2u * k4, dx + 2u * k4, idesc, (kk > 0 || k4 > 0) ? 1u : 0u);
+                    for (int b = 0; b < KC; ++b) {
+                        const uint64_t dw = make_smem_desc(sw + b * sub_bytes);
+                        const uint64_t dx = make_smem_desc(sw + b * sub_bytes + kWTile);
+#pragma unroll
+                        for (int k4 = 0; k4 < kBK / 16; ++k4)
+                            umma_bf16(dt, dw + 2u * k4, dx + 2u * k4, idesc, (kk > 0 || b > 0 || k4 > 0) ? 1u : 0u);
+                    }
                     umma_commit(empty_bar(s));
                     if (++s == p.n_stages) { s = 0; ph ^= 1u; }
                 }
@@ -500,14 +512,15 @@ sk_gemm_kernel(const __grid_constant__ SkMaps maps, const SkParams p)
 // ---------------------------------------------------------------------------------------
 size_t sk_smem_bytes(const SkParams &p)
 {
-    const int stage = kWTile + 2 * p.r_pad * 128;
+    const int stage = p.kc * (kWTile + 2 * p.r_pad * 128);
     return (size_t)p.n_stages * stage + 1024 + 8 * (2 * p.n_stages + 4) + 16 + kAuxBytes;
 }
 
 void sk_finish_shape(SkParams &p, int grid)
 {
     // the ring always takes all the shared memory there is: it also parks the LM statistics
-    const int stage = kWTile + 2 * p.r_pad * 128;
+    if (p.kc < 1) p.kc = 1;
+    const int stage = p.kc * (kWTile + 2 * p.r_pad * 128);
     int ns = (kSmemBudget - 1024 - 256 - 16 - kAuxBytes) / stage;
     if (ns > 12) ns = 12;
     p.n_stages = ns;
@@ -556,10 +569,10 @@ bool sk_weight_maps(const TcState *s, SkMaps &maps, int part, const void *w, uin
     return true;
 }
 
-template <int KIND, int RP, bool MARGIN>
+template <int KIND, int RP, bool MARGIN, int KC = 1>
 cudaError_t sk_launch(const SkMaps &maps, const SkParams &p, int grid, cudaStream_t st, bool pdl)
 {
-    auto kern = sk_gemm_kernel<KIND, RP, MARGIN>;
+    auto kern = sk_gemm_kernel<KIND, RP, MARGIN, KC>;
     // the shared-memory limit of a kernel is set once per device (the attribute is per device)
     static std::atomic<unsigned long long> attr_devices{0};
     int dev = 0;
@@ -596,6 +609,11 @@ cudaError_t sk_launch_rp(const SkMaps &maps, const SkParams &p, int grid, cudaSt
         default: return sk_launch<KIND, 128, false>(maps, p, grid, st, pdl);
         }
     } else {
+        if (p.kc == 2) {
+            if (p.r_pad == 16)
+                return margin ? sk_launch<KIND, 16, true, 2>(maps, p, grid, st, pdl) : sk_launch<KIND, 16, false, 2>(maps, p, grid, st, pdl);
+            return margin ? sk_launch<KIND, 32, true, 2>(maps, p, grid, st, pdl) : sk_launch<KIND, 32, false, 2>(maps, p, grid, st, pdl);
+        }
         if (p.r_pad == 16)
             return margin ? sk_launch<KIND, 16, true>(maps, p, grid, st, pdl) : sk_launch<KIND, 16, false>(maps, p, grid, st, pdl);
         return margin ? sk_launch<KIND, 32, true>(maps, p, grid, st, pdl) : sk_launch<KIND, 32, false>(maps, p, grid, st, pdl);
@@ -685,6 +703,7 @@ cudaError_t sk_lm(Ctx *c, const float *logits0, const int32_t *row_index, int M,
     SkParams p;
     sk_common(c, p, M, K, out);
     p.units_total = V / 16; p.k_chunks = d / kBK; p.r_pad = sk_lm_pad(p.n_rs);
+    p.kc = (p.k_chunks % 2 == 0) ? 2 : 1;
     p.logits0 = logits0; p.row_index = row_index;
     p.partials = (Partial *)(c->ws + c->lay.partials); p.logits_out = out.logits_out;
     sk_finish_shape(p, G);
