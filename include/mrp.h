@@ -246,6 +246,17 @@ int mrp_reveal_remask_noalloc(const float *conf, const int32_t *token, const int
                               const mrp_select_params *params, const mrp_select_out *out,
                               void *cuda_stream);
 
+/*
+ * Self-test of the bounded waits (no counterpart in the paper).  Every wait inside the kernels
+ * (on an mbarrier, on another CTA) gives up after a fixed number of cycles, raises
+ * MRP_DEV_TIMEOUT in the status word and lets the kernel return, so that a lost signal can never
+ * hang the GPU.  This call launches one thread that waits, with the same helper and the same
+ * limit (about 1.5 s) as the real kernels, for a barrier nobody completes.  After
+ * synchronising, *status (DEVICE int32, may be NULL) and the context's own status word carry
+ * MRP_DEV_TIMEOUT; the context stays usable.  Errors: INVALID_ARG, CUDA.
+ */
+int mrp_selftest_wait_timeout(mrp_ctx *ctx, int32_t *status, void *cuda_stream);
+
 /* Number of kernels the last mrp_draft / mrp_reveal_remask / mrp_verify call on this
  * context launched (for accounting in benchmarks). */
 int32_t mrp_last_launch_count(const mrp_ctx *ctx);

@@ -30,7 +30,7 @@ MRP_DEV_NONFINITE, MRP_DEV_TIMEOUT = 1, 2
 EXPORTS = ("mrp_workspace_bytes", "mrp_create", "mrp_destroy", "mrp_draft", "mrp_reveal_remask",
            "mrp_verify", "mrp_last_launch_count", "mrp_kernel_family", "mrp_status_string",
            "mrp_profile_enable", "mrp_profile_read", "mrp_last_error",
-           "mrp_reveal_remask_noalloc")
+           "mrp_reveal_remask_noalloc", "mrp_selftest_wait_timeout")
 MRP_NOALLOC_MAX_POSITIONS = 65536
 MRP_ERR_CAPACITY = 7
 
@@ -95,6 +95,8 @@ def _load():
                                       ctypes.POINTER(mrp_select_out), ctypes.c_void_p]
     lib.mrp_reveal_remask_noalloc.restype = ctypes.c_int
     lib.mrp_reveal_remask_noalloc.argtypes = lib.mrp_reveal_remask.argtypes[1:]
+    lib.mrp_selftest_wait_timeout.restype = ctypes.c_int
+    lib.mrp_selftest_wait_timeout.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
     lib.mrp_verify.restype = ctypes.c_int
     lib.mrp_verify.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
                                ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p,
@@ -282,6 +284,14 @@ def mrp_reveal_remask_noalloc(conf, token, row_index, M, K, B, L, mode, tau=0.9,
                                        _stream(stream))
     if rc != 0:
         raise MrpError("mrp_reveal_remask_noalloc", rc)
+
+
+def mrp_selftest_wait_timeout(ctx: Context, status, stream=None) -> None:
+    """Launch the bounded-wait self-test: after a sync, ``status`` carries MRP_DEV_TIMEOUT."""
+    _check(status, torch.int32, "status")
+    rc = lib.mrp_selftest_wait_timeout(ctx.handle, _ptr(status), _stream(stream))
+    if rc != 0:
+        raise MrpError("mrp_selftest_wait_timeout", rc)
 
 
 def mrp_verify(ctx: Context, draft_tok, verify_tok, draft_len, B, Kd, positionwise, accept_len,

@@ -263,6 +263,15 @@ int mrp_verify(mrp_ctx *ctx, const int32_t *draft_tok, const int32_t *verify_tok
     return e == cudaSuccess ? MRP_OK : MRP_ERR_CUDA;
 }
 
+int mrp_selftest_wait_timeout(mrp_ctx *ctx, int32_t *status, void *cuda_stream)
+{
+    if (!ctx) return MRP_ERR_INVALID_ARG;
+    Ctx &c = ctx->c;
+    DeviceGuard guard(c.cfg.device);
+    if (guard.err != cudaSuccess) return MRP_ERR_CUDA;
+    return tc_selftest_timeout(&c, status, (cudaStream_t)cuda_stream) == cudaSuccess ? MRP_OK : MRP_ERR_CUDA;
+}
+
 int32_t mrp_last_launch_count(const mrp_ctx *ctx) { return ctx ? ctx->c.launches : 0; }
 
 const char *mrp_last_error(const mrp_ctx *ctx) { return ctx ? ctx->c.err : ""; }

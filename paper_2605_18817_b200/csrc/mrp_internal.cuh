@@ -144,6 +144,9 @@ cudaError_t launch_verify(Ctx *c, const int32_t *draft_tok, const int32_t *verif
                           const int32_t *draft_len, int B, int Kd, int positionwise,
                           int32_t *accept_len, int8_t *accept_mask, cudaStream_t st);
 
+// Launches the bounded-wait self-test kernel (tc_kernels.cu).
+cudaError_t tc_selftest_timeout(Ctx *c, int32_t *user_status, cudaStream_t st);
+
 // ---- tensor-core kernel family (tc_*.cu) ---------------------------------------------
 bool tc_supported(const mrp_config &cfg, const mrp_head_weights *heads, const void *w_lm);
 cudaError_t tc_create(Ctx *c);

@@ -387,6 +387,20 @@ __global__ void to_half_kernel(const __nv_bfloat16 *__restrict__ src, __half *__
     if (bad) atomicOr(flag, 1);
 }
 
+// One thread waits for an mbarrier nobody completes: the bounded wait must give up and report.
+struct SelfTestParams { int32_t *status, *user_status; };
+__global__ void selftest_timeout_kernel(SelfTestParams p)
+{
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bar), 1);
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        mbar_wait(smem_u32(&bar), 0u, &abort_flag, p);
+    }
+}
+
 // ---------------------------------------------------------------------------------------
 // Host side
 // ---------------------------------------------------------------------------------------
@@ -461,6 +475,15 @@ cudaError_t launch_tc(const CUtensorMap &a, const CUtensorMap &b0, const CUtenso
 }
 
 }  // namespace
+
+cudaError_t tc_selftest_timeout(Ctx *c, int32_t *user_status, cudaStream_t st)
+{
+    SelfTestParams p;
+    p.status = (int32_t *)(c->ws + c->lay.status);
+    p.user_status = user_status;
+    selftest_timeout_kernel<<<1, 32, 0, st>>>(p);
+    return cudaGetLastError();
+}
 
 bool tc_supported(const mrp_config &cfg, const mrp_head_weights *heads, const void *w_lm)
 {

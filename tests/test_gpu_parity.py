@@ -297,3 +297,21 @@ def test_non_finite_logits_raise_the_status_bit_and_leave_the_context_usable(fla
     ref = oracle.draft(inp.hidden, inp.logits0, w.heads, w.w_lm, K=2)
     check_stats(good, ref, "bf16")
     binding.mrp_destroy(ctx)
+
+
+def test_a_wait_that_nothing_completes_gives_up_and_reports():
+    """Failure detection without a fault: the kernels' waits are bounded.  A barrier that nobody
+    completes makes the wait run out (about 1.5 s); the kernel returns, the status word carries
+    MRP_DEV_TIMEOUT and the context goes on working."""
+    w = synth.make_weights(128, 256, 2048, 1, "bf16", 9, head_std=0.05)
+    inp = synth.make_inputs(w, 1, 4, 9, 1.0, 4.0)
+    heads, w_lm = harness.upload_weights(w, DEV)
+    ctx = binding.mrp_create(w.d, w.F, w.V, heads, w_lm, max_rows=4, max_seqs=1, block_len=4)
+    st = torch.zeros(1, device=DEV, dtype=torch.int32)
+    binding.mrp_selftest_wait_timeout(ctx, st)
+    torch.cuda.synchronize()
+    assert int(st.item()) & binding.MRP_DEV_TIMEOUT
+    out, _ = run_gpu_draft(w, inp, 1, ctx=ctx)
+    ref = oracle.draft(inp.hidden, inp.logits0, w.heads, w.w_lm, K=1)
+    check_stats(out, ref, "bf16")
+    binding.mrp_destroy(ctx)
