@@ -31,6 +31,7 @@ WorkspaceLayout workspace_layout(const mrp_config &cfg)
     l.dense_row = take((size_t)cfg.max_seqs * (size_t)cfg.block_len * 4);
     l.sk_scratch = take((size_t)kSkScratchBytes);
     l.sk_counters = take((size_t)kSkMaxTiles * 4);
+    l.ssq_fix = take((size_t)5 * 128 * 8);
     l.has_f16 = cfg.dtype == MRP_BF16 && !(cfg.flags & (MRP_FLAG_FORCE_SIMT | MRP_FLAG_EXACT_OPERANDS)) &&
                 ((long long)cfg.n_heads + 1) * cfg.max_rows >= kF16MinRowSteps && cfg.d % 64 == 0 &&
                 cfg.d_ff % 64 == 0 && cfg.vocab % 16 == 0 && cfg.n_heads <= 4;

@@ -32,6 +32,7 @@ struct WorkspaceLayout {
     size_t dense_row;   // int32 [max_seqs*block_len] dense position -> masked row or -1
     size_t sk_scratch;  // fp32 [CTAs][r_pad][128] partial accumulators of the few-row head kernels
     size_t sk_counters; // int32 [kSkMaxTiles] arrivals per weight tile (zero between launches)
+    size_t ssq_fix;     // uint64 [5][128]: sums of squares per (head, row) in 2^-24 fixed point (chain kernel)
     size_t w16;         // fp16 [V, d] copy of the LM head (0 bytes unless the fp16 LM path can run)
     size_t xt16;        // fp16 [n_heads*max_rows, d] rows h_k - h_0 for that path
     bool has_f16;
@@ -164,7 +165,8 @@ cudaError_t sk_down(Ctx *c, int k, int M, int K, const mrp_draft_out &out, cudaS
                     int *n_ss_out, bool f16_lm);
 bool sk_heads_ok(const mrp_config &cfg);
 // The whole head chain as one cooperative kernel (tc_chain.cu); cudaErrorNotSupported = use the others.
-cudaError_t sk_chain(Ctx *c, int M, int K, const mrp_draft_out &out, cudaStream_t st, bool f16_lm);
+cudaError_t sk_chain(Ctx *c, int M, int K, const mrp_draft_out &out, cudaStream_t st, bool f16_lm,
+                     bool check_only);
 cudaError_t sk_lm(Ctx *c, const float *logits0, const int32_t *row_index, int M, int K,
                   const mrp_draft_out &out, cudaStream_t st, bool pdl);
 

@@ -24,12 +24,12 @@ namespace {
 
 constexpr int kChThreads = 192;
 constexpr int kChWTile = 128 * 128;
-constexpr int kChAuxBytes = 12288;
+constexpr int kChAuxBytes = 20480;
 constexpr int kChAuxRstd = 0;              // float[128]
 constexpr int kChAuxVote = 768;            // int
 constexpr int kChAuxReleased = 772;        // int: phases whose barrier this CTA has seen released
-constexpr int kChAuxSq = 4096;             // float[2048]: squares of a share's outputs
-constexpr int kChMaxShare = 2048;          // outputs a CTA finishes per down-projection phase, at most
+constexpr int kChAuxSq = 4096;             // float[4096]: squares of a share's outputs
+constexpr int kChMaxShare = 4096;          // outputs a CTA finishes per down-projection phase, at most
 constexpr int kChTilesPerPhase = 448;      // arrival counters per phase
 constexpr int kChMaxPhases = 8;
 constexpr long long kBarrierCycles = 1000000000LL;   // bound on a grid-barrier wait (about 0.5 s)
@@ -47,7 +47,7 @@ struct ChainPhase {
     int n_split;         // CTAs per tile, each a slice of the contraction
     int w_rows;          // weight rows (GU: gate rows)
     int map_x, map_w0, map_w1;
-    int n_ss;            // GU: slices of sums of squares to add up
+    int ssq_idx;         // GU: head index whose sums of squares normalise the input; DN: the one it adds to
     const __nv_bfloat16 *gamma_next;   // DN
     __nv_bfloat16 *xg_next;
     __nv_bfloat16 *xt_k;
@@ -64,7 +64,8 @@ struct ChainParams {
     __nv_bfloat16 *act;
     float *hcur;
     const float *h0f;
-    float *sumsq;            // [slices][M]: read by GU, written (one slice per CTA) by DN
+    unsigned long long *ssq_fix;   // [5][128] sums of squares in 2^-24 fixed point: integer adds commute,
+                                   // so the CTAs of a phase can add their shares in any order
     float *scratch;          // partial accumulators [cta][RP][128]
     int32_t *counters;       // arrivals per (phase, tile) (zero at launch)
     unsigned int *grid_bar;  // CTAs that have finished a phase, summed over phases (zero at launch)
@@ -280,13 +281,10 @@ sk_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant__ 
             if (active) {
                 const int split = cta % ph.n_split;
                 if (ph.kind == CH_GU) {
-                    // rstd of row m from the slices of sums of squares: warp per row, lanes over slices
-                    for (int m = q; m < p.M; m += 4) {
-                        float s = 0.f;
-                        for (int j = lane; j < ph.n_ss; j += 32) s += __ldcg(p.sumsq + (size_t)j * p.M + m);
-#pragma unroll
-                        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-                        if (lane == 0) rstd_s[m] = rsqrtf(s / (float)p.d + p.eps);
+                    if (t < p.M) {
+                        const unsigned long long v = __ldcg(p.ssq_fix + ph.ssq_idx * 128 + t);
+                        const float s = (float)((double)v * (1.0 / 16777216.0));
+                        rstd_s[t] = rsqrtf(s / (float)p.d + p.eps);
                     }
                 }
                 const int acc = n_acc & 1, use = n_acc >> 1;
@@ -381,11 +379,12 @@ sk_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant__ 
                         sq_s[e] = sq;
                     }
                     ch_epi_sync();
-                    // one slice of sums of squares per CTA: its rows, in row order
+                    // this CTA's rows, in row order, then one integer add per row of the batch
                     for (int m = t; m < p.M; m += 128) {
                         float s = 0.f;
                         for (int r = 0; r < n_r; ++r) s += sq_s[m * n_r + r];
-                        p.sumsq[(size_t)cta * p.M + m] = s;
+                        atomicAdd(p.ssq_fix + ph.ssq_idx * 128 + m,
+                                  (unsigned long long)__double2ll_rn((double)s * 16777216.0));
                     }
                 }
             }
@@ -446,20 +445,32 @@ cudaError_t chain_launch(const ChainMaps &maps, const ChainParams &p, int grid, 
 // The whole head chain (K heads) for M <= 64 rows as one kernel.  Returns cudaErrorNotSupported
 // (nothing launched) if the shape does not fit this form; the caller then runs the chain as
 // separate kernels.
-cudaError_t sk_chain(Ctx *c, int M, int K, const mrp_draft_out &out, cudaStream_t st, bool f16_lm)
+cudaError_t sk_chain(Ctx *c, int M, int K, const mrp_draft_out &out, cudaStream_t st, bool f16_lm, bool check_only)
 {
     const TcState *s = (const TcState *)c->tc_state;
     const int d = c->cfg.d, F = c->cfg.d_ff, G = c->sm_count;
-    if (K < 1 || K > 4 || 2 * K > kChMaxPhases || M < 1 || M > 64) return cudaErrorNotSupported;
+    if (K < 1 || K > 4 || 2 * K > kChMaxPhases || M < 1 || M > 128) return cudaErrorNotSupported;
     // Worth it while a GEMM of the chain is latency-bound (a few tens of MB of weights): measured
     // 71 vs 77 us at d = 2048, F = 4096, but 201 vs 183 us at d = 4096, F = 8192 (M = 4).
-    if ((long long)d * F > (12ll << 20)) return cudaErrorNotSupported;
-    const int r_pad = M <= 16 ? 16 : M <= 32 ? 32 : 64;
+    // Above 64 rows the alternative is the row-major kernels, whose narrow weight tiles cost far more.
+    if (M <= 64 && (long long)d * F > (12ll << 20)) return cudaErrorNotSupported;
+    const int r_pad = sk_head_pad(M);
     const int gu_tiles = F / 64, dn_tiles = (d + 127) / 128;
     if (gu_tiles > G || dn_tiles > G || G > kSumsqSlices || gu_tiles > kChTilesPerPhase ||
         kChMaxPhases * kChTilesPerPhase >= kSkMaxTiles)
         return cudaErrorNotSupported;
     if ((size_t)G * r_pad * 128 * 4 > (size_t)kSkScratchBytes) return cudaErrorNotSupported;
+
+    {
+        // a down-projection share must fit the shared-memory buffer of squares
+        int S = G / dn_tiles;
+        if (S < 1) S = 1;
+        if (S > F / kBK) S = F / kBK;
+        const int cps = (F / kBK + S - 1) / S;
+        S = (F / kBK + cps - 1) / cps;
+        if (M * ((128 + S - 1) / S) > kChMaxShare) return cudaErrorNotSupported;
+    }
+    if (check_only) return cudaSuccess;
 
     ChainParams p;
     memset(&p, 0, sizeof(p));
@@ -470,7 +481,7 @@ cudaError_t sk_chain(Ctx *c, int M, int K, const mrp_draft_out &out, cudaStream_
     p.lo_x = c->lo_x; p.lo_xt = c->lo_xt;
     p.act = (__nv_bfloat16 *)(c->ws + c->lay.act);
     p.hcur = (float *)(c->ws + c->lay.hcur); p.h0f = (const float *)(c->ws + c->lay.h0f);
-    p.sumsq = (float *)(c->ws + c->lay.sumsq);
+    p.ssq_fix = (unsigned long long *)(c->ws + c->lay.ssq_fix);
     p.scratch = (float *)(c->ws + c->lay.sk_scratch);
     p.counters = (int32_t *)(c->ws + c->lay.sk_counters);
     p.grid_bar = (unsigned int *)(c->ws + c->lay.sk_counters) + (kSkMaxTiles - 1);
@@ -505,9 +516,10 @@ cudaError_t sk_chain(Ctx *c, int M, int K, const mrp_draft_out &out, cudaStream_
         ChainPhase &gu = p.ph[2 * (k - 1)], &dn = p.ph[2 * (k - 1) + 1];
         gu.kind = CH_GU; gu.k_chunks = d / kBK; gu.n_tiles = gu_tiles; gu.n_split = split(gu_tiles, gu.k_chunks);
         gu.w_rows = F; gu.map_x = 0; gu.map_w0 = b; gu.map_w1 = b + 1;
-        gu.n_ss = (k == 1) ? 1 : dn_tiles * split(dn_tiles, F / kBK);
+        gu.ssq_idx = k - 1;
         dn.kind = CH_DN; dn.k_chunks = F / kBK; dn.n_tiles = dn_tiles; dn.n_split = split(dn_tiles, dn.k_chunks);
         if (M * ((128 + dn.n_split - 1) / dn.n_split) > kChMaxShare) return cudaErrorNotSupported;
+        dn.ssq_idx = k;
         dn.w_rows = d; dn.map_x = 1; dn.map_w0 = b + 2; dn.map_w1 = b + 2;
         dn.gamma_next = (k < K) ? (const __nv_bfloat16 *)c->heads[k].rms_gamma : nullptr;
         dn.xg_next = (k < K) ? xg : nullptr;
@@ -519,7 +531,8 @@ cudaError_t sk_chain(Ctx *c, int M, int K, const mrp_draft_out &out, cudaStream_
     switch (r_pad) {
     case 16: e = chain_launch<16>(maps, p, G, smem, st); break;
     case 32: e = chain_launch<32>(maps, p, G, smem, st); break;
-    default: e = chain_launch<64>(maps, p, G, smem, st); break;
+    case 64: e = chain_launch<64>(maps, p, G, smem, st); break;
+    default: e = chain_launch<128>(maps, p, G, smem, st); break;
     }
     c->launches++;
     return note_err(c, e, "head-chain kernel");

@@ -334,7 +334,8 @@ __global__ void tc_prep_kernel(const __nv_bfloat16 *__restrict__ hidden, const i
                                int d, int lo_x, int lo_xt, const __nv_bfloat16 *__restrict__ gamma1,
                                float *__restrict__ h0f, float *__restrict__ hcur, __nv_bfloat16 *__restrict__ xg,
                                __nv_bfloat16 *__restrict__ xt0, float *__restrict__ sumsq,
-                               int32_t *__restrict__ counters, int n_counters)
+                               int32_t *__restrict__ counters, int n_counters,
+                               unsigned long long *__restrict__ ssq_fix)
 {
     pdl_trigger();
     pdl_wait();
@@ -368,6 +369,11 @@ __global__ void tc_prep_kernel(const __nv_bfloat16 *__restrict__ hidden, const i
         float t = 0.f;
         for (int i = 0; i < (int)(blockDim.x >> 5); ++i) t += red[i];
         sumsq[m] = t;
+        if (m < 128) {
+            // the chain kernel keeps sums of squares in 2^-24 fixed point (integer adds commute)
+            ssq_fix[m] = (unsigned long long)__double2ll_rn((double)t * 16777216.0);
+            for (int k = 1; k < 5; ++k) ssq_fix[k * 128 + m] = 0ull;
+        }
     }
 }
 
@@ -560,23 +566,26 @@ cudaError_t tc_draft(Ctx *c, const void *hidden, const float *logits0, const int
                           !(c->cfg.flags & MRP_FLAG_ROW_MAJOR_ONLY);
     const bool lm_few = sk_rows_ok(n_rs) && !(c->cfg.flags & MRP_FLAG_ROW_MAJOR_ONLY);
     const bool f16_lm = c->use_f16_lm && n_rs >= kF16MinRowSteps && !lm_few;
-    c->lo_x = few_rows ? sk_head_pad(M) : M;
+    const bool chain = !(c->cfg.flags & (MRP_FLAG_ROW_MAJOR_ONLY | MRP_FLAG_NO_CHAIN)) && sk_heads_ok(c->cfg) &&
+                       sk_chain(c, M, K, out, st, f16_lm, true) == cudaSuccess;
+    c->lo_x = (few_rows || chain) ? sk_head_pad(M) : M;
     c->lo_xt = lm_few ? sk_lm_pad(n_rs) : n_rs;
 
     prof_mark(c, 0, st);
     cudaError_t e = note_err(c, launch_k(tc_prep_kernel, dim3(M), dim3(256), 0, st, !(c->cfg.flags & MRP_FLAG_NO_PDL),
                                          (const __nv_bfloat16 *)hidden, row_index, d, c->lo_x, c->lo_xt,
                                       (const __nv_bfloat16 *)c->heads[0].rms_gamma, h0f, hcur, xg, xt, sumsq,
-                                      (int32_t *)(c->ws + c->lay.sk_counters), kSkMaxTiles), "tc_prep_kernel");
+                                      (int32_t *)(c->ws + c->lay.sk_counters), kSkMaxTiles,
+                                      (unsigned long long *)(c->ws + c->lay.ssq_fix)), "tc_prep_kernel");
     c->launches++;
     if (e != cudaSuccess) return e;
 
     int n_ss = 1;
     bool chain_done = false;
-    if (few_rows && !(c->cfg.flags & MRP_FLAG_NO_CHAIN)) {
-        e = sk_chain(c, M, K, out, st, f16_lm);
-        if (e == cudaSuccess) chain_done = true;
-        else if (e != cudaErrorNotSupported) return e;
+    if (chain) {
+        e = sk_chain(c, M, K, out, st, f16_lm, false);
+        if (e != cudaSuccess) return e;
+        chain_done = true;
     }
     for (int k = 1; k <= K && !chain_done; ++k) {
         if (few_rows) {
