@@ -39,8 +39,8 @@ enum { SK_GU = 0, SK_DN = 1, SK_LM = 2 };
 
 struct SkMaps {
     CUtensorMap x;      // activation operand, box = r_pad rows
-    CUtensorMap w[6];   // [part * 3 + kind]: part 0 = gate / the matrix, 1 = up;
-                        // kind 0 = full tile, 1 / 2 = the two short-tile box heights
+    CUtensorMap w[6];   // w[0] = 128-row tiles of gate / the matrix, w[3] = 128-row tiles of up;
+                        // w[1], w[2], w[4], w[5] = LM tiles of the other heights (lm_h[0..3])
 };
 
 struct SkParams {
@@ -48,7 +48,7 @@ struct SkParams {
     int k_chunks;        // contraction extent / 64
     int n_stages;
     int kc;              // 64-element k-chunks per ring stage
-    int r_pad;           // activation rows per part (16 or 32); MMA N = 2 * r_pad
+    int r_pad;           // activation rows per part (16, 32, 64 or 128; LM: 16 or 32); MMA N = 2 * r_pad
     int tmem_cols;       // allocated TMEM columns (power of two >= 2 buffers * 2 * r_pad)
     int lo_x, lo_xt;     // row offset of the lo block in the head operands / the LM-head operand
     int lm_h[4];         // LM: tile heights (units) other than 8, fetched through maps w[1], w[2], w[4], w[5]
