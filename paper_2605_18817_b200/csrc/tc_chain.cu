@@ -220,34 +220,41 @@ sk_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant__ 
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
-        if (lane == 0) {
-            const uint32_t idesc = make_idesc(2 * RP);
-            int it = 0, n_acc = 0;
-            bool ok = true;
-            for (int i = 0; i < p.n_phases && ok; ++i) {
-                int tile, kc0, nk;
-                if (!share(i, tile, kc0, nk)) continue;
-                const int acc = n_acc & 1, use = n_acc >> 1;
-                if (use > 0 && !mbar_wait(tempty_bar(acc), (uint32_t)((use - 1) & 1), abort_flag, p)) break;
+        // The whole warp walks the loop (all values are warp-uniform); the elected lane issues.
+        const uint32_t idesc = make_idesc(2 * RP);
+        int n_acc = 0;
+        int s = 0;                        // ring stage and its barrier phase, advanced chunk by chunk
+        uint32_t ph_bit = 0;
+        bool ok = true;
+        for (int i = 0; i < p.n_phases && ok; ++i) {
+            int tile, kc0, nk;
+            if (!share(i, tile, kc0, nk)) continue;
+            const int acc = n_acc & 1, use = n_acc >> 1;
+            if (use > 0) ok = __all_sync(0xffffffffu, mbar_wait(tempty_bar(acc), (uint32_t)((use - 1) & 1), abort_flag, p));
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t dt = __shfl_sync(0xffffffffu, tmem_base, 0) + (uint32_t)(acc * 2 * RP);
+            for (int kk = 0; kk < nk; ++kk) {
+                const uint32_t sw = base + (uint32_t)s * stage_bytes;
+                const uint64_t dw = make_smem_desc(sw);
+                const uint64_t dx = make_smem_desc(sw + kChWTile);
+                const uint32_t later = kk > 0 ? 1u : 0u;
+                ok = __all_sync(0xffffffffu, mbar_wait(full_bar(s), ph_bit, abort_flag, p));
+                if (!ok) break;
                 tc_fence_after();
-                const uint32_t dt = tmem_base + (uint32_t)(acc * 2 * RP);
-                for (int kk = 0; kk < nk; ++kk) {
-                    const int s = (it + kk) % p.n_stages;
-                    if (!mbar_wait(full_bar(s), (uint32_t)(((it + kk) / p.n_stages) & 1), abort_flag, p)) { ok = false; break; }
-                    tc_fence_after();
-                    const uint32_t sw = base + (uint32_t)s * stage_bytes;
-                    const uint64_t dw = make_smem_desc(sw);
-                    const uint64_t dx = make_smem_desc(sw + kChWTile);
+                if (elect_one()) {
+                    umma_bf16(dt, dw, dx, idesc, later);
 #pragma unroll
-                    for (int k4 = 0; k4 < kBK / 16; ++k4)
-                        umma_bf16(dt, dw + 2u * k4, dx + 2u * k4, idesc, (kk > 0 || k4 > 0) ? 1u : 0u);
+                    for (int k4 = 1; k4 < kBK / 16; ++k4) umma_bf16(dt, dw + 2u * k4, dx + 2u * k4, idesc, 1u);
                     umma_commit(empty_bar(s));
                 }
-                if (!ok) break;
-                umma_commit(tfull_bar(acc));
-                it += nk;
-                ++n_acc;
+                __syncwarp();
+                if (++s == p.n_stages) { s = 0; ph_bit ^= 1u; }
             }
+            if (!ok) break;
+            if (elect_one()) umma_commit(tfull_bar(acc));
+            __syncwarp();
+            ++n_acc;
         }
     } else {
         // ---------------- epilogue warps ----------------

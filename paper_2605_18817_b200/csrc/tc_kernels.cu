@@ -1,6 +1,6 @@
 // Tensor-core kernel family, row-major form (sm_100a): tcgen05.mma with TMEM accumulators, operands
 // staged in shared memory by TMA (128-byte swizzle), warp-specialised: one TMA producer thread,
-// one MMA issuer thread, four epilogue warps that read the accumulators back with tcgen05.ld.
+// one MMA issuer warp (one elected lane issues), four epilogue warps that read the accumulators back with tcgen05.ld.
 // Used where there are many activation rows; tc_skinny.cu holds the few-row form.
 //
 // All three GEMMs of the drafting pass share one main loop and differ in the epilogue:
@@ -158,36 +158,43 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
-        if (lane == 0) {
-            const uint32_t idesc = F16 ? make_idesc_f16(p.bn) : make_idesc(p.bn);
-            int s = 0, acc = 0;
-            uint32_t ph = 0, acc_ph = 0;
-            bool ok = true;
-            for (int mb = grp; mb < p.n_rb && ok; mb += p.n_groups) {
-                for (int t = 0; t < n_t && ok; ++t) {
-                    if (!mbar_wait(tempty_bar(acc), acc_ph ^ 1u, abort_flag, p)) { ok = false; break; }
+        // The whole warp walks the loop (all values are warp-uniform); the elected lane issues.
+        const uint32_t idesc = F16 ? make_idesc_f16(p.bn) : make_idesc(p.bn);
+        const uint32_t tm = __shfl_sync(0xffffffffu, tmem_base, 0);
+        int s = 0, acc = 0;
+        uint32_t ph = 0, acc_ph = 0;
+        bool ok = true;
+        for (int mb = grp; mb < p.n_rb && ok; mb += p.n_groups) {
+            for (int t = 0; t < n_t && ok; ++t) {
+                ok = __all_sync(0xffffffffu, mbar_wait(tempty_bar(acc), acc_ph ^ 1u, abort_flag, p));
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t dt = tm + (uint32_t)(acc * kAccCols);
+                for (int kk = 0; kk < p.k_chunks; ++kk) {
+                    const uint32_t sa = base + (uint32_t)s * stage_bytes;
+                    const uint64_t db = make_smem_desc(sa + PARTS * kATile);
+                    const uint32_t later = kk > 0 ? 1u : 0u;
+                    ok = __all_sync(0xffffffffu, mbar_wait(full_bar(s), ph, abort_flag, p));
+                    if (!ok) break;
                     tc_fence_after();
-                    const uint32_t dt = tmem_base + (uint32_t)(acc * kAccCols);
-                    for (int kk = 0; kk < p.k_chunks; ++kk) {
-                        if (!mbar_wait(full_bar(s), ph, abort_flag, p)) { ok = false; break; }
-                        tc_fence_after();
-                        const uint32_t sa = base + (uint32_t)s * stage_bytes;
-                        const uint64_t db = make_smem_desc(sa + PARTS * kATile);
+                    if (elect_one()) {
 #pragma unroll
                         for (int a = 0; a < PARTS; ++a) {
                             const uint64_t da = make_smem_desc(sa + a * kATile);
 #pragma unroll
                             for (int k4 = 0; k4 < kBK / 16; ++k4)
-                                umma_bf16(dt, da + 2u * k4, db + 2u * k4, idesc, (kk > 0 || k4 > 0 || a > 0) ? 1u : 0u);
+                                umma_bf16(dt, da + 2u * k4, db + 2u * k4, idesc, (k4 > 0 || a > 0) ? 1u : later);
                         }
                         umma_commit(empty_bar(s));
-                        if (++s == p.n_stages) { s = 0; ph ^= 1u; }
                     }
-                    if (!ok) break;
-                    umma_commit(tfull_bar(acc));
-                    acc ^= 1;
-                    if (acc == 0) acc_ph ^= 1u;
+                    __syncwarp();
+                    if (++s == p.n_stages) { s = 0; ph ^= 1u; }
                 }
+                if (!ok) break;
+                if (elect_one()) umma_commit(tfull_bar(acc));
+                __syncwarp();
+                acc ^= 1;
+                if (acc == 0) acc_ph ^= 1u;
             }
         }
     } else {

@@ -214,35 +214,42 @@ sk_gemm_kernel(const __grid_constant__ SkMaps maps, const SkParams p)
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
-        if (lane == 0) {
-            const uint32_t idesc = make_idesc(2 * RP);
-            int s = 0, acc = 0;
-            uint32_t ph = 0, acc_ph = 0;
-            bool ok = true;
-            for (int t = 0; t < n_tiles && ok; ++t) {
-                if (!mbar_wait(tempty_bar(acc), acc_ph ^ 1u, abort_flag, p)) break;
+        // The whole warp walks the loop (all values are warp-uniform); the elected lane issues.
+        const uint32_t idesc = make_idesc(2 * RP);
+        const uint32_t tm = __shfl_sync(0xffffffffu, tmem_base, 0);
+        int s = 0, acc = 0;
+        uint32_t ph = 0, acc_ph = 0;
+        bool ok = true;
+        for (int t = 0; t < n_tiles && ok; ++t) {
+            ok = __all_sync(0xffffffffu, mbar_wait(tempty_bar(acc), acc_ph ^ 1u, abort_flag, p));
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t dt = tm + (uint32_t)(acc * 2 * RP);
+            for (int kk = 0; kk < nk; ++kk) {
+                const uint32_t sw = base + (uint32_t)s * stage_bytes;
+                const uint32_t later = kk > 0 ? 1u : 0u;
+                ok = __all_sync(0xffffffffu, mbar_wait(full_bar(s), ph, abort_flag, p));
+                if (!ok) break;
                 tc_fence_after();
-                const uint32_t dt = tmem_base + (uint32_t)(acc * 2 * RP);
-                for (int kk = 0; kk < nk; ++kk) {
-                    if (!mbar_wait(full_bar(s), ph, abort_flag, p)) { ok = false; break; }
-                    tc_fence_after();
-                    const uint32_t sw = base + (uint32_t)s * stage_bytes;
+                if (elect_one()) {
 #pragma unroll
                     for (int b = 0; b < KC; ++b) {
                         const uint64_t dw = make_smem_desc(sw + b * sub_bytes);
                         const uint64_t dx = make_smem_desc(sw + b * sub_bytes + kWTile);
 #pragma unroll
                         for (int k4 = 0; k4 < kBK / 16; ++k4)
-                            umma_bf16(dt, dw + 2u * k4, dx + 2u * k4, idesc, (kk > 0 || b > 0 || k4 > 0) ? 1u : 0u);
+                            umma_bf16(dt, dw + 2u * k4, dx + 2u * k4, idesc, (b > 0 || k4 > 0) ? 1u : later);
                     }
                     umma_commit(empty_bar(s));
-                    if (++s == p.n_stages) { s = 0; ph ^= 1u; }
                 }
-                if (!ok) break;
-                umma_commit(tfull_bar(acc));
-                acc ^= 1;
-                if (acc == 0) acc_ph ^= 1u;
+                __syncwarp();
+                if (++s == p.n_stages) { s = 0; ph ^= 1u; }
             }
+            if (!ok) break;
+            if (elect_one()) umma_commit(tfull_bar(acc));
+            __syncwarp();
+            acc ^= 1;
+            if (acc == 0) acc_ph ^= 1u;
         }
     } else {
         // ---------------- epilogue warps: thread t owns TMEM lane t = weight row t of the tile ----
