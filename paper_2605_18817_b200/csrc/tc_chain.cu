@@ -105,14 +105,16 @@ __device__ __forceinline__ bool grid_bar_wait(const unsigned int *bar, unsigned 
     return true;
 }
 
-template <int RP>
+template <int RP, int KC>
 __global__ void __launch_bounds__(kChThreads, 1)
 sk_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainParams p)
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     constexpr int x_bytes = 2 * RP * 128;            // hi rows then lo rows of one k-chunk
-    constexpr int stage_bytes = kChWTile + x_bytes;
+    constexpr int sub_bytes = kChWTile + x_bytes;     // one k-chunk: weight tile, then activation rows
+    constexpr int stage_bytes = KC * sub_bytes;       // a ring stage holds KC k-chunks: one barrier wait and
+                                                      // one commit per 4 * KC MMAs
     const uint32_t bars = base + (uint32_t)p.n_stages * stage_bytes;
     auto full_bar = [&](int s) { return bars + 8u * s; };
     auto empty_bar = [&](int s) { return bars + 8u * (p.n_stages + s); };
@@ -172,23 +174,31 @@ sk_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant__ 
                 auto claim = [&](int n) {     // wait until the stage of chunk n is free, arm its barrier
                     const int s = stage_of(n), use = n / p.n_stages;
                     if (use > 0 && !mbar_wait(empty_bar(s), (uint32_t)((use - 1) & 1), abort_flag, p)) return false;
-                    mbar_expect_tx(full_bar(s), (uint32_t)(kChWTile + x_bytes));
+                    mbar_expect_tx(full_bar(s), (uint32_t)stage_bytes);
                     return true;
                 };
                 auto load_w = [&](int n, int kk) {
-                    const uint32_t sw = base + (uint32_t)stage_of(n) * stage_bytes;
-                    if (ph.kind == CH_GU) {
-                        tma_load_2d_hint(sw, &maps.m[ph.map_w0], (kc0 + kk) * kBK, tile * 64, full_bar(stage_of(n)), pol_w);
-                        tma_load_2d_hint(sw + 64 * 128, &maps.m[ph.map_w1], (kc0 + kk) * kBK, tile * 64, full_bar(stage_of(n)), pol_w);
-                    } else {
-                        tma_load_2d_hint(sw, &maps.m[ph.map_w0], (kc0 + kk) * kBK, tile * 128, full_bar(stage_of(n)), pol_w);
+#pragma unroll
+                    for (int b = 0; b < KC; ++b) {
+                        const uint32_t sw = base + (uint32_t)stage_of(n) * stage_bytes + b * sub_bytes;
+                        const int col = (kc0 + kk * KC + b) * kBK;
+                        if (ph.kind == CH_GU) {
+                            tma_load_2d_hint(sw, &maps.m[ph.map_w0], col, tile * 64, full_bar(stage_of(n)), pol_w);
+                            tma_load_2d_hint(sw + 64 * 128, &maps.m[ph.map_w1], col, tile * 64, full_bar(stage_of(n)), pol_w);
+                        } else {
+                            tma_load_2d_hint(sw, &maps.m[ph.map_w0], col, tile * 128, full_bar(stage_of(n)), pol_w);
+                        }
                     }
                 };
                 auto load_x = [&](int n, int kk) {
-                    const uint32_t sx = base + (uint32_t)stage_of(n) * stage_bytes + kChWTile;
-                    // one box: RP hi rows, then (the lo block starts at row RP of the buffer) RP lo rows
-                    tma_load_2d_hint(sx, &maps.m[ph.map_x], (kc0 + kk) * kBK, 0, full_bar(stage_of(n)), pol_x);
+#pragma unroll
+                    for (int b = 0; b < KC; ++b) {
+                        const uint32_t sx = base + (uint32_t)stage_of(n) * stage_bytes + b * sub_bytes + kChWTile;
+                        // one box: RP hi rows, then (the lo block starts at row RP of the buffer) RP lo rows
+                        tma_load_2d_hint(sx, &maps.m[ph.map_x], (kc0 + kk * KC + b) * kBK, 0, full_bar(stage_of(n)), pol_x);
+                    }
                 };
+                nk /= KC;                     // ring steps of this slice (KC divides every slice)
                 // weights depend on nothing: put as many chunks of them in flight as the ring holds
                 const int pre = min(p.n_stages, nk);
                 for (int kk = 0; kk < pre && ok; ++kk) {
@@ -234,18 +244,22 @@ sk_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant__ 
             if (!ok) break;
             tc_fence_after();
             const uint32_t dt = __shfl_sync(0xffffffffu, tmem_base, 0) + (uint32_t)(acc * 2 * RP);
+            nk /= KC;
             for (int kk = 0; kk < nk; ++kk) {
                 const uint32_t sw = base + (uint32_t)s * stage_bytes;
-                const uint64_t dw = make_smem_desc(sw);
-                const uint64_t dx = make_smem_desc(sw + kChWTile);
                 const uint32_t later = kk > 0 ? 1u : 0u;
                 ok = __all_sync(0xffffffffu, mbar_wait(full_bar(s), ph_bit, abort_flag, p));
                 if (!ok) break;
                 tc_fence_after();
                 if (elect_one()) {
-                    umma_bf16(dt, dw, dx, idesc, later);
 #pragma unroll
-                    for (int k4 = 1; k4 < kBK / 16; ++k4) umma_bf16(dt, dw + 2u * k4, dx + 2u * k4, idesc, 1u);
+                    for (int b = 0; b < KC; ++b) {
+                        const uint64_t dw = make_smem_desc(sw + b * sub_bytes);
+                        const uint64_t dx = make_smem_desc(sw + b * sub_bytes + kChWTile);
+#pragma unroll
+                        for (int k4 = 0; k4 < kBK / 16; ++k4)
+                            umma_bf16(dt, dw + 2u * k4, dx + 2u * k4, idesc, (b > 0 || k4 > 0) ? 1u : later);
+                    }
                     umma_commit(empty_bar(s));
                 }
                 __syncwarp();
@@ -417,10 +431,10 @@ sk_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant__ 
     }
 }
 
-template <int RP>
+template <int RP, int KC>
 cudaError_t chain_launch(const ChainMaps &maps, const ChainParams &p, int grid, size_t smem, cudaStream_t st)
 {
-    auto kern = sk_chain_kernel<RP>;
+    auto kern = sk_chain_kernel<RP, KC>;
     // the shared-memory limit of a kernel is set once per device (the attribute is per device)
     static std::atomic<unsigned long long> attr_devices{0};
     int dev = 0;
@@ -493,7 +507,18 @@ cudaError_t sk_chain(Ctx *c, int M, int K, const mrp_draft_out &out, cudaStream_
     p.counters = (int32_t *)(c->ws + c->lay.sk_counters);
     p.grid_bar = (unsigned int *)(c->ws + c->lay.sk_counters) + (kSkMaxTiles - 1);
     p.status = (int32_t *)(c->ws + c->lay.status); p.user_status = out.status;
-    const int stage = kChWTile + 2 * r_pad * 128;
+    auto split = [&](int n_tiles, int k_chunks) {
+        int S = G / n_tiles;
+        if (S < 1) S = 1;
+        if (S > k_chunks) S = k_chunks;
+        const int cps = (k_chunks + S - 1) / S;
+        return (k_chunks + cps - 1) / cps;          // no empty slice
+    };
+    const int gu_split = split(gu_tiles, d / kBK), dn_split = split(dn_tiles, F / kBK);
+    // two k-chunks per ring stage where every slice of both GEMMs has an even number of them
+    const bool even = (d / kBK) % (2 * gu_split) == 0 && (F / kBK) % (2 * dn_split) == 0;
+    const int kc = (even && r_pad <= 32) ? 2 : 1;
+    const int stage = kc * (kChWTile + 2 * r_pad * 128);
     int ns = (kSmemBudget - 1024 - 256 - 16 - kChAuxBytes) / stage;
     if (ns > 12) ns = 12;
     p.n_stages = ns;
@@ -502,13 +527,6 @@ cudaError_t sk_chain(Ctx *c, int M, int K, const mrp_draft_out &out, cudaStream_
     p.tmem_cols = cols;
     const size_t smem = (size_t)ns * stage + 1024 + 8 * (2 * ns + 4) + 16 + kChAuxBytes;
 
-    auto split = [&](int n_tiles, int k_chunks) {
-        int S = G / n_tiles;
-        if (S < 1) S = 1;
-        if (S > k_chunks) S = k_chunks;
-        const int cps = (k_chunks + S - 1) / S;
-        return (k_chunks + cps - 1) / cps;          // no empty slice
-    };
     __nv_bfloat16 *xg = (__nv_bfloat16 *)(c->ws + c->lay.xg);
     __nv_bfloat16 *xt = (__nv_bfloat16 *)(c->ws + c->lay.xt);
     if (!make_map(s, &maps.m[0], xg, d, 2 * (uint64_t)r_pad, 2 * r_pad) ||
@@ -521,10 +539,10 @@ cudaError_t sk_chain(Ctx *c, int M, int K, const mrp_draft_out &out, cudaStream_
             !make_map(s, &maps.m[b + 2], hw.w_down, F, d, 128))
             return note_err(c, cudaErrorInvalidValue, "tensor map (head chain, weights)");
         ChainPhase &gu = p.ph[2 * (k - 1)], &dn = p.ph[2 * (k - 1) + 1];
-        gu.kind = CH_GU; gu.k_chunks = d / kBK; gu.n_tiles = gu_tiles; gu.n_split = split(gu_tiles, gu.k_chunks);
+        gu.kind = CH_GU; gu.k_chunks = d / kBK; gu.n_tiles = gu_tiles; gu.n_split = gu_split;
         gu.w_rows = F; gu.map_x = 0; gu.map_w0 = b; gu.map_w1 = b + 1;
         gu.ssq_idx = k - 1;
-        dn.kind = CH_DN; dn.k_chunks = F / kBK; dn.n_tiles = dn_tiles; dn.n_split = split(dn_tiles, dn.k_chunks);
+        dn.kind = CH_DN; dn.k_chunks = F / kBK; dn.n_tiles = dn_tiles; dn.n_split = dn_split;
         if (M * ((128 + dn.n_split - 1) / dn.n_split) > kChMaxShare) return cudaErrorNotSupported;
         dn.ssq_idx = k;
         dn.w_rows = d; dn.map_x = 1; dn.map_w0 = b + 2; dn.map_w1 = b + 2;
@@ -536,10 +554,10 @@ cudaError_t sk_chain(Ctx *c, int M, int K, const mrp_draft_out &out, cudaStream_
     }
     cudaError_t e;
     switch (r_pad) {
-    case 16: e = chain_launch<16>(maps, p, G, smem, st); break;
-    case 32: e = chain_launch<32>(maps, p, G, smem, st); break;
-    case 64: e = chain_launch<64>(maps, p, G, smem, st); break;
-    default: e = chain_launch<128>(maps, p, G, smem, st); break;
+    case 16: e = kc == 2 ? chain_launch<16, 2>(maps, p, G, smem, st) : chain_launch<16, 1>(maps, p, G, smem, st); break;
+    case 32: e = kc == 2 ? chain_launch<32, 2>(maps, p, G, smem, st) : chain_launch<32, 1>(maps, p, G, smem, st); break;
+    case 64: e = chain_launch<64, 1>(maps, p, G, smem, st); break;
+    default: e = chain_launch<128, 1>(maps, p, G, smem, st); break;
     }
     c->launches++;
     return note_err(c, e, "head-chain kernel");
