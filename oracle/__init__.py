@@ -43,6 +43,7 @@ def _load():
         _lib.mrp_oracle_cap.restype = ctypes.c_int
         _lib.mrp_oracle_cap.argtypes = [ctypes.c_int, ctypes.c_int]
         _lib.mrp_oracle_draft.restype = ctypes.c_int
+        _lib.mrp_oracle_draft_from_hidden.restype = ctypes.c_int
         _lib.mrp_oracle_select.restype = ctypes.c_int
         _lib.mrp_oracle_verify.restype = ctypes.c_int
     return _lib
@@ -80,20 +81,30 @@ class DraftResult:
 
 
 def draft(hidden, logits0, heads, w_lm, K=None, row_index=None, eps=1e-6,
-          want_logits=False, want_hidden=False) -> DraftResult:
+          want_logits=False, want_hidden=False, final_gamma=None) -> DraftResult:
     """Head chain + shared LM head + softmax statistics (Algorithm 2, inner loop).
 
     ``heads`` is a sequence of dicts with float32-representable arrays ``gamma`` [d],
     ``w_gate`` [F,d], ``w_up`` [F,d], ``w_down`` [d,F]; ``hidden`` [rows,d]; ``logits0``
     [rows,V]; ``w_lm`` [V,d]; ``row_index`` selects the masked rows (None = all rows).
+    ``logits0=None``: the backbone logits are computed from the hidden states with the shared
+    LM head, ``l_0 = W_lm n_0``, ``n_0 = h_0`` or ``RMSNorm(h_0) * final_gamma``.
     """
     lib = _load()
     hidden = _f32(hidden)
-    logits0 = _f32(logits0)
+    from_hidden = logits0 is None
     w_lm = _f32(w_lm)
     n_rows, d = hidden.shape
     V = w_lm.shape[0]
-    assert w_lm.shape[1] == d and logits0.shape == (n_rows, V)
+    assert w_lm.shape[1] == d
+    if not from_hidden:
+        assert final_gamma is None
+        logits0 = _f32(logits0)
+        assert logits0.shape == (n_rows, V)
+    fg = None
+    if final_gamma is not None:
+        fg = _f32(final_gamma)
+        assert fg.shape == (d,)
     K = len(heads) if K is None else int(K)
     assert 0 <= K <= len(heads)
     ri = None
@@ -120,9 +131,11 @@ def draft(hidden, logits0, heads, w_lm, K=None, row_index=None, eps=1e-6,
     token = np.zeros((K + 1, M), np.int32)
     logits = np.zeros((K, M, V), np.float64) if want_logits else None
     hid = np.zeros((M, d), np.float64) if want_hidden else None
-    rc = lib.mrp_oracle_draft(
+    fn = lib.mrp_oracle_draft_from_hidden if from_hidden else lib.mrp_oracle_draft
+    rc = fn(
         ctypes.c_int(d), ctypes.c_int(F), ctypes.c_int(V), ctypes.c_int(K), ctypes.c_int(M),
-        ctypes.c_double(eps), _p(hidden, ctypes.c_float), _p(logits0, ctypes.c_float),
+        ctypes.c_double(eps), _p(hidden, ctypes.c_float),
+        _p(fg, ctypes.c_float) if from_hidden else _p(logits0, ctypes.c_float),
         _p(ri, ctypes.c_int32), arrs["gamma"], arrs["w_gate"], arrs["w_up"], arrs["w_down"],
         _p(w_lm, ctypes.c_float), _p(conf, ctypes.c_double), _p(lse, ctypes.c_double),
         _p(token, ctypes.c_int32), _p(margin, ctypes.c_double), _p(logits, ctypes.c_double),

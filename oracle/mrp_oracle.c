@@ -28,7 +28,10 @@
  *
  * Parity pins live in tests/ (zero-residual heads, softmax normalisation, linearity of the
  * chain in the residual, brute force on tiny vocabularies, a second implementation on
- * library routines, closed forms for the cap and the accepted-prefix length).
+ * library routines, closed forms for the cap and the accepted-prefix length; for the base
+ * logits computed from the hidden states: exact agreement with the precomputed-logits pass on
+ * integer data, l_k = W_lm h_k without a final norm, the one-hot closed form and the scale
+ * invariance of the final norm).
  */
 #include <math.h>
 #include <stdint.h>
@@ -82,13 +85,14 @@ static void softmax_stats(const double *l, int V, double *conf, double *lse, int
  *   hidden_out  optional [M, d]     (h after step K)
  * Returns 0, or -1 on allocation failure / bad arguments.
  */
-int mrp_oracle_draft(int d, int F, int V, int K, int M, double eps,
-                     const float *hidden, const float *logits0, const int32_t *row_index,
-                     const float *const *gamma, const float *const *w_gate,
-                     const float *const *w_up, const float *const *w_down,
-                     const float *w_lm,
-                     double *conf, double *lse, int32_t *token, double *margin,
-                     double *logits_out, double *hidden_out)
+static int draft_rows(int d, int F, int V, int K, int M, double eps,
+                      const float *hidden, const float *logits0, int from_hidden,
+                      const float *final_gamma, const int32_t *row_index,
+                      const float *const *gamma, const float *const *w_gate,
+                      const float *const *w_up, const float *const *w_down,
+                      const float *w_lm,
+                      double *conf, double *lse, int32_t *token, double *margin,
+                      double *logits_out, double *hidden_out)
 {
     if (d <= 0 || F <= 0 || V <= 0 || K < 0 || M < 0) return -1;
     double *h = (double *)malloc(sizeof(double) * (size_t)d);
@@ -101,7 +105,26 @@ int mrp_oracle_draft(int d, int F, int V, int K, int M, double eps,
     for (int m = 0; m < M; ++m) {
         const size_t row = row_index ? (size_t)row_index[m] : (size_t)m;
         for (int j = 0; j < d; ++j) h[j] = (double)hidden[row * (size_t)d + j];
-        for (int v = 0; v < V; ++v) l[v] = (double)logits0[row * (size_t)V + v];
+        if (!from_hidden) {
+            for (int v = 0; v < V; ++v) l[v] = (double)logits0[row * (size_t)V + v];
+        } else {
+            /* l = W_lm n, n = h (final_gamma NULL) or RMSNorm(h) * final_gamma: the backbone's
+             * own LM head applied to the same hidden states ("h, l <- f(x_t)") */
+            double rstd0 = 1.0;
+            if (final_gamma) {
+                double ss0 = 0.0;
+                for (int j = 0; j < d; ++j) ss0 += h[j] * h[j];
+                rstd0 = 1.0 / sqrt(ss0 / (double)d + eps);
+            }
+            for (int j = 0; j < d; ++j) xh[j] = final_gamma ? h[j] * rstd0 * (double)final_gamma[j] : h[j];
+#pragma omp parallel for schedule(static)
+            for (int v = 0; v < V; ++v) {
+                double s = 0.0;
+                const float *wr = w_lm + (size_t)v * d;
+                for (int j = 0; j < d; ++j) s += (double)wr[j] * xh[j];
+                l[v] = s;
+            }
+        }
         softmax_stats(l, V, &conf[m], &lse[m], &token[m], &margin[m]);
 
         for (int k = 1; k <= K; ++k) {
@@ -148,6 +171,37 @@ int mrp_oracle_draft(int d, int F, int V, int K, int M, double eps,
     }
     free(h); free(xh); free(a); free(r); free(l);
     return 0;
+}
+
+int mrp_oracle_draft(int d, int F, int V, int K, int M, double eps,
+                     const float *hidden, const float *logits0, const int32_t *row_index,
+                     const float *const *gamma, const float *const *w_gate,
+                     const float *const *w_up, const float *const *w_down,
+                     const float *w_lm,
+                     double *conf, double *lse, int32_t *token, double *margin,
+                     double *logits_out, double *hidden_out)
+{
+    if (!logits0) return -1;
+    return draft_rows(d, F, V, K, M, eps, hidden, logits0, 0, NULL, row_index, gamma, w_gate, w_up, w_down,
+                      w_lm, conf, lse, token, margin, logits_out, hidden_out);
+}
+
+/*
+ * The same pass when the backbone hands over hidden states only (Algorithm 2: h and l come out
+ * of one forward, and Sec. 3.2: the module reuses the backbone's LM head): l_0 = W_lm n_0 with
+ * n_0 = h_0, or n_0 = RMSNorm(h_0) * final_gamma when the hidden states are taken before the
+ * backbone's final norm (final_gamma [d], NULL = none).  Everything else as mrp_oracle_draft.
+ */
+int mrp_oracle_draft_from_hidden(int d, int F, int V, int K, int M, double eps,
+                                 const float *hidden, const float *final_gamma, const int32_t *row_index,
+                                 const float *const *gamma, const float *const *w_gate,
+                                 const float *const *w_up, const float *const *w_down,
+                                 const float *w_lm,
+                                 double *conf, double *lse, int32_t *token, double *margin,
+                                 double *logits_out, double *hidden_out)
+{
+    return draft_rows(d, F, V, K, M, eps, hidden, NULL, 1, final_gamma, row_index, gamma, w_gate, w_up, w_down,
+                      w_lm, conf, lse, token, margin, logits_out, hidden_out);
 }
 
 /* Max-accept cap (Sec. 4.4): m = min(max(floor(0.7 n), 5), L). */

@@ -244,6 +244,7 @@ def test_config0_static_selection_end_to_end():
     (128, 256, 2048, 32, 1, 2),     # few-row head kernels at 32 rows, row-major LM head
     (64, 12288, 2304, 5, 1, 2),     # gate/up: full 128-row weight tiles plus short tiles
     (19008, 64, 512, 3, 1, 1),      # down projection: full weight tiles plus short tiles
+    (1024, 2048, 2048, 20, 1, 2),   # head chain with 32-row operands and two k-chunks per ring stage
 ])
 def test_tensor_core_family_small_shapes(d, F, V, B, L, K):
     # residuals of order one at every shape (the very long contraction gets smaller weights)

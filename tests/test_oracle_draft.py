@@ -224,3 +224,77 @@ def test_generator_confidence_calibration():
         inp = synth.make_inputs(w, 64, 1, 9, s, s)
         r = oracle.draft(inp.hidden, inp.logits0, [], w.w_lm, K=0)
         assert lo < np.median(r.conf[0]) < hi, (s, np.median(r.conf[0]))
+
+
+# ---- backbone logits from the hidden states (logits0=None): l_0 = W_lm n_0 ----
+
+def test_from_hidden_equals_the_pass_on_precomputed_base_logits():
+    """With base logits that are exactly representable the two entry points must agree: integer
+    weights and hidden states make W_lm h an exact float32 matrix, so nothing is rounded."""
+    rng = np.random.default_rng(3)
+    w, inp = small_problem(seed=5)
+    W = rng.integers(-3, 4, size=w.w_lm.shape).astype(np.float32)
+    H = rng.integers(-2, 3, size=inp.hidden.shape).astype(np.float32)
+    l0 = (H.astype(np.float64) @ W.astype(np.float64).T).astype(np.float32)
+    a = oracle.draft(H, l0, w.heads, W, want_logits=True, want_hidden=True)
+    b = oracle.draft(H, None, w.heads, W, want_logits=True, want_hidden=True)
+    np.testing.assert_allclose(b.logits, a.logits, rtol=0, atol=1e-12)
+    np.testing.assert_allclose(b.lse, a.lse, rtol=0, atol=1e-12)
+    np.testing.assert_array_equal(b.token, a.token)
+    np.testing.assert_allclose(b.hidden, a.hidden, rtol=0, atol=0)
+
+
+def test_from_hidden_without_final_norm_every_step_is_the_lm_head_of_that_hidden_state():
+    """l_k = l_0 + W_lm (h_k - h_0) = W_lm h_k: checked through two different outputs of the
+    oracle (step-accumulated logits vs. a library matmul on its final hidden state)."""
+    w, inp = small_problem(seed=8)
+    for K in (1, 3):
+        r = oracle.draft(inp.hidden, None, w.heads, w.w_lm, K=K, want_logits=True, want_hidden=True)
+        direct = r.hidden @ w.w_lm.astype(np.float64).T
+        np.testing.assert_allclose(r.logits[K - 1], direct, rtol=0, atol=1e-10)
+        np.testing.assert_allclose(r.lse[K], logsumexp(direct, axis=1), rtol=0, atol=1e-10)
+
+
+def test_from_hidden_final_norm_closed_form_on_one_hot_rows():
+    """h_0 = c e_j: RMSNorm gives sqrt(d) sign(c) e_j (eps -> 0), so l_0 = sqrt(d) sign(c) g_j W_lm[:, j]."""
+    d, V = 24, 96
+    w, _ = small_problem(seed=9, d=d, V=V)
+    g = (1.0 + 0.5 * np.sin(np.arange(d))).astype(np.float32)
+    js = [0, 5, 23, 11]
+    cs = [2.0, -3.0, 0.5, 7.0]
+    H = np.zeros((4, d), np.float32)
+    for i, (j, c) in enumerate(zip(js, cs)):
+        H[i, j] = c
+    r = oracle.draft(H, None, w.heads, w.w_lm, K=0, eps=0.0, final_gamma=g)
+    for i, (j, c) in enumerate(zip(js, cs)):
+        l = math.sqrt(d) * np.sign(c) * float(g[j]) * w.w_lm[:, j].astype(np.float64)
+        assert r.token[0, i] == int(np.argmax(l))
+        np.testing.assert_allclose(r.lse[0, i], logsumexp(l), rtol=0, atol=1e-12)
+        np.testing.assert_allclose(r.conf[0, i], np.exp(l.max() - logsumexp(l)), rtol=0, atol=1e-12)
+
+
+def test_from_hidden_final_norm_ignores_the_scale_of_the_hidden_state_at_step_zero():
+    w, inp = small_problem(seed=10)
+    g = (1.0 + 0.25 * np.cos(np.arange(w.d))).astype(np.float32)
+    H = inp.hidden.astype(np.float32)
+    a = oracle.draft(H, None, w.heads, w.w_lm, K=0, eps=0.0, final_gamma=g)
+    b = oracle.draft(4.0 * H, None, w.heads, w.w_lm, K=0, eps=0.0, final_gamma=g)
+    np.testing.assert_allclose(b.lse, a.lse, rtol=0, atol=1e-10)
+    # and the library form of the same definition, with eps
+    n0 = H.astype(np.float64) / np.sqrt(np.mean(H.astype(np.float64) ** 2, axis=1, keepdims=True) + 1e-6) * g
+    c = oracle.draft(H, None, w.heads, w.w_lm, K=0, eps=1e-6, final_gamma=g)
+    np.testing.assert_allclose(c.lse[0], logsumexp(n0 @ w.w_lm.astype(np.float64).T, axis=1), rtol=0, atol=1e-10)
+
+
+def test_from_hidden_matches_library_implementation_with_final_norm():
+    w, inp = small_problem(seed=12)
+    g = (1.0 + 0.25 * np.cos(np.arange(w.d))).astype(np.float32)
+    H = inp.hidden.astype(np.float64)
+    n0 = H / np.sqrt(np.mean(H * H, axis=1, keepdims=True) + 1e-6) * g
+    l0 = n0 @ w.w_lm.astype(np.float64).T
+    stats, logits, _ = library_draft(inp.hidden, l0, w.heads, w.w_lm, 1e-6)
+    r = oracle.draft(inp.hidden, None, w.heads, w.w_lm, eps=1e-6, final_gamma=g, want_logits=True)
+    for k in range(len(w.heads) + 1):
+        np.testing.assert_allclose(r.conf[k], stats[k][0], rtol=0, atol=1e-10)
+        np.testing.assert_allclose(r.lse[k], stats[k][1], rtol=0, atol=1e-10)
+        np.testing.assert_array_equal(r.token[k], stats[k][2])
