@@ -154,6 +154,24 @@ typedef struct {
 int mrp_draft(mrp_ctx *ctx, const void *hidden, const float *logits0, const int32_t *row_index,
               int32_t M, int32_t K, const mrp_draft_out *out, void *cuda_stream);
 
+/*
+ * The drafting pass when the backbone hands over hidden states only.  In Algorithm 2 the
+ * hidden states and the logits come out of the same forward ("h, l <- f(x_t)") and the module
+ * reuses the backbone's LM head (Sec. 3.2); here that head is applied once for both: the pass
+ * over W_lm that produces the residual logits also produces the base logits
+ *     l_0 = W_lm n_0,   n_0 = h_0                               (final_norm_gamma == NULL)
+ *                       n_0 = RMSNorm(h_0; rms_eps) * final_norm_gamma   (hidden states taken
+ *                                                  before the backbone's final norm)
+ * and step k's logits are W_lm (n_0 + h_k - h_0).  No [n_rows, V] input is read, and the backbone
+ * needs no LM-head pass of its own for these rows.
+ *   final_norm_gamma [d] in the context's dtype, or NULL; the other arguments and the outputs
+ *   are those of mrp_draft.  On the tensor-core kernels the operand rows are always carried as
+ *   bf16 hi + lo pairs in this mode.  Errors: INVALID_ARG, CUDA.
+ */
+int mrp_draft_from_hidden(mrp_ctx *ctx, const void *hidden, const void *final_norm_gamma,
+                          const int32_t *row_index, int32_t M, int32_t K, const mrp_draft_out *out,
+                          void *cuda_stream);
+
 typedef enum { MRP_SELECT_STATIC = 0, MRP_SELECT_DYNAMIC_REMASK = 1 } mrp_select_mode;
 
 typedef struct {

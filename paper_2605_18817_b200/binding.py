@@ -30,7 +30,7 @@ MRP_DEV_NONFINITE, MRP_DEV_TIMEOUT = 1, 2
 EXPORTS = ("mrp_workspace_bytes", "mrp_create", "mrp_destroy", "mrp_draft", "mrp_reveal_remask",
            "mrp_verify", "mrp_last_launch_count", "mrp_kernel_family", "mrp_status_string",
            "mrp_profile_enable", "mrp_profile_read", "mrp_last_error",
-           "mrp_reveal_remask_noalloc", "mrp_selftest_wait_timeout")
+           "mrp_reveal_remask_noalloc", "mrp_selftest_wait_timeout", "mrp_draft_from_hidden")
 MRP_NOALLOC_MAX_POSITIONS = 65536
 MRP_ERR_CAPACITY = 7
 
@@ -87,6 +87,10 @@ def _load():
     lib.mrp_draft.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
                               ctypes.c_int32, ctypes.c_int32, ctypes.POINTER(mrp_draft_out),
                               ctypes.c_void_p]
+    lib.mrp_draft_from_hidden.restype = ctypes.c_int
+    lib.mrp_draft_from_hidden.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                                          ctypes.c_int32, ctypes.c_int32, ctypes.POINTER(mrp_draft_out),
+                                          ctypes.c_void_p]
     lib.mrp_reveal_remask.restype = ctypes.c_int
     lib.mrp_reveal_remask.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
                                       ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32,
@@ -235,6 +239,26 @@ def mrp_draft(ctx: Context, hidden, logits0, row_index, M, K, conf, lse, token, 
                        ctypes.byref(out), _stream(stream))
     if rc != 0:
         raise MrpError("mrp_draft", rc, lib.mrp_last_error(ctx.handle).decode())
+
+
+def mrp_draft_from_hidden(ctx: Context, hidden, final_norm_gamma, row_index, M, K, conf, lse, token,
+                          margin=None, logits_out=None, hidden_out=None, status=None, stream=None) -> None:
+    """Enqueue one drafting pass that computes the base logits itself (l_0 = W_lm n_0)."""
+    dt_ctx = torch.float32 if ctx.cfg.dtype == MRP_F32 else torch.bfloat16
+    _check(hidden, dt_ctx, "hidden")
+    _check(final_norm_gamma, dt_ctx, "final_norm_gamma")
+    _check(row_index, torch.int32, "row_index")
+    for t, dt, nm in ((conf, torch.float32, "conf"), (lse, torch.float32, "lse"),
+                      (token, torch.int32, "token"), (margin, torch.float32, "margin"),
+                      (logits_out, torch.float32, "logits_out"),
+                      (hidden_out, torch.float32, "hidden_out"), (status, torch.int32, "status")):
+        _check(t, dt, nm)
+    out = mrp_draft_out(_ptr(conf), _ptr(lse), _ptr(token), _ptr(margin), _ptr(logits_out),
+                        _ptr(hidden_out), _ptr(status))
+    rc = lib.mrp_draft_from_hidden(ctx.handle, _ptr(hidden), _ptr(final_norm_gamma), _ptr(row_index),
+                                   int(M), int(K), ctypes.byref(out), _stream(stream))
+    if rc != 0:
+        raise MrpError("mrp_draft_from_hidden", rc, lib.mrp_last_error(ctx.handle).decode())
 
 
 def mrp_reveal_remask(ctx: Context, conf, token, row_index, M, K, B, L, mode, tau=0.9, r_reveal=1,

@@ -201,24 +201,40 @@ void mrp_destroy(mrp_ctx *ctx)
     delete ctx;
 }
 
-int mrp_draft(mrp_ctx *ctx, const void *hidden, const float *logits0, const int32_t *row_index,
-              int32_t M, int32_t K, const mrp_draft_out *out, void *cuda_stream)
+static int draft_call(mrp_ctx *ctx, const void *hidden, const float *logits0, bool from_hidden,
+                      const void *final_gamma, const int32_t *row_index, int32_t M, int32_t K,
+                      const mrp_draft_out *out, void *cuda_stream)
 {
     if (!ctx || !out) return MRP_ERR_INVALID_ARG;
     Ctx &c = ctx->c;
     if (M < 0 || M > c.cfg.max_rows || K < 0 || K > c.cfg.n_heads) return MRP_ERR_INVALID_ARG;
     c.launches = 0;
     if (M == 0) return MRP_OK;
-    if (!hidden || !logits0 || !out->conf || !out->lse || !out->token) return MRP_ERR_INVALID_ARG;
+    if (!hidden || (!from_hidden && !logits0) || !out->conf || !out->lse || !out->token) return MRP_ERR_INVALID_ARG;
     if (((uintptr_t)hidden & 15u) || ((uintptr_t)logits0 & 15u)) return MRP_ERR_INVALID_ARG;
     DeviceGuard guard(c.cfg.device);
     if (guard.err != cudaSuccess) return MRP_ERR_CUDA;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     c.err[0] = 0;
+    c.from_hidden = from_hidden;
+    c.final_gamma = from_hidden ? final_gamma : nullptr;
     cudaError_t e = c.use_tc ? tc_draft(&c, hidden, logits0, row_index, M, K, *out, st)
                              : simt_draft(&c, hidden, logits0, row_index, M, K, *out, st);
     if (e != cudaSuccess && !c.err[0]) note_err(&c, e, "mrp_draft");
     return e == cudaSuccess ? MRP_OK : MRP_ERR_CUDA;
+}
+
+int mrp_draft(mrp_ctx *ctx, const void *hidden, const float *logits0, const int32_t *row_index,
+              int32_t M, int32_t K, const mrp_draft_out *out, void *cuda_stream)
+{
+    return draft_call(ctx, hidden, logits0, false, nullptr, row_index, M, K, out, cuda_stream);
+}
+
+int mrp_draft_from_hidden(mrp_ctx *ctx, const void *hidden, const void *final_norm_gamma,
+                          const int32_t *row_index, int32_t M, int32_t K, const mrp_draft_out *out,
+                          void *cuda_stream)
+{
+    return draft_call(ctx, hidden, nullptr, true, final_norm_gamma, row_index, M, K, out, cuda_stream);
 }
 
 int mrp_reveal_remask(mrp_ctx *ctx, const float *conf, const int32_t *token,

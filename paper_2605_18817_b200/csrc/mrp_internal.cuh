@@ -58,6 +58,10 @@ struct Ctx {
     WorkspaceLayout lay;
     bool use_tc;
     bool use_f16_lm;           // the fp16 copy of W_lm exists and is usable
+    // Set per call by mrp_draft_from_hidden: no base logits are given (logits0 == nullptr); the
+    // LM-head pass computes them as W_lm n_0, n_0 = h_0 or RMSNorm(h_0) * final_gamma.
+    bool from_hidden;
+    const void *final_gamma;
     // Row offset of the bf16 lo block behind the hi block in this call's operand buffers: M and
     // (K+1)M for the row-major kernels, the padded row count for the few-row kernels (which then
     // fetch hi and lo rows of a k-chunk with one TMA box).
@@ -133,9 +137,10 @@ struct TopFix {
 cudaError_t launch_combine(Ctx *c, const Partial *partials, int n_slices, int n_rowsteps,
                            const mrp_draft_out &out, int32_t *status, cudaStream_t st,
                            const TopFix *fix = nullptr);
-// Shared by both families: gather masked rows of `hidden` into fp32 h0f / hcur.
+// CUDA-core family: gather masked rows of `hidden` into fp32 h0f / hcur (xt0: where the step-0
+// operand rows n_0 go when the base logits are computed in the LM-head pass, else nullptr).
 cudaError_t launch_prep(Ctx *c, const void *hidden, const int32_t *row_index, int M,
-                        cudaStream_t st);
+                        cudaStream_t st, float *xt0);
 
 // ---- selection / verification (select_verify.cu) ------------------------------------
 cudaError_t launch_select(Ctx *c, const float *conf, const int32_t *token, const int32_t *row_index,

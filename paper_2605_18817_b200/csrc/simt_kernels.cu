@@ -27,30 +27,50 @@ __device__ __forceinline__ float warp_sum(float v)
 // ---- a0: gather masked rows into the fp32 residual stream --------------------------------
 template <typename T>
 __global__ void prep_kernel(const T *__restrict__ hidden, const int32_t *__restrict__ row_index,
-                            int d, float *__restrict__ h0f, float *__restrict__ hcur)
+                            int d, float *__restrict__ h0f, float *__restrict__ hcur, float *__restrict__ xt0,
+                            const T *__restrict__ final_gamma, float eps)
 {
     pdl_trigger();
     pdl_wait();
+    __shared__ float red[32];
     const int m = blockIdx.x;
     const size_t row = row_index ? (size_t)row_index[m] : (size_t)m;
+    float ss = 0.f;
     for (int j = threadIdx.x; j < d; j += blockDim.x) {
         const float v = ld_f(hidden, row * d + j);
-        h0f[(size_t)m * d + j] = v;
+        if (!xt0) h0f[(size_t)m * d + j] = v;
         hcur[(size_t)m * d + j] = v;
+        ss = fmaf(v, v, ss);
+    }
+    if (!xt0) return;
+    // No base logits: the LM-head operand of step 0 is n_0 = h_0, or RMSNorm(h_0) * final_gamma,
+    // and h0f holds h_0 - n_0, so that the down projections emit n_0 + (h_k - h_0).
+    ss = warp_sum(ss);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+    __syncthreads();
+    float t = 0.f;
+    for (int i = 0; i < (int)(blockDim.x >> 5); ++i) t += red[i];
+    const float rstd0 = final_gamma ? rsqrtf(t / (float)d + eps) : 1.f;
+    for (int j = threadIdx.x; j < d; j += blockDim.x) {
+        const float v = ld_f(hidden, row * d + j);
+        const float n0 = final_gamma ? v * rstd0 * ld_f(final_gamma, j) : v;
+        h0f[(size_t)m * d + j] = v - n0;
+        xt0[(size_t)m * d + j] = n0;
     }
 }
 
-cudaError_t launch_prep(Ctx *c, const void *hidden, const int32_t *row_index, int M, cudaStream_t st)
+cudaError_t launch_prep(Ctx *c, const void *hidden, const int32_t *row_index, int M, cudaStream_t st, float *xt0)
 {
     if (M == 0) return cudaSuccess;
     float *h0f = (float *)(c->ws + c->lay.h0f), *hcur = (float *)(c->ws + c->lay.hcur);
     const bool pdl = !(c->cfg.flags & MRP_FLAG_NO_PDL);
     cudaError_t e;
     if (c->cfg.dtype == MRP_F32)
-        e = launch_k(prep_kernel<float>, dim3(M), dim3(256), 0, st, pdl, (const float *)hidden, row_index, c->cfg.d, h0f, hcur);
+        e = launch_k(prep_kernel<float>, dim3(M), dim3(256), 0, st, pdl, (const float *)hidden, row_index, c->cfg.d, h0f, hcur,
+                     xt0, (const float *)c->final_gamma, c->cfg.rms_eps);
     else
         e = launch_k(prep_kernel<__nv_bfloat16>, dim3(M), dim3(256), 0, st, pdl, (const __nv_bfloat16 *)hidden, row_index,
-                     c->cfg.d, h0f, hcur);
+                     c->cfg.d, h0f, hcur, xt0, (const __nv_bfloat16 *)c->final_gamma, c->cfg.rms_eps);
     c->launches++;
     return e;
 }
@@ -163,7 +183,7 @@ constexpr int kLR = 8;
 
 template <typename T, int SLICE>
 __global__ void __launch_bounds__(256)
-lm_simt_kernel(const T *__restrict__ w_lm, const float *__restrict__ xt,
+lm_simt_kernel(const T *__restrict__ w_lm, const float *__restrict__ xt, const float *__restrict__ xt0,
                const float *__restrict__ logits0, const int32_t *__restrict__ row_index, int M,
                int K, int d, int V, int n_slices, Partial *__restrict__ partials,
                float *__restrict__ logits_out)
@@ -191,8 +211,10 @@ lm_simt_kernel(const T *__restrict__ w_lm, const float *__restrict__ xt,
 #pragma unroll
                         for (int r = 0; r < kLR; ++r) {
                             const int rs = rs0 + r;
-                            if (rs < n_rs && rs >= M)   // step 0 has no residual
+                            if (rs < n_rs && rs >= M)   // step 0 has no residual ...
                                 acc[r] = fmaf(a, xt[(size_t)(rs - M) * d + j], acc[r]);
+                            else if (rs < M && xt0)     // ... unless its logits are computed here
+                                acc[r] = fmaf(a, xt0[(size_t)rs * d + j], acc[r]);
                         }
                     }
                 }
@@ -205,7 +227,7 @@ lm_simt_kernel(const T *__restrict__ w_lm, const float *__restrict__ xt,
                         if (v < V && rs < n_rs) {
                             const int m = rs % M;
                             const size_t row = row_index ? (size_t)row_index[m] : (size_t)m;
-                            l = logits0[row * (size_t)V + v] + s;
+                            l = (logits0 ? logits0[row * (size_t)V + v] : 0.f) + s;
                         }
                         tile[r][vl] = l;
                     }
@@ -352,10 +374,12 @@ static cudaError_t simt_draft_t(Ctx *c, const void *hidden, const float *logits0
     int32_t *status = (int32_t *)(c->ws + c->lay.status);
     const bool pdl = !(c->cfg.flags & MRP_FLAG_NO_PDL);
     prof_mark(c, 0, st);
-    cudaError_t e = launch_prep(c, hidden, row_index, M, st);
+    // without base logits the operand rows of step 0 (n_0) follow those of steps 1..K
+    float *xt0 = c->from_hidden ? xt + (size_t)K * M * d : nullptr;
+    cudaError_t e = launch_prep(c, hidden, row_index, M, st, xt0);
     if (e != cudaSuccess) return e;
     if (K == 0 && out.hidden_out)
-        cudaMemcpyAsync(out.hidden_out, h0f, sizeof(float) * (size_t)M * d, cudaMemcpyDeviceToDevice, st);
+        cudaMemcpyAsync(out.hidden_out, hcur, sizeof(float) * (size_t)M * d, cudaMemcpyDeviceToDevice, st);
     for (int k = 1; k <= K; ++k) {
         const mrp_head_weights &hw = c->heads[k - 1];
         e = launch_k(rmsnorm_kernel<T>, dim3(M), dim3(256), 0, st, pdl, (const float *)hcur, (const T *)hw.rms_gamma, d,
@@ -378,10 +402,11 @@ static cudaError_t simt_draft_t(Ctx *c, const void *hidden, const float *logits0
     const int grid = n_slices < kSimtMaxBlocks ? n_slices : kSimtMaxBlocks;
     if (narrow)
         e = launch_k(lm_simt_kernel<T, 32>, dim3(grid), dim3(256), 0, st, pdl, (const T *)c->w_lm, (const float *)xt,
-                     logits0, row_index, M, K, d, V, n_slices, partials, out.logits_out);
+                     (const float *)xt0, logits0, row_index, M, K, d, V, n_slices, partials, out.logits_out);
     else
         e = launch_k(lm_simt_kernel<T, kSimtSliceV>, dim3(grid), dim3(256), 0, st, pdl, (const T *)c->w_lm,
-                     (const float *)xt, logits0, row_index, M, K, d, V, n_slices, partials, out.logits_out);
+                     (const float *)xt, (const float *)xt0, logits0, row_index, M, K, d, V, n_slices, partials,
+                     out.logits_out);
     c->launches++;
     if (e != cudaSuccess) return e;
     prof_mark(c, 2, st);

@@ -51,6 +51,7 @@ struct TcParams {
     int n_rb;            // 128-row activation blocks
     int rows;            // valid activation rows (GU/DN: M; LM: K*M row-steps of steps 1..K)
     int a_row_base;      // A row coordinate of row 0 (hi part)
+    int step_base;       // LM: MRP step of row 0 (1: step 0 rides on the rows of step 1; 0: it has its own rows)
     int a_part_rows;     // A row offset from the hi part to the lo part
     int M, K, V, d, F;
     int n_rs;            // (K+1)*M
@@ -218,11 +219,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 st.init();
                 st0.init();
                 if (valid) {
-                    k_of_row = r / p.M + 1;
-                    m_of_row = r - (k_of_row - 1) * p.M;
-                    first_step = (k_of_row == 1);
+                    k_of_row = r / p.M + p.step_base;
+                    m_of_row = r - (k_of_row - p.step_base) * p.M;
+                    first_step = (k_of_row == 1 && p.step_base == 1);
                     const size_t row = p.row_index ? (size_t)p.row_index[m_of_row] : (size_t)m_of_row;
-                    l0p = p.logits0 + row * (size_t)p.V;
+                    if (p.logits0) l0p = p.logits0 + row * (size_t)p.V;
                 }
             } else if (KIND == KIND_GU && valid) {
                 float s = 0.f;
@@ -241,14 +242,17 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     for (int c = 0; c < units_here; ++c) {
                         const int v = v_tile + c * 16;
                         float l0[16], a[16];
-                        if (valid) load16(l0p + v, l0);
+                        if (valid && l0p) load16(l0p + v, l0);
                         tmem_ld16(tacc + c * 16, a);
                         if (valid) {
-                            if (first_step) st0.template update<MARGIN>(l0, v);
+                            if (l0p) {
+                                if (first_step) st0.template update<MARGIN>(l0, v);
 #pragma unroll
-                            for (int j = 0; j < 16; ++j) a[j] += l0[j];
+                                for (int j = 0; j < 16; ++j) a[j] += l0[j];
+                            }
                             st.template update<MARGIN>(a, v);
-                            if (p.logits_out) store16(p.logits_out + (size_t)r * p.V + v, a);
+                            if (p.logits_out && k_of_row >= 1)
+                                store16(p.logits_out + ((size_t)(k_of_row - 1) * p.M + m_of_row) * p.V + v, a);
                         }
                     }
                 } else if (KIND == KIND_GU) {
@@ -337,12 +341,17 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
 // Gather masked rows: fp32 copies of h_0, the first head's operand bf16(h_0 * gamma_1), the
 // row sums of squares, and the zero rows that stand for step 0 in the stacked LM-head operand.
+// Without base logits (from_hidden) the LM-head operand of step k is n_0 + (h_k - h_0), so that
+// the pass itself yields l_k = W_lm n_0 + W_lm (h_k - h_0): the step-0 rows hold n_0 = h_0, or
+// RMSNorm(h_0) * final_gamma, and h0f holds h_0 - n_0, which is what the down-projection
+// epilogues subtract from h_k.
 __global__ void tc_prep_kernel(const __nv_bfloat16 *__restrict__ hidden, const int32_t *__restrict__ row_index,
                                int d, int lo_x, int lo_xt, const __nv_bfloat16 *__restrict__ gamma1,
                                float *__restrict__ h0f, float *__restrict__ hcur, __nv_bfloat16 *__restrict__ xg,
                                __nv_bfloat16 *__restrict__ xt0, float *__restrict__ sumsq,
                                int32_t *__restrict__ counters, int n_counters,
-                               unsigned long long *__restrict__ ssq_fix)
+                               unsigned long long *__restrict__ ssq_fix, int from_hidden,
+                               const __nv_bfloat16 *__restrict__ final_gamma, float eps)
 {
     pdl_trigger();
     pdl_wait();
@@ -350,13 +359,14 @@ __global__ void tc_prep_kernel(const __nv_bfloat16 *__restrict__ hidden, const i
     if (blockIdx.x == 0)
         for (int i = threadIdx.x; i < n_counters; i += blockDim.x) counters[i] = 0;
     __shared__ float red[8];
+    __shared__ float total_s;
     const int m = blockIdx.x;
     const size_t row = row_index ? (size_t)row_index[m] : (size_t)m;
     float ss = 0.f;
     for (int j = threadIdx.x; j < d; j += blockDim.x) {
         const float v = __bfloat162float(hidden[row * d + j]);
         const size_t o = (size_t)m * d + j;
-        h0f[o] = v;
+        if (!from_hidden) h0f[o] = v;
         hcur[o] = v;
         if (gamma1) {
             const float x = v * __bfloat162float(gamma1[j]);
@@ -364,8 +374,10 @@ __global__ void tc_prep_kernel(const __nv_bfloat16 *__restrict__ hidden, const i
             xg[o] = hi;
             xg[(size_t)lo_x * d + o] = __float2bfloat16_rn(x - __bfloat162float(hi));
         }
-        xt0[o] = __float2bfloat16(0.f);
-        xt0[(size_t)lo_xt * d + o] = __float2bfloat16(0.f);
+        if (!from_hidden) {
+            xt0[o] = __float2bfloat16(0.f);
+            xt0[(size_t)lo_xt * d + o] = __float2bfloat16(0.f);
+        }
         ss = fmaf(v, v, ss);
     }
 #pragma unroll
@@ -380,6 +392,20 @@ __global__ void tc_prep_kernel(const __nv_bfloat16 *__restrict__ hidden, const i
             // the chain kernel keeps sums of squares in 2^-24 fixed point (integer adds commute)
             ssq_fix[m] = (unsigned long long)__double2ll_rn((double)t * 16777216.0);
             for (int k = 1; k < 5; ++k) ssq_fix[k * 128 + m] = 0ull;
+        }
+        total_s = t;
+    }
+    if (from_hidden) {
+        __syncthreads();
+        const float rstd0 = final_gamma ? rsqrtf(total_s / (float)d + eps) : 1.f;
+        for (int j = threadIdx.x; j < d; j += blockDim.x) {
+            const float v = __bfloat162float(hidden[row * d + j]);
+            const float n0 = final_gamma ? v * rstd0 * __bfloat162float(final_gamma[j]) : v;
+            const size_t o = (size_t)m * d + j;
+            h0f[o] = v - n0;
+            const __nv_bfloat16 hi = __float2bfloat16_rn(n0);
+            xt0[o] = hi;
+            xt0[(size_t)lo_xt * d + o] = __float2bfloat16_rn(n0 - __bfloat162float(hi));
         }
     }
 }
@@ -572,7 +598,8 @@ cudaError_t tc_draft(Ctx *c, const void *hidden, const float *logits0, const int
     const bool few_rows = sk_head_rows_ok(M) && sk_heads_ok(c->cfg) &&
                           !(c->cfg.flags & MRP_FLAG_ROW_MAJOR_ONLY);
     const bool lm_few = sk_rows_ok(n_rs) && !(c->cfg.flags & MRP_FLAG_ROW_MAJOR_ONLY);
-    const bool f16_lm = c->use_f16_lm && n_rs >= kF16MinRowSteps && !lm_few;
+    // base logits computed in the pass need the operand exact to 2^-17: no fp16 operand there
+    const bool f16_lm = c->use_f16_lm && n_rs >= kF16MinRowSteps && !lm_few && !c->from_hidden;
     const bool chain = !(c->cfg.flags & (MRP_FLAG_ROW_MAJOR_ONLY | MRP_FLAG_NO_CHAIN)) && sk_heads_ok(c->cfg) &&
                        sk_chain(c, M, K, out, st, f16_lm, true) == cudaSuccess;
     c->lo_x = (few_rows || chain) ? sk_head_pad(M) : M;
@@ -583,7 +610,8 @@ cudaError_t tc_draft(Ctx *c, const void *hidden, const float *logits0, const int
                                          (const __nv_bfloat16 *)hidden, row_index, d, c->lo_x, c->lo_xt,
                                       (const __nv_bfloat16 *)c->heads[0].rms_gamma, h0f, hcur, xg, xt, sumsq,
                                       (int32_t *)(c->ws + c->lay.sk_counters), kSkMaxTiles,
-                                      (unsigned long long *)(c->ws + c->lay.ssq_fix)), "tc_prep_kernel");
+                                      (unsigned long long *)(c->ws + c->lay.ssq_fix), c->from_hidden ? 1 : 0,
+                                      (const __nv_bfloat16 *)c->final_gamma, c->cfg.rms_eps), "tc_prep_kernel");
     c->launches++;
     if (e != cudaSuccess) return e;
 
@@ -651,13 +679,15 @@ cudaError_t tc_draft(Ctx *c, const void *hidden, const float *logits0, const int
         memset(&p, 0, sizeof(p));
         // Row-steps of steps 1..K in 128-row blocks; CTA = (vocabulary range, group of row blocks).
         // Pick the split with the shortest longest CTA (in tiles), the fewest passes on ties.
-        const int rows = K * M, n_rb = (rows + 127) / 128, U = V / 16;
+        // (with the base logits computed in the pass, step 0 has rows of its own)
+        const int step_base = c->from_hidden ? 0 : 1;
+        const int rows = (K + 1 - step_base) * M, n_rb = (rows + 127) / 128, U = V / 16;
         const int best_g = choose_groups(n_rb, U, G);
         p.n_groups = best_g;
         n_slices = G / best_g;
         p.n_rb = n_rb; p.rows = rows;
         p.units_total = U; p.unit_rows = 16; p.n_boxes = 1; p.k_chunks = d / kBK;
-        p.a_row_base = M; p.a_part_rows = n_rs;
+        p.a_row_base = step_base * M; p.a_part_rows = n_rs; p.step_base = step_base;
         p.M = M; p.K = K; p.V = V; p.d = d; p.F = F; p.n_rs = n_rs;
         p.logits0 = logits0; p.row_index = row_index; p.partials = partials; p.logits_out = out.logits_out;
         p.status = status; p.user_status = out.status;

@@ -297,7 +297,7 @@ sk_gemm_kernel(const __grid_constant__ SkMaps maps, const SkParams p)
                 float a[RP];
 #pragma unroll
                 for (int j = 0; j < RP; ++j)
-                    a[j] = (valid && j < p.n_rs) ? __ldg(p.logits0 + rowoff_s[j] + v) : 0.f;
+                    a[j] = (valid && j < p.n_rs && p.logits0) ? __ldg(p.logits0 + rowoff_s[j] + v) : 0.f;
                 ok = __all_sync(0xffffffffu, mbar_wait(tfull_bar(acc), acc_ph, abort_flag, p));
                 if (!ok) break;
                 tc_fence_after();

@@ -64,6 +64,12 @@ def draft(ctx, hidden, logits0, row_index, M, K, out: DraftOut, stream=None):
     return out
 
 
+def draft_from_hidden(ctx, hidden, final_gamma, row_index, M, K, out: DraftOut, stream=None):
+    binding.mrp_draft_from_hidden(ctx, hidden, final_gamma, row_index, M, K, out.conf, out.lse, out.token,
+                                  out.margin, out.logits, out.hidden, out.status, stream=stream)
+    return out
+
+
 @dataclass
 class SelectOut:
     reveal_mask: torch.Tensor

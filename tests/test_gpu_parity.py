@@ -37,6 +37,25 @@ def run_gpu_draft(w, inp, K, flags=0, margin=True, logits=False, hidden=False, r
     return out, fam
 
 
+def run_gpu_draft_from_hidden(w, inp, K, final_gamma=None, flags=0, logits=False, hidden=False,
+                              row_index="inp"):
+    """mrp_draft_from_hidden on the same inputs: no base logits are handed over."""
+    heads, w_lm = harness.upload_weights(w, DEV)
+    ctx = binding.mrp_create(w.d, w.F, w.V, heads, w_lm, max_rows=max(inp.B * inp.L, 1),
+                             max_seqs=inp.B, block_len=inp.L, flags=flags)
+    ri = inp.row_index if isinstance(row_index, str) else row_index
+    M = inp.hidden.shape[0] if ri is None else len(ri)
+    hid = harness.to_device(inp.hidden, w.dtype, DEV)
+    g = None if final_gamma is None else harness.to_device(final_gamma, w.dtype, DEV)
+    ri_t = None if ri is None else torch.from_numpy(np.asarray(ri, np.int32)).to(DEV)
+    out = harness.alloc_draft_out(M, K, w.V, w.d, DEV, margin=True, logits=logits, hidden=hidden)
+    harness.draft_from_hidden(ctx, hid, g, ri_t, M, K, out)
+    torch.cuda.synchronize()
+    fam = ctx.family
+    binding.mrp_destroy(ctx)
+    return out, fam
+
+
 def check_stats(out, ref, dtype, cols=None):
     """Compare conf/lse/token of the GPU (all rows, or the columns `cols`) with the oracle."""
     tol = TOL[dtype]
@@ -316,3 +335,44 @@ def test_a_wait_that_nothing_completes_gives_up_and_reports():
     ref = oracle.draft(inp.hidden, inp.logits0, w.heads, w.w_lm, K=1)
     check_stats(out, ref, "bf16")
     binding.mrp_destroy(ctx)
+
+
+# ---- base logits computed from the hidden states in the LM-head pass (mrp_draft_from_hidden) ----
+
+@pytest.mark.parametrize("dtype,flags,d,F,V,B,L,K", [
+    ("f32", 0, 72, 136, 1000, 5, 3, 3),                                # CUDA-core kernels, ragged sizes
+    ("bf16", binding.MRP_FLAG_FORCE_SIMT, 72, 136, 1000, 5, 3, 2),
+    ("bf16", 0, 256, 512, 4096, 2, 4, 2),                              # few-row LM head + head chain
+    ("bf16", 0, 2048, 4096, 4096, 1, 4, 3),                            # the same at the 1.7B-class width
+    ("bf16", 0, 128, 256, 2048, 10, 4, 3),                             # row-major LM head, 160 row-steps
+    ("bf16", 0, 192, 320, 4112, 150, 1, 2),                            # two row blocks + step-0 rows of their own
+    ("bf16", binding.MRP_FLAG_ROW_MAJOR_ONLY, 256, 512, 4096, 2, 4, 2),
+])
+def test_base_logits_from_hidden_states(dtype, flags, d, F, V, B, L, K):
+    w = synth.make_weights(d, F, V, K, dtype, 55, head_std=0.05 if d <= 256 else 0.02)
+    inp = synth.make_inputs(w, B, L, 55, 1.0, 4.0)
+    gam = (1.0 + 0.25 * np.cos(np.arange(d))).astype(np.float32)
+    if dtype == "bf16":
+        gam = synth.bf16_round(gam)
+    for g in (None, gam):
+        out, fam = run_gpu_draft_from_hidden(w, inp, K, final_gamma=g, flags=flags, logits=True, hidden=True)
+        assert fam == ("simt" if (dtype == "f32" or flags & binding.MRP_FLAG_FORCE_SIMT) else "tcgen05")
+        ref = oracle.draft(inp.hidden, None, w.heads, w.w_lm, K=K, row_index=inp.row_index,
+                           final_gamma=g, want_logits=True, want_hidden=True)
+        check_stats(out, ref, dtype)
+        lg = out.logits.cpu().numpy().astype(np.float64)
+        rms = np.sqrt((ref.logits ** 2).mean(axis=2, keepdims=True))
+        rel = 1e-4 if dtype == "f32" else 2e-2
+        assert np.all(np.abs(lg - ref.logits) <= rel * np.maximum(np.abs(ref.logits), rms))
+        assert np.abs(out.hidden.cpu().numpy() - ref.hidden).max() <= (1e-4 if dtype == "f32" else 2e-2)
+    # a row subset, a shorter chain, and no chain at all (step 0 only)
+    sub = inp.row_index[::2]
+    for k in (max(K - 1, 1), 0):
+        out, _ = run_gpu_draft_from_hidden(w, inp, k, final_gamma=gam, flags=flags, row_index=sub, hidden=True)
+        ref = oracle.draft(inp.hidden, None, w.heads, w.w_lm, K=k, row_index=sub, final_gamma=gam, want_hidden=True)
+        check_stats(out, ref, dtype)
+        assert np.abs(out.hidden.cpu().numpy() - ref.hidden).max() <= (1e-4 if dtype == "f32" else 2e-2)
+    # the ordinary entry point afterwards on a fresh context: nothing of the mode lingers
+    out, _ = run_gpu_draft(w, inp, K, flags=flags)
+    ref = oracle.draft(inp.hidden, inp.logits0, w.heads, w.w_lm, K=K, row_index=inp.row_index)
+    check_stats(out, ref, dtype)
