@@ -44,6 +44,9 @@ def parse_args():
     ap.add_argument("--flags", type=int, default=0, help="mrp_config.flags (MRP_FLAG_* bits) for A/B timing")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--from-hidden", action="store_true",
+                    help="draft with mrp_draft_from_hidden: the base logits are computed in the LM-head pass "
+                         "instead of being an input (no [rows, V] read or host copy)")
     return ap.parse_args()
 
 
@@ -137,12 +140,16 @@ def replica_throughput(dist, device, units_per_rank, seconds):
     return world * units_per_rank / seconds, seconds
 
 
-def lm_head_roofline(cfg, M, lm_ms, peaks, peaks_kind, traffic):
+def lm_head_roofline(cfg, M, lm_ms, peaks, peaks_kind, traffic, from_hidden=False):
     """Roofline of the fused LM-head kernel: algorithmic bytes 2Vd + 4MV + 2KMd (one read of
-    the LM head, one read of l_0, the stacked residual rows), flops 2KMVd."""
+    the LM head, one read of l_0, the stacked residual rows), flops 2KMVd.  With the base
+    logits computed in the pass: bytes 2Vd + 2(K+1)Md, flops 2(K+1)MVd."""
     V, d, K = cfg["V"], cfg["d"], cfg["K"]
     nbytes = 2.0 * V * d + 4.0 * M * V + 2.0 * K * M * d
     flops = 2.0 * K * M * V * d
+    if from_hidden:
+        nbytes = 2.0 * V * d + 2.0 * (K + 1) * M * d
+        flops = 2.0 * (K + 1) * M * V * d
     t_hbm = nbytes / (peaks["hbm_gbs"] * 1e9)
     t_tc = flops / (peaks["bf16_tflops_sustained"] * 1e12)
     sec = lm_ms * 1e-3
@@ -359,7 +366,10 @@ def main():
     launches = [0]
 
     def step():
-        harness.draft(ctx, hid, l0, ri, M, K, out)
+        if args.from_hidden:
+            harness.draft_from_hidden(ctx, hid, None, ri, M, K, out)
+        else:
+            harness.draft(ctx, hid, l0, ri, M, K, out)
         n = ctx.last_launch_count
         harness.select(ctx, out.conf, out.token, ri, M, K, B, L, mode, sel, tau=cfg["tau"])
         n += ctx.last_launch_count
@@ -422,7 +432,8 @@ def main():
     n_calls = max(n_calls, 1)
     peaks, peaks_kind = load_peaks()
     roofline = lm_head_roofline(cfg, M, ms_lm / n_calls, peaks, peaks_kind,
-                                NCU_TRAFFIC_BYTES.get(cfg["name"]))
+                                None if args.from_hidden else NCU_TRAFFIC_BYTES.get(cfg["name"]),
+                                from_hidden=args.from_hidden)
     phases = {"heads_ms": ms_heads / n_calls, "lm_head_ms": ms_lm / n_calls,
               "combine_ms": ms_comb / n_calls, "family": ctx.family}
 
@@ -435,13 +446,16 @@ def main():
         h_ri = ri.cpu().pin_memory()
         res = [out.conf, out.token, sel.reveal_mask, sel.remask_mask, sel.out_token, sel.draft_len, alen]
         h_res = [torch.empty_like(t, device="cpu").pin_memory() for t in res]
-        bi = h_hid.numel() * h_hid.element_size() + h_l0.numel() * 4 + h_ri.numel() * 4
+        bi = h_hid.numel() * h_hid.element_size() + h_ri.numel() * 4
+        if not args.from_hidden:
+            bi += h_l0.numel() * 4
         bo = sum(t.numel() * t.element_size() for t in res)
         n_e2e = max(3, min(args.steps, 300))
 
         def e2e_body():
             hid.copy_(h_hid, non_blocking=True)
-            l0.copy_(h_l0, non_blocking=True)
+            if not args.from_hidden:
+                l0.copy_(h_l0, non_blocking=True)
             ri.copy_(h_ri, non_blocking=True)
             step()
             for s, dcpu in zip(res, h_res):
@@ -499,6 +513,7 @@ def main():
             "dtype": "bf16" if cfg["dtype"] == "bf16" else "f32", "data": "synthetic",
             "config": {"workload": cfg["name"], "rows": M, "chain": K, "d": cfg["d"], "d_ff": cfg["F"],
                        "vocab": cfg["V"], "seqs": B, "block_len": L, "mode": cfg["mode"],
+                       "entry": "mrp_draft_from_hidden" if args.from_hidden else "mrp_draft",
                        "l2": "weights streamed per step (%.0f MB) exceed the 126 MB L2; no flush"
                              % ((2.0 * cfg["V"] * cfg["d"] + K * 6.0 * cfg["d"] * cfg["F"]) / 1e6),
                        "parallelism": "replicas x%d" % world},

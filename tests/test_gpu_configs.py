@@ -74,6 +74,39 @@ def test_config1_decode_shape_all_rows():
     binding.mrp_destroy(ctx)
 
 
+def test_config1_decode_shape_base_logits_from_hidden_states():
+    """Config 1 through mrp_draft_from_hidden (no base logits handed over), with and without the
+    backbone's final norm; all rows and all vocabulary entries against the oracle."""
+    cfg = synth.CONFIGS[1]
+    w = synth.make_weights(cfg["d"], cfg["F"], cfg["V"], cfg["n_heads"], cfg["dtype"], cfg["seed"])
+    dev = Device(w)
+    _, inp = synth.make_config(cfg, w)
+    ctx = dev.ctx(4, 1, 4)
+    K, M = cfg["K"], 4
+    hid = harness.to_device(inp.hidden, w.dtype, DEV)
+    ri = torch.from_numpy(inp.row_index).to(DEV)
+    gam = synth.bf16_round((1.0 + 0.25 * np.cos(np.arange(w.d))).astype(np.float32))
+    for g in (None, gam):
+        out = harness.alloc_draft_out(M, K, w.V, w.d, DEV, logits=True, hidden=True)
+        harness.draft_from_hidden(ctx, hid, None if g is None else harness.to_device(g, w.dtype, DEV),
+                                  ri, M, K, out)
+        torch.cuda.synchronize()
+        ref = oracle.draft(inp.hidden, None, w.heads, w.w_lm, K=K, row_index=inp.row_index,
+                           final_gamma=g, want_logits=True, want_hidden=True)
+        check_stats(out, ref, "bf16")
+        lg = out.logits.cpu().numpy().astype(np.float64)
+        rms = np.sqrt((ref.logits ** 2).mean(axis=2, keepdims=True))
+        assert np.all(np.abs(lg - ref.logits) <= 2e-2 * np.maximum(np.abs(ref.logits), rms))
+    # without a final norm the synthetic base logits are W_lm h_0 rounded to fp32: the ordinary
+    # entry point on those must give the same statistics up to that rounding
+    out_b, _ = gpu_draft(dev, ctx, inp, K)
+    out_a = harness.alloc_draft_out(M, K, w.V, w.d, DEV)
+    harness.draft_from_hidden(ctx, hid, None, ri, M, K, out_a)
+    torch.cuda.synchronize()
+    assert torch.allclose(out_a.lse, out_b.lse, atol=1e-3) and torch.allclose(out_a.conf, out_b.conf, atol=1e-3)
+    binding.mrp_destroy(ctx)
+
+
 def test_config2_speculative_shape_sampled_rows_and_verify():
     cfg = synth.CONFIGS[2]
     w = synth.make_weights(cfg["d"], cfg["F"], cfg["V"], cfg["n_heads"], cfg["dtype"], cfg["seed"])
@@ -179,6 +212,27 @@ def test_sweep_points_sampled_rows(sweep_dev, M, K):
     l0 = torch.from_numpy(inp.logits0).to(DEV)
     assert torch.equal(l0.argmax(dim=1).int().cpu(), out.token[0].cpu())
     assert torch.allclose(torch.logsumexp(l0, dim=1), out.lse[0], atol=2e-3)
+    binding.mrp_destroy(ctx)
+
+
+@pytest.mark.parametrize("M,K", [(4, 2), (64, 2), (256, 4), (1024, 1)])
+def test_sweep_points_base_logits_from_hidden_states(sweep_dev, M, K):
+    dev = sweep_dev
+    cfg = synth.sweep_config(M, K)
+    _, inp = synth.make_config(cfg, dev.w, logits_fn=dev.logits_fn)
+    ctx = dev.ctx(M, M, 1, n_heads=K)
+    hid = harness.to_device(inp.hidden, dev.w.dtype, DEV)
+    ri = torch.from_numpy(inp.row_index).to(DEV)
+    gam = synth.bf16_round((1.0 + 0.25 * np.cos(np.arange(dev.w.d))).astype(np.float32))
+    out = harness.alloc_draft_out(M, K, dev.w.V, dev.w.d, DEV, margin=False)
+    harness.draft_from_hidden(ctx, hid, harness.to_device(gam, dev.w.dtype, DEV), ri, M, K, out)
+    torch.cuda.synchronize()
+    sample = np.unique(np.array([0, M // 3, M // 2, M - 1]))
+    ref = oracle.draft(inp.hidden, None, dev.w.heads, dev.w.w_lm, K=K, row_index=inp.row_index[sample],
+                       final_gamma=gam)
+    check_stats(out, ref, "bf16", cols=sample)
+    conf = out.conf.cpu().numpy()
+    assert np.all(conf > 1.0 / dev.w.V) and np.all(conf <= 1.0 + 1e-6)
     binding.mrp_destroy(ctx)
 
 
