@@ -165,8 +165,7 @@ int mrp_draft(mrp_ctx *ctx, const void *hidden, const float *logits0, const int3
  * and step k's logits are W_lm (n_0 + h_k - h_0).  No [n_rows, V] input is read, and the backbone
  * needs no LM-head pass of its own for these rows.
  *   final_norm_gamma [d] in the context's dtype, or NULL; the other arguments and the outputs
- *   are those of mrp_draft.  On the tensor-core kernels the operand rows are always carried as
- *   bf16 hi + lo pairs in this mode.  Errors: INVALID_ARG, CUDA.
+ *   are those of mrp_draft.  Errors: INVALID_ARG, CUDA.
  */
 int mrp_draft_from_hidden(mrp_ctx *ctx, const void *hidden, const void *final_norm_gamma,
                           const int32_t *row_index, int32_t M, int32_t K, const mrp_draft_out *out,

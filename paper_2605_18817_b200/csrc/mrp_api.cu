@@ -36,7 +36,7 @@ WorkspaceLayout workspace_layout(const mrp_config &cfg)
                 ((long long)cfg.n_heads + 1) * cfg.max_rows >= kF16MinRowSteps && cfg.d % 64 == 0 &&
                 cfg.d_ff % 64 == 0 && cfg.vocab % 16 == 0 && cfg.n_heads <= 4;
     l.w16 = take(l.has_f16 ? (size_t)cfg.vocab * d * 2 : 0);
-    l.xt16 = take(l.has_f16 ? (size_t)cfg.n_heads * rows * d * 2 : 0);
+    l.xt16 = take(l.has_f16 ? (size_t)steps * rows * d * 2 : 0);
     l.total = off;
     return l;
 }

@@ -313,8 +313,9 @@ __global__ void combine_kernel(const Partial *__restrict__ partials, int n_slice
         p = (lane & o) ? merge_partial(q, p) : merge_partial(p, q);
     }
     float top = p.mx;      // the top logit as the sum of exponentials saw it
-    if (fix.w && rs >= fix.M) {
+    if (fix.w && (rs >= fix.M || !fix.logits0)) {
         // exact top logit: l_0[row, tok] + W[tok] . (hi + lo), fp32, fixed summation order
+        // (no l_0 term, and step 0 included, when the base logits are computed in the pass)
         const int tok = __shfl_sync(0xffffffffu, p.idx, 0);
         const int m = rs % fix.M;
         const size_t row = fix.row_index ? (size_t)fix.row_index[m] : (size_t)m;
@@ -330,7 +331,7 @@ __global__ void combine_kernel(const Partial *__restrict__ partials, int n_slice
             dot = fmaf(w2.y, h2.y + l2.y, dot);
         }
         dot = warp_sum(dot);
-        top = fix.logits0[row * (size_t)fix.V + tok] + dot;
+        top = (fix.logits0 ? fix.logits0[row * (size_t)fix.V + tok] : 0.f) + dot;
     }
     if (lane == 0) {
         // the term of the top token entered the sum as exp(0) = 1: swap in its exact value

@@ -549,7 +549,7 @@ cudaError_t sk_chain(Ctx *c, int M, int K, const mrp_draft_out &out, cudaStream_
         dn.gamma_next = (k < K) ? (const __nv_bfloat16 *)c->heads[k].rms_gamma : nullptr;
         dn.xg_next = (k < K) ? xg : nullptr;
         dn.xt_k = xt + (size_t)k * M * d;
-        dn.xt16_k = f16_lm ? (__half *)(c->ws + c->lay.xt16) + (size_t)(k - 1) * M * d : nullptr;
+        dn.xt16_k = f16_lm ? (__half *)(c->ws + c->lay.xt16) + (size_t)(k - (c->from_hidden ? 0 : 1)) * M * d : nullptr;
         dn.hidden_out = (k == K) ? out.hidden_out : nullptr;
     }
     cudaError_t e;

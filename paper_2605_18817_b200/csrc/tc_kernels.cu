@@ -351,7 +351,7 @@ __global__ void tc_prep_kernel(const __nv_bfloat16 *__restrict__ hidden, const i
                                __nv_bfloat16 *__restrict__ xt0, float *__restrict__ sumsq,
                                int32_t *__restrict__ counters, int n_counters,
                                unsigned long long *__restrict__ ssq_fix, int from_hidden,
-                               const __nv_bfloat16 *__restrict__ final_gamma, float eps)
+                               const __nv_bfloat16 *__restrict__ final_gamma, float eps, __half *__restrict__ xt16_0)
 {
     pdl_trigger();
     pdl_wait();
@@ -406,6 +406,7 @@ __global__ void tc_prep_kernel(const __nv_bfloat16 *__restrict__ hidden, const i
             const __nv_bfloat16 hi = __float2bfloat16_rn(n0);
             xt0[o] = hi;
             xt0[(size_t)lo_xt * d + o] = __float2bfloat16_rn(n0 - __bfloat162float(hi));
+            if (xt16_0) xt16_0[o] = __float2half_rn(n0);
         }
     }
 }
@@ -598,8 +599,7 @@ cudaError_t tc_draft(Ctx *c, const void *hidden, const float *logits0, const int
     const bool few_rows = sk_head_rows_ok(M) && sk_heads_ok(c->cfg) &&
                           !(c->cfg.flags & MRP_FLAG_ROW_MAJOR_ONLY);
     const bool lm_few = sk_rows_ok(n_rs) && !(c->cfg.flags & MRP_FLAG_ROW_MAJOR_ONLY);
-    // base logits computed in the pass need the operand exact to 2^-17: no fp16 operand there
-    const bool f16_lm = c->use_f16_lm && n_rs >= kF16MinRowSteps && !lm_few && !c->from_hidden;
+    const bool f16_lm = c->use_f16_lm && n_rs >= kF16MinRowSteps && !lm_few;
     const bool chain = !(c->cfg.flags & (MRP_FLAG_ROW_MAJOR_ONLY | MRP_FLAG_NO_CHAIN)) && sk_heads_ok(c->cfg) &&
                        sk_chain(c, M, K, out, st, f16_lm, true) == cudaSuccess;
     c->lo_x = (few_rows || chain) ? sk_head_pad(M) : M;
@@ -611,7 +611,9 @@ cudaError_t tc_draft(Ctx *c, const void *hidden, const float *logits0, const int
                                       (const __nv_bfloat16 *)c->heads[0].rms_gamma, h0f, hcur, xg, xt, sumsq,
                                       (int32_t *)(c->ws + c->lay.sk_counters), kSkMaxTiles,
                                       (unsigned long long *)(c->ws + c->lay.ssq_fix), c->from_hidden ? 1 : 0,
-                                      (const __nv_bfloat16 *)c->final_gamma, c->cfg.rms_eps), "tc_prep_kernel");
+                                      (const __nv_bfloat16 *)c->final_gamma, c->cfg.rms_eps,
+                                      (c->from_hidden && f16_lm) ? (__half *)(c->ws + c->lay.xt16) : (__half *)nullptr),
+                             "tc_prep_kernel");
     c->launches++;
     if (e != cudaSuccess) return e;
 
@@ -656,7 +658,7 @@ cudaError_t tc_draft(Ctx *c, const void *hidden, const float *logits0, const int
         p.gamma_next = (k < K) ? (const __nv_bfloat16 *)c->heads[k].rms_gamma : nullptr;
         p.xg_next = (k < K) ? xg : nullptr;
         p.xt_k = xt + (size_t)k * M * d;
-        p.xt16_k = f16_lm ? (__half *)(c->ws + c->lay.xt16) + (size_t)(k - 1) * M * d : nullptr;
+        p.xt16_k = f16_lm ? (__half *)(c->ws + c->lay.xt16) + (size_t)(k - (c->from_hidden ? 0 : 1)) * M * d : nullptr;
         p.sumsq_out = sumsq;
         p.hidden_out = (k == K) ? out.hidden_out : nullptr;
         p.status = status; p.user_status = out.status;

@@ -685,7 +685,7 @@ cudaError_t sk_down(Ctx *c, int k, int M, int K, const mrp_draft_out &out, cudaS
     p.gamma_next = (k < K) ? (const __nv_bfloat16 *)c->heads[k].rms_gamma : nullptr;
     p.xg_next = (k < K) ? (__nv_bfloat16 *)(c->ws + c->lay.xg) : nullptr;
     p.xt_k = (__nv_bfloat16 *)(c->ws + c->lay.xt) + (size_t)k * M * d;
-    p.xt16_k = f16_lm ? (__half *)(c->ws + c->lay.xt16) + (size_t)(k - 1) * M * d : nullptr;
+    p.xt16_k = f16_lm ? (__half *)(c->ws + c->lay.xt16) + (size_t)(k - (c->from_hidden ? 0 : 1)) * M * d : nullptr;
     p.sumsq_out = (float *)(c->ws + c->lay.sumsq);
     p.hidden_out = (k == K) ? out.hidden_out : nullptr;
     sk_finish_shape(p, 0);

@@ -260,3 +260,32 @@ def test_fp16_operand_mode_stays_close_to_exact_operands_on_every_row(sweep_dev,
     clear = b.margin > 1e-2
     assert torch.equal(a.token[clear], b.token[clear])
     assert torch.equal(a.conf[0], b.conf[0])          # step 0 never touches the operands
+
+
+@pytest.mark.parametrize("M,K", [(16, 2), (64, 4), (256, 1), (1024, 2), (4096, 1)])
+def test_fp16_operand_mode_of_the_base_logits_pass_stays_close_to_exact_operands(sweep_dev, M, K):
+    """The same comparison for mrp_draft_from_hidden, where the base logits go through the
+    operand as well: every row-step, step 0 included, against MRP_FLAG_EXACT_OPERANDS."""
+    dev = sweep_dev
+    cfg = synth.sweep_config(M, K)
+    _, inp = synth.make_config(cfg, dev.w, logits_fn=dev.logits_fn)
+    hid = harness.to_device(inp.hidden, dev.w.dtype, DEV)
+    ri = torch.from_numpy(inp.row_index).to(DEV)
+    gam = harness.to_device(synth.bf16_round((1.0 + 0.25 * np.cos(np.arange(dev.w.d))).astype(np.float32)),
+                            dev.w.dtype, DEV)
+    for g in (None, gam):
+        outs = []
+        for flags in (0, binding.MRP_FLAG_EXACT_OPERANDS):
+            ctx = dev.ctx(M, M, 1, n_heads=K, flags=flags)
+            out = harness.alloc_draft_out(M, K, dev.w.V, dev.w.d, DEV, margin=True)
+            harness.draft_from_hidden(ctx, hid, g, ri, M, K, out)
+            torch.cuda.synchronize()
+            outs.append(out)
+            binding.mrp_destroy(ctx)
+        a, b = outs
+        dconf = (a.conf - b.conf).abs().max().item()
+        dlse = (a.lse - b.lse).abs().max().item()
+        print("M=%d K=%d norm=%s max|dconf|=%.2e max|dlse|=%.2e" % (M, K, g is not None, dconf, dlse))
+        assert dconf <= 1.5e-3 and dlse <= 1.5e-3
+        clear = b.margin > 1e-2
+        assert torch.equal(a.token[clear], b.token[clear])
