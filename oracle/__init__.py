@@ -6,7 +6,8 @@ may import this package; the product path never does.  Nothing here touches CUDA
 
 The functions mirror the paper's steps (Algorithms 2-4): ``draft`` runs the head chain and
 the shared LM head and returns per-step softmax statistics, ``select`` applies the static /
-dynamic reveal rules and the remask rule, ``verify`` computes accepted draft prefixes.
+dynamic reveal rules and the remask rule, ``verify`` computes accepted draft prefixes, ``commit``
+applies the outcome to the block state (x_t -> x_{t-1}) and lists the positions still masked.
 """
 from __future__ import annotations
 
@@ -208,3 +209,42 @@ def verify(draft_tok, verify_tok, draft_len, positionwise=False):
     if rc != 0:
         raise RuntimeError("mrp_oracle_verify failed (%d)" % rc)
     return accept_len, accept_mask
+
+
+@dataclass
+class CommitResult:
+    tokens: np.ndarray        # [B*L] int32, -1 = still masked
+    row_index: np.ndarray     # [n_masked] int32, dense positions still masked, ascending
+    block_masked: np.ndarray  # [B] int32
+
+
+def commit(tokens, sel: SelectResult, B, L, accept_mask=None) -> CommitResult:
+    """One transition x_t -> x_{t-1} of the block state (the last lines of Algorithms 2-4).
+
+    ``tokens`` [B*L] holds the committed token of every position, -1 while it is masked.
+    ``accept_mask=None``: every position the selection took is unmasked with its token --
+    the reveals of all steps in direct decoding (Algorithm 2), the members of R that survived
+    remasking in the dynamic regime (Algorithm 4).  With ``accept_mask`` [B, Kd] (speculative
+    decoding, Algorithm 3): the step-0 reveals are unmasked, a drafted position only where the
+    backbone accepted the draft; rejected drafts stay masked.  Plain loops, no arithmetic.
+    """
+    tokens = np.array(tokens, dtype=np.int32).reshape(B * L).copy()
+    for p in range(B * L):
+        if tokens[p] >= 0:
+            continue
+        if accept_mask is None:
+            if sel.out_token[p] >= 0:
+                tokens[p] = sel.out_token[p]
+        elif sel.step_of[p] == 0:
+            tokens[p] = sel.out_token[p]
+    if accept_mask is not None:
+        accept_mask = np.asarray(accept_mask).reshape(B, -1)
+        for b in range(B):
+            for s in range(accept_mask.shape[1]):
+                if accept_mask[b, s] and sel.draft_pos[b, s] >= 0:
+                    p = b * L + int(sel.draft_pos[b, s])
+                    if tokens[p] < 0:
+                        tokens[p] = sel.draft_tok[b, s]
+    row_index = np.array([p for p in range(B * L) if tokens[p] < 0], dtype=np.int32)
+    block_masked = np.array([int(np.sum(tokens[b * L:(b + 1) * L] < 0)) for b in range(B)], dtype=np.int32)
+    return CommitResult(tokens, row_index, block_masked)

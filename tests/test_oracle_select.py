@@ -202,3 +202,81 @@ def test_verify_accept_length_is_first_mismatch_and_geometric_mean():
     expect = sum(0.7 ** j for j in range(1, 5))
     sd = alen.std() / np.sqrt(B)
     assert abs(alen.mean() - expect) < 4 * sd + 1e-3
+
+
+# ---- the block-state transition x_t -> x_{t-1} (oracle.commit) ----
+
+def _stats(rng, K, M, V=1000):
+    return rng.random((K + 1, M)).astype(np.float32), rng.integers(0, V, (K + 1, M)).astype(np.int32)
+
+
+def test_commit_hand_example_for_the_three_decoding_modes():
+    # one block of 6 positions, position 2 already holds token 7
+    tokens = np.array([-1, -1, 7, -1, -1, -1], np.int32)
+    ri = np.array([0, 1, 3, 4, 5], np.int32)
+    conf = np.array([[0.9, 0.2, 0.5, 0.1, 0.3],      # step 0: position 0 is the most confident
+                     [0.0, 0.3, 0.8, 0.2, 0.1],      # step 1: position 3
+                     [0.0, 0.6, 0.0, 0.7, 0.2]], np.float32)   # step 2: position 4
+    tok = np.array([[10, 11, 13, 14, 15], [20, 21, 23, 24, 25], [30, 31, 33, 34, 35]], np.int32)
+    sel = oracle.select(conf, tok, ri, 1, 6, oracle.STATIC)
+    # Algorithm 2: reveals of every step are unmasked
+    c = oracle.commit(tokens, sel, 1, 6)
+    assert c.tokens.tolist() == [10, -1, 7, 23, 34, -1]
+    assert c.row_index.tolist() == [1, 5] and c.block_masked.tolist() == [2]
+    # Algorithm 3: the backbone accepts the first draft only
+    c = oracle.commit(tokens, sel, 1, 6, accept_mask=np.array([[1, 0]], np.int8))
+    assert c.tokens.tolist() == [10, -1, 7, 23, -1, -1]
+    assert c.row_index.tolist() == [1, 4, 5]
+    c = oracle.commit(tokens, sel, 1, 6, accept_mask=np.array([[0, 0]], np.int8))
+    assert c.tokens.tolist() == [10, -1, 7, -1, -1, -1]
+    # Algorithm 4: R = {0, 3} at tau = 0.45; the update drops position 0 below tau, so it is remasked
+    sel = oracle.select(conf[:2], tok[:2], ri, 1, 6, oracle.DYNAMIC_REMASK, tau=0.45)
+    assert sel.reveal_mask.tolist() == [1, 0, 0, 1, 0, 0] and sel.remask_mask.tolist() == [1, 0, 0, 0, 0, 0]
+    c = oracle.commit(tokens, sel, 1, 6)
+    assert c.tokens.tolist() == [-1, -1, 7, 13, -1, -1]
+
+
+def test_commit_invariants_on_random_states():
+    rng = np.random.default_rng(5)
+    for case in range(30):
+        B, L, K = 1 + case % 5, 1 + (case * 7) % 13, case % 4
+        tokens = np.where(rng.random(B * L) < 0.6, -1, rng.integers(0, 99, B * L)).astype(np.int32)
+        ri = np.flatnonzero(tokens < 0).astype(np.int32)
+        if ri.size == 0:
+            continue
+        conf, tok = _stats(rng, K, ri.size)
+        mode = oracle.STATIC if case % 2 == 0 else oracle.DYNAMIC_REMASK
+        sel = oracle.select(conf, tok, ri, B, L, mode, tau=0.5, r_reveal=1 + case % 2, r_draft=1)
+        acc = None
+        if mode == oracle.STATIC and case % 4 == 0 and K > 0:
+            vt = np.where(rng.random((B, K)) < 0.6, sel.draft_tok, -5).astype(np.int32)
+            _, acc = oracle.verify(sel.draft_tok, vt, sel.draft_len)
+        c = oracle.commit(tokens, sel, B, L, accept_mask=acc)
+        was_masked = tokens < 0
+        newly = was_masked & (c.tokens >= 0)
+        assert np.array_equal(c.tokens[~was_masked], tokens[~was_masked])      # committed tokens never change
+        assert np.array_equal(c.tokens[newly], sel.out_token[newly])            # new ones are the selected tokens
+        assert np.array_equal(c.row_index, np.flatnonzero(c.tokens < 0))
+        assert c.block_masked.sum() == c.row_index.size
+        if acc is None:
+            assert newly.sum() == (sel.out_token >= 0).sum()
+        else:
+            assert newly.sum() == (sel.step_of == 0).sum() + acc.sum()
+
+
+def test_direct_decoding_loop_needs_ceil_L_over_K_plus_one_forwards():
+    """Algorithm 2 with r = 1: every backbone forward unmasks min(K + 1, masked) positions of a
+    block, so a block of L positions is done after ceil(L / (K + 1)) forwards, whatever the statistics."""
+    rng = np.random.default_rng(9)
+    for L, K in ((4, 1), (7, 2), (32, 3), (5, 0)):
+        B = 3
+        tokens = np.full(B * L, -1, np.int32)
+        n = 0
+        while (tokens < 0).any():
+            ri = np.flatnonzero(tokens < 0).astype(np.int32)
+            conf, tok = _stats(rng, K, ri.size)
+            sel = oracle.select(conf, tok, ri, B, L, oracle.STATIC)
+            tokens = oracle.commit(tokens, sel, B, L).tokens
+            n += 1
+            assert n <= L
+        assert n == -(-L // (K + 1))
