@@ -236,6 +236,39 @@ int mrp_verify(mrp_ctx *ctx, const int32_t *draft_tok, const int32_t *verify_tok
                int32_t *accept_len, int8_t *accept_mask, void *cuda_stream);
 
 /*
+ * Block state kept on the device between backbone forwards, and its transition x_t -> x_{t-1}.
+ *   tokens       [B*L] int32, in/out: token committed at the position, -1 while it is masked
+ *   row_index    [B*L] int32, out: dense positions b*L+i still masked after the call, ascending
+ *                (its first *n_masked entries; the argument of the next mrp_draft and
+ *                mrp_reveal_remask)
+ *   n_masked     [1] int32, out
+ *   block_masked [B] int32, out: positions still masked per block (0 = the block is done)
+ */
+typedef struct {
+    int32_t *tokens;
+    int32_t *row_index;
+    int32_t *n_masked;
+    int32_t *block_masked;
+} mrp_block_state;
+
+/*
+ * Apply the outcome of one pass to the block state (the closing lines of Algorithms 2-4).
+ *   accept_mask == NULL: every position the selection took (sel->out_token >= 0) is unmasked
+ *     with that token: the reveals of all steps in direct decoding (Algorithm 2 "Reveal r
+ *     tokens" at k = 0..K), and in the dynamic regime the members of R that survived remasking
+ *     (Algorithm 4 "Remask positions i in R where confidence is below tau").
+ *   accept_mask [B, Kd] int8 (from mrp_verify; speculative decoding, Algorithm 3): the step-0
+ *     reveals are unmasked; drafted position sel->draft_pos[b, s] takes sel->draft_tok[b, s]
+ *     only where accept_mask[b, s] != 0 ("Reject drafted positions ...; remask rejected
+ *     positions").
+ * Positions that already hold a token are never changed.  sel is the mrp_select_out of this
+ * pass (reveal_mask and remask_mask are not read); Kd as in mrp_reveal_remask; 1 <= B <=
+ * max_seqs, 1 <= L <= block_len.  Errors: INVALID_ARG, CUDA.
+ */
+int mrp_commit(mrp_ctx *ctx, const mrp_select_out *sel, const int8_t *accept_mask, int32_t B,
+               int32_t L, int32_t Kd, const mrp_block_state *state, void *cuda_stream);
+
+/*
  * mrp_reveal_remask without a context and without any allocation (the paper has no
  * counterpart: this is a packaging variant of the call above, same rules, same outputs).
  *

@@ -30,7 +30,7 @@ MRP_DEV_NONFINITE, MRP_DEV_TIMEOUT = 1, 2
 EXPORTS = ("mrp_workspace_bytes", "mrp_create", "mrp_destroy", "mrp_draft", "mrp_reveal_remask",
            "mrp_verify", "mrp_last_launch_count", "mrp_kernel_family", "mrp_status_string",
            "mrp_profile_enable", "mrp_profile_read", "mrp_last_error",
-           "mrp_reveal_remask_noalloc", "mrp_selftest_wait_timeout", "mrp_draft_from_hidden")
+           "mrp_reveal_remask_noalloc", "mrp_selftest_wait_timeout", "mrp_draft_from_hidden", "mrp_commit")
 MRP_NOALLOC_MAX_POSITIONS = 65536
 MRP_ERR_CAPACITY = 7
 
@@ -67,6 +67,11 @@ class mrp_select_out(ctypes.Structure):
                 ("draft_len", ctypes.c_void_p)]
 
 
+class mrp_block_state(ctypes.Structure):
+    _fields_ = [("tokens", ctypes.c_void_p), ("row_index", ctypes.c_void_p),
+                ("n_masked", ctypes.c_void_p), ("block_masked", ctypes.c_void_p)]
+
+
 def _load():
     if not os.path.exists(LIB_PATH):
         raise ImportError(
@@ -87,6 +92,9 @@ def _load():
     lib.mrp_draft.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
                               ctypes.c_int32, ctypes.c_int32, ctypes.POINTER(mrp_draft_out),
                               ctypes.c_void_p]
+    lib.mrp_commit.restype = ctypes.c_int
+    lib.mrp_commit.argtypes = [ctypes.c_void_p, ctypes.POINTER(mrp_select_out), ctypes.c_void_p, ctypes.c_int32,
+                               ctypes.c_int32, ctypes.c_int32, ctypes.POINTER(mrp_block_state), ctypes.c_void_p]
     lib.mrp_draft_from_hidden.restype = ctypes.c_int
     lib.mrp_draft_from_hidden.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
                                           ctypes.c_int32, ctypes.c_int32, ctypes.POINTER(mrp_draft_out),
@@ -316,6 +324,23 @@ def mrp_selftest_wait_timeout(ctx: Context, status, stream=None) -> None:
     rc = lib.mrp_selftest_wait_timeout(ctx.handle, _ptr(status), _stream(stream))
     if rc != 0:
         raise MrpError("mrp_selftest_wait_timeout", rc)
+
+
+def mrp_commit(ctx: Context, B, L, Kd, *, out_token, step_of, draft_pos, draft_tok, accept_mask=None,
+               tokens, row_index, n_masked, block_masked, stream=None) -> None:
+    """Apply one pass's selection (and, if given, verification) to the block state."""
+    for t, dt, nm in ((out_token, torch.int32, "out_token"), (step_of, torch.int8, "step_of"),
+                      (draft_pos, torch.int32, "draft_pos"), (draft_tok, torch.int32, "draft_tok"),
+                      (accept_mask, torch.int8, "accept_mask"), (tokens, torch.int32, "tokens"),
+                      (row_index, torch.int32, "row_index"), (n_masked, torch.int32, "n_masked"),
+                      (block_masked, torch.int32, "block_masked")):
+        _check(t, dt, nm)
+    sel = mrp_select_out(None, None, _ptr(out_token), _ptr(step_of), _ptr(draft_pos), _ptr(draft_tok), None)
+    state = mrp_block_state(_ptr(tokens), _ptr(row_index), _ptr(n_masked), _ptr(block_masked))
+    rc = lib.mrp_commit(ctx.handle, ctypes.byref(sel), _ptr(accept_mask), int(B), int(L), int(Kd),
+                        ctypes.byref(state), _stream(stream))
+    if rc != 0:
+        raise MrpError("mrp_commit", rc, lib.mrp_last_error(ctx.handle).decode())
 
 
 def mrp_verify(ctx: Context, draft_tok, verify_tok, draft_len, B, Kd, positionwise, accept_len,

@@ -280,6 +280,23 @@ int mrp_verify(mrp_ctx *ctx, const int32_t *draft_tok, const int32_t *verify_tok
     return e == cudaSuccess ? MRP_OK : MRP_ERR_CUDA;
 }
 
+int mrp_commit(mrp_ctx *ctx, const mrp_select_out *sel, const int8_t *accept_mask, int32_t B, int32_t L,
+               int32_t Kd, const mrp_block_state *state, void *cuda_stream)
+{
+    if (!ctx || !sel || !state) return MRP_ERR_INVALID_ARG;
+    Ctx &c = ctx->c;
+    if (B < 1 || B > c.cfg.max_seqs || L < 1 || L > c.cfg.block_len || Kd < 0) return MRP_ERR_INVALID_ARG;
+    if (!state->tokens || !state->row_index || !state->n_masked || !state->block_masked) return MRP_ERR_INVALID_ARG;
+    if (!sel->out_token || (accept_mask && !sel->step_of)) return MRP_ERR_INVALID_ARG;
+    if (accept_mask && Kd > 0 && (!sel->draft_pos || !sel->draft_tok)) return MRP_ERR_INVALID_ARG;
+    c.launches = 0;
+    DeviceGuard guard(c.cfg.device);
+    if (guard.err != cudaSuccess) return MRP_ERR_CUDA;
+    c.err[0] = 0;
+    cudaError_t e = launch_commit(&c, *sel, accept_mask, B, L, Kd, *state, (cudaStream_t)cuda_stream);
+    return e == cudaSuccess ? MRP_OK : MRP_ERR_CUDA;
+}
+
 int mrp_selftest_wait_timeout(mrp_ctx *ctx, int32_t *status, void *cuda_stream)
 {
     if (!ctx) return MRP_ERR_INVALID_ARG;

@@ -143,6 +143,8 @@ cudaError_t launch_prep(Ctx *c, const void *hidden, const int32_t *row_index, in
                         cudaStream_t st, float *xt0);
 
 // ---- selection / verification (select_verify.cu) ------------------------------------
+cudaError_t launch_commit(Ctx *c, const mrp_select_out &sel, const int8_t *accept_mask, int B, int L, int Kd,
+                          const mrp_block_state &state, cudaStream_t st);
 cudaError_t launch_select(Ctx *c, const float *conf, const int32_t *token, const int32_t *row_index,
                           int M, int K, int B, int L, const mrp_select_params &p,
                           const mrp_select_out &out, cudaStream_t st);

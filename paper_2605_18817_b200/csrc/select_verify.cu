@@ -231,6 +231,106 @@ cudaError_t launch_verify(Ctx *c, const int32_t *draft_tok, const int32_t *verif
                     draft_tok, verify_tok, draft_len, B, Kd, positionwise, accept_len, accept_mask);
 }
 
+// ---- block-state transition x_t -> x_{t-1}: one warp per block -----------------------------
+__global__ void commit_kernel(int32_t *__restrict__ tokens, const int32_t *__restrict__ out_token,
+                              const int8_t *__restrict__ step_of, const int32_t *__restrict__ draft_pos,
+                              const int32_t *__restrict__ draft_tok, const int8_t *__restrict__ accept_mask,
+                              int L, int Kd, int32_t *__restrict__ block_masked)
+{
+    pdl_trigger();
+    pdl_wait();
+    const int b = blockIdx.x, lane = threadIdx.x;
+    int32_t *tk = tokens + (size_t)b * L;
+    for (int i = lane; i < L; i += 32) {
+        const size_t p = (size_t)b * L + i;
+        if (tk[i] >= 0) continue;
+        const int32_t t = out_token[p];
+        if (accept_mask ? (step_of[p] == 0) : (t >= 0)) tk[i] = t;
+    }
+    __syncwarp();
+    if (accept_mask) {
+        // accepted drafts (distinct positions of this block)
+        for (int s = lane; s < Kd; s += 32) {
+            const int pos = draft_pos[(size_t)b * Kd + s];
+            if (accept_mask[(size_t)b * Kd + s] && pos >= 0 && tk[pos] < 0) tk[pos] = draft_tok[(size_t)b * Kd + s];
+        }
+        __syncwarp();
+    }
+    int n = 0;
+    for (int i0 = 0; i0 < L; i0 += 32) {
+        const int i = i0 + lane;
+        n += __popc(__ballot_sync(0xffffffffu, i < L && tk[i] < 0));
+    }
+    if (lane == 0) block_masked[b] = n;
+}
+
+// Exclusive prefix sum of the per-block counts (one CTA; counts of 1024 blocks per round).
+__global__ void __launch_bounds__(1024) commit_scan_kernel(const int32_t *__restrict__ block_masked, int B,
+                                                           int32_t *__restrict__ block_off, int32_t *__restrict__ n_masked)
+{
+    pdl_trigger();
+    pdl_wait();
+    __shared__ int warp_tot[32];
+    __shared__ int carry_s;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0) carry_s = 0;
+    __syncthreads();
+    for (int b0 = 0; b0 < B; b0 += 1024) {
+        const int b = b0 + threadIdx.x;
+        const int v = b < B ? block_masked[b] : 0;
+        int inc = v;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int t = __shfl_up_sync(0xffffffffu, inc, o);
+            if (lane >= o) inc += t;
+        }
+        if (lane == 31) warp_tot[warp] = inc;
+        __syncthreads();
+        int before = carry_s;
+        for (int w = 0; w < warp; ++w) before += warp_tot[w];
+        if (b < B) block_off[b] = before + inc - v;
+        __syncthreads();
+        if (threadIdx.x == 1023) carry_s = before + inc;
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) *n_masked = carry_s;
+}
+
+// Every block lists its still-masked positions, in order, from its offset on.
+__global__ void commit_list_kernel(const int32_t *__restrict__ tokens, const int32_t *__restrict__ block_off, int L,
+                                   int32_t *__restrict__ row_index)
+{
+    pdl_trigger();
+    pdl_wait();
+    const int b = blockIdx.x, lane = threadIdx.x;
+    int off = block_off[b];
+    for (int i0 = 0; i0 < L; i0 += 32) {
+        const int i = i0 + lane;
+        const bool masked = i < L && tokens[(size_t)b * L + i] < 0;
+        const unsigned bal = __ballot_sync(0xffffffffu, masked);
+        if (masked) row_index[off + __popc(bal & ((1u << lane) - 1u))] = b * L + i;
+        off += __popc(bal);
+    }
+}
+
+cudaError_t launch_commit(Ctx *c, const mrp_select_out &sel, const int8_t *accept_mask, int B, int L, int Kd,
+                          const mrp_block_state &state, cudaStream_t st)
+{
+    const bool pdl = !(c->cfg.flags & MRP_FLAG_NO_PDL);
+    int32_t *block_off = (int32_t *)(c->ws + c->lay.dense_row);     // B <= max_seqs entries fit
+    cudaError_t e = launch_k(commit_kernel, dim3(B), dim3(32), 0, st, pdl, state.tokens, (const int32_t *)sel.out_token,
+                             (const int8_t *)sel.step_of, (const int32_t *)sel.draft_pos, (const int32_t *)sel.draft_tok,
+                             accept_mask, L, Kd, state.block_masked);
+    if (e == cudaSuccess)
+        e = launch_k(commit_scan_kernel, dim3(1), dim3(1024), 0, st, pdl, (const int32_t *)state.block_masked, B, block_off,
+                     state.n_masked);
+    if (e == cudaSuccess)
+        e = launch_k(commit_list_kernel, dim3(B), dim3(32), 0, st, pdl, (const int32_t *)state.tokens,
+                     (const int32_t *)block_off, L, state.row_index);
+    c->launches += 3;
+    return note_err(c, e, "commit kernels");
+}
+
 }  // namespace mrp
 
 // ---------------------------------------------------------------------------------------

@@ -64,6 +64,28 @@ def draft(ctx, hidden, logits0, row_index, M, K, out: DraftOut, stream=None):
     return out
 
 
+@dataclass
+class BlockState:
+    tokens: torch.Tensor        # [B*L] int32, -1 = masked
+    row_index: torch.Tensor     # [B*L] int32
+    n_masked: torch.Tensor      # [1] int32
+    block_masked: torch.Tensor  # [B] int32
+
+
+def alloc_block_state(B, L, device) -> BlockState:
+    i32 = dict(device=device, dtype=torch.int32)
+    return BlockState(torch.full((B * L,), -1, **i32), torch.arange(B * L, **i32),
+                      torch.full((1,), B * L, **i32), torch.full((B,), L, **i32))
+
+
+def commit(ctx, sel, state: BlockState, B, L, Kd, accept_mask=None, stream=None):
+    binding.mrp_commit(ctx, B, L, Kd, out_token=sel.out_token, step_of=sel.step_of, draft_pos=sel.draft_pos,
+                       draft_tok=sel.draft_tok, accept_mask=accept_mask, tokens=state.tokens,
+                       row_index=state.row_index, n_masked=state.n_masked, block_masked=state.block_masked,
+                       stream=stream)
+    return state
+
+
 def draft_from_hidden(ctx, hidden, final_gamma, row_index, M, K, out: DraftOut, stream=None):
     binding.mrp_draft_from_hidden(ctx, hidden, final_gamma, row_index, M, K, out.conf, out.lse, out.token,
                                   out.margin, out.logits, out.hidden, out.status, stream=stream)

@@ -57,6 +57,8 @@ def test_null_arguments_are_rejected_on_the_host():
     assert lib.mrp_create(None, None, None, None, 0, ctypes.byref(h)) == 1
     assert lib.mrp_draft(None, None, None, None, 1, 1, None, None) == 1
     assert lib.mrp_verify(None, None, None, None, 1, 1, 0, None, None, None) == 1
+    assert lib.mrp_draft_from_hidden(None, None, None, None, 1, 1, None, None) == 1
+    assert lib.mrp_commit(None, None, None, 1, 1, 0, None, None) == 1
     lib.mrp_destroy(None)
 
 

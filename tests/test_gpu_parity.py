@@ -376,3 +376,126 @@ def test_base_logits_from_hidden_states(dtype, flags, d, F, V, B, L, K):
     out, _ = run_gpu_draft(w, inp, K, flags=flags)
     ref = oracle.draft(inp.hidden, inp.logits0, w.heads, w.w_lm, K=K, row_index=inp.row_index)
     check_stats(out, ref, dtype)
+
+
+# ---- block-state transition (mrp_commit) ----
+
+def _state_to_device(tokens, B, L):
+    st = harness.alloc_block_state(B, L, DEV)
+    st.tokens.copy_(torch.from_numpy(tokens))
+    return st
+
+
+def _assert_state_equal(st, ref):
+    n = int(st.n_masked.item())
+    assert n == ref.row_index.size
+    assert np.array_equal(st.tokens.cpu().numpy(), ref.tokens)
+    assert np.array_equal(st.row_index.cpu().numpy()[:n], ref.row_index)
+    assert np.array_equal(st.block_masked.cpu().numpy(), ref.block_masked)
+
+
+@pytest.mark.parametrize("L", [1, 4, 31, 32, 33, 100, 1024])
+def test_commit_bit_exact_for_the_three_decoding_modes(select_ctx, L):
+    rng = np.random.default_rng(100 + L)
+    for case in range(8):
+        K = case % 4
+        B = 1 + (case * 7) % 23
+        tokens = np.where(rng.random(B * L) < 0.3 + 0.08 * case, -1, rng.integers(0, 999, B * L)).astype(np.int32)
+        ri = np.flatnonzero(tokens < 0).astype(np.int32)
+        if ri.size == 0:
+            continue
+        conf = rng.random((K + 1, ri.size)).astype(np.float32)
+        tok = rng.integers(0, 1000, (K + 1, ri.size)).astype(np.int32)
+        mode = binding.MRP_SELECT_STATIC if case % 3 else binding.MRP_SELECT_DYNAMIC_REMASK
+        kw = dict(tau=0.5) if mode == binding.MRP_SELECT_DYNAMIC_REMASK else dict(r_reveal=1 + case % 2, r_draft=1)
+        sel = _gpu_select(select_ctx, conf, tok, ri, B, L, mode, **kw)
+        osel = oracle.select(conf, tok, ri, B, L, oracle.STATIC if mode == binding.MRP_SELECT_STATIC else oracle.DYNAMIC_REMASK, **kw)
+        _assert_select_equal(sel, osel)
+        # direct decoding / remasking: everything selected is unmasked
+        st = _state_to_device(tokens, B, L)
+        harness.commit(select_ctx, sel, st, B, L, K)
+        torch.cuda.synchronize()
+        _assert_state_equal(st, oracle.commit(tokens, osel, B, L))
+        # speculative decoding: drafts only where the backbone agreed
+        if mode == binding.MRP_SELECT_STATIC and K > 0:
+            vt = np.where(rng.random((B, K)) < 0.6, osel.draft_tok, -5).astype(np.int32)
+            alen = torch.empty(B, device=DEV, dtype=torch.int32)
+            amask = torch.empty((B, K), device=DEV, dtype=torch.int8)
+            binding.mrp_verify(select_ctx, sel.draft_tok, torch.from_numpy(vt).to(DEV), sel.draft_len, B, K,
+                               bool(case & 4), alen, amask)
+            _, oacc = oracle.verify(osel.draft_tok, vt, osel.draft_len, positionwise=bool(case & 4))
+            st = _state_to_device(tokens, B, L)
+            harness.commit(select_ctx, sel, st, B, L, K, accept_mask=amask)
+            torch.cuda.synchronize()
+            _assert_state_equal(st, oracle.commit(tokens, osel, B, L, accept_mask=oacc))
+
+
+@pytest.mark.parametrize("mode", ["direct", "speculative", "remask"])
+def test_denoising_loop_with_the_block_state_on_the_device(select_ctx, mode):
+    """Algorithms 2-4 as a loop: the statistics of every forward are synthetic (one random table
+    per forward, gathered at the masked positions), selection, verification and the state
+    transition run on the device; the oracle runs the same loop.  States must agree after
+    every forward, and both must finish together."""
+    rng = np.random.default_rng({"direct": 1, "speculative": 2, "remask": 3}[mode])
+    B, L, K = 9, 32, 2 if mode != "remask" else 1
+    tokens = np.full(B * L, -1, np.int32)
+    st = _state_to_device(tokens, B, L)
+    n_forwards = 0
+    while (tokens < 0).any():
+        conf_full = rng.random((K + 1, B * L)).astype(np.float32)
+        tok_full = rng.integers(0, 1000, (K + 1, B * L)).astype(np.int32)
+        n = int(st.n_masked.item())
+        ri_dev = st.row_index[:n].clone()              # the device's own list of masked positions
+        ri = np.flatnonzero(tokens < 0).astype(np.int32)
+        assert np.array_equal(ri_dev.cpu().numpy(), ri)
+        conf, tok = conf_full[:, ri], tok_full[:, ri]
+        sel = harness.alloc_select_out(B, L, K, DEV)
+        c, t = torch.from_numpy(np.ascontiguousarray(conf)).to(DEV), torch.from_numpy(np.ascontiguousarray(tok)).to(DEV)
+        if mode == "remask":
+            harness.select(select_ctx, c, t, ri_dev, n, K, B, L, binding.MRP_SELECT_DYNAMIC_REMASK, sel, tau=0.6)
+            osel = oracle.select(conf, tok, ri, B, L, oracle.DYNAMIC_REMASK, tau=0.6)
+            harness.commit(select_ctx, sel, st, B, L, K)
+            ref = oracle.commit(tokens, osel, B, L)
+        else:
+            harness.select(select_ctx, c, t, ri_dev, n, K, B, L, binding.MRP_SELECT_STATIC, sel)
+            osel = oracle.select(conf, tok, ri, B, L, oracle.STATIC)
+            if mode == "direct":
+                harness.commit(select_ctx, sel, st, B, L, K)
+                ref = oracle.commit(tokens, osel, B, L)
+            else:
+                vt = np.where(rng.random((B, K)) < 0.7, osel.draft_tok, -5).astype(np.int32)
+                alen = torch.empty(B, device=DEV, dtype=torch.int32)
+                amask = torch.empty((B, K), device=DEV, dtype=torch.int8)
+                binding.mrp_verify(select_ctx, sel.draft_tok, torch.from_numpy(vt).to(DEV), sel.draft_len, B, K,
+                                   False, alen, amask)
+                harness.commit(select_ctx, sel, st, B, L, K, accept_mask=amask)
+                _, oacc = oracle.verify(osel.draft_tok, vt, osel.draft_len)
+                ref = oracle.commit(tokens, osel, B, L, accept_mask=oacc)
+        torch.cuda.synchronize()
+        _assert_state_equal(st, ref)
+        assert ref.row_index.size < ri.size                  # every forward makes progress
+        tokens = ref.tokens
+        n_forwards += 1
+        assert n_forwards <= L
+    if mode == "direct":
+        assert n_forwards == -(-L // (K + 1))
+    assert int(st.n_masked.item()) == 0 and int(st.block_masked.sum().item()) == 0
+
+
+def test_commit_with_more_blocks_than_one_round_of_the_prefix_sum():
+    w = synth.make_weights(16, 16, 32, 0, "f32", 1)
+    heads, w_lm = harness.upload_weights(w, DEV)
+    B, L, K = 2500, 3, 1
+    ctx = binding.mrp_create(16, 16, 32, heads, w_lm, max_rows=4, max_seqs=B, block_len=L)
+    rng = np.random.default_rng(77)
+    tokens = np.where(rng.random(B * L) < 0.7, -1, rng.integers(0, 999, B * L)).astype(np.int32)
+    ri = np.flatnonzero(tokens < 0).astype(np.int32)
+    conf = rng.random((K + 1, ri.size)).astype(np.float32)
+    tok = rng.integers(0, 1000, (K + 1, ri.size)).astype(np.int32)
+    sel = _gpu_select(ctx, conf, tok, ri, B, L, binding.MRP_SELECT_STATIC)
+    osel = oracle.select(conf, tok, ri, B, L, oracle.STATIC)
+    st = _state_to_device(tokens, B, L)
+    harness.commit(ctx, sel, st, B, L, K)
+    torch.cuda.synchronize()
+    _assert_state_equal(st, oracle.commit(tokens, osel, B, L))
+    binding.mrp_destroy(ctx)
