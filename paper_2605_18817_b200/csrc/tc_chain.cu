@@ -316,6 +316,34 @@ sk_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant__ 
                 ch_epi_sync();                      // also publishes rstd_s
                 if (*vote_s == 1) { alive = false; break; }
                 tc_fence_after();
+                if (ph.kind == CH_GU && ph.n_split == 1) {
+                    // The tile is this CTA's alone: no slices to add, so the outputs are finished straight
+                    // from the accumulator.  Gate row c and up row c of an output sit in lanes c and c + 64:
+                    // they meet through shared memory, 16 batch rows at a time.
+                    float *exch = sq_s;                              // [16][128]
+#pragma unroll 1
+                    for (int ch = 0; ch < n_ch; ++ch) {
+                        float v[16], w[16];
+                        tmem_ld16(lane_addr + ch * 16, v);
+                        tmem_ld16(lane_addr + RP + ch * 16, w);
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) exch[j * 128 + t] = v[j] + w[j];
+                        ch_epi_sync();
+                        const int c = t & 63, f = tile * 64 + c;
+#pragma unroll
+                        for (int q = 0; q < 8; ++q) {
+                            const int j = (t >> 6) * 8 + q, m = ch * 16 + j;
+                            if (m < p.M && f < ph.w_rows) {
+                                const float g = exch[j * 128 + c] * rstd_s[m], u = exch[j * 128 + 64 + c] * rstd_s[m];
+                                ch_store_hi_lo(p.act + (size_t)m * p.F + f, (size_t)p.lo_x * p.F, g / (1.f + __expf(-g)) * u);
+                            }
+                        }
+                        ch_epi_sync();
+                    }
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(tempty_bar(acc));     // the accumulator buffer is free again
+                } else {
                 // (1) park this slice: scratch[cta][column][lane]
                 float *mine = p.scratch + ((size_t)cta * RP) * 128;
 #pragma unroll 1
@@ -408,6 +436,7 @@ sk_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant__ 
                                   (unsigned long long)__double2ll_rn((double)s * 16777216.0));
                     }
                 }
+                }   // slices parked and added
             }
             // this CTA's part of the phase is in memory: arrive at the grid barrier
             __threadfence();

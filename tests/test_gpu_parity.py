@@ -264,6 +264,10 @@ def test_config0_static_selection_end_to_end():
     (64, 12288, 2304, 5, 1, 2),     # gate/up: full 128-row weight tiles plus short tiles
     (19008, 64, 512, 3, 1, 1),      # down projection: full weight tiles plus short tiles
     (1024, 2048, 2048, 20, 1, 2),   # head chain with 32-row operands and two k-chunks per ring stage
+    (512, 1024, 2048, 100, 1, 2),   # head chain with 128-row operands
+    (128, 192, 2048, 90, 1, 2),     # the same with an odd number of gate/up weight tiles
+    (64, 6144, 1024, 100, 1, 1),    # head chain, gate/up tiles not split: outputs finished straight from TMEM
+    (64, 6144, 1024, 5, 1, 2),      # the same with few rows
 ])
 def test_tensor_core_family_small_shapes(d, F, V, B, L, K):
     # residuals of order one at every shape (the very long contraction gets smaller weights)
