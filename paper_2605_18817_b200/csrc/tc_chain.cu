@@ -80,6 +80,15 @@ __device__ __forceinline__ void ch_store_hi_lo(__nv_bfloat16 *dst, size_t lo_off
     dst[0] = hi;
     dst[lo_off] = __float2bfloat16_rn(v - __bfloat162float(hi));
 }
+// four consecutive values as bf16 hi + lo pairs, one 8-byte store each
+__device__ __forceinline__ void ch_store_split4(__nv_bfloat16 *dst, size_t lo_off, const float *v)
+{
+    uint32_t hi[2], lo[2];
+    split_bf16(v[0], v[1], hi[0], lo[0]);
+    split_bf16(v[2], v[3], hi[1], lo[1]);
+    *reinterpret_cast<uint2 *>(dst) = make_uint2(hi[0], hi[1]);
+    *reinterpret_cast<uint2 *>(dst + lo_off) = make_uint2(lo[0], lo[1]);
+}
 __device__ __forceinline__ unsigned int ld_acquire_u32(const unsigned int *p)
 {
     unsigned int v;
@@ -400,6 +409,58 @@ sk_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant__ 
                         }
                     }
                 } else {
+                    int n_sq = n_r;                      // entries of the buffer of squares per batch row
+                    bool done = false;
+                    if constexpr (RP >= 64) {
+                        // Many batch rows: a share is thousands of outputs, so four consecutive output
+                        // rows are handled per item with 16-byte loads and 8-byte stores.
+                        if ((per & 3) == 0 && (ph.w_rows & 3) == 0 && n_r > 0) {
+                            const int n_g = n_r >> 2;
+                            n_sq = n_g;
+                            done = true;
+#pragma unroll 2
+                            for (int e = t; e < n_g * p.M; e += 128) {
+                                const int m = e / n_g, row = r0 + ((e - m * n_g) << 2);
+                                const int j = tile * 128 + row;
+                                float sq = 0.f;
+                                if (j < ph.w_rows) {
+                                    const size_t o = (size_t)m * p.d + j;
+                                    const float4 hc = __ldcg(reinterpret_cast<const float4 *>(p.hcur + o));
+                                    const float4 h0 = __ldg(reinterpret_cast<const float4 *>(p.h0f + o));
+                                    float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+                                    for (int s0 = 0; s0 < ph.n_split; s0 += 8) {  // slice order; 8 slices' loads in flight
+                                        float4 as[8];
+#pragma unroll
+                                        for (int k = 0; k < 8; ++k)
+                                            as[k] = (s0 + k < ph.n_split)
+                                                        ? __ldcg(reinterpret_cast<const float4 *>(first + ((size_t)(s0 + k) * RP + m) * 128 + row))
+                                                        : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                                        for (int k = 0; k < 8; ++k) { a.x += as[k].x; a.y += as[k].y; a.z += as[k].z; a.w += as[k].w; }
+                                    }
+                                    const float h[4] = {hc.x + a.x, hc.y + a.y, hc.z + a.z, hc.w + a.w};
+                                    const float hz[4] = {h0.x, h0.y, h0.z, h0.w};
+                                    *reinterpret_cast<float4 *>(p.hcur + o) = make_float4(h[0], h[1], h[2], h[3]);
+                                    if (ph.hidden_out) *reinterpret_cast<float4 *>(ph.hidden_out + o) = make_float4(h[0], h[1], h[2], h[3]);
+                                    sq = (h[0] * h[0] + h[1] * h[1]) + (h[2] * h[2] + h[3] * h[3]);
+                                    float r[4], xn[4];
+#pragma unroll
+                                    for (int k = 0; k < 4; ++k) {
+                                        r[k] = h[k] - hz[k];
+                                        xn[k] = ph.xg_next ? h[k] * __bfloat162float(ph.gamma_next[j + k]) : 0.f;
+                                    }
+                                    ch_store_split4(ph.xt_k + o, (size_t)p.lo_xt * p.d, r);
+                                    if (ph.xt16_k) {
+                                        __half2 hh[2] = {__floats2half2_rn(r[0], r[1]), __floats2half2_rn(r[2], r[3])};
+                                        *reinterpret_cast<uint2 *>(ph.xt16_k + o) = *reinterpret_cast<uint2 *>(hh);
+                                    }
+                                    if (ph.xg_next) ch_store_split4(ph.xg_next + o, (size_t)p.lo_x * p.d, xn);
+                                }
+                                sq_s[e] = sq;
+                            }
+                        }
+                    }
+                    if (!done) {
 #pragma unroll 2
                     for (int e = t; e < n_items; e += 128) {
                         const int m = e / n_r, row = r0 + (e - m * n_r);
@@ -427,11 +488,12 @@ sk_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant__ 
                         }
                         sq_s[e] = sq;
                     }
+                    }
                     ch_epi_sync();
                     // this CTA's rows, in row order, then one integer add per row of the batch
                     for (int m = t; m < p.M; m += 128) {
                         float s = 0.f;
-                        for (int r = 0; r < n_r; ++r) s += sq_s[m * n_r + r];
+                        for (int r = 0; r < n_sq; ++r) s += sq_s[m * n_sq + r];
                         atomicAdd(p.ssq_fix + ph.ssq_idx * 128 + m,
                                   (unsigned long long)__double2ll_rn((double)s * 16777216.0));
                     }
