@@ -338,14 +338,22 @@ sk_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant__ 
 #pragma unroll
                         for (int j = 0; j < 16; ++j) exch[j * 128 + t] = v[j] + w[j];
                         ch_epi_sync();
-                        const int c = t & 63, f = tile * 64 + c;
+                        // thread = (batch row j of the 16, 8 consecutive outputs): two 16-byte stores
+                        const int j = t >> 3, c0 = (t & 7) * 8, m = ch * 16 + j, f0 = tile * 64 + c0;
+                        if (m < p.M && f0 < ph.w_rows) {
+                            const float4 *gp = reinterpret_cast<const float4 *>(exch + j * 128 + c0);
+                            const float4 *up = reinterpret_cast<const float4 *>(exch + j * 128 + 64 + c0);
+                            const float4 g0 = gp[0], g1 = gp[1], u0 = up[0], u1 = up[1];
+                            const float gg[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
+                            const float uu[8] = {u0.x, u0.y, u0.z, u0.w, u1.x, u1.y, u1.z, u1.w};
+                            const float rs = rstd_s[m];
+                            float av[8];
 #pragma unroll
-                        for (int q = 0; q < 8; ++q) {
-                            const int j = (t >> 6) * 8 + q, m = ch * 16 + j;
-                            if (m < p.M && f < ph.w_rows) {
-                                const float g = exch[j * 128 + c] * rstd_s[m], u = exch[j * 128 + 64 + c] * rstd_s[m];
-                                ch_store_hi_lo(p.act + (size_t)m * p.F + f, (size_t)p.lo_x * p.F, g / (1.f + __expf(-g)) * u);
+                            for (int q = 0; q < 8; ++q) {
+                                const float g = gg[q] * rs;
+                                av[q] = g / (1.f + __expf(-g)) * (uu[q] * rs);
                             }
+                            store_split<8>(p.act + (size_t)m * p.F + f0, (size_t)p.lo_x * p.F, av);
                         }
                         ch_epi_sync();
                     }
