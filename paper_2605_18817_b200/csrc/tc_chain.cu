@@ -394,6 +394,45 @@ sk_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant__ 
                 const int n_items = n_r * p.M;
                 const float *first = p.scratch + ((size_t)tile * ph.n_split * RP) * 128;
                 if (ph.kind == CH_GU) {
+                    bool done = false;
+                    if constexpr (RP >= 32) {
+                        // many batch rows: four consecutive outputs per item, 16-byte loads, 8-byte stores
+                        if ((per & 3) == 0 && (ph.w_rows & 3) == 0 && n_r > 0) {
+                            const int n_g = n_r >> 2;
+                            done = true;
+#pragma unroll 2
+                            for (int e = t; e < n_g * p.M; e += 128) {
+                                const int m = e / n_g, row = r0 + ((e - m * n_g) << 2);
+                                const int f = tile * 64 + row;
+                                if (f < ph.w_rows) {
+                                    float4 g = make_float4(0.f, 0.f, 0.f, 0.f), u = g;
+                                    for (int s0 = 0; s0 < ph.n_split; s0 += 4) {  // slice order; 4 slices' loads in flight
+                                        float4 gs[4], us[4];
+#pragma unroll
+                                        for (int k = 0; k < 4; ++k) {
+                                            const float *src = first + ((size_t)(s0 + k) * RP + m) * 128 + row;
+                                            const bool in = s0 + k < ph.n_split;
+                                            gs[k] = in ? __ldcg(reinterpret_cast<const float4 *>(src)) : make_float4(0.f, 0.f, 0.f, 0.f);
+                                            us[k] = in ? __ldcg(reinterpret_cast<const float4 *>(src + 64)) : make_float4(0.f, 0.f, 0.f, 0.f);
+                                        }
+#pragma unroll
+                                        for (int k = 0; k < 4; ++k) {
+                                            g.x += gs[k].x; g.y += gs[k].y; g.z += gs[k].z; g.w += gs[k].w;
+                                            u.x += us[k].x; u.y += us[k].y; u.z += us[k].z; u.w += us[k].w;
+                                        }
+                                    }
+                                    const float rs = rstd_s[m];
+                                    const float gg[4] = {g.x * rs, g.y * rs, g.z * rs, g.w * rs};
+                                    const float uu[4] = {u.x * rs, u.y * rs, u.z * rs, u.w * rs};
+                                    float av[4];
+#pragma unroll
+                                    for (int k = 0; k < 4; ++k) av[k] = gg[k] / (1.f + __expf(-gg[k])) * uu[k];
+                                    ch_store_split4(p.act + (size_t)m * p.F + f, (size_t)p.lo_x * p.F, av);
+                                }
+                            }
+                        }
+                    }
+                    if (!done) {
 #pragma unroll 2
                     for (int e = t; e < n_items; e += 128) {
                         const int m = e / n_r, row = r0 + (e - m * n_r);
@@ -416,10 +455,11 @@ sk_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant__ 
                             ch_store_hi_lo(p.act + (size_t)m * p.F + f, (size_t)p.lo_x * p.F, g / (1.f + __expf(-g)) * u);
                         }
                     }
+                    }
                 } else {
                     int n_sq = n_r;                      // entries of the buffer of squares per batch row
                     bool done = false;
-                    if constexpr (RP >= 64) {
+                    if constexpr (RP >= 32) {
                         // Many batch rows: a share is thousands of outputs, so four consecutive output
                         // rows are handled per item with 16-byte loads and 8-byte stores.
                         if ((per & 3) == 0 && (ph.w_rows & 3) == 0 && n_r > 0) {
