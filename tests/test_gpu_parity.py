@@ -503,3 +503,36 @@ def test_commit_with_more_blocks_than_one_round_of_the_prefix_sum():
     torch.cuda.synchronize()
     _assert_state_equal(st, oracle.commit(tokens, osel, B, L))
     binding.mrp_destroy(ctx)
+
+
+@pytest.mark.parametrize("d,F,V,B,L,K", [
+    (2048, 4096, 4096, 1, 4, 3),      # head chain with grid barriers, few-row LM head
+    (512, 1024, 2048, 100, 1, 2),     # 128-row chain: parked slices, tile barriers, row-major LM head
+    (256, 512, 4096, 75, 4, 2),       # row-major kernels throughout
+])
+def test_repeated_calls_give_bit_identical_outputs(d, F, V, B, L, K):
+    """Sums over CTAs are taken in a fixed order (slice order, fixed-point integer adds for the row
+    sums of squares, fixed merge order of the softmax partials): 200 calls, no bit may move."""
+    w = synth.make_weights(d, F, V, K, "bf16", 91, head_std=0.05 if d <= 512 else 0.02)
+    inp = synth.make_inputs(w, B, L, 91, 1.0, 4.0)
+    heads, w_lm = harness.upload_weights(w, DEV)
+    ctx = binding.mrp_create(w.d, w.F, w.V, heads, w_lm, max_rows=B * L, max_seqs=B, block_len=L)
+    M = B * L
+    hid = harness.to_device(inp.hidden, w.dtype, DEV)
+    l0 = torch.from_numpy(inp.logits0).to(DEV)
+    out = harness.alloc_draft_out(M, K, w.V, w.d, DEV, margin=True, hidden=True)
+    for from_hidden in (False, True):
+        ref = None
+        for i in range(200):
+            if from_hidden:
+                harness.draft_from_hidden(ctx, hid, None, None, M, K, out)
+            else:
+                harness.draft(ctx, hid, l0, None, M, K, out)
+            if i % 40 == 0 or i == 199:
+                torch.cuda.synchronize()
+                cur = [t.clone() for t in (out.conf, out.lse, out.token, out.margin, out.hidden)]
+                if ref is None:
+                    ref = cur
+                assert all(torch.equal(a, b) for a, b in zip(cur, ref)), i
+        assert int(out.status.item()) == 0
+    binding.mrp_destroy(ctx)
