@@ -307,6 +307,18 @@ int mrp_reveal_remask_noalloc(const float *conf, const int32_t *token, const int
  */
 int mrp_selftest_wait_timeout(mrp_ctx *ctx, int32_t *status, void *cuda_stream);
 
+/*
+ * Let mrp_draft wait for the base logits separately from the hidden states.  In Algorithm 2
+ * ("h, l <- f(x_t)") the logits are the last thing the backbone forward produces, and the head
+ * chain needs only h: an engine can run its own LM head (or, with host buffers, the copy of
+ * logits0) on another stream while the head chain runs.  After this call every mrp_draft on
+ * the context enqueues a wait for cuda_event (a cudaEvent_t the caller records, before calling
+ * mrp_draft, on the stream that produces logits0) immediately before the LM-head kernel, and
+ * reads logits0 nowhere earlier.  NULL restores the default (logits0 ready when mrp_draft is
+ * called).  mrp_draft_from_hidden ignores the event.  Errors: INVALID_ARG.
+ */
+int mrp_set_logits0_event(mrp_ctx *ctx, void *cuda_event);
+
 /* Number of kernels the last mrp_draft / mrp_reveal_remask / mrp_verify call on this
  * context launched (for accounting in benchmarks). */
 int32_t mrp_last_launch_count(const mrp_ctx *ctx);

@@ -30,7 +30,8 @@ MRP_DEV_NONFINITE, MRP_DEV_TIMEOUT = 1, 2
 EXPORTS = ("mrp_workspace_bytes", "mrp_create", "mrp_destroy", "mrp_draft", "mrp_reveal_remask",
            "mrp_verify", "mrp_last_launch_count", "mrp_kernel_family", "mrp_status_string",
            "mrp_profile_enable", "mrp_profile_read", "mrp_last_error",
-           "mrp_reveal_remask_noalloc", "mrp_selftest_wait_timeout", "mrp_draft_from_hidden", "mrp_commit")
+           "mrp_reveal_remask_noalloc", "mrp_selftest_wait_timeout", "mrp_draft_from_hidden", "mrp_commit",
+           "mrp_set_logits0_event")
 MRP_NOALLOC_MAX_POSITIONS = 65536
 MRP_ERR_CAPACITY = 7
 
@@ -92,6 +93,8 @@ def _load():
     lib.mrp_draft.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
                               ctypes.c_int32, ctypes.c_int32, ctypes.POINTER(mrp_draft_out),
                               ctypes.c_void_p]
+    lib.mrp_set_logits0_event.restype = ctypes.c_int
+    lib.mrp_set_logits0_event.argtypes = [ctypes.c_void_p, ctypes.c_void_p]
     lib.mrp_commit.restype = ctypes.c_int
     lib.mrp_commit.argtypes = [ctypes.c_void_p, ctypes.POINTER(mrp_select_out), ctypes.c_void_p, ctypes.c_int32,
                                ctypes.c_int32, ctypes.c_int32, ctypes.POINTER(mrp_block_state), ctypes.c_void_p]
@@ -324,6 +327,14 @@ def mrp_selftest_wait_timeout(ctx: Context, status, stream=None) -> None:
     rc = lib.mrp_selftest_wait_timeout(ctx.handle, _ptr(status), _stream(stream))
     if rc != 0:
         raise MrpError("mrp_selftest_wait_timeout", rc)
+
+
+def mrp_set_logits0_event(ctx: Context, event) -> None:
+    """``event``: a recorded ``torch.cuda.Event`` (or None): mrp_draft waits for it right before the LM head."""
+    h = None if event is None else ctypes.c_void_p(event.cuda_event)
+    rc = lib.mrp_set_logits0_event(ctx.handle, h)
+    if rc != 0:
+        raise MrpError("mrp_set_logits0_event", rc)
 
 
 def mrp_commit(ctx: Context, B, L, Kd, *, out_token, step_of, draft_pos, draft_tok, accept_mask=None,

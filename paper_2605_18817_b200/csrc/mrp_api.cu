@@ -280,6 +280,13 @@ int mrp_verify(mrp_ctx *ctx, const int32_t *draft_tok, const int32_t *verify_tok
     return e == cudaSuccess ? MRP_OK : MRP_ERR_CUDA;
 }
 
+int mrp_set_logits0_event(mrp_ctx *ctx, void *cuda_event)
+{
+    if (!ctx) return MRP_ERR_INVALID_ARG;
+    ctx->c.l0_event = (cudaEvent_t)cuda_event;
+    return MRP_OK;
+}
+
 int mrp_commit(mrp_ctx *ctx, const mrp_select_out *sel, const int8_t *accept_mask, int32_t B, int32_t L,
                int32_t Kd, const mrp_block_state *state, void *cuda_stream)
 {

@@ -62,6 +62,7 @@ struct Ctx {
     // LM-head pass computes them as W_lm n_0, n_0 = h_0 or RMSNorm(h_0) * final_gamma.
     bool from_hidden;
     const void *final_gamma;
+    cudaEvent_t l0_event;      // mrp_set_logits0_event: awaited right before the LM-head kernel, or nullptr
     // Row offset of the bf16 lo block behind the hi block in this call's operand buffers: M and
     // (K+1)M for the row-major kernels, the padded row count for the few-row kernels (which then
     // fetch hi and lo rows of a k-chunk with one TMA box).
@@ -85,6 +86,13 @@ inline cudaError_t note_err(Ctx *c, cudaError_t e, const char *where)
 
 constexpr int kProfSlots = 1024;
 constexpr int kProfMarks = 4;   // start, after head chain, after LM head, after combine
+
+// The base logits may become ready later than the hidden states (mrp_set_logits0_event).
+inline cudaError_t wait_logits0(Ctx *c, cudaStream_t st)
+{
+    if (!c->l0_event || c->from_hidden) return cudaSuccess;
+    return cudaStreamWaitEvent(st, c->l0_event, 0);
+}
 
 inline void prof_mark(Ctx *c, int mark, cudaStream_t st)
 {

@@ -396,6 +396,8 @@ static cudaError_t simt_draft_t(Ctx *c, const void *hidden, const float *logits0
         c->launches += 3;
     }
     prof_mark(c, 1, st);
+    e = note_err(c, wait_logits0(c, st), "wait for the base logits");
+    if (e != cudaSuccess) return e;
     // small vocabularies: narrower slices so that every SM gets a block
     const bool narrow = (V + kSimtSliceV - 1) / kSimtSliceV < 2 * c->sm_count;
     const int slice_v = narrow ? 32 : kSimtSliceV;

@@ -671,6 +671,8 @@ cudaError_t tc_draft(Ctx *c, const void *hidden, const float *logits0, const int
         n_ss = p.n_vr;
     }
     prof_mark(c, 1, st);
+    e = note_err(c, wait_logits0(c, st), "wait for the base logits");
+    if (e != cudaSuccess) return e;
     int n_slices = G;
     if (lm_few) {
         e = sk_lm(c, logits0, row_index, M, K, out, st, pdl);

@@ -59,6 +59,7 @@ def test_null_arguments_are_rejected_on_the_host():
     assert lib.mrp_verify(None, None, None, None, 1, 1, 0, None, None, None) == 1
     assert lib.mrp_draft_from_hidden(None, None, None, None, 1, 1, None, None) == 1
     assert lib.mrp_commit(None, None, None, 1, 1, 0, None, None) == 1
+    assert lib.mrp_set_logits0_event(None, None) == 1
     lib.mrp_destroy(None)
 
 

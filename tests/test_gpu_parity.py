@@ -536,3 +536,33 @@ def test_repeated_calls_give_bit_identical_outputs(d, F, V, B, L, K):
                 assert all(torch.equal(a, b) for a, b in zip(cur, ref)), i
         assert int(out.status.item()) == 0
     binding.mrp_destroy(ctx)
+
+
+def test_draft_waits_for_the_base_logits_event_before_the_lm_head():
+    """mrp_set_logits0_event: the base logits arrive late on another stream (after a sleep kernel);
+    the call enqueued meanwhile must give the results of a call that had them from the start."""
+    w = synth.make_weights(256, 512, 4096, 2, "bf16", 17, head_std=0.05)
+    inp = synth.make_inputs(w, 2, 4, 17, 1.0, 4.0)
+    heads, w_lm = harness.upload_weights(w, DEV)
+    M, K = 8, 2
+    hid = harness.to_device(inp.hidden, w.dtype, DEV)
+    l0_host = torch.from_numpy(inp.logits0).pin_memory()
+    for flags in (0, binding.MRP_FLAG_FORCE_SIMT, binding.MRP_FLAG_ROW_MAJOR_ONLY):
+        ctx = binding.mrp_create(w.d, w.F, w.V, heads, w_lm, max_rows=M, max_seqs=2, block_len=4, flags=flags)
+        ref = harness.alloc_draft_out(M, K, w.V, w.d, DEV)
+        harness.draft(ctx, hid, l0_host.to(DEV), None, M, K, ref)
+        torch.cuda.synchronize()
+        l0 = torch.full((M, w.V), 1e30, device=DEV)          # poison until the late copy lands
+        side, ready = torch.cuda.Stream(), torch.cuda.Event()
+        with torch.cuda.stream(side):
+            torch.cuda._sleep(40_000_000)                     # some 20 ms
+            l0.copy_(l0_host, non_blocking=True)
+            ready.record(side)
+        binding.mrp_set_logits0_event(ctx, ready)
+        out = harness.alloc_draft_out(M, K, w.V, w.d, DEV)
+        harness.draft(ctx, hid, l0, None, M, K, out)
+        torch.cuda.synchronize()
+        assert torch.equal(out.conf, ref.conf) and torch.equal(out.token, ref.token) and torch.equal(out.lse, ref.lse)
+        assert int(out.status.item()) == 0
+        binding.mrp_set_logits0_event(ctx, None)
+        binding.mrp_destroy(ctx)
