@@ -252,7 +252,7 @@ __global__ void commit_kernel(int32_t *__restrict__ tokens, const int32_t *__res
         // accepted drafts (distinct positions of this block)
         for (int s = lane; s < Kd; s += 32) {
             const int pos = draft_pos[(size_t)b * Kd + s];
-            if (accept_mask[(size_t)b * Kd + s] && pos >= 0 && tk[pos] < 0) tk[pos] = draft_tok[(size_t)b * Kd + s];
+            if (accept_mask[(size_t)b * Kd + s] && pos >= 0 && pos < L && tk[pos] < 0) tk[pos] = draft_tok[(size_t)b * Kd + s];
         }
         __syncwarp();
     }
