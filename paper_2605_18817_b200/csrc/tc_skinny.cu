@@ -395,9 +395,12 @@ sk_gemm_kernel(const __grid_constant__ SkMaps maps, const SkParams p)
                     for (int j = 0; j < 16; ++j)
                         if (ch * 16 + j < p.M) mine[(ch * 16 + j) * 128 + t] = v[j] + w[j];
                 }
-                __threadfence();
+                // one thread's fence after the barrier publishes every thread's stores (fences are cumulative)
                 epi_sync();
-                if (t == 0) *vote_s = (atomicAdd(p.counters + tile, 1) == p.n_split - 1) ? 2 : 0;
+                if (t == 0) {
+                    __threadfence();
+                    *vote_s = (atomicAdd(p.counters + tile, 1) == p.n_split - 1) ? 2 : 0;
+                }
                 epi_sync();
                 finisher = (*vote_s == 2);
                 if (finisher) {
