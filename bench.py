@@ -30,7 +30,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the fused LM-head kernel,
 # from the ncu captures summarised under profiles/ (bytes per launch; None = not captured).
-NCU_TRAFFIC_BYTES = {"decode_1p7b": 628789760}   # profiles/sk_gemm_kernel_decode_1p7b.md
+NCU_TRAFFIC_BYTES = {"decode_1p7b": 628542208}   # profiles/sk_gemm_kernel_decode_1p7b.md
 
 
 def parse_args():
