@@ -629,12 +629,11 @@ cudaError_t sk_chain(Ctx *c, int M, int K, const mrp_draft_out &out, cudaStream_
     const TcState *s = (const TcState *)c->tc_state;
     const int d = c->cfg.d, F = c->cfg.d_ff, G = c->sm_count;
     if (K < 1 || K > 4 || 2 * K > kChMaxPhases || M < 1 || M > 128) return cudaErrorNotSupported;
-    // Up to 32 rows: worth it while a GEMM of the chain is latency-bound (a few tens of MB of
-    // weights): measured 67 vs 77 us at d = 2048, F = 4096 (M = 4, K = 3); at d = 4096, F = 8192 the
-    // two forms tie (173 vs 172 us at M = 4, K = 4; 59 vs 54 us at M = 16, K = 1), so the separate
-    // kernels stay there.  From 33 rows on this kernel wins at every size (M = 64, d = 4096:
-    // 69 vs 84 us for one head, 231-275 vs 286 us for four): its finish is spread over all CTAs.
-    if (M <= 32 && (long long)d * F > (12ll << 20)) return cudaErrorNotSupported;
+    // Measured against one kernel per GEMM (programmatic dependent launch between them), whole
+    // mrp_draft call: d = 2048, F = 4096, M = 4, K = 3: 60 vs 77 us for the heads; d = 4096,
+    // F = 8192: M = 1, K = 1 0.244 vs 0.247 ms, M = 4, K = 4 0.371 vs 0.378 ms, M = 16, K = 4
+    // 0.398 vs 0.412 ms, M = 64, K = 1 69 vs 84 us for the head (M = 16, K = 1 is the one point
+    // where the separate kernels are ahead, by 2 us).  So every shape that fits runs here.
     const int r_pad = sk_head_pad(M);
     const int gu_tiles = F / 64, dn_tiles = (d + 127) / 128;
     if (gu_tiles > G || dn_tiles > G || G > kSumsqSlices || gu_tiles > kChTilesPerPhase ||
