@@ -8,8 +8,14 @@
 // axis, bf16 hi + lo activation rows stacked on N, one 128-row weight tile and one slice of the
 // contraction per CTA and phase).  A phase needs the previous phase's activations, so the
 // CTAs meet at a grid barrier between phases -- but the weights depend on nothing: the producer
-// fills the ring with the next phase's weight tiles before it waits, and only the activation
-// tiles are fetched after the barrier.
+// fills the ring with the next phase's weight tiles before it waits
+// (three stages at once, the rest of the ring once the CTA has parked its own slice), and only
+// the activation tiles are fetched after the barrier.
+// A weight tile that is split over several CTAs is finished in three steps: every CTA parks its
+// slice of the accumulator in scratch, the CTAs of the tile meet at a counter, and each finishes
+// its share of the tile's output rows from the parked slices, added in slice order (so every SM
+// takes part in the element-wise work, and the result does not depend on arrival order).  A
+// gate/up tile that one CTA owns alone is finished straight from the accumulator.
 // Every wait is bounded: a barrier or mbarrier wait that runs out sets MRP_DEV_TIMEOUT and the
 // CTA leaves; the others then run out as well.
 #include <cuda_fp16.h>
@@ -376,193 +382,193 @@ sk_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant__ 
                     __syncwarp();
                     if (lane == 0) mbar_arrive(tempty_bar(acc));     // the accumulator buffer is free again
                 } else {
-                // (1) park this slice: scratch[cta][column][lane]
-                float *mine = p.scratch + ((size_t)cta * RP) * 128;
+                    // (1) park this slice: scratch[cta][column][lane]
+                    float *mine = p.scratch + ((size_t)cta * RP) * 128;
 #pragma unroll 1
-                for (int ch = 0; ch < n_ch; ++ch) {
-                    float v[16], w[16];
-                    tmem_ld16(lane_addr + ch * 16, v);
-                    tmem_ld16(lane_addr + RP + ch * 16, w);
+                    for (int ch = 0; ch < n_ch; ++ch) {
+                        float v[16], w[16];
+                        tmem_ld16(lane_addr + ch * 16, v);
+                        tmem_ld16(lane_addr + RP + ch * 16, w);
 #pragma unroll
-                    for (int j = 0; j < 16; ++j)
-                        if (ch * 16 + j < p.M) mine[(ch * 16 + j) * 128 + t] = v[j] + w[j];
-                }
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(tempty_bar(acc));     // the accumulator buffer is free again
-                // (2) meet the other CTAs of the tile.  One thread's fence after the CTA barrier publishes
-                // every thread's stores (fences are cumulative), and costs one wait instead of four.
-                ch_epi_sync();
-                if (t == 0) {
-                    __threadfence();
-                    *reinterpret_cast<volatile int *>(aux + kChAuxParked) = i + 1;
-                    unsigned int *cnt = reinterpret_cast<unsigned int *>(p.counters) + i * kChTilesPerPhase + tile;
-                    atomicAdd(cnt, 1u);
-                    if (!grid_bar_wait(cnt, (unsigned int)ph.n_split, abort_flag, p)) *vote_s = 1;
-                }
-                ch_epi_sync();
-                if (*vote_s == 1) { alive = false; break; }
-                // (3) this CTA's share of the tile's output rows, element by element from the parked slices
-                const int rows_tile = ph.kind == CH_GU ? 64 : 128;
-                const int per = (rows_tile + ph.n_split - 1) / ph.n_split;
-                const int r0 = split * per;
-                const int n_r = max(0, min(rows_tile, r0 + per) - r0);
-                const int n_items = n_r * p.M;
-                const float *first = p.scratch + ((size_t)tile * ph.n_split * RP) * 128;
-                if (ph.kind == CH_GU) {
-                    bool done = false;
-                    if constexpr (RP >= 32) {
-                        // many batch rows: four consecutive outputs per item, 16-byte loads, 8-byte stores
-                        if ((per & 3) == 0 && (ph.w_rows & 3) == 0 && n_r > 0) {
-                            const int n_g = n_r >> 2;
-                            done = true;
+                        for (int j = 0; j < 16; ++j)
+                            if (ch * 16 + j < p.M) mine[(ch * 16 + j) * 128 + t] = v[j] + w[j];
+                    }
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(tempty_bar(acc));     // the accumulator buffer is free again
+                    // (2) meet the other CTAs of the tile.  One thread's fence after the CTA barrier publishes
+                    // every thread's stores (fences are cumulative), and costs one wait instead of four.
+                    ch_epi_sync();
+                    if (t == 0) {
+                        __threadfence();
+                        *reinterpret_cast<volatile int *>(aux + kChAuxParked) = i + 1;
+                        unsigned int *cnt = reinterpret_cast<unsigned int *>(p.counters) + i * kChTilesPerPhase + tile;
+                        atomicAdd(cnt, 1u);
+                        if (!grid_bar_wait(cnt, (unsigned int)ph.n_split, abort_flag, p)) *vote_s = 1;
+                    }
+                    ch_epi_sync();
+                    if (*vote_s == 1) { alive = false; break; }
+                    // (3) this CTA's share of the tile's output rows, element by element from the parked slices
+                    const int rows_tile = ph.kind == CH_GU ? 64 : 128;
+                    const int per = (rows_tile + ph.n_split - 1) / ph.n_split;
+                    const int r0 = split * per;
+                    const int n_r = max(0, min(rows_tile, r0 + per) - r0);
+                    const int n_items = n_r * p.M;
+                    const float *first = p.scratch + ((size_t)tile * ph.n_split * RP) * 128;
+                    if (ph.kind == CH_GU) {
+                        bool done = false;
+                        if constexpr (RP >= 32) {
+                            // many batch rows: four consecutive outputs per item, 16-byte loads, 8-byte stores
+                            if ((per & 3) == 0 && (ph.w_rows & 3) == 0 && n_r > 0) {
+                                const int n_g = n_r >> 2;
+                                done = true;
 #pragma unroll 2
-                            for (int e = t; e < n_g * p.M; e += 128) {
-                                const int m = e / n_g, row = r0 + ((e - m * n_g) << 2);
+                                for (int e = t; e < n_g * p.M; e += 128) {
+                                    const int m = e / n_g, row = r0 + ((e - m * n_g) << 2);
+                                    const int f = tile * 64 + row;
+                                    if (f < ph.w_rows) {
+                                        float4 g = make_float4(0.f, 0.f, 0.f, 0.f), u = g;
+                                        for (int s0 = 0; s0 < ph.n_split; s0 += 4) {  // slice order; 4 slices' loads in flight
+                                            float4 gs[4], us[4];
+#pragma unroll
+                                            for (int k = 0; k < 4; ++k) {
+                                                const float *src = first + ((size_t)(s0 + k) * RP + m) * 128 + row;
+                                                const bool in = s0 + k < ph.n_split;
+                                                gs[k] = in ? __ldcg(reinterpret_cast<const float4 *>(src)) : make_float4(0.f, 0.f, 0.f, 0.f);
+                                                us[k] = in ? __ldcg(reinterpret_cast<const float4 *>(src + 64)) : make_float4(0.f, 0.f, 0.f, 0.f);
+                                            }
+#pragma unroll
+                                            for (int k = 0; k < 4; ++k) {
+                                                g.x += gs[k].x; g.y += gs[k].y; g.z += gs[k].z; g.w += gs[k].w;
+                                                u.x += us[k].x; u.y += us[k].y; u.z += us[k].z; u.w += us[k].w;
+                                            }
+                                        }
+                                        const float rs = rstd_s[m];
+                                        const float gg[4] = {g.x * rs, g.y * rs, g.z * rs, g.w * rs};
+                                        const float uu[4] = {u.x * rs, u.y * rs, u.z * rs, u.w * rs};
+                                        float av[4];
+#pragma unroll
+                                        for (int k = 0; k < 4; ++k) av[k] = gg[k] / (1.f + __expf(-gg[k])) * uu[k];
+                                        ch_store_split4(p.act + (size_t)m * p.F + f, (size_t)p.lo_x * p.F, av);
+                                    }
+                                }
+                            }
+                        }
+                        if (!done) {
+#pragma unroll 2
+                            for (int e = t; e < n_items; e += 128) {
+                                const int m = e / n_r, row = r0 + (e - m * n_r);
                                 const int f = tile * 64 + row;
                                 if (f < ph.w_rows) {
-                                    float4 g = make_float4(0.f, 0.f, 0.f, 0.f), u = g;
-                                    for (int s0 = 0; s0 < ph.n_split; s0 += 4) {  // slice order; 4 slices' loads in flight
-                                        float4 gs[4], us[4];
+                                    float g = 0.f, u = 0.f;
+                                    for (int s0 = 0; s0 < ph.n_split; s0 += 8) {  // slice order; 8 slices' loads in flight
+                                        float gs[8], us[8];
 #pragma unroll
-                                        for (int k = 0; k < 4; ++k) {
+                                        for (int k = 0; k < 8; ++k) {
                                             const float *src = first + ((size_t)(s0 + k) * RP + m) * 128 + row;
-                                            const bool in = s0 + k < ph.n_split;
-                                            gs[k] = in ? __ldcg(reinterpret_cast<const float4 *>(src)) : make_float4(0.f, 0.f, 0.f, 0.f);
-                                            us[k] = in ? __ldcg(reinterpret_cast<const float4 *>(src + 64)) : make_float4(0.f, 0.f, 0.f, 0.f);
+                                            gs[k] = (s0 + k < ph.n_split) ? __ldcg(src) : 0.f;
+                                            us[k] = (s0 + k < ph.n_split) ? __ldcg(src + 64) : 0.f;
                                         }
+#pragma unroll
+                                        for (int k = 0; k < 8; ++k) { g += gs[k]; u += us[k]; }
+                                    }
+                                    g *= rstd_s[m];
+                                    u *= rstd_s[m];
+                                    ch_store_hi_lo(p.act + (size_t)m * p.F + f, (size_t)p.lo_x * p.F, g / (1.f + __expf(-g)) * u);
+                                }
+                            }
+                        }
+                    } else {
+                        int n_sq = n_r;                      // entries of the buffer of squares per batch row
+                        bool done = false;
+                        if constexpr (RP >= 32) {
+                            // Many batch rows: a share is thousands of outputs, so four consecutive output
+                            // rows are handled per item with 16-byte loads and 8-byte stores.
+                            if ((per & 3) == 0 && (ph.w_rows & 3) == 0 && n_r > 0) {
+                                const int n_g = n_r >> 2;
+                                n_sq = n_g;
+                                done = true;
+#pragma unroll 2
+                                for (int e = t; e < n_g * p.M; e += 128) {
+                                    const int m = e / n_g, row = r0 + ((e - m * n_g) << 2);
+                                    const int j = tile * 128 + row;
+                                    float sq = 0.f;
+                                    if (j < ph.w_rows) {
+                                        const size_t o = (size_t)m * p.d + j;
+                                        const float4 hc = __ldcg(reinterpret_cast<const float4 *>(p.hcur + o));
+                                        const float4 h0 = __ldg(reinterpret_cast<const float4 *>(p.h0f + o));
+                                        float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+                                        for (int s0 = 0; s0 < ph.n_split; s0 += 8) {  // slice order; 8 slices' loads in flight
+                                            float4 as[8];
+#pragma unroll
+                                            for (int k = 0; k < 8; ++k)
+                                                as[k] = (s0 + k < ph.n_split)
+                                                            ? __ldcg(reinterpret_cast<const float4 *>(first + ((size_t)(s0 + k) * RP + m) * 128 + row))
+                                                            : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                                            for (int k = 0; k < 8; ++k) { a.x += as[k].x; a.y += as[k].y; a.z += as[k].z; a.w += as[k].w; }
+                                        }
+                                        const float h[4] = {hc.x + a.x, hc.y + a.y, hc.z + a.z, hc.w + a.w};
+                                        const float hz[4] = {h0.x, h0.y, h0.z, h0.w};
+                                        *reinterpret_cast<float4 *>(p.hcur + o) = make_float4(h[0], h[1], h[2], h[3]);
+                                        if (ph.hidden_out) *reinterpret_cast<float4 *>(ph.hidden_out + o) = make_float4(h[0], h[1], h[2], h[3]);
+                                        sq = (h[0] * h[0] + h[1] * h[1]) + (h[2] * h[2] + h[3] * h[3]);
+                                        float r[4], xn[4];
 #pragma unroll
                                         for (int k = 0; k < 4; ++k) {
-                                            g.x += gs[k].x; g.y += gs[k].y; g.z += gs[k].z; g.w += gs[k].w;
-                                            u.x += us[k].x; u.y += us[k].y; u.z += us[k].z; u.w += us[k].w;
+                                            r[k] = h[k] - hz[k];
+                                            xn[k] = ph.xg_next ? h[k] * __bfloat162float(ph.gamma_next[j + k]) : 0.f;
                                         }
+                                        ch_store_split4(ph.xt_k + o, (size_t)p.lo_xt * p.d, r);
+                                        if (ph.xt16_k) {
+                                            __half2 hh[2] = {__floats2half2_rn(r[0], r[1]), __floats2half2_rn(r[2], r[3])};
+                                            *reinterpret_cast<uint2 *>(ph.xt16_k + o) = *reinterpret_cast<uint2 *>(hh);
+                                        }
+                                        if (ph.xg_next) ch_store_split4(ph.xg_next + o, (size_t)p.lo_x * p.d, xn);
                                     }
-                                    const float rs = rstd_s[m];
-                                    const float gg[4] = {g.x * rs, g.y * rs, g.z * rs, g.w * rs};
-                                    const float uu[4] = {u.x * rs, u.y * rs, u.z * rs, u.w * rs};
-                                    float av[4];
-#pragma unroll
-                                    for (int k = 0; k < 4; ++k) av[k] = gg[k] / (1.f + __expf(-gg[k])) * uu[k];
-                                    ch_store_split4(p.act + (size_t)m * p.F + f, (size_t)p.lo_x * p.F, av);
+                                    sq_s[e] = sq;
                                 }
                             }
                         }
-                    }
-                    if (!done) {
+                        if (!done) {
 #pragma unroll 2
-                    for (int e = t; e < n_items; e += 128) {
-                        const int m = e / n_r, row = r0 + (e - m * n_r);
-                        const int f = tile * 64 + row;
-                        if (f < ph.w_rows) {
-                            float g = 0.f, u = 0.f;
-                            for (int s0 = 0; s0 < ph.n_split; s0 += 8) {  // slice order; 8 slices' loads in flight
-                                float gs[8], us[8];
-#pragma unroll
-                                for (int k = 0; k < 8; ++k) {
-                                    const float *src = first + ((size_t)(s0 + k) * RP + m) * 128 + row;
-                                    gs[k] = (s0 + k < ph.n_split) ? __ldcg(src) : 0.f;
-                                    us[k] = (s0 + k < ph.n_split) ? __ldcg(src + 64) : 0.f;
-                                }
-#pragma unroll
-                                for (int k = 0; k < 8; ++k) { g += gs[k]; u += us[k]; }
-                            }
-                            g *= rstd_s[m];
-                            u *= rstd_s[m];
-                            ch_store_hi_lo(p.act + (size_t)m * p.F + f, (size_t)p.lo_x * p.F, g / (1.f + __expf(-g)) * u);
-                        }
-                    }
-                    }
-                } else {
-                    int n_sq = n_r;                      // entries of the buffer of squares per batch row
-                    bool done = false;
-                    if constexpr (RP >= 32) {
-                        // Many batch rows: a share is thousands of outputs, so four consecutive output
-                        // rows are handled per item with 16-byte loads and 8-byte stores.
-                        if ((per & 3) == 0 && (ph.w_rows & 3) == 0 && n_r > 0) {
-                            const int n_g = n_r >> 2;
-                            n_sq = n_g;
-                            done = true;
-#pragma unroll 2
-                            for (int e = t; e < n_g * p.M; e += 128) {
-                                const int m = e / n_g, row = r0 + ((e - m * n_g) << 2);
+                            for (int e = t; e < n_items; e += 128) {
+                                const int m = e / n_r, row = r0 + (e - m * n_r);
                                 const int j = tile * 128 + row;
                                 float sq = 0.f;
                                 if (j < ph.w_rows) {
                                     const size_t o = (size_t)m * p.d + j;
-                                    const float4 hc = __ldcg(reinterpret_cast<const float4 *>(p.hcur + o));
-                                    const float4 h0 = __ldg(reinterpret_cast<const float4 *>(p.h0f + o));
-                                    float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+                                    const float hc = __ldcg(p.hcur + o), h0 = __ldg(p.h0f + o);
+                                    float a = 0.f;
                                     for (int s0 = 0; s0 < ph.n_split; s0 += 8) {  // slice order; 8 slices' loads in flight
-                                        float4 as[8];
+                                        float as[8];
 #pragma unroll
                                         for (int k = 0; k < 8; ++k)
-                                            as[k] = (s0 + k < ph.n_split)
-                                                        ? __ldcg(reinterpret_cast<const float4 *>(first + ((size_t)(s0 + k) * RP + m) * 128 + row))
-                                                        : make_float4(0.f, 0.f, 0.f, 0.f);
+                                            as[k] = (s0 + k < ph.n_split) ? __ldcg(first + ((size_t)(s0 + k) * RP + m) * 128 + row) : 0.f;
 #pragma unroll
-                                        for (int k = 0; k < 8; ++k) { a.x += as[k].x; a.y += as[k].y; a.z += as[k].z; a.w += as[k].w; }
+                                        for (int k = 0; k < 8; ++k) a += as[k];
                                     }
-                                    const float h[4] = {hc.x + a.x, hc.y + a.y, hc.z + a.z, hc.w + a.w};
-                                    const float hz[4] = {h0.x, h0.y, h0.z, h0.w};
-                                    *reinterpret_cast<float4 *>(p.hcur + o) = make_float4(h[0], h[1], h[2], h[3]);
-                                    if (ph.hidden_out) *reinterpret_cast<float4 *>(ph.hidden_out + o) = make_float4(h[0], h[1], h[2], h[3]);
-                                    sq = (h[0] * h[0] + h[1] * h[1]) + (h[2] * h[2] + h[3] * h[3]);
-                                    float r[4], xn[4];
-#pragma unroll
-                                    for (int k = 0; k < 4; ++k) {
-                                        r[k] = h[k] - hz[k];
-                                        xn[k] = ph.xg_next ? h[k] * __bfloat162float(ph.gamma_next[j + k]) : 0.f;
-                                    }
-                                    ch_store_split4(ph.xt_k + o, (size_t)p.lo_xt * p.d, r);
-                                    if (ph.xt16_k) {
-                                        __half2 hh[2] = {__floats2half2_rn(r[0], r[1]), __floats2half2_rn(r[2], r[3])};
-                                        *reinterpret_cast<uint2 *>(ph.xt16_k + o) = *reinterpret_cast<uint2 *>(hh);
-                                    }
-                                    if (ph.xg_next) ch_store_split4(ph.xg_next + o, (size_t)p.lo_x * p.d, xn);
+                                    const float h = hc + a;
+                                    p.hcur[o] = h;
+                                    if (ph.hidden_out) ph.hidden_out[o] = h;
+                                    sq = h * h;
+                                    ch_store_hi_lo(ph.xt_k + o, (size_t)p.lo_xt * p.d, h - h0);
+                                    if (ph.xt16_k) ph.xt16_k[o] = __float2half_rn(h - h0);
+                                    if (ph.xg_next) ch_store_hi_lo(ph.xg_next + o, (size_t)p.lo_x * p.d, h * __bfloat162float(ph.gamma_next[j]));
                                 }
                                 sq_s[e] = sq;
                             }
                         }
-                    }
-                    if (!done) {
-#pragma unroll 2
-                    for (int e = t; e < n_items; e += 128) {
-                        const int m = e / n_r, row = r0 + (e - m * n_r);
-                        const int j = tile * 128 + row;
-                        float sq = 0.f;
-                        if (j < ph.w_rows) {
-                            const size_t o = (size_t)m * p.d + j;
-                            const float hc = __ldcg(p.hcur + o), h0 = __ldg(p.h0f + o);
-                            float a = 0.f;
-                            for (int s0 = 0; s0 < ph.n_split; s0 += 8) {  // slice order; 8 slices' loads in flight
-                                float as[8];
-#pragma unroll
-                                for (int k = 0; k < 8; ++k)
-                                    as[k] = (s0 + k < ph.n_split) ? __ldcg(first + ((size_t)(s0 + k) * RP + m) * 128 + row) : 0.f;
-#pragma unroll
-                                for (int k = 0; k < 8; ++k) a += as[k];
-                            }
-                            const float h = hc + a;
-                            p.hcur[o] = h;
-                            if (ph.hidden_out) ph.hidden_out[o] = h;
-                            sq = h * h;
-                            ch_store_hi_lo(ph.xt_k + o, (size_t)p.lo_xt * p.d, h - h0);
-                            if (ph.xt16_k) ph.xt16_k[o] = __float2half_rn(h - h0);
-                            if (ph.xg_next) ch_store_hi_lo(ph.xg_next + o, (size_t)p.lo_x * p.d, h * __bfloat162float(ph.gamma_next[j]));
+                        ch_epi_sync();
+                        // this CTA's rows, in row order, then one integer add per row of the batch
+                        for (int m = t; m < p.M; m += 128) {
+                            float s = 0.f;
+                            for (int r = 0; r < n_sq; ++r) s += sq_s[m * n_sq + r];
+                            atomicAdd(p.ssq_fix + ph.ssq_idx * 128 + m,
+                                      (unsigned long long)__double2ll_rn((double)s * 16777216.0));
                         }
-                        sq_s[e] = sq;
-                    }
-                    }
-                    ch_epi_sync();
-                    // this CTA's rows, in row order, then one integer add per row of the batch
-                    for (int m = t; m < p.M; m += 128) {
-                        float s = 0.f;
-                        for (int r = 0; r < n_sq; ++r) s += sq_s[m * n_sq + r];
-                        atomicAdd(p.ssq_fix + ph.ssq_idx * 128 + m,
-                                  (unsigned long long)__double2ll_rn((double)s * 16777216.0));
                     }
                 }
-                }   // slices parked and added
             }
             // this CTA's part of the phase is in memory: arrive at the grid barrier
             ch_epi_sync();
