@@ -129,10 +129,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_holder;
+    // launched behind its predecessor with programmatic dependent launch: everything above overlaps
+    // the predecessor's tail; the roles that touch its outputs wait for it first
+    pdl_trigger();
 
     if (warp == 0) {
         // ---------------- TMA producer ----------------
         if (lane == 0) {
+            pdl_wait();
             const uint32_t tx = (uint32_t)(PARTS * kATile + p.bn * 128);
             const int box_rows = p.bn / p.n_boxes;
             int s = 0;
@@ -200,6 +204,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
     } else {
         // ---------------- epilogue warps (TMEM lane quadrant = warp % 4) ----------------
+        pdl_wait();
         const int q = warp & 3;
         const int rl = q * 32 + lane;
         const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
@@ -495,7 +500,7 @@ size_t smem_bytes(const TcParams &p, int parts)
 
 template <int KIND, bool MARGIN, bool F16 = false>
 cudaError_t launch_tc(const CUtensorMap &a, const CUtensorMap &b0, const CUtensorMap &b1, const TcParams &p,
-                      int grid, cudaStream_t st)
+                      int grid, cudaStream_t st, bool pdl)
 {
     auto kern = tc_gemm_kernel<KIND, MARGIN, F16>;
     const size_t smem = smem_bytes(p, F16 ? 1 : 2);
@@ -510,8 +515,7 @@ cudaError_t launch_tc(const CUtensorMap &a, const CUtensorMap &b0, const CUtenso
         if (ea != cudaSuccess) return ea;
         attr_devices.fetch_or(bit);
     }
-    kern<<<grid, kThreads, smem, st>>>(a, b0, b1, p);
-    return cudaGetLastError();
+    return launch_k(kern, dim3(grid), dim3(kThreads), smem, st, pdl, a, b0, b1, p);
 }
 
 }  // namespace
@@ -646,7 +650,7 @@ cudaError_t tc_draft(Ctx *c, const void *hidden, const float *logits0, const int
         if (!make_map(s, &mA, xg, d, 2 * (uint64_t)M, 128) || !make_map(s, &mB0, hw.w_gate, d, F, p.bn / 2) ||
             !make_map(s, &mB1, hw.w_up, d, F, p.bn / 2))
             return note_err(c, cudaErrorInvalidValue, "tensor map (gate/up)");
-        e = note_err(c, launch_tc<KIND_GU, false>(mA, mB0, mB1, p, p.n_groups * p.n_vr, st), "gate/up kernel");
+        e = note_err(c, launch_tc<KIND_GU, false>(mA, mB0, mB1, p, p.n_groups * p.n_vr, st, pdl), "gate/up kernel");
         c->launches++;
         if (e != cudaSuccess) return e;
         // down projection, residual add, next operands
@@ -665,7 +669,7 @@ cudaError_t tc_draft(Ctx *c, const void *hidden, const float *logits0, const int
         finish_shape(p, G / p.n_groups);
         if (!make_map(s, &mA, act, F, 2 * (uint64_t)M, 128) || !make_map(s, &mB0, hw.w_down, F, d, p.bn))
             return note_err(c, cudaErrorInvalidValue, "tensor map (down)");
-        e = note_err(c, launch_tc<KIND_DN, false>(mA, mB0, mB0, p, p.n_groups * p.n_vr, st), "down kernel");
+        e = note_err(c, launch_tc<KIND_DN, false>(mA, mB0, mB0, p, p.n_groups * p.n_vr, st, pdl), "down kernel");
         c->launches++;
         if (e != cudaSuccess) return e;
         n_ss = p.n_vr;
@@ -703,14 +707,14 @@ cudaError_t tc_draft(Ctx *c, const void *hidden, const float *logits0, const int
             if (!make_map(s, &mA, c->ws + c->lay.xt16, d, (uint64_t)rows, 128) ||
                 !make_map(s, &mB, c->ws + c->lay.w16, d, V, p.bn))
                 return note_err(c, cudaErrorInvalidValue, "tensor map (LM head, fp16)");
-            e = note_err(c, out.margin ? launch_tc<KIND_LM, true, true>(mA, mB, mB, p, grid, st)
-                                       : launch_tc<KIND_LM, false, true>(mA, mB, mB, p, grid, st),
+            e = note_err(c, out.margin ? launch_tc<KIND_LM, true, true>(mA, mB, mB, p, grid, st, pdl)
+                                       : launch_tc<KIND_LM, false, true>(mA, mB, mB, p, grid, st, pdl),
                          "LM-head kernel (fp16 operands)");
         } else {
             if (!make_map(s, &mA, xt, d, 2 * (uint64_t)n_rs, 128) || !make_map(s, &mB, c->w_lm, d, V, p.bn))
                 return note_err(c, cudaErrorInvalidValue, "tensor map (LM head)");
-            e = note_err(c, out.margin ? launch_tc<KIND_LM, true>(mA, mB, mB, p, grid, st)
-                                       : launch_tc<KIND_LM, false>(mA, mB, mB, p, grid, st), "LM-head kernel");
+            e = note_err(c, out.margin ? launch_tc<KIND_LM, true>(mA, mB, mB, p, grid, st, pdl)
+                                       : launch_tc<KIND_LM, false>(mA, mB, mB, p, grid, st, pdl), "LM-head kernel");
         }
         c->launches++;
         if (e != cudaSuccess) return e;
