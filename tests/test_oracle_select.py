@@ -280,3 +280,21 @@ def test_direct_decoding_loop_needs_ceil_L_over_K_plus_one_forwards():
             n += 1
             assert n <= L
         assert n == -(-L // (K + 1))
+
+
+def test_commit_positionwise_acceptance_keeps_a_later_match():
+    """Algorithm 3 read literally (per position): a later draft that the backbone confirms is kept
+    even though an earlier one was rejected; with prefix acceptance it is not."""
+    tokens = np.array([-1, -1, -1, -1], np.int32)
+    ri = np.arange(4, dtype=np.int32)
+    conf = np.array([[0.9, 0.1, 0.2, 0.3], [0.0, 0.8, 0.2, 0.3], [0.0, 0.0, 0.7, 0.3]], np.float32)
+    tok = np.array([[1, 2, 3, 4], [11, 12, 13, 14], [21, 22, 23, 24]], np.int32)
+    sel = oracle.select(conf, tok, ri, 1, 4, oracle.STATIC)
+    assert sel.draft_pos.tolist() == [[1, 2]] and sel.draft_tok.tolist() == [[12, 23]]
+    verify_tok = np.array([[99, 23]], np.int32)          # first draft rejected, second confirmed
+    alen, amask = oracle.verify(sel.draft_tok, verify_tok, sel.draft_len, positionwise=False)
+    assert alen.tolist() == [0] and amask.tolist() == [[0, 0]]
+    assert oracle.commit(tokens, sel, 1, 4, accept_mask=amask).tokens.tolist() == [1, -1, -1, -1]
+    alen, amask = oracle.verify(sel.draft_tok, verify_tok, sel.draft_len, positionwise=True)
+    assert alen.tolist() == [1] and amask.tolist() == [[0, 1]]
+    assert oracle.commit(tokens, sel, 1, 4, accept_mask=amask).tokens.tolist() == [1, -1, 23, -1]
