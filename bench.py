@@ -362,6 +362,25 @@ def main():
     ri = torch.from_numpy(inp.row_index).to(dev)
     out = harness.alloc_draft_out(M, K, w.V, w.d, dev, margin=False)
     sel = harness.alloc_select_out(B, L, K, dev)
+    alen = torch.empty(B, device=dev, dtype=torch.int32)
+    # The results a caller reads back after a step live in one device arena (the library only
+    # sees pointers), so the end-to-end leg returns them with a single device-to-host copy.
+    res_names = [(out, "conf"), (out, "token"), (sel, "reveal_mask"), (sel, "remask_mask"),
+                 (sel, "out_token"), (sel, "draft_len")]
+    res_shapes = [(getattr(o, n).shape, getattr(o, n).dtype) for o, n in res_names] + [(alen.shape, alen.dtype)]
+    offs, total = [], 0
+    for shp, dt in res_shapes:
+        offs.append(total)
+        nbytes = int(np.prod(shp)) * torch.empty((), dtype=dt).element_size()
+        total += (nbytes + 15) // 16 * 16
+    arena = torch.zeros(total, device=dev, dtype=torch.uint8)
+    views = []
+    for (shp, dt), o in zip(res_shapes, offs):
+        nbytes = int(np.prod(shp)) * torch.empty((), dtype=dt).element_size()
+        views.append(arena[o:o + nbytes].view(dt).view(shp))
+    for (o, n), v in zip(res_names, views[:-1]):
+        setattr(o, n, v)
+    alen = views[-1]
     mode = binding.MRP_SELECT_STATIC if static else binding.MRP_SELECT_DYNAMIC_REMASK
     launches = [0]
 
@@ -378,7 +397,6 @@ def main():
             n += ctx.last_launch_count
         launches[0] = n
 
-    alen = torch.empty(B, device=dev, dtype=torch.int32)
     amask = torch.empty((B, K), device=dev, dtype=torch.int8)
     vt = torch.zeros((B, K), device=dev, dtype=torch.int32)
     step()
@@ -444,12 +462,11 @@ def main():
         h_hid = hid.cpu().pin_memory()
         h_l0 = l0.cpu().pin_memory()
         h_ri = ri.cpu().pin_memory()
-        res = [out.conf, out.token, sel.reveal_mask, sel.remask_mask, sel.out_token, sel.draft_len, alen]
-        h_res = [torch.empty_like(t, device="cpu").pin_memory() for t in res]
+        h_arena = torch.empty_like(arena, device="cpu").pin_memory()
         bi = h_hid.numel() * h_hid.element_size() + h_ri.numel() * 4
         if not args.from_hidden:
             bi += h_l0.numel() * 4
-        bo = sum(t.numel() * t.element_size() for t in res)
+        bo = arena.numel()
         n_e2e = max(3, min(args.steps, 300))
 
         # The base logits are needed by the LM-head kernel only: their copy (the bulk of the input
@@ -471,8 +488,7 @@ def main():
             hid.copy_(h_hid, non_blocking=True)
             ri.copy_(h_ri, non_blocking=True)
             step()
-            for s, dcpu in zip(res, h_res):
-                dcpu.copy_(s, non_blocking=True)
+            h_arena.copy_(arena, non_blocking=True)
 
         # The library's calls are stream-ordered and allocate nothing, so a caller can record
         # the whole step (input copies, the three C-ABI calls, result copies) in a CUDA graph
