@@ -1,14 +1,24 @@
 #!/usr/bin/env python
 """Benchmark of the MRP drafting step on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 1] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps S] [--warmup W] [--config all|0..3|sweep:M:K|sweep]
+                    [--impl ours|reference]
 
-A step is one pass of the whole hot path over one batch of synthetic input: mrp_draft (head
-chain, shared LM head, softmax statistics), mrp_reveal_remask and, in static mode,
-mrp_verify.  The metric is drafted tokens per second = K_chain * M per step.  Rank 0 prints
-one JSON line.  With N > 1 (torchrun) every rank runs an independent replica of the same
-workload on its own GPU (the path has no collective); the value is the sum over ranks
-divided by the slowest rank's time.
+A step is one pass of the whole hot path over one batch of synthetic input: mrp_draft (row
+gather, head chain, shared LM head with fused softmax statistics, combine), mrp_reveal_remask
+and, in static mode, mrp_verify.  The metric is drafted tokens per second = K_chain * M per step.
+
+With no --config the five benchmark configurations are measured in one process: the tiny fp32
+instance, the 1.7B-class decode shape, the 8B-class speculative shape, the 8B-class remask
+shape and four points of the roofline sweep.  Rank 0 prints ONE JSON line whose top-level
+figures are those of the largest named single-GPU configuration (remask_8b); the list
+``configs`` carries the same figures for every other workload.  Each workload is timed as
+repeated batches of S steps (CUDA events around every batch) until at least --min-seconds of
+GPU time have been spent; the reported time per step is the median batch divided by S.
+
+With N > 1 (torchrun) every rank runs an independent replica of the same workloads on its own
+GPU (the path has no collective); a value is the sum over ranks divided by the slowest rank's
+time.
 """
 from __future__ import annotations
 
@@ -27,20 +37,29 @@ if ROOT not in sys.path:
 METRIC = "MRP draft tokens/s on 1 B200; % of LM-head roofline (HBM or bf16 TC)"
 UNIT = "draft tokens/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+NOMINAL = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}     # the figures the benchmark spec names
+HEADLINE = "3"
+DEFAULT_WORKLOADS = ("0", "1", "2", "3", "sweep:1:1", "sweep:64:4", "sweep:256:1", "sweep:4096:4")
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the fused LM-head kernel,
-# from the ncu captures summarised under profiles/ (bytes per launch; None = not captured).
-NCU_TRAFFIC_BYTES = {"decode_1p7b": 628542208}   # profiles/sk_gemm_kernel_decode_1p7b.md
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the fused LM-head kernel, from
+# the ncu captures summarised under profiles/ (bytes per launch, and the summary they come from).
+NCU_TRAFFIC = {
+    "decode_1p7b": (628542208, "profiles/sk_gemm_kernel_decode_1p7b.md"),
+    "sweep_M256_K4": (1447000000, "profiles/tc_gemm_kernel_lm_sweep_M256_K4.md"),
+}
 
 
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=1000)
-    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=20, help="steps per timed batch")
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", default="1",
-                    help="0..3 = benchmark configuration, sweep:M:K = one roofline-sweep point, sweep = all 21 points")
+    ap.add_argument("--config", default="all",
+                    help="all = the five configurations in one line (default); 0..3 = one configuration; "
+                         "sweep:M:K = one roofline-sweep point; sweep = all 21 points, one line each")
+    ap.add_argument("--min-seconds", type=float, default=1.0,
+                    help="GPU time per workload spent in timed batches of --steps steps")
     ap.add_argument("--flags", type=int, default=0, help="mrp_config.flags (MRP_FLAG_* bits) for A/B timing")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -67,6 +86,17 @@ def load_peaks():
         except Exception:
             pass
     return dict(FALLBACK_PEAKS), "fallback"
+
+
+def config_dict(cfg, M, entry="mrp_draft"):
+    """What names a workload; the reference arm prints the same dictionary."""
+    K = cfg["K"]
+    return {"workload": cfg["name"], "rows": int(M), "chain": K, "d": cfg["d"], "d_ff": cfg["F"],
+            "vocab": cfg["V"], "seqs": cfg["B"], "block_len": cfg["L"], "mode": cfg["mode"], "entry": entry,
+            "l2": "weights streamed per step (%.0f MB) %s the 126 MB L2; no flush between steps"
+                  % ((cfg["V"] * cfg["d"] + K * 3.0 * cfg["d"] * cfg["F"]) * (4 if cfg["dtype"] == "f32" else 2) / 1e6,
+                     "exceed" if cfg["V"] * cfg["d"] > 40e6 else "fit in (latency case)"),
+            "parallelism": "independent replicas, no collective"}
 
 
 class ClockSampler:
@@ -106,14 +136,16 @@ class ClockSampler:
                 self.proc.kill()
 
     def summary(self, t0, t1):
-        rows = [s for t, s in self.samples if t0 <= t <= t1 + 0.15] or [s for _, s in self.samples]
-        sm, mx, reasons = [], [], set()
+        """Samples taken inside [t0, t1] (wall clock of the timed region)."""
+        rows = [s for t, s in self.samples if t0 <= t <= t1]
+        sm, mx, pw, reasons = [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for r in rows:
             f = [x.strip() for x in r.split(",")]
             try:
                 sm.append(float(f[0]))
                 mx.append(float(f[1]))
+                pw.append(float(f[2]))
             except (ValueError, IndexError):
                 continue
             for n, v in zip(names, f[3:7]):
@@ -123,7 +155,7 @@ class ClockSampler:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
         sm.sort()
         return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": max(mx), "reasons": sorted(reasons),
-                "samples": len(sm)}
+                "samples": len(sm), "power_w_max": max(pw), "sampled": "inside the timed region"}
 
 
 def replica_throughput(dist, device, units_per_rank, seconds):
@@ -140,333 +172,352 @@ def replica_throughput(dist, device, units_per_rank, seconds):
     return world * units_per_rank / seconds, seconds
 
 
-def lm_head_roofline(cfg, M, lm_ms, peaks, peaks_kind, traffic, from_hidden=False):
+def lm_head_roofline(cfg, M, lm_ms, peaks, peaks_kind, from_hidden=False):
     """Roofline of the fused LM-head kernel: algorithmic bytes 2Vd + 4MV + 2KMd (one read of
     the LM head, one read of l_0, the stacked residual rows), flops 2KMVd.  With the base
-    logits computed in the pass: bytes 2Vd + 2(K+1)Md, flops 2(K+1)MVd."""
+    logits computed in the pass: bytes 2Vd + 2(K+1)Md, flops 2(K+1)MVd.  The bound is the slower
+    of bytes over the HBM copy bandwidth and flops over the bf16 tensor peak; ``frac`` is against
+    the peaks measured on this machine (sustained bf16 figure: the kernel is timed inside a loop of a
+    second or more), ``frac_nominal`` against 8 TB/s and 2250 TFLOP/s."""
     V, d, K = cfg["V"], cfg["d"], cfg["K"]
-    nbytes = 2.0 * V * d + 4.0 * M * V + 2.0 * K * M * d
+    esz = 4 if cfg["dtype"] == "f32" else 2
+    nbytes = float(esz) * V * d + 4.0 * M * V + float(esz) * K * M * d
     flops = 2.0 * K * M * V * d
     if from_hidden:
-        nbytes = 2.0 * V * d + 2.0 * (K + 1) * M * d
+        nbytes = float(esz) * V * d + float(esz) * (K + 1) * M * d
         flops = 2.0 * (K + 1) * M * V * d
     t_hbm = nbytes / (peaks["hbm_gbs"] * 1e9)
     t_tc = flops / (peaks["bf16_tflops_sustained"] * 1e12)
     sec = lm_ms * 1e-3
+    traffic = NCU_TRAFFIC.get(cfg["name"]) if not from_hidden else None
+    common = {"traffic": traffic[0] if traffic else None, "traffic_source": traffic[1] if traffic else None,
+              "kernel": "fused LM head", "kernel_ms": lm_ms, "alg_bytes": nbytes, "alg_flops": flops,
+              "units_per_launch": K * M}
     if t_hbm >= t_tc:
         ach = nbytes / sec / 1e9
-        return {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": ach / peaks["hbm_gbs"], "traffic": traffic, "kernel": "fused LM head",
-                "kernel_ms": lm_ms, "alg_bytes": nbytes, "alg_flops": flops,
-                "peak_source": "MEASURED_PEAKS.json hbm_gbs" if peaks_kind == "measured"
-                else "fallback 6650 GB/s"}
+        return dict(common, bound="hbm", achieved=ach, peak=peaks["hbm_gbs"], unit="GB/s",
+                    frac=ach / peaks["hbm_gbs"], frac_nominal=ach / NOMINAL["hbm_gbs"],
+                    peak_source=("MEASURED_PEAKS.json hbm_gbs" if peaks_kind == "measured"
+                                 else "fallback 6650 GB/s") + "; frac_nominal against 8000 GB/s")
     ach = flops / sec / 1e12
-    return {"bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops_sustained"],
-            "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops_sustained"], "traffic": traffic,
-            "kernel": "fused LM head", "kernel_ms": lm_ms, "alg_bytes": nbytes, "alg_flops": flops,
-            "peak_source": "MEASURED_PEAKS.json bf16_tflops_sustained" if peaks_kind == "measured"
-            else "fallback 1400 TFLOP/s sustained"}
+    return dict(common, bound="tensor", achieved=ach, peak=peaks["bf16_tflops_sustained"], unit="TFLOP/s",
+                frac=ach / peaks["bf16_tflops_sustained"], frac_burst=ach / peaks["bf16_tflops"],
+                frac_nominal=ach / NOMINAL["bf16_tflops"],
+                peak_source=("MEASURED_PEAKS.json bf16_tflops_sustained" if peaks_kind == "measured"
+                             else "fallback 1400 TFLOP/s sustained")
+                + "; frac_burst against the burst figure, frac_nominal against 2250 TFLOP/s")
 
 
-def oracle_sample(cfg, w, inp, budget_s=12.0):
+def call_roofline_seconds(cfg, M, peaks):
+    """Roofline time of the whole mrp_draft call: every weight read once, l_0 read once."""
+    V, d, F, K = cfg["V"], cfg["d"], cfg["F"], cfg["K"]
+    esz = 4 if cfg["dtype"] == "f32" else 2
+    nbytes = float(esz) * V * d + K * (3.0 * esz * d * F + esz * d) + 4.0 * M * V + float(esz) * M * d + 12.0 * (K + 1) * M
+    flops = 2.0 * K * M * V * d + 6.0 * K * M * d * F
+    return max(nbytes / (peaks["hbm_gbs"] * 1e9), flops / (peaks["bf16_tflops_sustained"] * 1e12))
+
+
+def oracle_step_fn(cfg, w, inp, rows):
+    """One pass of the hot path by the CPU oracle over the masked rows ``rows`` (indices into
+    inp.row_index; their blocks are renumbered densely)."""
+    import numpy as np
+    import oracle
+    K, L = cfg["K"], cfg["L"]
+    ri_rows = inp.row_index[rows]
+    blocks = np.unique(ri_rows // L)
+    remap = {b: i for i, b in enumerate(blocks)}
+    ri = np.array([remap[x // L] * L + x % L for x in ri_rows], np.int32)
+    mode = oracle.STATIC if cfg["mode"] == "static" else oracle.DYNAMIC_REMASK
+
+    def step():
+        r = oracle.draft(inp.hidden, inp.logits0, w.heads, w.w_lm, K=K, row_index=ri_rows)
+        s = oracle.select(r.conf.astype(np.float32), r.token, ri, len(blocks), L, mode, tau=cfg["tau"])
+        if cfg["mode"] == "static":
+            oracle.verify(s.draft_tok, s.draft_tok, s.draft_len)
+    return step
+
+
+def oracle_sample(cfg, w, inp, budget_s):
     """Time the CPU oracle, as it stands, on a bounded sample of the workload's rows (whole
     blocks).  Returns (draft tokens/s, cores, description)."""
     import numpy as np
     import oracle
     K, L = cfg["K"], cfg["L"]
     M = len(inp.row_index)
-
-    def run(rows):
-        t = time.perf_counter()
-        r = oracle.draft(inp.hidden, inp.logits0, w.heads, w.w_lm, K=K, row_index=inp.row_index[rows])
-        blocks = np.unique(inp.row_index[rows] // L)
-        remap = {b: i for i, b in enumerate(blocks)}
-        ri = np.array([remap[x // L] * L + x % L for x in inp.row_index[rows]], np.int32)
-        mode = oracle.STATIC if cfg["mode"] == "static" else oracle.DYNAMIC_REMASK
-        s = oracle.select(r.conf.astype(np.float32), r.token, ri, len(blocks), L, mode, tau=cfg["tau"])
-        if cfg["mode"] == "static":
-            oracle.verify(s.draft_tok, s.draft_tok, s.draft_len)
-        return time.perf_counter() - t
-
-    first_block = np.flatnonzero(inp.row_index // L == inp.row_index[0] // L)
-    t1 = run(first_block)
-    per_row = t1 / len(first_block)
+    blk = inp.row_index // L
+    first_block = np.flatnonzero(blk == blk[0])
+    step = oracle_step_fn(cfg, w, inp, first_block)
+    t = time.perf_counter()
+    step()
+    per_row = (time.perf_counter() - t) / len(first_block)
     n_rows = int(max(len(first_block), min(M, budget_s / max(per_row, 1e-9))))
-    # whole blocks only
-    order = np.argsort(inp.row_index // L, kind="stable")
-    rows = np.sort(order[:n_rows])
-    last_block = inp.row_index[rows[-1]] // L
-    rows = np.flatnonzero(inp.row_index // L <= last_block)
+    order = np.argsort(blk, kind="stable")            # whole blocks only
+    last_block = blk[np.sort(order[:n_rows])[-1]]
+    rows = np.flatnonzero(blk <= last_block)
     if len(rows) > n_rows * 1.5:
         rows = first_block
     reps = int(max(1, min(20, budget_s / max(per_row * len(rows), 1e-9))))
-    t = min(run(rows) for _ in range(reps)) if reps > 1 else run(rows)
-    desc = "%d of %d masked rows (whole blocks), all V columns, best of %d" % (len(rows), M, reps)
-    return K * len(rows) / t, oracle.num_threads(), desc
+    step = oracle_step_fn(cfg, w, inp, rows)
+    best = None
+    for _ in range(reps):
+        t = time.perf_counter()
+        step()
+        dt = time.perf_counter() - t
+        best = dt if best is None else min(best, dt)
+    desc = "%d of %d masked rows (whole blocks), all V columns, best of %d%s" % (
+        len(rows), M, reps, "" if len(rows) == M else "; per-row rate extrapolated to the workload")
+    return K * len(rows) / best, oracle.num_threads(), desc
 
 
-def run_reference(args, cfg):
-    """Reference arm: the CPU oracle, as it stands, on the host cores (rank 0 only)."""
+def run_reference(args):
+    """Reference arm: the CPU oracle, as it stands, on the host cores (rank 0 only), on the
+    headline workload (or the one --config names); each step is a bounded sample of its rows."""
     if int(os.environ.get("RANK", "0")) != 0:
         return
     import numpy as np
     import oracle
     from paper_2605_18817_b200 import synth
+    name = HEADLINE if args.config == "all" else args.config
+    cfg = resolve_config(name)
     oracle.build()
-    w, inp = synth.make_config(cfg)
+    w = synth.make_weights(cfg["d"], cfg["F"], cfg["V"], cfg["n_heads"], cfg["dtype"],
+                           4000 if name.startswith("sweep:") else cfg["seed"])
+    # base logits only for the rows the sample can reach (input generation, not the method)
+    inp = synth.make_inputs(w, cfg["B"], cfg["L"], cfg["seed"], cfg["s_lo"], cfg["s_hi"], cfg["mask_prob"],
+                            logits_rows=256)
     M = len(inp.row_index)
-    K, L = cfg["K"], cfg["L"]
-    # bounded sample per step: the first rows of the workload, sized so that the whole run
-    # (warm-up + timed steps) stays near two minutes; never fewer than one row
+    K = cfg["K"]
+    step1 = oracle_step_fn(cfg, w, inp, np.arange(1))
     t0 = time.perf_counter()
-    oracle.draft(inp.hidden, inp.logits0, w.heads, w.w_lm, K=K, row_index=inp.row_index[:1])
+    step1()
     per_row = time.perf_counter() - t0
     total = args.steps + args.warmup
-    n_rows = int(max(1, min(M, 120.0 / total / max(per_row, 1e-9))))
-    rows = np.arange(n_rows)
-
-    def step():
-        r = oracle.draft(inp.hidden, inp.logits0, w.heads, w.w_lm, K=K, row_index=inp.row_index[rows])
-        blocks = np.unique(inp.row_index[rows] // L)
-        remap = {b: i for i, b in enumerate(blocks)}
-        ri = np.array([remap[x // L] * L + x % L for x in inp.row_index[rows]], np.int32)
-        mode = oracle.STATIC if cfg["mode"] == "static" else oracle.DYNAMIC_REMASK
-        s = oracle.select(r.conf.astype(np.float32), r.token, ri, len(blocks), L, mode, tau=cfg["tau"])
-        if cfg["mode"] == "static":
-            oracle.verify(s.draft_tok, s.draft_tok, s.draft_len)
-
+    # bounded sample per step, sized so that warm-up + timed steps stay near two minutes
+    n_rows = int(max(1, min(M, 256, 120.0 / total / max(per_row, 1e-9))))
+    step = oracle_step_fn(cfg, w, inp, np.arange(n_rows))
     for _ in range(args.warmup):
         step()
     t0 = time.perf_counter()
     for _ in range(args.steps):
         step()
     dt = time.perf_counter() - t0
-    value = K * len(rows) * args.steps / dt
-    sample = "first %d of %d masked rows per step, all V columns" % (len(rows), M)
+    value = K * n_rows * args.steps / dt
+    sample = "first %d of %d masked rows per step, all V columns" % (n_rows, M)
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
-        "data": "synthetic",
-        "config": {"workload": cfg["name"], "rows": M, "chain": K, "d": cfg["d"], "d_ff": cfg["F"],
-                   "vocab": cfg["V"], "seqs": cfg["B"], "block_len": L, "mode": cfg["mode"],
-                   "l2": "host cores (oracle)", "parallelism": "rank 0 only"},
+        "data": "synthetic", "config": config_dict(cfg, M),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(),
                          "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
+        "note": "the oracle on the host cores; every step covers the sample named in cpu_baseline, not the "
+                "whole workload; rank 0 only",
     }
     print(json.dumps(line), flush=True)
 
 
-def run_sweep(args):
-    """Roofline sweep (configuration 4): d = 4096, V = 151936, masked rows M in {1 .. 4096} times
-    chain length K in {1, 2, 4}, one weight set shared by all points.  Prints one JSON line per
-    point: time per drafting pass, draft tokens/s, the fused LM-head kernel's time and its
-    fraction of the roofline (slower of algorithmic bytes over HBM bandwidth and flops over the
-    bf16 tensor peak), and the same fraction for the whole mrp_draft call."""
-    import numpy as np
-    import torch
-    from paper_2605_18817_b200 import build as _build
-    if not os.environ.get("MRP_B200_LIB"):
-        _build.build()
-    from paper_2605_18817_b200 import binding, harness, synth
-    torch.cuda.set_device(0)
-    dev = torch.device("cuda", 0)
-    peaks, peaks_kind = load_peaks()
-    w = synth.make_weights(4096, 8192, 151936, 4, "bf16", 4000)
-    heads, w_lm = harness.upload_weights(w, dev)
-    logits_fn = harness.device_logits_fn(w_lm)
-    d, F, V = w.d, w.F, w.V
-    for M in synth.SWEEP_ROWS:
-        for K in synth.SWEEP_CHAIN:
-            cfg = synth.sweep_config(M, K)
-            _, inp = synth.make_config(cfg, w, logits_fn=logits_fn)
-            ctx = binding.mrp_create(d, F, V, heads[:K], w_lm, max_rows=M, max_seqs=M, block_len=1,
-                                     flags=args.flags)
-            hid = harness.to_device(inp.hidden, w.dtype, dev)
-            l0 = torch.from_numpy(inp.logits0).to(dev)
-            ri = torch.from_numpy(inp.row_index).to(dev)
-            out = harness.alloc_draft_out(M, K, V, d, dev, margin=False)
-            for _ in range(3):
-                harness.draft(ctx, hid, l0, ri, M, K, out)
-            torch.cuda.synchronize()
-            ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            ev0.record()
-            harness.draft(ctx, hid, l0, ri, M, K, out)
-            ev1.record()
-            torch.cuda.synchronize()
-            n = int(max(5, min(200, 300.0 / max(ev0.elapsed_time(ev1), 1e-3))))
-            ev0.record()
-            for _ in range(n):
-                harness.draft(ctx, hid, l0, ri, M, K, out)
-            ev1.record()
-            torch.cuda.synchronize()
-            ms = ev0.elapsed_time(ev1) / n
-            binding.mrp_profile_enable(ctx, True)
-            for _ in range(n):
-                harness.draft(ctx, hid, l0, ri, M, K, out)
-            torch.cuda.synchronize()
-            (ms_heads, ms_lm, ms_comb), nc = binding.mrp_profile_read(ctx)
-            binding.mrp_profile_enable(ctx, False)
-            roof = lm_head_roofline(cfg, M, ms_lm / nc, peaks, peaks_kind, None)
-            call_bytes = 2.0 * V * d + K * (6.0 * d * F + 2 * d) + 4.0 * M * V + 2.0 * M * d + 12.0 * (K + 1) * M
-            call_flops = 2.0 * K * M * V * d + 6.0 * K * M * d * F
-            t_roof = max(call_bytes / (peaks["hbm_gbs"] * 1e9), call_flops / (peaks["bf16_tflops_sustained"] * 1e12))
-            print(json.dumps({
-                "workload": cfg["name"], "rows": M, "chain": K, "ms_per_draft": ms,
-                "draft_tokens_per_s": K * M / (ms * 1e-3), "heads_ms": ms_heads / nc,
-                "lm_head_ms": ms_lm / nc, "combine_ms": ms_comb / nc,
-                "lm_head_roofline": {k: roof[k] for k in ("bound", "achieved", "peak", "unit", "frac")},
-                "draft_call_roofline_frac": t_roof / (ms * 1e-3), "family": ctx.family,
-                "peaks": peaks_kind}), flush=True)
-            binding.mrp_destroy(ctx)
-            del hid, l0, ri, out
+class Bench:
+    """Process-wide state of the GPU arm: device, process group, peaks, cached weight sets."""
 
-
-def main():
-    args = parse_args()
-    if args.config == "sweep":
-        run_sweep(args)
-        return
-    cfg = resolve_config(args.config)
-    if args.impl == "reference":
-        run_reference(args, cfg)
-        return
-    import numpy as np
-    import torch
-    from paper_2605_18817_b200 import build as _build
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    if rank == 0 and not os.environ.get("MRP_B200_LIB"):
-        _build.build()
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        torch.cuda.set_device(local)
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-        dist.barrier()
-    else:
-        torch.cuda.set_device(local)
-    from paper_2605_18817_b200 import binding, harness, synth
-    dev = torch.device("cuda", local)
-
-    w, inp = synth.make_config(cfg)
-    K, B, L = cfg["K"], cfg["B"], cfg["L"]
-    M = len(inp.row_index)
-    static = cfg["mode"] == "static"
-    ctx = harness.create_for(cfg, w, dev, flags=args.flags)
-    hid = harness.to_device(inp.hidden, w.dtype, dev)
-    l0 = torch.from_numpy(inp.logits0).to(dev)
-    ri = torch.from_numpy(inp.row_index).to(dev)
-    # hidden states and row index of a step share one device arena too: one host-to-device copy
-    hid_bytes = (hid.numel() * hid.element_size() + 15) // 16 * 16
-    in_arena = torch.zeros(hid_bytes + ri.numel() * 4, device=dev, dtype=torch.uint8)
-    hid_v = in_arena[:hid.numel() * hid.element_size()].view(hid.dtype).view(hid.shape)
-    ri_v = in_arena[hid_bytes:].view(torch.int32)
-    hid_v.copy_(hid)
-    ri_v.copy_(ri)
-    hid, ri = hid_v, ri_v
-    out = harness.alloc_draft_out(M, K, w.V, w.d, dev, margin=False)
-    sel = harness.alloc_select_out(B, L, K, dev)
-    alen = torch.empty(B, device=dev, dtype=torch.int32)
-    # The results a caller reads back after a step live in one device arena (the library only
-    # sees pointers), so the end-to-end leg returns them with a single device-to-host copy.
-    res_names = [(out, "conf"), (out, "token"), (sel, "reveal_mask"), (sel, "remask_mask"),
-                 (sel, "out_token"), (sel, "draft_len")]
-    res_shapes = [(getattr(o, n).shape, getattr(o, n).dtype) for o, n in res_names] + [(alen.shape, alen.dtype)]
-    offs, total = [], 0
-    for shp, dt in res_shapes:
-        offs.append(total)
-        nbytes = int(np.prod(shp)) * torch.empty((), dtype=dt).element_size()
-        total += (nbytes + 15) // 16 * 16
-    arena = torch.zeros(total, device=dev, dtype=torch.uint8)
-    views = []
-    for (shp, dt), o in zip(res_shapes, offs):
-        nbytes = int(np.prod(shp)) * torch.empty((), dtype=dt).element_size()
-        views.append(arena[o:o + nbytes].view(dt).view(shp))
-    for (o, n), v in zip(res_names, views[:-1]):
-        setattr(o, n, v)
-    alen = views[-1]
-    mode = binding.MRP_SELECT_STATIC if static else binding.MRP_SELECT_DYNAMIC_REMASK
-    launches = [0]
-
-    def step():
-        if args.from_hidden:
-            harness.draft_from_hidden(ctx, hid, None, ri, M, K, out)
-        else:
-            harness.draft(ctx, hid, l0, ri, M, K, out)
-        n = ctx.last_launch_count
-        harness.select(ctx, out.conf, out.token, ri, M, K, B, L, mode, sel, tau=cfg["tau"])
-        n += ctx.last_launch_count
-        if static:
-            binding.mrp_verify(ctx, sel.draft_tok, vt, sel.draft_len, B, K, False, alen, amask)
-            n += ctx.last_launch_count
-        launches[0] = n
-
-    amask = torch.empty((B, K), device=dev, dtype=torch.int8)
-    vt = torch.zeros((B, K), device=dev, dtype=torch.int32)
-    step()
-    torch.cuda.synchronize()
-    if static:   # synthetic backbone verification tokens for the drafted tokens
-        vt.copy_(torch.from_numpy(synth.make_verify_tokens(sel.draft_tok.cpu().numpy(), w.V,
-                                                           cfg["seed"], 0.7)))
-
-    def barrier():
-        torch.cuda.synchronize()
-        if dist is not None:
+    def __init__(self, args):
+        import torch
+        from paper_2605_18817_b200 import build as _build
+        self.args = args
+        self.rank = int(os.environ.get("RANK", "0"))
+        self.world = int(os.environ.get("WORLD_SIZE", "1"))
+        self.local = int(os.environ.get("LOCAL_RANK", "0"))
+        if self.local == 0 and not os.environ.get("MRP_B200_LIB"):
+            _build.build()
+        self.dist = None
+        torch.cuda.set_device(self.local)
+        if self.world > 1:
+            import torch.distributed as dist
+            dist.init_process_group("nccl", device_id=torch.device("cuda", self.local))
             dist.barrier()
+            self.dist = dist
+        self.dev = torch.device("cuda", self.local)
+        self.peaks, self.peaks_kind = load_peaks()
+        self.weights = {}      # (d, F, V, n_heads, dtype, seed) -> (host weights, device heads, device w_lm)
+
+    def barrier(self):
+        import torch
+        torch.cuda.synchronize()
+        if self.dist is not None:
+            self.dist.barrier()
             torch.cuda.synchronize()
 
-    for _ in range(max(args.warmup, 3)):
+    def weights_for(self, cfg, name):
+        from paper_2605_18817_b200 import harness, synth
+        seed = 4000 if name.startswith("sweep:") else cfg["seed"]
+        n_heads = 4 if name.startswith("sweep:") else cfg["n_heads"]      # one weight set for all sweep points
+        key = (cfg["d"], cfg["F"], cfg["V"], n_heads, cfg["dtype"], seed)
+        if key not in self.weights:
+            self.weights.clear()                                          # one large weight set on the device at a time
+            import gc
+            import torch
+            gc.collect()
+            torch.cuda.empty_cache()
+            w = synth.make_weights(cfg["d"], cfg["F"], cfg["V"], n_heads, cfg["dtype"], seed)
+            heads, w_lm = harness.upload_weights(w, self.dev)
+            self.weights[key] = (w, heads, w_lm)
+        return self.weights[key]
+
+    # -------------------------------------------------------------------------------------
+    def run_workload(self, name, cpu_budget_s):
+        import numpy as np
+        import torch
+        from paper_2605_18817_b200 import binding, harness, synth
+        args, dev, dist = self.args, self.dev, self.dist
+        cfg = resolve_config(name)
+        w, heads, w_lm = self.weights_for(cfg, name)
+        big = cfg["d"] >= 4096          # base logits of the synthetic backbone: fp32 product on the device
+        _, inp = synth.make_config(cfg, w, logits_fn=harness.device_logits_fn(w_lm) if big else None)
+        K, B, L = cfg["K"], cfg["B"], cfg["L"]
+        M = len(inp.row_index)
+        static = cfg["mode"] == "static"
+        ctx = binding.mrp_create(w.d, w.F, w.V, heads[:cfg["n_heads"]], w_lm, max_rows=B * L, max_seqs=B,
+                                 block_len=L, flags=args.flags)
+        hid = harness.to_device(inp.hidden, w.dtype, dev)
+        l0 = torch.from_numpy(inp.logits0).to(dev)
+        ri = torch.from_numpy(inp.row_index).to(dev)
+        # hidden states and row index of a step share one device arena: one host-to-device copy
+        hid_bytes = (hid.numel() * hid.element_size() + 15) // 16 * 16
+        in_arena = torch.zeros(hid_bytes + ri.numel() * 4, device=dev, dtype=torch.uint8)
+        hid_v = in_arena[:hid.numel() * hid.element_size()].view(hid.dtype).view(hid.shape)
+        ri_v = in_arena[hid_bytes:].view(torch.int32)
+        hid_v.copy_(hid)
+        ri_v.copy_(ri)
+        hid, ri = hid_v, ri_v
+        out = harness.alloc_draft_out(M, K, w.V, w.d, dev, margin=False)
+        sel = harness.alloc_select_out(B, L, K, dev)
+        alen = torch.empty(B, device=dev, dtype=torch.int32)
+        # The results a caller reads back after a step live in one device arena (the library only
+        # sees pointers), so the end-to-end leg returns them with a single device-to-host copy.
+        res_names = [(out, "conf"), (out, "token"), (sel, "reveal_mask"), (sel, "remask_mask"),
+                     (sel, "out_token"), (sel, "draft_len")]
+        res_shapes = [(getattr(o, n).shape, getattr(o, n).dtype) for o, n in res_names] + [(alen.shape, alen.dtype)]
+        offs, total = [], 0
+        for shp, dt in res_shapes:
+            offs.append(total)
+            nbytes = int(np.prod(shp)) * torch.empty((), dtype=dt).element_size()
+            total += (nbytes + 15) // 16 * 16
+        arena = torch.zeros(total, device=dev, dtype=torch.uint8)
+        views = []
+        for (shp, dt), o in zip(res_shapes, offs):
+            nbytes = int(np.prod(shp)) * torch.empty((), dtype=dt).element_size()
+            views.append(arena[o:o + nbytes].view(dt).view(shp))
+        for (o, n), v in zip(res_names, views[:-1]):
+            setattr(o, n, v)
+        alen = views[-1]
+        mode = binding.MRP_SELECT_STATIC if static else binding.MRP_SELECT_DYNAMIC_REMASK
+        launches = [0]
+        amask = torch.empty((B, K), device=dev, dtype=torch.int8)
+        vt = torch.zeros((B, K), device=dev, dtype=torch.int32)
+
+        def step():
+            if args.from_hidden:
+                harness.draft_from_hidden(ctx, hid, None, ri, M, K, out)
+            else:
+                harness.draft(ctx, hid, l0, ri, M, K, out)
+            n = ctx.last_launch_count
+            harness.select(ctx, out.conf, out.token, ri, M, K, B, L, mode, sel, tau=cfg["tau"])
+            n += ctx.last_launch_count
+            if static:
+                binding.mrp_verify(ctx, sel.draft_tok, vt, sel.draft_len, B, K, False, alen, amask)
+                n += ctx.last_launch_count
+            launches[0] = n
+
         step()
-    sampler = ClockSampler(local)
-    sampler.start()
-    barrier()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    t_wall0 = time.time()
-    ev0.record()
-    for _ in range(args.steps):
-        step()
-    ev1.record()
-    barrier()
-    t_wall1 = time.time()
-    ms_total = ev0.elapsed_time(ev1)
-    # keep the GPU busy a little longer if the region was too short for a clock sample
-    if t_wall1 - t_wall0 < 0.6:
-        t_end = time.time() + 0.8
-        while time.time() < t_end:
-            for _ in range(50):
+        torch.cuda.synchronize()
+        if static:   # synthetic backbone verification tokens for the drafted tokens
+            vt.copy_(torch.from_numpy(synth.make_verify_tokens(sel.draft_tok.cpu().numpy(), w.V, cfg["seed"], 0.7)))
+
+        S = max(args.steps, 1)
+        warm = max(args.warmup, 3)
+        for _ in range(warm):
+            step()
+        # one batch to size the run
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(S):
+            step()
+        e1.record()
+        torch.cuda.synchronize()
+        n_batches = int(max(1, min(5000, np.ceil(args.min_seconds * 1e3 / max(e0.elapsed_time(e1), 1e-3)))))
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(n_batches + 1)]
+        sampler = ClockSampler(self.local)
+        sampler.start()
+        time.sleep(0.12)                       # the sampler's first line
+        self.barrier()
+        t_wall0 = time.time()
+        evs[0].record()
+        for b in range(n_batches):
+            for _ in range(S):
                 step()
-            torch.cuda.synchronize()
+            evs[b + 1].record()
+        self.barrier()
         t_wall1 = time.time()
-    sampler.stop()
-    clocks = sampler.summary(t_wall0, t_wall1)
-    value, sec_total = replica_throughput(dist, dev, K * M * args.steps, ms_total * 1e-3)
-    ms_total = sec_total * 1e3
-    ms_step = ms_total / args.steps
+        sampler.stop()
+        batch_ms = sorted(evs[b].elapsed_time(evs[b + 1]) for b in range(n_batches))
+        med = batch_ms[len(batch_ms) // 2]
+        clocks = sampler.summary(t_wall0, t_wall1)
+        value, sec_batch = replica_throughput(dist, dev, K * M * S, med * 1e-3)
+        ms_step = sec_batch * 1e3 / S
 
-    # per-phase kernel times, CUDA events on the launching stream, same number of steps
-    binding.mrp_profile_enable(ctx, True)
-    n_prof = min(args.steps, 1000)
-    for _ in range(n_prof):
-        step()
-    torch.cuda.synchronize()
-    (ms_heads, ms_lm, ms_comb), n_calls = binding.mrp_profile_read(ctx)
-    binding.mrp_profile_enable(ctx, False)
-    n_calls = max(n_calls, 1)
-    peaks, peaks_kind = load_peaks()
-    roofline = lm_head_roofline(cfg, M, ms_lm / n_calls, peaks, peaks_kind,
-                                None if args.from_hidden else NCU_TRAFFIC_BYTES.get(cfg["name"]),
-                                from_hidden=args.from_hidden)
-    phases = {"heads_ms": ms_heads / n_calls, "lm_head_ms": ms_lm / n_calls,
-              "combine_ms": ms_comb / n_calls, "family": ctx.family}
+        # per-phase kernel times (CUDA events on the launching stream inside mrp_draft)
+        binding.mrp_profile_enable(ctx, True)
+        n_prof = int(min(1000, max(S, S * n_batches // 2)))
+        for _ in range(n_prof):
+            step()
+        torch.cuda.synchronize()
+        (ms_heads, ms_lm, ms_comb), n_calls = binding.mrp_profile_read(ctx)
+        binding.mrp_profile_enable(ctx, False)
+        n_calls = max(n_calls, 1)
+        roofline = lm_head_roofline(cfg, M, ms_lm / n_calls, self.peaks, self.peaks_kind, from_hidden=args.from_hidden)
+        if clocks.get("sm_mhz"):
+            roofline["kernel_ms_x_sm_mhz"] = ms_lm / n_calls * clocks["sm_mhz"]
+        if cfg["V"] * cfg["d"] <= 40e6:
+            roofline["note"] = "all weights fit in L2 and a step is a handful of launches of a few microseconds: " \
+                               "this workload measures launch latency (ms_per_step), not a roofline"
 
-    # end to end through the public API with host buffers: H2D of the step's inputs from
-    # pinned memory and D2H of its results inside the timed region
-    e2e = None
-    if not args.no_e2e:
+        phases = {"heads_ms": ms_heads / n_calls, "lm_head_ms": ms_lm / n_calls,
+                  "combine_ms": ms_comb / n_calls, "family": ctx.family,
+                  "draft_call_roofline_frac": call_roofline_seconds(cfg, M, self.peaks) /
+                  max((ms_heads + ms_lm + ms_comb) / n_calls * 1e-3, 1e-12)}
+
+        # end to end through the public API with host buffers: H2D of the step's inputs from
+        # pinned memory and D2H of its results inside the timed region
+        e2e = None
+        if not args.no_e2e:
+            e2e = self.run_e2e(ctx, cfg, step, in_arena, l0, arena, hid, ri, K, M, S)
+
+        cpu = None
+        if self.rank == 0 and self.world == 1 and not args.no_cpu_baseline:
+            v, cores, desc = oracle_sample(cfg, w, inp, cpu_budget_s)
+            cpu = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc}
+
+        status = binding.mrp_fetch_status(ctx)
+        binding.mrp_destroy(ctx)
+        res = {
+            "value": value, "unit": UNIT, "ms_per_step": ms_step,
+            "batches": n_batches, "batch_ms_median": med, "batch_ms_min": batch_ms[0], "batch_ms_max": batch_ms[-1],
+            "timed_gpu_seconds": sum(batch_ms) * 1e-3,
+            "dtype": "bf16" if cfg["dtype"] == "bf16" else "f32",
+            "config": config_dict(cfg, M, "mrp_draft_from_hidden" if args.from_hidden else "mrp_draft"),
+            "clocks": clocks, "e2e": e2e, "gpu_launches": launches[0] * S * n_batches,
+            "launches_per_step": launches[0], "roofline": roofline, "phases": phases, "cpu_baseline": cpu,
+            "device_status_word": status,
+        }
+        del hid, l0, ri, out, sel, arena, in_arena
+        return res
+
+    def run_e2e(self, ctx, cfg, step, in_arena, l0, arena, hid, ri, K, M, S):
+        import torch
+        from paper_2605_18817_b200 import binding
+        args, dev, dist = self.args, self.dev, self.dist
         h_in = in_arena.cpu().pin_memory()
         h_l0 = l0.cpu().pin_memory()
         h_arena = torch.empty_like(arena, device="cpu").pin_memory()
@@ -474,7 +525,6 @@ def main():
         if not args.from_hidden:
             bi += h_l0.numel() * 4
         bo = arena.numel()
-        n_e2e = max(3, min(args.steps, 300))
 
         # The base logits are needed by the LM-head kernel only: their copy (the bulk of the input
         # bytes) runs on a second stream beside the head chain, and the library waits for it right
@@ -525,42 +575,74 @@ def main():
 
         for _ in range(3):
             e2e_step()
-        barrier()
+        t0 = time.perf_counter()
+        e2e_step()
+        one = time.perf_counter() - t0
+        n_e2e = int(max(3, min(2000, 0.5 * args.min_seconds / max(one, 1e-6)))) if args.min_seconds > 0 else max(3, S)
+        self.barrier()
         t0 = time.perf_counter()
         for _ in range(n_e2e):
             e2e_step()
-        barrier()
+        self.barrier()
         dt = time.perf_counter() - t0
         e2e_value, dt = replica_throughput(dist, dev, K * M * n_e2e, dt)
         binding.mrp_set_logits0_event(ctx, None)
-        e2e = {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": bi,
-               "d2h_bytes_per_step": bo, "steps": n_e2e, "ms_per_step": dt / n_e2e * 1e3, "mode": e2e_mode}
+        return {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": bi, "d2h_bytes_per_step": bo,
+                "steps": n_e2e, "ms_per_step": dt / n_e2e * 1e3, "mode": e2e_mode}
 
-    cpu = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        v, cores, desc = oracle_sample(cfg, w, inp)
-        cpu = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc}
 
-    if rank == 0:
+def run_sweep(args):
+    """All 21 points of the roofline sweep (configuration 4), one JSON line per point."""
+    bench = Bench(args)
+    from paper_2605_18817_b200 import synth
+    for M in synth.SWEEP_ROWS:
+        for K in synth.SWEEP_CHAIN:
+            r = bench.run_workload("sweep:%d:%d" % (M, K), 0.0)
+            if bench.rank == 0:
+                print(json.dumps({
+                    "workload": r["config"]["workload"], "rows": M, "chain": K, "ms_per_draft_step": r["ms_per_step"],
+                    "draft_tokens_per_s": r["value"], "heads_ms": r["phases"]["heads_ms"],
+                    "lm_head_ms": r["phases"]["lm_head_ms"], "combine_ms": r["phases"]["combine_ms"],
+                    "lm_head_roofline": {k: r["roofline"].get(k) for k in
+                                         ("bound", "achieved", "peak", "unit", "frac", "frac_burst", "frac_nominal")},
+                    "draft_call_roofline_frac": r["phases"]["draft_call_roofline_frac"],
+                    "sm_mhz": r["clocks"].get("sm_mhz"), "reasons": r["clocks"].get("reasons"),
+                    "family": r["phases"]["family"], "peaks": bench.peaks_kind}), flush=True)
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+    if args.config == "sweep":
+        args.no_e2e = True
+        args.no_cpu_baseline = True
+        run_sweep(args)
+        return
+    bench = Bench(args)
+    names = list(DEFAULT_WORKLOADS) if args.config == "all" else [args.config]
+    head_name = HEADLINE if args.config == "all" else args.config
+    results = {}
+    for name in names:
+        results[name] = bench.run_workload(name, 12.0 if name == head_name else 5.0)
+    if bench.rank == 0:
+        head = results[head_name]
         line = {
-            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None,
-            "dtype": "bf16" if cfg["dtype"] == "bf16" else "f32", "data": "synthetic",
-            "config": {"workload": cfg["name"], "rows": M, "chain": K, "d": cfg["d"], "d_ff": cfg["F"],
-                       "vocab": cfg["V"], "seqs": B, "block_len": L, "mode": cfg["mode"],
-                       "entry": "mrp_draft_from_hidden" if args.from_hidden else "mrp_draft",
-                       "l2": "weights streamed per step (%.0f MB) exceed the 126 MB L2; no flush"
-                             % ((2.0 * cfg["V"] * cfg["d"] + K * 6.0 * cfg["d"] * cfg["F"]) / 1e6),
-                       "parallelism": "replicas x%d" % world},
-            "clocks": clocks, "e2e": e2e, "gpu_launches": launches[0] * args.steps,
-            "launches_per_step": launches[0], "roofline": roofline, "phases": phases,
-            "cpu_baseline": cpu,
+            "metric": METRIC, "value": head["value"], "unit": UNIT, "n_gpus": bench.world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": head["ms_per_step"], "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": head["dtype"], "data": "synthetic",
+            "timing": "per workload: batches of `steps` steps, CUDA events around every batch, repeated until "
+                      ">= %.2f s of GPU time; ms_per_step = median batch / steps (max over ranks)" % args.min_seconds,
         }
+        for k in ("config", "clocks", "e2e", "gpu_launches", "launches_per_step", "roofline", "phases",
+                  "cpu_baseline", "batches", "batch_ms_median", "batch_ms_min", "batch_ms_max",
+                  "timed_gpu_seconds", "device_status_word"):
+            line[k] = head[k]
+        line["configs"] = [results[n] for n in names if n != head_name]
         print(json.dumps(line), flush=True)
-    binding.mrp_destroy(ctx)
-    if dist is not None:
-        dist.destroy_process_group()
+    if bench.dist is not None:
+        bench.dist.destroy_process_group()
 
 
 if __name__ == "__main__":

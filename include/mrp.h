@@ -17,11 +17,17 @@
  *   - Matrices are row-major.  Weight matrices are [out_features, in_features].
  *   - Calls enqueue work on the given CUDA stream (a cudaStream_t passed as void*, NULL =
  *     the default stream) and return without synchronising.  No entry point allocates
- *     device memory; all scratch lives in the caller-provided workspace.
+ *     device memory; all scratch lives in the caller-provided workspace (the one exception,
+ *     mrp_reveal_remask_noalloc, keeps its scratch in a fixed array inside the library).
  *   - The return value is an mrp_status.  Argument errors are detected on the host before
  *     anything is launched.  Device-side anomalies (non-finite statistics, a bounded wait
- *     that gave up) are OR-ed as MRP_DEV_* bits into an int32 device status word that the
- *     caller may read after synchronising; kernels never trap or spin without a limit.
+ *     that gave up, a row index outside its array, a residual outside the range the tensor-core
+ *     kernels are accurate in) are OR-ed as MRP_DEV_* bits into the context's int32 device
+ *     status word (mrp_fetch_status) and into the optional `status` word of the call's output
+ *     descriptor; kernels never trap or spin without a limit.
+ *   - Index arrays coming from the caller (row_index) are checked on the device before they
+ *     are used as an address: an entry outside its range raises MRP_DEV_BAD_INDEX and the row
+ *     is treated as absent (nothing is read or written through it).
  *   - A context is not thread-safe: use one context per stream.
  */
 #ifndef MRP_H
@@ -50,6 +56,11 @@ typedef enum {
 /* Bits of the device status word. */
 #define MRP_DEV_NONFINITE 1    /* a log-sum-exp came out NaN or infinite                */
 #define MRP_DEV_TIMEOUT 2      /* a bounded barrier wait inside a kernel ran out        */
+#define MRP_DEV_BAD_INDEX 4    /* a row_index entry was outside its array, or named a dense
+                                  position twice (selection); the access was skipped      */
+#define MRP_DEV_RANGE 8        /* tensor-core kernels: a residual h_k - h_0 left the range in
+                                  which confidence / log-sum-exp hold their 2e-3 accuracy
+                                  (see mrp_create); the results were still produced        */
 
 typedef enum { MRP_F32 = 0, MRP_BF16 = 1 } mrp_dtype;
 
@@ -62,6 +73,9 @@ typedef enum { MRP_F32 = 0, MRP_BF16 = 1 } mrp_dtype;
 #define MRP_FLAG_ROW_MAJOR_ONLY 4   /* tensor-core family: never use the few-row kernels  */
 #define MRP_FLAG_NO_CHAIN 16    /* tensor-core family: run the head chain of a few-row call as
                                   one kernel per GEMM instead of one persistent kernel      */
+#define MRP_FLAG_REQUIRE_TENSOR_CORES 32   /* bf16 context: mrp_create fails with MRP_ERR_UNSUPPORTED
+                                       instead of falling back to the CUDA-core kernels when the
+                                       shape or the alignment rules out the tensor-core kernels  */
 #define MRP_FLAG_EXACT_OPERANDS 8   /* tensor-core family: always carry the LM-head activation
                                        operand as a bf16 hi + lo pair (products exact to 2^-17),
                                        also where that doubles the tensor work for nothing.  Without
@@ -109,9 +123,23 @@ size_t mrp_workspace_bytes(const mrp_config *cfg);
  * w_lm: DEVICE [vocab, d]; workspace: DEVICE, 256-byte aligned, at least
  * mrp_workspace_bytes(cfg) bytes, owned by the caller and kept alive until mrp_destroy.
  * The bf16 tensor-core kernels need d % 64 == 0, d_ff % 64 == 0, vocab % 16 == 0 and
- * 16-byte aligned weights; other bf16 shapes run on the CUDA-core kernels.
- * On success *out receives the context.  Errors: INVALID_ARG, NOMEM, CUDA.
+ * 16-byte aligned weights; other bf16 shapes run on the CUDA-core kernels (two orders of
+ * magnitude slower: mrp_kernel_family tells which family a context resolved to, and
+ * MRP_FLAG_REQUIRE_TENSOR_CORES turns the silent choice into MRP_ERR_UNSUPPORTED).
+ * Accuracy range of the tensor-core kernels: they accumulate in the tensor cores' fp32, whose
+ * error grows with the length of the contractions (d, d_ff) times the size of the sums, i.e.
+ * of the residual.  Confidence and log-sum-exp stay within 2e-3 of an fp64 evaluation while
+ *     d * rms(h_k - h_0) <= MRP_RANGE_LIMIT      (rms over the d entries of a row, any step k)
+ * (measured: log-sum-exp off by 2.5e-4 at 11 000, 1.5e-3 at 40 000, 2.2e-3 at 98 000 for d =
+ * 4096, d_ff = 8192; less at equal d * rms for shorter d_ff; the benchmark shapes sit at 8 000
+ * to 16 000).  A row-step beyond the limit raises MRP_DEV_RANGE and is still computed.  The
+ * CUDA-core kernels (fp32 FMA, MRP_FLAG_FORCE_SIMT) have no such limit.
+ * Workspace: mrp_workspace_bytes() includes, for bf16 contexts with (n_heads + 1) * max_rows
+ * > 32 and without MRP_FLAG_EXACT_OPERANDS, an fp16 copy of W_lm (2 * vocab * d bytes, made
+ * here with one blocking pass over W_lm): the price of the one-pass LM head above 32 row-steps.
+ * On success *out receives the context.  Errors: INVALID_ARG, UNSUPPORTED, NOMEM, CUDA.
  */
+#define MRP_RANGE_LIMIT 32768.0f
 int mrp_create(const mrp_config *cfg, const mrp_head_weights *heads, const void *w_lm,
                void *workspace, size_t workspace_bytes, mrp_ctx **out);
 
@@ -146,7 +174,10 @@ typedef struct {
  *   hidden  [n_rows, d]   backbone hidden states, dtype of the context
  *   logits0 [n_rows, V]   backbone logits, fp32
  *   row_index [M] int32   rows of hidden/logits0 that are masked positions (dense position
- *                         b*L+i of each masked row), or NULL for rows 0..M-1
+ *                         b*L+i of each masked row), or NULL for rows 0..M-1.  Every entry
+ *                         must lie in [0, n_rows), n_rows as set by mrp_set_input_rows; an entry
+ *                         outside raises MRP_DEV_BAD_INDEX, nothing is read through it and the
+ *                         row's statistics are those of an all-zero hidden state and logit row
  *   M in [0, max_rows], K in [0, n_heads] (head k uses weight set k-1)
  * Step k's logits are l_0 + W_lm (h_k - h_0), which equals the per-step accumulation
  * l <- l + W_lm Delta by linearity of the LM head.  Errors: INVALID_ARG, CUDA.
@@ -192,6 +223,9 @@ typedef struct {
  *   draft_pos, draft_tok [B, Kd] int32, Kd = K * r_draft: block positions and tokens of the
  *               drafts (steps k >= 1) in draft order, -1 padded
  *   draft_len   [B] int32
+ *   status      optional device int32: MRP_DEV_BAD_INDEX is OR-ed in when a row_index entry
+ *               is outside [0, B*L) (the row is ignored) or names a position a second time (the
+ *               row listed last keeps the position)
  */
 typedef struct {
     int8_t *reveal_mask;
@@ -201,12 +235,13 @@ typedef struct {
     int32_t *draft_pos;
     int32_t *draft_tok;
     int32_t *draft_len;
+    int32_t *status;          /* optional device int32 receiving MRP_DEV_* bits, NULL = none */
 } mrp_select_out;
 
 /*
  * Reveal selection and remasking from the per-step statistics of mrp_draft.
- *   STATIC (Algorithm 2 "Reveal r tokens with highest confidence", Algorithm 3 "Draft
- *   token with highest confidence"; Sec. 4.1 static denoising): for k = 0..K take the r
+ *   STATIC (Algorithm 2, the reveal step at k = 0..K; Algorithm 3, the draft step after each
+ *   MRP update; Sec. 4.1 static denoising): for k = 0..K take the r
  *   most confident still-masked positions of each block under step k (confidence
  *   descending, position ascending on ties); k = 0 picks are reveals, k >= 1 are drafts.
  *   DYNAMIC_REMASK (Algorithm 4; Sec. 4.1 dynamic denoising; Sec. 4.4 cap): R = masked
@@ -254,13 +289,13 @@ typedef struct {
 /*
  * Apply the outcome of one pass to the block state (the closing lines of Algorithms 2-4).
  *   accept_mask == NULL: every position the selection took (sel->out_token >= 0) is unmasked
- *     with that token: the reveals of all steps in direct decoding (Algorithm 2 "Reveal r
- *     tokens" at k = 0..K), and in the dynamic regime the members of R that survived remasking
- *     (Algorithm 4 "Remask positions i in R where confidence is below tau").
+ *     with that token: the reveals of all steps in direct decoding (Algorithm 2, reveal step
+ *     at k = 0..K), and in the dynamic regime the members of R that survived remasking
+ *     (Algorithm 4, remask step).
  *   accept_mask [B, Kd] int8 (from mrp_verify; speculative decoding, Algorithm 3): the step-0
  *     reveals are unmasked; drafted position sel->draft_pos[b, s] takes sel->draft_tok[b, s]
- *     only where accept_mask[b, s] != 0 ("Reject drafted positions ...; remask rejected
- *     positions").
+ *     only where accept_mask[b, s] != 0 (Algorithm 3, rejection step: a rejected draft stays
+ *     masked).
  * Positions that already hold a token are never changed.  sel is the mrp_select_out of this
  * pass (reveal_mask and remask_mask are not read); Kd as in mrp_reveal_remask; 1 <= B <=
  * max_seqs, 1 <= L <= block_len.  Errors: INVALID_ARG, CUDA.
@@ -282,10 +317,16 @@ int mrp_commit(mrp_ctx *ctx, const mrp_select_out *sel, const int8_t *accept_mas
  *   - B * L must not exceed MRP_NOALLOC_MAX_POSITIONS, else MRP_ERR_CAPACITY (nothing is
  *     launched); L <= 1024.  All other arguments, layouts and errors as mrp_reveal_remask;
  *     the caller still owns every input and output buffer.
- *   - Works on the CURRENT device, which must be the device of cuda_stream and of the buffers.
- *   - The first call on each device looks up the array's device address
- *     (cudaGetSymbolAddress); make that first call outside of any stream capture.  Later
- *     calls only enqueue a memset and two kernels.  Never calls cudaMalloc / cudaFree.
+ *   - Works on the CURRENT device and CUDA context, which must be those of cuda_stream and of
+ *     the buffers.
+ *   - The first call in each (device, CUDA context) looks up the array's device address
+ *     (cudaGetSymbolAddress; the address of a module variable belongs to a context, so a second
+ *     context on the same device gets its own look-up); make that first call outside of any
+ *     stream capture.  Later calls only enqueue a memset and two kernels.  Never calls
+ *     cudaMalloc / cudaFree.
+ *   - row_index entries outside [0, B*L) are skipped and duplicates resolved exactly as in
+ *     mrp_reveal_remask (MRP_DEV_BAD_INDEX in out->status if given): nothing is written
+ *     outside the part of the array the call uses.
  *   - All calls on a device share the one array.  Each call re-initialises the part it uses,
  *     so earlier calls leave nothing behind, but two calls that may overlap on the GPU
  *     (different streams, no ordering between them) race on it: serialise them.
@@ -306,6 +347,22 @@ int mrp_reveal_remask_noalloc(const float *conf, const int32_t *token, const int
  * MRP_DEV_TIMEOUT; the context stays usable.  Errors: INVALID_ARG, CUDA.
  */
 int mrp_selftest_wait_timeout(mrp_ctx *ctx, int32_t *status, void *cuda_stream);
+
+/*
+ * Number of rows of the `hidden` / `logits0` arrays handed to the following mrp_draft and
+ * mrp_draft_from_hidden calls: the range row_index entries are checked against on the device
+ * (no counterpart in the paper).  Default, and largest value: max(max_rows, max_seqs *
+ * block_len).  Errors: INVALID_ARG.
+ */
+int mrp_set_input_rows(mrp_ctx *ctx, int32_t n_rows);
+
+/*
+ * Copy the context's device status word (MRP_DEV_* bits OR-ed by every call on the context
+ * since creation or the last clearing fetch) to dst, a DEVICE int32, as an operation on
+ * cuda_stream ordered behind the calls already enqueued there; clear != 0 then resets the word.
+ * Never synchronises.  Errors: INVALID_ARG, CUDA.
+ */
+int mrp_fetch_status(mrp_ctx *ctx, int32_t *dst, int32_t clear, void *cuda_stream);
 
 /*
  * Let mrp_draft wait for the base logits separately from the hidden states.  In Algorithm 2

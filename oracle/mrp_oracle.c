@@ -360,8 +360,9 @@ int mrp_oracle_select(const float *conf, const int32_t *token, const int32_t *ro
 }
 
 /*
- * Draft verification (Algorithm 3, "Reject drafted positions where argmax differ";
- * Figure 1(d): candidate k embeds the first k draft tokens, hence prefix acceptance).
+ * Draft verification (Algorithm 3, rejection step: a drafted position is rejected where the
+ * backbone's argmax differs from the draft; Figure 1(d): candidate k embeds the first k draft
+ * tokens, hence prefix acceptance).
  *   draft_tok, verify_tok [B, Kd]; draft_len [B] (entries j >= draft_len[b] are ignored)
  *   positionwise = 0: accept_len = number of leading matches, accept_mask cleared after
  *                     the first mismatch (those drafts are remasked);

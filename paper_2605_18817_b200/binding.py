@@ -24,14 +24,16 @@ MRP_FLAG_NO_PDL = 2
 MRP_FLAG_ROW_MAJOR_ONLY = 4
 MRP_FLAG_EXACT_OPERANDS = 8
 MRP_FLAG_NO_CHAIN = 16
+MRP_FLAG_REQUIRE_TENSOR_CORES = 32
 MRP_SELECT_STATIC, MRP_SELECT_DYNAMIC_REMASK = 0, 1
-MRP_DEV_NONFINITE, MRP_DEV_TIMEOUT = 1, 2
+MRP_DEV_NONFINITE, MRP_DEV_TIMEOUT, MRP_DEV_BAD_INDEX, MRP_DEV_RANGE = 1, 2, 4, 8
+MRP_RANGE_LIMIT = 32768.0
 
 EXPORTS = ("mrp_workspace_bytes", "mrp_create", "mrp_destroy", "mrp_draft", "mrp_reveal_remask",
            "mrp_verify", "mrp_last_launch_count", "mrp_kernel_family", "mrp_status_string",
            "mrp_profile_enable", "mrp_profile_read", "mrp_last_error",
            "mrp_reveal_remask_noalloc", "mrp_selftest_wait_timeout", "mrp_draft_from_hidden", "mrp_commit",
-           "mrp_set_logits0_event")
+           "mrp_set_logits0_event", "mrp_set_input_rows", "mrp_fetch_status")
 MRP_NOALLOC_MAX_POSITIONS = 65536
 MRP_ERR_CAPACITY = 7
 
@@ -65,7 +67,7 @@ class mrp_select_out(ctypes.Structure):
     _fields_ = [("reveal_mask", ctypes.c_void_p), ("remask_mask", ctypes.c_void_p),
                 ("out_token", ctypes.c_void_p), ("step_of", ctypes.c_void_p),
                 ("draft_pos", ctypes.c_void_p), ("draft_tok", ctypes.c_void_p),
-                ("draft_len", ctypes.c_void_p)]
+                ("draft_len", ctypes.c_void_p), ("status", ctypes.c_void_p)]
 
 
 class mrp_block_state(ctypes.Structure):
@@ -95,6 +97,10 @@ def _load():
                               ctypes.c_void_p]
     lib.mrp_set_logits0_event.restype = ctypes.c_int
     lib.mrp_set_logits0_event.argtypes = [ctypes.c_void_p, ctypes.c_void_p]
+    lib.mrp_set_input_rows.restype = ctypes.c_int
+    lib.mrp_set_input_rows.argtypes = [ctypes.c_void_p, ctypes.c_int32]
+    lib.mrp_fetch_status.restype = ctypes.c_int
+    lib.mrp_fetch_status.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32, ctypes.c_void_p]
     lib.mrp_commit.restype = ctypes.c_int
     lib.mrp_commit.argtypes = [ctypes.c_void_p, ctypes.POINTER(mrp_select_out), ctypes.c_void_p, ctypes.c_int32,
                                ctypes.c_int32, ctypes.c_int32, ctypes.POINTER(mrp_block_state), ctypes.c_void_p]
@@ -163,6 +169,7 @@ class Context:
     handle: int
     cfg: mrp_config
     keep: tuple           # weights + workspace kept alive for the context's lifetime
+    guards: tuple = ()    # (buffer, workspace offset, workspace bytes, guard bytes) for workspace_guards_intact
 
     @property
     def family(self) -> str:
@@ -178,9 +185,11 @@ def mrp_workspace_bytes(cfg: mrp_config) -> int:
 
 
 def mrp_create(d, d_ff, vocab, heads, w_lm, max_rows, max_seqs, block_len, rms_eps=1e-6,
-               flags=0) -> Context:
+               flags=0, guard_bytes=0) -> Context:
     """heads: list of dicts of CUDA tensors gamma [d], w_gate [F,d], w_up [F,d], w_down [d,F];
-    w_lm: CUDA tensor [V,d]; dtype (float32 or bfloat16) is taken from w_lm."""
+    w_lm: CUDA tensor [V,d]; dtype (float32 or bfloat16) is taken from w_lm.  ``guard_bytes``
+    (a multiple of 256) surrounds the workspace with bands of that many 0xA5 bytes, which
+    ``workspace_guards_intact`` checks: a way for tests to see a write outside the workspace."""
     tdtype = w_lm.dtype
     if tdtype not in (torch.float32, torch.bfloat16):
         raise TypeError("weights must be float32 or bfloat16")
@@ -200,15 +209,43 @@ def mrp_create(d, d_ff, vocab, heads, w_lm, max_rows, max_seqs, block_len, rms_e
     nbytes = mrp_workspace_bytes(cfg)
     if nbytes == 0:
         raise MrpError("mrp_workspace_bytes", 1)
-    ws = torch.empty(nbytes + 256, dtype=torch.uint8, device=w_lm.device)
-    off = (-ws.data_ptr()) % 256
+    guard_bytes = (int(guard_bytes) + 255) // 256 * 256
+    ws = torch.full((nbytes + 256 + 2 * guard_bytes,), 0xA5, dtype=torch.uint8, device=w_lm.device)
+    off = (-ws.data_ptr()) % 256 + guard_bytes
     keep.append(ws)
     handle = ctypes.c_void_p()
     rc = lib.mrp_create(ctypes.byref(cfg), harr, _ptr(w_lm), ctypes.c_void_p(ws.data_ptr() + off),
                         ctypes.c_size_t(nbytes), ctypes.byref(handle))
     if rc != 0:
         raise MrpError("mrp_create", rc)
-    return Context(handle.value, cfg, tuple(keep))
+    ctx = Context(handle.value, cfg, tuple(keep))
+    ctx.guards = (ws, off, nbytes, guard_bytes)
+    return ctx
+
+
+def workspace_guards_intact(ctx: Context) -> bool:
+    """True if the bands around the workspace (``guard_bytes`` of mrp_create) still hold their
+    fill pattern; synchronises."""
+    ws, off, nbytes, g = ctx.guards
+    if g == 0:
+        return True
+    before, after = ws[off - g:off], ws[off + nbytes:off + nbytes + g]
+    return bool((before == 0xA5).all().item()) and bool((after == 0xA5).all().item())
+
+
+def mrp_set_input_rows(ctx: Context, n_rows: int) -> None:
+    rc = lib.mrp_set_input_rows(ctx.handle, int(n_rows))
+    if rc != 0:
+        raise MrpError("mrp_set_input_rows", rc)
+
+
+def mrp_fetch_status(ctx: Context, clear: bool = False, stream=None) -> int:
+    """The context's device status word (MRP_DEV_* bits); synchronises to return it as an int."""
+    dst = torch.zeros(1, dtype=torch.int32, device="cuda:%d" % ctx.cfg.device)
+    rc = lib.mrp_fetch_status(ctx.handle, _ptr(dst), int(bool(clear)), _stream(stream))
+    if rc != 0:
+        raise MrpError("mrp_fetch_status", rc)
+    return int(dst.item())
 
 
 def mrp_destroy(ctx: Context) -> None:
@@ -275,19 +312,19 @@ def mrp_draft_from_hidden(ctx: Context, hidden, final_norm_gamma, row_index, M, 
 def mrp_reveal_remask(ctx: Context, conf, token, row_index, M, K, B, L, mode, tau=0.9, r_reveal=1,
                       r_draft=1, use_cap=False, remask_policy=0, ensure_progress=True, *,
                       reveal_mask, remask_mask, out_token, step_of, draft_pos, draft_tok, draft_len,
-                      stream=None) -> None:
+                      status=None, stream=None) -> None:
     _check(conf, torch.float32, "conf")
     _check(token, torch.int32, "token")
     _check(row_index, torch.int32, "row_index")
     for t, dt, nm in ((reveal_mask, torch.int8, "reveal_mask"), (remask_mask, torch.int8, "remask_mask"),
                       (out_token, torch.int32, "out_token"), (step_of, torch.int8, "step_of"),
                       (draft_pos, torch.int32, "draft_pos"), (draft_tok, torch.int32, "draft_tok"),
-                      (draft_len, torch.int32, "draft_len")):
+                      (draft_len, torch.int32, "draft_len"), (status, torch.int32, "status")):
         _check(t, dt, nm)
     p = mrp_select_params(int(mode), float(tau), int(r_reveal), int(r_draft), int(bool(use_cap)),
                           int(remask_policy), int(bool(ensure_progress)))
     o = mrp_select_out(_ptr(reveal_mask), _ptr(remask_mask), _ptr(out_token), _ptr(step_of),
-                       _ptr(draft_pos), _ptr(draft_tok), _ptr(draft_len))
+                       _ptr(draft_pos), _ptr(draft_tok), _ptr(draft_len), _ptr(status))
     rc = lib.mrp_reveal_remask(ctx.handle, _ptr(conf), _ptr(token), _ptr(row_index), int(M), int(K),
                                int(B), int(L), ctypes.byref(p), ctypes.byref(o), _stream(stream))
     if rc != 0:
@@ -297,7 +334,7 @@ def mrp_reveal_remask(ctx: Context, conf, token, row_index, M, K, B, L, mode, ta
 def mrp_reveal_remask_noalloc(conf, token, row_index, M, K, B, L, mode, tau=0.9, r_reveal=1,
                               r_draft=1, use_cap=False, remask_policy=0, ensure_progress=True, *,
                               reveal_mask, remask_mask, out_token, step_of, draft_pos, draft_tok,
-                              draft_len, stream=None) -> None:
+                              draft_len, status=None, stream=None) -> None:
     """Reveal selection for callers that cannot allocate device memory: no context and no
     workspace, the position map lives in a fixed array inside the library (B * L at most
     MRP_NOALLOC_MAX_POSITIONS).  The tensors' device must be the current device.  Calls on
@@ -308,12 +345,12 @@ def mrp_reveal_remask_noalloc(conf, token, row_index, M, K, B, L, mode, tau=0.9,
     for t, dt, nm in ((reveal_mask, torch.int8, "reveal_mask"), (remask_mask, torch.int8, "remask_mask"),
                       (out_token, torch.int32, "out_token"), (step_of, torch.int8, "step_of"),
                       (draft_pos, torch.int32, "draft_pos"), (draft_tok, torch.int32, "draft_tok"),
-                      (draft_len, torch.int32, "draft_len")):
+                      (draft_len, torch.int32, "draft_len"), (status, torch.int32, "status")):
         _check(t, dt, nm)
     p = mrp_select_params(int(mode), float(tau), int(r_reveal), int(r_draft), int(bool(use_cap)),
                           int(remask_policy), int(bool(ensure_progress)))
     o = mrp_select_out(_ptr(reveal_mask), _ptr(remask_mask), _ptr(out_token), _ptr(step_of),
-                       _ptr(draft_pos), _ptr(draft_tok), _ptr(draft_len))
+                       _ptr(draft_pos), _ptr(draft_tok), _ptr(draft_len), _ptr(status))
     rc = lib.mrp_reveal_remask_noalloc(_ptr(conf), _ptr(token), _ptr(row_index), int(M), int(K),
                                        int(B), int(L), ctypes.byref(p), ctypes.byref(o),
                                        _stream(stream))
@@ -346,7 +383,7 @@ def mrp_commit(ctx: Context, B, L, Kd, *, out_token, step_of, draft_pos, draft_t
                       (row_index, torch.int32, "row_index"), (n_masked, torch.int32, "n_masked"),
                       (block_masked, torch.int32, "block_masked")):
         _check(t, dt, nm)
-    sel = mrp_select_out(None, None, _ptr(out_token), _ptr(step_of), _ptr(draft_pos), _ptr(draft_tok), None)
+    sel = mrp_select_out(None, None, _ptr(out_token), _ptr(step_of), _ptr(draft_pos), _ptr(draft_tok), None, None)
     state = mrp_block_state(_ptr(tokens), _ptr(row_index), _ptr(n_masked), _ptr(block_masked))
     rc = lib.mrp_commit(ctx.handle, ctypes.byref(sel), _ptr(accept_mask), int(B), int(L), int(Kd),
                         ctypes.byref(state), _stream(stream))

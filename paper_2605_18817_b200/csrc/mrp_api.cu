@@ -34,7 +34,7 @@ WorkspaceLayout workspace_layout(const mrp_config &cfg)
     l.ssq_fix = take((size_t)5 * 128 * 8);
     l.has_f16 = cfg.dtype == MRP_BF16 && !(cfg.flags & (MRP_FLAG_FORCE_SIMT | MRP_FLAG_EXACT_OPERANDS)) &&
                 ((long long)cfg.n_heads + 1) * cfg.max_rows >= kF16MinRowSteps && cfg.d % 64 == 0 &&
-                cfg.d_ff % 64 == 0 && cfg.vocab % 16 == 0 && cfg.n_heads <= 4;
+                cfg.d_ff % 64 == 0 && cfg.vocab % 16 == 0;
     l.w16 = take(l.has_f16 ? (size_t)cfg.vocab * d * 2 : 0);
     l.xt16 = take(l.has_f16 ? (size_t)steps * rows * d * 2 : 0);
     l.total = off;
@@ -126,6 +126,13 @@ int mrp_create(const mrp_config *cfg, const mrp_head_weights *heads, const void 
     c.sm_count = sm;
     c.use_tc = (cfg->dtype == MRP_BF16) && !(cfg->flags & MRP_FLAG_FORCE_SIMT) &&
                tc_supported(*cfg, c.heads, w_lm);
+    if ((cfg->flags & MRP_FLAG_REQUIRE_TENSOR_CORES) && !c.use_tc) {
+        free(c.heads); delete ctx; return MRP_ERR_UNSUPPORTED;
+    }
+    {
+        const long long dense = (long long)cfg->max_seqs * cfg->block_len;
+        c.input_rows = (int)(dense > cfg->max_rows ? dense : cfg->max_rows);
+    }
     if (c.use_tc) {
         if (tc_create(&c) != cudaSuccess) { free(c.heads); delete ctx; return MRP_ERR_CUDA; }
     }
@@ -211,6 +218,7 @@ static int draft_call(mrp_ctx *ctx, const void *hidden, const float *logits0, bo
     c.launches = 0;
     if (M == 0) return MRP_OK;
     if (!hidden || (!from_hidden && !logits0) || !out->conf || !out->lse || !out->token) return MRP_ERR_INVALID_ARG;
+    if (!row_index && M > c.input_rows) return MRP_ERR_INVALID_ARG;      // rows 0..M-1 must exist
     if (((uintptr_t)hidden & 15u) || ((uintptr_t)logits0 & 15u)) return MRP_ERR_INVALID_ARG;
     DeviceGuard guard(c.cfg.device);
     if (guard.err != cudaSuccess) return MRP_ERR_CUDA;
@@ -278,6 +286,30 @@ int mrp_verify(mrp_ctx *ctx, const int32_t *draft_tok, const int32_t *verify_tok
     cudaError_t e = launch_verify(&c, draft_tok, verify_tok, draft_len, B, Kd, positionwise ? 1 : 0,
                                   accept_len, accept_mask, (cudaStream_t)cuda_stream);
     return e == cudaSuccess ? MRP_OK : MRP_ERR_CUDA;
+}
+
+int mrp_set_input_rows(mrp_ctx *ctx, int32_t n_rows)
+{
+    if (!ctx) return MRP_ERR_INVALID_ARG;
+    const mrp_config &cfg = ctx->c.cfg;
+    const long long dense = (long long)cfg.max_seqs * cfg.block_len;
+    const long long most = dense > cfg.max_rows ? dense : (long long)cfg.max_rows;
+    if (n_rows < 1 || n_rows > most) return MRP_ERR_INVALID_ARG;
+    ctx->c.input_rows = n_rows;
+    return MRP_OK;
+}
+
+int mrp_fetch_status(mrp_ctx *ctx, int32_t *dst, int32_t clear, void *cuda_stream)
+{
+    if (!ctx || !dst) return MRP_ERR_INVALID_ARG;
+    Ctx &c = ctx->c;
+    DeviceGuard guard(c.cfg.device);
+    if (guard.err != cudaSuccess) return MRP_ERR_CUDA;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    int32_t *word = (int32_t *)(c.ws + c.lay.status);
+    if (cudaMemcpyAsync(dst, word, sizeof(int32_t), cudaMemcpyDeviceToDevice, st) != cudaSuccess) return MRP_ERR_CUDA;
+    if (clear && cudaMemsetAsync(word, 0, sizeof(int32_t), st) != cudaSuccess) return MRP_ERR_CUDA;
+    return MRP_OK;
 }
 
 int mrp_set_logits0_event(mrp_ctx *ctx, void *cuda_event)

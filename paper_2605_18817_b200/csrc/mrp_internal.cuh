@@ -63,6 +63,7 @@ struct Ctx {
     bool from_hidden;
     const void *final_gamma;
     cudaEvent_t l0_event;      // mrp_set_logits0_event: awaited right before the LM-head kernel, or nullptr
+    int input_rows;            // rows of the caller's hidden / logits0 arrays: row_index entries must be below
     // Row offset of the bf16 lo block behind the hi block in this call's operand buffers: M and
     // (K+1)M for the row-major kernels, the padded row count for the few-row kernels (which then
     // fetch hi and lo rows of a k-chunk with one TMA box).
@@ -134,12 +135,18 @@ cudaError_t simt_draft(Ctx *c, const void *hidden, const float *logits0, const i
 // fp32 from the bf16 hi + lo rows, which removes the dominant token's rounding error from
 // log-sum-exp and confidence.  w == nullptr: off.
 struct TopFix {
-    const __nv_bfloat16 *w;      // [V, d]
-    const __nv_bfloat16 *xt;     // [2 * n_rs, d]: hi rows then lo rows, row-step major
+    const __nv_bfloat16 *w;      // [V, d]; nullptr: no recomputation
+    const __nv_bfloat16 *xt;     // hi rows [n_rs, d] of the stacked LM-head operand, row-step major, then (from
+                                 // row n_rs on, only read when w is set) the lo rows; nullptr: nothing to check
     const float *logits0;
     const int32_t *row_index;
     int d, V, M, n_rs;
+    int n_rows_in;               // row_index entries at or above are invalid (their l_0 reads as zero)
+    float range_limit;           // > 0: raise MRP_DEV_RANGE for a row-step whose operand has d * rms above it
 };
+
+// A caller-provided row index is used as an address only if it lies inside the caller's array.
+__device__ __forceinline__ bool row_ok(int idx, int n_rows_in) { return (unsigned)idx < (unsigned)n_rows_in; }
 
 // Shared by both families: merge per-slice partials into conf/lse/token/margin.
 cudaError_t launch_combine(Ctx *c, const Partial *partials, int n_slices, int n_rowsteps,
@@ -148,7 +155,7 @@ cudaError_t launch_combine(Ctx *c, const Partial *partials, int n_slices, int n_
 // CUDA-core family: gather masked rows of `hidden` into fp32 h0f / hcur (xt0: where the step-0
 // operand rows n_0 go when the base logits are computed in the LM-head pass, else nullptr).
 cudaError_t launch_prep(Ctx *c, const void *hidden, const int32_t *row_index, int M,
-                        cudaStream_t st, float *xt0);
+                        cudaStream_t st, float *xt0, int32_t *user_status);
 
 // ---- selection / verification (select_verify.cu) ------------------------------------
 cudaError_t launch_commit(Ctx *c, const mrp_select_out &sel, const int8_t *accept_mask, int B, int L, int Kd,

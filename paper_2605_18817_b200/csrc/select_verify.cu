@@ -1,12 +1,13 @@
 // Reveal selection, remasking and draft verification: one warp per (sequence, block).
 //
-// STATIC   (Algorithm 2 "Reveal r tokens with highest confidence"; Algorithm 3 "Draft token
-//           with highest confidence"): for k = 0..K the r most confident still-masked
+// STATIC   (Algorithm 2, reveal step at k = 0..K; Algorithm 3, draft step after each MRP
+//           update): for k = 0..K the r most confident still-masked
 //           positions under step k, confidence descending then position ascending.
 // DYNAMIC  (Algorithm 4; Sec. 4.1 dynamic denoising; Sec. 4.4 cap): R = {conf_0 >= tau},
 //           at least one, optionally capped; remask members of R whose updated confidence
 //           is below the same tau.
-// VERIFY   (Algorithm 3 "Reject drafted positions where argmax differ"; Figure 1(d)).
+// VERIFY   (Algorithm 3, rejection step: a draft that differs from the backbone's argmax is
+//           rejected; Figure 1(d): prefix acceptance).
 // Lane l owns block positions l, l+32, ... (up to 32 strides, i.e. L <= 1024); membership
 // sets are per-lane bit masks over the strides.
 #include <limits.h>
@@ -17,11 +18,24 @@
 
 namespace mrp {
 
-__global__ void scatter_rows_kernel(const int32_t *__restrict__ row_index, int M,
-                                    int32_t *__restrict__ dense_row)
+__device__ __forceinline__ void raise_bad_index(int32_t *status, int32_t *user_status)
+{
+    if (status) atomicOr(status, MRP_DEV_BAD_INDEX);
+    if (user_status) atomicOr(user_status, MRP_DEV_BAD_INDEX);
+}
+
+// dense_row[position] = masked row, over n_pos = B * L positions preset to -1.  A row whose
+// position is outside [0, n_pos) is skipped; of several rows naming one position the one listed
+// last (highest m) keeps it, whatever the order the threads run in.  Both raise MRP_DEV_BAD_INDEX.
+__global__ void scatter_rows_kernel(const int32_t *__restrict__ row_index, int M, int n_pos,
+                                    int32_t *__restrict__ dense_row, int32_t *__restrict__ status,
+                                    int32_t *__restrict__ user_status)
 {
     const int m = blockIdx.x * blockDim.x + threadIdx.x;
-    if (m < M) dense_row[row_index ? row_index[m] : m] = m;
+    if (m >= M) return;
+    const int idx = row_index ? row_index[m] : m;
+    if (!row_ok(idx, n_pos)) { raise_bad_index(status, user_status); return; }
+    if (atomicMax(dense_row + idx, m) != -1) raise_bad_index(status, user_status);
 }
 
 // Most confident position among the lanes' candidate bit sets under confidences c[row]:
@@ -58,7 +72,7 @@ __device__ __forceinline__ int warp_popc(uint32_t bits)
 __global__ void __launch_bounds__(32)
 select_kernel(const float *__restrict__ conf, const int32_t *__restrict__ token,
               const int32_t *__restrict__ dense_row, int M, int K, int L, mrp_select_params p,
-              mrp_select_out out, int Kd, const int32_t *__restrict__ row_index)
+              mrp_select_out out, int Kd, const int32_t *__restrict__ row_index, int32_t *__restrict__ status)
 {
     pdl_trigger();
     pdl_wait();
@@ -72,10 +86,16 @@ select_kernel(const float *__restrict__ conf, const int32_t *__restrict__ token,
     } else {
         for (int i = lane; i < L; i += 32) rows_s[i] = -1;
         __syncwarp();
-        const long long lo = (long long)b * L;
+        // rows of other blocks are skipped, and with them any index outside [0, B * L) (block 0
+        // reports those); of several rows naming one position the one listed last keeps it
+        const long long lo = (long long)b * L, n_pos = (long long)gridDim.x * L;
         for (int m = lane; m < M; m += 32) {
             const long long idx = row_index ? row_index[m] : m;
-            if (idx >= lo && idx < lo + L) rows_s[idx - lo] = m;
+            if (idx >= lo && idx < lo + L) {
+                if (atomicMax(&rows_s[idx - lo], m) != -1) raise_bad_index(status, out.status);
+            } else if (b == 0 && (idx < 0 || idx >= n_pos)) {
+                raise_bad_index(status, out.status);
+            }
         }
         __syncwarp();
     }
@@ -203,20 +223,21 @@ cudaError_t launch_select(Ctx *c, const float *conf, const int32_t *token, const
                           const mrp_select_out &out, cudaStream_t st)
 {
     const int Kd = K * (p.r_draft > 0 ? p.r_draft : 0);
+    int32_t *status = (int32_t *)(c->ws + c->lay.status);
     if ((long long)B * M <= (1ll << 22)) {
         // few rows: every block finds its rows itself, one launch instead of three
         c->launches++;
         return launch_k(select_kernel, dim3(B), dim3(32), 0, st, !(c->cfg.flags & MRP_FLAG_NO_PDL), conf, token,
-                        (const int32_t *)nullptr, M, K, L, p, out, Kd, row_index);
+                        (const int32_t *)nullptr, M, K, L, p, out, Kd, row_index, status);
     }
     int32_t *dense_row = (int32_t *)(c->ws + c->lay.dense_row);
     cudaError_t e = cudaMemsetAsync(dense_row, 0xFF, sizeof(int32_t) * (size_t)B * L, st);
     if (e != cudaSuccess) return e;
     if (M > 0) {
-        scatter_rows_kernel<<<(M + 255) / 256, 256, 0, st>>>(row_index, M, dense_row);
+        scatter_rows_kernel<<<(M + 255) / 256, 256, 0, st>>>(row_index, M, B * L, dense_row, status, out.status);
         c->launches++;
     }
-    select_kernel<<<B, 32, 0, st>>>(conf, token, dense_row, M, K, L, p, out, Kd, nullptr);
+    select_kernel<<<B, 32, 0, st>>>(conf, token, dense_row, M, K, L, p, out, Kd, nullptr, status);
     c->launches++;
     return cudaGetLastError();
 }
@@ -346,11 +367,36 @@ cudaError_t launch_commit(Ctx *c, const mrp_select_out &sel, const int8_t *accep
 static __device__ __align__(256) int32_t mrp_noalloc_dense_row[MRP_NOALLOC_MAX_POSITIONS];
 
 namespace {
-constexpr int kNoAllocMaxDevices = 64;
-// Device address of mrp_noalloc_dense_row on each device, resolved on first use.  In host
-// code the array's name is only a handle for the runtime, never a device address.
-int32_t *g_noalloc_ptr[kNoAllocMaxDevices];
+// Device address of mrp_noalloc_dense_row, resolved on first use and remembered per (device,
+// CUDA context): a module variable has one address per context, so a second context on the
+// same device must not be handed the first one's pointer.  In host code the array's name is only
+// a handle for the runtime, never a device address.
+constexpr int kNoAllocSlots = 64;
+struct NoAllocSlot { int dev; void *cuctx; int32_t *ptr; };
+NoAllocSlot g_noalloc[kNoAllocSlots];
+int g_noalloc_n = 0;
 std::mutex g_noalloc_mu;
+
+typedef int (*CtxGetCurrentFn)(void **);   // CUresult cuCtxGetCurrent(CUcontext *)
+
+// The CUDA context current to this thread (nullptr if the driver entry point is not available:
+// every call then resolves the address anew).
+void *current_cuda_context()
+{
+    static CtxGetCurrentFn fn = nullptr;
+    static bool looked = false;
+    if (!looked) {
+        void *f = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuCtxGetCurrent", &f, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = (CtxGetCurrentFn)f;
+        looked = true;
+    }
+    void *cur = nullptr;
+    if (!fn || fn(&cur) != 0) return nullptr;
+    return cur;
+}
 }  // namespace
 
 extern "C" int mrp_reveal_remask_noalloc(const float *conf, const int32_t *token,
@@ -375,23 +421,29 @@ extern "C" int mrp_reveal_remask_noalloc(const float *conf, const int32_t *token
 
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess) return MRP_ERR_CUDA;
-    if (dev < 0 || dev >= kNoAllocMaxDevices) return MRP_ERR_UNSUPPORTED;
     int32_t *dense_row = nullptr;
     {
         std::lock_guard<std::mutex> lock(g_noalloc_mu);
-        if (!g_noalloc_ptr[dev]) {
-            // once per device, with that device current
+        void *cuctx = current_cuda_context();      // nullptr before the thread has a context: resolve, do not remember
+        for (int i = 0; i < g_noalloc_n && cuctx; ++i)
+            if (g_noalloc[i].dev == dev && g_noalloc[i].cuctx == cuctx) dense_row = g_noalloc[i].ptr;
+        if (!dense_row) {
+            // once per (device, context), with that device current
             void *p = nullptr;
             if (cudaGetSymbolAddress(&p, mrp_noalloc_dense_row) != cudaSuccess || !p) return MRP_ERR_CUDA;
-            g_noalloc_ptr[dev] = (int32_t *)p;
+            dense_row = (int32_t *)p;
+            if (cuctx && g_noalloc_n < kNoAllocSlots) g_noalloc[g_noalloc_n++] = NoAllocSlot{dev, cuctx, dense_row};
         }
-        dense_row = g_noalloc_ptr[dev];
     }
     cudaStream_t st = (cudaStream_t)cuda_stream;
     // the array still holds the previous call's map: every position of this call starts at -1
     if (cudaMemsetAsync(dense_row, 0xFF, sizeof(int32_t) * (size_t)B * L, st) != cudaSuccess)
         return MRP_ERR_CUDA;
-    if (M > 0) scatter_rows_kernel<<<(M + 255) / 256, 256, 0, st>>>(row_index, M, dense_row);
-    select_kernel<<<B, 32, 0, st>>>(conf, token, dense_row, M, K, L, *params, *out, Kd, nullptr);
+    // rows whose position is outside [0, B * L) are skipped: nothing is written outside the part
+    // of the array this call has just reset
+    if (M > 0)
+        scatter_rows_kernel<<<(M + 255) / 256, 256, 0, st>>>(row_index, M, B * L, dense_row, (int32_t *)nullptr,
+                                                              out->status);
+    select_kernel<<<B, 32, 0, st>>>(conf, token, dense_row, M, K, L, *params, *out, Kd, nullptr, (int32_t *)nullptr);
     return cudaGetLastError() == cudaSuccess ? MRP_OK : MRP_ERR_CUDA;
 }

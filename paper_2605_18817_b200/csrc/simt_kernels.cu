@@ -28,16 +28,24 @@ __device__ __forceinline__ float warp_sum(float v)
 template <typename T>
 __global__ void prep_kernel(const T *__restrict__ hidden, const int32_t *__restrict__ row_index,
                             int d, float *__restrict__ h0f, float *__restrict__ hcur, float *__restrict__ xt0,
-                            const T *__restrict__ final_gamma, float eps)
+                            const T *__restrict__ final_gamma, float eps, int n_rows_in,
+                            int32_t *__restrict__ status, int32_t *__restrict__ user_status)
 {
     pdl_trigger();
     pdl_wait();
     __shared__ float red[32];
     const int m = blockIdx.x;
-    const size_t row = row_index ? (size_t)row_index[m] : (size_t)m;
+    const int idx = row_index ? row_index[m] : m;
+    // an index outside the caller's array is never used as an address: the row reads as zeros
+    const bool bad = row_index && !row_ok(idx, n_rows_in);
+    if (bad && threadIdx.x == 0) {
+        atomicOr(status, MRP_DEV_BAD_INDEX);
+        if (user_status) atomicOr(user_status, MRP_DEV_BAD_INDEX);
+    }
+    const size_t row = bad ? 0 : (size_t)idx;
     float ss = 0.f;
     for (int j = threadIdx.x; j < d; j += blockDim.x) {
-        const float v = ld_f(hidden, row * d + j);
+        const float v = bad ? 0.f : ld_f(hidden, row * d + j);
         if (!xt0) h0f[(size_t)m * d + j] = v;
         hcur[(size_t)m * d + j] = v;
         ss = fmaf(v, v, ss);
@@ -52,25 +60,28 @@ __global__ void prep_kernel(const T *__restrict__ hidden, const int32_t *__restr
     for (int i = 0; i < (int)(blockDim.x >> 5); ++i) t += red[i];
     const float rstd0 = final_gamma ? rsqrtf(t / (float)d + eps) : 1.f;
     for (int j = threadIdx.x; j < d; j += blockDim.x) {
-        const float v = ld_f(hidden, row * d + j);
+        const float v = bad ? 0.f : ld_f(hidden, row * d + j);
         const float n0 = final_gamma ? v * rstd0 * ld_f(final_gamma, j) : v;
         h0f[(size_t)m * d + j] = v - n0;
         xt0[(size_t)m * d + j] = n0;
     }
 }
 
-cudaError_t launch_prep(Ctx *c, const void *hidden, const int32_t *row_index, int M, cudaStream_t st, float *xt0)
+cudaError_t launch_prep(Ctx *c, const void *hidden, const int32_t *row_index, int M, cudaStream_t st, float *xt0,
+                        int32_t *user_status)
 {
     if (M == 0) return cudaSuccess;
     float *h0f = (float *)(c->ws + c->lay.h0f), *hcur = (float *)(c->ws + c->lay.hcur);
+    int32_t *status = (int32_t *)(c->ws + c->lay.status);
     const bool pdl = !(c->cfg.flags & MRP_FLAG_NO_PDL);
     cudaError_t e;
     if (c->cfg.dtype == MRP_F32)
         e = launch_k(prep_kernel<float>, dim3(M), dim3(256), 0, st, pdl, (const float *)hidden, row_index, c->cfg.d, h0f, hcur,
-                     xt0, (const float *)c->final_gamma, c->cfg.rms_eps);
+                     xt0, (const float *)c->final_gamma, c->cfg.rms_eps, c->input_rows, status, user_status);
     else
         e = launch_k(prep_kernel<__nv_bfloat16>, dim3(M), dim3(256), 0, st, pdl, (const __nv_bfloat16 *)hidden, row_index,
-                     c->cfg.d, h0f, hcur, xt0, (const __nv_bfloat16 *)c->final_gamma, c->cfg.rms_eps);
+                     c->cfg.d, h0f, hcur, xt0, (const __nv_bfloat16 *)c->final_gamma, c->cfg.rms_eps, c->input_rows,
+                     status, user_status);
     c->launches++;
     return e;
 }
@@ -186,7 +197,7 @@ __global__ void __launch_bounds__(256)
 lm_simt_kernel(const T *__restrict__ w_lm, const float *__restrict__ xt, const float *__restrict__ xt0,
                const float *__restrict__ logits0, const int32_t *__restrict__ row_index, int M,
                int K, int d, int V, int n_slices, Partial *__restrict__ partials,
-               float *__restrict__ logits_out)
+               float *__restrict__ logits_out, int n_rows_in)
 {
     pdl_trigger();
     pdl_wait();
@@ -226,8 +237,9 @@ lm_simt_kernel(const T *__restrict__ w_lm, const float *__restrict__ xt, const f
                         float l = -INFINITY;
                         if (v < V && rs < n_rs) {
                             const int m = rs % M;
-                            const size_t row = row_index ? (size_t)row_index[m] : (size_t)m;
-                            l = (logits0 ? logits0[row * (size_t)V + v] : 0.f) + s;
+                            const int idx = row_index ? row_index[m] : m;
+                            const bool have = logits0 && (!row_index || row_ok(idx, n_rows_in));
+                            l = (have ? logits0[(size_t)idx * (size_t)V + v] : 0.f) + s;
                         }
                         tile[r][vl] = l;
                     }
@@ -313,12 +325,15 @@ __global__ void combine_kernel(const Partial *__restrict__ partials, int n_slice
         p = (lane & o) ? merge_partial(q, p) : merge_partial(p, q);
     }
     float top = p.mx;      // the top logit as the sum of exponentials saw it
-    if (fix.w && (rs >= fix.M || !fix.logits0)) {
+    const bool has_operand = fix.xt && (rs >= fix.M || !fix.logits0);   // step 0 of mrp_draft has none
+    float ssq = 0.f;       // sum of squares of the row-step's LM-head operand (hi part)
+    if (fix.w && has_operand) {
         // exact top logit: l_0[row, tok] + W[tok] . (hi + lo), fp32, fixed summation order
         // (no l_0 term, and step 0 included, when the base logits are computed in the pass)
         const int tok = __shfl_sync(0xffffffffu, p.idx, 0);
         const int m = rs % fix.M;
-        const size_t row = fix.row_index ? (size_t)fix.row_index[m] : (size_t)m;
+        const int idx = fix.row_index ? fix.row_index[m] : m;
+        const bool have = fix.logits0 && (!fix.row_index || row_ok(idx, fix.n_rows_in));
         const __nv_bfloat16 *wr = fix.w + (size_t)tok * fix.d;
         const __nv_bfloat16 *xh = fix.xt + (size_t)rs * fix.d, *xl = xh + (size_t)fix.n_rs * fix.d;
         float dot = 0.f;
@@ -329,9 +344,31 @@ __global__ void combine_kernel(const Partial *__restrict__ partials, int n_slice
             const float2 l2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(xl + j));
             dot = fmaf(w2.x, h2.x + l2.x, dot);
             dot = fmaf(w2.y, h2.y + l2.y, dot);
+            ssq = fmaf(h2.x, h2.x, fmaf(h2.y, h2.y, ssq));
         }
         dot = warp_sum(dot);
-        top = (fix.logits0 ? fix.logits0[row * (size_t)fix.V + tok] : 0.f) + dot;
+        top = (have ? fix.logits0[(size_t)idx * (size_t)fix.V + tok] : 0.f) + dot;
+    } else if (fix.range_limit > 0.f && has_operand) {
+        // only the size of the operand row is needed: 16-byte loads of its hi part (d % 64 == 0)
+        const uint4 *xh = reinterpret_cast<const uint4 *>(fix.xt + (size_t)rs * fix.d);
+#pragma unroll 4
+        for (int j = lane; j < fix.d / 8; j += 32) {
+            const uint4 q = xh[j];
+            const uint32_t w4[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float2 h2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&w4[i]));
+                ssq = fmaf(h2.x, h2.x, fmaf(h2.y, h2.y, ssq));
+            }
+        }
+    }
+    if (fix.range_limit > 0.f && has_operand) {
+        // accuracy range of the tensor-core path: d * rms(operand row) = sqrt(d * sum of squares)
+        ssq = warp_sum(ssq);
+        if (lane == 0 && sqrtf(ssq * (float)fix.d) > fix.range_limit) {
+            atomicOr(status, MRP_DEV_RANGE);
+            if (user_status) atomicOr(user_status, MRP_DEV_RANGE);
+        }
     }
     if (lane == 0) {
         // the term of the top token entered the sum as exp(0) = 1: swap in its exact value
@@ -377,7 +414,7 @@ static cudaError_t simt_draft_t(Ctx *c, const void *hidden, const float *logits0
     prof_mark(c, 0, st);
     // without base logits the operand rows of step 0 (n_0) follow those of steps 1..K
     float *xt0 = c->from_hidden ? xt + (size_t)K * M * d : nullptr;
-    cudaError_t e = launch_prep(c, hidden, row_index, M, st, xt0);
+    cudaError_t e = launch_prep(c, hidden, row_index, M, st, xt0, out.status);
     if (e != cudaSuccess) return e;
     if (K == 0 && out.hidden_out)
         cudaMemcpyAsync(out.hidden_out, hcur, sizeof(float) * (size_t)M * d, cudaMemcpyDeviceToDevice, st);
@@ -405,11 +442,12 @@ static cudaError_t simt_draft_t(Ctx *c, const void *hidden, const float *logits0
     const int grid = n_slices < kSimtMaxBlocks ? n_slices : kSimtMaxBlocks;
     if (narrow)
         e = launch_k(lm_simt_kernel<T, 32>, dim3(grid), dim3(256), 0, st, pdl, (const T *)c->w_lm, (const float *)xt,
-                     (const float *)xt0, logits0, row_index, M, K, d, V, n_slices, partials, out.logits_out);
+                     (const float *)xt0, logits0, row_index, M, K, d, V, n_slices, partials, out.logits_out,
+                     c->input_rows);
     else
         e = launch_k(lm_simt_kernel<T, kSimtSliceV>, dim3(grid), dim3(256), 0, st, pdl, (const T *)c->w_lm,
                      (const float *)xt, (const float *)xt0, logits0, row_index, M, K, d, V, n_slices, partials,
-                     out.logits_out);
+                     out.logits_out, c->input_rows);
     c->launches++;
     if (e != cudaSuccess) return e;
     prof_mark(c, 2, st);

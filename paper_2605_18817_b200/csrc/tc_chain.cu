@@ -595,12 +595,15 @@ sk_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant__ 
     }
 }
 
+// Sets the kernel's shared-memory limit (once per device: the attribute is per device) and asks
+// whether `grid` CTAs of it can be resident together, which the phase barriers need: on a
+// context that may use only part of the SMs (MPS with a thread percentage, a partitioned
+// device) they cannot, and the caller then runs the chain as one kernel per GEMM.
 template <int RP, int KC>
-cudaError_t chain_launch(const ChainMaps &maps, const ChainParams &p, int grid, size_t smem, cudaStream_t st)
+cudaError_t chain_prepare(int grid, size_t smem, int sm_count, bool *fits)
 {
     auto kern = sk_chain_kernel<RP, KC>;
-    // the shared-memory limit of a kernel is set once per device (the attribute is per device)
-    static std::atomic<unsigned long long> attr_devices{0};
+    static std::atomic<unsigned long long> attr_devices{0}, fit_devices{0}, nofit_devices{0};
     int dev = 0;
     cudaError_t ea = cudaGetDevice(&dev);
     if (ea != cudaSuccess) return ea;
@@ -610,6 +613,20 @@ cudaError_t chain_launch(const ChainMaps &maps, const ChainParams &p, int grid, 
         if (ea != cudaSuccess) return ea;
         attr_devices.fetch_or(bit);
     }
+    if (!((fit_devices.load() | nofit_devices.load()) & bit)) {
+        int per_sm = 0;
+        ea = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kChThreads, smem);
+        if (ea != cudaSuccess) return ea;
+        ((long long)per_sm * sm_count >= grid ? fit_devices : nofit_devices).fetch_or(bit);
+    }
+    if (fits) *fits = (fit_devices.load() & bit) != 0;
+    return cudaSuccess;
+}
+
+template <int RP, int KC>
+cudaError_t chain_launch(const ChainMaps &maps, const ChainParams &p, int grid, size_t smem, cudaStream_t st)
+{
+    auto kern = sk_chain_kernel<RP, KC>;
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));
     cfg.gridDim = dim3(grid);
@@ -656,6 +673,33 @@ cudaError_t sk_chain(Ctx *c, int M, int K, const mrp_draft_out &out, cudaStream_
         S = (F / kBK + cps - 1) / cps;
         if (M * ((128 + S - 1) / S) > kChMaxShare) return cudaErrorNotSupported;
     }
+    auto split = [&](int n_tiles, int k_chunks) {
+        int S = G / n_tiles;
+        if (S < 1) S = 1;
+        if (S > k_chunks) S = k_chunks;
+        const int cps = (k_chunks + S - 1) / S;
+        return (k_chunks + cps - 1) / cps;          // no empty slice
+    };
+    const int gu_split = split(gu_tiles, d / kBK), dn_split = split(dn_tiles, F / kBK);
+    // two k-chunks per ring stage where every slice of both GEMMs has an even number of them
+    const bool even = (d / kBK) % (2 * gu_split) == 0 && (F / kBK) % (2 * dn_split) == 0;
+    const int kc = (even && r_pad <= 32) ? 2 : 1;
+    const int stage = kc * (kChWTile + 2 * r_pad * 128);
+    int ns = (kSmemBudget - 1024 - 256 - 16 - kChAuxBytes) / stage;
+    if (ns > 12) ns = 12;
+    const size_t smem = (size_t)ns * stage + 1024 + 8 * (2 * ns + 4) + 16 + kChAuxBytes;
+    {
+        // all G CTAs must be resident at once (they wait for one another)
+        bool fits = false;
+        cudaError_t eq;
+        switch (r_pad) {
+        case 16: eq = kc == 2 ? chain_prepare<16, 2>(G, smem, G, &fits) : chain_prepare<16, 1>(G, smem, G, &fits); break;
+        case 32: eq = kc == 2 ? chain_prepare<32, 2>(G, smem, G, &fits) : chain_prepare<32, 1>(G, smem, G, &fits); break;
+        case 64: eq = chain_prepare<64, 1>(G, smem, G, &fits); break;
+        default: eq = chain_prepare<128, 1>(G, smem, G, &fits); break;
+        }
+        if (eq != cudaSuccess || !fits) return cudaErrorNotSupported;
+    }
     if (check_only) return cudaSuccess;
 
     ChainParams p;
@@ -672,25 +716,10 @@ cudaError_t sk_chain(Ctx *c, int M, int K, const mrp_draft_out &out, cudaStream_
     p.counters = (int32_t *)(c->ws + c->lay.sk_counters);
     p.grid_bar = (unsigned int *)(c->ws + c->lay.sk_counters) + (kSkMaxTiles - 1);
     p.status = (int32_t *)(c->ws + c->lay.status); p.user_status = out.status;
-    auto split = [&](int n_tiles, int k_chunks) {
-        int S = G / n_tiles;
-        if (S < 1) S = 1;
-        if (S > k_chunks) S = k_chunks;
-        const int cps = (k_chunks + S - 1) / S;
-        return (k_chunks + cps - 1) / cps;          // no empty slice
-    };
-    const int gu_split = split(gu_tiles, d / kBK), dn_split = split(dn_tiles, F / kBK);
-    // two k-chunks per ring stage where every slice of both GEMMs has an even number of them
-    const bool even = (d / kBK) % (2 * gu_split) == 0 && (F / kBK) % (2 * dn_split) == 0;
-    const int kc = (even && r_pad <= 32) ? 2 : 1;
-    const int stage = kc * (kChWTile + 2 * r_pad * 128);
-    int ns = (kSmemBudget - 1024 - 256 - 16 - kChAuxBytes) / stage;
-    if (ns > 12) ns = 12;
     p.n_stages = ns;
     int cols = 32;
     while (cols < 2 * 2 * r_pad) cols <<= 1;
     p.tmem_cols = cols;
-    const size_t smem = (size_t)ns * stage + 1024 + 8 * (2 * ns + 4) + 16 + kChAuxBytes;
 
     __nv_bfloat16 *xg = (__nv_bfloat16 *)(c->ws + c->lay.xg);
     __nv_bfloat16 *xt = (__nv_bfloat16 *)(c->ws + c->lay.xt);

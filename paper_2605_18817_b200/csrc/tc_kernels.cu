@@ -58,6 +58,7 @@ struct TcParams {
     // LM
     const float *logits0;
     const int32_t *row_index;
+    int n_rows_in;       // row_index entries at or above are invalid: their base logits read as zero
     Partial *partials;
     float *logits_out;
     // GU
@@ -136,29 +137,49 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     if (warp == 0) {
         // ---------------- TMA producer ----------------
         if (lane == 0) {
-            pdl_wait();
             const uint32_t tx = (uint32_t)(PARTS * kATile + p.bn * 128);
             const int box_rows = p.bn / p.n_boxes;
+            // the CTA's work as one sequence of ring steps: row blocks mb = grp, grp + n_groups, ...,
+            // for each its n_t weight tiles, for each tile the k-chunks
+            auto advance = [&](int &mb_, int &t_, int &kk_) {
+                if (++kk_ == p.k_chunks) { kk_ = 0; if (++t_ == n_t) { t_ = 0; mb_ += p.n_groups; } }
+            };
+            auto load_b = [&](int t_, int kk_, int s_) {
+                const int n0 = (u0 + t_ * p.w_units) * p.unit_rows;
+                const uint32_t sb = base + (uint32_t)s_ * stage_bytes + PARTS * kATile;
+                tma_load_2d(sb, &tmB0, kk_ * kBK, n0, full_bar(s_));
+                if (KIND == KIND_GU) tma_load_2d(sb + box_rows * 128, &tmB1, kk_ * kBK, n0, full_bar(s_));
+            };
+            auto load_a = [&](int mb_, int kk_, int s_) {
+                const uint32_t sa = base + (uint32_t)s_ * stage_bytes;
+                tma_load_2d(sa, &tmA, kk_ * kBK, p.a_row_base + mb_ * 128, full_bar(s_));
+                if (!F16) tma_load_2d(sa + kATile, &tmA, kk_ * kBK, p.a_part_rows + p.a_row_base + mb_ * 128, full_bar(s_));
+            };
+            const int my_blocks = grp < p.n_rb ? (p.n_rb - 1 - grp) / p.n_groups + 1 : 0;
+            const long long total_it = (long long)my_blocks * n_t * p.k_chunks;
+            const int pre = (int)(total_it < p.n_stages ? total_it : p.n_stages);
+            // the weight tiles depend on nothing: the ring is filled with them while the previous
+            // kernel of the stream drains; only the activation tiles wait for it
+            int mb = grp, t = 0, kk = 0;
+            for (int it = 0; it < pre; ++it) {
+                mbar_expect_tx(full_bar(it), tx);
+                load_b(t, kk, it);
+                advance(mb, t, kk);
+            }
+            pdl_wait();
+            {
+                int mb2 = grp, t2 = 0, kk2 = 0;
+                for (int it = 0; it < pre; ++it) { load_a(mb2, kk2, it); advance(mb2, t2, kk2); }
+            }
             int s = 0;
-            uint32_t ph = 0;
-            bool ok = true;
-            for (int mb = grp; mb < p.n_rb && ok; mb += p.n_groups) {
-                for (int t = 0; t < n_t && ok; ++t) {
-                    const int n0 = (u0 + t * p.w_units) * p.unit_rows;
-                    for (int kk = 0; kk < p.k_chunks; ++kk) {
-                        if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p)) { ok = false; break; }
-                        mbar_expect_tx(full_bar(s), tx);
-                        const uint32_t sa = base + (uint32_t)s * stage_bytes;
-                        tma_load_2d(sa, &tmA, kk * kBK, p.a_row_base + mb * 128, full_bar(s));
-                        if (!F16)
-                            tma_load_2d(sa + kATile, &tmA, kk * kBK, p.a_part_rows + p.a_row_base + mb * 128, full_bar(s));
-                        const uint32_t sb = sa + PARTS * kATile;
-                        tma_load_2d(sb, &tmB0, kk * kBK, n0, full_bar(s));
-                        if (KIND == KIND_GU)
-                            tma_load_2d(sb + box_rows * 128, &tmB1, kk * kBK, n0, full_bar(s));
-                        if (++s == p.n_stages) { s = 0; ph ^= 1u; }
-                    }
-                }
+            uint32_t ph = 1;              // the ring has been filled once
+            for (long long it = pre; it < total_it; ++it) {
+                if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p)) break;
+                mbar_expect_tx(full_bar(s), tx);
+                load_a(mb, kk, s);
+                load_b(t, kk, s);
+                advance(mb, t, kk);
+                if (++s == p.n_stages) { s = 0; ph ^= 1u; }
             }
         }
     } else if (warp == 1) {
@@ -227,8 +248,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     k_of_row = r / p.M + p.step_base;
                     m_of_row = r - (k_of_row - p.step_base) * p.M;
                     first_step = (k_of_row == 1 && p.step_base == 1);
-                    const size_t row = p.row_index ? (size_t)p.row_index[m_of_row] : (size_t)m_of_row;
-                    if (p.logits0) l0p = p.logits0 + row * (size_t)p.V;
+                    const int idx = p.row_index ? p.row_index[m_of_row] : m_of_row;
+                    if (p.logits0 && (!p.row_index || row_ok(idx, p.n_rows_in)))
+                        l0p = p.logits0 + (size_t)idx * (size_t)p.V;
                 }
             } else if (KIND == KIND_GU && valid) {
                 float s = 0.f;
@@ -247,10 +269,17 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     for (int c = 0; c < units_here; ++c) {
                         const int v = v_tile + c * 16;
                         float l0[16], a[16];
-                        if (valid && l0p) load16(l0p + v, l0);
+                        if (valid && p.logits0) {
+                            if (l0p) {
+                                load16(l0p + v, l0);
+                            } else {          // the caller's row index was out of range: an all-zero logit row
+#pragma unroll
+                                for (int j = 0; j < 16; ++j) l0[j] = 0.f;
+                            }
+                        }
                         tmem_ld16(tacc + c * 16, a);
                         if (valid) {
-                            if (l0p) {
+                            if (p.logits0) {
                                 if (first_step) st0.template update<MARGIN>(l0, v);
 #pragma unroll
                                 for (int j = 0; j < 16; ++j) a[j] += l0[j];
@@ -356,7 +385,8 @@ __global__ void tc_prep_kernel(const __nv_bfloat16 *__restrict__ hidden, const i
                                __nv_bfloat16 *__restrict__ xt0, float *__restrict__ sumsq,
                                int32_t *__restrict__ counters, int n_counters,
                                unsigned long long *__restrict__ ssq_fix, int from_hidden,
-                               const __nv_bfloat16 *__restrict__ final_gamma, float eps, __half *__restrict__ xt16_0)
+                               const __nv_bfloat16 *__restrict__ final_gamma, float eps, __half *__restrict__ xt16_0,
+                               int n_rows_in, int32_t *__restrict__ status, int32_t *__restrict__ user_status)
 {
     pdl_trigger();
     pdl_wait();
@@ -366,10 +396,17 @@ __global__ void tc_prep_kernel(const __nv_bfloat16 *__restrict__ hidden, const i
     __shared__ float red[8];
     __shared__ float total_s;
     const int m = blockIdx.x;
-    const size_t row = row_index ? (size_t)row_index[m] : (size_t)m;
+    const int idx = row_index ? row_index[m] : m;
+    // an index outside the caller's array is never used as an address: the row reads as zeros
+    const bool bad = row_index && !row_ok(idx, n_rows_in);
+    if (bad && threadIdx.x == 0) {
+        atomicOr(status, MRP_DEV_BAD_INDEX);
+        if (user_status) atomicOr(user_status, MRP_DEV_BAD_INDEX);
+    }
+    const size_t row = bad ? 0 : (size_t)idx;
     float ss = 0.f;
     for (int j = threadIdx.x; j < d; j += blockDim.x) {
-        const float v = __bfloat162float(hidden[row * d + j]);
+        const float v = bad ? 0.f : __bfloat162float(hidden[row * d + j]);
         const size_t o = (size_t)m * d + j;
         if (!from_hidden) h0f[o] = v;
         hcur[o] = v;
@@ -404,7 +441,7 @@ __global__ void tc_prep_kernel(const __nv_bfloat16 *__restrict__ hidden, const i
         __syncthreads();
         const float rstd0 = final_gamma ? rsqrtf(total_s / (float)d + eps) : 1.f;
         for (int j = threadIdx.x; j < d; j += blockDim.x) {
-            const float v = __bfloat162float(hidden[row * d + j]);
+            const float v = bad ? 0.f : __bfloat162float(hidden[row * d + j]);
             const float n0 = final_gamma ? v * rstd0 * __bfloat162float(final_gamma[j]) : v;
             const size_t o = (size_t)m * d + j;
             h0f[o] = v - n0;
@@ -533,7 +570,6 @@ bool tc_supported(const mrp_config &cfg, const mrp_head_weights *heads, const vo
 {
     if (cfg.dtype != MRP_BF16) return false;
     if (cfg.d % 64 || cfg.d_ff % 64 || cfg.vocab % 16) return false;
-    if (cfg.n_heads > 4) return false;
     if ((uintptr_t)w_lm & 15u) return false;
     for (int k = 0; k < cfg.n_heads; ++k)
         if (((uintptr_t)heads[k].rms_gamma & 1u) || ((uintptr_t)heads[k].w_gate & 15u) ||
@@ -616,7 +652,8 @@ cudaError_t tc_draft(Ctx *c, const void *hidden, const float *logits0, const int
                                       (int32_t *)(c->ws + c->lay.sk_counters), kSkMaxTiles,
                                       (unsigned long long *)(c->ws + c->lay.ssq_fix), c->from_hidden ? 1 : 0,
                                       (const __nv_bfloat16 *)c->final_gamma, c->cfg.rms_eps,
-                                      (c->from_hidden && f16_lm) ? (__half *)(c->ws + c->lay.xt16) : (__half *)nullptr),
+                                      (c->from_hidden && f16_lm) ? (__half *)(c->ws + c->lay.xt16) : (__half *)nullptr,
+                                      c->input_rows, status, out.status),
                              "tc_prep_kernel");
     c->launches++;
     if (e != cudaSuccess) return e;
@@ -698,6 +735,7 @@ cudaError_t tc_draft(Ctx *c, const void *hidden, const float *logits0, const int
         p.a_row_base = step_base * M; p.a_part_rows = n_rs; p.step_base = step_base;
         p.M = M; p.K = K; p.V = V; p.d = d; p.F = F; p.n_rs = n_rs;
         p.logits0 = logits0; p.row_index = row_index; p.partials = partials; p.logits_out = out.logits_out;
+        p.n_rows_in = c->input_rows;
         p.status = status; p.user_status = out.status;
         finish_shape(p, n_slices, f16_lm ? 1 : 2);
         const int grid = p.n_groups * p.n_vr;
@@ -722,11 +760,12 @@ cudaError_t tc_draft(Ctx *c, const void *hidden, const float *logits0, const int
     prof_mark(c, 2, st);
     TopFix fix;
     memset(&fix, 0, sizeof(fix));
-    if (f16_lm) {
-        fix.w = (const __nv_bfloat16 *)c->w_lm; fix.xt = xt; fix.logits0 = logits0; fix.row_index = row_index;
-        fix.d = d; fix.V = V; fix.M = M; fix.n_rs = n_rs;
-    }
-    e = launch_combine(c, partials, n_slices, (K + 1) * M, out, status, st, f16_lm ? &fix : nullptr);
+    // every call: the size of the operand rows against the accuracy range; fp16 mode: the exact top logit
+    fix.xt = xt; fix.logits0 = logits0; fix.row_index = row_index;
+    fix.d = d; fix.V = V; fix.M = M; fix.n_rs = n_rs; fix.n_rows_in = c->input_rows;
+    fix.range_limit = MRP_RANGE_LIMIT;
+    if (f16_lm) fix.w = (const __nv_bfloat16 *)c->w_lm;
+    e = launch_combine(c, partials, n_slices, (K + 1) * M, out, status, st, &fix);
     prof_mark(c, 3, st);
     return e;
 }

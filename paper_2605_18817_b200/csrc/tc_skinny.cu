@@ -60,6 +60,7 @@ struct SkParams {
     // LM
     const float *logits0;
     const int32_t *row_index;
+    int n_rows_in;       // row_index entries at or above are invalid: their base logits read as zero
     Partial *partials;
     float *logits_out;
     // GU
@@ -267,7 +268,9 @@ sk_gemm_kernel(const __grid_constant__ SkMaps maps, const SkParams p)
         if (KIND == SK_LM) {
             if (t < p.n_rs) {
                 const int m = t % p.M;
-                rowoff_s[t] = (long long)(p.row_index ? p.row_index[m] : m) * p.V;
+                const int idx = p.row_index ? p.row_index[m] : m;
+                // -1: no base logits for this row-step (none given, or the caller's index is out of range)
+                rowoff_s[t] = (p.logits0 && (!p.row_index || row_ok(idx, p.n_rows_in))) ? (long long)idx * p.V : -1ll;
             }
         } else if (KIND == SK_GU) {
             if (t < p.M) {
@@ -297,7 +300,7 @@ sk_gemm_kernel(const __grid_constant__ SkMaps maps, const SkParams p)
                 float a[RP];
 #pragma unroll
                 for (int j = 0; j < RP; ++j)
-                    a[j] = (valid && j < p.n_rs && p.logits0) ? __ldg(p.logits0 + rowoff_s[j] + v) : 0.f;
+                    a[j] = (valid && j < p.n_rs && rowoff_s[j] >= 0) ? __ldg(p.logits0 + rowoff_s[j] + v) : 0.f;
                 ok = __all_sync(0xffffffffu, mbar_wait(tfull_bar(acc), acc_ph, abort_flag, p));
                 if (!ok) break;
                 tc_fence_after();
@@ -714,7 +717,7 @@ cudaError_t sk_lm(Ctx *c, const float *logits0, const int32_t *row_index, int M,
     sk_common(c, p, M, K, out);
     p.units_total = V / 16; p.k_chunks = d / kBK; p.r_pad = sk_lm_pad(p.n_rs);
     p.kc = (p.k_chunks % 2 == 0) ? 2 : 1;
-    p.logits0 = logits0; p.row_index = row_index;
+    p.logits0 = logits0; p.row_index = row_index; p.n_rows_in = c->input_rows;
     p.partials = (Partial *)(c->ws + c->lay.partials); p.logits_out = out.logits_out;
     sk_finish_shape(p, G);
     SkMaps maps;

@@ -116,18 +116,23 @@ class Inputs:
 
 
 def make_inputs(w: Weights, B: int, L: int, seed: int, s_lo: float, s_hi: float,
-                mask_prob: float = 1.0, calibrated: bool = True, logits_fn=None) -> Inputs:
+                mask_prob: float = 1.0, calibrated: bool = True, logits_fn=None,
+                logits_rows: int | None = None, planted=None) -> Inputs:
     """Backbone outputs for one active block per sequence.
 
     ``mask_prob`` < 1 masks each position independently (at least one per block, by
     resampling the block); 1.0 masks every position.  ``logits_fn(hidden_rows)`` may replace
     the host matrix product that produces the base logits (e.g. an fp32 product on another
-    device); whatever it returns is the input both sides then share.
+    device); whatever it returns is the input both sides then share.  ``logits_rows`` limits the
+    base logits to the first that many masked rows (the others stay zero: for consumers that only
+    touch a sample of the rows).  ``planted`` [B*L] overrides the uniformly drawn planted tokens
+    (e.g. to put the top token of some rows at the two ends of the vocabulary).
     """
     n = B * L
     d, V = w.d, w.V
     z = _rng(seed, _S_Z).standard_normal((n, d), dtype=np.float32)
-    planted = _rng(seed, _S_TOK).integers(0, V, size=n, dtype=np.int64).astype(np.int32)
+    drawn = _rng(seed, _S_TOK).integers(0, V, size=n, dtype=np.int64).astype(np.int32)
+    planted = drawn if planted is None else np.asarray(planted, np.int32).reshape(n)
     u = _rng(seed, _S_STRENGTH).random(n)
     strength = (s_lo + (s_hi - s_lo) * u).astype(np.float32)
     rows = w.w_lm[planted]                                   # [n, d]
@@ -150,8 +155,9 @@ def make_inputs(w: Weights, B: int, L: int, seed: int, s_lo: float, s_hi: float,
     row_index = np.flatnonzero(mask.reshape(-1)).astype(np.int32)
     logits0 = np.zeros((n, V), np.float32)
     step = 256
-    for i in range(0, row_index.size, step):                 # base logits = LM head on h
-        idx = row_index[i:i + step]
+    n_logits = row_index.size if logits_rows is None else min(row_index.size, int(logits_rows))
+    for i in range(0, n_logits, step):                       # base logits = LM head on h
+        idx = row_index[i:min(i + step, n_logits)]
         logits0[idx] = logits_fn(hidden[idx]) if logits_fn else hidden[idx] @ w.w_lm.T
     return Inputs(B, L, hidden, logits0, row_index, planted, strength)
 
@@ -189,11 +195,11 @@ def sweep_config(M: int, K: int) -> dict:
                 mode="static", seed=4000 + p)
 
 
-def make_config(cfg: dict, weights: Weights | None = None, logits_fn=None):
+def make_config(cfg: dict, weights: Weights | None = None, logits_fn=None, planted=None):
     """Weights (unless given) and inputs of a configuration dict."""
     if weights is None:
         weights = make_weights(cfg["d"], cfg["F"], cfg["V"], cfg["n_heads"], cfg["dtype"],
                                cfg["seed"])
     inp = make_inputs(weights, cfg["B"], cfg["L"], cfg["seed"], cfg["s_lo"], cfg["s_hi"],
-                      cfg["mask_prob"], logits_fn=logits_fn)
+                      cfg["mask_prob"], logits_fn=logits_fn, planted=planted)
     return weights, inp

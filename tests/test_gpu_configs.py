@@ -1,5 +1,9 @@
 """Full-size parity: the five benchmark configurations run through the C ABI at their real
-shapes; the oracle recomputes sampled rows (all V columns) or whole sampled blocks."""
+shapes, in the launch configuration the benchmark times (default flags); the oracle recomputes
+every row where there are at most 256, else 256 or more rows (whole blocks) spread so that every
+128-row block of the stacked row-steps is hit, over all V columns.  Some of the compared rows have
+their top token planted in the first and in the last 16 entries of the vocabulary, i.e. in the
+first and the last CTA's range."""
 import gc
 
 import numpy as np
@@ -36,6 +40,23 @@ class Device:
         heads = self.heads if n_heads is None else self.heads[:n_heads]
         return binding.mrp_create(self.w.d, self.w.F, self.w.V, heads, self.w_lm, max_rows=rows,
                                   max_seqs=seqs, block_len=block, flags=flags)
+
+
+def spread_rows(M, n=256):
+    """n row numbers spread evenly over 0..M-1 (all of them if M <= n), first and last included."""
+    if M <= n:
+        return np.arange(M)
+    return np.unique(np.round(np.linspace(0, M - 1, n)).astype(np.int64))
+
+
+def plant_vocabulary_ends(cfg, rows):
+    """Planted tokens of a configuration with those of the dense positions `rows` moved to the two
+    ends of the vocabulary, alternating."""
+    n, V = cfg["B"] * cfg["L"], cfg["V"]
+    planted = synth._rng(cfg["seed"], synth._S_TOK).integers(0, V, size=n, dtype=np.int64).astype(np.int32)
+    for i, r in enumerate(rows):
+        planted[r] = (i // 2) % 16 if i % 2 == 0 else V - 1 - (i // 2) % 16
+    return planted
 
 
 def gpu_draft(dev, ctx, inp, K, **kw):
@@ -111,15 +132,16 @@ def test_config2_speculative_shape_sampled_rows_and_verify():
     cfg = synth.CONFIGS[2]
     w = synth.make_weights(cfg["d"], cfg["F"], cfg["V"], cfg["n_heads"], cfg["dtype"], cfg["seed"])
     dev = Device(w)
-    _, inp = synth.make_config(cfg, w, logits_fn=dev.logits_fn)
+    _, inp = synth.make_config(cfg, w, logits_fn=dev.logits_fn, planted=plant_vocabulary_ends(cfg, range(0, 8)))
     K, B, L = cfg["K"], cfg["B"], cfg["L"]
     M = len(inp.row_index)
     assert M == 128
     ctx = dev.ctx(M, B, L)
     out, ri = gpu_draft(dev, ctx, inp, K)
-    sample = np.array([0, 37, 64, 101, 126, 127])
-    ref = oracle.draft(inp.hidden, inp.logits0, w.heads, w.w_lm, K=K, row_index=inp.row_index[sample])
-    check_stats(out, ref, "bf16", cols=sample)
+    # every row of the configuration against the oracle
+    ref = oracle.draft(inp.hidden, inp.logits0, w.heads, w.w_lm, K=K, row_index=inp.row_index)
+    check_stats(out, ref, "bf16")
+    assert ref.token[0, 0] == 0 and ref.token[0, 1] == w.V - 1       # the planted ends of the vocabulary
     # selection on the device's own statistics is bit-exact against the oracle's rules
     sel = harness.alloc_select_out(B, L, K, DEV)
     harness.select(ctx, out.conf, out.token, ri, M, K, B, L, binding.MRP_SELECT_STATIC, sel)
@@ -144,7 +166,7 @@ def test_config3_remask_shape_sampled_blocks():
     cfg = synth.CONFIGS[3]
     w = synth.make_weights(cfg["d"], cfg["F"], cfg["V"], cfg["n_heads"], cfg["dtype"], cfg["seed"])
     dev = Device(w)
-    _, inp = synth.make_config(cfg, w, logits_fn=dev.logits_fn)
+    _, inp = synth.make_config(cfg, w, logits_fn=dev.logits_fn, planted=plant_vocabulary_ends(cfg, range(0, 32)))
     K, B, L, tau = cfg["K"], cfg["B"], cfg["L"], cfg["tau"]
     M = len(inp.row_index)
     assert 850 < M < 1200
@@ -160,9 +182,11 @@ def test_config3_remask_shape_sampled_blocks():
                              oracle.DYNAMIC_REMASK, tau=tau, remask_policy=policy)
         _assert_select_equal(sel, osel)
         assert 0 < osel.remask_mask.sum() < osel.reveal_mask.sum()
-    # (ii) end to end on three whole blocks, recomputed by the oracle
-    blocks = [0, 31, 63]
+    # (ii) end to end on every fourth block and the last (some 270 rows, two or more in every 128-row
+    # block of the stacked row-steps), recomputed by the oracle
+    blocks = sorted(set(range(0, B, 4)) | {B - 1})
     rows = np.flatnonzero(np.isin(inp.row_index // L, blocks))
+    assert rows.size >= 256 and np.all(np.diff(rows) < 128)
     ref = oracle.draft(inp.hidden, inp.logits0, w.heads, w.w_lm, K=K, row_index=inp.row_index[rows])
     check_stats(out, ref, "bf16", cols=rows)
     checked = 0
@@ -180,7 +204,7 @@ def test_config3_remask_shape_sampled_blocks():
         assert np.array_equal(sel_np["remask_mask"][sl], o.remask_mask)
         assert np.array_equal(sel_np["out_token"][sl], o.out_token)
         checked += 1
-    assert checked >= 1
+    assert checked >= 2
     binding.mrp_destroy(ctx)
     del dev, w
     gc.collect()
@@ -197,10 +221,11 @@ def sweep_dev():
 def test_sweep_points_sampled_rows(sweep_dev, M, K):
     dev = sweep_dev
     cfg = synth.sweep_config(M, K)
-    _, inp = synth.make_config(cfg, dev.w, logits_fn=dev.logits_fn)
+    sample = spread_rows(M)
+    _, inp = synth.make_config(cfg, dev.w, logits_fn=dev.logits_fn,
+                               planted=plant_vocabulary_ends(cfg, [sample[0], sample[-1]]))
     ctx = dev.ctx(M, M, 1, n_heads=K)
     out, _ = gpu_draft(dev, ctx, inp, K, margin=False)
-    sample = np.unique(np.array([0, M // 3, M // 2, M - 1]))
     ref = oracle.draft(inp.hidden, inp.logits0, dev.w.heads, dev.w.w_lm, K=K,
                        row_index=inp.row_index[sample])
     check_stats(out, ref, "bf16", cols=sample)
@@ -227,7 +252,7 @@ def test_sweep_points_base_logits_from_hidden_states(sweep_dev, M, K):
     out = harness.alloc_draft_out(M, K, dev.w.V, dev.w.d, DEV, margin=False)
     harness.draft_from_hidden(ctx, hid, harness.to_device(gam, dev.w.dtype, DEV), ri, M, K, out)
     torch.cuda.synchronize()
-    sample = np.unique(np.array([0, M // 3, M // 2, M - 1]))
+    sample = spread_rows(M)
     ref = oracle.draft(inp.hidden, None, dev.w.heads, dev.w.w_lm, K=K, row_index=inp.row_index[sample],
                        final_gamma=gam)
     check_stats(out, ref, "bf16", cols=sample)

@@ -270,8 +270,9 @@ def test_config0_static_selection_end_to_end():
     (64, 6144, 1024, 5, 1, 2),      # the same with few rows
 ])
 def test_tensor_core_family_small_shapes(d, F, V, B, L, K):
-    # residuals of order one at every shape (the very long contraction gets smaller weights)
-    w = synth.make_weights(d, F, V, K, "bf16", 77, head_std=0.05 if d < 4096 else 0.03)
+    # residuals inside the accuracy range the header states for the tensor-core kernels
+    # (d * rms(h_k - h_0) <= MRP_RANGE_LIMIT; check_stats asserts that no status bit was raised)
+    w = synth.make_weights(d, F, V, K, "bf16", 77, head_std=0.05 if d < 4096 else 0.02)
     for k, h in enumerate(w.heads):
         h["gamma"] = synth.bf16_round((1.0 + 0.25 * np.cos(np.arange(d) + k)).astype(np.float32))
     inp = synth.make_inputs(w, B, L, 77, 1.0, 4.0)
@@ -298,6 +299,32 @@ def test_tensor_core_family_small_shapes(d, F, V, B, L, K):
     # the head chain as one kernel per GEMM instead of one persistent kernel
     out5, _ = run_gpu_draft(w, inp, K, flags=binding.MRP_FLAG_NO_CHAIN)
     check_stats(out5, ref, "bf16")
+
+
+@pytest.mark.parametrize("d,F,V,M,K,std,beyond", [
+    (19008, 64, 512, 3, 1, 0.02, False),        # d * rms about 14 000
+    (19008, 64, 512, 3, 1, 0.05, True),         # about 220 000
+    (4096, 8192, 4096, 40, 2, 0.02, False),     # the benchmark shapes' weights: about 11 000
+    (4096, 8192, 4096, 40, 2, 0.04, True),      # about 98 000: beyond the range, and beyond the tolerance
+])
+def test_residuals_beyond_the_accuracy_range_raise_the_range_bit(d, F, V, M, K, std, beyond):
+    """The tensor-core kernels keep confidence and log-sum-exp within 2e-3 while d * rms(h_k - h_0)
+    stays below MRP_RANGE_LIMIT; a row-step beyond it is still computed but raises MRP_DEV_RANGE
+    (the CUDA-core kernels, which accumulate by fp32 FMA, take the same input without the bit)."""
+    w = synth.make_weights(d, F, V, K, "bf16", 77, head_std=std)
+    inp = synth.make_inputs(w, M, 1, 77, 1.0, 4.0)
+    ref = oracle.draft(inp.hidden, inp.logits0, w.heads, w.w_lm, K=K, want_hidden=True)
+    d_rms = d * np.sqrt(((ref.hidden - inp.hidden.astype(np.float64)) ** 2).mean(axis=1)).max()
+    assert (d_rms > 2 * binding.MRP_RANGE_LIMIT) if beyond else (d_rms < 0.5 * binding.MRP_RANGE_LIMIT)
+    out, fam = run_gpu_draft(w, inp, K)
+    assert fam == "tcgen05"
+    assert int(out.status.item()) == (binding.MRP_DEV_RANGE if beyond else 0)
+    assert torch.isfinite(out.lse).all()
+    if not beyond:
+        check_stats(out, ref, "bf16")
+    out_s, fam_s = run_gpu_draft(w, inp, K, flags=binding.MRP_FLAG_FORCE_SIMT)
+    assert fam_s == "simt" and int(out_s.status.item()) == 0
+    check_stats(out_s, ref, "bf16")
 
 
 @pytest.mark.parametrize("flags", [0, binding.MRP_FLAG_FORCE_SIMT])

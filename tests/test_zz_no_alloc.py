@@ -3,9 +3,10 @@
 It serves callers that cannot allocate device memory (an engine whose pool owns the GPU, a
 plugin inside a foreign CUDA context, a path where cudaMalloc is forbidden) and so cannot
 give `mrp_create` a workspace: its scratch is a fixed array inside the library.  The checks:
-its outputs equal those of the context-based `mrp_reveal_remask` on two calls in a row (the
-second on a smaller problem, so anything the first call left in the shared array would show),
-and sizes beyond the built-in capacity are refused on the host.
+its outputs equal the CPU oracle's selection and those of the context-based
+`mrp_reveal_remask` on several calls in a row (later ones on smaller problems, so anything an
+earlier call left in the shared array would show), and sizes beyond the built-in capacity are
+refused on the host.
 
 This file sorts last on purpose: a run that stops at the first failure has by then run
 every other test.
@@ -16,6 +17,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2605_18817_b200 import binding, harness, synth
 
 DEV = "cuda:0"
@@ -45,7 +47,11 @@ def _both(ctx, ri, conf, token, B, L, mode, **kw):
     binding.mrp_reveal_remask_noalloc(c, t, r, M, K, B, L, mode, **kw,
                                       **{n: getattr(got, n) for n in NAMES})
     torch.cuda.synchronize()
+    omode = oracle.STATIC if mode == binding.MRP_SELECT_STATIC else oracle.DYNAMIC_REMASK
+    want = oracle.select(conf, token, ri, B, L, omode, **kw)
     for n in NAMES:
+        w = getattr(want, n)
+        assert np.array_equal(getattr(got, n).cpu().numpy().reshape(w.shape), w), n
         assert torch.equal(getattr(got, n), getattr(ref, n)), n
 
 
@@ -54,8 +60,10 @@ def test_noalloc_selection_matches_context_entry_point_twice_in_a_row():
     w = synth.make_weights(16, 16, 32, 0, "f32", 1)
     heads, w_lm = harness.upload_weights(w, DEV)
     ctx = binding.mrp_create(16, 16, 32, heads, w_lm, max_rows=4, max_seqs=2048, block_len=128)
-    # first call: the full capacity (B * L = 65536 positions), densely masked
+    # first call: the full capacity (B * L = 65536 positions), densely masked; B * M > 2^22, the size
+    # from which the context entry point goes through a dense position map as well
     ri, conf, token = _case(11, 2, 2048, 32, 0.9)
+    assert 2048 * ri.size > (1 << 22)
     _both(ctx, ri, conf, token, 2048, 32, binding.MRP_SELECT_DYNAMIC_REMASK, tau=0.5)
     # second call: fewer, sparsely masked positions over the same part of the shared array
     ri, conf, token = _case(12, 3, 40, 16, 0.3)
@@ -69,7 +77,7 @@ def test_noalloc_selection_matches_context_entry_point_twice_in_a_row():
 def test_noalloc_selection_refuses_sizes_beyond_its_capacity_on_the_host():
     lib = binding.lib
     p = binding.mrp_select_params(0, 0.5, 1, 1, 0, 0, 1)
-    o = binding.mrp_select_out(8, 8, 8, 8, 8, 8, 8)          # never dereferenced: refused first
+    o = binding.mrp_select_out(8, 8, 8, 8, 8, 8, 8, None)    # never dereferenced: refused first
     B, L = binding.MRP_NOALLOC_MAX_POSITIONS // 32 + 1, 32
     rc = lib.mrp_reveal_remask_noalloc(None, None, None, 0, 1, B, L, ctypes.byref(p),
                                        ctypes.byref(o), None)
