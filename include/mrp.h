@@ -157,6 +157,9 @@ void mrp_destroy(mrp_ctx *ctx);
  *                never written to memory
  *   hidden_out = optional [M, d] fp32: h after step K; NULL = skip
  *   status = optional device int32 that receives MRP_DEV_* bits (OR-ed, never cleared)
+ *   conf_first = optional [(K+1), M]: softmax probability, under step k's logits, of the token
+ *            that is on top at step 0 (the token a reveal at step 0 commits); equals conf where
+ *            the argmax has not moved; read by remask_policy 2 of mrp_reveal_remask; NULL = skip
  */
 typedef struct {
     float *conf;
@@ -166,6 +169,7 @@ typedef struct {
     float *logits_out;
     float *hidden_out;
     int32_t *status;
+    float *conf_first;
 } mrp_draft_out;
 
 /*
@@ -209,9 +213,19 @@ typedef struct {
     float tau;                /* confidence threshold (dynamic mode)                     */
     int32_t r_reveal;         /* static: positions revealed from the backbone step k=0   */
     int32_t r_draft;          /* static: positions drafted per MRP step k>=1             */
-    int32_t use_cap;          /* dynamic: cap |R| at min(max(floor(0.7 n),5),L), Sec.4.4 */
-    int32_t remask_policy;    /* 0 = min over steps 1..K must stay >= tau, 1 = step K    */
+    int32_t use_cap;          /* dynamic: cap |R| at min(max(floor(0.7 n),5),L), Sec.4.4
+                                 (the setting of the paper's dynamic-mode experiments)   */
+    int32_t remask_policy;    /* which updated quantity revokes a member of R (Algorithm 4
+                                 remask step; the paper has K = 1 and the top-1 probability):
+                                 0 = min over steps 1..K of the updated confidence < tau,
+                                 1 = updated confidence of step K < tau,
+                                 2 = min over steps 1..K of conf_first (probability of the
+                                     token revealed at step 0) < tau,
+                                 3 = the argmax differs from the revealed token at some
+                                     step 1..K                                            */
     int32_t ensure_progress;  /* keep at least one reveal per block                      */
+    const float *conf_first;  /* DEVICE [(K+1), M], mrp_draft_out.conf_first: read by
+                                 remask_policy 2 only, NULL otherwise                     */
 } mrp_select_params;
 
 /*
@@ -247,8 +261,9 @@ typedef struct {
  *   DYNAMIC_REMASK (Algorithm 4; Sec. 4.1 dynamic denoising; Sec. 4.4 cap): R = masked
  *   positions with conf_0 >= tau (the most confident one if none and ensure_progress;
  *   the cap's most confident ones if use_cap and |R| exceeds it); remask members of R whose
- *   updated confidence (policy) is < tau; if that revokes all of R and ensure_progress, the
- *   most confident member stays.  Comparisons are fp32.
+ *   updated confidence (remask_policy; variants 2 and 3 follow the revealed token instead of
+ *   the top one) is < tau; if that revokes all of R and ensure_progress, the most confident
+ *   member stays.  Comparisons are fp32.
  * conf, token: [(K+1), M]; row_index [M] (unique, < B*L) or NULL; 1 <= L <= block_len,
  * 1 <= B <= max_seqs.  Errors: INVALID_ARG, CUDA.
  */

@@ -45,6 +45,7 @@ def _load():
         _lib.mrp_oracle_cap.argtypes = [ctypes.c_int, ctypes.c_int]
         _lib.mrp_oracle_draft.restype = ctypes.c_int
         _lib.mrp_oracle_draft_from_hidden.restype = ctypes.c_int
+        _lib.mrp_oracle_draft_kl.restype = ctypes.c_int
         _lib.mrp_oracle_select.restype = ctypes.c_int
         _lib.mrp_oracle_verify.restype = ctypes.c_int
     return _lib
@@ -79,6 +80,7 @@ class DraftResult:
     margin: np.ndarray    # [(K+1), M] float64, top-1 minus top-2 logit
     logits: np.ndarray | None   # [K, M, V] float64
     hidden: np.ndarray | None   # [M, d] float64
+    conf_first: np.ndarray | None = None   # [(K+1), M] float64: probability under step k of the step-0 argmax token
 
 
 def draft(hidden, logits0, heads, w_lm, K=None, row_index=None, eps=1e-6,
@@ -132,6 +134,7 @@ def draft(hidden, logits0, heads, w_lm, K=None, row_index=None, eps=1e-6,
     token = np.zeros((K + 1, M), np.int32)
     logits = np.zeros((K, M, V), np.float64) if want_logits else None
     hid = np.zeros((M, d), np.float64) if want_hidden else None
+    conf_first = np.zeros((K + 1, M), np.float64)
     fn = lib.mrp_oracle_draft_from_hidden if from_hidden else lib.mrp_oracle_draft
     rc = fn(
         ctypes.c_int(d), ctypes.c_int(F), ctypes.c_int(V), ctypes.c_int(K), ctypes.c_int(M),
@@ -140,10 +143,50 @@ def draft(hidden, logits0, heads, w_lm, K=None, row_index=None, eps=1e-6,
         _p(ri, ctypes.c_int32), arrs["gamma"], arrs["w_gate"], arrs["w_up"], arrs["w_down"],
         _p(w_lm, ctypes.c_float), _p(conf, ctypes.c_double), _p(lse, ctypes.c_double),
         _p(token, ctypes.c_int32), _p(margin, ctypes.c_double), _p(logits, ctypes.c_double),
-        _p(hid, ctypes.c_double))
+        _p(hid, ctypes.c_double), _p(conf_first, ctypes.c_double))
     if rc != 0:
         raise RuntimeError("mrp_oracle_draft failed (%d)" % rc)
-    return DraftResult(conf, lse, token, margin, logits, hid)
+    return DraftResult(conf, lse, token, margin, logits, hid, conf_first)
+
+
+def draft_kl(hidden, logits0, teacher, heads, w_lm, K=None, row_index=None, eps=1e-6):
+    """The drafting pass with the training objective (Algorithm 1, Eq. (3)): ``teacher`` [K, M, V]
+    are the backbone's logits of every unrolled step's revealed sequence at the masked rows; returns
+    (DraftResult, kl [K, M]) with kl = KL(softmax(teacher_k) || softmax(l_k))."""
+    lib = _load()
+    hidden, logits0, w_lm, teacher = _f32(hidden), _f32(logits0), _f32(w_lm), _f32(teacher)
+    n_rows, d = hidden.shape
+    V = w_lm.shape[0]
+    K = len(heads) if K is None else int(K)
+    ri, M = None, n_rows
+    if row_index is not None:
+        ri = _i32(row_index)
+        M = ri.shape[0]
+        assert M == 0 or (ri.min() >= 0 and ri.max() < n_rows)
+    assert teacher.shape == (K, M, V) and logits0.shape == (n_rows, V) and K >= 1
+    F = heads[0]["w_gate"].shape[0]
+    PtrArr = ctypes.POINTER(ctypes.c_float) * K
+    keep, arrs = [], {}
+    for name, shape in (("gamma", (d,)), ("w_gate", (F, d)), ("w_up", (F, d)), ("w_down", (d, F))):
+        lst = []
+        for k in range(K):
+            a = _f32(heads[k][name])
+            assert a.shape == shape
+            keep.append(a)
+            lst.append(_p(a, ctypes.c_float))
+        arrs[name] = PtrArr(*lst)
+    conf, lse, margin = (np.zeros((K + 1, M), np.float64) for _ in range(3))
+    token = np.zeros((K + 1, M), np.int32)
+    kl = np.zeros((K, M), np.float64)
+    rc = lib.mrp_oracle_draft_kl(
+        ctypes.c_int(d), ctypes.c_int(F), ctypes.c_int(V), ctypes.c_int(K), ctypes.c_int(M),
+        ctypes.c_double(eps), _p(hidden, ctypes.c_float), _p(logits0, ctypes.c_float), _p(ri, ctypes.c_int32),
+        arrs["gamma"], arrs["w_gate"], arrs["w_up"], arrs["w_down"], _p(w_lm, ctypes.c_float),
+        _p(teacher, ctypes.c_float), _p(conf, ctypes.c_double), _p(lse, ctypes.c_double),
+        _p(token, ctypes.c_int32), _p(margin, ctypes.c_double), _p(kl, ctypes.c_double))
+    if rc != 0:
+        raise RuntimeError("mrp_oracle_draft_kl failed (%d)" % rc)
+    return DraftResult(conf, lse, token, margin, None, None), kl
 
 
 @dataclass
@@ -162,11 +205,18 @@ DYNAMIC_REMASK = 1
 
 
 def select(conf, token, row_index, B, L, mode, tau=0.9, r_reveal=1, r_draft=1,
-           use_cap=False, remask_policy=0, ensure_progress=True) -> SelectResult:
-    """Static top-r reveal/draft or dynamic threshold reveal + remask (Algorithms 2-4)."""
+           use_cap=False, remask_policy=0, ensure_progress=True, conf_first=None) -> SelectResult:
+    """Static top-r reveal/draft or dynamic threshold reveal + remask (Algorithms 2-4).
+    ``remask_policy``: 0 = min over steps 1..K of the updated confidence, 1 = step K only,
+    2 = min over steps of ``conf_first`` (probability of the token revealed at step 0),
+    3 = revoke when the argmax left that token at any step."""
     lib = _load()
     conf = _f32(conf)
     token = _i32(token)
+    cf = None
+    if conf_first is not None:
+        cf = _f32(conf_first)
+        assert cf.shape == conf.shape
     Kp1, M = conf.shape
     assert token.shape == conf.shape
     K = Kp1 - 1
@@ -185,7 +235,7 @@ def select(conf, token, row_index, B, L, mode, tau=0.9, r_reveal=1, r_draft=1,
         _p(out.reveal_mask, ctypes.c_int8), _p(out.remask_mask, ctypes.c_int8),
         _p(out.out_token, ctypes.c_int32), _p(out.step_of, ctypes.c_int8),
         _p(out.draft_pos, ctypes.c_int32), _p(out.draft_tok, ctypes.c_int32),
-        _p(out.draft_len, ctypes.c_int32))
+        _p(out.draft_len, ctypes.c_int32), _p(cf, ctypes.c_float))
     if rc != 0:
         raise RuntimeError("mrp_oracle_select failed (%d)" % rc)
     return out

@@ -71,6 +71,23 @@ static void softmax_stats(const double *l, int V, double *conf, double *lse, int
     *margin = (V > 1) ? (mx - second) : INFINITY;
 }
 
+/* Forward KL divergence KL(softmax(t) || softmax(l)) of two logit rows (Eq. (3)), from the
+ * definition: sum_v p_v (log p_v - log q_v) with p = softmax(t), q = softmax(l). */
+static double kl_rows(const double *t, const double *l, int V)
+{
+    double mt = t[0], ml = l[0];
+    for (int v = 1; v < V; ++v) { if (t[v] > mt) mt = t[v]; if (l[v] > ml) ml = l[v]; }
+    double st = 0.0, sl = 0.0;
+    for (int v = 0; v < V; ++v) { st += exp(t[v] - mt); sl += exp(l[v] - ml); }
+    const double lse_t = mt + log(st), lse_l = ml + log(sl);
+    double kl = 0.0;
+    for (int v = 0; v < V; ++v) {
+        const double logp = t[v] - lse_t, logq = l[v] - lse_l;
+        kl += exp(logp) * (logp - logq);
+    }
+    return kl;
+}
+
 /*
  * One drafting pass over M masked rows (Algorithm 2, lines "for k = 1..K").
  *   hidden  [n_rows, d]   backbone hidden states h
@@ -83,6 +100,10 @@ static void softmax_stats(const double *l, int V, double *conf, double *lse, int
  *   conf, lse, margin [(K+1), M] double; token [(K+1), M] int32
  *   logits_out  optional [K, M, V]  (l after step k = 1..K)
  *   hidden_out  optional [M, d]     (h after step K)
+ *   conf_first  optional [(K+1), M] softmax probability, under step k's logits, of the row's
+ *               step-0 argmax token (the token a reveal at step 0 commits; Algorithm 4 remasks by
+ *               the confidence of the updated logits, and this is the variant that follows the
+ *               committed token itself)
  * Returns 0, or -1 on allocation failure / bad arguments.
  */
 static int draft_rows(int d, int F, int V, int K, int M, double eps,
@@ -92,15 +113,18 @@ static int draft_rows(int d, int F, int V, int K, int M, double eps,
                       const float *const *w_up, const float *const *w_down,
                       const float *w_lm,
                       double *conf, double *lse, int32_t *token, double *margin,
-                      double *logits_out, double *hidden_out)
+                      double *logits_out, double *hidden_out, double *conf_first,
+                      const float *teacher, double *kl)
 {
     if (d <= 0 || F <= 0 || V <= 0 || K < 0 || M < 0) return -1;
+    if ((teacher != NULL) != (kl != NULL)) return -1;
     double *h = (double *)malloc(sizeof(double) * (size_t)d);
     double *xh = (double *)malloc(sizeof(double) * (size_t)d);
     double *a = (double *)malloc(sizeof(double) * (size_t)F);
     double *r = (double *)malloc(sizeof(double) * (size_t)d);
     double *l = (double *)malloc(sizeof(double) * (size_t)V);
-    if (!h || !xh || !a || !r || !l) { free(h); free(xh); free(a); free(r); free(l); return -1; }
+    double *tt = (double *)malloc(sizeof(double) * (size_t)V);
+    if (!h || !xh || !a || !r || !l || !tt) { free(h); free(xh); free(a); free(r); free(l); free(tt); return -1; }
 
     for (int m = 0; m < M; ++m) {
         const size_t row = row_index ? (size_t)row_index[m] : (size_t)m;
@@ -126,6 +150,7 @@ static int draft_rows(int d, int F, int V, int K, int M, double eps,
             }
         }
         softmax_stats(l, V, &conf[m], &lse[m], &token[m], &margin[m]);
+        if (conf_first) conf_first[m] = conf[m];
 
         for (int k = 1; k <= K; ++k) {
             const float *g_k = gamma[k - 1];
@@ -164,12 +189,21 @@ static int draft_rows(int d, int F, int V, int K, int M, double eps,
             }
             const size_t o = (size_t)k * M + m;
             softmax_stats(l, V, &conf[o], &lse[o], &token[o], &margin[o]);
+            /* probability, under the updated logits, of the token that was on top at step 0 */
+            if (conf_first) conf_first[o] = exp(l[token[m]] - lse[o]);
+            /* training objective of this unrolled step (Eq. (3), Algorithm 1): the teacher logits of the
+             * step against the corrected logits l = l_t + delta */
+            if (teacher) {
+                const float *tr = teacher + ((size_t)(k - 1) * M + m) * (size_t)V;
+                for (int v = 0; v < V; ++v) tt[v] = (double)tr[v];
+                kl[(size_t)(k - 1) * M + m] = kl_rows(tt, l, V);
+            }
             if (logits_out)
                 memcpy(logits_out + ((size_t)(k - 1) * M + m) * V, l, sizeof(double) * (size_t)V);
         }
         if (hidden_out) memcpy(hidden_out + (size_t)m * d, h, sizeof(double) * (size_t)d);
     }
-    free(h); free(xh); free(a); free(r); free(l);
+    free(h); free(xh); free(a); free(r); free(l); free(tt);
     return 0;
 }
 
@@ -179,11 +213,29 @@ int mrp_oracle_draft(int d, int F, int V, int K, int M, double eps,
                      const float *const *w_up, const float *const *w_down,
                      const float *w_lm,
                      double *conf, double *lse, int32_t *token, double *margin,
-                     double *logits_out, double *hidden_out)
+                     double *logits_out, double *hidden_out, double *conf_first)
 {
     if (!logits0) return -1;
     return draft_rows(d, F, V, K, M, eps, hidden, logits0, 0, NULL, row_index, gamma, w_gate, w_up, w_down,
-                      w_lm, conf, lse, token, margin, logits_out, hidden_out);
+                      w_lm, conf, lse, token, margin, logits_out, hidden_out, conf_first, NULL, NULL);
+}
+
+/*
+ * The drafting pass with the training objective (Algorithm 1; Eq. (3)): teacher [K, M, V] holds, for
+ * every unrolled step k = 1..K and masked row m, the backbone's logits on the sequence that has the
+ * step's ground-truth tokens revealed (l_{t-1} in the paper's one-step notation); kl [K, M] receives
+ * KL(softmax(teacher_k) || softmax(l_k)), l_k = l_{k-1} + delta_k the corrected logits of the step.
+ */
+int mrp_oracle_draft_kl(int d, int F, int V, int K, int M, double eps,
+                        const float *hidden, const float *logits0, const int32_t *row_index,
+                        const float *const *gamma, const float *const *w_gate,
+                        const float *const *w_up, const float *const *w_down,
+                        const float *w_lm, const float *teacher,
+                        double *conf, double *lse, int32_t *token, double *margin, double *kl)
+{
+    if (!logits0 || !teacher || !kl) return -1;
+    return draft_rows(d, F, V, K, M, eps, hidden, logits0, 0, NULL, row_index, gamma, w_gate, w_up, w_down,
+                      w_lm, conf, lse, token, margin, NULL, NULL, NULL, teacher, kl);
 }
 
 /*
@@ -198,10 +250,10 @@ int mrp_oracle_draft_from_hidden(int d, int F, int V, int K, int M, double eps,
                                  const float *const *w_up, const float *const *w_down,
                                  const float *w_lm,
                                  double *conf, double *lse, int32_t *token, double *margin,
-                                 double *logits_out, double *hidden_out)
+                                 double *logits_out, double *hidden_out, double *conf_first)
 {
     return draft_rows(d, F, V, K, M, eps, hidden, NULL, 1, final_gamma, row_index, gamma, w_gate, w_up, w_down,
-                      w_lm, conf, lse, token, margin, logits_out, hidden_out);
+                      w_lm, conf, lse, token, margin, logits_out, hidden_out, conf_first, NULL, NULL);
 }
 
 /* Max-accept cap (Sec. 4.4): m = min(max(floor(0.7 n), 5), L). */
@@ -239,7 +291,12 @@ static int best_candidate(const int *cand, int n, const uint8_t *taken, const fl
  *            ensure_progress, R = {most confident}; if use_cap and |R| > m keep the m most
  *            confident; remask i in R whose updated confidence c'(i) < tau, where
  *            c'(i) = min_{k=1..K} conf[k,i] (remask_policy 0) or conf[K,i] (policy 1);
+ *            policy 2 follows the committed token instead of the top one: c'(i) =
+ *            min_{k=1..K} conf_first[k,i], the probability the updated logits give the token
+ *            revealed at step 0; policy 3 revokes i when the argmax moved away from that token
+ *            at any step, token[k,i] != token[0,i] for some k in 1..K;
  *            if everything was revoked and ensure_progress, the most confident of R stays.
+ *   conf_first [(K+1), M] float32: read by policy 2 only (NULL otherwise).
  * Outputs (all written for every dense position / block):
  *   reveal_mask, remask_mask [B*L] int8; out_token [B*L] int32 (-1 = nothing committed
  *   or drafted); step_of [B*L] int8 (-1 = untouched); draft_pos, draft_tok [B, Kd] int32
@@ -251,9 +308,10 @@ int mrp_oracle_select(const float *conf, const int32_t *token, const int32_t *ro
                       int r_draft, int use_cap, int remask_policy, int ensure_progress,
                       int8_t *reveal_mask, int8_t *remask_mask, int32_t *out_token,
                       int8_t *step_of, int32_t *draft_pos, int32_t *draft_tok,
-                      int32_t *draft_len)
+                      int32_t *draft_len, const float *conf_first)
 {
     if (M < 0 || K < 0 || B <= 0 || L <= 0) return -1;
+    if (mode == 1 && remask_policy == 2 && !conf_first) return -1;
     const int Kd = K * (r_draft > 0 ? r_draft : 0);
     for (int i = 0; i < B * L; ++i) {
         reveal_mask[i] = 0; remask_mask[i] = 0; out_token[i] = -1; step_of[i] = -1;
@@ -330,17 +388,26 @@ int mrp_oracle_select(const float *conf, const int32_t *token, const int32_t *ro
                 const int m = cand[i];
                 const int dense = b * L + pos[m];
                 reveal_mask[dense] = 1;
-                float c2;
-                if (K == 0) {
-                    c2 = conf[m];
-                } else if (remask_policy == 1) {
-                    c2 = conf[(size_t)K * M + m];
+                int revoke;
+                if (remask_policy == 3) {
+                    revoke = 0;
+                    for (int k = 1; k <= K; ++k)
+                        if (token[(size_t)k * M + m] != token[m]) revoke = 1;
                 } else {
-                    c2 = conf[(size_t)1 * M + m];
-                    for (int k = 2; k <= K; ++k)
-                        if (conf[(size_t)k * M + m] < c2) c2 = conf[(size_t)k * M + m];
+                    const float *cu = (remask_policy == 2) ? conf_first : conf;
+                    float c2;
+                    if (K == 0) {
+                        c2 = cu[m];
+                    } else if (remask_policy == 1) {
+                        c2 = cu[(size_t)K * M + m];
+                    } else {
+                        c2 = cu[(size_t)1 * M + m];
+                        for (int k = 2; k <= K; ++k)
+                            if (cu[(size_t)k * M + m] < c2) c2 = cu[(size_t)k * M + m];
+                    }
+                    revoke = (c2 < tau);
                 }
-                if (c2 < tau) remask_mask[dense] = 1; else ++kept;
+                if (revoke) remask_mask[dense] = 1; else ++kept;
             }
             if (kept == 0 && nR > 0 && ensure_progress) {
                 for (int i = 0; i < n; ++i) taken[i] = !inR[i];

@@ -54,13 +54,15 @@ class mrp_head_weights(ctypes.Structure):
 class mrp_draft_out(ctypes.Structure):
     _fields_ = [("conf", ctypes.c_void_p), ("lse", ctypes.c_void_p), ("token", ctypes.c_void_p),
                 ("margin", ctypes.c_void_p), ("logits_out", ctypes.c_void_p),
-                ("hidden_out", ctypes.c_void_p), ("status", ctypes.c_void_p)]
+                ("hidden_out", ctypes.c_void_p), ("status", ctypes.c_void_p),
+                ("conf_first", ctypes.c_void_p)]
 
 
 class mrp_select_params(ctypes.Structure):
     _fields_ = [("mode", ctypes.c_int32), ("tau", ctypes.c_float), ("r_reveal", ctypes.c_int32),
                 ("r_draft", ctypes.c_int32), ("use_cap", ctypes.c_int32),
-                ("remask_policy", ctypes.c_int32), ("ensure_progress", ctypes.c_int32)]
+                ("remask_policy", ctypes.c_int32), ("ensure_progress", ctypes.c_int32),
+                ("conf_first", ctypes.c_void_p)]
 
 
 class mrp_select_out(ctypes.Structure):
@@ -271,7 +273,7 @@ def mrp_profile_read(ctx: Context):
 
 
 def mrp_draft(ctx: Context, hidden, logits0, row_index, M, K, conf, lse, token, margin=None,
-              logits_out=None, hidden_out=None, status=None, stream=None) -> None:
+              logits_out=None, hidden_out=None, status=None, stream=None, conf_first=None) -> None:
     """Enqueue one drafting pass; outputs are written into the given CUDA tensors."""
     _check(hidden, torch.float32 if ctx.cfg.dtype == MRP_F32 else torch.bfloat16, "hidden")
     _check(logits0, torch.float32, "logits0")
@@ -279,10 +281,11 @@ def mrp_draft(ctx: Context, hidden, logits0, row_index, M, K, conf, lse, token, 
     for t, dt, nm in ((conf, torch.float32, "conf"), (lse, torch.float32, "lse"),
                       (token, torch.int32, "token"), (margin, torch.float32, "margin"),
                       (logits_out, torch.float32, "logits_out"),
-                      (hidden_out, torch.float32, "hidden_out"), (status, torch.int32, "status")):
+                      (hidden_out, torch.float32, "hidden_out"), (status, torch.int32, "status"),
+                      (conf_first, torch.float32, "conf_first")):
         _check(t, dt, nm)
     out = mrp_draft_out(_ptr(conf), _ptr(lse), _ptr(token), _ptr(margin), _ptr(logits_out),
-                        _ptr(hidden_out), _ptr(status))
+                        _ptr(hidden_out), _ptr(status), _ptr(conf_first))
     rc = lib.mrp_draft(ctx.handle, _ptr(hidden), _ptr(logits0), _ptr(row_index), int(M), int(K),
                        ctypes.byref(out), _stream(stream))
     if rc != 0:
@@ -290,7 +293,8 @@ def mrp_draft(ctx: Context, hidden, logits0, row_index, M, K, conf, lse, token, 
 
 
 def mrp_draft_from_hidden(ctx: Context, hidden, final_norm_gamma, row_index, M, K, conf, lse, token,
-                          margin=None, logits_out=None, hidden_out=None, status=None, stream=None) -> None:
+                          margin=None, logits_out=None, hidden_out=None, status=None, stream=None,
+                          conf_first=None) -> None:
     """Enqueue one drafting pass that computes the base logits itself (l_0 = W_lm n_0)."""
     dt_ctx = torch.float32 if ctx.cfg.dtype == MRP_F32 else torch.bfloat16
     _check(hidden, dt_ctx, "hidden")
@@ -299,10 +303,11 @@ def mrp_draft_from_hidden(ctx: Context, hidden, final_norm_gamma, row_index, M, 
     for t, dt, nm in ((conf, torch.float32, "conf"), (lse, torch.float32, "lse"),
                       (token, torch.int32, "token"), (margin, torch.float32, "margin"),
                       (logits_out, torch.float32, "logits_out"),
-                      (hidden_out, torch.float32, "hidden_out"), (status, torch.int32, "status")):
+                      (hidden_out, torch.float32, "hidden_out"), (status, torch.int32, "status"),
+                      (conf_first, torch.float32, "conf_first")):
         _check(t, dt, nm)
     out = mrp_draft_out(_ptr(conf), _ptr(lse), _ptr(token), _ptr(margin), _ptr(logits_out),
-                        _ptr(hidden_out), _ptr(status))
+                        _ptr(hidden_out), _ptr(status), _ptr(conf_first))
     rc = lib.mrp_draft_from_hidden(ctx.handle, _ptr(hidden), _ptr(final_norm_gamma), _ptr(row_index),
                                    int(M), int(K), ctypes.byref(out), _stream(stream))
     if rc != 0:
@@ -310,7 +315,7 @@ def mrp_draft_from_hidden(ctx: Context, hidden, final_norm_gamma, row_index, M, 
 
 
 def mrp_reveal_remask(ctx: Context, conf, token, row_index, M, K, B, L, mode, tau=0.9, r_reveal=1,
-                      r_draft=1, use_cap=False, remask_policy=0, ensure_progress=True, *,
+                      r_draft=1, use_cap=False, remask_policy=0, ensure_progress=True, conf_first=None, *,
                       reveal_mask, remask_mask, out_token, step_of, draft_pos, draft_tok, draft_len,
                       status=None, stream=None) -> None:
     _check(conf, torch.float32, "conf")
@@ -321,8 +326,9 @@ def mrp_reveal_remask(ctx: Context, conf, token, row_index, M, K, B, L, mode, ta
                       (draft_pos, torch.int32, "draft_pos"), (draft_tok, torch.int32, "draft_tok"),
                       (draft_len, torch.int32, "draft_len"), (status, torch.int32, "status")):
         _check(t, dt, nm)
+    _check(conf_first, torch.float32, "conf_first")
     p = mrp_select_params(int(mode), float(tau), int(r_reveal), int(r_draft), int(bool(use_cap)),
-                          int(remask_policy), int(bool(ensure_progress)))
+                          int(remask_policy), int(bool(ensure_progress)), _ptr(conf_first))
     o = mrp_select_out(_ptr(reveal_mask), _ptr(remask_mask), _ptr(out_token), _ptr(step_of),
                        _ptr(draft_pos), _ptr(draft_tok), _ptr(draft_len), _ptr(status))
     rc = lib.mrp_reveal_remask(ctx.handle, _ptr(conf), _ptr(token), _ptr(row_index), int(M), int(K),
@@ -332,7 +338,7 @@ def mrp_reveal_remask(ctx: Context, conf, token, row_index, M, K, B, L, mode, ta
 
 
 def mrp_reveal_remask_noalloc(conf, token, row_index, M, K, B, L, mode, tau=0.9, r_reveal=1,
-                              r_draft=1, use_cap=False, remask_policy=0, ensure_progress=True, *,
+                              r_draft=1, use_cap=False, remask_policy=0, ensure_progress=True, conf_first=None, *,
                               reveal_mask, remask_mask, out_token, step_of, draft_pos, draft_tok,
                               draft_len, status=None, stream=None) -> None:
     """Reveal selection for callers that cannot allocate device memory: no context and no
@@ -347,8 +353,9 @@ def mrp_reveal_remask_noalloc(conf, token, row_index, M, K, B, L, mode, tau=0.9,
                       (draft_pos, torch.int32, "draft_pos"), (draft_tok, torch.int32, "draft_tok"),
                       (draft_len, torch.int32, "draft_len"), (status, torch.int32, "status")):
         _check(t, dt, nm)
+    _check(conf_first, torch.float32, "conf_first")
     p = mrp_select_params(int(mode), float(tau), int(r_reveal), int(r_draft), int(bool(use_cap)),
-                          int(remask_policy), int(bool(ensure_progress)))
+                          int(remask_policy), int(bool(ensure_progress)), _ptr(conf_first))
     o = mrp_select_out(_ptr(reveal_mask), _ptr(remask_mask), _ptr(out_token), _ptr(step_of),
                        _ptr(draft_pos), _ptr(draft_tok), _ptr(draft_len), _ptr(status))
     rc = lib.mrp_reveal_remask_noalloc(_ptr(conf), _ptr(token), _ptr(row_index), int(M), int(K),

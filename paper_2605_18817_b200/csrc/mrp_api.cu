@@ -257,7 +257,9 @@ int mrp_reveal_remask(mrp_ctx *ctx, const float *conf, const int32_t *token,
     if (params->mode != MRP_SELECT_STATIC && params->mode != MRP_SELECT_DYNAMIC_REMASK)
         return MRP_ERR_INVALID_ARG;
     if (params->r_reveal < 0 || params->r_draft < 0) return MRP_ERR_INVALID_ARG;
-    if (params->remask_policy != 0 && params->remask_policy != 1) return MRP_ERR_INVALID_ARG;
+    if (params->remask_policy < 0 || params->remask_policy > 3) return MRP_ERR_INVALID_ARG;
+    if (params->mode == MRP_SELECT_DYNAMIC_REMASK && params->remask_policy == 2 && M > 0 && !params->conf_first)
+        return MRP_ERR_INVALID_ARG;
     if (!out->reveal_mask || !out->remask_mask || !out->out_token || !out->step_of || !out->draft_len)
         return MRP_ERR_INVALID_ARG;
     const int Kd = K * params->r_draft;

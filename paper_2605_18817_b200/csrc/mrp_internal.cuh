@@ -152,6 +152,24 @@ __device__ __forceinline__ bool row_ok(int idx, int n_rows_in) { return (unsigne
 cudaError_t launch_combine(Ctx *c, const Partial *partials, int n_slices, int n_rowsteps,
                            const mrp_draft_out &out, int32_t *status, cudaStream_t st,
                            const TopFix *fix = nullptr);
+// Probability, under every step's logits, of the token on top at step 0 (mrp_draft_out.conf_first):
+// l_k[tok_0] = l_0[row, tok_0] + W_lm[tok_0] . x_k exactly in fp32, then exp(l_k[tok_0] - lse_k).  Runs
+// after the combine, which provides token and lse.  x: the stacked LM-head operand rows, either fp32
+// (CUDA-core family: step k >= 1 at row (k-1)*M + m) or bf16 hi + lo (tensor-core family: row k*M + m, lo
+// rows lo_rows further on).
+struct FirstTok {
+    const void *w;            // [V, d], fp32 or bf16
+    int w_bf16;
+    const float *logits0;     // nullptr: base logits computed in the pass (their operand rows are part of x)
+    const int32_t *row_index;
+    int n_rows_in;
+    const void *x;
+    int x_bf16;               // 0: fp32 rows, 1: bf16 hi + lo rows
+    long long lo_rows;
+    int M, K, d, V;
+};
+cudaError_t launch_first_token_prob(Ctx *c, const FirstTok &f, const mrp_draft_out &out, cudaStream_t st);
+
 // CUDA-core family: gather masked rows of `hidden` into fp32 h0f / hcur (xt0: where the step-0
 // operand rows n_0 go when the base logits are computed in the LM-head pass, else nullptr).
 cudaError_t launch_prep(Ctx *c, const void *hidden, const int32_t *row_index, int M,

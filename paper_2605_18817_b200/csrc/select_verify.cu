@@ -165,16 +165,26 @@ select_kernel(const float *__restrict__ conf, const int32_t *__restrict__ token,
         for (uint32_t c = inR; c; c &= c - 1) {
             const int s = __ffs(c) - 1;
             const int m = rows[lane + 32 * s];
-            float c2;
-            if (K == 0) {
-                c2 = conf[m];
-            } else if (p.remask_policy == 1) {
-                c2 = conf[(size_t)K * M + m];
+            bool revoke;
+            if (p.remask_policy == 3) {
+                // the argmax moved away from the revealed token at some step
+                revoke = false;
+                for (int k = 1; k <= K; ++k) revoke |= token[(size_t)k * M + m] != token[m];
             } else {
-                c2 = conf[(size_t)M + m];
-                for (int k = 2; k <= K; ++k) c2 = fminf(c2, conf[(size_t)k * M + m]);
+                // policy 2 follows the revealed token's own probability instead of the top one
+                const float *cu = (p.remask_policy == 2) ? p.conf_first : conf;
+                float c2;
+                if (K == 0) {
+                    c2 = cu[m];
+                } else if (p.remask_policy == 1) {
+                    c2 = cu[(size_t)K * M + m];
+                } else {
+                    c2 = cu[(size_t)M + m];
+                    for (int k = 2; k <= K; ++k) c2 = fminf(c2, cu[(size_t)k * M + m]);
+                }
+                revoke = c2 < p.tau;
             }
-            if (c2 < p.tau) rem |= 1u << s;
+            if (revoke) rem |= 1u << s;
         }
         const int kept = warp_popc(inR & ~rem);
         if (kept == 0 && nR > 0 && p.ensure_progress) {
@@ -413,7 +423,9 @@ extern "C" int mrp_reveal_remask_noalloc(const float *conf, const int32_t *token
     if (params->mode != MRP_SELECT_STATIC && params->mode != MRP_SELECT_DYNAMIC_REMASK)
         return MRP_ERR_INVALID_ARG;
     if (params->r_reveal < 0 || params->r_draft < 0) return MRP_ERR_INVALID_ARG;
-    if (params->remask_policy != 0 && params->remask_policy != 1) return MRP_ERR_INVALID_ARG;
+    if (params->remask_policy < 0 || params->remask_policy > 3) return MRP_ERR_INVALID_ARG;
+    if (params->mode == MRP_SELECT_DYNAMIC_REMASK && params->remask_policy == 2 && M > 0 && !params->conf_first)
+        return MRP_ERR_INVALID_ARG;
     if (!out->reveal_mask || !out->remask_mask || !out->out_token || !out->step_of || !out->draft_len)
         return MRP_ERR_INVALID_ARG;
     const int Kd = K * params->r_draft;

@@ -399,6 +399,57 @@ cudaError_t launch_combine(Ctx *c, const Partial *partials, int n_slices, int n_
                     out.token, out.margin, status, out.status, f);
 }
 
+// ---- conf_first: probability of the step-0 argmax token under every step's logits ----------
+__global__ void first_token_prob_kernel(const FirstTok f, const int32_t *__restrict__ token,
+                                        const float *__restrict__ lse, const float *__restrict__ conf,
+                                        float *__restrict__ conf_first)
+{
+    pdl_trigger();
+    pdl_wait();
+    const int rs = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (rs >= (f.K + 1) * f.M) return;
+    const int k = rs / f.M, m = rs - k * f.M;
+    if (k == 0) {                     // the step-0 token is the top token of step 0
+        if (lane == 0) conf_first[rs] = conf[rs];
+        return;
+    }
+    const int tok = token[m];
+    float dot = 0.f;
+    if (f.x_bf16) {
+        const __nv_bfloat16 *xh = (const __nv_bfloat16 *)f.x + (size_t)rs * f.d;
+        const __nv_bfloat16 *xl = xh + (size_t)f.lo_rows * f.d;
+        const __nv_bfloat16 *wr = (const __nv_bfloat16 *)f.w + (size_t)tok * f.d;
+        for (int j = lane; j < f.d; j += 32)
+            dot = fmaf(__bfloat162float(wr[j]), __bfloat162float(xh[j]) + __bfloat162float(xl[j]), dot);
+    } else {
+        // the row of step k holds h_k - h_0, or n_0 + h_k - h_0 when the base logits are computed in the pass
+        const float *xr = (const float *)f.x + (size_t)(k - 1) * f.M * f.d + (size_t)m * f.d;
+        for (int j = lane; j < f.d; j += 32) {
+            const float wv = f.w_bf16 ? __bfloat162float(((const __nv_bfloat16 *)f.w)[(size_t)tok * f.d + j])
+                                      : ((const float *)f.w)[(size_t)tok * f.d + j];
+            dot = fmaf(wv, xr[j], dot);
+        }
+    }
+    dot = warp_sum(dot);
+    if (lane == 0) {
+        const int idx = f.row_index ? f.row_index[m] : m;
+        const bool have = f.logits0 && (!f.row_index || row_ok(idx, f.n_rows_in));
+        const float l = (have ? f.logits0[(size_t)idx * (size_t)f.V + tok] : 0.f) + dot;
+        conf_first[rs] = fminf(expf(l - lse[rs]), conf[rs]);     // never above the top probability
+    }
+}
+
+cudaError_t launch_first_token_prob(Ctx *c, const FirstTok &f, const mrp_draft_out &out, cudaStream_t st)
+{
+    if (!out.conf_first) return cudaSuccess;
+    const int n = (f.K + 1) * f.M, warps = 4;
+    c->launches++;
+    return launch_k(first_token_prob_kernel, dim3((n + warps - 1) / warps), dim3(warps * 32), 0, st,
+                    !(c->cfg.flags & MRP_FLAG_NO_PDL), f, (const int32_t *)out.token, (const float *)out.lse,
+                    (const float *)out.conf, out.conf_first);
+}
+
 template <typename T>
 static cudaError_t simt_draft_t(Ctx *c, const void *hidden, const float *logits0,
                                 const int32_t *row_index, int M, int K, const mrp_draft_out &out,
@@ -453,7 +504,12 @@ static cudaError_t simt_draft_t(Ctx *c, const void *hidden, const float *logits0
     prof_mark(c, 2, st);
     e = launch_combine(c, partials, grid, (K + 1) * M, out, status, st);
     prof_mark(c, 3, st);
-    return e;
+    if (e != cudaSuccess) return e;
+    FirstTok ft;
+    memset(&ft, 0, sizeof(ft));
+    ft.w = c->w_lm; ft.w_bf16 = c->cfg.dtype == MRP_BF16; ft.logits0 = logits0; ft.row_index = row_index;
+    ft.n_rows_in = c->input_rows; ft.x = xt; ft.x_bf16 = 0; ft.M = M; ft.K = K; ft.d = d; ft.V = V;
+    return launch_first_token_prob(c, ft, out, st);
 }
 
 cudaError_t simt_draft(Ctx *c, const void *hidden, const float *logits0, const int32_t *row_index,

@@ -767,7 +767,12 @@ cudaError_t tc_draft(Ctx *c, const void *hidden, const float *logits0, const int
     if (f16_lm) fix.w = (const __nv_bfloat16 *)c->w_lm;
     e = launch_combine(c, partials, n_slices, (K + 1) * M, out, status, st, &fix);
     prof_mark(c, 3, st);
-    return e;
+    if (e != cudaSuccess) return e;
+    FirstTok ft;
+    memset(&ft, 0, sizeof(ft));
+    ft.w = c->w_lm; ft.w_bf16 = 1; ft.logits0 = logits0; ft.row_index = row_index; ft.n_rows_in = c->input_rows;
+    ft.x = xt; ft.x_bf16 = 1; ft.lo_rows = c->lo_xt; ft.M = M; ft.K = K; ft.d = d; ft.V = V;
+    return launch_first_token_prob(c, ft, out, st);
 }
 
 }  // namespace mrp

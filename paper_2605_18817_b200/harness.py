@@ -45,9 +45,10 @@ class DraftOut:
     logits: torch.Tensor | None
     hidden: torch.Tensor | None
     status: torch.Tensor
+    conf_first: torch.Tensor | None = None
 
 
-def alloc_draft_out(M, K, V, d, device, margin=True, logits=False, hidden=False) -> DraftOut:
+def alloc_draft_out(M, K, V, d, device, margin=True, logits=False, hidden=False, conf_first=False) -> DraftOut:
     f = dict(device=device, dtype=torch.float32)
     return DraftOut(
         torch.empty((K + 1, M), **f), torch.empty((K + 1, M), **f),
@@ -55,12 +56,13 @@ def alloc_draft_out(M, K, V, d, device, margin=True, logits=False, hidden=False)
         torch.empty((K + 1, M), **f) if margin else None,
         torch.empty((K, M, V), **f) if logits else None,
         torch.empty((M, d), **f) if hidden else None,
-        torch.zeros(1, device=device, dtype=torch.int32))
+        torch.zeros(1, device=device, dtype=torch.int32),
+        torch.empty((K + 1, M), **f) if conf_first else None)
 
 
 def draft(ctx, hidden, logits0, row_index, M, K, out: DraftOut, stream=None):
     binding.mrp_draft(ctx, hidden, logits0, row_index, M, K, out.conf, out.lse, out.token,
-                      out.margin, out.logits, out.hidden, out.status, stream=stream)
+                      out.margin, out.logits, out.hidden, out.status, stream=stream, conf_first=out.conf_first)
     return out
 
 
@@ -88,7 +90,8 @@ def commit(ctx, sel, state: BlockState, B, L, Kd, accept_mask=None, stream=None)
 
 def draft_from_hidden(ctx, hidden, final_gamma, row_index, M, K, out: DraftOut, stream=None):
     binding.mrp_draft_from_hidden(ctx, hidden, final_gamma, row_index, M, K, out.conf, out.lse, out.token,
-                                  out.margin, out.logits, out.hidden, out.status, stream=stream)
+                                  out.margin, out.logits, out.hidden, out.status, stream=stream,
+                                  conf_first=out.conf_first)
     return out
 
 

@@ -148,6 +148,8 @@ def _rand_select_case(rng, K, B, L, mask_prob):
         conf[:, 1] = conf[:, 0]
         conf[0, 2] = np.float32(0.5)
     token = rng.integers(0, 1000, (K + 1, M)).astype(np.int32)
+    # in about half of the row-steps the argmax is still the step-0 token
+    token = np.where(rng.random((K + 1, M)) < 0.5, token[:1], token).astype(np.int32)
     return ri, conf, token
 
 
@@ -165,6 +167,8 @@ def _gpu_select(ctx, conf, token, ri, B, L, mode, **kw):
     M = conf.shape[1]
     Kd = K * kw.get("r_draft", 1)
     out = harness.alloc_select_out(B, L, Kd, DEV)
+    if kw.get("conf_first") is not None:
+        kw = dict(kw, conf_first=torch.from_numpy(kw["conf_first"]).to(DEV))
     c = torch.from_numpy(conf).to(DEV)
     t = torch.from_numpy(token).to(DEV)
     r = torch.from_numpy(ri).to(DEV) if ri is not None else None
@@ -194,11 +198,16 @@ def test_select_bit_exact_on_shared_statistics(select_ctx, L):
         g = _gpu_select(select_ctx, conf, token, ri, B, L, binding.MRP_SELECT_STATIC, **kw)
         o = oracle.select(conf, token, ri, B, L, oracle.STATIC, **kw)
         _assert_select_equal(g, o)
+        # the revealed token's own probability: the top probability where the token stayed, less where it moved
+        moved = token != token[:1]
+        conf_first = np.where(moved, conf * np.float32(0.5), conf).astype(np.float32)
         for tau in (0.0, 0.3, 0.5, 0.8, 1.5):
             for cap in (False, True):
-                for policy in (0, 1):
+                for policy in (0, 1, 2, 3):
                     for prog in (True, False):
                         kw = dict(tau=tau, use_cap=cap, remask_policy=policy, ensure_progress=prog)
+                        if policy == 2:
+                            kw["conf_first"] = conf_first
                         g = _gpu_select(select_ctx, conf, token, ri, B, L,
                                         binding.MRP_SELECT_DYNAMIC_REMASK, **kw)
                         o = oracle.select(conf, token, ri, B, L, oracle.DYNAMIC_REMASK, **kw)
@@ -365,6 +374,59 @@ def test_a_wait_that_nothing_completes_gives_up_and_reports():
     out, _ = run_gpu_draft(w, inp, 1, ctx=ctx)
     ref = oracle.draft(inp.hidden, inp.logits0, w.heads, w.w_lm, K=1)
     check_stats(out, ref, "bf16")
+    binding.mrp_destroy(ctx)
+
+
+@pytest.mark.parametrize("dtype,flags,d,F,V,B,L,K", [
+    ("f32", 0, 72, 136, 1000, 5, 3, 3),                                # CUDA-core kernels
+    ("bf16", binding.MRP_FLAG_FORCE_SIMT, 72, 136, 1000, 5, 3, 2),
+    ("bf16", 0, 256, 512, 4096, 2, 4, 3),                              # few-row tensor-core kernels
+    ("bf16", 0, 128, 256, 2048, 30, 4, 3),                             # row-major LM head, fp16 operand
+    ("bf16", binding.MRP_FLAG_EXACT_OPERANDS, 128, 256, 2048, 30, 4, 2),
+])
+def test_probability_of_the_step_zero_token_under_the_updated_logits(dtype, flags, d, F, V, B, L, K):
+    """mrp_draft_out.conf_first against the oracle, with and without base logits handed over, and
+    remask policy 2 / 3 driven by it end to end."""
+    w = synth.make_weights(d, F, V, K, dtype, 61, head_std=0.12 if d < 128 else 0.08)   # residuals that move argmaxes
+    inp = synth.make_inputs(w, B, L, 61, 0.5, 2.5)
+    heads, w_lm = harness.upload_weights(w, DEV)
+    M = B * L
+    ctx = binding.mrp_create(d, F, V, heads, w_lm, max_rows=M, max_seqs=B, block_len=L, flags=flags)
+    hid = harness.to_device(inp.hidden, w.dtype, DEV)
+    l0 = torch.from_numpy(inp.logits0).to(DEV)
+    tol = TOL[dtype]
+    moved_total = 0
+    for from_hidden in (False, True):
+        out = harness.alloc_draft_out(M, K, V, d, DEV, conf_first=True)
+        out.conf_first.fill_(-1.0)
+        if from_hidden:
+            harness.draft_from_hidden(ctx, hid, None, None, M, K, out)
+        else:
+            harness.draft(ctx, hid, l0, None, M, K, out)
+        torch.cuda.synchronize()
+        ref = oracle.draft(inp.hidden, None if from_hidden else inp.logits0, w.heads, w.w_lm, K=K)
+        check_stats(out, ref, dtype)
+        # compare where the step-0 token is unambiguous (else the two sides may follow different tokens)
+        clear0 = ref.margin[0] > 1e-2
+        got = out.conf_first.cpu().numpy().astype(np.float64)
+        assert np.abs(got - ref.conf_first)[:, clear0].max() <= tol
+        assert np.array_equal(got[0], out.conf.cpu().numpy()[0].astype(np.float64))
+        assert np.all(got <= out.conf.cpu().numpy() + 1e-7)
+        moved_total += int((ref.token[1:] != ref.token[:1]).sum())
+        # selection driven by the device's own statistics, policies 2 and 3, bit-exact against the oracle's rules
+        for policy in (2, 3):
+            sel = harness.alloc_select_out(B, L, K, DEV)
+            harness.select(ctx, out.conf, out.token, None, M, K, B, L, binding.MRP_SELECT_DYNAMIC_REMASK, sel,
+                           tau=0.3, remask_policy=policy, conf_first=out.conf_first)
+            torch.cuda.synchronize()
+            osel = oracle.select(out.conf.cpu().numpy(), out.token.cpu().numpy(), None, B, L, oracle.DYNAMIC_REMASK,
+                                 tau=0.3, remask_policy=policy, conf_first=out.conf_first.cpu().numpy())
+            _assert_select_equal(sel, osel)
+    assert moved_total > 0
+    with pytest.raises(binding.MrpError):          # policy 2 needs the array
+        sel = harness.alloc_select_out(B, L, K, DEV)
+        harness.select(ctx, out.conf, out.token, None, M, K, B, L, binding.MRP_SELECT_DYNAMIC_REMASK, sel,
+                       tau=0.3, remask_policy=2)
     binding.mrp_destroy(ctx)
 
 

@@ -298,3 +298,93 @@ def test_from_hidden_matches_library_implementation_with_final_norm():
         np.testing.assert_allclose(r.conf[k], stats[k][0], rtol=0, atol=1e-10)
         np.testing.assert_allclose(r.lse[k], stats[k][1], rtol=0, atol=1e-10)
         np.testing.assert_array_equal(r.token[k], stats[k][2])
+
+
+# ---- probability of the step-0 argmax token under the updated logits (conf_first) ----
+
+def test_conf_first_is_the_softmax_probability_of_the_step_zero_token():
+    # library evaluation from the materialised logits: exp(l_k[tok_0] - logsumexp(l_k))
+    w, inp = small_problem(seed=19, head_std=0.5)
+    r = oracle.draft(inp.hidden, inp.logits0, w.heads, w.w_lm, want_logits=True)
+    assert np.array_equal(r.conf_first[0], r.conf[0])
+    tok0 = r.token[0]
+    rows = np.arange(tok0.size)
+    moved = 0
+    for k in range(1, 4):
+        l = r.logits[k - 1]
+        want = np.exp(l[rows, tok0] - logsumexp(l, axis=1))
+        assert np.allclose(r.conf_first[k], want, rtol=0, atol=1e-14)
+        same = r.token[k] == tok0
+        assert np.array_equal(r.conf_first[k][same], r.conf[k][same])      # still on top: the confidence itself
+        assert np.all(r.conf_first[k][~same] < r.conf[k][~same])           # displaced: strictly below the top
+        moved += int((~same).sum())
+    assert moved > 0                                                        # the case is exercised
+
+
+def test_conf_first_with_zero_residual_heads_stays_at_the_backbone_confidence():
+    w, inp = small_problem()
+    for hd in w.heads:
+        hd["w_down"] = np.zeros_like(hd["w_down"])
+    r = oracle.draft(inp.hidden, inp.logits0, w.heads, w.w_lm)
+    for k in range(4):
+        assert np.array_equal(r.conf_first[k], r.conf[0])
+
+
+# ---- the training objective: forward KL of the teacher against the corrected logits (Eq. (3)) ----
+
+def _teacher(rng, logits, scale):
+    """Teacher logits near the corrected logits (the residual is a small correction, Sec. 3.1)."""
+    return (logits + scale * rng.standard_normal(logits.shape)).astype(np.float32)
+
+
+def test_kl_matches_library_relative_entropy_and_is_zero_on_equal_distributions():
+    from scipy.special import rel_entr, softmax
+    w, inp = small_problem(seed=23, head_std=0.4)
+    K, M, V = 3, inp.hidden.shape[0], w.V
+    base = oracle.draft(inp.hidden, inp.logits0, w.heads, w.w_lm, want_logits=True)
+    rng = np.random.default_rng(5)
+    teacher = _teacher(rng, base.logits, 0.7)
+    r, kl = oracle.draft_kl(inp.hidden, inp.logits0, teacher, w.heads, w.w_lm)
+    assert np.array_equal(r.conf, base.conf) and np.array_equal(r.token, base.token)
+    want = rel_entr(softmax(teacher.astype(np.float64), axis=2), softmax(base.logits, axis=2)).sum(axis=2)
+    assert kl.shape == (K, M) and np.all(kl > 0)
+    assert np.allclose(kl, want, rtol=1e-10, atol=1e-13)
+    # the direction matters: KL(q || p) differs
+    other = rel_entr(softmax(base.logits, axis=2), softmax(teacher.astype(np.float64), axis=2)).sum(axis=2)
+    assert np.abs(other - want).max() > 1e-3
+    # a teacher that equals the corrected logits up to a constant per row is the same distribution: KL = 0
+    # (the logits are unnormalised log-densities: the normalising constants cancel)
+    # (fp32-exact inputs so that "equal" is exact: heads that produce nothing)
+    for hd in w.heads:
+        hd["w_down"] = np.zeros_like(hd["w_down"])
+    t0 = np.repeat(inp.logits0[None, :, :], K, axis=0) + np.float32(2.5)
+    _, kl0 = oracle.draft_kl(inp.hidden, inp.logits0, t0, w.heads, w.w_lm)
+    assert np.abs(kl0).max() < 1e-12
+
+
+def test_kl_two_token_closed_form():
+    # V = 2, zero heads: KL((a, 1-a) || (b, 1-b)) = a ln(a/b) + (1-a) ln((1-a)/(1-b)), with a, b the
+    # logistic function of the logit differences
+    d, F, V = 8, 8, 2
+    w = synth.make_weights(d, F, V, 1, "f32", 3)
+    w.heads[0]["w_down"] = np.zeros_like(w.heads[0]["w_down"])
+    hidden = np.ones((2, d), np.float32)
+    logits0 = np.array([[0.5, -0.25], [2.0, 3.0]], np.float32)
+    teacher = np.array([[[1.5, 0.0], [-1.0, 0.5]]], np.float32)
+    _, kl = oracle.draft_kl(hidden, logits0, teacher, w.heads, w.w_lm)
+    for m in range(2):
+        a = 1.0 / (1.0 + math.exp(-(float(teacher[0, m, 0]) - float(teacher[0, m, 1]))))
+        b = 1.0 / (1.0 + math.exp(-(float(logits0[m, 0]) - float(logits0[m, 1]))))
+        want = a * math.log(a / b) + (1 - a) * math.log((1 - a) / (1 - b))
+        assert abs(kl[0, m] - want) < 1e-14
+
+
+def test_kl_row_index_and_chain_truncation():
+    w, inp = small_problem(seed=29, rows=7)
+    rng = np.random.default_rng(8)
+    full = oracle.draft(inp.hidden, inp.logits0, w.heads, w.w_lm, want_logits=True)
+    teacher = _teacher(rng, full.logits, 0.5)
+    _, kl = oracle.draft_kl(inp.hidden, inp.logits0, teacher, w.heads, w.w_lm)
+    sub = np.array([5, 0, 3], np.int32)
+    _, kl_sub = oracle.draft_kl(inp.hidden, inp.logits0, teacher[:2][:, sub], w.heads, w.w_lm, K=2, row_index=sub)
+    assert np.array_equal(kl_sub, kl[:2][:, sub])

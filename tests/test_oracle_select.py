@@ -298,3 +298,65 @@ def test_commit_positionwise_acceptance_keeps_a_later_match():
     alen, amask = oracle.verify(sel.draft_tok, verify_tok, sel.draft_len, positionwise=True)
     assert alen.tolist() == [1] and amask.tolist() == [[0, 1]]
     assert oracle.commit(tokens, sel, 1, 4, accept_mask=amask).tokens.tolist() == [1, -1, 23, -1]
+
+
+def test_remask_by_the_revealed_token_hand_example():
+    # one block of four masked positions, K = 2, tau = 0.5.  Position 0: stays confident and on the same
+    # token.  Position 1: the top probability stays high but moves to another token at step 2, the
+    # revealed token's own probability falls to 0.1.  Position 2: same token, confidence dips below tau
+    # at step 1.  Position 3: never clears tau.
+    conf = np.array([[0.9, 0.8, 0.7, 0.3],
+                     [0.9, 0.8, 0.4, 0.3],
+                     [0.9, 0.85, 0.7, 0.3]], np.float32)
+    token = np.array([[5, 6, 7, 8],
+                      [5, 6, 7, 8],
+                      [5, 9, 7, 8]], np.int32)
+    conf_first = np.array([[0.9, 0.8, 0.7, 0.3],
+                           [0.9, 0.8, 0.4, 0.3],
+                           [0.9, 0.1, 0.7, 0.3]], np.float32)
+    want = {0: [0, 0, 1, 0],      # updated top-1 probability, all steps
+            1: [0, 0, 0, 0],      # updated top-1 probability, last step
+            2: [0, 1, 1, 0],      # probability of the revealed token, all steps
+            3: [0, 1, 0, 0]}      # the argmax left the revealed token
+    for policy, remask in want.items():
+        s = oracle.select(conf, token, None, 1, 4, oracle.DYNAMIC_REMASK, tau=0.5, remask_policy=policy,
+                          conf_first=conf_first)
+        assert list(s.reveal_mask) == [1, 1, 1, 0], policy
+        assert list(s.remask_mask) == remask, policy
+        assert list(s.out_token) == [5 if not remask[0] else -1, 6 if not remask[1] else -1,
+                                     7 if not remask[2] else -1, -1], policy
+
+
+def test_remask_by_the_revealed_token_relations_between_the_policies():
+    rng = np.random.default_rng(21)
+    K, B, L = 3, 8, 16
+    mask, ri, conf, token = random_stats(rng, K, B, L)
+    M = ri.size
+    # tokens move away from the step-0 token in some row-steps; where they stay, the revealed token's
+    # probability is the top probability, where they move it is strictly smaller
+    moved = rng.random((K + 1, M)) < 0.3
+    moved[0] = False
+    token = np.where(moved, token[0][None, :] + 1, token[0][None, :]).astype(np.int32)
+    conf_first = np.where(moved, conf * rng.random((K + 1, M)).astype(np.float32) * 0.9, conf).astype(np.float32)
+    for tau in (0.3, 0.5, 0.7):
+        kw = dict(tau=tau, ensure_progress=False)
+        p0 = oracle.select(conf, token, ri, B, L, oracle.DYNAMIC_REMASK, remask_policy=0, **kw)
+        p2 = oracle.select(conf, token, ri, B, L, oracle.DYNAMIC_REMASK, remask_policy=2, conf_first=conf_first, **kw)
+        p3 = oracle.select(conf, token, ri, B, L, oracle.DYNAMIC_REMASK, remask_policy=3, **kw)
+        assert np.array_equal(p0.reveal_mask, p2.reveal_mask) and np.array_equal(p0.reveal_mask, p3.reveal_mask)
+        # the revealed token's probability never exceeds the top probability: policy 2 revokes a superset
+        assert np.all(p2.remask_mask >= p0.remask_mask)
+        # policy 3 from its definition: revealed and moved at some step
+        dense_moved = np.zeros(B * L, bool)
+        dense_moved[ri] = moved[1:].any(axis=0)
+        assert np.array_equal(p3.remask_mask.astype(bool), p3.reveal_mask.astype(bool) & dense_moved)
+        # policy 2 from its definition
+        dense_min = np.full(B * L, 2.0, np.float32)
+        dense_min[ri] = conf_first[1:].min(axis=0)
+        assert np.array_equal(p2.remask_mask.astype(bool), p2.reveal_mask.astype(bool) & (dense_min < np.float32(tau)))
+    # with tokens that never move and conf_first = conf, policy 2 is policy 0 and policy 3 revokes nothing
+    still = np.repeat(token[:1], K + 1, axis=0)
+    a = oracle.select(conf, still, ri, B, L, oracle.DYNAMIC_REMASK, tau=0.5, remask_policy=0)
+    b = oracle.select(conf, still, ri, B, L, oracle.DYNAMIC_REMASK, tau=0.5, remask_policy=2, conf_first=conf)
+    c = oracle.select(conf, still, ri, B, L, oracle.DYNAMIC_REMASK, tau=0.5, remask_policy=3)
+    assert np.array_equal(a.remask_mask, b.remask_mask) and not c.remask_mask.any()
