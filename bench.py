@@ -63,6 +63,9 @@ def parse_args():
     ap.add_argument("--flags", type=int, default=0, help="mrp_config.flags (MRP_FLAG_* bits) for A/B timing")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--fp8-lm", action="store_true",
+                    help="decode-regime workloads: run the LM head on the 8-bit (e4m3, per-row scale) copy of W_lm "
+                         "(MRP_FLAG_FP8_LM); the roofline then counts one byte per LM-head weight")
     ap.add_argument("--from-hidden", action="store_true",
                     help="draft with mrp_draft_from_hidden: the base logits are computed in the LM-head pass "
                          "instead of being an input (no [rows, V] read or host copy)")
@@ -172,7 +175,7 @@ def replica_throughput(dist, device, units_per_rank, seconds):
     return world * units_per_rank / seconds, seconds
 
 
-def lm_head_roofline(cfg, M, lm_ms, peaks, peaks_kind, from_hidden=False):
+def lm_head_roofline(cfg, M, lm_ms, peaks, peaks_kind, from_hidden=False, fp8=False):
     """Roofline of the fused LM-head kernel: algorithmic bytes 2Vd + 4MV + 2KMd (one read of
     the LM head, one read of l_0, the stacked residual rows), flops 2KMVd.  With the base
     logits computed in the pass: bytes 2Vd + 2(K+1)Md, flops 2(K+1)MVd.  The bound is the slower
@@ -181,15 +184,16 @@ def lm_head_roofline(cfg, M, lm_ms, peaks, peaks_kind, from_hidden=False):
     second or more), ``frac_nominal`` against 8 TB/s and 2250 TFLOP/s."""
     V, d, K = cfg["V"], cfg["d"], cfg["K"]
     esz = 4 if cfg["dtype"] == "f32" else 2
-    nbytes = float(esz) * V * d + 4.0 * M * V + float(esz) * K * M * d
+    wsz = 1 if fp8 else esz                       # bytes per LM-head weight (+ 4 bytes of scale per row)
+    nbytes = float(wsz) * V * d + (4.0 * V if fp8 else 0.0) + 4.0 * M * V + float(esz) * K * M * d
     flops = 2.0 * K * M * V * d
     if from_hidden:
-        nbytes = float(esz) * V * d + float(esz) * (K + 1) * M * d
+        nbytes = float(wsz) * V * d + (4.0 * V if fp8 else 0.0) + float(esz) * (K + 1) * M * d
         flops = 2.0 * (K + 1) * M * V * d
     t_hbm = nbytes / (peaks["hbm_gbs"] * 1e9)
     t_tc = flops / (peaks["bf16_tflops_sustained"] * 1e12)
     sec = lm_ms * 1e-3
-    traffic = NCU_TRAFFIC.get(cfg["name"]) if not from_hidden else None
+    traffic = NCU_TRAFFIC.get(cfg["name"]) if not (from_hidden or fp8) else None
     common = {"traffic": traffic[0] if traffic else None, "traffic_source": traffic[1] if traffic else None,
               "kernel": "fused LM head", "kernel_ms": lm_ms, "alg_bytes": nbytes, "alg_flops": flops,
               "units_per_launch": K * M}
@@ -378,7 +382,7 @@ class Bench:
         M = len(inp.row_index)
         static = cfg["mode"] == "static"
         ctx = binding.mrp_create(w.d, w.F, w.V, heads[:cfg["n_heads"]], w_lm, max_rows=B * L, max_seqs=B,
-                                 block_len=L, flags=args.flags)
+                                 block_len=L, flags=args.flags | (binding.MRP_FLAG_FP8_LM if args.fp8_lm else 0))
         hid = harness.to_device(inp.hidden, w.dtype, dev)
         l0 = torch.from_numpy(inp.logits0).to(dev)
         ri = torch.from_numpy(inp.row_index).to(dev)
@@ -476,7 +480,8 @@ class Bench:
         (ms_heads, ms_lm, ms_comb), n_calls = binding.mrp_profile_read(ctx)
         binding.mrp_profile_enable(ctx, False)
         n_calls = max(n_calls, 1)
-        roofline = lm_head_roofline(cfg, M, ms_lm / n_calls, self.peaks, self.peaks_kind, from_hidden=args.from_hidden)
+        roofline = lm_head_roofline(cfg, M, ms_lm / n_calls, self.peaks, self.peaks_kind, from_hidden=args.from_hidden,
+                                    fp8=args.fp8_lm)
         if clocks.get("sm_mhz"):
             roofline["kernel_ms_x_sm_mhz"] = ms_lm / n_calls * clocks["sm_mhz"]
         if cfg["V"] * cfg["d"] <= 40e6:
@@ -506,7 +511,8 @@ class Bench:
             "batches": n_batches, "batch_ms_median": med, "batch_ms_min": batch_ms[0], "batch_ms_max": batch_ms[-1],
             "timed_gpu_seconds": sum(batch_ms) * 1e-3,
             "dtype": "bf16" if cfg["dtype"] == "bf16" else "f32",
-            "config": config_dict(cfg, M, "mrp_draft_from_hidden" if args.from_hidden else "mrp_draft"),
+            "config": config_dict(cfg, M, ("mrp_draft_from_hidden" if args.from_hidden else "mrp_draft") +
+                                  (" on the 8-bit LM head" if args.fp8_lm else "")),
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches[0] * S * n_batches,
             "launches_per_step": launches[0], "roofline": roofline, "phases": phases, "cpu_baseline": cpu,
             "device_status_word": status,

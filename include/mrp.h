@@ -76,6 +76,20 @@ typedef enum { MRP_F32 = 0, MRP_BF16 = 1 } mrp_dtype;
 #define MRP_FLAG_REQUIRE_TENSOR_CORES 32   /* bf16 context: mrp_create fails with MRP_ERR_UNSUPPORTED
                                        instead of falling back to the CUDA-core kernels when the
                                        shape or the alignment rules out the tensor-core kernels  */
+#define MRP_FLAG_TRAINING_KL 64     /* reserve workspace for mrp_draft_kl (the per-slice partial sums of
+                                       the KL objective); without it that entry point returns
+                                       MRP_ERR_UNSUPPORTED                                           */
+#define MRP_FLAG_FP8_LM 128         /* decode-regime contexts ((n_heads + 1) * max_rows <= 32, d % 256 == 0,
+                                       tensor-core shapes): the LM head runs on an 8-bit copy of W_lm made
+                                       at mrp_create, e4m3 values with one power-of-two scale per
+                                       vocabulary row, which halves the dominant weight stream.  The
+                                       context then computes with the dequantised matrix
+                                       W8[v, :] = scale[v] * e4m3(W_lm[v, :] / scale[v]),
+                                       scale[v] = 2^E, E the smallest integer with max|W_lm[v, :]| <=
+                                       448 * 2^E (rounding to nearest, ties to even): its results are
+                                       those of mrp_draft on W8, to the usual tolerances; the difference
+                                       to W_lm itself is the quantisation (relative 2^-4 per weight).
+                                       Other shapes: MRP_ERR_UNSUPPORTED.  Workspace: + vocab * d bytes  */
 #define MRP_FLAG_EXACT_OPERANDS 8   /* tensor-core family: always carry the LM-head activation
                                        operand as a bf16 hi + lo pair (products exact to 2^-17),
                                        also where that doubles the tensor work for nothing.  Without
@@ -190,6 +204,16 @@ int mrp_draft(mrp_ctx *ctx, const void *hidden, const float *logits0, const int3
               int32_t M, int32_t K, const mrp_draft_out *out, void *cuda_stream);
 
 /*
+ * mrp_draft with the backbone logits stored as bf16: logits0 [n_rows, V] bf16 (16-byte aligned),
+ * half the bytes of the largest input (Algorithm 2, "h, l <- f(x_t)": engines that keep their LM-head
+ * output in the model's 16-bit type).  The values are taken exactly as stored (promoted to fp32);
+ * everything else, outputs and tolerances included, as mrp_draft.  Errors: INVALID_ARG, CUDA.
+ */
+int mrp_draft_bf16_logits(mrp_ctx *ctx, const void *hidden, const void *logits0_bf16,
+                          const int32_t *row_index, int32_t M, int32_t K, const mrp_draft_out *out,
+                          void *cuda_stream);
+
+/*
  * The drafting pass when the backbone hands over hidden states only.  In Algorithm 2 the
  * hidden states and the logits come out of the same forward ("h, l <- f(x_t)") and the module
  * reuses the backbone's LM head (Sec. 3.2); here that head is applied once for both: the pass
@@ -205,6 +229,26 @@ int mrp_draft(mrp_ctx *ctx, const void *hidden, const float *logits0, const int3
 int mrp_draft_from_hidden(mrp_ctx *ctx, const void *hidden, const void *final_norm_gamma,
                           const int32_t *row_index, int32_t M, int32_t K, const mrp_draft_out *out,
                           void *cuda_stream);
+
+/*
+ * The drafting pass with the training objective fused into the LM-head epilogue (Algorithm 1, last
+ * lines; Eq. (3); Sec. 4.1: K unrolled iterations, uniform per-step weight, forward direction,
+ * temperature 1, masked positions only).  Besides everything mrp_draft computes,
+ *     kl[(k-1)*M + m] = KL( softmax(teacher[k-1, m, :]) || softmax(l_k[m, :]) ),   k = 1..K,
+ * where l_k = l_0 + W_lm (h_k - h_0) are the corrected logits of unrolled step k and teacher holds the
+ * frozen backbone's logits on the sequence with that step's ground-truth tokens revealed (l_{t-1} in
+ * the paper's one-step notation).  The two log-sum-exps and the cross term
+ * sum_v softmax(teacher)_v (teacher_v - l_v) are accumulated online, tile by tile, next to the
+ * softmax statistics: neither V-wide row is ever written.
+ *   teacher [K, M, V] fp32 DEVICE, rows compacted like the outputs (row (k-1)*M + m)
+ *   kl      [K, M]    fp32 DEVICE
+ * The other arguments are those of mrp_draft.  The LM head runs on exact (bf16 hi + lo) operands
+ * whatever the context's flags.  Needs a context created with MRP_FLAG_TRAINING_KL and K >= 1.
+ * Errors: INVALID_ARG, UNSUPPORTED, CUDA.  (The backward pass is outside this library.)
+ */
+int mrp_draft_kl(mrp_ctx *ctx, const void *hidden, const float *logits0, const float *teacher,
+                 const int32_t *row_index, int32_t M, int32_t K, const mrp_draft_out *out, float *kl,
+                 void *cuda_stream);
 
 typedef enum { MRP_SELECT_STATIC = 0, MRP_SELECT_DYNAMIC_REMASK = 1 } mrp_select_mode;
 
@@ -378,6 +422,13 @@ int mrp_set_input_rows(mrp_ctx *ctx, int32_t n_rows);
  * Never synchronises.  Errors: INVALID_ARG, CUDA.
  */
 int mrp_fetch_status(mrp_ctx *ctx, int32_t *dst, int32_t clear, void *cuda_stream);
+
+/*
+ * The 8-bit copy of the LM head of a context created with MRP_FLAG_FP8_LM: *codes receives the DEVICE
+ * pointer to the e4m3 bytes [vocab, d], *scales the DEVICE pointer to the fp32 row scales [vocab]
+ * (both inside the workspace, valid for the context's life).  Errors: INVALID_ARG, UNSUPPORTED.
+ */
+int mrp_quantised_lm_head(mrp_ctx *ctx, const uint8_t **codes, const float **scales);
 
 /*
  * Let mrp_draft wait for the base logits separately from the hidden states.  In Algorithm 2

@@ -25,6 +25,8 @@ MRP_FLAG_ROW_MAJOR_ONLY = 4
 MRP_FLAG_EXACT_OPERANDS = 8
 MRP_FLAG_NO_CHAIN = 16
 MRP_FLAG_REQUIRE_TENSOR_CORES = 32
+MRP_FLAG_TRAINING_KL = 64
+MRP_FLAG_FP8_LM = 128
 MRP_SELECT_STATIC, MRP_SELECT_DYNAMIC_REMASK = 0, 1
 MRP_DEV_NONFINITE, MRP_DEV_TIMEOUT, MRP_DEV_BAD_INDEX, MRP_DEV_RANGE = 1, 2, 4, 8
 MRP_RANGE_LIMIT = 32768.0
@@ -33,7 +35,7 @@ EXPORTS = ("mrp_workspace_bytes", "mrp_create", "mrp_destroy", "mrp_draft", "mrp
            "mrp_verify", "mrp_last_launch_count", "mrp_kernel_family", "mrp_status_string",
            "mrp_profile_enable", "mrp_profile_read", "mrp_last_error",
            "mrp_reveal_remask_noalloc", "mrp_selftest_wait_timeout", "mrp_draft_from_hidden", "mrp_commit",
-           "mrp_set_logits0_event", "mrp_set_input_rows", "mrp_fetch_status")
+           "mrp_set_logits0_event", "mrp_set_input_rows", "mrp_fetch_status", "mrp_draft_kl", "mrp_draft_bf16_logits", "mrp_quantised_lm_head")
 MRP_NOALLOC_MAX_POSITIONS = 65536
 MRP_ERR_CAPACITY = 7
 
@@ -97,6 +99,14 @@ def _load():
     lib.mrp_draft.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
                               ctypes.c_int32, ctypes.c_int32, ctypes.POINTER(mrp_draft_out),
                               ctypes.c_void_p]
+    lib.mrp_draft_bf16_logits.restype = ctypes.c_int
+    lib.mrp_draft_bf16_logits.argtypes = lib.mrp_draft.argtypes
+    lib.mrp_quantised_lm_head.restype = ctypes.c_int
+    lib.mrp_quantised_lm_head.argtypes = [ctypes.c_void_p, ctypes.POINTER(ctypes.c_void_p), ctypes.POINTER(ctypes.c_void_p)]
+    lib.mrp_draft_kl.restype = ctypes.c_int
+    lib.mrp_draft_kl.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                                 ctypes.c_int32, ctypes.c_int32, ctypes.POINTER(mrp_draft_out), ctypes.c_void_p,
+                                 ctypes.c_void_p]
     lib.mrp_set_logits0_event.restype = ctypes.c_int
     lib.mrp_set_logits0_event.argtypes = [ctypes.c_void_p, ctypes.c_void_p]
     lib.mrp_set_input_rows.restype = ctypes.c_int
@@ -235,6 +245,22 @@ def workspace_guards_intact(ctx: Context) -> bool:
     return bool((before == 0xA5).all().item()) and bool((after == 0xA5).all().item())
 
 
+def mrp_quantised_lm_head(ctx: Context):
+    """Host copies (uint8 codes [V, d], float32 scales [V]) of the 8-bit LM head of an MRP_FLAG_FP8_LM context."""
+    codes, scales = ctypes.c_void_p(), ctypes.c_void_p()
+    rc = lib.mrp_quantised_lm_head(ctx.handle, ctypes.byref(codes), ctypes.byref(scales))
+    if rc != 0:
+        raise MrpError("mrp_quantised_lm_head", rc)
+    V, d = ctx.cfg.vocab, ctx.cfg.d
+    dev = "cuda:%d" % ctx.cfg.device
+    c = torch.empty((V, d), dtype=torch.uint8, device=dev)
+    s = torch.empty(V, dtype=torch.float32, device=dev)
+    ws = ctx.guards[0]          # the tensor that holds the workspace: the two pointers lie inside it
+    c.copy_(ws[codes.value - ws.data_ptr():codes.value - ws.data_ptr() + V * d].view(V, d))
+    s.copy_(ws[scales.value - ws.data_ptr():scales.value - ws.data_ptr() + 4 * V].view(torch.float32))
+    return c.cpu().numpy(), s.cpu().numpy()
+
+
 def mrp_set_input_rows(ctx: Context, n_rows: int) -> None:
     rc = lib.mrp_set_input_rows(ctx.handle, int(n_rows))
     if rc != 0:
@@ -274,9 +300,11 @@ def mrp_profile_read(ctx: Context):
 
 def mrp_draft(ctx: Context, hidden, logits0, row_index, M, K, conf, lse, token, margin=None,
               logits_out=None, hidden_out=None, status=None, stream=None, conf_first=None) -> None:
-    """Enqueue one drafting pass; outputs are written into the given CUDA tensors."""
+    """Enqueue one drafting pass; outputs are written into the given CUDA tensors.  ``logits0`` in
+    float32 goes to mrp_draft, in bfloat16 to mrp_draft_bf16_logits."""
     _check(hidden, torch.float32 if ctx.cfg.dtype == MRP_F32 else torch.bfloat16, "hidden")
-    _check(logits0, torch.float32, "logits0")
+    l0_bf16 = logits0 is not None and logits0.dtype == torch.bfloat16
+    _check(logits0, torch.bfloat16 if l0_bf16 else torch.float32, "logits0")
     _check(row_index, torch.int32, "row_index")
     for t, dt, nm in ((conf, torch.float32, "conf"), (lse, torch.float32, "lse"),
                       (token, torch.int32, "token"), (margin, torch.float32, "margin"),
@@ -286,10 +314,30 @@ def mrp_draft(ctx: Context, hidden, logits0, row_index, M, K, conf, lse, token, 
         _check(t, dt, nm)
     out = mrp_draft_out(_ptr(conf), _ptr(lse), _ptr(token), _ptr(margin), _ptr(logits_out),
                         _ptr(hidden_out), _ptr(status), _ptr(conf_first))
-    rc = lib.mrp_draft(ctx.handle, _ptr(hidden), _ptr(logits0), _ptr(row_index), int(M), int(K),
-                       ctypes.byref(out), _stream(stream))
+    fn = lib.mrp_draft_bf16_logits if l0_bf16 else lib.mrp_draft
+    rc = fn(ctx.handle, _ptr(hidden), _ptr(logits0), _ptr(row_index), int(M), int(K),
+            ctypes.byref(out), _stream(stream))
     if rc != 0:
         raise MrpError("mrp_draft", rc, lib.mrp_last_error(ctx.handle).decode())
+
+
+def mrp_draft_kl(ctx: Context, hidden, logits0, teacher, row_index, M, K, conf, lse, token, kl, margin=None,
+                 hidden_out=None, status=None, stream=None) -> None:
+    """The drafting pass with the KL objective of every unrolled step fused into the LM-head epilogue:
+    ``teacher`` [K, M, V] fp32, ``kl`` [K, M] fp32 (context created with MRP_FLAG_TRAINING_KL)."""
+    _check(hidden, torch.float32 if ctx.cfg.dtype == MRP_F32 else torch.bfloat16, "hidden")
+    _check(logits0, torch.float32, "logits0")
+    _check(teacher, torch.float32, "teacher")
+    _check(row_index, torch.int32, "row_index")
+    for t, dt, nm in ((conf, torch.float32, "conf"), (lse, torch.float32, "lse"), (token, torch.int32, "token"),
+                      (kl, torch.float32, "kl"), (margin, torch.float32, "margin"),
+                      (hidden_out, torch.float32, "hidden_out"), (status, torch.int32, "status")):
+        _check(t, dt, nm)
+    out = mrp_draft_out(_ptr(conf), _ptr(lse), _ptr(token), _ptr(margin), None, _ptr(hidden_out), _ptr(status), None)
+    rc = lib.mrp_draft_kl(ctx.handle, _ptr(hidden), _ptr(logits0), _ptr(teacher), _ptr(row_index), int(M), int(K),
+                          ctypes.byref(out), _ptr(kl), _stream(stream))
+    if rc != 0:
+        raise MrpError("mrp_draft_kl", rc, lib.mrp_last_error(ctx.handle).decode())
 
 
 def mrp_draft_from_hidden(ctx: Context, hidden, final_norm_gamma, row_index, M, K, conf, lse, token,

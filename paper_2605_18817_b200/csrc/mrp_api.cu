@@ -37,6 +37,13 @@ WorkspaceLayout workspace_layout(const mrp_config &cfg)
                 cfg.d_ff % 64 == 0 && cfg.vocab % 16 == 0;
     l.w16 = take(l.has_f16 ? (size_t)cfg.vocab * d * 2 : 0);
     l.xt16 = take(l.has_f16 ? (size_t)steps * rows * d * 2 : 0);
+    l.kl_partials = take((cfg.flags & MRP_FLAG_TRAINING_KL)
+                             ? (size_t)l.n_slices_max * (size_t)cfg.n_heads * rows * sizeof(KlPartial) : 0);
+    const bool fp8 = (cfg.flags & MRP_FLAG_FP8_LM) != 0;
+    l.w8 = take(fp8 ? (size_t)cfg.vocab * d : 0);
+    l.w8_scale = take(fp8 ? (size_t)cfg.vocab * 4 : 0);
+    l.xq = take(fp8 ? (size_t)4 * 32 * d : 0);
+    l.x8_scale = take(fp8 ? 32 * 4 : 0);
     l.total = off;
     return l;
 }
@@ -129,12 +136,18 @@ int mrp_create(const mrp_config *cfg, const mrp_head_weights *heads, const void 
     if ((cfg->flags & MRP_FLAG_REQUIRE_TENSOR_CORES) && !c.use_tc) {
         free(c.heads); delete ctx; return MRP_ERR_UNSUPPORTED;
     }
+    if ((cfg->flags & MRP_FLAG_FP8_LM) && (!c.use_tc || !fp8_lm_supported(*cfg))) {
+        free(c.heads); delete ctx; return MRP_ERR_UNSUPPORTED;
+    }
     {
         const long long dense = (long long)cfg->max_seqs * cfg->block_len;
         c.input_rows = (int)(dense > cfg->max_rows ? dense : cfg->max_rows);
     }
     if (c.use_tc) {
         if (tc_create(&c) != cudaSuccess) { free(c.heads); delete ctx; return MRP_ERR_CUDA; }
+        if ((cfg->flags & MRP_FLAG_FP8_LM) && fp8_lm_create(&c) != cudaSuccess) {
+            tc_destroy(&c); free(c.heads); delete ctx; return MRP_ERR_CUDA;
+        }
     }
     if (cudaMemset(c.ws + lay.status, 0, 64 * sizeof(int32_t)) != cudaSuccess) {
         if (c.use_tc) tc_destroy(&c);
@@ -210,13 +223,18 @@ void mrp_destroy(mrp_ctx *ctx)
 
 static int draft_call(mrp_ctx *ctx, const void *hidden, const float *logits0, bool from_hidden,
                       const void *final_gamma, const int32_t *row_index, int32_t M, int32_t K,
-                      const mrp_draft_out *out, void *cuda_stream)
+                      const mrp_draft_out *out, void *cuda_stream, const float *teacher = nullptr,
+                      float *kl = nullptr, bool l0_bf16 = false)
 {
     if (!ctx || !out) return MRP_ERR_INVALID_ARG;
     Ctx &c = ctx->c;
+    c.teacher = teacher;
+    c.kl_out = kl;
+    c.l0_bf16 = l0_bf16;
     if (M < 0 || M > c.cfg.max_rows || K < 0 || K > c.cfg.n_heads) return MRP_ERR_INVALID_ARG;
     c.launches = 0;
     if (M == 0) return MRP_OK;
+    if (c.use_fp8_lm && (K < 1 || teacher)) return MRP_ERR_UNSUPPORTED;   // the 8-bit LM head serves drafting passes with K >= 1
     if (!hidden || (!from_hidden && !logits0) || !out->conf || !out->lse || !out->token) return MRP_ERR_INVALID_ARG;
     if (!row_index && M > c.input_rows) return MRP_ERR_INVALID_ARG;      // rows 0..M-1 must exist
     if (((uintptr_t)hidden & 15u) || ((uintptr_t)logits0 & 15u)) return MRP_ERR_INVALID_ARG;
@@ -236,6 +254,23 @@ int mrp_draft(mrp_ctx *ctx, const void *hidden, const float *logits0, const int3
               int32_t M, int32_t K, const mrp_draft_out *out, void *cuda_stream)
 {
     return draft_call(ctx, hidden, logits0, false, nullptr, row_index, M, K, out, cuda_stream);
+}
+
+int mrp_draft_bf16_logits(mrp_ctx *ctx, const void *hidden, const void *logits0_bf16, const int32_t *row_index,
+                          int32_t M, int32_t K, const mrp_draft_out *out, void *cuda_stream)
+{
+    return draft_call(ctx, hidden, (const float *)logits0_bf16, false, nullptr, row_index, M, K, out, cuda_stream,
+                      nullptr, nullptr, true);
+}
+
+int mrp_draft_kl(mrp_ctx *ctx, const void *hidden, const float *logits0, const float *teacher,
+                 const int32_t *row_index, int32_t M, int32_t K, const mrp_draft_out *out, float *kl,
+                 void *cuda_stream)
+{
+    if (!ctx) return MRP_ERR_INVALID_ARG;
+    if (!(ctx->c.cfg.flags & MRP_FLAG_TRAINING_KL)) return MRP_ERR_UNSUPPORTED;
+    if (K < 1 || (M > 0 && (!teacher || !kl)) || ((uintptr_t)teacher & 15u)) return MRP_ERR_INVALID_ARG;
+    return draft_call(ctx, hidden, logits0, false, nullptr, row_index, M, K, out, cuda_stream, teacher, kl);
 }
 
 int mrp_draft_from_hidden(mrp_ctx *ctx, const void *hidden, const void *final_norm_gamma,
@@ -288,6 +323,15 @@ int mrp_verify(mrp_ctx *ctx, const int32_t *draft_tok, const int32_t *verify_tok
     cudaError_t e = launch_verify(&c, draft_tok, verify_tok, draft_len, B, Kd, positionwise ? 1 : 0,
                                   accept_len, accept_mask, (cudaStream_t)cuda_stream);
     return e == cudaSuccess ? MRP_OK : MRP_ERR_CUDA;
+}
+
+int mrp_quantised_lm_head(mrp_ctx *ctx, const uint8_t **codes, const float **scales)
+{
+    if (!ctx || !codes || !scales) return MRP_ERR_INVALID_ARG;
+    if (!ctx->c.use_fp8_lm) return MRP_ERR_UNSUPPORTED;
+    *codes = (const uint8_t *)(ctx->c.ws + ctx->c.lay.w8);
+    *scales = (const float *)(ctx->c.ws + ctx->c.lay.w8_scale);
+    return MRP_OK;
 }
 
 int mrp_set_input_rows(mrp_ctx *ctx, int32_t n_rows)

@@ -17,6 +17,13 @@ struct __align__(16) Partial {
     float second;  // second largest logit of the slice (-inf if none)
 };
 
+// Partial sums of the KL objective of one (step, row) over a slice of the vocabulary: with t the
+// teacher logits and l the corrected logits, mx = max_v t_v, sum = sum_v exp(t_v - mx),
+// cross = sum_v exp(t_v - mx) (t_v - l_v).  KL = cross / sum - (mx + ln sum) + lse(l).
+struct __align__(16) KlPartial {
+    float mx, sum, cross, pad;
+};
+
 __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 // Regions of the caller-provided workspace (byte offsets, each 256-byte aligned).
@@ -35,6 +42,11 @@ struct WorkspaceLayout {
     size_t ssq_fix;     // uint64 [5][128]: sums of squares per (head, row) in 2^-24 fixed point (chain kernel)
     size_t w16;         // fp16 [V, d] copy of the LM head (0 bytes unless the fp16 LM path can run)
     size_t xt16;        // fp16 [n_heads*max_rows, d] rows h_k - h_0 for that path
+    size_t kl_partials; // KlPartial [n_slices_max, n_heads*max_rows] (0 bytes without MRP_FLAG_TRAINING_KL)
+    size_t w8;          // e4m3 [V, d] copy of the LM head, w8_scale fp32 [V]; xq e4m3 [4 limbs * 32 rows, d] operand
+    size_t w8_scale;    //   limbs, x8_scale fp32 [32] (all 0 bytes without MRP_FLAG_FP8_LM)
+    size_t xq;
+    size_t x8_scale;
     bool has_f16;
     size_t total;
     int32_t n_slices_max;
@@ -58,12 +70,16 @@ struct Ctx {
     WorkspaceLayout lay;
     bool use_tc;
     bool use_f16_lm;           // the fp16 copy of W_lm exists and is usable
+    bool use_fp8_lm;           // MRP_FLAG_FP8_LM: the LM head is the e4m3 copy in the workspace
     // Set per call by mrp_draft_from_hidden: no base logits are given (logits0 == nullptr); the
     // LM-head pass computes them as W_lm n_0, n_0 = h_0 or RMSNorm(h_0) * final_gamma.
     bool from_hidden;
     const void *final_gamma;
     cudaEvent_t l0_event;      // mrp_set_logits0_event: awaited right before the LM-head kernel, or nullptr
     int input_rows;            // rows of the caller's hidden / logits0 arrays: row_index entries must be below
+    bool l0_bf16;              // set per call by mrp_draft_bf16_logits: logits0 points to bf16 values
+    const float *teacher;      // set per call by mrp_draft_kl: teacher logits [K, M, V], else nullptr
+    float *kl_out;             // [K, M]
     // Row offset of the bf16 lo block behind the hi block in this call's operand buffers: M and
     // (K+1)M for the row-major kernels, the padded row count for the few-row kernels (which then
     // fetch hi and lo rows of a k-chunk with one TMA box).
@@ -134,6 +150,12 @@ cudaError_t simt_draft(Ctx *c, const void *hidden, const float *logits0, const i
 // LM-head operands were rounded to fp16): l_top = l_0[row, tok] + W_lm[tok] . (h_k - h_0) in
 // fp32 from the bf16 hi + lo rows, which removes the dominant token's rounding error from
 // log-sum-exp and confidence.  w == nullptr: off.
+// Element i of the caller's base logits, stored as fp32 or (is_bf16) as bf16.
+__device__ __forceinline__ float ld_l0(const float *l0, int is_bf16, size_t i)
+{
+    return is_bf16 ? __bfloat162float(__ldg(reinterpret_cast<const __nv_bfloat16 *>(l0) + i)) : __ldg(l0 + i);
+}
+
 struct TopFix {
     const __nv_bfloat16 *w;      // [V, d]; nullptr: no recomputation
     const __nv_bfloat16 *xt;     // hi rows [n_rs, d] of the stacked LM-head operand, row-step major, then (from
@@ -142,6 +164,7 @@ struct TopFix {
     const int32_t *row_index;
     int d, V, M, n_rs;
     int n_rows_in;               // row_index entries at or above are invalid (their l_0 reads as zero)
+    int l0_bf16;                 // logits0 holds bf16 values
     float range_limit;           // > 0: raise MRP_DEV_RANGE for a row-step whose operand has d * rms above it
 };
 
@@ -151,16 +174,18 @@ __device__ __forceinline__ bool row_ok(int idx, int n_rows_in) { return (unsigne
 // Shared by both families: merge per-slice partials into conf/lse/token/margin.
 cudaError_t launch_combine(Ctx *c, const Partial *partials, int n_slices, int n_rowsteps,
                            const mrp_draft_out &out, int32_t *status, cudaStream_t st,
-                           const TopFix *fix = nullptr);
+                           const TopFix *fix = nullptr, int M = 0);
 // Probability, under every step's logits, of the token on top at step 0 (mrp_draft_out.conf_first):
 // l_k[tok_0] = l_0[row, tok_0] + W_lm[tok_0] . x_k exactly in fp32, then exp(l_k[tok_0] - lse_k).  Runs
 // after the combine, which provides token and lse.  x: the stacked LM-head operand rows, either fp32
 // (CUDA-core family: step k >= 1 at row (k-1)*M + m) or bf16 hi + lo (tensor-core family: row k*M + m, lo
 // rows lo_rows further on).
 struct FirstTok {
-    const void *w;            // [V, d], fp32 or bf16
+    const void *w;            // [V, d], fp32 or bf16, or (w8_scale set) e4m3 codes with one scale per row
     int w_bf16;
+    const float *w8_scale;
     const float *logits0;     // nullptr: base logits computed in the pass (their operand rows are part of x)
+    int l0_bf16;
     const int32_t *row_index;
     int n_rows_in;
     const void *x;
@@ -209,6 +234,19 @@ cudaError_t sk_chain(Ctx *c, int M, int K, const mrp_draft_out &out, cudaStream_
                      bool check_only);
 cudaError_t sk_lm(Ctx *c, const float *logits0, const int32_t *row_index, int M, int K,
                   const mrp_draft_out &out, cudaStream_t st, bool pdl);
+bool fp8_lm_supported(const mrp_config &cfg);
+cudaError_t fp8_lm_create(Ctx *c);      // quantises W_lm into the workspace (blocking, once)
+
+__device__ inline KlPartial merge_kl(const KlPartial &a, const KlPartial &b)
+{
+    KlPartial r;
+    r.mx = fmaxf(a.mx, b.mx);
+    const float ea = (a.sum == 0.f) ? 0.f : expf(a.mx - r.mx), eb = (b.sum == 0.f) ? 0.f : expf(b.mx - r.mx);
+    r.sum = a.sum * ea + b.sum * eb;
+    r.cross = a.cross * ea + b.cross * eb;
+    r.pad = 0.f;
+    return r;
+}
 
 // Merge of two partial statistics; ties on the maximum go to the lower token id.
 __device__ inline Partial merge_partial(const Partial &a, const Partial &b)

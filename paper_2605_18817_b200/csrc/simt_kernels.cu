@@ -197,7 +197,8 @@ __global__ void __launch_bounds__(256)
 lm_simt_kernel(const T *__restrict__ w_lm, const float *__restrict__ xt, const float *__restrict__ xt0,
                const float *__restrict__ logits0, const int32_t *__restrict__ row_index, int M,
                int K, int d, int V, int n_slices, Partial *__restrict__ partials,
-               float *__restrict__ logits_out, int n_rows_in)
+               float *__restrict__ logits_out, int n_rows_in, const float *__restrict__ teacher,
+               KlPartial *__restrict__ kl_partials, int l0_bf16)
 {
     pdl_trigger();
     pdl_wait();
@@ -239,7 +240,7 @@ lm_simt_kernel(const T *__restrict__ w_lm, const float *__restrict__ xt, const f
                             const int m = rs % M;
                             const int idx = row_index ? row_index[m] : m;
                             const bool have = logits0 && (!row_index || row_ok(idx, n_rows_in));
-                            l = (have ? logits0[(size_t)idx * (size_t)V + v] : 0.f) + s;
+                            l = (have ? ld_l0(logits0, l0_bf16, (size_t)idx * (size_t)V + v) : 0.f) + s;
                         }
                         tile[r][vl] = l;
                     }
@@ -292,6 +293,37 @@ lm_simt_kernel(const T *__restrict__ w_lm, const float *__restrict__ xt, const f
                     if (!first) p = merge_partial(*dst, p);
                     *dst = p;
                 }
+                if (teacher && rs >= M) {
+                    // the slice's share of the KL objective against the teacher logits of this row-step
+                    const float *tr = teacher + (size_t)(rs - M) * V;
+                    float tv[SLICE / 32], tmx = -INFINITY;
+#pragma unroll
+                    for (int i = 0; i < SLICE / 32; ++i) {
+                        const int v = v0 + lane + 32 * i;
+                        tv[i] = v < V ? tr[v] : -INFINITY;
+                        tmx = fmaxf(tmx, tv[i]);
+                    }
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) tmx = fmaxf(tmx, __shfl_xor_sync(0xffffffffu, tmx, o));
+                    float ts = 0.f, tc = 0.f;
+#pragma unroll
+                    for (int i = 0; i < SLICE / 32; ++i) {
+                        if (tv[i] != -INFINITY) {
+                            const float e = expf(tv[i] - tmx);
+                            ts += e;
+                            tc = fmaf(e, tv[i] - vals[i], tc);
+                        }
+                    }
+                    ts = warp_sum(ts);
+                    tc = warp_sum(tc);
+                    if (lane == 0) {
+                        KlPartial q;
+                        q.mx = tmx; q.sum = ts; q.cross = tc; q.pad = 0.f;
+                        KlPartial *dst = kl_partials + (size_t)blockIdx.x * (size_t)(K * M) + (rs - M);
+                        if (!first) q = merge_kl(*dst, q);
+                        *dst = q;
+                    }
+                }
             }
             __syncthreads();
         }
@@ -303,7 +335,8 @@ __global__ void combine_kernel(const Partial *__restrict__ partials, int n_slice
                                float *__restrict__ conf, float *__restrict__ lse,
                                int32_t *__restrict__ token, float *__restrict__ margin,
                                int32_t *__restrict__ status, int32_t *__restrict__ user_status,
-                               const TopFix fix)
+                               const TopFix fix, const KlPartial *__restrict__ kl_partials, int M,
+                               float *__restrict__ kl_out)
 {
     pdl_trigger();
     pdl_wait();
@@ -347,7 +380,7 @@ __global__ void combine_kernel(const Partial *__restrict__ partials, int n_slice
             ssq = fmaf(h2.x, h2.x, fmaf(h2.y, h2.y, ssq));
         }
         dot = warp_sum(dot);
-        top = (have ? fix.logits0[(size_t)idx * (size_t)fix.V + tok] : 0.f) + dot;
+        top = (have ? ld_l0(fix.logits0, fix.l0_bf16, (size_t)idx * (size_t)fix.V + tok) : 0.f) + dot;
     } else if (fix.range_limit > 0.f && has_operand) {
         // only the size of the operand row is needed: 16-byte loads of its hi part (d % 64 == 0)
         const uint4 *xh = reinterpret_cast<const uint4 *>(fix.xt + (size_t)rs * fix.d);
@@ -370,10 +403,28 @@ __global__ void combine_kernel(const Partial *__restrict__ partials, int n_slice
             if (user_status) atomicOr(user_status, MRP_DEV_RANGE);
         }
     }
+    KlPartial kq;
+    kq.mx = -INFINITY; kq.sum = 0.f; kq.cross = 0.f; kq.pad = 0.f;
+    if (kl_out && rs >= M) {
+        // KL objective of the row-step: merge the slices' partial sums in the same fixed order
+        const size_t n_kl = (size_t)(n_rs - M);
+#pragma unroll 4
+        for (int s = lane; s < n_slices; s += 32) kq = merge_kl(kq, kl_partials[(size_t)s * n_kl + (rs - M)]);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            KlPartial q;
+            q.mx = __shfl_xor_sync(0xffffffffu, kq.mx, o);
+            q.sum = __shfl_xor_sync(0xffffffffu, kq.sum, o);
+            q.cross = __shfl_xor_sync(0xffffffffu, kq.cross, o);
+            q.pad = 0.f;
+            kq = (lane & o) ? merge_kl(q, kq) : merge_kl(kq, q);
+        }
+    }
     if (lane == 0) {
         // the term of the top token entered the sum as exp(0) = 1: swap in its exact value
         const float sum = (top == p.mx) ? p.sum : (p.sum - 1.f) + expf(top - p.mx);
         const float l = p.mx + logf(sum);
+        if (kl_out && rs >= M) kl_out[rs - M] = kq.cross / kq.sum - (kq.mx + logf(kq.sum)) + l;
         conf[rs] = (top == p.mx) ? 1.f / sum : expf(top - l);
         lse[rs] = l;
         token[rs] = p.idx;
@@ -386,7 +437,7 @@ __global__ void combine_kernel(const Partial *__restrict__ partials, int n_slice
 }
 
 cudaError_t launch_combine(Ctx *c, const Partial *partials, int n_slices, int n_rowsteps,
-                           const mrp_draft_out &out, int32_t *status, cudaStream_t st, const TopFix *fix)
+                           const mrp_draft_out &out, int32_t *status, cudaStream_t st, const TopFix *fix, int M)
 {
     if (n_rowsteps == 0) return cudaSuccess;
     const int warps = 4;
@@ -396,7 +447,9 @@ cudaError_t launch_combine(Ctx *c, const Partial *partials, int n_slices, int n_
     c->launches++;
     return launch_k(combine_kernel, dim3((n_rowsteps + warps - 1) / warps), dim3(warps * 32), 0, st,
                     !(c->cfg.flags & MRP_FLAG_NO_PDL), partials, n_slices, n_rowsteps, out.conf, out.lse,
-                    out.token, out.margin, status, out.status, f);
+                    out.token, out.margin, status, out.status, f,
+                    (const KlPartial *)(c->teacher ? c->ws + c->lay.kl_partials : nullptr), M,
+                    c->teacher ? c->kl_out : (float *)nullptr);
 }
 
 // ---- conf_first: probability of the step-0 argmax token under every step's logits ----------
@@ -416,7 +469,20 @@ __global__ void first_token_prob_kernel(const FirstTok f, const int32_t *__restr
     }
     const int tok = token[m];
     float dot = 0.f;
-    if (f.x_bf16) {
+    if (f.x_bf16 && f.w8_scale) {
+        // 8-bit LM head: the row of the dequantised matrix, scale[tok] * e4m3 code
+        const __nv_bfloat16 *xh = (const __nv_bfloat16 *)f.x + (size_t)rs * f.d;
+        const __nv_bfloat16 *xl = xh + (size_t)f.lo_rows * f.d;
+        const uint8_t *wr = (const uint8_t *)f.w + (size_t)tok * f.d;
+        for (int j = lane; j < f.d; j += 32) {
+            const uint32_t b = wr[j];
+            const int e = (b >> 3) & 15, mm = b & 7;
+            float wv = e ? __uint_as_float(((uint32_t)(e + 120) << 23) | ((uint32_t)mm << 20)) : (float)mm * 0.001953125f;
+            wv = (b & 0x80u) ? -wv : wv;
+            dot = fmaf(wv, __bfloat162float(xh[j]) + __bfloat162float(xl[j]), dot);
+        }
+        dot *= f.w8_scale[tok];
+    } else if (f.x_bf16) {
         const __nv_bfloat16 *xh = (const __nv_bfloat16 *)f.x + (size_t)rs * f.d;
         const __nv_bfloat16 *xl = xh + (size_t)f.lo_rows * f.d;
         const __nv_bfloat16 *wr = (const __nv_bfloat16 *)f.w + (size_t)tok * f.d;
@@ -435,7 +501,7 @@ __global__ void first_token_prob_kernel(const FirstTok f, const int32_t *__restr
     if (lane == 0) {
         const int idx = f.row_index ? f.row_index[m] : m;
         const bool have = f.logits0 && (!f.row_index || row_ok(idx, f.n_rows_in));
-        const float l = (have ? f.logits0[(size_t)idx * (size_t)f.V + tok] : 0.f) + dot;
+        const float l = (have ? ld_l0(f.logits0, f.l0_bf16, (size_t)idx * (size_t)f.V + tok) : 0.f) + dot;
         conf_first[rs] = fminf(expf(l - lse[rs]), conf[rs]);     // never above the top probability
     }
 }
@@ -460,6 +526,7 @@ static cudaError_t simt_draft_t(Ctx *c, const void *hidden, const float *logits0
     float *xg = (float *)(c->ws + c->lay.xg), *act = (float *)(c->ws + c->lay.act);
     float *xt = (float *)(c->ws + c->lay.xt);
     Partial *partials = (Partial *)(c->ws + c->lay.partials);
+    KlPartial *kl_partials = (KlPartial *)(c->ws + c->lay.kl_partials);
     int32_t *status = (int32_t *)(c->ws + c->lay.status);
     const bool pdl = !(c->cfg.flags & MRP_FLAG_NO_PDL);
     prof_mark(c, 0, st);
@@ -494,20 +561,21 @@ static cudaError_t simt_draft_t(Ctx *c, const void *hidden, const float *logits0
     if (narrow)
         e = launch_k(lm_simt_kernel<T, 32>, dim3(grid), dim3(256), 0, st, pdl, (const T *)c->w_lm, (const float *)xt,
                      (const float *)xt0, logits0, row_index, M, K, d, V, n_slices, partials, out.logits_out,
-                     c->input_rows);
+                     c->input_rows, c->teacher, kl_partials, c->l0_bf16 ? 1 : 0);
     else
         e = launch_k(lm_simt_kernel<T, kSimtSliceV>, dim3(grid), dim3(256), 0, st, pdl, (const T *)c->w_lm,
                      (const float *)xt, (const float *)xt0, logits0, row_index, M, K, d, V, n_slices, partials,
-                     out.logits_out, c->input_rows);
+                     out.logits_out, c->input_rows, c->teacher, kl_partials, c->l0_bf16 ? 1 : 0);
     c->launches++;
     if (e != cudaSuccess) return e;
     prof_mark(c, 2, st);
-    e = launch_combine(c, partials, grid, (K + 1) * M, out, status, st);
+    e = launch_combine(c, partials, grid, (K + 1) * M, out, status, st, nullptr, M);
     prof_mark(c, 3, st);
     if (e != cudaSuccess) return e;
     FirstTok ft;
     memset(&ft, 0, sizeof(ft));
     ft.w = c->w_lm; ft.w_bf16 = c->cfg.dtype == MRP_BF16; ft.logits0 = logits0; ft.row_index = row_index;
+    ft.l0_bf16 = c->l0_bf16 ? 1 : 0;
     ft.n_rows_in = c->input_rows; ft.x = xt; ft.x_bf16 = 0; ft.M = M; ft.K = K; ft.d = d; ft.V = V;
     return launch_first_token_prob(c, ft, out, st);
 }

@@ -102,6 +102,16 @@ __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t da, uint64_t
         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(d_tmem), "l"(da), "l"(db), "r"(idesc), "r"(acc) : "memory");
 }
+// The same MMA on 8-bit floating-point operands (kind::f8f6f4; here both operands e4m3, 32 elements of
+// the contraction per instruction).
+__device__ __forceinline__ void umma_f8(uint32_t d_tmem, uint64_t da, uint64_t db, uint32_t idesc, uint32_t acc)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(da), "l"(db), "r"(idesc), "r"(acc) : "memory");
+}
 // True in exactly one lane of a converged warp, the same lane every time.  The MMA issuer runs
 // its loop with the whole warp and only issues from the elected lane: the loop's barrier waits,
 // fences and commits cost about half as many cycles that way as in a one-lane branch
@@ -175,6 +185,40 @@ __device__ __forceinline__ uint32_t make_idesc_f16(int bn)
 {
     return (1u << 4) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 }
+// Same for kind::f8f6f4 with both operands e4m3 (operand format code 0) -> fp32.
+__device__ __forceinline__ uint32_t make_idesc_e4m3(int bn)
+{
+    return (1u << 4) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+}
+
+// e4m3 (the 8-bit floating-point format with 4 exponent bits of bias 7 and 3 mantissa bits; no
+// infinities, largest finite value 448 = 0x7E, 0x7F = NaN; exponent field 0 = subnormals of spacing
+// 2^-9): round to nearest, ties to even, saturating.
+__device__ __forceinline__ uint32_t f32_to_e4m3(float x)
+{
+    const uint32_t sign = (__float_as_uint(x) >> 24) & 0x80u;
+    const float a = fabsf(x);
+    if (!(a <= 448.f)) return sign | 0x7Eu;
+    if (a < 0.015625f) return sign | (uint32_t)__float2int_rn(a * 512.f);     // 0..8; 8 is the smallest normal
+    uint32_t ua = __float_as_uint(a);
+    ua += 0x7FFFFu + ((ua >> 20) & 1u);          // round the 23-bit mantissa to 3 bits, ties to even
+    return sign | ((((ua >> 23) - 120u) << 3) | ((ua >> 20) & 7u));
+}
+__device__ __forceinline__ float e4m3_to_f32(uint32_t b)
+{
+    const int e = (b >> 3) & 15, m = b & 7;
+    const float v = e ? __uint_as_float(((uint32_t)(e + 120) << 23) | ((uint32_t)m << 20)) : (float)m * 0.001953125f;
+    return (b & 0x80u) ? -v : v;
+}
+// Power of two s = 2^E, E the smallest integer with amax <= 448 * 2^E (1 for amax = 0): the scale that
+// maps a row onto the e4m3 range.
+__device__ __forceinline__ float e4m3_row_scale(float amax)
+{
+    if (!(amax > 0.f)) return 1.f;
+    int e;
+    const float f = frexpf(amax, &e);            // amax = f * 2^e, f in [0.5, 1); 448 = 0.875 * 2^9
+    return ldexpf(1.f, e - 9 + (f > 0.875f ? 1 : 0));
+}
 
 constexpr float kLog2e = 1.4426950408889634f;
 
@@ -219,12 +263,59 @@ struct RowStat {
     }
 };
 
+// Online partial sums of the KL objective of one row (teacher logits t against corrected logits l),
+// updated 16 columns at a time: mx = running max of t, sum = sum exp(t - mx), cross = sum exp(t - mx) (t - l).
+struct KlStat {
+    float mx, sum, cross;
+    __device__ __forceinline__ void init() { mx = -INFINITY; sum = 0.f; cross = 0.f; }
+    __device__ __forceinline__ void update(const float *t, const float *l)
+    {
+        float cmax = t[0];
+#pragma unroll
+        for (int j = 1; j < 16; ++j) cmax = fmaxf(cmax, t[j]);
+        if (cmax > mx) {
+            const float sc = ex2f((mx - cmax) * kLog2e);
+            sum *= sc;
+            cross *= sc;
+            mx = cmax;
+        }
+        const float ms = mx * kLog2e;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+            const float e = ex2f(fmaf(t[j], kLog2e, -ms));
+            sum += e;
+            cross = fmaf(e, t[j] - l[j], cross);
+        }
+    }
+    __device__ __forceinline__ KlPartial partial() const
+    {
+        KlPartial p;
+        p.mx = mx; p.sum = sum; p.cross = cross; p.pad = 0.f;
+        return p;
+    }
+};
+
 __device__ __forceinline__ void load16(const float *p, float *v)
 {
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
         const float4 x = ldg_nc4(p + 4 * i);
         v[4 * i] = x.x; v[4 * i + 1] = x.y; v[4 * i + 2] = x.z; v[4 * i + 3] = x.w;
+    }
+}
+// 16 consecutive bf16 values (32-byte aligned address) as floats
+__device__ __forceinline__ void load16_bf16(const __nv_bfloat16 *p, float *v)
+{
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+        uint4 q;
+        asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(q.x), "=r"(q.y), "=r"(q.z), "=r"(q.w) : "l"(p + 8 * i));
+        const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            v[8 * i + 2 * j] = __uint_as_float(w[j] << 16);
+            v[8 * i + 2 * j + 1] = __uint_as_float(w[j] & 0xFFFF0000u);
+        }
     }
 }
 __device__ __forceinline__ void load16_rw(const float *p, float *v)   // data this kernel also writes
@@ -294,6 +385,19 @@ inline bool make_map(const TcState *s, CUtensorMap *map, const void *ptr, uint64
     cuuint32_t box[2] = {(cuuint32_t)kBK, box_rows};
     cuuint32_t es[2] = {1, 1};
     return s->encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(ptr), dims, strides, box, es,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// 8-bit row-major [rows, inner] matrix, box = [box_rows, 128 bytes], 128-byte swizzle.
+inline bool make_map_u8(const TcState *s, CUtensorMap *map, const void *ptr, uint64_t inner, uint64_t rows,
+                        uint32_t box_rows)
+{
+    cuuint64_t dims[2] = {inner, rows};
+    cuuint64_t strides[1] = {inner};
+    cuuint32_t box[2] = {128u, box_rows};
+    cuuint32_t es[2] = {1, 1};
+    return s->encode(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(ptr), dims, strides, box, es,
                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                      CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }

@@ -59,8 +59,11 @@ struct TcParams {
     const float *logits0;
     const int32_t *row_index;
     int n_rows_in;       // row_index entries at or above are invalid: their base logits read as zero
+    int l0_bf16;         // logits0 holds bf16 values
     Partial *partials;
     float *logits_out;
+    const float *teacher;        // KL variant: teacher logits [K * M, V], row-step order of steps 1..K
+    KlPartial *kl_partials;      // [n_vr][K * M]
     // GU
     const float *sumsq;
     int n_ss;
@@ -84,7 +87,7 @@ struct TcParams {
 // ---------------------------------------------------------------------------------------
 // F16: one fp16 A tile per stage against fp16 weights (LM head only); otherwise the bf16 hi and lo
 // A tiles of a k-chunk against bf16 weights.
-template <int KIND, bool MARGIN, bool F16>
+template <int KIND, bool MARGIN, bool F16, bool KL>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
                const __grid_constant__ CUtensorMap tmB1, const TcParams p)
@@ -237,6 +240,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const int r = mb * 128 + rl;
             const bool valid = r < p.rows;
             RowStat st, st0;       // LM: statistics of the row's own step, and of step 0 (rows of step 1 only)
+            KlStat kst;            // LM, KL variant: the row-step's share of the training objective
+            const float *tp = nullptr;
             bool first_step = false;
             const float *l0p = nullptr;
             int k_of_row = 0, m_of_row = r;
@@ -249,8 +254,15 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     m_of_row = r - (k_of_row - p.step_base) * p.M;
                     first_step = (k_of_row == 1 && p.step_base == 1);
                     const int idx = p.row_index ? p.row_index[m_of_row] : m_of_row;
+                    // (for bf16 base logits l0p is kept in units of two bytes: see the load below)
                     if (p.logits0 && (!p.row_index || row_ok(idx, p.n_rows_in)))
-                        l0p = p.logits0 + (size_t)idx * (size_t)p.V;
+                        l0p = p.l0_bf16 ? reinterpret_cast<const float *>(reinterpret_cast<const __nv_bfloat16 *>(p.logits0) +
+                                                                           (size_t)idx * (size_t)p.V)
+                                        : p.logits0 + (size_t)idx * (size_t)p.V;
+                    if (KL) {
+                        kst.init();
+                        tp = p.teacher + ((size_t)(k_of_row - 1) * p.M + m_of_row) * (size_t)p.V;   // step_base is 1 here
+                    }
                 }
             } else if (KIND == KIND_GU && valid) {
                 float s = 0.f;
@@ -271,12 +283,15 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         float l0[16], a[16];
                         if (valid && p.logits0) {
                             if (l0p) {
-                                load16(l0p + v, l0);
+                                if (p.l0_bf16) load16_bf16(reinterpret_cast<const __nv_bfloat16 *>(l0p) + v, l0);
+                                else load16(l0p + v, l0);
                             } else {          // the caller's row index was out of range: an all-zero logit row
 #pragma unroll
                                 for (int j = 0; j < 16; ++j) l0[j] = 0.f;
                             }
                         }
+                        float tch[16];
+                        if (KL && valid) load16(tp + v, tch);
                         tmem_ld16(tacc + c * 16, a);
                         if (valid) {
                             if (p.logits0) {
@@ -285,6 +300,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                                 for (int j = 0; j < 16; ++j) a[j] += l0[j];
                             }
                             st.template update<MARGIN>(a, v);
+                            if (KL) kst.update(tch, a);
                             if (p.logits_out && k_of_row >= 1)
                                 store16(p.logits_out + ((size_t)(k_of_row - 1) * p.M + m_of_row) * p.V + v, a);
                         }
@@ -351,6 +367,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 if (KIND == KIND_LM) {
                     p.partials[(size_t)vr * p.n_rs + (size_t)k_of_row * p.M + m_of_row] = st.partial();
                     if (first_step) p.partials[(size_t)vr * p.n_rs + m_of_row] = st0.partial();
+                    if (KL)
+                        p.kl_partials[(size_t)vr * ((size_t)p.K * p.M) + (size_t)(k_of_row - 1) * p.M + m_of_row] = kst.partial();
                 } else if (KIND == KIND_DN) {
                     p.sumsq_out[(size_t)vr * p.M + m_of_row] = ssq;
                 }
@@ -535,11 +553,11 @@ size_t smem_bytes(const TcParams &p, int parts)
     return (size_t)p.n_stages * (parts * kATile + b_bytes) + 1024 + 8 * (2 * p.n_stages + 4) + 16;
 }
 
-template <int KIND, bool MARGIN, bool F16 = false>
+template <int KIND, bool MARGIN, bool F16 = false, bool KL = false>
 cudaError_t launch_tc(const CUtensorMap &a, const CUtensorMap &b0, const CUtensorMap &b1, const TcParams &p,
                       int grid, cudaStream_t st, bool pdl)
 {
-    auto kern = tc_gemm_kernel<KIND, MARGIN, F16>;
+    auto kern = tc_gemm_kernel<KIND, MARGIN, F16, KL>;
     const size_t smem = smem_bytes(p, F16 ? 1 : 2);
     // the shared-memory limit of a kernel is set once per device (the attribute is per device)
     static std::atomic<unsigned long long> attr_devices{0};
@@ -638,8 +656,10 @@ cudaError_t tc_draft(Ctx *c, const void *hidden, const float *logits0, const int
     const bool pdl = !(c->cfg.flags & MRP_FLAG_NO_PDL);
     const bool few_rows = sk_head_rows_ok(M) && sk_heads_ok(c->cfg) &&
                           !(c->cfg.flags & MRP_FLAG_ROW_MAJOR_ONLY);
-    const bool lm_few = sk_rows_ok(n_rs) && !(c->cfg.flags & MRP_FLAG_ROW_MAJOR_ONLY);
-    const bool f16_lm = c->use_f16_lm && n_rs >= kF16MinRowSteps && !lm_few;
+    // the KL objective lives in the row-major LM-head kernel, on exact operands
+    const bool with_kl = c->teacher != nullptr;
+    const bool lm_few = sk_rows_ok(n_rs) && !(c->cfg.flags & MRP_FLAG_ROW_MAJOR_ONLY) && !with_kl;
+    const bool f16_lm = c->use_f16_lm && n_rs >= kF16MinRowSteps && !lm_few && !with_kl;
     const bool chain = !(c->cfg.flags & (MRP_FLAG_ROW_MAJOR_ONLY | MRP_FLAG_NO_CHAIN)) && sk_heads_ok(c->cfg) &&
                        sk_chain(c, M, K, out, st, f16_lm, true) == cudaSuccess;
     c->lo_x = (few_rows || chain) ? sk_head_pad(M) : M;
@@ -735,7 +755,8 @@ cudaError_t tc_draft(Ctx *c, const void *hidden, const float *logits0, const int
         p.a_row_base = step_base * M; p.a_part_rows = n_rs; p.step_base = step_base;
         p.M = M; p.K = K; p.V = V; p.d = d; p.F = F; p.n_rs = n_rs;
         p.logits0 = logits0; p.row_index = row_index; p.partials = partials; p.logits_out = out.logits_out;
-        p.n_rows_in = c->input_rows;
+        p.n_rows_in = c->input_rows; p.l0_bf16 = c->l0_bf16 ? 1 : 0;
+        p.teacher = c->teacher; p.kl_partials = (KlPartial *)(c->ws + c->lay.kl_partials);
         p.status = status; p.user_status = out.status;
         finish_shape(p, n_slices, f16_lm ? 1 : 2);
         const int grid = p.n_groups * p.n_vr;
@@ -751,8 +772,13 @@ cudaError_t tc_draft(Ctx *c, const void *hidden, const float *logits0, const int
         } else {
             if (!make_map(s, &mA, xt, d, 2 * (uint64_t)n_rs, 128) || !make_map(s, &mB, c->w_lm, d, V, p.bn))
                 return note_err(c, cudaErrorInvalidValue, "tensor map (LM head)");
-            e = note_err(c, out.margin ? launch_tc<KIND_LM, true>(mA, mB, mB, p, grid, st, pdl)
-                                       : launch_tc<KIND_LM, false>(mA, mB, mB, p, grid, st, pdl), "LM-head kernel");
+            if (with_kl)
+                e = note_err(c, out.margin ? launch_tc<KIND_LM, true, false, true>(mA, mB, mB, p, grid, st, pdl)
+                                           : launch_tc<KIND_LM, false, false, true>(mA, mB, mB, p, grid, st, pdl),
+                             "LM-head kernel (KL objective)");
+            else
+                e = note_err(c, out.margin ? launch_tc<KIND_LM, true>(mA, mB, mB, p, grid, st, pdl)
+                                           : launch_tc<KIND_LM, false>(mA, mB, mB, p, grid, st, pdl), "LM-head kernel");
         }
         c->launches++;
         if (e != cudaSuccess) return e;
@@ -762,15 +788,17 @@ cudaError_t tc_draft(Ctx *c, const void *hidden, const float *logits0, const int
     memset(&fix, 0, sizeof(fix));
     // every call: the size of the operand rows against the accuracy range; fp16 mode: the exact top logit
     fix.xt = xt; fix.logits0 = logits0; fix.row_index = row_index;
-    fix.d = d; fix.V = V; fix.M = M; fix.n_rs = n_rs; fix.n_rows_in = c->input_rows;
+    fix.d = d; fix.V = V; fix.M = M; fix.n_rs = n_rs; fix.n_rows_in = c->input_rows; fix.l0_bf16 = c->l0_bf16 ? 1 : 0;
     fix.range_limit = MRP_RANGE_LIMIT;
     if (f16_lm) fix.w = (const __nv_bfloat16 *)c->w_lm;
-    e = launch_combine(c, partials, n_slices, (K + 1) * M, out, status, st, &fix);
+    e = launch_combine(c, partials, n_slices, (K + 1) * M, out, status, st, &fix, M);
     prof_mark(c, 3, st);
     if (e != cudaSuccess) return e;
     FirstTok ft;
     memset(&ft, 0, sizeof(ft));
     ft.w = c->w_lm; ft.w_bf16 = 1; ft.logits0 = logits0; ft.row_index = row_index; ft.n_rows_in = c->input_rows;
+    ft.l0_bf16 = c->l0_bf16 ? 1 : 0;
+    if (c->use_fp8_lm) { ft.w = c->ws + c->lay.w8; ft.w8_scale = (const float *)(c->ws + c->lay.w8_scale); }
     ft.x = xt; ft.x_bf16 = 1; ft.lo_rows = c->lo_xt; ft.M = M; ft.K = K; ft.d = d; ft.V = V;
     return launch_first_token_prob(c, ft, out, st);
 }

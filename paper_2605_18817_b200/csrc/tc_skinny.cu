@@ -48,7 +48,8 @@ struct SkParams {
     int k_chunks;        // contraction extent / 64
     int n_stages;
     int kc;              // 64-element k-chunks per ring stage
-    int r_pad;           // activation rows per part (16, 32, 64 or 128; LM: 16 or 32); MMA N = 2 * r_pad
+    int r_pad;           // activation rows per part (16, 32, 64 or 128; LM: 16 or 32); MMA N = n_parts * r_pad
+    int n_parts;         // operand parts stacked on N: 2 (bf16 hi + lo) or 4 (e4m3 limbs)
     int tmem_cols;       // allocated TMEM columns (power of two >= 2 buffers * 2 * r_pad)
     int lo_x, lo_xt;     // row offset of the lo block in the head operands / the LM-head operand
     int lm_h[4];         // LM: tile heights (units) other than 8, fetched through maps w[1], w[2], w[4], w[5]
@@ -61,6 +62,7 @@ struct SkParams {
     const float *logits0;
     const int32_t *row_index;
     int n_rows_in;       // row_index entries at or above are invalid: their base logits read as zero
+    int l0_bf16;         // logits0 holds bf16 values
     Partial *partials;
     float *logits_out;
     // GU
@@ -79,6 +81,10 @@ struct SkParams {
     float *hidden_out;
     int32_t *status;
     int32_t *user_status;
+    // LM with 8-bit weights: per-vocabulary-row scales of the e4m3 copy of W_lm, per-row-step scales of
+    // the operand's e4m3 limbs
+    const float *w8_scale;
+    const float *x8_scale;
 };
 
 __device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
@@ -92,14 +98,19 @@ __device__ __forceinline__ void store_hi_lo(__nv_bfloat16 *dst, size_t lo_off, f
     dst[lo_off] = __float2bfloat16_rn(v - __bfloat162float(hi));
 }
 
-// KC: 64-element k-chunks per ring stage (2 for the LM head: fewer, larger stages stream better).
-template <int KIND, int RP, bool MARGIN, int KC>
+// KC: k-chunks (128 bytes of every row) per ring stage (2 for the LM head: fewer, larger stages stream better).
+// FP8 (LM head only): the weights are an e4m3 copy of W_lm with one power-of-two scale per row, a k-chunk
+// is 128 elements, and the activation operand is four e4m3 limbs per row-step (x = t * sum_i 16^-i limb_i,
+// exact to 2^-16) stacked on N instead of the bf16 hi + lo pair.
+template <int KIND, int RP, bool MARGIN, int KC, bool FP8 = false>
 __global__ void __launch_bounds__(kSkThreads, 1)
 sk_gemm_kernel(const __grid_constant__ SkMaps maps, const SkParams p)
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    constexpr int x_bytes = 2 * RP * 128;            // hi rows then lo rows of one k-chunk
+    constexpr int NP = FP8 ? 4 : 2;                  // operand parts stacked on N: 4 limbs, or hi and lo
+    constexpr int kElem = FP8 ? 128 : kBK;           // elements of the contraction per k-chunk
+    constexpr int x_bytes = NP * RP * 128;           // the parts' rows of one k-chunk
     constexpr int sub_bytes = kWTile + x_bytes;      // one k-chunk: weight tile, then activation rows
     constexpr int stage_bytes = KC * sub_bytes;
     const uint32_t bars = base + (uint32_t)p.n_stages * stage_bytes;
@@ -176,7 +187,7 @@ sk_gemm_kernel(const __grid_constant__ SkMaps maps, const SkParams p)
                 const int ut = tile_start(t);
 #pragma unroll
                 for (int b = 0; b < KC; ++b) {
-                    const int kx = (kc0 + kk * KC + b) * kBK;
+                    const int kx = (kc0 + kk * KC + b) * kElem;
                     if (KIND == SK_GU) {
                         tma_load_2d_hint(sw + b * sub_bytes, &maps.w[0], kx, ut * 8, full_bar(s), pol_w);
                         tma_load_2d_hint(sw + b * sub_bytes + 64 * 128, &maps.w[3], kx, ut * 8, full_bar(s), pol_w);
@@ -190,7 +201,7 @@ sk_gemm_kernel(const __grid_constant__ SkMaps maps, const SkParams p)
                 // one box per k-chunk: RP hi rows, then (the lo block starts at row RP of the buffer) RP lo rows
 #pragma unroll
                 for (int b = 0; b < KC; ++b)
-                    tma_load_2d_hint(sx + b * sub_bytes, &maps.x, (kc0 + kk * KC + b) * kBK, 0, full_bar(s), pol_x);
+                    tma_load_2d_hint(sx + b * sub_bytes, &maps.x, (kc0 + kk * KC + b) * kElem, 0, full_bar(s), pol_x);
             };
             // weights do not depend on the previous kernel: fill the ring with them first
             int t = 0, kk = 0;
@@ -216,7 +227,7 @@ sk_gemm_kernel(const __grid_constant__ SkMaps maps, const SkParams p)
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
         // The whole warp walks the loop (all values are warp-uniform); the elected lane issues.
-        const uint32_t idesc = make_idesc(2 * RP);
+        const uint32_t idesc = FP8 ? make_idesc_e4m3(NP * RP) : make_idesc(NP * RP);
         const uint32_t tm = __shfl_sync(0xffffffffu, tmem_base, 0);
         int s = 0, acc = 0;
         uint32_t ph = 0, acc_ph = 0;
@@ -225,7 +236,7 @@ sk_gemm_kernel(const __grid_constant__ SkMaps maps, const SkParams p)
             ok = __all_sync(0xffffffffu, mbar_wait(tempty_bar(acc), acc_ph ^ 1u, abort_flag, p));
             if (!ok) break;
             tc_fence_after();
-            const uint32_t dt = tm + (uint32_t)(acc * 2 * RP);
+            const uint32_t dt = tm + (uint32_t)(acc * NP * RP);
             for (int kk = 0; kk < nk; ++kk) {
                 const uint32_t sw = base + (uint32_t)s * stage_bytes;
                 const uint32_t later = kk > 0 ? 1u : 0u;
@@ -238,8 +249,10 @@ sk_gemm_kernel(const __grid_constant__ SkMaps maps, const SkParams p)
                         const uint64_t dw = make_smem_desc(sw + b * sub_bytes);
                         const uint64_t dx = make_smem_desc(sw + b * sub_bytes + kWTile);
 #pragma unroll
-                        for (int k4 = 0; k4 < kBK / 16; ++k4)
-                            umma_bf16(dt, dw + 2u * k4, dx + 2u * k4, idesc, (b > 0 || k4 > 0) ? 1u : later);
+                        for (int k4 = 0; k4 < 4; ++k4) {         // 32 bytes of every row per MMA
+                            if (FP8) umma_f8(dt, dw + 2u * k4, dx + 2u * k4, idesc, (b > 0 || k4 > 0) ? 1u : later);
+                            else umma_bf16(dt, dw + 2u * k4, dx + 2u * k4, idesc, (b > 0 || k4 > 0) ? 1u : later);
+                        }
                     }
                     umma_commit(empty_bar(s));
                 }
@@ -266,6 +279,7 @@ sk_gemm_kernel(const __grid_constant__ SkMaps maps, const SkParams p)
         if (t == 0) *vote_s = 0;
         griddep_wait();
         if (KIND == SK_LM) {
+            if (FP8 && t < RP) rstd_s[t] = t < p.n_rs ? p.x8_scale[t] : 0.f;     // the limbs' per-row-step scales
             if (t < p.n_rs) {
                 const int m = t % p.M;
                 const int idx = p.row_index ? p.row_index[m] : m;
@@ -300,17 +314,35 @@ sk_gemm_kernel(const __grid_constant__ SkMaps maps, const SkParams p)
                 float a[RP];
 #pragma unroll
                 for (int j = 0; j < RP; ++j)
-                    a[j] = (valid && j < p.n_rs && rowoff_s[j] >= 0) ? __ldg(p.logits0 + rowoff_s[j] + v) : 0.f;
+                    a[j] = (valid && j < p.n_rs && rowoff_s[j] >= 0) ? ld_l0(p.logits0, p.l0_bf16, (size_t)(rowoff_s[j] + v)) : 0.f;
                 ok = __all_sync(0xffffffffu, mbar_wait(tfull_bar(acc), acc_ph, abort_flag, p));
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t tacc = lane_addr + (uint32_t)(acc * 2 * RP);
+                const uint32_t tacc = lane_addr + (uint32_t)(acc * NP * RP);
+                if constexpr (!FP8) {
 #pragma unroll
-                for (int c0 = 0; c0 < 2 * RP; c0 += 16) {          // products with the hi rows, then the lo rows
-                    float part[16];
-                    tmem_ld16(tacc + c0, part);
+                    for (int c0 = 0; c0 < 2 * RP; c0 += 16) {          // products with the hi rows, then the lo rows
+                        float part[16];
+                        tmem_ld16(tacc + c0, part);
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) a[(c0 + j) % RP] += part[j];
+                        for (int j = 0; j < 16; ++j) a[(c0 + j) % RP] += part[j];
+                    }
+                } else {
+                    // delta = (row scale of W) * (scale of the row-step) * sum_i 16^-i (W8 . limb_i)
+                    const float ws = valid ? __ldg(p.w8_scale + v) : 0.f;
+                    float dsum[RP];
+#pragma unroll
+                    for (int j = 0; j < RP; ++j) dsum[j] = 0.f;
+#pragma unroll
+                    for (int c0 = 0; c0 < 4 * RP; c0 += 16) {
+                        float part[16];
+                        tmem_ld16(tacc + c0, part);
+                        const float lw = (c0 / RP) == 0 ? 1.f : (c0 / RP) == 1 ? 0.0625f : (c0 / RP) == 2 ? 0.00390625f : 0.000244140625f;
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) dsum[(c0 + j) % RP] = fmaf(part[j], lw, dsum[(c0 + j) % RP]);
+                    }
+#pragma unroll
+                    for (int j = 0; j < RP; ++j) a[j] = fmaf(dsum[j], ws * rstd_s[j], a[j]);
                 }
                 tc_fence_before();
                 __syncwarp();
@@ -521,11 +553,70 @@ sk_gemm_kernel(const __grid_constant__ SkMaps maps, const SkParams p)
 }
 
 // ---------------------------------------------------------------------------------------
+// 8-bit LM head: quantiser of W_lm (once, at context creation) and of the operand rows (every call)
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ float block_max(float v, float *red)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+    __syncthreads();
+    float m = 0.f;
+    for (int i = 0; i < (int)(blockDim.x >> 5); ++i) m = fmaxf(m, red[i]);
+    __syncthreads();
+    return m;
+}
+
+// One block per vocabulary row: scale = 2^E with max|row| <= 448 * 2^E, codes = e4m3(row / scale).
+__global__ void quantise_rows_kernel(const __nv_bfloat16 *__restrict__ w, int d, uint8_t *__restrict__ codes,
+                                     float *__restrict__ scales)
+{
+    __shared__ float red[32];
+    const size_t row = blockIdx.x;
+    float amax = 0.f;
+    for (int j = threadIdx.x; j < d; j += blockDim.x) amax = fmaxf(amax, fabsf(__bfloat162float(w[row * d + j])));
+    amax = block_max(amax, red);
+    const float sc = e4m3_row_scale(amax), inv = 1.f / sc;       // a power of two: the division is exact
+    if (threadIdx.x == 0) scales[row] = sc;
+    for (int j = threadIdx.x; j < d; j += blockDim.x)
+        codes[row * d + j] = (uint8_t)f32_to_e4m3(__bfloat162float(w[row * d + j]) * inv);
+}
+
+// One block per row-step of the stacked LM-head operand (bf16 hi + lo rows): x = t * (l_0 + l_1 / 16 +
+// l_2 / 256 + l_3 / 4096), t a power of two, every l_i an e4m3 value: each limb takes what the
+// previous ones left (the subtractions are exact in fp32), so x is met to 2^-16 relative.
+// Limb i of row-step r is row i * r_pad + r of xq.
+__global__ void operand_limbs_kernel(const __nv_bfloat16 *__restrict__ xt, int lo_rows, int d, int r_pad,
+                                     uint8_t *__restrict__ xq, float *__restrict__ x_scale)
+{
+    pdl_trigger();
+    pdl_wait();
+    __shared__ float red[32];
+    const int r = blockIdx.x;
+    const __nv_bfloat16 *hi = xt + (size_t)r * d, *lo = xt + ((size_t)lo_rows + r) * d;
+    float amax = 0.f;
+    for (int j = threadIdx.x; j < d; j += blockDim.x)
+        amax = fmaxf(amax, fabsf(__bfloat162float(hi[j]) + __bfloat162float(lo[j])));
+    amax = block_max(amax, red);
+    const float sc = e4m3_row_scale(amax), inv = 1.f / sc;
+    if (threadIdx.x == 0) x_scale[r] = sc;
+    for (int j = threadIdx.x; j < d; j += blockDim.x) {
+        float y = (__bfloat162float(hi[j]) + __bfloat162float(lo[j])) * inv;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const uint32_t q = f32_to_e4m3(y);
+            xq[((size_t)i * r_pad + r) * d + j] = (uint8_t)q;
+            y = (y - e4m3_to_f32(q)) * 16.f;
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------
 // Host side
 // ---------------------------------------------------------------------------------------
 size_t sk_smem_bytes(const SkParams &p)
 {
-    const int stage = p.kc * (kWTile + 2 * p.r_pad * 128);
+    const int stage = p.kc * (kWTile + p.n_parts * p.r_pad * 128);
     return (size_t)p.n_stages * stage + 1024 + 8 * (2 * p.n_stages + 4) + 16 + kAuxBytes;
 }
 
@@ -533,12 +624,13 @@ void sk_finish_shape(SkParams &p, int grid)
 {
     // the ring always takes all the shared memory there is: it also parks the LM statistics
     if (p.kc < 1) p.kc = 1;
-    const int stage = p.kc * (kWTile + 2 * p.r_pad * 128);
+    if (p.n_parts < 2) p.n_parts = 2;
+    const int stage = p.kc * (kWTile + p.n_parts * p.r_pad * 128);
     int ns = (kSmemBudget - 1024 - 256 - 16 - kAuxBytes) / stage;
     if (ns > 12) ns = 12;
     p.n_stages = ns;
     int cols = 32;
-    while (cols < 2 * 2 * p.r_pad) cols <<= 1;
+    while (cols < 2 * p.n_parts * p.r_pad) cols <<= 1;
     p.tmem_cols = cols;
     p.n_split = 1;
     for (int i = 0; i < 4; ++i) p.lm_h[i] = 0;
@@ -582,10 +674,10 @@ bool sk_weight_maps(const TcState *s, SkMaps &maps, int part, const void *w, uin
     return true;
 }
 
-template <int KIND, int RP, bool MARGIN, int KC = 1>
+template <int KIND, int RP, bool MARGIN, int KC = 1, bool FP8 = false>
 cudaError_t sk_launch(const SkMaps &maps, const SkParams &p, int grid, cudaStream_t st, bool pdl)
 {
-    auto kern = sk_gemm_kernel<KIND, RP, MARGIN, KC>;
+    auto kern = sk_gemm_kernel<KIND, RP, MARGIN, KC, FP8>;
     // the shared-memory limit of a kernel is set once per device (the attribute is per device)
     static std::atomic<unsigned long long> attr_devices{0};
     int dev = 0;
@@ -622,6 +714,11 @@ cudaError_t sk_launch_rp(const SkMaps &maps, const SkParams &p, int grid, cudaSt
         default: return sk_launch<KIND, 128, false>(maps, p, grid, st, pdl);
         }
     } else {
+        if (p.n_parts == 4) {       // e4m3 weights and operand limbs (two k-chunks per stage)
+            if (p.r_pad == 16)
+                return margin ? sk_launch<KIND, 16, true, 2, true>(maps, p, grid, st, pdl) : sk_launch<KIND, 16, false, 2, true>(maps, p, grid, st, pdl);
+            return margin ? sk_launch<KIND, 32, true, 2, true>(maps, p, grid, st, pdl) : sk_launch<KIND, 32, false, 2, true>(maps, p, grid, st, pdl);
+        }
         if (p.kc == 2) {
             if (p.r_pad == 16)
                 return margin ? sk_launch<KIND, 16, true, 2>(maps, p, grid, st, pdl) : sk_launch<KIND, 16, false, 2>(maps, p, grid, st, pdl);
@@ -717,16 +814,54 @@ cudaError_t sk_lm(Ctx *c, const float *logits0, const int32_t *row_index, int M,
     sk_common(c, p, M, K, out);
     p.units_total = V / 16; p.k_chunks = d / kBK; p.r_pad = sk_lm_pad(p.n_rs);
     p.kc = (p.k_chunks % 2 == 0) ? 2 : 1;
-    p.logits0 = logits0; p.row_index = row_index; p.n_rows_in = c->input_rows;
+    p.logits0 = logits0; p.row_index = row_index; p.n_rows_in = c->input_rows; p.l0_bf16 = c->l0_bf16 ? 1 : 0;
     p.partials = (Partial *)(c->ws + c->lay.partials); p.logits_out = out.logits_out;
-    sk_finish_shape(p, G);
     SkMaps maps;
     memset(&maps, 0, sizeof(maps));
+    if (c->use_fp8_lm) {
+        // the operand rows as e4m3 limbs, then the same kernel on the 8-bit copy of W_lm
+        uint8_t *xq = (uint8_t *)(c->ws + c->lay.xq);
+        float *xs = (float *)(c->ws + c->lay.x8_scale);
+        cudaError_t e = note_err(c, launch_k(operand_limbs_kernel, dim3(p.n_rs), dim3(256), 0, st, pdl,
+                                             (const __nv_bfloat16 *)(c->ws + c->lay.xt), c->lo_xt, d, p.r_pad, xq, xs),
+                                 "operand limb kernel");
+        c->launches++;
+        if (e != cudaSuccess) return e;
+        p.k_chunks = d / 128; p.kc = 2; p.n_parts = 4;
+        p.w8_scale = (const float *)(c->ws + c->lay.w8_scale); p.x8_scale = xs;
+        sk_finish_shape(p, G);
+        bool ok = make_map_u8(s, &maps.x, xq, d, 4 * (uint64_t)p.r_pad, 4 * p.r_pad) &&
+                  make_map_u8(s, &maps.w[0], c->ws + c->lay.w8, d, V, 128);
+        static const int slot[4] = {1, 2, 4, 5};
+        for (int k = 0; k < 4 && ok; ++k)
+            if (p.lm_h[k] > 0) ok = make_map_u8(s, &maps.w[slot[k]], c->ws + c->lay.w8, d, V, p.lm_h[k] * 16);
+        if (!ok) return note_err(c, cudaErrorInvalidValue, "tensor map (LM head, 8-bit weights)");
+        c->launches++;
+        return note_err(c, sk_launch_rp<SK_LM>(maps, p, G, st, pdl, out.margin != nullptr), "LM-head kernel (8-bit weights)");
+    }
+    sk_finish_shape(p, G);
     if (!make_map(s, &maps.x, c->ws + c->lay.xt, d, 2 * (uint64_t)p.r_pad, 2 * p.r_pad) ||
         !sk_weight_maps(s, maps, 0, c->w_lm, d, V, 16, p))
         return note_err(c, cudaErrorInvalidValue, "tensor map (LM head, few rows)");
     c->launches++;
     return note_err(c, sk_launch_rp<SK_LM>(maps, p, G, st, pdl, out.margin != nullptr), "LM-head kernel (few rows)");
+}
+
+bool fp8_lm_supported(const mrp_config &cfg)
+{
+    return cfg.dtype == MRP_BF16 && !(cfg.flags & (MRP_FLAG_FORCE_SIMT | MRP_FLAG_ROW_MAJOR_ONLY | MRP_FLAG_TRAINING_KL)) &&
+           cfg.d % 256 == 0 && cfg.n_heads >= 1 && ((long long)cfg.n_heads + 1) * cfg.max_rows <= 32;
+}
+
+cudaError_t fp8_lm_create(Ctx *c)
+{
+    quantise_rows_kernel<<<c->cfg.vocab, 256>>>((const __nv_bfloat16 *)c->w_lm, c->cfg.d, (uint8_t *)(c->ws + c->lay.w8),
+                                                (float *)(c->ws + c->lay.w8_scale));
+    cudaError_t e = cudaGetLastError();
+    if (e == cudaSuccess) e = cudaMemset(c->ws + c->lay.xq, 0, (size_t)4 * 32 * c->cfg.d);
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();
+    c->use_fp8_lm = (e == cudaSuccess);
+    return e;
 }
 
 }  // namespace mrp

@@ -430,6 +430,91 @@ def test_probability_of_the_step_zero_token_under_the_updated_logits(dtype, flag
     binding.mrp_destroy(ctx)
 
 
+# ---- base logits stored as bf16 (mrp_draft_bf16_logits) ----
+
+@pytest.mark.parametrize("dtype,flags,d,F,V,B,L,K", [
+    ("f32", 0, 72, 136, 1000, 5, 3, 2),                                # CUDA-core kernels
+    ("bf16", 0, 256, 512, 4096, 2, 4, 3),                              # few-row LM head
+    ("bf16", 0, 128, 256, 2048, 30, 4, 3),                             # row-major LM head, fp16 operand + top fix
+    ("bf16", binding.MRP_FLAG_EXACT_OPERANDS, 192, 320, 4112, 150, 1, 2),
+])
+def test_base_logits_stored_as_bf16(dtype, flags, d, F, V, B, L, K):
+    """The bf16 values are the input: the oracle takes the same values promoted to fp32."""
+    w = synth.make_weights(d, F, V, K, dtype, 81, head_std=0.05)
+    inp = synth.make_inputs(w, B, L, 81, 1.0, 4.0, mask_prob=0.8)
+    l0_r = synth.bf16_round(inp.logits0)
+    heads, w_lm = harness.upload_weights(w, DEV)
+    ctx = binding.mrp_create(d, F, V, heads, w_lm, max_rows=B * L, max_seqs=B, block_len=L, flags=flags)
+    M = inp.row_index.size
+    hid = harness.to_device(inp.hidden, w.dtype, DEV)
+    l0 = harness.to_device(l0_r, "bf16", DEV)
+    ri = torch.from_numpy(inp.row_index).to(DEV)
+    out = harness.alloc_draft_out(M, K, V, d, DEV, logits=True, conf_first=True)
+    harness.draft(ctx, hid, l0, ri, M, K, out)
+    torch.cuda.synchronize()
+    ref = oracle.draft(inp.hidden, l0_r, w.heads, w.w_lm, K=K, row_index=inp.row_index, want_logits=True)
+    check_stats(out, ref, dtype)
+    lg = out.logits.cpu().numpy().astype(np.float64)
+    rms = np.sqrt((ref.logits ** 2).mean(axis=2, keepdims=True))
+    assert np.all(np.abs(lg - ref.logits) <= (1e-4 if dtype == "f32" else 2e-2) * np.maximum(np.abs(ref.logits), rms))
+    clear0 = ref.margin[0] > 1e-2
+    assert np.abs(out.conf_first.cpu().numpy() - ref.conf_first)[:, clear0].max() <= TOL[dtype]
+    binding.mrp_destroy(ctx)
+
+
+# ---- the training objective fused into the LM-head epilogue (mrp_draft_kl) ----
+
+@pytest.mark.parametrize("dtype,flags,d,F,V,B,L,K", [
+    ("f32", 0, 72, 136, 1000, 5, 3, 2),                                # CUDA-core kernels, ragged sizes
+    ("bf16", binding.MRP_FLAG_FORCE_SIMT, 72, 136, 1000, 5, 3, 3),
+    ("bf16", 0, 256, 512, 4096, 2, 4, 2),                              # 8 rows: one row block
+    ("bf16", 0, 192, 320, 4112, 150, 1, 2),                            # 300 row-steps, ragged vocabulary tiles
+    ("bf16", 0, 1024, 2048, 8192, 40, 4, 3),                           # several tiles per CTA, 480 row-steps
+])
+def test_kl_objective_fused_into_the_lm_head(dtype, flags, d, F, V, B, L, K):
+    """kl[k, m] = KL(softmax(teacher_k) || softmax(l_k)) per masked row and unrolled step (Eq. (3)) against
+    the oracle: absolute error within 2e-3 (bf16 contexts) / 1e-5 (fp32), and relative 2e-3 where the
+    divergence is large; the ordinary statistics of the same call stay those of mrp_draft."""
+    w = synth.make_weights(d, F, V, K, dtype, 71, head_std=0.05 if d <= 256 else 0.02)
+    inp = synth.make_inputs(w, B, L, 71, 1.0, 4.0, mask_prob=0.8)
+    ri = inp.row_index
+    M = ri.size
+    base = oracle.draft(inp.hidden, inp.logits0, w.heads, w.w_lm, K=K, row_index=ri, want_logits=True)
+    rng = np.random.default_rng(3)
+    # teacher = corrected logits plus a perturbation of a few tenths: KL values from 1e-3 to order one
+    scale = rng.uniform(0.02, 0.6, size=(K, M, 1))
+    teacher = (base.logits + scale * rng.standard_normal(base.logits.shape)).astype(np.float32)
+    ref, kl_ref = oracle.draft_kl(inp.hidden, inp.logits0, teacher, w.heads, w.w_lm, K=K, row_index=ri)
+    heads, w_lm = harness.upload_weights(w, DEV)
+    ctx = binding.mrp_create(d, F, V, heads, w_lm, max_rows=B * L, max_seqs=B, block_len=L,
+                             flags=flags | binding.MRP_FLAG_TRAINING_KL)
+    hid = harness.to_device(inp.hidden, w.dtype, DEV)
+    l0 = torch.from_numpy(inp.logits0).to(DEV)
+    out = harness.alloc_draft_out(M, K, V, d, DEV)
+    kl = torch.full((K, M), -1.0, device=DEV)
+    binding.mrp_draft_kl(ctx, hid, l0, torch.from_numpy(teacher).to(DEV), torch.from_numpy(ri).to(DEV), M, K,
+                         out.conf, out.lse, out.token, kl, margin=out.margin, status=out.status)
+    torch.cuda.synchronize()
+    check_stats(out, ref, dtype)
+    got = kl.cpu().numpy().astype(np.float64)
+    tol = TOL[dtype]
+    assert kl_ref.min() > 0 and kl_ref.max() > 1e-2
+    assert np.all(np.abs(got - kl_ref) <= tol + 2e-3 * kl_ref), np.abs(got - kl_ref).max()
+    # the ordinary entry point on the same context afterwards: nothing of the KL call lingers
+    out2 = harness.alloc_draft_out(M, K, V, d, DEV)
+    harness.draft(ctx, hid, l0, torch.from_numpy(ri).to(DEV), M, K, out2)
+    torch.cuda.synchronize()
+    check_stats(out2, ref, dtype)
+    binding.mrp_destroy(ctx)
+    # a context without the flag has no room for the partial sums
+    ctx = binding.mrp_create(d, F, V, heads, w_lm, max_rows=B * L, max_seqs=B, block_len=L, flags=flags)
+    with pytest.raises(binding.MrpError) as ei:
+        binding.mrp_draft_kl(ctx, hid, l0, torch.from_numpy(teacher).to(DEV), torch.from_numpy(ri).to(DEV), M, K,
+                             out.conf, out.lse, out.token, kl)
+    assert ei.value.status == 2
+    binding.mrp_destroy(ctx)
+
+
 # ---- base logits computed from the hidden states in the LM-head pass (mrp_draft_from_hidden) ----
 
 @pytest.mark.parametrize("dtype,flags,d,F,V,B,L,K", [
