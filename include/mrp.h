@@ -250,6 +250,62 @@ int mrp_draft_kl(mrp_ctx *ctx, const void *hidden, const float *logits0, const f
                  const int32_t *row_index, int32_t M, int32_t K, const mrp_draft_out *out, float *kl,
                  void *cuda_stream);
 
+/*
+ * The token-conditioned MRP module (Sec. 3.2; Fig. 1(a,c); Algorithm 2, "Delta, delta <- g(x_t, h)"),
+ * one application per call so that the caller can reveal tokens between MRP steps: unlike the reduced
+ * head above, this module reads the embeddings of the tokens revealed so far, so step k + 1 depends on
+ * the reveals of step k and the LM head runs once per step.
+ * The paper fixes the parts and leaves the details open; the form implemented (first slice: CUDA-core
+ * kernels for the module itself, the context's own LM-head kernels behind it):
+ *     e_i = emb[x_i]  (emb[mask_token] where x_i = -1);   z_i = W_proj [h_i ; e_i]
+ *     n_layers times:  z += W_o Attn(RMSNorm(z) g_attn),  attention over the positions of the same block,
+ *                      bidirectional, n_attn_heads heads, no positional term;
+ *                      z += W_down( silu(W_gate n) * (W_up n) ),  n = RMSNorm(z) g_mlp
+ *     Delta_i = z_i;   h_i <- h_i + Delta_i  (every position);   l_i <- l_i + W_lm Delta_i  (masked rows)
+ * All matrices row-major [out, in] in the context's dtype, no biases.
+ */
+typedef struct {
+    const void *g_attn, *w_q, *w_k, *w_v, *w_o;     /* [d], [d, d] x 4        */
+    const void *g_mlp, *w_gate, *w_up, *w_down;     /* [d], [d_ff, d] x 2, [d, d_ff] */
+} mrp_module_layer;
+
+typedef struct {
+    int32_t n_layers;               /* D (the paper: 3); 0 = the fusion projection alone          */
+    int32_t n_attn_heads;           /* divides d                                                   */
+    int32_t mask_token;             /* row of emb that stands for a masked position                */
+    int32_t emb_rows;               /* rows of emb: tokens are checked against it on the device     */
+    const void *emb;                /* [emb_rows, d] frozen token embeddings                        */
+    const void *w_proj;             /* [d, 2 d]                                                     */
+    const mrp_module_layer *layers; /* HOST array [n_layers] of DEVICE pointers                     */
+} mrp_module_weights;
+
+/* Bytes of additional device workspace the module needs on this context (0 on bad arguments). */
+size_t mrp_module_workspace_bytes(const mrp_config *cfg, const mrp_module_weights *w);
+
+/*
+ * Attach a module to a context (weights and workspace borrowed until mrp_destroy or the next attach;
+ * workspace DEVICE, 256-byte aligned, at least mrp_module_workspace_bytes).  Errors: INVALID_ARG, NOMEM.
+ */
+int mrp_module_attach(mrp_ctx *ctx, const mrp_module_weights *w, void *workspace, size_t workspace_bytes);
+
+/*
+ * One MRP step of the attached module over B blocks of L positions.
+ *   tokens   [B*L] int32   the sequence x_t of the active blocks: token id, or -1 where still masked; an id
+ *                          outside [0, emb_rows) raises MRP_DEV_BAD_INDEX and is read as masked
+ *   hidden0  [B*L, d]      backbone hidden states h_0 (context dtype)
+ *   h_state  [B*L, d] fp32 running hidden states h, in/out: h <- h + Delta; with first_step != 0 the call
+ *                          first sets it to h_0, so the caller never converts
+ *   logits0, row_index, M  as mrp_draft (row_index entries in [0, B*L))
+ *   out      conf / lse / token (margin, conf_first optional) are [2, M]: entry 0 the backbone's own
+ *            logits, entry 1 the logits after this step, l_0 + W_lm (h - h_0), which by linearity is the
+ *            running sum l <- l + delta of Algorithm 2; hidden_out optional [M, d]; logits_out [1, M, V]
+ * The caller reveals from entry 1 (mrp_reveal_remask with K = 0 on it, mrp_commit), updates tokens and
+ * calls again.  Errors: INVALID_ARG, UNSUPPORTED (no module attached), CUDA.
+ */
+int mrp_module_step(mrp_ctx *ctx, const int32_t *tokens, const void *hidden0, float *h_state,
+                    const float *logits0, const int32_t *row_index, int32_t M, int32_t B, int32_t L,
+                    int32_t first_step, const mrp_draft_out *out, void *cuda_stream);
+
 typedef enum { MRP_SELECT_STATIC = 0, MRP_SELECT_DYNAMIC_REMASK = 1 } mrp_select_mode;
 
 typedef struct {

@@ -46,6 +46,7 @@ def _load():
         _lib.mrp_oracle_draft.restype = ctypes.c_int
         _lib.mrp_oracle_draft_from_hidden.restype = ctypes.c_int
         _lib.mrp_oracle_draft_kl.restype = ctypes.c_int
+        _lib.mrp_oracle_module.restype = ctypes.c_int
         _lib.mrp_oracle_select.restype = ctypes.c_int
         _lib.mrp_oracle_verify.restype = ctypes.c_int
     return _lib
@@ -187,6 +188,60 @@ def draft_kl(hidden, logits0, teacher, heads, w_lm, K=None, row_index=None, eps=
     if rc != 0:
         raise RuntimeError("mrp_oracle_draft_kl failed (%d)" % rc)
     return DraftResult(conf, lse, token, margin, None, None), kl
+
+
+MODULE_LAYER_KEYS = ("g_attn", "w_q", "w_k", "w_v", "w_o", "g_mlp", "w_gate", "w_up", "w_down")
+
+
+def module(hidden, tokens, B, L, emb, w_proj, layers, w_lm, n_attn_heads, mask_token, row_index=None, eps=1e-6):
+    """One application of the token-conditioned MRP module g(x_t, h) (Sec. 3.2; Algorithm 2) to the L
+    positions of each of B blocks: returns (delta_h [B*L, d], delta_l [M, V]) in float64.  ``layers`` is a
+    sequence of dicts with the arrays named in MODULE_LAYER_KEYS; ``tokens`` [B*L] with -1 = masked."""
+    lib = _load()
+    hidden, emb, w_proj, w_lm = _f32(hidden), _f32(emb), _f32(w_proj), _f32(w_lm)
+    tokens = _i32(tokens)
+    n, d = hidden.shape
+    assert n == B * L and tokens.shape == (n,) and w_proj.shape == (d, 2 * d) and emb.shape[1] == d
+    V = w_lm.shape[0]
+    D = len(layers)
+    F = layers[0]["w_gate"].shape[0] if D else 1
+    shapes = dict(g_attn=(d,), w_q=(d, d), w_k=(d, d), w_v=(d, d), w_o=(d, d), g_mlp=(d,), w_gate=(F, d), w_up=(F, d),
+                  w_down=(d, F))
+    PtrArr = ctypes.POINTER(ctypes.c_float) * max(D, 1)
+    keep, arrs = [], {}
+    for name in MODULE_LAYER_KEYS:
+        lst = []
+        for lay in layers:
+            a = _f32(lay[name])
+            assert a.shape == shapes[name], (name, a.shape)
+            keep.append(a)
+            lst.append(_p(a, ctypes.c_float))
+        arrs[name] = PtrArr(*lst) if D else PtrArr()
+    ri, M = None, 0
+    if row_index is not None:
+        ri = _i32(row_index)
+        M = ri.shape[0]
+    delta_h = np.zeros((n, d), np.float64)
+    delta_l = np.zeros((M, V), np.float64)
+    rc = lib.mrp_oracle_module(
+        ctypes.c_int(d), ctypes.c_int(F), ctypes.c_int(V), ctypes.c_int(D), ctypes.c_int(n_attn_heads), ctypes.c_int(B),
+        ctypes.c_int(L), ctypes.c_int(mask_token), ctypes.c_double(eps), _p(hidden, ctypes.c_float),
+        _p(tokens, ctypes.c_int32), _p(emb, ctypes.c_float), _p(w_proj, ctypes.c_float),
+        *[arrs[k] for k in MODULE_LAYER_KEYS], _p(w_lm, ctypes.c_float), _p(ri, ctypes.c_int32), ctypes.c_int(M),
+        _p(delta_h, ctypes.c_double), _p(delta_l, ctypes.c_double))
+    if rc != 0:
+        raise RuntimeError("mrp_oracle_module failed (%d)" % rc)
+    return delta_h, delta_l
+
+
+def stats(logits):
+    """(conf, lse, token, margin) of logit rows [M, V] by the definitions of Sec. 2, in float64."""
+    l = np.asarray(logits, np.float64)
+    mx = l.max(axis=1)
+    tok = l.argmax(axis=1).astype(np.int32)
+    lse = mx + np.log(np.exp(l - mx[:, None]).sum(axis=1))
+    second = np.sort(l, axis=1)[:, -2] if l.shape[1] > 1 else np.full(l.shape[0], -np.inf)
+    return np.exp(mx - lse), lse, tok, mx - second
 
 
 @dataclass

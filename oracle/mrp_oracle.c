@@ -455,3 +455,134 @@ int mrp_oracle_verify(const int32_t *draft_tok, const int32_t *verify_tok,
     }
     return 0;
 }
+
+/* ------------------------------------------------------------------------------------------------
+ * The token-conditioned MRP module (Sec. 3.2; Fig. 1(a,c); Algorithm 2, "Delta, delta <- g(x_t, h)").
+ *
+ * One application of g to the L positions of each of B active blocks.  Sec. 3.2 fixes the parts --
+ * the backbone's hidden states and the token embeddings of the (partly revealed) sequence, fused by a
+ * learned projection; a small number D of transformer layers; the backbone's LM head on the result --
+ * and leaves their details open.  The reading taken here (listed with the other readings in the
+ * design notes):
+ *     e_i = E[x_i]  (E the frozen embedding table; the [MASK] embedding where x_i = -1)
+ *     z_i = W_p [h_i ; e_i]                                    (W_p [d, 2d], no bias)
+ *     D times:  n = RMSNorm(z; g_attn);  q, k, v = W_q n, W_k n, W_v n;
+ *               o_i = sum_j softmax_j(q_i . k_j / sqrt(d_head)) v_j   per attention head, j over the
+ *                     positions of the same block (bidirectional, block-local, no positional term);
+ *               z += W_o o;   n' = RMSNorm(z; g_mlp);   z += W_down( silu(W_gate n') * (W_up n') )
+ *     Delta_i = z_i   (hidden residual),   delta_i = W_lm Delta_i   (logit residual)
+ * Outputs: delta_h [B*L, d] double for every position; delta_l [M, V] double for the masked rows
+ * listed in row_index (may be NULL with M = 0).  tokens [B*L] int32, -1 = masked.
+ * Layer weights: arrays of D pointers each.  Returns 0, or -1 on bad arguments.
+ */
+int mrp_oracle_module(int d, int F, int V, int D, int n_attn_heads, int B, int L, int mask_token, double eps,
+                      const float *hidden, const int32_t *tokens, const float *emb, const float *w_proj,
+                      const float *const *g_attn, const float *const *w_q, const float *const *w_k,
+                      const float *const *w_v, const float *const *w_o, const float *const *g_mlp,
+                      const float *const *w_gate, const float *const *w_up, const float *const *w_down,
+                      const float *w_lm, const int32_t *row_index, int M, double *delta_h, double *delta_l)
+{
+    if (d <= 0 || F <= 0 || V <= 0 || D < 0 || n_attn_heads <= 0 || d % n_attn_heads || B <= 0 || L <= 0) return -1;
+    const int dh = d / n_attn_heads;
+    const size_t n = (size_t)B * L;
+    double *z = (double *)malloc(sizeof(double) * n * d), *nn = (double *)malloc(sizeof(double) * n * d);
+    double *q = (double *)malloc(sizeof(double) * n * d), *k = (double *)malloc(sizeof(double) * n * d);
+    double *v = (double *)malloc(sizeof(double) * n * d), *o = (double *)malloc(sizeof(double) * n * d);
+    double *a = (double *)malloc(sizeof(double) * (size_t)F), *p = (double *)malloc(sizeof(double) * (size_t)L);
+    if (!z || !nn || !q || !k || !v || !o || !a || !p) { free(z); free(nn); free(q); free(k); free(v); free(o); free(a); free(p); return -1; }
+
+    /* fusion of hidden state and token embedding */
+    for (size_t i = 0; i < n; ++i) {
+        const int tok = tokens[i] >= 0 ? tokens[i] : mask_token;
+        const float *hi = hidden + i * (size_t)d, *ei = emb + (size_t)tok * d;
+        for (int j = 0; j < d; ++j) {
+            const float *wr = w_proj + (size_t)j * 2 * d;
+            double s = 0.0;
+            for (int c = 0; c < d; ++c) s += (double)wr[c] * (double)hi[c];
+            for (int c = 0; c < d; ++c) s += (double)wr[d + c] * (double)ei[c];
+            z[i * d + j] = s;
+        }
+    }
+    for (int layer = 0; layer < D; ++layer) {
+        /* attention sub-layer */
+        for (size_t i = 0; i < n; ++i) {
+            double ss = 0.0;
+            for (int j = 0; j < d; ++j) ss += z[i * d + j] * z[i * d + j];
+            const double rstd = 1.0 / sqrt(ss / (double)d + eps);
+            for (int j = 0; j < d; ++j) nn[i * d + j] = z[i * d + j] * rstd * (double)g_attn[layer][j];
+        }
+        for (size_t i = 0; i < n; ++i)
+            for (int j = 0; j < d; ++j) {
+                double sq = 0.0, sk = 0.0, sv = 0.0;
+                for (int c = 0; c < d; ++c) {
+                    const double x = nn[i * d + c];
+                    sq += (double)w_q[layer][(size_t)j * d + c] * x;
+                    sk += (double)w_k[layer][(size_t)j * d + c] * x;
+                    sv += (double)w_v[layer][(size_t)j * d + c] * x;
+                }
+                q[i * d + j] = sq; k[i * d + j] = sk; v[i * d + j] = sv;
+            }
+        for (int b = 0; b < B; ++b)
+            for (int hd = 0; hd < n_attn_heads; ++hd)
+                for (int i = 0; i < L; ++i) {
+                    const size_t ri = ((size_t)b * L + i) * d + (size_t)hd * dh;
+                    double mx = -INFINITY;
+                    for (int j = 0; j < L; ++j) {
+                        const size_t rj = ((size_t)b * L + j) * d + (size_t)hd * dh;
+                        double s = 0.0;
+                        for (int c = 0; c < dh; ++c) s += q[ri + c] * k[rj + c];
+                        p[j] = s / sqrt((double)dh);
+                        if (p[j] > mx) mx = p[j];
+                    }
+                    double sum = 0.0;
+                    for (int j = 0; j < L; ++j) { p[j] = exp(p[j] - mx); sum += p[j]; }
+                    for (int c = 0; c < dh; ++c) {
+                        double s = 0.0;
+                        for (int j = 0; j < L; ++j) s += p[j] * v[((size_t)b * L + j) * d + (size_t)hd * dh + c];
+                        o[ri + c] = s / sum;
+                    }
+                }
+        for (size_t i = 0; i < n; ++i)
+            for (int j = 0; j < d; ++j) {
+                double s = 0.0;
+                for (int c = 0; c < d; ++c) s += (double)w_o[layer][(size_t)j * d + c] * o[i * d + c];
+                nn[i * d + j] = s;                 /* held apart until every output of the row is done */
+            }
+        for (size_t i = 0; i < n * d; ++i) z[i] += nn[i];
+        /* SwiGLU sub-layer */
+        for (size_t i = 0; i < n; ++i) {
+            double ss = 0.0;
+            for (int j = 0; j < d; ++j) ss += z[i * d + j] * z[i * d + j];
+            const double rstd = 1.0 / sqrt(ss / (double)d + eps);
+            for (int j = 0; j < d; ++j) nn[i * d + j] = z[i * d + j] * rstd * (double)g_mlp[layer][j];
+            for (int f = 0; f < F; ++f) {
+                double g = 0.0, u = 0.0;
+                for (int c = 0; c < d; ++c) {
+                    g += (double)w_gate[layer][(size_t)f * d + c] * nn[i * d + c];
+                    u += (double)w_up[layer][(size_t)f * d + c] * nn[i * d + c];
+                }
+                a[f] = g / (1.0 + exp(-g)) * u;
+            }
+            for (int j = 0; j < d; ++j) {
+                double s = 0.0;
+                for (int f = 0; f < F; ++f) s += (double)w_down[layer][(size_t)j * F + f] * a[f];
+                q[i * d + j] = s;
+            }
+        }
+        for (size_t i = 0; i < n * d; ++i) z[i] += q[i];
+    }
+    for (size_t i = 0; i < n * d; ++i) delta_h[i] = z[i];
+    /* logit residual of the masked rows through the shared LM head */
+    for (int m = 0; m < M; ++m) {
+        const size_t row = row_index ? (size_t)row_index[m] : (size_t)m;
+        if (row >= n) { free(z); free(nn); free(q); free(k); free(v); free(o); free(a); free(p); return -1; }
+#pragma omp parallel for schedule(static)
+        for (int t = 0; t < V; ++t) {
+            double s = 0.0;
+            for (int c = 0; c < d; ++c) s += (double)w_lm[(size_t)t * d + c] * z[row * d + c];
+            delta_l[(size_t)m * V + t] = s;
+        }
+    }
+    free(z); free(nn); free(q); free(k); free(v); free(o); free(a); free(p);
+    return 0;
+}

@@ -35,7 +35,8 @@ EXPORTS = ("mrp_workspace_bytes", "mrp_create", "mrp_destroy", "mrp_draft", "mrp
            "mrp_verify", "mrp_last_launch_count", "mrp_kernel_family", "mrp_status_string",
            "mrp_profile_enable", "mrp_profile_read", "mrp_last_error",
            "mrp_reveal_remask_noalloc", "mrp_selftest_wait_timeout", "mrp_draft_from_hidden", "mrp_commit",
-           "mrp_set_logits0_event", "mrp_set_input_rows", "mrp_fetch_status", "mrp_draft_kl", "mrp_draft_bf16_logits", "mrp_quantised_lm_head")
+           "mrp_set_logits0_event", "mrp_set_input_rows", "mrp_fetch_status", "mrp_draft_kl", "mrp_draft_bf16_logits", "mrp_quantised_lm_head",
+           "mrp_module_workspace_bytes", "mrp_module_attach", "mrp_module_step")
 MRP_NOALLOC_MAX_POSITIONS = 65536
 MRP_ERR_CAPACITY = 7
 
@@ -74,6 +75,16 @@ class mrp_select_out(ctypes.Structure):
                 ("draft_len", ctypes.c_void_p), ("status", ctypes.c_void_p)]
 
 
+class mrp_module_layer(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in ("g_attn", "w_q", "w_k", "w_v", "w_o", "g_mlp", "w_gate", "w_up", "w_down")]
+
+
+class mrp_module_weights(ctypes.Structure):
+    _fields_ = [("n_layers", ctypes.c_int32), ("n_attn_heads", ctypes.c_int32), ("mask_token", ctypes.c_int32),
+                ("emb_rows", ctypes.c_int32), ("emb", ctypes.c_void_p), ("w_proj", ctypes.c_void_p),
+                ("layers", ctypes.POINTER(mrp_module_layer))]
+
+
 class mrp_block_state(ctypes.Structure):
     _fields_ = [("tokens", ctypes.c_void_p), ("row_index", ctypes.c_void_p),
                 ("n_masked", ctypes.c_void_p), ("block_masked", ctypes.c_void_p)]
@@ -103,6 +114,14 @@ def _load():
     lib.mrp_draft_bf16_logits.argtypes = lib.mrp_draft.argtypes
     lib.mrp_quantised_lm_head.restype = ctypes.c_int
     lib.mrp_quantised_lm_head.argtypes = [ctypes.c_void_p, ctypes.POINTER(ctypes.c_void_p), ctypes.POINTER(ctypes.c_void_p)]
+    lib.mrp_module_workspace_bytes.restype = ctypes.c_size_t
+    lib.mrp_module_workspace_bytes.argtypes = [ctypes.POINTER(mrp_config), ctypes.POINTER(mrp_module_weights)]
+    lib.mrp_module_attach.restype = ctypes.c_int
+    lib.mrp_module_attach.argtypes = [ctypes.c_void_p, ctypes.POINTER(mrp_module_weights), ctypes.c_void_p, ctypes.c_size_t]
+    lib.mrp_module_step.restype = ctypes.c_int
+    lib.mrp_module_step.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                                    ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
+                                    ctypes.POINTER(mrp_draft_out), ctypes.c_void_p]
     lib.mrp_draft_kl.restype = ctypes.c_int
     lib.mrp_draft_kl.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
                                  ctypes.c_int32, ctypes.c_int32, ctypes.POINTER(mrp_draft_out), ctypes.c_void_p,
@@ -259,6 +278,54 @@ def mrp_quantised_lm_head(ctx: Context):
     c.copy_(ws[codes.value - ws.data_ptr():codes.value - ws.data_ptr() + V * d].view(V, d))
     s.copy_(ws[scales.value - ws.data_ptr():scales.value - ws.data_ptr() + 4 * V].view(torch.float32))
     return c.cpu().numpy(), s.cpu().numpy()
+
+
+def mrp_module_attach(ctx: Context, emb, w_proj, layers, n_attn_heads, mask_token) -> None:
+    """Attach the token-conditioned module: ``emb`` [rows, d], ``w_proj`` [d, 2d], ``layers`` a list of dicts
+    of CUDA tensors named like the fields of mrp_module_layer.  Allocates the module's workspace (a torch
+    tensor kept alive with the context)."""
+    tdtype = torch.float32 if ctx.cfg.dtype == MRP_F32 else torch.bfloat16
+    _check(emb, tdtype, "emb")
+    _check(w_proj, tdtype, "w_proj")
+    larr = (mrp_module_layer * max(len(layers), 1))()
+    keep = [emb, w_proj]
+    for i, lay in enumerate(layers):
+        vals = []
+        for name, _ in mrp_module_layer._fields_:
+            _check(lay[name], tdtype, name)
+            keep.append(lay[name])
+            vals.append(lay[name].data_ptr())
+        larr[i] = mrp_module_layer(*vals)
+    w = mrp_module_weights(len(layers), int(n_attn_heads), int(mask_token), int(emb.shape[0]), emb.data_ptr(),
+                           w_proj.data_ptr(), larr)
+    nbytes = int(lib.mrp_module_workspace_bytes(ctypes.byref(ctx.cfg), ctypes.byref(w)))
+    if nbytes == 0:
+        raise MrpError("mrp_module_workspace_bytes", 1)
+    ws = torch.empty(nbytes + 256, dtype=torch.uint8, device=emb.device)
+    off = (-ws.data_ptr()) % 256
+    rc = lib.mrp_module_attach(ctx.handle, ctypes.byref(w), ctypes.c_void_p(ws.data_ptr() + off), ctypes.c_size_t(nbytes))
+    if rc != 0:
+        raise MrpError("mrp_module_attach", rc)
+    ctx.keep = tuple(ctx.keep) + tuple(keep) + (ws,)
+
+
+def mrp_module_step(ctx: Context, tokens, hidden0, h_state, logits0, row_index, M, B, L, first_step, conf, lse, token,
+                    margin=None, logits_out=None, hidden_out=None, status=None, conf_first=None, stream=None) -> None:
+    """One step of the attached module; conf / lse / token are [2, M] (backbone, after this step)."""
+    tdtype = torch.float32 if ctx.cfg.dtype == MRP_F32 else torch.bfloat16
+    for t, dt, nm in ((tokens, torch.int32, "tokens"), (hidden0, tdtype, "hidden0"), (h_state, torch.float32, "h_state"),
+                      (logits0, torch.float32, "logits0"), (row_index, torch.int32, "row_index"),
+                      (conf, torch.float32, "conf"), (lse, torch.float32, "lse"), (token, torch.int32, "token"),
+                      (margin, torch.float32, "margin"), (logits_out, torch.float32, "logits_out"),
+                      (hidden_out, torch.float32, "hidden_out"), (status, torch.int32, "status"),
+                      (conf_first, torch.float32, "conf_first")):
+        _check(t, dt, nm)
+    out = mrp_draft_out(_ptr(conf), _ptr(lse), _ptr(token), _ptr(margin), _ptr(logits_out), _ptr(hidden_out),
+                        _ptr(status), _ptr(conf_first))
+    rc = lib.mrp_module_step(ctx.handle, _ptr(tokens), _ptr(hidden0), _ptr(h_state), _ptr(logits0), _ptr(row_index),
+                             int(M), int(B), int(L), int(bool(first_step)), ctypes.byref(out), _stream(stream))
+    if rc != 0:
+        raise MrpError("mrp_module_step", rc, lib.mrp_last_error(ctx.handle).decode())
 
 
 def mrp_set_input_rows(ctx: Context, n_rows: int) -> None:

@@ -217,6 +217,7 @@ void mrp_destroy(mrp_ctx *ctx)
     if (!ctx) return;
     prof_release(ctx->c);
     if (ctx->c.use_tc) tc_destroy(&ctx->c);
+    free(ctx->c.module_layers);
     free(ctx->c.heads);
     delete ctx;
 }
@@ -322,6 +323,70 @@ int mrp_verify(mrp_ctx *ctx, const int32_t *draft_tok, const int32_t *verify_tok
     if (guard.err != cudaSuccess) return MRP_ERR_CUDA;
     cudaError_t e = launch_verify(&c, draft_tok, verify_tok, draft_len, B, Kd, positionwise ? 1 : 0,
                                   accept_len, accept_mask, (cudaStream_t)cuda_stream);
+    return e == cudaSuccess ? MRP_OK : MRP_ERR_CUDA;
+}
+
+static bool module_ok(const mrp_config *cfg, const mrp_module_weights *w)
+{
+    if (!cfg || !w || w->n_layers < 0 || w->n_layers > 64 || w->n_attn_heads < 1 || cfg->d % w->n_attn_heads) return false;
+    if (w->emb_rows < 1 || w->mask_token < 0 || w->mask_token >= w->emb_rows || !w->emb || !w->w_proj) return false;
+    if (w->n_layers > 0 && !w->layers) return false;
+    for (int l = 0; l < w->n_layers; ++l) {
+        const mrp_module_layer &y = w->layers[l];
+        if (!y.g_attn || !y.w_q || !y.w_k || !y.w_v || !y.w_o || !y.g_mlp || !y.w_gate || !y.w_up || !y.w_down) return false;
+    }
+    return true;
+}
+
+size_t mrp_module_workspace_bytes(const mrp_config *cfg, const mrp_module_weights *w)
+{
+    if (!config_ok(cfg) || !module_ok(cfg, w)) return 0;
+    return module_workspace_bytes(*cfg, w->n_layers);
+}
+
+int mrp_module_attach(mrp_ctx *ctx, const mrp_module_weights *w, void *workspace, size_t workspace_bytes)
+{
+    if (!ctx || !workspace || ((uintptr_t)workspace & 255u)) return MRP_ERR_INVALID_ARG;
+    Ctx &c = ctx->c;
+    if (!module_ok(&c.cfg, w)) return MRP_ERR_INVALID_ARG;
+    if (workspace_bytes < module_workspace_bytes(c.cfg, w->n_layers)) return MRP_ERR_NOMEM;
+    mrp_module_layer *copy = nullptr;
+    if (w->n_layers > 0) {
+        copy = (mrp_module_layer *)malloc(sizeof(mrp_module_layer) * (size_t)w->n_layers);
+        if (!copy) return MRP_ERR_NOMEM;
+        memcpy(copy, w->layers, sizeof(mrp_module_layer) * (size_t)w->n_layers);
+    }
+    free(c.module_layers);
+    c.module_layers = copy;
+    c.module = *w;
+    c.module.layers = copy;
+    c.module_ws = (char *)workspace;
+    c.has_module = true;
+    return MRP_OK;
+}
+
+int mrp_module_step(mrp_ctx *ctx, const int32_t *tokens, const void *hidden0, float *h_state, const float *logits0,
+                    const int32_t *row_index, int32_t M, int32_t B, int32_t L, int32_t first_step,
+                    const mrp_draft_out *out, void *cuda_stream)
+{
+    if (!ctx || !out) return MRP_ERR_INVALID_ARG;
+    Ctx &c = ctx->c;
+    if (!c.has_module || c.use_fp8_lm) return MRP_ERR_UNSUPPORTED;
+    if (B < 1 || B > c.cfg.max_seqs || L < 1 || L > c.cfg.block_len) return MRP_ERR_INVALID_ARG;
+    if (M < 0 || M > c.cfg.max_rows || (long long)M > (long long)B * L) return MRP_ERR_INVALID_ARG;
+    if (!tokens || !hidden0 || !h_state || ((uintptr_t)hidden0 & 15u) || ((uintptr_t)h_state & 15u)) return MRP_ERR_INVALID_ARG;
+    if (M > 0 && (!logits0 || ((uintptr_t)logits0 & 15u) || !out->conf || !out->lse || !out->token)) return MRP_ERR_INVALID_ARG;
+    c.launches = 0;
+    DeviceGuard guard(c.cfg.device);
+    if (guard.err != cudaSuccess) return MRP_ERR_CUDA;
+    c.err[0] = 0;
+    c.from_hidden = false; c.final_gamma = nullptr; c.teacher = nullptr; c.kl_out = nullptr; c.l0_bf16 = false;
+    const int saved_rows = c.input_rows;
+    c.input_rows = B * L;                       // the dense arrays of this call have B * L rows
+    cudaError_t e = module_step(&c, tokens, hidden0, h_state, logits0, row_index, M, B, L, first_step != 0, *out,
+                                (cudaStream_t)cuda_stream);
+    c.input_rows = saved_rows;
+    if (e != cudaSuccess && !c.err[0]) note_err(&c, e, "mrp_module_step");
     return e == cudaSuccess ? MRP_OK : MRP_ERR_CUDA;
 }
 

@@ -88,6 +88,11 @@ struct Ctx {
     int sm_count;
     void *tc_state;            // tensor-core path state (tensor maps), owned by tc_*.cu
     // Optional per-phase timing of mrp_draft (CUDA events on the call's stream).
+    // the token-conditioned module attached with mrp_module_attach (weights and workspace borrowed)
+    bool has_module;
+    mrp_module_weights module;
+    mrp_module_layer *module_layers;   // host copy [n_layers]
+    char *module_ws;
     char err[192];             // detail of the last failure ("" if none)
     bool prof_enabled;
     cudaEvent_t *prof_events;  // [kProfSlots][kProfMarks]
@@ -219,6 +224,27 @@ cudaError_t tc_create(Ctx *c);
 void tc_destroy(Ctx *c);
 cudaError_t tc_draft(Ctx *c, const void *hidden, const float *logits0, const int32_t *row_index,
                      int M, int K, const mrp_draft_out &out, cudaStream_t st);
+
+// Which kernels serve a call of M rows and K steps (tc_plan also sets the lo-block offsets lo_x / lo_xt of
+// the context for the call), and the part of a drafting pass behind the head chain: LM head on the stacked
+// operand rows already in the workspace (xt; xt16 in fp16 mode), combine, per-token probability.
+struct TcPlan {
+    bool pdl, few_rows, lm_few, f16_lm, chain, with_kl;
+    int n_rs;
+};
+TcPlan tc_plan(Ctx *c, int M, int K, const mrp_draft_out &out, cudaStream_t st, bool want_chain);
+cudaError_t tc_lm_tail(Ctx *c, const TcPlan &pl, const float *logits0, const int32_t *row_index, int M, int K,
+                       const mrp_draft_out &out, cudaStream_t st);
+// The same for the CUDA-core family (operand rows: fp32 xt).
+cudaError_t simt_lm_tail(Ctx *c, const float *logits0, const int32_t *row_index, int M, int K,
+                         const mrp_draft_out &out, cudaStream_t st);
+
+// One step of the token-conditioned module (simt_kernels.cu): module forward on CUDA cores, then the
+// context's LM-head tail.
+cudaError_t module_step(Ctx *c, const int32_t *tokens, const void *hidden0, float *h_state, const float *logits0,
+                        const int32_t *row_index, int M, int B, int L, bool first_step, const mrp_draft_out &out,
+                        cudaStream_t st);
+size_t module_workspace_bytes(const mrp_config &cfg, int n_layers);
 
 // Few-row variants (tc_skinny.cu): weight rows on the MMA M axis; rows <= 32.
 bool sk_rows_ok(int rows);          // LM head: row-steps incl. step 0

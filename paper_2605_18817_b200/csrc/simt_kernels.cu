@@ -517,6 +517,55 @@ cudaError_t launch_first_token_prob(Ctx *c, const FirstTok &f, const mrp_draft_o
 }
 
 template <typename T>
+static cudaError_t simt_lm_tail_t(Ctx *c, const float *logits0, const int32_t *row_index, int M, int K,
+                                  const mrp_draft_out &out, cudaStream_t st)
+{
+    const int d = c->cfg.d, V = c->cfg.vocab;
+    float *xt = (float *)(c->ws + c->lay.xt);
+    Partial *partials = (Partial *)(c->ws + c->lay.partials);
+    KlPartial *kl_partials = (KlPartial *)(c->ws + c->lay.kl_partials);
+    int32_t *status = (int32_t *)(c->ws + c->lay.status);
+    const bool pdl = !(c->cfg.flags & MRP_FLAG_NO_PDL);
+    float *xt0 = c->from_hidden ? xt + (size_t)K * M * d : nullptr;
+    cudaError_t e;
+    prof_mark(c, 1, st);
+    e = note_err(c, wait_logits0(c, st), "wait for the base logits");
+    if (e != cudaSuccess) return e;
+    // small vocabularies: narrower slices so that every SM gets a block
+    const bool narrow = (V + kSimtSliceV - 1) / kSimtSliceV < 2 * c->sm_count;
+    const int slice_v = narrow ? 32 : kSimtSliceV;
+    const int n_slices = (V + slice_v - 1) / slice_v;
+    const int grid = n_slices < kSimtMaxBlocks ? n_slices : kSimtMaxBlocks;
+    if (narrow)
+        e = launch_k(lm_simt_kernel<T, 32>, dim3(grid), dim3(256), 0, st, pdl, (const T *)c->w_lm, (const float *)xt,
+                     (const float *)xt0, logits0, row_index, M, K, d, V, n_slices, partials, out.logits_out,
+                     c->input_rows, c->teacher, kl_partials, c->l0_bf16 ? 1 : 0);
+    else
+        e = launch_k(lm_simt_kernel<T, kSimtSliceV>, dim3(grid), dim3(256), 0, st, pdl, (const T *)c->w_lm,
+                     (const float *)xt, (const float *)xt0, logits0, row_index, M, K, d, V, n_slices, partials,
+                     out.logits_out, c->input_rows, c->teacher, kl_partials, c->l0_bf16 ? 1 : 0);
+    c->launches++;
+    if (e != cudaSuccess) return e;
+    prof_mark(c, 2, st);
+    e = launch_combine(c, partials, grid, (K + 1) * M, out, status, st, nullptr, M);
+    prof_mark(c, 3, st);
+    if (e != cudaSuccess) return e;
+    FirstTok ft;
+    memset(&ft, 0, sizeof(ft));
+    ft.w = c->w_lm; ft.w_bf16 = c->cfg.dtype == MRP_BF16; ft.logits0 = logits0; ft.row_index = row_index;
+    ft.l0_bf16 = c->l0_bf16 ? 1 : 0;
+    ft.n_rows_in = c->input_rows; ft.x = xt; ft.x_bf16 = 0; ft.M = M; ft.K = K; ft.d = d; ft.V = V;
+    return launch_first_token_prob(c, ft, out, st);
+}
+
+cudaError_t simt_lm_tail(Ctx *c, const float *logits0, const int32_t *row_index, int M, int K,
+                         const mrp_draft_out &out, cudaStream_t st)
+{
+    if (c->cfg.dtype == MRP_F32) return simt_lm_tail_t<float>(c, logits0, row_index, M, K, out, st);
+    return simt_lm_tail_t<__nv_bfloat16>(c, logits0, row_index, M, K, out, st);
+}
+
+template <typename T>
 static cudaError_t simt_draft_t(Ctx *c, const void *hidden, const float *logits0,
                                 const int32_t *row_index, int M, int K, const mrp_draft_out &out,
                                 cudaStream_t st)
@@ -550,34 +599,7 @@ static cudaError_t simt_draft_t(Ctx *c, const void *hidden, const float *logits0
         if (e != cudaSuccess) return e;
         c->launches += 3;
     }
-    prof_mark(c, 1, st);
-    e = note_err(c, wait_logits0(c, st), "wait for the base logits");
-    if (e != cudaSuccess) return e;
-    // small vocabularies: narrower slices so that every SM gets a block
-    const bool narrow = (V + kSimtSliceV - 1) / kSimtSliceV < 2 * c->sm_count;
-    const int slice_v = narrow ? 32 : kSimtSliceV;
-    const int n_slices = (V + slice_v - 1) / slice_v;
-    const int grid = n_slices < kSimtMaxBlocks ? n_slices : kSimtMaxBlocks;
-    if (narrow)
-        e = launch_k(lm_simt_kernel<T, 32>, dim3(grid), dim3(256), 0, st, pdl, (const T *)c->w_lm, (const float *)xt,
-                     (const float *)xt0, logits0, row_index, M, K, d, V, n_slices, partials, out.logits_out,
-                     c->input_rows, c->teacher, kl_partials, c->l0_bf16 ? 1 : 0);
-    else
-        e = launch_k(lm_simt_kernel<T, kSimtSliceV>, dim3(grid), dim3(256), 0, st, pdl, (const T *)c->w_lm,
-                     (const float *)xt, (const float *)xt0, logits0, row_index, M, K, d, V, n_slices, partials,
-                     out.logits_out, c->input_rows, c->teacher, kl_partials, c->l0_bf16 ? 1 : 0);
-    c->launches++;
-    if (e != cudaSuccess) return e;
-    prof_mark(c, 2, st);
-    e = launch_combine(c, partials, grid, (K + 1) * M, out, status, st, nullptr, M);
-    prof_mark(c, 3, st);
-    if (e != cudaSuccess) return e;
-    FirstTok ft;
-    memset(&ft, 0, sizeof(ft));
-    ft.w = c->w_lm; ft.w_bf16 = c->cfg.dtype == MRP_BF16; ft.logits0 = logits0; ft.row_index = row_index;
-    ft.l0_bf16 = c->l0_bf16 ? 1 : 0;
-    ft.n_rows_in = c->input_rows; ft.x = xt; ft.x_bf16 = 0; ft.M = M; ft.K = K; ft.d = d; ft.V = V;
-    return launch_first_token_prob(c, ft, out, st);
+    return simt_lm_tail(c, logits0, row_index, M, K, out, st);
 }
 
 cudaError_t simt_draft(Ctx *c, const void *hidden, const float *logits0, const int32_t *row_index,
@@ -587,6 +609,247 @@ cudaError_t simt_draft(Ctx *c, const void *hidden, const float *logits0, const i
     if (c->cfg.dtype == MRP_F32)
         return simt_draft_t<float>(c, hidden, logits0, row_index, M, K, out, st);
     return simt_draft_t<__nv_bfloat16>(c, hidden, logits0, row_index, M, K, out, st);
+}
+
+// ---------------------------------------------------------------------------------------
+// The token-conditioned MRP module (Sec. 3.2; Algorithm 2, "Delta, delta <- g(x_t, h)") on CUDA cores.
+// fp32 activations, weights in the context's dtype.  One step = embedding fusion, D transformer layers
+// with block-local attention, h <- h + Delta, the LM-head operand h - h_0 of the masked rows, and then the
+// context's own LM-head kernels.
+// ---------------------------------------------------------------------------------------
+// [h_i ; emb[x_i]] per dense position; a token outside the table reads as masked and raises the bit.
+template <typename T>
+__global__ void mod_concat_kernel(const float *h_state, const T *__restrict__ hidden0, int first_step,
+                                  const int32_t *__restrict__ tokens, const T *__restrict__ emb, int mask_token,
+                                  int emb_rows, int d, float *h_out /* = h_state */, float *__restrict__ cat,
+                                  int32_t *__restrict__ status, int32_t *__restrict__ user_status)
+{
+    pdl_trigger();
+    pdl_wait();
+    const int i = blockIdx.x;
+    int tok = tokens[i];
+    if (tok >= emb_rows || tok < -1) {
+        if (threadIdx.x == 0) {
+            atomicOr(status, MRP_DEV_BAD_INDEX);
+            if (user_status) atomicOr(user_status, MRP_DEV_BAD_INDEX);
+        }
+        tok = -1;
+    }
+    if (tok < 0) tok = mask_token;
+    for (int j = threadIdx.x; j < d; j += blockDim.x) {
+        const float h = first_step ? ld_f(hidden0, (size_t)i * d + j) : h_state[(size_t)i * d + j];
+        if (first_step) h_out[(size_t)i * d + j] = h;
+        cat[(size_t)i * 2 * d + j] = h;
+        cat[(size_t)i * 2 * d + d + j] = ld_f(emb, (size_t)tok * d + j);
+    }
+}
+
+// y[r, j] (+)= sum_c W[j, c] x[r, c]: one warp per output feature, kRC rows at a time.
+template <typename T>
+__global__ void linear_kernel(const T *__restrict__ w, const float *__restrict__ x, int rows, int n_in, int n_out,
+                              float *__restrict__ y, int accumulate)
+{
+    pdl_trigger();
+    pdl_wait();
+    const int j = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (j >= n_out) return;
+    const T *wr = w + (size_t)j * n_in;
+    for (int r0 = 0; r0 < rows; r0 += kRC) {
+        float s[kRC];
+#pragma unroll
+        for (int r = 0; r < kRC; ++r) s[r] = 0.f;
+        for (int c = lane; c < n_in; c += 32) {
+            const float a = ld_f(wr, c);
+#pragma unroll
+            for (int r = 0; r < kRC; ++r)
+                if (r0 + r < rows) s[r] = fmaf(a, x[(size_t)(r0 + r) * n_in + c], s[r]);
+        }
+#pragma unroll
+        for (int r = 0; r < kRC; ++r) {
+            const float v = warp_sum(s[r]);
+            if (lane == 0 && r0 + r < rows) {
+                const size_t o = (size_t)(r0 + r) * n_out + j;
+                y[o] = accumulate ? y[o] + v : v;
+            }
+        }
+    }
+}
+
+// Block-local bidirectional attention: CTA = (block b, attention head); a warp per query position, lanes
+// over the key positions for the scores and over the head's features for the output.
+__global__ void mod_attention_kernel(const float *__restrict__ q, const float *__restrict__ k,
+                                     const float *__restrict__ v, int L, int d, int dh, float *__restrict__ o)
+{
+    pdl_trigger();
+    pdl_wait();
+    extern __shared__ float prob[];                  // [warps][L]
+    const int b = blockIdx.x, hd = blockIdx.y;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, n_warps = blockDim.x >> 5;
+    float *p = prob + (size_t)warp * L;
+    const float scale = rsqrtf((float)dh);
+    for (int i = warp; i < L; i += n_warps) {
+        const float *qi = q + ((size_t)b * L + i) * d + (size_t)hd * dh;
+        float mx = -INFINITY;
+        for (int j = lane; j < L; j += 32) {
+            const float *kj = k + ((size_t)b * L + j) * d + (size_t)hd * dh;
+            float sdot = 0.f;
+            for (int c = 0; c < dh; ++c) sdot = fmaf(qi[c], kj[c], sdot);
+            sdot *= scale;
+            p[j] = sdot;
+            mx = fmaxf(mx, sdot);
+        }
+#pragma unroll
+        for (int w = 16; w > 0; w >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, w));
+        float sum = 0.f;
+        for (int j = lane; j < L; j += 32) {
+            const float e = expf(p[j] - mx);
+            p[j] = e;
+            sum += e;
+        }
+        sum = warp_sum(sum);
+        __syncwarp();
+        for (int c = lane; c < dh; c += 32) {
+            float acc = 0.f;
+            for (int j = 0; j < L; ++j) acc = fmaf(p[j], v[((size_t)b * L + j) * d + (size_t)hd * dh + c], acc);
+            o[((size_t)b * L + i) * d + (size_t)hd * dh + c] = acc / sum;
+        }
+        __syncwarp();
+    }
+}
+
+// h <- h + Delta for every dense position.
+__global__ void mod_add_kernel(float *__restrict__ h_state, const float *__restrict__ z, size_t n)
+{
+    pdl_trigger();
+    pdl_wait();
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
+        h_state[i] += z[i];
+}
+
+// LM-head operand of the masked rows: h - h_0, as the context's kernel family wants it (fp32 rows for the
+// CUDA-core family; bf16 hi + lo rows of step 1 behind zero rows of step 0, plus the fp16 copy when the
+// row-major fp16 LM head runs, for the tensor-core family).
+template <typename T>
+__global__ void mod_operand_kernel(const float *__restrict__ h_state, const T *__restrict__ hidden0,
+                                   const int32_t *__restrict__ row_index, int n_rows_in, int M, int d,
+                                   float *__restrict__ xt_f32, __nv_bfloat16 *__restrict__ xt_bf16, int lo_rows,
+                                   __half *__restrict__ xt16, float *__restrict__ hidden_out,
+                                   int32_t *__restrict__ status, int32_t *__restrict__ user_status)
+{
+    pdl_trigger();
+    pdl_wait();
+    const int m = blockIdx.x;
+    const int idx = row_index ? row_index[m] : m;
+    const bool bad = !row_ok(idx, n_rows_in);
+    if (bad && threadIdx.x == 0) {
+        atomicOr(status, MRP_DEV_BAD_INDEX);
+        if (user_status) atomicOr(user_status, MRP_DEV_BAD_INDEX);
+    }
+    for (int j = threadIdx.x; j < d; j += blockDim.x) {
+        const float h = bad ? 0.f : h_state[(size_t)idx * d + j];
+        const float r = bad ? 0.f : h - ld_f(hidden0, (size_t)idx * d + j);
+        if (hidden_out) hidden_out[(size_t)m * d + j] = h;
+        if (xt_f32) xt_f32[(size_t)m * d + j] = r;
+        if (xt_bf16) {
+            const __nv_bfloat16 hi = __float2bfloat16_rn(r);
+            xt_bf16[(size_t)m * d + j] = __float2bfloat16(0.f);                          // step 0 has no residual
+            xt_bf16[((size_t)lo_rows + m) * d + j] = __float2bfloat16(0.f);
+            xt_bf16[((size_t)M + m) * d + j] = hi;
+            xt_bf16[((size_t)lo_rows + M + m) * d + j] = __float2bfloat16_rn(r - __bfloat162float(hi));
+            if (xt16) xt16[(size_t)m * d + j] = __float2half_rn(r);
+        }
+    }
+}
+
+size_t module_workspace_bytes(const mrp_config &cfg, int n_layers)
+{
+    (void)n_layers;
+    const size_t n = (size_t)cfg.max_seqs * cfg.block_len, d = (size_t)cfg.d, F = (size_t)cfg.d_ff;
+    return align_up(n * 2 * d * 4, 256) + 6 * align_up(n * d * 4, 256) + align_up(n * F * 4, 256);
+}
+
+template <typename T>
+static cudaError_t module_step_t(Ctx *c, const int32_t *tokens, const void *hidden0, float *h_state, const float *logits0,
+                                 const int32_t *row_index, int M, int B, int L, bool first_step, const mrp_draft_out &out,
+                                 cudaStream_t st)
+{
+    const mrp_module_weights &w = c->module;
+    const int d = c->cfg.d, F = c->cfg.d_ff, n = B * L, dh = d / w.n_attn_heads;
+    const size_t cap = (size_t)c->cfg.max_seqs * c->cfg.block_len;
+    char *ws = c->module_ws;
+    auto take = [&](size_t bytes) { char *p0 = ws; ws += align_up(bytes, 256); return (float *)p0; };
+    float *cat = take(cap * 2 * d * 4), *z = take(cap * d * 4), *nn = take(cap * d * 4), *q = take(cap * d * 4);
+    float *k = take(cap * d * 4), *v = take(cap * d * 4), *o = take(cap * d * 4), *act = take(cap * F * 4);
+    int32_t *status = (int32_t *)(c->ws + c->lay.status);
+    const bool pdl = !(c->cfg.flags & MRP_FLAG_NO_PDL);
+    auto lin = [&](const void *wm, const float *x, int n_in, int n_out, float *y, int acc) {
+        c->launches++;
+        return launch_k(linear_kernel<T>, dim3((n_out + 7) / 8), dim3(256), 0, st, pdl, (const T *)wm, x, n, n_in, n_out, y, acc);
+    };
+    prof_mark(c, 0, st);
+    cudaError_t e = launch_k(mod_concat_kernel<T>, dim3(n), dim3(256), 0, st, pdl, (const float *)h_state, (const T *)hidden0,
+                             first_step ? 1 : 0, tokens, (const T *)w.emb, w.mask_token, w.emb_rows, d, h_state, cat, status,
+                             out.status);
+    c->launches++;
+    if (e == cudaSuccess) e = lin(w.w_proj, cat, 2 * d, d, z, 0);
+    for (int l = 0; l < w.n_layers && e == cudaSuccess; ++l) {
+        const mrp_module_layer &y = w.layers[l];
+        e = launch_k(rmsnorm_kernel<T>, dim3(n), dim3(256), 0, st, pdl, (const float *)z, (const T *)y.g_attn, d, c->cfg.rms_eps, nn);
+        c->launches++;
+        if (e == cudaSuccess) e = lin(y.w_q, nn, d, d, q, 0);
+        if (e == cudaSuccess) e = lin(y.w_k, nn, d, d, k, 0);
+        if (e == cudaSuccess) e = lin(y.w_v, nn, d, d, v, 0);
+        if (e == cudaSuccess) {
+            e = launch_k(mod_attention_kernel, dim3(B, w.n_attn_heads), dim3(128), (size_t)4 * L * 4, st, pdl, (const float *)q,
+                         (const float *)k, (const float *)v, L, d, dh, o);
+            c->launches++;
+        }
+        if (e == cudaSuccess) e = lin(y.w_o, o, d, d, z, 1);
+        if (e == cudaSuccess) {
+            e = launch_k(rmsnorm_kernel<T>, dim3(n), dim3(256), 0, st, pdl, (const float *)z, (const T *)y.g_mlp, d, c->cfg.rms_eps, nn);
+            c->launches++;
+        }
+        if (e == cudaSuccess) {
+            e = launch_k(gateup_kernel<T>, dim3((F + 7) / 8), dim3(256), 0, st, pdl, (const T *)y.w_gate, (const T *)y.w_up,
+                         (const float *)nn, n, d, F, act);
+            c->launches++;
+        }
+        if (e == cudaSuccess) e = lin(y.w_down, act, F, d, z, 1);
+    }
+    if (e == cudaSuccess) {
+        const size_t total = (size_t)n * d;
+        e = launch_k(mod_add_kernel, dim3((unsigned)((total + 255) / 256 < 1184 ? (total + 255) / 256 : 1184)), dim3(256), 0, st, pdl,
+                     h_state, (const float *)z, total);
+        c->launches++;
+    }
+    if (e != cudaSuccess || M == 0) return e;
+    // the LM-head operand of the masked rows, then the context's LM-head kernels (K = 1)
+    if (c->use_tc) {
+        const TcPlan pl = tc_plan(c, M, 1, out, st, false);
+        __nv_bfloat16 *xt = (__nv_bfloat16 *)(c->ws + c->lay.xt);
+        e = launch_k(mod_operand_kernel<T>, dim3(M), dim3(256), 0, st, pdl, (const float *)h_state, (const T *)hidden0, row_index,
+                     n, M, d, (float *)nullptr, xt, c->lo_xt, pl.f16_lm ? (__half *)(c->ws + c->lay.xt16) : (__half *)nullptr,
+                     out.hidden_out, status, out.status);
+        c->launches++;
+        if (e != cudaSuccess) return e;
+        return tc_lm_tail(c, pl, logits0, row_index, M, 1, out, st);
+    }
+    e = launch_k(mod_operand_kernel<T>, dim3(M), dim3(256), 0, st, pdl, (const float *)h_state, (const T *)hidden0, row_index, n,
+                 M, d, (float *)(c->ws + c->lay.xt), (__nv_bfloat16 *)nullptr, 0, (__half *)nullptr, out.hidden_out, status,
+                 out.status);
+    c->launches++;
+    if (e != cudaSuccess) return e;
+    return simt_lm_tail(c, logits0, row_index, M, 1, out, st);
+}
+
+cudaError_t module_step(Ctx *c, const int32_t *tokens, const void *hidden0, float *h_state, const float *logits0,
+                        const int32_t *row_index, int M, int B, int L, bool first_step, const mrp_draft_out &out,
+                        cudaStream_t st)
+{
+    if (c->cfg.dtype == MRP_F32)
+        return module_step_t<float>(c, tokens, hidden0, h_state, logits0, row_index, M, B, L, first_step, out, st);
+    return module_step_t<__nv_bfloat16>(c, tokens, hidden0, h_state, logits0, row_index, M, B, L, first_step, out, st);
 }
 
 }  // namespace mrp

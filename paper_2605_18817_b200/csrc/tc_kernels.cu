@@ -633,104 +633,36 @@ void tc_destroy(Ctx *c)
     c->tc_state = nullptr;
 }
 
-cudaError_t tc_draft(Ctx *c, const void *hidden, const float *logits0, const int32_t *row_index, int M,
-                     int K, const mrp_draft_out &out, cudaStream_t st)
+TcPlan tc_plan(Ctx *c, int M, int K, const mrp_draft_out &out, cudaStream_t st, bool want_chain)
 {
-    if (M == 0) return cudaSuccess;
-    if (K == 0) return simt_draft(c, hidden, logits0, row_index, M, K, out, st);
+    TcPlan pl;
+    pl.n_rs = (K + 1) * M;
+    pl.pdl = !(c->cfg.flags & MRP_FLAG_NO_PDL);
+    pl.few_rows = sk_head_rows_ok(M) && sk_heads_ok(c->cfg) && !(c->cfg.flags & MRP_FLAG_ROW_MAJOR_ONLY);
+    // the KL objective lives in the row-major LM-head kernel, on exact operands
+    pl.with_kl = c->teacher != nullptr;
+    pl.lm_few = sk_rows_ok(pl.n_rs) && !(c->cfg.flags & MRP_FLAG_ROW_MAJOR_ONLY) && !pl.with_kl;
+    pl.f16_lm = c->use_f16_lm && pl.n_rs >= kF16MinRowSteps && !pl.lm_few && !pl.with_kl;
+    pl.chain = want_chain && !(c->cfg.flags & (MRP_FLAG_ROW_MAJOR_ONLY | MRP_FLAG_NO_CHAIN)) && sk_heads_ok(c->cfg) &&
+               sk_chain(c, M, K, out, st, pl.f16_lm, true) == cudaSuccess;
+    c->lo_x = (pl.few_rows || pl.chain) ? sk_head_pad(M) : M;
+    c->lo_xt = pl.lm_few ? sk_lm_pad(pl.n_rs) : pl.n_rs;
+    return pl;
+}
+
+// The LM head on the stacked operand rows already in the workspace (xt, and xt16 in fp16 mode), the
+// combine and the optional per-token probability: everything of a drafting pass behind the head chain.
+cudaError_t tc_lm_tail(Ctx *c, const TcPlan &pl, const float *logits0, const int32_t *row_index, int M, int K,
+                              const mrp_draft_out &out, cudaStream_t st)
+{
     const TcState *s = (const TcState *)c->tc_state;
-    const int d = c->cfg.d, F = c->cfg.d_ff, V = c->cfg.vocab;
-    const int G = c->sm_count;
-    float *h0f = (float *)(c->ws + c->lay.h0f), *hcur = (float *)(c->ws + c->lay.hcur);
-    __nv_bfloat16 *xg = (__nv_bfloat16 *)(c->ws + c->lay.xg), *act = (__nv_bfloat16 *)(c->ws + c->lay.act);
+    const int d = c->cfg.d, F = c->cfg.d_ff, V = c->cfg.vocab, G = c->sm_count;
     __nv_bfloat16 *xt = (__nv_bfloat16 *)(c->ws + c->lay.xt);
-    float *sumsq = (float *)(c->ws + c->lay.sumsq);
     Partial *partials = (Partial *)(c->ws + c->lay.partials);
     int32_t *status = (int32_t *)(c->ws + c->lay.status);
-    if (G > kSumsqSlices || G > c->lay.n_slices_max)
-        return note_err(c, cudaErrorInvalidValue, "workspace slices");
-    const int n_mb = (M + 127) / 128;
-
-    const int n_rs = (K + 1) * M;
-    // which kernel family runs the head chain and the LM head of this call
-    const bool pdl = !(c->cfg.flags & MRP_FLAG_NO_PDL);
-    const bool few_rows = sk_head_rows_ok(M) && sk_heads_ok(c->cfg) &&
-                          !(c->cfg.flags & MRP_FLAG_ROW_MAJOR_ONLY);
-    // the KL objective lives in the row-major LM-head kernel, on exact operands
-    const bool with_kl = c->teacher != nullptr;
-    const bool lm_few = sk_rows_ok(n_rs) && !(c->cfg.flags & MRP_FLAG_ROW_MAJOR_ONLY) && !with_kl;
-    const bool f16_lm = c->use_f16_lm && n_rs >= kF16MinRowSteps && !lm_few && !with_kl;
-    const bool chain = !(c->cfg.flags & (MRP_FLAG_ROW_MAJOR_ONLY | MRP_FLAG_NO_CHAIN)) && sk_heads_ok(c->cfg) &&
-                       sk_chain(c, M, K, out, st, f16_lm, true) == cudaSuccess;
-    c->lo_x = (few_rows || chain) ? sk_head_pad(M) : M;
-    c->lo_xt = lm_few ? sk_lm_pad(n_rs) : n_rs;
-
-    prof_mark(c, 0, st);
-    cudaError_t e = note_err(c, launch_k(tc_prep_kernel, dim3(M), dim3(256), 0, st, !(c->cfg.flags & MRP_FLAG_NO_PDL),
-                                         (const __nv_bfloat16 *)hidden, row_index, d, c->lo_x, c->lo_xt,
-                                      (const __nv_bfloat16 *)c->heads[0].rms_gamma, h0f, hcur, xg, xt, sumsq,
-                                      (int32_t *)(c->ws + c->lay.sk_counters), kSkMaxTiles,
-                                      (unsigned long long *)(c->ws + c->lay.ssq_fix), c->from_hidden ? 1 : 0,
-                                      (const __nv_bfloat16 *)c->final_gamma, c->cfg.rms_eps,
-                                      (c->from_hidden && f16_lm) ? (__half *)(c->ws + c->lay.xt16) : (__half *)nullptr,
-                                      c->input_rows, status, out.status),
-                             "tc_prep_kernel");
-    c->launches++;
-    if (e != cudaSuccess) return e;
-
-    int n_ss = 1;
-    bool chain_done = false;
-    if (chain) {
-        e = sk_chain(c, M, K, out, st, f16_lm, false);
-        if (e != cudaSuccess) return e;
-        chain_done = true;
-    }
-    for (int k = 1; k <= K && !chain_done; ++k) {
-        if (few_rows) {
-            e = sk_gateup(c, k, M, K, n_ss, out, st, pdl);
-            if (e != cudaSuccess) return e;
-            e = sk_down(c, k, M, K, out, st, pdl, &n_ss, f16_lm);
-            if (e != cudaSuccess) return e;
-            continue;
-        }
-        const mrp_head_weights &hw = c->heads[k - 1];
-        CUtensorMap mA, mB0, mB1;
-        // gate/up + SwiGLU
-        TcParams p;
-        memset(&p, 0, sizeof(p));
-        p.units_total = F / 8; p.unit_rows = 8; p.n_boxes = 2; p.k_chunks = d / kBK;
-        p.n_groups = choose_groups(n_mb, p.units_total, G); p.n_rb = n_mb; p.rows = M; p.a_row_base = 0; p.a_part_rows = M;
-        p.M = M; p.K = K; p.V = V; p.d = d; p.F = F; p.n_rs = n_rs;
-        p.sumsq = sumsq; p.n_ss = n_ss; p.eps = c->cfg.rms_eps; p.act = act;
-        p.status = status; p.user_status = out.status;
-        finish_shape(p, G / p.n_groups);
-        if (!make_map(s, &mA, xg, d, 2 * (uint64_t)M, 128) || !make_map(s, &mB0, hw.w_gate, d, F, p.bn / 2) ||
-            !make_map(s, &mB1, hw.w_up, d, F, p.bn / 2))
-            return note_err(c, cudaErrorInvalidValue, "tensor map (gate/up)");
-        e = note_err(c, launch_tc<KIND_GU, false>(mA, mB0, mB1, p, p.n_groups * p.n_vr, st, pdl), "gate/up kernel");
-        c->launches++;
-        if (e != cudaSuccess) return e;
-        // down projection, residual add, next operands
-        memset(&p, 0, sizeof(p));
-        p.units_total = d / 16; p.unit_rows = 16; p.n_boxes = 1; p.k_chunks = F / kBK;
-        p.n_groups = choose_groups(n_mb, p.units_total, G); p.n_rb = n_mb; p.rows = M;
-        p.M = M; p.K = K; p.V = V; p.d = d; p.F = F; p.n_rs = n_rs; p.a_part_rows = M;
-        p.hcur = hcur; p.h0f = h0f;
-        p.gamma_next = (k < K) ? (const __nv_bfloat16 *)c->heads[k].rms_gamma : nullptr;
-        p.xg_next = (k < K) ? xg : nullptr;
-        p.xt_k = xt + (size_t)k * M * d;
-        p.xt16_k = f16_lm ? (__half *)(c->ws + c->lay.xt16) + (size_t)(k - (c->from_hidden ? 0 : 1)) * M * d : nullptr;
-        p.sumsq_out = sumsq;
-        p.hidden_out = (k == K) ? out.hidden_out : nullptr;
-        p.status = status; p.user_status = out.status;
-        finish_shape(p, G / p.n_groups);
-        if (!make_map(s, &mA, act, F, 2 * (uint64_t)M, 128) || !make_map(s, &mB0, hw.w_down, F, d, p.bn))
-            return note_err(c, cudaErrorInvalidValue, "tensor map (down)");
-        e = note_err(c, launch_tc<KIND_DN, false>(mA, mB0, mB0, p, p.n_groups * p.n_vr, st, pdl), "down kernel");
-        c->launches++;
-        if (e != cudaSuccess) return e;
-        n_ss = p.n_vr;
-    }
+    const int n_rs = pl.n_rs;
+    const bool pdl = pl.pdl, lm_few = pl.lm_few, f16_lm = pl.f16_lm, with_kl = pl.with_kl;
+    cudaError_t e;
     prof_mark(c, 1, st);
     e = note_err(c, wait_logits0(c, st), "wait for the base logits");
     if (e != cudaSuccess) return e;
@@ -801,6 +733,96 @@ cudaError_t tc_draft(Ctx *c, const void *hidden, const float *logits0, const int
     if (c->use_fp8_lm) { ft.w = c->ws + c->lay.w8; ft.w8_scale = (const float *)(c->ws + c->lay.w8_scale); }
     ft.x = xt; ft.x_bf16 = 1; ft.lo_rows = c->lo_xt; ft.M = M; ft.K = K; ft.d = d; ft.V = V;
     return launch_first_token_prob(c, ft, out, st);
+}
+cudaError_t tc_draft(Ctx *c, const void *hidden, const float *logits0, const int32_t *row_index, int M,
+                     int K, const mrp_draft_out &out, cudaStream_t st)
+{
+    if (M == 0) return cudaSuccess;
+    if (K == 0) return simt_draft(c, hidden, logits0, row_index, M, K, out, st);
+    const TcState *s = (const TcState *)c->tc_state;
+    const int d = c->cfg.d, F = c->cfg.d_ff, V = c->cfg.vocab;
+    const int G = c->sm_count;
+    float *h0f = (float *)(c->ws + c->lay.h0f), *hcur = (float *)(c->ws + c->lay.hcur);
+    __nv_bfloat16 *xg = (__nv_bfloat16 *)(c->ws + c->lay.xg), *act = (__nv_bfloat16 *)(c->ws + c->lay.act);
+    __nv_bfloat16 *xt = (__nv_bfloat16 *)(c->ws + c->lay.xt);
+    float *sumsq = (float *)(c->ws + c->lay.sumsq);
+    Partial *partials = (Partial *)(c->ws + c->lay.partials);
+    int32_t *status = (int32_t *)(c->ws + c->lay.status);
+    if (G > kSumsqSlices || G > c->lay.n_slices_max)
+        return note_err(c, cudaErrorInvalidValue, "workspace slices");
+    const int n_mb = (M + 127) / 128;
+
+    const TcPlan pl = tc_plan(c, M, K, out, st, true);
+    const int n_rs = pl.n_rs;
+    const bool pdl = pl.pdl, few_rows = pl.few_rows, f16_lm = pl.f16_lm, chain = pl.chain;
+
+    prof_mark(c, 0, st);
+    cudaError_t e = note_err(c, launch_k(tc_prep_kernel, dim3(M), dim3(256), 0, st, !(c->cfg.flags & MRP_FLAG_NO_PDL),
+                                         (const __nv_bfloat16 *)hidden, row_index, d, c->lo_x, c->lo_xt,
+                                      (const __nv_bfloat16 *)c->heads[0].rms_gamma, h0f, hcur, xg, xt, sumsq,
+                                      (int32_t *)(c->ws + c->lay.sk_counters), kSkMaxTiles,
+                                      (unsigned long long *)(c->ws + c->lay.ssq_fix), c->from_hidden ? 1 : 0,
+                                      (const __nv_bfloat16 *)c->final_gamma, c->cfg.rms_eps,
+                                      (c->from_hidden && f16_lm) ? (__half *)(c->ws + c->lay.xt16) : (__half *)nullptr,
+                                      c->input_rows, status, out.status),
+                             "tc_prep_kernel");
+    c->launches++;
+    if (e != cudaSuccess) return e;
+
+    int n_ss = 1;
+    bool chain_done = false;
+    if (chain) {
+        e = sk_chain(c, M, K, out, st, f16_lm, false);
+        if (e != cudaSuccess) return e;
+        chain_done = true;
+    }
+    for (int k = 1; k <= K && !chain_done; ++k) {
+        if (few_rows) {
+            e = sk_gateup(c, k, M, K, n_ss, out, st, pdl);
+            if (e != cudaSuccess) return e;
+            e = sk_down(c, k, M, K, out, st, pdl, &n_ss, f16_lm);
+            if (e != cudaSuccess) return e;
+            continue;
+        }
+        const mrp_head_weights &hw = c->heads[k - 1];
+        CUtensorMap mA, mB0, mB1;
+        // gate/up + SwiGLU
+        TcParams p;
+        memset(&p, 0, sizeof(p));
+        p.units_total = F / 8; p.unit_rows = 8; p.n_boxes = 2; p.k_chunks = d / kBK;
+        p.n_groups = choose_groups(n_mb, p.units_total, G); p.n_rb = n_mb; p.rows = M; p.a_row_base = 0; p.a_part_rows = M;
+        p.M = M; p.K = K; p.V = V; p.d = d; p.F = F; p.n_rs = n_rs;
+        p.sumsq = sumsq; p.n_ss = n_ss; p.eps = c->cfg.rms_eps; p.act = act;
+        p.status = status; p.user_status = out.status;
+        finish_shape(p, G / p.n_groups);
+        if (!make_map(s, &mA, xg, d, 2 * (uint64_t)M, 128) || !make_map(s, &mB0, hw.w_gate, d, F, p.bn / 2) ||
+            !make_map(s, &mB1, hw.w_up, d, F, p.bn / 2))
+            return note_err(c, cudaErrorInvalidValue, "tensor map (gate/up)");
+        e = note_err(c, launch_tc<KIND_GU, false>(mA, mB0, mB1, p, p.n_groups * p.n_vr, st, pdl), "gate/up kernel");
+        c->launches++;
+        if (e != cudaSuccess) return e;
+        // down projection, residual add, next operands
+        memset(&p, 0, sizeof(p));
+        p.units_total = d / 16; p.unit_rows = 16; p.n_boxes = 1; p.k_chunks = F / kBK;
+        p.n_groups = choose_groups(n_mb, p.units_total, G); p.n_rb = n_mb; p.rows = M;
+        p.M = M; p.K = K; p.V = V; p.d = d; p.F = F; p.n_rs = n_rs; p.a_part_rows = M;
+        p.hcur = hcur; p.h0f = h0f;
+        p.gamma_next = (k < K) ? (const __nv_bfloat16 *)c->heads[k].rms_gamma : nullptr;
+        p.xg_next = (k < K) ? xg : nullptr;
+        p.xt_k = xt + (size_t)k * M * d;
+        p.xt16_k = f16_lm ? (__half *)(c->ws + c->lay.xt16) + (size_t)(k - (c->from_hidden ? 0 : 1)) * M * d : nullptr;
+        p.sumsq_out = sumsq;
+        p.hidden_out = (k == K) ? out.hidden_out : nullptr;
+        p.status = status; p.user_status = out.status;
+        finish_shape(p, G / p.n_groups);
+        if (!make_map(s, &mA, act, F, 2 * (uint64_t)M, 128) || !make_map(s, &mB0, hw.w_down, F, d, p.bn))
+            return note_err(c, cudaErrorInvalidValue, "tensor map (down)");
+        e = note_err(c, launch_tc<KIND_DN, false>(mA, mB0, mB0, p, p.n_groups * p.n_vr, st, pdl), "down kernel");
+        c->launches++;
+        if (e != cudaSuccess) return e;
+        n_ss = p.n_vr;
+    }
+    return tc_lm_tail(c, pl, logits0, row_index, M, K, out, st);
 }
 
 }  // namespace mrp

@@ -315,6 +315,8 @@ sk_gemm_kernel(const __grid_constant__ SkMaps maps, const SkParams p)
 #pragma unroll
                 for (int j = 0; j < RP; ++j)
                     a[j] = (valid && j < p.n_rs && rowoff_s[j] >= 0) ? ld_l0(p.logits0, p.l0_bf16, (size_t)(rowoff_s[j] + v)) : 0.f;
+                float ws = 0.f;                              // 8-bit weights: the scale of this thread's vocabulary row
+                if (FP8 && valid) ws = __ldg(p.w8_scale + v);
                 ok = __all_sync(0xffffffffu, mbar_wait(tfull_bar(acc), acc_ph, abort_flag, p));
                 if (!ok) break;
                 tc_fence_after();
@@ -329,7 +331,6 @@ sk_gemm_kernel(const __grid_constant__ SkMaps maps, const SkParams p)
                     }
                 } else {
                     // delta = (row scale of W) * (scale of the row-step) * sum_i 16^-i (W8 . limb_i)
-                    const float ws = valid ? __ldg(p.w8_scale + v) : 0.f;
                     float dsum[RP];
 #pragma unroll
                     for (int j = 0; j < RP; ++j) dsum[j] = 0.f;

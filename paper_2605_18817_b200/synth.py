@@ -93,6 +93,41 @@ def make_weights(d: int, F: int, V: int, n_heads: int, dtype: str, seed: int,
     return Weights(d, F, V, dtype, w_lm, heads)
 
 
+@dataclass
+class ModuleWeights:
+    """Weights of the token-conditioned MRP module (Sec. 3.2): frozen embedding table, fusion projection,
+    D transformer layers.  float32 arrays (bf16-representable when dtype == "bf16")."""
+    D: int
+    n_attn_heads: int
+    mask_token: int
+    emb: np.ndarray                 # [V, d]
+    w_proj: np.ndarray              # [d, 2d]
+    layers: list = field(default_factory=list)   # dicts g_attn, w_q, w_k, w_v, w_o, g_mlp, w_gate, w_up, w_down
+
+
+def make_module_weights(d: int, F: int, V: int, D: int, n_attn_heads: int, dtype: str, seed: int,
+                        std: float = 0.02, proj_std: float | None = None) -> ModuleWeights:
+    """Embeddings ~ N(0, 1); projection ~ N(0, proj_std^2) (default 1/sqrt(2d): an output of order one);
+    layer matrices ~ N(0, std^2); norm weights 1 + 0.1 cos (non-trivial so that a dropped one shows)."""
+    ps = proj_std if proj_std is not None else 1.0 / math.sqrt(2.0 * d)
+    st = 500
+    emb = _normal(seed, st, (V, d), 1.0, dtype)
+    w_proj = _normal(seed, st + 1, (d, 2 * d), ps, dtype)
+    layers = []
+    for l in range(D):
+        b = st + 10 * (l + 1)
+        g1 = (1.0 + 0.1 * np.cos(np.arange(d) + l)).astype(np.float32)
+        g2 = (1.0 + 0.1 * np.sin(np.arange(d) + l)).astype(np.float32)
+        if dtype == "bf16":
+            g1, g2 = bf16_round(g1), bf16_round(g2)
+        layers.append({
+            "g_attn": g1, "w_q": _normal(seed, b, (d, d), std, dtype), "w_k": _normal(seed, b + 1, (d, d), std, dtype),
+            "w_v": _normal(seed, b + 2, (d, d), std, dtype), "w_o": _normal(seed, b + 3, (d, d), std, dtype),
+            "g_mlp": g2, "w_gate": _normal(seed, b + 4, (F, d), std, dtype), "w_up": _normal(seed, b + 5, (F, d), std, dtype),
+            "w_down": _normal(seed, b + 6, (d, F), std, dtype)})
+    return ModuleWeights(D, n_attn_heads, V - 1, emb, w_proj, layers)
+
+
 def planted_gain(s: np.ndarray, V: int, calibrated: bool = True) -> np.ndarray:
     """Logit advantage given to the planted token for a planted strength ``s``.
 

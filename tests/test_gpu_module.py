@@ -1,0 +1,113 @@
+"""The token-conditioned MRP module (mrp_module_step) against the oracle's module, step by step through
+the direct-decoding loop of Algorithm 2: after every MRP step the running hidden states, the statistics of
+the running logits l <- l + delta and the reveal they drive are compared, and the tokens revealed so far
+condition the next step on both sides."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2605_18817_b200 import binding, harness, synth
+from test_gpu_parity import DEV, TOL
+
+pytestmark = pytest.mark.gpu
+
+
+def upload_module(mw, dtype):
+    up = lambda a: harness.to_device(a, dtype, DEV)
+    return up(mw.emb), up(mw.w_proj), [{k: up(v) for k, v in lay.items()} for lay in mw.layers]
+
+
+@pytest.mark.parametrize("dtype,flags,d,F,V,D,heads,B,L,steps", [
+    ("f32", 0, 64, 96, 512, 2, 4, 3, 4, 3),                                 # CUDA-core LM head
+    ("bf16", binding.MRP_FLAG_FORCE_SIMT, 64, 96, 512, 1, 2, 2, 5, 2),
+    ("bf16", 0, 256, 512, 4096, 3, 4, 1, 4, 3),                             # the paper's depth; few-row tcgen05 LM head
+    ("bf16", 0, 128, 256, 2048, 2, 4, 10, 4, 2),                            # 80 row-steps: row-major LM head, fp16 operand
+    ("bf16", 0, 256, 512, 4096, 0, 4, 2, 4, 1),                             # the fusion projection alone
+])
+def test_module_steps_follow_the_oracle_through_direct_decoding(dtype, flags, d, F, V, D, heads, B, L, steps):
+    w = synth.make_weights(d, F, V, 1, dtype, 41)
+    mw = synth.make_module_weights(d, F, V, D, heads, dtype, 41, std=0.06, proj_std=0.3 / np.sqrt(2 * d))
+    inp = synth.make_inputs(w, B, L, 41, 1.0, 3.0)
+    n = B * L
+    heads_dev, w_lm = harness.upload_weights(w, DEV)
+    ctx = binding.mrp_create(d, F, V, heads_dev, w_lm, max_rows=n, max_seqs=B, block_len=L, flags=flags)
+    emb, w_proj, layers = upload_module(mw, dtype)
+    binding.mrp_module_attach(ctx, emb, w_proj, layers, heads, mw.mask_token)
+    hid0 = harness.to_device(inp.hidden, dtype, DEV)
+    l0 = torch.from_numpy(inp.logits0).to(DEV)
+    h_state = torch.empty((n, d), device=DEV, dtype=torch.float32)
+    tol = TOL[dtype] if dtype == "bf16" else 5e-5          # fp32: D layers of fp32 sums in front of the LM head
+
+    tokens = np.full(n, -1, np.int32)                       # x_t: the active blocks, fully masked
+    h_run = inp.hidden.astype(np.float64)                   # oracle's running h
+    l_run = inp.logits0.astype(np.float64)                  # oracle's running l
+    conf0, lse0, tok0, margin0 = oracle.stats(l_run)
+    # the backbone's own reveal (Algorithm 2: r tokens of highest confidence before the MRP steps)
+    sel = oracle.select(conf0[None, :].astype(np.float32), tok0[None, :], None, B, L, oracle.STATIC, r_reveal=1)
+    tokens = np.where(sel.out_token >= 0, sel.out_token, tokens).astype(np.int32)
+    for s in range(1, steps + 1):
+        ri = np.flatnonzero(tokens < 0).astype(np.int32)
+        M = ri.size
+        if M == 0:
+            break
+        out = harness.alloc_draft_out(M, 1, V, d, DEV, hidden=True)
+        binding.mrp_module_step(ctx, torch.from_numpy(tokens).to(DEV), hid0, h_state, l0, torch.from_numpy(ri).to(DEV),
+                                M, B, L, s == 1, out.conf, out.lse, out.token, margin=out.margin,
+                                hidden_out=out.hidden, status=out.status)
+        torch.cuda.synchronize()
+        assert int(out.status.item()) == 0
+        dh, dl = oracle.module(h_run.astype(np.float32), tokens, B, L, mw.emb, mw.w_proj, mw.layers, w.w_lm, heads,
+                               mw.mask_token, row_index=ri)
+        assert D == 0 or np.abs(dh).max() > 1e-2
+        h_run = h_run.astype(np.float32).astype(np.float64) + dh
+        l_run[ri] += dl
+        conf, lse, tok, margin = oracle.stats(l_run[ri])
+        assert np.abs(h_state.cpu().numpy() - h_run).max() <= 1e-3 * max(1.0, np.abs(h_run).max())
+        assert np.abs(out.hidden.cpu().numpy() - h_run[ri]).max() <= 1e-3 * max(1.0, np.abs(h_run).max())
+        g_conf, g_lse, g_tok = (t.cpu().numpy() for t in (out.conf, out.lse, out.token))
+        assert np.abs(g_conf[1] - conf).max() <= tol and np.abs(g_lse[1] - lse).max() <= tol
+        assert np.abs(g_conf[0] - conf0[ri]).max() <= tol and np.abs(g_lse[0] - lse0[ri]).max() <= tol
+        clear = margin > 1e-2
+        assert np.array_equal(g_tok[1][clear], tok[clear])
+        # reveal from the updated logits: the device's rule on its own statistics is the oracle's rule
+        gsel = harness.alloc_select_out(B, L, 0, DEV)
+        harness.select(ctx, out.conf[1:2].contiguous(), out.token[1:2].contiguous(), torch.from_numpy(ri).to(DEV), M, 0,
+                       B, L, binding.MRP_SELECT_STATIC, gsel, r_reveal=1)
+        torch.cuda.synchronize()
+        osel_g = oracle.select(g_conf[1:2], g_tok[1:2], ri, B, L, oracle.STATIC, r_reveal=1)
+        assert np.array_equal(gsel.out_token.cpu().numpy(), osel_g.out_token)
+        # the oracle's own reveal conditions the next step on both sides
+        osel = oracle.select(conf[None, :].astype(np.float32), tok[None, :], ri, B, L, oracle.STATIC, r_reveal=1)
+        tokens = np.where(osel.out_token >= 0, osel.out_token, tokens).astype(np.int32)
+    binding.mrp_destroy(ctx)
+
+
+def test_module_step_checks_tokens_and_needs_an_attached_module():
+    d, F, V = 64, 96, 512
+    w = synth.make_weights(d, F, V, 1, "f32", 43)
+    mw = synth.make_module_weights(d, F, V, 1, 2, "f32", 43, std=0.05)
+    inp = synth.make_inputs(w, 2, 4, 43, 1.0, 3.0)
+    heads_dev, w_lm = harness.upload_weights(w, DEV)
+    ctx = binding.mrp_create(d, F, V, heads_dev, w_lm, max_rows=8, max_seqs=2, block_len=4)
+    hid0 = harness.to_device(inp.hidden, "f32", DEV)
+    l0 = torch.from_numpy(inp.logits0).to(DEV)
+    h_state = torch.empty((8, d), device=DEV)
+    out = harness.alloc_draft_out(8, 1, V, d, DEV)
+    tok = torch.full((8,), -1, device=DEV, dtype=torch.int32)
+    with pytest.raises(binding.MrpError) as ei:
+        binding.mrp_module_step(ctx, tok, hid0, h_state, l0, None, 8, 2, 4, True, out.conf, out.lse, out.token)
+    assert ei.value.status == 2
+    emb, w_proj, layers = upload_module(mw, "f32")
+    binding.mrp_module_attach(ctx, emb, w_proj, layers, 2, mw.mask_token)
+    # a token id outside the embedding table is read as masked and raises the bit
+    bad = tok.clone()
+    bad[3] = V + 5
+    binding.mrp_module_step(ctx, bad, hid0, h_state, l0, None, 8, 2, 4, True, out.conf, out.lse, out.token, status=out.status)
+    torch.cuda.synchronize()
+    assert int(out.status.item()) == binding.MRP_DEV_BAD_INDEX
+    ref = harness.alloc_draft_out(8, 1, V, d, DEV)
+    binding.mrp_module_step(ctx, tok, hid0, h_state, l0, None, 8, 2, 4, True, ref.conf, ref.lse, ref.token, status=ref.status)
+    torch.cuda.synchronize()
+    assert int(ref.status.item()) == 0 and torch.equal(ref.conf, out.conf) and torch.equal(ref.token, out.token)
+    binding.mrp_destroy(ctx)
