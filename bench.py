@@ -39,7 +39,8 @@ UNIT = "draft tokens/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 NOMINAL = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}     # the figures the benchmark spec names
 HEADLINE = "3"
-DEFAULT_WORKLOADS = ("0", "1", "2", "3", "sweep:1:1", "sweep:64:4", "sweep:256:1", "sweep:4096:4")
+DEFAULT_WORKLOADS = ("0", "1", "module", "2", "3", "sweep:1:1", "sweep:64:4", "sweep:256:1", "sweep:4096:4")
+MODULE_LAYERS, MODULE_ATTN_HEADS = 3, 16      # the paper's depth D = 3 (Sec. 4.1); 128 features per attention head
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the fused LM-head kernel, from
 # the ncu captures summarised under profiles/ (bytes per launch, and the summary they come from).
@@ -368,6 +369,55 @@ class Bench:
             self.weights[key] = (w, heads, w_lm)
         return self.weights[key]
 
+    def time_step(self, step, units_per_step, launches, ctx=None, cfg=None, M=None):
+        """Warm-up, then batches of --steps steps (CUDA events around every batch) until --min-seconds of GPU
+        time; the median batch gives the time per step; clocks sampled inside the region.  With cfg: the
+        common keys of a workload's result."""
+        import numpy as np
+        import torch
+        args, dev, dist = self.args, self.dev, self.dist
+        S = max(args.steps, 1)
+        warm = max(args.warmup, 3)
+        for _ in range(warm):
+            step()
+        # one batch to size the run
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(S):
+            step()
+        e1.record()
+        torch.cuda.synchronize()
+        n_batches = int(max(1, min(5000, np.ceil(args.min_seconds * 1e3 / max(e0.elapsed_time(e1), 1e-3)))))
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(n_batches + 1)]
+        sampler = ClockSampler(self.local)
+        sampler.start()
+        time.sleep(0.12)                       # the sampler's first line
+        self.barrier()
+        t_wall0 = time.time()
+        evs[0].record()
+        for b in range(n_batches):
+            for _ in range(S):
+                step()
+            evs[b + 1].record()
+        self.barrier()
+        t_wall1 = time.time()
+        sampler.stop()
+        batch_ms = sorted(evs[b].elapsed_time(evs[b + 1]) for b in range(n_batches))
+        med = batch_ms[len(batch_ms) // 2]
+        clocks = sampler.summary(t_wall0, t_wall1)
+        value, sec_batch = replica_throughput(dist, dev, units_per_step * S, med * 1e-3)
+        ms_step = sec_batch * 1e3 / S
+
+        out = {"value": value, "unit": UNIT, "ms_per_step": ms_step, "steps_per_batch": S, "batches": n_batches,
+               "batch_ms_median": med, "batch_ms_min": batch_ms[0], "batch_ms_max": batch_ms[-1],
+               "timed_gpu_seconds": sum(batch_ms) * 1e-3, "clocks": clocks,
+               "gpu_launches": launches[0] * S * n_batches, "launches_per_step": launches[0]}
+        if cfg is not None:
+            out["dtype"] = "bf16" if cfg["dtype"] == "bf16" else "f32"
+            out["config"] = config_dict(cfg, M, "mrp_module_step x %d" % cfg["K"])
+        return out
+
     # -------------------------------------------------------------------------------------
     def run_workload(self, name, cpu_budget_s):
         import numpy as np
@@ -438,38 +488,9 @@ class Bench:
         if static:   # synthetic backbone verification tokens for the drafted tokens
             vt.copy_(torch.from_numpy(synth.make_verify_tokens(sel.draft_tok.cpu().numpy(), w.V, cfg["seed"], 0.7)))
 
-        S = max(args.steps, 1)
-        warm = max(args.warmup, 3)
-        for _ in range(warm):
-            step()
-        # one batch to size the run
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        torch.cuda.synchronize()
-        e0.record()
-        for _ in range(S):
-            step()
-        e1.record()
-        torch.cuda.synchronize()
-        n_batches = int(max(1, min(5000, np.ceil(args.min_seconds * 1e3 / max(e0.elapsed_time(e1), 1e-3)))))
-        evs = [torch.cuda.Event(enable_timing=True) for _ in range(n_batches + 1)]
-        sampler = ClockSampler(self.local)
-        sampler.start()
-        time.sleep(0.12)                       # the sampler's first line
-        self.barrier()
-        t_wall0 = time.time()
-        evs[0].record()
-        for b in range(n_batches):
-            for _ in range(S):
-                step()
-            evs[b + 1].record()
-        self.barrier()
-        t_wall1 = time.time()
-        sampler.stop()
-        batch_ms = sorted(evs[b].elapsed_time(evs[b + 1]) for b in range(n_batches))
-        med = batch_ms[len(batch_ms) // 2]
-        clocks = sampler.summary(t_wall0, t_wall1)
-        value, sec_batch = replica_throughput(dist, dev, K * M * S, med * 1e-3)
-        ms_step = sec_batch * 1e3 / S
+        timed = self.time_step(step, K * M, launches)
+        S, n_batches = timed["steps_per_batch"], timed["batches"]
+        clocks, value, ms_step = timed["clocks"], timed["value"], timed["ms_per_step"]
 
         # per-phase kernel times (CUDA events on the launching stream inside mrp_draft)
         binding.mrp_profile_enable(ctx, True)
@@ -508,8 +529,8 @@ class Bench:
         binding.mrp_destroy(ctx)
         res = {
             "value": value, "unit": UNIT, "ms_per_step": ms_step,
-            "batches": n_batches, "batch_ms_median": med, "batch_ms_min": batch_ms[0], "batch_ms_max": batch_ms[-1],
-            "timed_gpu_seconds": sum(batch_ms) * 1e-3,
+            "batches": n_batches, "batch_ms_median": timed["batch_ms_median"], "batch_ms_min": timed["batch_ms_min"],
+            "batch_ms_max": timed["batch_ms_max"], "timed_gpu_seconds": timed["timed_gpu_seconds"],
             "dtype": "bf16" if cfg["dtype"] == "bf16" else "f32",
             "config": config_dict(cfg, M, ("mrp_draft_from_hidden" if args.from_hidden else "mrp_draft") +
                                   (" on the 8-bit LM head" if args.fp8_lm else "")),
@@ -597,6 +618,120 @@ class Bench:
                 "steps": n_e2e, "ms_per_step": dt / n_e2e * 1e3, "mode": e2e_mode}
 
 
+def run_module_workload(bench, cpu_budget_s):
+    """The token-conditioned module at the decode shape (configuration 1's d, V, block): a step is the K = 3
+    MRP steps that follow one backbone forward in direct decoding (Algorithm 2), each = mrp_module_step
+    (module forward + one LM-head pass) + mrp_reveal_remask + mrp_commit, the reveals of a step
+    conditioning the next.  Drafted tokens per step: K (one reveal per MRP step)."""
+    import numpy as np
+    import torch
+    import oracle
+    from paper_2605_18817_b200 import binding, harness, synth
+    args, dev, dist = bench.args, bench.dev, bench.dist
+    cfg = dict(synth.CONFIGS[1], name="module_decode_1p7b")
+    w, heads, w_lm = bench.weights_for(synth.CONFIGS[1], "1")
+    _, inp = synth.make_config(synth.CONFIGS[1], w)
+    K, B, L, d, V, F = cfg["K"], cfg["B"], cfg["L"], cfg["d"], cfg["V"], cfg["F"]
+    n = B * L
+    mw = synth.make_module_weights(d, F, V, MODULE_LAYERS, MODULE_ATTN_HEADS, "bf16", 11, std=0.02)
+    ctx = binding.mrp_create(d, F, V, heads[:1], w_lm, max_rows=n, max_seqs=B, block_len=L, flags=args.flags)
+    up = lambda a: harness.to_device(a, "bf16", dev)
+    binding.mrp_module_attach(ctx, up(mw.emb), up(mw.w_proj), [{k: up(v) for k, v in lay.items()} for lay in mw.layers],
+                              MODULE_ATTN_HEADS, mw.mask_token)
+    hid0 = harness.to_device(inp.hidden, "bf16", dev)
+    l0 = torch.from_numpy(inp.logits0).to(dev)
+    h_state = torch.empty((n, d), device=dev)
+    # block state after the backbone's own reveal of one token (position 0 here: any would do for timing)
+    tokens0 = np.full(n, -1, np.int32)
+    tokens0[0] = 17
+    state = harness.alloc_block_state(B, L, dev)
+    tok_init = torch.from_numpy(tokens0).to(dev)
+    out = harness.alloc_draft_out(n, 1, V, d, dev, margin=False)
+    sel = harness.alloc_select_out(B, L, 0, dev)
+    launches = [0]
+    conf_flat, token_flat = out.conf.view(-1), out.token.view(-1)
+
+    def step():
+        state.tokens.copy_(tok_init)
+        m = n - 1                                   # rows still masked: one fewer after every MRP step
+        ri = torch.arange(1, n, device=dev, dtype=torch.int32)
+        cnt = 1                                     # the tensor fill above
+        for k in range(K):
+            rows = ri[:m] if k == 0 else state.row_index[:m]
+            # a call with m rows writes [2, m] step-major into the front of the [2, n] buffers
+            binding.mrp_module_step(ctx, state.tokens, hid0, h_state, l0, rows, m, B, L, k == 0, out.conf, out.lse, out.token)
+            cnt += ctx.last_launch_count
+            harness.select(ctx, conf_flat[m:2 * m].view(1, m), token_flat[m:2 * m].view(1, m), rows, m, 0, B, L,
+                           binding.MRP_SELECT_STATIC, sel, r_reveal=1)
+            cnt += ctx.last_launch_count
+            harness.commit(ctx, sel, state, B, L, 0)
+            cnt += ctx.last_launch_count
+            m -= 1
+        launches[0] = cnt
+
+    step()
+    torch.cuda.synchronize()
+    res = bench.time_step(step, K, launches, ctx, cfg, n - 1)
+    res.pop("steps_per_batch")
+    # roofline of the dominant kernel: the LM-head kernel, launched once per MRP step (K weight streams)
+    binding.mrp_profile_enable(ctx, True)
+    for _ in range(50):
+        step()
+    torch.cuda.synchronize()
+    (ms_mod, ms_lm, ms_comb), n_calls = binding.mrp_profile_read(ctx)
+    binding.mrp_profile_enable(ctx, False)
+    one = dict(cfg, K=1)
+    roofline = lm_head_roofline(one, n - 2, ms_lm / max(n_calls, 1), bench.peaks, bench.peaks_kind)
+    roofline["kernel"] = "fused LM head, one launch per MRP step (K = %d weight streams per backbone forward)" % K
+    roofline["units_per_launch"] = 1
+    res["roofline"] = roofline
+    res["phases"] = {"module_ms_per_mrp_step": ms_mod / max(n_calls, 1), "lm_head_ms_per_mrp_step": ms_lm / max(n_calls, 1),
+                     "combine_ms_per_mrp_step": ms_comb / max(n_calls, 1), "family": ctx.family,
+                     "module": "D = %d layers, %d attention heads, CUDA-core kernels" % (MODULE_LAYERS, MODULE_ATTN_HEADS)}
+    # end to end with host buffers: hidden states, base logits and the block's tokens in, the block state out
+    e2e = None
+    if not args.no_e2e:
+        h_hid, h_l0, h_tok = hid0.cpu().pin_memory(), l0.cpu().pin_memory(), tok_init.cpu().pin_memory()
+        h_out = torch.empty_like(state.tokens, device="cpu").pin_memory()
+
+        def e2e_step():
+            hid0.copy_(h_hid, non_blocking=True)
+            l0.copy_(h_l0, non_blocking=True)
+            tok_init.copy_(h_tok, non_blocking=True)
+            step()
+            h_out.copy_(state.tokens, non_blocking=True)
+            torch.cuda.current_stream().synchronize()
+        for _ in range(3):
+            e2e_step()
+        n_e2e = 200 if args.min_seconds > 0 else 3
+        bench.barrier()
+        t0 = time.perf_counter()
+        for _ in range(n_e2e):
+            e2e_step()
+        bench.barrier()
+        dt = time.perf_counter() - t0
+        v, dt = replica_throughput(dist, dev, K * n_e2e, dt)
+        e2e = {"value": v, "unit": UNIT, "h2d_bytes_per_step": h_hid.numel() * 2 + h_l0.numel() * 4 + h_tok.numel() * 4,
+               "d2h_bytes_per_step": h_out.numel() * 4, "steps": n_e2e, "ms_per_step": dt / n_e2e * 1e3, "mode": "eager calls"}
+    res["e2e"] = e2e
+    cpu = None
+    if bench.rank == 0 and bench.world == 1 and not args.no_cpu_baseline:
+        ri = np.arange(1, n, dtype=np.int32)
+        t0 = time.perf_counter()
+        reps = 0
+        while time.perf_counter() - t0 < min(cpu_budget_s, 6.0) or reps == 0:
+            for k in range(K):
+                oracle.module(inp.hidden, tokens0, B, L, mw.emb, mw.w_proj, mw.layers, w.w_lm, MODULE_ATTN_HEADS,
+                              mw.mask_token, row_index=ri[:n - 1 - k])
+            reps += 1
+        cpu = {"value": K * reps / (time.perf_counter() - t0), "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+               "sample": "the module oracle, K = %d applications on the whole block, %d repetitions" % (K, reps)}
+    res["cpu_baseline"] = cpu
+    res["device_status_word"] = binding.mrp_fetch_status(ctx)
+    binding.mrp_destroy(ctx)
+    return res
+
+
 def run_sweep(args):
     """All 21 points of the roofline sweep (configuration 4), one JSON line per point."""
     bench = Bench(args)
@@ -631,7 +766,10 @@ def main():
     head_name = HEADLINE if args.config == "all" else args.config
     results = {}
     for name in names:
-        results[name] = bench.run_workload(name, 12.0 if name == head_name else 5.0)
+        if name == "module":
+            results[name] = run_module_workload(bench, 5.0)
+        else:
+            results[name] = bench.run_workload(name, 12.0 if name == head_name else 5.0)
     if bench.rank == 0:
         head = results[head_name]
         line = {

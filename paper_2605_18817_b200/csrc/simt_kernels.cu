@@ -10,6 +10,8 @@
 #include <limits.h>
 #include <string.h>
 
+#include <type_traits>
+
 #include "mrp_internal.cuh"
 
 namespace mrp {
@@ -22,6 +24,46 @@ __device__ __forceinline__ float warp_sum(float v)
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
     return v;
+}
+
+constexpr int kRC = 4;     // activation rows a warp handles per pass over a weight row
+
+// Lane-partial dot products of one weight row with up to kRC activation rows (x: fp32 [rows, n_in]); the
+// caller adds the lanes.  bf16 weight rows whose length is a multiple of 256 are read 16 bytes per lane.
+template <typename T>
+__device__ __forceinline__ void row_dots(const T *__restrict__ wr, const float *__restrict__ x, int rows, int n_in, int lane,
+                                         float *s)
+{
+#pragma unroll
+    for (int r = 0; r < kRC; ++r) s[r] = 0.f;
+    if (std::is_same<T, __nv_bfloat16>::value && (n_in & 255) == 0) {
+#pragma unroll 4
+        for (int c = lane * 8; c < n_in; c += 256) {
+            const uint4 q = __ldg(reinterpret_cast<const uint4 *>(reinterpret_cast<const __nv_bfloat16 *>(wr) + c));
+            const float wv[8] = {__uint_as_float(q.x << 16), __uint_as_float(q.x & 0xFFFF0000u),
+                                 __uint_as_float(q.y << 16), __uint_as_float(q.y & 0xFFFF0000u),
+                                 __uint_as_float(q.z << 16), __uint_as_float(q.z & 0xFFFF0000u),
+                                 __uint_as_float(q.w << 16), __uint_as_float(q.w & 0xFFFF0000u)};
+#pragma unroll
+            for (int r = 0; r < kRC; ++r) {
+                if (r < rows) {
+                    const float4 a = *reinterpret_cast<const float4 *>(x + (size_t)r * n_in + c);
+                    const float4 b = *reinterpret_cast<const float4 *>(x + (size_t)r * n_in + c + 4);
+                    float t = s[r];
+                    t = fmaf(wv[0], a.x, t); t = fmaf(wv[1], a.y, t); t = fmaf(wv[2], a.z, t); t = fmaf(wv[3], a.w, t);
+                    t = fmaf(wv[4], b.x, t); t = fmaf(wv[5], b.y, t); t = fmaf(wv[6], b.z, t); t = fmaf(wv[7], b.w, t);
+                    s[r] = t;
+                }
+            }
+        }
+    } else {
+        for (int c = lane; c < n_in; c += 32) {
+            const float a = ld_f(wr, c);
+#pragma unroll
+            for (int r = 0; r < kRC; ++r)
+                if (r < rows) s[r] = fmaf(a, x[(size_t)r * n_in + c], s[r]);
+        }
+    }
 }
 
 // ---- a0: gather masked rows into the fp32 residual stream --------------------------------
@@ -112,8 +154,7 @@ __global__ void rmsnorm_kernel(const float *__restrict__ hcur, const T *__restri
         xg[(size_t)m * d + j] = h[j] * rstd * ld_f(gamma, j);
 }
 
-// ---- a1: gate/up projections + SwiGLU; one warp per inner feature, 4 rows at a time -------
-constexpr int kRC = 4;
+// ---- a1: gate/up projections + SwiGLU; one warp per inner feature, kRC rows at a time -------
 
 template <typename T>
 __global__ void gateup_kernel(const T *__restrict__ w_gate, const T *__restrict__ w_up,
@@ -128,19 +169,8 @@ __global__ void gateup_kernel(const T *__restrict__ w_gate, const T *__restrict_
     const T *wg = w_gate + (size_t)f * d, *wu = w_up + (size_t)f * d;
     for (int m0 = 0; m0 < M; m0 += kRC) {
         float g[kRC], u[kRC];
-#pragma unroll
-        for (int r = 0; r < kRC; ++r) g[r] = u[r] = 0.f;
-        for (int j = lane; j < d; j += 32) {
-            const float a = ld_f(wg, j), b = ld_f(wu, j);
-#pragma unroll
-            for (int r = 0; r < kRC; ++r) {
-                if (m0 + r < M) {
-                    const float x = xg[(size_t)(m0 + r) * d + j];
-                    g[r] = fmaf(a, x, g[r]);
-                    u[r] = fmaf(b, x, u[r]);
-                }
-            }
-        }
+        row_dots<T>(wg, xg + (size_t)m0 * d, M - m0, d, lane, g);
+        row_dots<T>(wu, xg + (size_t)m0 * d, M - m0, d, lane, u);
 #pragma unroll
         for (int r = 0; r < kRC; ++r) {
             const float gs = warp_sum(g[r]), us = warp_sum(u[r]);
@@ -164,14 +194,7 @@ __global__ void down_kernel(const T *__restrict__ w_down, const float *__restric
     const T *wd = w_down + (size_t)j * F;
     for (int m0 = 0; m0 < M; m0 += kRC) {
         float s[kRC];
-#pragma unroll
-        for (int r = 0; r < kRC; ++r) s[r] = 0.f;
-        for (int f = lane; f < F; f += 32) {
-            const float a = ld_f(wd, f);
-#pragma unroll
-            for (int r = 0; r < kRC; ++r)
-                if (m0 + r < M) s[r] = fmaf(a, act[(size_t)(m0 + r) * F + f], s[r]);
-        }
+        row_dots<T>(wd, act + (size_t)m0 * F, M - m0, F, lane, s);
 #pragma unroll
         for (int r = 0; r < kRC; ++r) {
             const float v = warp_sum(s[r]);
@@ -644,7 +667,8 @@ __global__ void mod_concat_kernel(const float *h_state, const T *__restrict__ hi
     }
 }
 
-// y[r, j] (+)= sum_c W[j, c] x[r, c]: one warp per output feature, kRC rows at a time.
+// y[r, j] (+)= sum_c W[j, c] x[r, c]: one warp per output feature, kRC rows at a time; bf16 weights
+// with n_in a multiple of 256 are read 16 bytes per lane.
 template <typename T>
 __global__ void linear_kernel(const T *__restrict__ w, const float *__restrict__ x, int rows, int n_in, int n_out,
                               float *__restrict__ y, int accumulate)
@@ -657,14 +681,7 @@ __global__ void linear_kernel(const T *__restrict__ w, const float *__restrict__
     const T *wr = w + (size_t)j * n_in;
     for (int r0 = 0; r0 < rows; r0 += kRC) {
         float s[kRC];
-#pragma unroll
-        for (int r = 0; r < kRC; ++r) s[r] = 0.f;
-        for (int c = lane; c < n_in; c += 32) {
-            const float a = ld_f(wr, c);
-#pragma unroll
-            for (int r = 0; r < kRC; ++r)
-                if (r0 + r < rows) s[r] = fmaf(a, x[(size_t)(r0 + r) * n_in + c], s[r]);
-        }
+        row_dots<T>(wr, x + (size_t)r0 * n_in, rows - r0, n_in, lane, s);
 #pragma unroll
         for (int r = 0; r < kRC; ++r) {
             const float v = warp_sum(s[r]);
