@@ -45,8 +45,12 @@ MODULE_LAYERS, MODULE_ATTN_HEADS = 3, 16      # the paper's depth D = 3 (Sec. 4.
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the fused LM-head kernel, from
 # the ncu captures summarised under profiles/ (bytes per launch, and the summary they come from).
 NCU_TRAFFIC = {
-    "decode_1p7b": (628542208, "profiles/sk_gemm_kernel_decode_1p7b.md"),
-    "sweep_M256_K4": (1447000000, "profiles/tc_gemm_kernel_lm_sweep_M256_K4.md"),
+    "decode_1p7b": (627908096, "profiles/lm_head_dram_traffic.md"),
+    "spec_8b": (1362025984, "profiles/lm_head_dram_traffic.md"),
+    "remask_8b": (1899798528, "profiles/lm_head_dram_traffic.md"),
+    "sweep_M64_K4": (1369512704, "profiles/lm_head_dram_traffic.md"),
+    "sweep_M256_K1": (1487823104, "profiles/lm_head_dram_traffic.md"),
+    "sweep_M4096_K4": (20161282048, "profiles/lm_head_dram_traffic.md"),
 }
 
 
