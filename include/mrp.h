@@ -90,6 +90,8 @@ typedef enum { MRP_F32 = 0, MRP_BF16 = 1 } mrp_dtype;
                                        those of mrp_draft on W8, to the usual tolerances; the difference
                                        to W_lm itself is the quantisation (relative 2^-4 per weight).
                                        Other shapes: MRP_ERR_UNSUPPORTED.  Workspace: + vocab * d bytes  */
+#define MRP_FLAG_NO_CTA_PAIRS 256   /* tensor-core family: run the row-major kernels one CTA per tile instead
+                                     * of two-CTA clusters that share each MMA (for comparison)             */
 #define MRP_FLAG_EXACT_OPERANDS 8   /* tensor-core family: always carry the LM-head activation
                                        operand as a bf16 hi + lo pair (products exact to 2^-17),
                                        also where that doubles the tensor work for nothing.  Without

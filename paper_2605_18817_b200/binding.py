@@ -27,6 +27,7 @@ MRP_FLAG_NO_CHAIN = 16
 MRP_FLAG_REQUIRE_TENSOR_CORES = 32
 MRP_FLAG_TRAINING_KL = 64
 MRP_FLAG_FP8_LM = 128
+MRP_FLAG_NO_CTA_PAIRS = 256
 MRP_SELECT_STATIC, MRP_SELECT_DYNAMIC_REMASK = 0, 1
 MRP_DEV_NONFINITE, MRP_DEV_TIMEOUT, MRP_DEV_BAD_INDEX, MRP_DEV_RANGE = 1, 2, 4, 8
 MRP_RANGE_LIMIT = 32768.0

@@ -112,6 +112,56 @@ __device__ __forceinline__ void umma_f8(uint32_t d_tmem, uint64_t da, uint64_t d
         "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(d_tmem), "l"(da), "l"(db), "r"(idesc), "r"(acc) : "memory");
 }
+// ---- CTA pairs (a cluster of two CTAs working on one 256-row MMA tile, cta_group::2) ----------------
+// Shared-memory addresses carry the CTA's rank within the cluster in bit 24; clearing it names the same
+// offset in the pair's leader (rank 0).
+constexpr uint32_t kLeaderMask = 0xFEFFFFFFu;
+__device__ __forceinline__ uint32_t cluster_ctarank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// All threads of both CTAs meet (release / acquire at cluster scope).
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// TMA load into this CTA's shared memory whose completion is counted by the LEADER's barrier at `bar`'s offset
+// (no multicast: every CTA fetches its own tiles).
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap *map, int c0, int c1, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar & kLeaderMask), "r"(c0), "r"(c1) : "memory");
+}
+// 256 x N x 16 MMA over the pair: rows 0-127 of A from the leader's shared memory, 128-255 from the peer's;
+// each CTA holds N / 2 rows of B; each CTA's tensor memory receives its 128 rows of D.  Issued by the leader.
+__device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t da, uint64_t db, uint32_t idesc, uint32_t acc)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(da), "l"(db), "r"(idesc), "r"(acc) : "memory");
+}
+// Arrival on the barrier at `bar`'s offset in BOTH CTAs once the pair's MMAs issued so far have completed.
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"((unsigned short)3) : "memory");
+}
+// Arrival on the leader's barrier from either CTA of the pair.
+__device__ __forceinline__ void mbar_arrive_leader(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(bar & kLeaderMask) : "memory");
+}
+// Instruction descriptor of the pair's MMA: M = 256, N = bn, fp32 accumulation; bf16 (1) or fp16 (0) operands.
+__device__ __forceinline__ uint32_t make_idesc_pair(int bn, bool f16)
+{
+    return (1u << 4) | (f16 ? 0u : ((1u << 7) | (1u << 10))) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+}
+
 // True in exactly one lane of a converged warp, the same lane every time.  The MMA issuer runs
 // its loop with the whole warp and only issues from the elected lane: the loop's barrier waits,
 // fences and commits cost about half as many cycles that way as in a one-lane branch

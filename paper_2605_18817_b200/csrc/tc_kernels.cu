@@ -87,16 +87,23 @@ struct TcParams {
 // ---------------------------------------------------------------------------------------
 // F16: one fp16 A tile per stage against fp16 weights (LM head only); otherwise the bf16 hi and lo
 // A tiles of a k-chunk against bf16 weights.
-template <int KIND, bool MARGIN, bool F16, bool KL>
+// PAIR: the grid is launched in clusters of two CTAs that share every MMA (cta_group::2, M = 256): CTA r of
+// a pair owns row block 2 pb + r and loads its own A tiles plus HALF of the B tile (rows r * bn / 2 ...),
+// which halves the weight bytes a CTA pulls from L2 per MMA cycle and so deepens the ring.  The leader
+// (rank 0) issues the MMAs; both CTAs' loads complete on the leader's full barrier; the MMA commits
+// arrive on both CTAs' empty / accumulator-full barriers; both CTAs' epilogue warps arrive on the
+// leader's accumulator-empty barrier.  No load is multicast: each CTA fetches its own tiles.
+template <int KIND, bool MARGIN, bool F16, bool KL, bool PAIR = false>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
                const __grid_constant__ CUtensorMap tmB1, const TcParams p)
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    // a stage holds the A tile(s) of a k-chunk and one B tile
+    // a stage holds the A tile(s) of a k-chunk and one B tile (PAIR: this CTA's half of it)
     constexpr int PARTS = F16 ? 1 : 2;
-    const int b_bytes = (p.bn * 128 + 1023) & ~1023;
+    const int bn_own = PAIR ? p.bn / 2 : p.bn;           // B rows in this CTA's shared memory
+    const int b_bytes = (bn_own * 128 + 1023) & ~1023;
     const int stage_bytes = PARTS * kATile + b_bytes;
     const uint32_t bars = base + (uint32_t)p.n_stages * stage_bytes;   // 8-byte aligned
     // barrier slots: full[s], empty[s], tmem_full[2], tmem_empty[2]
@@ -109,7 +116,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_holder + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int cta = blockIdx.x;
+    // PAIR: `cta` numbers the pair, `rank` the CTA in it; a pair walks PAIRS of row blocks (p.n_rb counts pairs,
+    // row block of this CTA = 2 * pair-block + rank)
+    const int rank = PAIR ? (int)cluster_ctarank() : 0;
+    const int cta = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
     const int vr = cta % p.n_vr, grp = cta / p.n_vr;
     const int u0 = (int)((long long)vr * p.units_total / p.n_vr);
     const int u1 = (int)((long long)(vr + 1) * p.units_total / p.n_vr);
@@ -117,7 +127,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.n_stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-        for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
+        for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), PAIR ? 8 : 4); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         prefetch_tmap(&tmA);
@@ -125,12 +135,19 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (KIND == KIND_GU) prefetch_tmap(&tmB1);
     }
     if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                     ::"r"(smem_u32(tmem_holder)), "r"(2u * kAccCols) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        if (PAIR) {
+            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                         ::"r"(smem_u32(tmem_holder)), "r"(2u * kAccCols) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+        } else {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                         ::"r"(smem_u32(tmem_holder)), "r"(2u * kAccCols) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        }
     }
     tc_fence_before();
     __syncthreads();
+    if (PAIR) cluster_sync_all();       // both CTAs' barriers exist before either signals the other's
     tc_fence_after();
     const uint32_t tmem_base = *tmem_holder;
     // launched behind its predecessor with programmatic dependent launch: everything above overlaps
@@ -140,7 +157,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     if (warp == 0) {
         // ---------------- TMA producer ----------------
         if (lane == 0) {
-            const uint32_t tx = (uint32_t)(PARTS * kATile + p.bn * 128);
+            // PAIR: both CTAs' loads are counted by the leader's barrier, which its producer arms for both
+            const uint32_t tx = (uint32_t)(PARTS * kATile + bn_own * 128) * (PAIR ? 2u : 1u);
             const int box_rows = p.bn / p.n_boxes;
             // the CTA's work as one sequence of ring steps: row blocks mb = grp, grp + n_groups, ...,
             // for each its n_t weight tiles, for each tile the k-chunks
@@ -150,14 +168,28 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             auto load_b = [&](int t_, int kk_, int s_) {
                 const int n0 = (u0 + t_ * p.w_units) * p.unit_rows;
                 const uint32_t sb = base + (uint32_t)s_ * stage_bytes + PARTS * kATile;
-                tma_load_2d(sb, &tmB0, kk_ * kBK, n0, full_bar(s_));
-                if (KIND == KIND_GU) tma_load_2d(sb + box_rows * 128, &tmB1, kk_ * kBK, n0, full_bar(s_));
+                if (PAIR) {
+                    // this CTA's half of the B tile: rows [rank * bn / 2, ...) of a one-box tile; of a gate/up tile
+                    // the gate rows (leader) or the up rows (peer), so that the columns stay [gate | up]
+                    if (KIND == KIND_GU) tma_load_2d_pair(sb, rank ? &tmB1 : &tmB0, kk_ * kBK, n0, full_bar(s_));
+                    else tma_load_2d_pair(sb, &tmB0, kk_ * kBK, n0 + rank * bn_own, full_bar(s_));
+                } else {
+                    tma_load_2d(sb, &tmB0, kk_ * kBK, n0, full_bar(s_));
+                    if (KIND == KIND_GU) tma_load_2d(sb + box_rows * 128, &tmB1, kk_ * kBK, n0, full_bar(s_));
+                }
             };
             auto load_a = [&](int mb_, int kk_, int s_) {
                 const uint32_t sa = base + (uint32_t)s_ * stage_bytes;
-                tma_load_2d(sa, &tmA, kk_ * kBK, p.a_row_base + mb_ * 128, full_bar(s_));
-                if (!F16) tma_load_2d(sa + kATile, &tmA, kk_ * kBK, p.a_part_rows + p.a_row_base + mb_ * 128, full_bar(s_));
+                const int row0 = p.a_row_base + (PAIR ? 2 * mb_ + rank : mb_) * 128;
+                if (PAIR) {
+                    tma_load_2d_pair(sa, &tmA, kk_ * kBK, row0, full_bar(s_));
+                    if (!F16) tma_load_2d_pair(sa + kATile, &tmA, kk_ * kBK, p.a_part_rows + row0, full_bar(s_));
+                } else {
+                    tma_load_2d(sa, &tmA, kk_ * kBK, row0, full_bar(s_));
+                    if (!F16) tma_load_2d(sa + kATile, &tmA, kk_ * kBK, p.a_part_rows + row0, full_bar(s_));
+                }
             };
+            auto arm = [&](int s_) { if (!PAIR || rank == 0) mbar_expect_tx(full_bar(s_), tx); };
             const int my_blocks = grp < p.n_rb ? (p.n_rb - 1 - grp) / p.n_groups + 1 : 0;
             const long long total_it = (long long)my_blocks * n_t * p.k_chunks;
             const int pre = (int)(total_it < p.n_stages ? total_it : p.n_stages);
@@ -165,7 +197,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             // kernel of the stream drains; only the activation tiles wait for it
             int mb = grp, t = 0, kk = 0;
             for (int it = 0; it < pre; ++it) {
-                mbar_expect_tx(full_bar(it), tx);
+                arm(it);
                 load_b(t, kk, it);
                 advance(mb, t, kk);
             }
@@ -178,22 +210,30 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             uint32_t ph = 1;              // the ring has been filled once
             for (long long it = pre; it < total_it; ++it) {
                 if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p)) break;
-                mbar_expect_tx(full_bar(s), tx);
+                arm(s);
                 load_a(mb, kk, s);
                 load_b(t, kk, s);
                 advance(mb, t, kk);
                 if (++s == p.n_stages) { s = 0; ph ^= 1u; }
             }
+            if (PAIR) {
+                // the leader's last commits also arrive here: let them land before this CTA may leave
+                for (int i = 0; i < pre && !*abort_flag; ++i) {
+                    if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p)) break;
+                    if (++s == p.n_stages) { s = 0; ph ^= 1u; }
+                }
+            }
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
         // The whole warp walks the loop (all values are warp-uniform); the elected lane issues.
-        const uint32_t idesc = F16 ? make_idesc_f16(p.bn) : make_idesc(p.bn);
+        const uint32_t idesc = PAIR ? make_idesc_pair(p.bn, F16) : F16 ? make_idesc_f16(p.bn) : make_idesc(p.bn);
         const uint32_t tm = __shfl_sync(0xffffffffu, tmem_base, 0);
         int s = 0, acc = 0;
         uint32_t ph = 0, acc_ph = 0;
         bool ok = true;
-        for (int mb = grp; mb < p.n_rb && ok; mb += p.n_groups) {
+        // PAIR: the leader's warp issues for both CTAs; the peer's warp only holds the TMEM allocation
+        for (int mb = grp; mb < p.n_rb && ok && rank == 0; mb += p.n_groups) {
             for (int t = 0; t < n_t && ok; ++t) {
                 ok = __all_sync(0xffffffffu, mbar_wait(tempty_bar(acc), acc_ph ^ 1u, abort_flag, p));
                 if (!ok) break;
@@ -211,16 +251,22 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         for (int a = 0; a < PARTS; ++a) {
                             const uint64_t da = make_smem_desc(sa + a * kATile);
 #pragma unroll
-                            for (int k4 = 0; k4 < kBK / 16; ++k4)
-                                umma_bf16(dt, da + 2u * k4, db + 2u * k4, idesc, (k4 > 0 || a > 0) ? 1u : later);
+                            for (int k4 = 0; k4 < kBK / 16; ++k4) {
+                                if (PAIR) umma_bf16_pair(dt, da + 2u * k4, db + 2u * k4, idesc, (k4 > 0 || a > 0) ? 1u : later);
+                                else umma_bf16(dt, da + 2u * k4, db + 2u * k4, idesc, (k4 > 0 || a > 0) ? 1u : later);
+                            }
                         }
-                        umma_commit(empty_bar(s));
+                        if (PAIR) umma_commit_pair(empty_bar(s));
+                        else umma_commit(empty_bar(s));
                     }
                     __syncwarp();
                     if (++s == p.n_stages) { s = 0; ph ^= 1u; }
                 }
                 if (!ok) break;
-                if (elect_one()) umma_commit(tfull_bar(acc));
+                if (elect_one()) {
+                    if (PAIR) umma_commit_pair(tfull_bar(acc));
+                    else umma_commit(tfull_bar(acc));
+                }
                 __syncwarp();
                 acc ^= 1;
                 if (acc == 0) acc_ph ^= 1u;
@@ -237,7 +283,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         bool ok = true;
         for (int mb = grp; mb < p.n_rb && ok; mb += p.n_groups) {
             // ---- per-block state: this thread's activation row ----
-            const int r = mb * 128 + rl;
+            const int r = (PAIR ? 2 * mb + rank : mb) * 128 + rl;
             const bool valid = r < p.rows;
             RowStat st, st0;       // LM: statistics of the row's own step, and of step 0 (rows of step 1 only)
             KlStat kst;            // LM, KL variant: the row-step's share of the training objective
@@ -358,7 +404,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 }
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(tempty_bar(acc));
+                if (lane == 0) {
+                    if (PAIR) mbar_arrive_leader(tempty_bar(acc));
+                    else mbar_arrive(tempty_bar(acc));
+                }
                 acc ^= 1;
                 if (acc == 0) acc_ph ^= 1u;
             }
@@ -385,9 +434,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         while (clock64() - t0 < 200000) __nanosleep(1000);
         __syncthreads();
     }
+    // PAIR: neither CTA leaves, nor frees the shared allocation, while the other may still signal its barriers
+    if (PAIR) cluster_sync_all();
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(2u * kAccCols) : "memory");
+        if (PAIR)
+            asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(2u * kAccCols) : "memory");
+        else
+            asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(2u * kAccCols) : "memory");
     }
 }
 
@@ -529,7 +583,14 @@ int choose_groups(int n_rb, int units_total, int G)
     return best_g;
 }
 
-void finish_shape(TcParams &p, int n_vr, int parts = 2)
+// CTA pairs need an even number of SMs, all of which clusters of two can occupy at once (otherwise the
+// grid would run in waves), and can be switched off per context.
+bool pair_ok(const Ctx *c)
+{
+    return !(c->cfg.flags & MRP_FLAG_NO_CTA_PAIRS) && (c->sm_count % 2 == 0);
+}
+
+void finish_shape(TcParams &p, int n_vr, int parts = 2, bool pair = false)
 {
     p.n_vr = n_vr;
     const int maxunits = (p.units_total + n_vr - 1) / n_vr;
@@ -540,25 +601,26 @@ void finish_shape(TcParams &p, int n_vr, int parts = 2)
     if (w_max < 1) w_max = 1;
     p.w_units = choose_tile_units(maxunits < 1 ? 1 : maxunits, w_max);
     p.bn = p.w_units * rows_per_unit;
-    const int b_bytes = (p.bn * 128 + 1023) & ~1023;
+    const int b_bytes = ((pair ? p.bn / 2 : p.bn) * 128 + 1023) & ~1023;
     const int stage = parts * kATile + b_bytes;
     int ns = (kSmemBudget - 1024 - 512) / stage;
     if (ns > 12) ns = 12;
     p.n_stages = ns;
 }
 
-size_t smem_bytes(const TcParams &p, int parts)
+size_t smem_bytes(const TcParams &p, int parts, bool pair)
 {
-    const int b_bytes = (p.bn * 128 + 1023) & ~1023;
+    const int b_bytes = ((pair ? p.bn / 2 : p.bn) * 128 + 1023) & ~1023;
     return (size_t)p.n_stages * (parts * kATile + b_bytes) + 1024 + 8 * (2 * p.n_stages + 4) + 16;
 }
 
-template <int KIND, bool MARGIN, bool F16 = false, bool KL = false>
+// PAIR: `grid` counts CTAs (two per pair); the launch carries the cluster shape (2, 1, 1).
+template <int KIND, bool MARGIN, bool F16 = false, bool KL = false, bool PAIR = false>
 cudaError_t launch_tc(const CUtensorMap &a, const CUtensorMap &b0, const CUtensorMap &b1, const TcParams &p,
                       int grid, cudaStream_t st, bool pdl)
 {
-    auto kern = tc_gemm_kernel<KIND, MARGIN, F16, KL>;
-    const size_t smem = smem_bytes(p, F16 ? 1 : 2);
+    auto kern = tc_gemm_kernel<KIND, MARGIN, F16, KL, PAIR>;
+    const size_t smem = smem_bytes(p, F16 ? 1 : 2, PAIR);
     // the shared-memory limit of a kernel is set once per device (the attribute is per device)
     static std::atomic<unsigned long long> attr_devices{0};
     int dev = 0;
@@ -569,6 +631,21 @@ cudaError_t launch_tc(const CUtensorMap &a, const CUtensorMap &b0, const CUtenso
         ea = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
         if (ea != cudaSuccess) return ea;
         attr_devices.fetch_or(bit);
+    }
+    if (PAIR) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(grid);
+        cfg.blockDim = dim3(kThreads);
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = st;
+        cudaLaunchAttribute at[2];
+        at[0].id = cudaLaunchAttributeClusterDimension;
+        at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+        at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        at[1].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = at;
+        cfg.numAttrs = pdl ? 2 : 1;
+        return cudaLaunchKernelEx(&cfg, kern, a, b0, b1, p);
     }
     return launch_k(kern, dim3(grid), dim3(kThreads), smem, st, pdl, a, b0, b1, p);
 }
@@ -679,10 +756,14 @@ cudaError_t tc_lm_tail(Ctx *c, const TcPlan &pl, const float *logits0, const int
         // (with the base logits computed in the pass, step 0 has rows of its own)
         const int step_base = c->from_hidden ? 0 : 1;
         const int rows = (K + 1 - step_base) * M, n_rb = (rows + 127) / 128, U = V / 16;
-        const int best_g = choose_groups(n_rb, U, G);
+        // Two row blocks or more: CTA pairs, each MMA covering two row blocks (the kernel then counts pairs of
+        // row blocks and pairs of CTAs); needs an even SM count the device can fill with clusters of two.
+        const bool pair = pair_ok(c) && n_rb >= 2 && n_rb % 2 == 0 && !with_kl;
+        const int n_cta = pair ? G / 2 : G, n_blk = pair ? (n_rb + 1) / 2 : n_rb;
+        const int best_g = choose_groups(n_blk, U, n_cta);
         p.n_groups = best_g;
-        n_slices = G / best_g;
-        p.n_rb = n_rb; p.rows = rows;
+        n_slices = n_cta / best_g;
+        p.n_rb = n_blk; p.rows = rows;
         p.units_total = U; p.unit_rows = 16; p.n_boxes = 1; p.k_chunks = d / kBK;
         p.a_row_base = step_base * M; p.a_part_rows = n_rs; p.step_base = step_base;
         p.M = M; p.K = K; p.V = V; p.d = d; p.F = F; p.n_rs = n_rs;
@@ -690,21 +771,31 @@ cudaError_t tc_lm_tail(Ctx *c, const TcPlan &pl, const float *logits0, const int
         p.n_rows_in = c->input_rows; p.l0_bf16 = c->l0_bf16 ? 1 : 0;
         p.teacher = c->teacher; p.kl_partials = (KlPartial *)(c->ws + c->lay.kl_partials);
         p.status = status; p.user_status = out.status;
-        finish_shape(p, n_slices, f16_lm ? 1 : 2);
-        const int grid = p.n_groups * p.n_vr;
+        finish_shape(p, n_slices, f16_lm ? 1 : 2, pair);
+        const int grid = p.n_groups * p.n_vr * (pair ? 2 : 1);
+        const int b_box = pair ? p.bn / 2 : p.bn;
         if (f16_lm) {
             // 16-bit elements either way: the bf16 tensor-map type only moves the bytes
             p.a_row_base = 0;
             if (!make_map(s, &mA, c->ws + c->lay.xt16, d, (uint64_t)rows, 128) ||
-                !make_map(s, &mB, c->ws + c->lay.w16, d, V, p.bn))
+                !make_map(s, &mB, c->ws + c->lay.w16, d, V, b_box))
                 return note_err(c, cudaErrorInvalidValue, "tensor map (LM head, fp16)");
-            e = note_err(c, out.margin ? launch_tc<KIND_LM, true, true>(mA, mB, mB, p, grid, st, pdl)
-                                       : launch_tc<KIND_LM, false, true>(mA, mB, mB, p, grid, st, pdl),
-                         "LM-head kernel (fp16 operands)");
+            if (pair)
+                e = note_err(c, out.margin ? launch_tc<KIND_LM, true, true, false, true>(mA, mB, mB, p, grid, st, pdl)
+                                           : launch_tc<KIND_LM, false, true, false, true>(mA, mB, mB, p, grid, st, pdl),
+                             "LM-head kernel (fp16 operands, CTA pairs)");
+            else
+                e = note_err(c, out.margin ? launch_tc<KIND_LM, true, true>(mA, mB, mB, p, grid, st, pdl)
+                                           : launch_tc<KIND_LM, false, true>(mA, mB, mB, p, grid, st, pdl),
+                             "LM-head kernel (fp16 operands)");
         } else {
-            if (!make_map(s, &mA, xt, d, 2 * (uint64_t)n_rs, 128) || !make_map(s, &mB, c->w_lm, d, V, p.bn))
+            if (!make_map(s, &mA, xt, d, 2 * (uint64_t)n_rs, 128) || !make_map(s, &mB, c->w_lm, d, V, b_box))
                 return note_err(c, cudaErrorInvalidValue, "tensor map (LM head)");
-            if (with_kl)
+            if (pair)
+                e = note_err(c, out.margin ? launch_tc<KIND_LM, true, false, false, true>(mA, mB, mB, p, grid, st, pdl)
+                                           : launch_tc<KIND_LM, false, false, false, true>(mA, mB, mB, p, grid, st, pdl),
+                             "LM-head kernel (CTA pairs)");
+            else if (with_kl)
                 e = note_err(c, out.margin ? launch_tc<KIND_LM, true, false, true>(mA, mB, mB, p, grid, st, pdl)
                                            : launch_tc<KIND_LM, false, false, true>(mA, mB, mB, p, grid, st, pdl),
                              "LM-head kernel (KL objective)");
@@ -751,6 +842,10 @@ cudaError_t tc_draft(Ctx *c, const void *hidden, const float *logits0, const int
     if (G > kSumsqSlices || G > c->lay.n_slices_max)
         return note_err(c, cudaErrorInvalidValue, "workspace slices");
     const int n_mb = (M + 127) / 128;
+    // The head GEMMs can run on CTA pairs like the LM head (see tc_lm_tail), but gain nothing from it: with
+    // two MMA passes per loaded tile (bf16 hi + lo) they are bound by the tensor pipe, not by the tile feed.
+    const bool pair = false;
+    const int n_cta = pair ? G / 2 : G, n_blk = pair ? (n_mb + 1) / 2 : n_mb;
 
     const TcPlan pl = tc_plan(c, M, K, out, st, true);
     const int n_rs = pl.n_rs;
@@ -790,21 +885,22 @@ cudaError_t tc_draft(Ctx *c, const void *hidden, const float *logits0, const int
         TcParams p;
         memset(&p, 0, sizeof(p));
         p.units_total = F / 8; p.unit_rows = 8; p.n_boxes = 2; p.k_chunks = d / kBK;
-        p.n_groups = choose_groups(n_mb, p.units_total, G); p.n_rb = n_mb; p.rows = M; p.a_row_base = 0; p.a_part_rows = M;
+        p.n_groups = choose_groups(n_blk, p.units_total, n_cta); p.n_rb = n_blk; p.rows = M; p.a_row_base = 0; p.a_part_rows = M;
         p.M = M; p.K = K; p.V = V; p.d = d; p.F = F; p.n_rs = n_rs;
         p.sumsq = sumsq; p.n_ss = n_ss; p.eps = c->cfg.rms_eps; p.act = act;
         p.status = status; p.user_status = out.status;
-        finish_shape(p, G / p.n_groups);
+        finish_shape(p, n_cta / p.n_groups, 2, pair);
         if (!make_map(s, &mA, xg, d, 2 * (uint64_t)M, 128) || !make_map(s, &mB0, hw.w_gate, d, F, p.bn / 2) ||
             !make_map(s, &mB1, hw.w_up, d, F, p.bn / 2))
             return note_err(c, cudaErrorInvalidValue, "tensor map (gate/up)");
-        e = note_err(c, launch_tc<KIND_GU, false>(mA, mB0, mB1, p, p.n_groups * p.n_vr, st, pdl), "gate/up kernel");
+        e = note_err(c, pair ? launch_tc<KIND_GU, false, false, false, true>(mA, mB0, mB1, p, 2 * p.n_groups * p.n_vr, st, pdl)
+                             : launch_tc<KIND_GU, false>(mA, mB0, mB1, p, p.n_groups * p.n_vr, st, pdl), "gate/up kernel");
         c->launches++;
         if (e != cudaSuccess) return e;
         // down projection, residual add, next operands
         memset(&p, 0, sizeof(p));
         p.units_total = d / 16; p.unit_rows = 16; p.n_boxes = 1; p.k_chunks = F / kBK;
-        p.n_groups = choose_groups(n_mb, p.units_total, G); p.n_rb = n_mb; p.rows = M;
+        p.n_groups = choose_groups(n_blk, p.units_total, n_cta); p.n_rb = n_blk; p.rows = M;
         p.M = M; p.K = K; p.V = V; p.d = d; p.F = F; p.n_rs = n_rs; p.a_part_rows = M;
         p.hcur = hcur; p.h0f = h0f;
         p.gamma_next = (k < K) ? (const __nv_bfloat16 *)c->heads[k].rms_gamma : nullptr;
@@ -814,10 +910,11 @@ cudaError_t tc_draft(Ctx *c, const void *hidden, const float *logits0, const int
         p.sumsq_out = sumsq;
         p.hidden_out = (k == K) ? out.hidden_out : nullptr;
         p.status = status; p.user_status = out.status;
-        finish_shape(p, G / p.n_groups);
-        if (!make_map(s, &mA, act, F, 2 * (uint64_t)M, 128) || !make_map(s, &mB0, hw.w_down, F, d, p.bn))
+        finish_shape(p, n_cta / p.n_groups, 2, pair);
+        if (!make_map(s, &mA, act, F, 2 * (uint64_t)M, 128) || !make_map(s, &mB0, hw.w_down, F, d, pair ? p.bn / 2 : p.bn))
             return note_err(c, cudaErrorInvalidValue, "tensor map (down)");
-        e = note_err(c, launch_tc<KIND_DN, false>(mA, mB0, mB0, p, p.n_groups * p.n_vr, st, pdl), "down kernel");
+        e = note_err(c, pair ? launch_tc<KIND_DN, false, false, false, true>(mA, mB0, mB0, p, 2 * p.n_groups * p.n_vr, st, pdl)
+                             : launch_tc<KIND_DN, false>(mA, mB0, mB0, p, p.n_groups * p.n_vr, st, pdl), "down kernel");
         c->launches++;
         if (e != cudaSuccess) return e;
         n_ss = p.n_vr;

@@ -277,6 +277,8 @@ def test_config0_static_selection_end_to_end():
     (128, 192, 2048, 90, 1, 2),     # the same with an odd number of gate/up weight tiles
     (64, 6144, 1024, 100, 1, 1),    # head chain, gate/up tiles not split: outputs finished straight from TMEM
     (64, 6144, 1024, 5, 1, 2),      # the same with few rows
+    (64, 128, 160, 257, 1, 1),      # CTA pairs: three row blocks (the second pair half empty), fewer units than pairs
+    (128, 256, 2064, 129, 1, 3),    # CTA pairs: one row past a block in the heads, four row blocks in the LM head
 ])
 def test_tensor_core_family_small_shapes(d, F, V, B, L, K):
     # residuals inside the accuracy range the header states for the tensor-core kernels
@@ -308,6 +310,10 @@ def test_tensor_core_family_small_shapes(d, F, V, B, L, K):
     # the head chain as one kernel per GEMM instead of one persistent kernel
     out5, _ = run_gpu_draft(w, inp, K, flags=binding.MRP_FLAG_NO_CHAIN)
     check_stats(out5, ref, "bf16")
+    # the row-major kernels one CTA per tile instead of CTA pairs
+    if B * L > 128:
+        out6, _ = run_gpu_draft(w, inp, K, flags=binding.MRP_FLAG_NO_CTA_PAIRS)
+        check_stats(out6, ref, "bf16")
 
 
 @pytest.mark.parametrize("d,F,V,M,K,std,beyond", [
