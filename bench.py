@@ -46,11 +46,11 @@ MODULE_LAYERS, MODULE_ATTN_HEADS = 3, 16      # the paper's depth D = 3 (Sec. 4.
 # the ncu captures summarised under profiles/ (bytes per launch, and the summary they come from).
 NCU_TRAFFIC = {
     "decode_1p7b": (627908096, "profiles/lm_head_dram_traffic.md"),
-    "spec_8b": (1362025984, "profiles/lm_head_dram_traffic.md"),
-    "remask_8b": (1899798528, "profiles/lm_head_dram_traffic.md"),
-    "sweep_M64_K4": (1369512704, "profiles/lm_head_dram_traffic.md"),
-    "sweep_M256_K1": (1487823104, "profiles/lm_head_dram_traffic.md"),
-    "sweep_M4096_K4": (20161282048, "profiles/lm_head_dram_traffic.md"),
+    "spec_8b": (1366403328, "profiles/lm_head_dram_traffic.md"),
+    "remask_8b": (2794008320, "profiles/lm_head_dram_traffic.md"),
+    "sweep_M64_K4": (1368513792, "profiles/lm_head_dram_traffic.md"),
+    "sweep_M256_K1": (1486397184, "profiles/lm_head_dram_traffic.md"),
+    "sweep_M4096_K4": (35227708160, "profiles/lm_head_dram_traffic.md"),
 }
 
 
