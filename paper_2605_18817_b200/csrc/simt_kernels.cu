@@ -10,6 +10,7 @@
 #include <limits.h>
 #include <string.h>
 
+#include <atomic>
 #include <type_traits>
 
 #include "mrp_internal.cuh"
@@ -28,10 +29,27 @@ __device__ __forceinline__ float warp_sum(float v)
 
 constexpr int kRC = 4;     // activation rows a warp handles per pass over a weight row
 
+// Loads of buffers that another CTA of the SAME kernel may have written in an earlier phase (the one-kernel
+// pass below): CG = true reads through L2 (ld.global.cg), never from a line this SM cached before the write.
+template <bool CG> __device__ __forceinline__ float ldx(const float *p) { return CG ? __ldcg(p) : *p; }
+template <bool CG> __device__ __forceinline__ float4 ldx4(const float *p)
+{
+    return CG ? __ldcg(reinterpret_cast<const float4 *>(p)) : *reinterpret_cast<const float4 *>(p);
+}
+template <bool CG> __device__ __forceinline__ int ldxi(const int32_t *p) { return CG ? __ldcg(p) : *p; }
+template <bool CG> __device__ __forceinline__ Partial ld_partial(const Partial *p)
+{
+    if (!CG) return *p;
+    const float4 q = __ldcg(reinterpret_cast<const float4 *>(p));
+    Partial r;
+    r.mx = q.x; r.sum = q.y; r.idx = __float_as_int(q.z); r.second = q.w;
+    return r;
+}
+
 // Lane-partial dot products of one weight row with up to kRC activation rows (x: fp32 [rows, n_in]); the
 // caller adds the lanes.  bf16 weight rows whose length is a multiple of 256 are read 16 bytes per lane.
-template <typename T>
-__device__ __forceinline__ void row_dots(const T *__restrict__ wr, const float *__restrict__ x, int rows, int n_in, int lane,
+template <typename T, bool CG = false>
+__device__ __forceinline__ void row_dots(const T *__restrict__ wr, const float *x, int rows, int n_in, int lane,
                                          float *s)
 {
 #pragma unroll
@@ -47,8 +65,8 @@ __device__ __forceinline__ void row_dots(const T *__restrict__ wr, const float *
 #pragma unroll
             for (int r = 0; r < kRC; ++r) {
                 if (r < rows) {
-                    const float4 a = *reinterpret_cast<const float4 *>(x + (size_t)r * n_in + c);
-                    const float4 b = *reinterpret_cast<const float4 *>(x + (size_t)r * n_in + c + 4);
+                    const float4 a = ldx4<CG>(x + (size_t)r * n_in + c);
+                    const float4 b = ldx4<CG>(x + (size_t)r * n_in + c + 4);
                     float t = s[r];
                     t = fmaf(wv[0], a.x, t); t = fmaf(wv[1], a.y, t); t = fmaf(wv[2], a.z, t); t = fmaf(wv[3], a.w, t);
                     t = fmaf(wv[4], b.x, t); t = fmaf(wv[5], b.y, t); t = fmaf(wv[6], b.z, t); t = fmaf(wv[7], b.w, t);
@@ -57,11 +75,12 @@ __device__ __forceinline__ void row_dots(const T *__restrict__ wr, const float *
             }
         }
     } else {
+#pragma unroll 8
         for (int c = lane; c < n_in; c += 32) {
             const float a = ld_f(wr, c);
 #pragma unroll
             for (int r = 0; r < kRC; ++r)
-                if (r < rows) s[r] = fmaf(a, x[(size_t)r * n_in + c], s[r]);
+                if (r < rows) s[r] = fmaf(a, ldx<CG>(x + (size_t)r * n_in + c), s[r]);
         }
     }
 }
@@ -215,21 +234,20 @@ __global__ void down_kernel(const T *__restrict__ w_down, const float *__restric
 // tile l = l_0 + delta goes to shared memory, and warp w reduces row-step w of the chunk.
 constexpr int kLR = 8;
 
+// The work of CTA `cta` of `n_cta` (256 threads); `tile` is kLR * SLICE floats of its shared memory.
 template <typename T, int SLICE>
-__global__ void __launch_bounds__(256)
-lm_simt_kernel(const T *__restrict__ w_lm, const float *__restrict__ xt, const float *__restrict__ xt0,
-               const float *__restrict__ logits0, const int32_t *__restrict__ row_index, int M,
-               int K, int d, int V, int n_slices, Partial *__restrict__ partials,
-               float *__restrict__ logits_out, int n_rows_in, const float *__restrict__ teacher,
-               KlPartial *__restrict__ kl_partials, int l0_bf16)
+__device__ __forceinline__ void
+lm_simt_body(float (*tile)[SLICE], int cta, int n_cta,
+             const T *__restrict__ w_lm, const float *__restrict__ xt, const float *__restrict__ xt0,
+             const float *__restrict__ logits0, const int32_t *__restrict__ row_index, int M,
+             int K, int d, int V, int n_slices, Partial *__restrict__ partials,
+             float *__restrict__ logits_out, int n_rows_in, const float *__restrict__ teacher,
+             KlPartial *__restrict__ kl_partials, int l0_bf16)
 {
-    pdl_trigger();
-    pdl_wait();
-    __shared__ float tile[kLR][SLICE];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n_rs = (K + 1) * M;
     bool first = true;
-    for (int slice = blockIdx.x; slice < n_slices; slice += gridDim.x, first = false) {
+    for (int slice = cta; slice < n_slices; slice += n_cta, first = false) {
         const int v0 = slice * SLICE;
         for (int rs0 = 0; rs0 < n_rs; rs0 += kLR) {
             // delta for entries v0 + warp*16 .. +16, row-steps rs0 .. rs0+kLR
@@ -312,7 +330,7 @@ lm_simt_kernel(const T *__restrict__ w_lm, const float *__restrict__ xt, const f
                 if (lane == 0) {
                     Partial p;
                     p.mx = mx; p.sum = sum; p.idx = idx; p.second = sec;
-                    Partial *dst = partials + (size_t)blockIdx.x * n_rs + rs;
+                    Partial *dst = partials + (size_t)cta * n_rs + rs;
                     if (!first) p = merge_partial(*dst, p);
                     *dst = p;
                 }
@@ -342,7 +360,7 @@ lm_simt_kernel(const T *__restrict__ w_lm, const float *__restrict__ xt, const f
                     if (lane == 0) {
                         KlPartial q;
                         q.mx = tmx; q.sum = ts; q.cross = tc; q.pad = 0.f;
-                        KlPartial *dst = kl_partials + (size_t)blockIdx.x * (size_t)(K * M) + (rs - M);
+                        KlPartial *dst = kl_partials + (size_t)cta * (size_t)(K * M) + (rs - M);
                         if (!first) q = merge_kl(*dst, q);
                         *dst = q;
                     }
@@ -353,23 +371,35 @@ lm_simt_kernel(const T *__restrict__ w_lm, const float *__restrict__ xt, const f
     }
 }
 
-// ---- a4: combine per-slice partials -------------------------------------------------------
-__global__ void combine_kernel(const Partial *__restrict__ partials, int n_slices, int n_rs,
-                               float *__restrict__ conf, float *__restrict__ lse,
-                               int32_t *__restrict__ token, float *__restrict__ margin,
-                               int32_t *__restrict__ status, int32_t *__restrict__ user_status,
-                               const TopFix fix, const KlPartial *__restrict__ kl_partials, int M,
-                               float *__restrict__ kl_out)
+template <typename T, int SLICE>
+__global__ void __launch_bounds__(256)
+lm_simt_kernel(const T *__restrict__ w_lm, const float *__restrict__ xt, const float *__restrict__ xt0,
+               const float *__restrict__ logits0, const int32_t *__restrict__ row_index, int M,
+               int K, int d, int V, int n_slices, Partial *__restrict__ partials,
+               float *__restrict__ logits_out, int n_rows_in, const float *__restrict__ teacher,
+               KlPartial *__restrict__ kl_partials, int l0_bf16)
 {
     pdl_trigger();
     pdl_wait();
-    const int rs = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    const int lane = threadIdx.x & 31;
-    if (rs >= n_rs) return;
+    __shared__ float tile[kLR][SLICE];
+    lm_simt_body<T, SLICE>(tile, blockIdx.x, gridDim.x, w_lm, xt, xt0, logits0, row_index, M, K, d, V, n_slices, partials,
+                           logits_out, n_rows_in, teacher, kl_partials, l0_bf16);
+}
+
+// ---- a4: combine per-slice partials -------------------------------------------------------
+// One warp merges the slices of row-step rs.
+template <bool CG = false>
+__device__ __forceinline__ void combine_body(int rs, int lane, const Partial *partials, int n_slices, int n_rs,
+                                             float *__restrict__ conf, float *__restrict__ lse,
+                                             int32_t *__restrict__ token, float *__restrict__ margin,
+                                             int32_t *__restrict__ status, int32_t *__restrict__ user_status,
+                                             const TopFix &fix, const KlPartial *__restrict__ kl_partials, int M,
+                                             float *__restrict__ kl_out)
+{
     Partial p;
     p.mx = -INFINITY; p.sum = 0.f; p.idx = INT_MAX; p.second = -INFINITY;
 #pragma unroll 8
-    for (int s = lane; s < n_slices; s += 32) p = merge_partial(p, partials[(size_t)s * n_rs + rs]);
+    for (int s = lane; s < n_slices; s += 32) p = merge_partial(p, ld_partial<CG>(partials + (size_t)s * n_rs + rs));
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
         Partial q;
@@ -459,6 +489,21 @@ __global__ void combine_kernel(const Partial *__restrict__ partials, int n_slice
     }
 }
 
+__global__ void combine_kernel(const Partial *__restrict__ partials, int n_slices, int n_rs,
+                               float *__restrict__ conf, float *__restrict__ lse,
+                               int32_t *__restrict__ token, float *__restrict__ margin,
+                               int32_t *__restrict__ status, int32_t *__restrict__ user_status,
+                               const TopFix fix, const KlPartial *__restrict__ kl_partials, int M,
+                               float *__restrict__ kl_out)
+{
+    pdl_trigger();
+    pdl_wait();
+    const int rs = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (rs >= n_rs) return;
+    combine_body(rs, threadIdx.x & 31, partials, n_slices, n_rs, conf, lse, token, margin, status, user_status, fix,
+                 kl_partials, M, kl_out);
+}
+
 cudaError_t launch_combine(Ctx *c, const Partial *partials, int n_slices, int n_rowsteps,
                            const mrp_draft_out &out, int32_t *status, cudaStream_t st, const TopFix *fix, int M)
 {
@@ -476,21 +521,16 @@ cudaError_t launch_combine(Ctx *c, const Partial *partials, int n_slices, int n_
 }
 
 // ---- conf_first: probability of the step-0 argmax token under every step's logits ----------
-__global__ void first_token_prob_kernel(const FirstTok f, const int32_t *__restrict__ token,
-                                        const float *__restrict__ lse, const float *__restrict__ conf,
-                                        float *__restrict__ conf_first)
+template <bool CG = false>
+__device__ __forceinline__ void first_token_prob_body(int rs, int lane, const FirstTok &f, const int32_t *token,
+                                                      const float *lse, const float *conf, float *conf_first)
 {
-    pdl_trigger();
-    pdl_wait();
-    const int rs = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    const int lane = threadIdx.x & 31;
-    if (rs >= (f.K + 1) * f.M) return;
     const int k = rs / f.M, m = rs - k * f.M;
     if (k == 0) {                     // the step-0 token is the top token of step 0
-        if (lane == 0) conf_first[rs] = conf[rs];
+        if (lane == 0) conf_first[rs] = ldx<CG>(conf + rs);
         return;
     }
-    const int tok = token[m];
+    const int tok = ldxi<CG>(token + m);
     float dot = 0.f;
     if (f.x_bf16 && f.w8_scale) {
         // 8-bit LM head: the row of the dequantised matrix, scale[tok] * e4m3 code
@@ -517,7 +557,7 @@ __global__ void first_token_prob_kernel(const FirstTok f, const int32_t *__restr
         for (int j = lane; j < f.d; j += 32) {
             const float wv = f.w_bf16 ? __bfloat162float(((const __nv_bfloat16 *)f.w)[(size_t)tok * f.d + j])
                                       : ((const float *)f.w)[(size_t)tok * f.d + j];
-            dot = fmaf(wv, xr[j], dot);
+            dot = fmaf(wv, ldx<CG>(xr + j), dot);
         }
     }
     dot = warp_sum(dot);
@@ -525,8 +565,19 @@ __global__ void first_token_prob_kernel(const FirstTok f, const int32_t *__restr
         const int idx = f.row_index ? f.row_index[m] : m;
         const bool have = f.logits0 && (!f.row_index || row_ok(idx, f.n_rows_in));
         const float l = (have ? ld_l0(f.logits0, f.l0_bf16, (size_t)idx * (size_t)f.V + tok) : 0.f) + dot;
-        conf_first[rs] = fminf(expf(l - lse[rs]), conf[rs]);     // never above the top probability
+        conf_first[rs] = fminf(expf(l - ldx<CG>(lse + rs)), ldx<CG>(conf + rs));     // never above the top probability
     }
+}
+
+__global__ void first_token_prob_kernel(const FirstTok f, const int32_t *__restrict__ token,
+                                        const float *__restrict__ lse, const float *__restrict__ conf,
+                                        float *__restrict__ conf_first)
+{
+    pdl_trigger();
+    pdl_wait();
+    const int rs = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (rs >= (f.K + 1) * f.M) return;
+    first_token_prob_body(rs, threadIdx.x & 31, f, token, lse, conf, conf_first);
 }
 
 cudaError_t launch_first_token_prob(Ctx *c, const FirstTok &f, const mrp_draft_out &out, cudaStream_t st)
@@ -625,10 +676,411 @@ static cudaError_t simt_draft_t(Ctx *c, const void *hidden, const float *logits0
     return simt_lm_tail(c, logits0, row_index, M, K, out, st);
 }
 
+// ---- the whole pass as ONE kernel, for a few short rows ---------------------------------------
+// A small shape (the tiny configuration: 4 rows of 256) is a dozen launches of a few microseconds each when
+// every step is a kernel of its own; here the same steps are phases of one cooperative kernel, separated by
+// grid barriers: gather -> per head [RMSNorm + gate/up + SwiGLU | down projection + residual] -> LM head with
+// per-CTA softmax partials -> combine -> (probability of the step-0 token).  The phases run the code of the
+// separate kernels (row_dots, lm_simt_body, combine_body), reading what earlier phases wrote through L2.
+// The barrier is a counter that only grows: a launch reads where the last one left it (bar[1]), barrier i
+// is passed once the counter reaches base + (i + 1) * gridDim.x, and CTA 0 leaves base + n_barriers *
+// gridDim.x behind for the next launch.  A wait that runs out (about half a second) raises MRP_DEV_TIMEOUT,
+// and the CTA adds the arrivals it still owes before it returns, so that the counter ends where the next
+// launch expects it whatever happened.
+constexpr int kFusedMaxRows = 8;
+constexpr int kFusedMaxD = 512;
+constexpr int kFusedMaxHeads = 8;
+constexpr int kFusedMaxRowSteps = 32;  // (K + 1) * M: a lane per row-step in the LM-head phase
+constexpr int kFusedEntries = 4;       // vocabulary entries a warp works on at a time in the LM-head phase
+constexpr size_t kFusedMaxSmem = 160 * 1024;
+constexpr long long kFusedBarrierCycles = 1000000000LL;
+
+template <typename T>
+struct FusedParams {
+    const T *hidden, *w_lm, *final_gamma;
+    const T *gamma[kFusedMaxHeads], *w_gate[kFusedMaxHeads], *w_up[kFusedMaxHeads], *w_down[kFusedMaxHeads];
+    const int32_t *row_index;
+    const float *logits0;
+    int M, K, d, F, V, n_rows_in, l0_bf16;
+    float eps;
+    float *h0f, *hcur, *act, *xt, *xt0;     // workspace (xt0: operand rows of step 0, or nullptr)
+    Partial *partials;
+    float *conf, *lse, *margin, *logits_out, *hidden_out, *conf_first;
+    int32_t *token;
+    int32_t *status, *user_status;
+    unsigned int *bar;                      // [0] arrivals so far, [1] their number when this launch began
+    FirstTok ft;
+};
+
+struct FusedSync {
+    unsigned int base;
+    int done, total;
+};
+
+// All threads of all CTAs.  False: the wait ran out (the caller returns; the owed arrivals are already paid).
+template <typename T>
+__device__ __forceinline__ bool fused_barrier(const FusedParams<T> &p, FusedSync &sy)
+{
+    __syncthreads();
+    int ok = 1;
+    sy.done++;
+    if (threadIdx.x == 0) {
+        __threadfence();
+        atomicAdd(p.bar, 1u);
+        const unsigned int target = sy.base + (unsigned int)sy.done * gridDim.x;
+        const long long t0 = clock64();
+        while ((int)(*reinterpret_cast<volatile unsigned int *>(p.bar) - target) < 0) {
+            if (clock64() - t0 > kFusedBarrierCycles) { ok = 0; break; }
+        }
+        __threadfence();
+        if (!ok) {
+            atomicOr(p.status, MRP_DEV_TIMEOUT);
+            if (p.user_status) atomicOr(p.user_status, MRP_DEV_TIMEOUT);
+            if (sy.total > sy.done) atomicAdd(p.bar, (unsigned int)(sy.total - sy.done));
+        }
+    }
+    return __syncthreads_and(ok) != 0;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256)
+simt_fused_kernel(const FusedParams<T> p)
+{
+    // normalised rows [M, d] in the head phases; in the LM-head phase the operand rows [(K+1) M, d + 1],
+    // one weight row per warp [8, d] and the warps' partials [8, 32]
+    extern __shared__ __align__(16) float sh[];
+    __shared__ float red[8];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int G = gridDim.x, cta = blockIdx.x;
+    const int gw = cta * 8 + warp, n_gw = G * 8;
+    const int M = p.M, K = p.K, d = p.d, F = p.F;
+    FusedSync sy;
+    sy.base = *reinterpret_cast<volatile unsigned int *>(p.bar + 1);
+    sy.done = 0;
+    sy.total = 2 * K + 3 + (p.conf_first ? 1 : 0);
+    // what CTA 0 leaves for the next launch, on every way out
+    auto leave = [&]() {
+        if (cta == 0 && threadIdx.x == 0) {
+            *reinterpret_cast<volatile unsigned int *>(p.bar + 1) = sy.base + (unsigned int)sy.total * G;
+            __threadfence();
+        }
+    };
+
+    // ---- gather the masked rows (CTA per row) ----
+    for (int m = cta; m < M; m += G) {
+        const int idx = p.row_index ? p.row_index[m] : m;
+        const bool bad = p.row_index && !row_ok(idx, p.n_rows_in);
+        if (bad && threadIdx.x == 0) {
+            atomicOr(p.status, MRP_DEV_BAD_INDEX);
+            if (p.user_status) atomicOr(p.user_status, MRP_DEV_BAD_INDEX);
+        }
+        const size_t row = bad ? 0 : (size_t)idx;
+        float ss = 0.f;
+        for (int j = threadIdx.x; j < d; j += blockDim.x) {
+            const float v = bad ? 0.f : ld_f(p.hidden, row * d + j);
+            if (!p.xt0) p.h0f[(size_t)m * d + j] = v;
+            p.hcur[(size_t)m * d + j] = v;
+            ss = fmaf(v, v, ss);
+        }
+        if (p.xt0) {
+            // no base logits: step 0's operand is n_0 = h_0 or RMSNorm(h_0) * final_gamma, h0f = h_0 - n_0
+            ss = warp_sum(ss);
+            __syncthreads();
+            if (lane == 0) red[warp] = ss;
+            __syncthreads();
+            float t = 0.f;
+            for (int i = 0; i < 8; ++i) t += red[i];
+            const float rstd0 = p.final_gamma ? rsqrtf(t / (float)d + p.eps) : 1.f;
+            for (int j = threadIdx.x; j < d; j += blockDim.x) {
+                const float v = bad ? 0.f : ld_f(p.hidden, row * d + j);
+                const float n0 = p.final_gamma ? v * rstd0 * ld_f(p.final_gamma, j) : v;
+                p.h0f[(size_t)m * d + j] = v - n0;
+                p.xt0[(size_t)m * d + j] = n0;
+            }
+        }
+    }
+    if (!fused_barrier(p, sy)) { leave(); return; }
+
+    for (int k = 1; k <= K; ++k) {
+        // ---- RMSNorm of all rows into shared memory (every CTA its own copy), then gate/up + SwiGLU ----
+        for (int m = warp; m < M; m += 8) {
+            float ss = 0.f;
+#pragma unroll 8
+            for (int j = lane; j < d; j += 32) {
+                const float v = __ldcg(p.hcur + (size_t)m * d + j);
+                sh[m * d + j] = v;
+                ss = fmaf(v, v, ss);
+            }
+            ss = warp_sum(ss);
+            const float rstd = rsqrtf(ss / (float)d + p.eps);
+            for (int j = lane; j < d; j += 32) sh[m * d + j] = sh[m * d + j] * rstd * ld_f(p.gamma[k - 1], j);
+        }
+        __syncthreads();
+        for (int f = gw; f < F; f += n_gw) {
+            const T *wg = p.w_gate[k - 1] + (size_t)f * d, *wu = p.w_up[k - 1] + (size_t)f * d;
+            for (int m0 = 0; m0 < M; m0 += kRC) {
+                float g[kRC], u[kRC];
+                row_dots<T>(wg, sh + (size_t)m0 * d, M - m0, d, lane, g);
+                row_dots<T>(wu, sh + (size_t)m0 * d, M - m0, d, lane, u);
+#pragma unroll
+                for (int r = 0; r < kRC; ++r) {
+                    const float gs = warp_sum(g[r]), us = warp_sum(u[r]);
+                    if (lane == 0 && m0 + r < M) p.act[(size_t)(m0 + r) * F + f] = gs / (1.f + expf(-gs)) * us;
+                }
+            }
+        }
+        if (!fused_barrier(p, sy)) { leave(); return; }
+        // ---- down projection, h <- h + Delta, LM-head operand h_k - h_0 ----
+        if (cta * 8 < d) {             // CTAs with an output feature: the activations [M, F] into shared memory, through L2
+            for (int i = threadIdx.x * 4; i < M * F; i += blockDim.x * 4) {
+                if (((M * F) & 3) == 0) *reinterpret_cast<float4 *>(sh + i) = __ldcg(reinterpret_cast<const float4 *>(p.act + i));
+                else for (int e = i; e < i + 4 && e < M * F; ++e) sh[e] = __ldcg(p.act + e);
+            }
+        }
+        __syncthreads();
+        for (int j = gw; j < d; j += n_gw) {
+            const T *wd = p.w_down[k - 1] + (size_t)j * F;
+            for (int m0 = 0; m0 < M; m0 += kRC) {
+                float s[kRC];
+                row_dots<T>(wd, sh + (size_t)m0 * F, M - m0, F, lane, s);
+#pragma unroll
+                for (int r = 0; r < kRC; ++r) {
+                    const float v = warp_sum(s[r]);
+                    if (lane == 0 && m0 + r < M) {
+                        const size_t o = (size_t)(m0 + r) * d + j;
+                        const float hn = __ldcg(p.hcur + o) + v;
+                        p.hcur[o] = hn;
+                        p.xt[(size_t)(k - 1) * M * d + o] = hn - __ldcg(p.h0f + o);
+                        if (k == K && p.hidden_out) p.hidden_out[o] = hn;
+                    }
+                }
+            }
+        }
+        if (!fused_barrier(p, sy)) { leave(); return; }
+    }
+
+    // ---- LM head on the residuals, added to l_0 (Eq. 2), softmax statistics per CTA ----
+    // Lane = row-step: a warp takes one vocabulary entry at a time, puts its weight row into shared memory,
+    // and every lane forms the whole dot product of its own operand row with it; the lane then folds the logit
+    // into the running statistics of its row-step, so nothing is exchanged between lanes until the end.
+    const int n_rs = (K + 1) * M;
+    {
+        const int ldx_s = d + 1;                       // odd pitch: lanes read one column of 32 rows without conflicts
+        const size_t xs_floats = ((size_t)n_rs * ldx_s + 3) & ~(size_t)3;
+        const size_t w_floats = ((size_t)8 * kFusedEntries * d + 3) & ~(size_t)3;
+        float *xs = sh, *wrow = sh + xs_floats + (size_t)warp * kFusedEntries * d;
+        Partial *wp = reinterpret_cast<Partial *>(sh + xs_floats + w_floats);
+        const bool vec = (d & 3) == 0;                 // 16-byte reads of the (broadcast) weight rows
+        if (vec) {
+#pragma unroll 4
+            for (int i = threadIdx.x * 4; i < n_rs * d; i += blockDim.x * 4) {
+                const int rs = i / d, j = i - rs * d;
+                float4 v = make_float4(0.f, 0.f, 0.f, 0.f);              // step 0 has no residual ...
+                if (rs >= M) v = __ldcg(reinterpret_cast<const float4 *>(p.xt + (size_t)(rs - M) * d + j));
+                else if (p.xt0) v = __ldcg(reinterpret_cast<const float4 *>(p.xt0 + (size_t)rs * d + j));   // ... unless computed here
+                float *dst = xs + rs * ldx_s + j;
+                dst[0] = v.x; dst[1] = v.y; dst[2] = v.z; dst[3] = v.w;
+            }
+        } else {
+#pragma unroll 4
+            for (int i = threadIdx.x; i < n_rs * d; i += blockDim.x) {
+                const int rs = i / d, j = i - rs * d;
+                float v = 0.f;
+                if (rs >= M) v = __ldcg(p.xt + (size_t)(rs - M) * d + j);
+                else if (p.xt0) v = __ldcg(p.xt0 + (size_t)rs * d + j);
+                xs[rs * ldx_s + j] = v;
+            }
+        }
+        __syncthreads();
+        Partial st;
+        st.mx = -INFINITY; st.sum = 0.f; st.idx = INT_MAX; st.second = -INFINITY;
+        const bool mine = lane < n_rs;
+        const int m = mine ? lane % M : 0;
+        const int idx = p.row_index ? p.row_index[m] : m;
+        const bool have = mine && p.logits0 && (!p.row_index || row_ok(idx, p.n_rows_in));
+        const float *xr = xs + (size_t)(mine ? lane : 0) * ldx_s;
+        // kFusedEntries consecutive entries per warp and round: every operand element read from shared memory
+        // feeds that many products
+        for (int v0 = gw * kFusedEntries; v0 < p.V; v0 += n_gw * kFusedEntries) {
+            const int n_e = min(kFusedEntries, p.V - v0);
+            float l0[kFusedEntries];
+#pragma unroll
+            for (int e = 0; e < kFusedEntries; ++e)
+                l0[e] = (have && e < n_e) ? ld_l0(p.logits0, p.l0_bf16, (size_t)idx * (size_t)p.V + v0 + e) : 0.f;
+#pragma unroll 8
+            for (int i = lane; i < n_e * d; i += 32) wrow[i] = ld_f(p.w_lm, (size_t)v0 * d + i);
+            for (int i = n_e * d + lane; i < kFusedEntries * d; i += 32) wrow[i] = 0.f;
+            __syncwarp();
+            // two running sums per entry, each over every other group of four (short chains keep the fp32
+            // rounding of a long dot product small)
+            float a[kFusedEntries][2];
+#pragma unroll
+            for (int e = 0; e < kFusedEntries; ++e) a[e][0] = a[e][1] = 0.f;
+            int j = 0;
+            if (vec) {
+                for (; j + 8 <= d; j += 8) {
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        const float x0 = xr[j + 4 * h], x1 = xr[j + 4 * h + 1], x2 = xr[j + 4 * h + 2], x3 = xr[j + 4 * h + 3];
+#pragma unroll
+                        for (int e = 0; e < kFusedEntries; ++e) {
+                            const float4 w4 = *reinterpret_cast<const float4 *>(wrow + e * d + j + 4 * h);
+                            float t = a[e][h];
+                            t = fmaf(w4.x, x0, t); t = fmaf(w4.y, x1, t); t = fmaf(w4.z, x2, t); t = fmaf(w4.w, x3, t);
+                            a[e][h] = t;
+                        }
+                    }
+                }
+            }
+            for (; j < d; ++j) {
+                const float x0 = xr[j];
+#pragma unroll
+                for (int e = 0; e < kFusedEntries; ++e) a[e][j & 1] = fmaf(wrow[e * d + j], x0, a[e][j & 1]);
+            }
+            __syncwarp();
+            if (mine) {
+#pragma unroll
+                for (int e = 0; e < kFusedEntries; ++e) {
+                    if (e < n_e) {
+                        const int v = v0 + e;
+                        const float l = l0[e] + (a[e][0] + a[e][1]);
+                        if (l > st.mx) {                 // entries come in ascending order: the lowest id keeps a tie
+                            st.sum = st.sum * expf(st.mx - l) + 1.f;
+                            st.second = st.mx; st.mx = l; st.idx = v;
+                        } else {
+                            st.sum += expf(l - st.mx);
+                            if (l > st.second) st.second = l;
+                        }
+                        if (p.logits_out && lane >= M) p.logits_out[(size_t)(lane - M) * p.V + v] = l;
+                    }
+                }
+            }
+        }
+        wp[warp * 32 + lane] = st;
+        __syncthreads();
+        if (warp == 0 && mine) {
+            Partial t = wp[lane];
+#pragma unroll
+            for (int w8 = 1; w8 < 8; ++w8) t = merge_partial(t, wp[w8 * 32 + lane]);
+            p.partials[(size_t)cta * n_rs + lane] = t;
+        }
+    }
+    if (!fused_barrier(p, sy)) { leave(); return; }
+
+    // ---- combine the CTAs' partials (warp per row-step) ----
+    const int n_parts = G;
+    TopFix nofix;
+    memset(&nofix, 0, sizeof(nofix));
+    for (int rs = gw; rs < n_rs; rs += n_gw)
+        combine_body<true>(rs, lane, p.partials, n_parts, n_rs, p.conf, p.lse, p.token, p.margin, p.status, p.user_status,
+                           nofix, nullptr, M, nullptr);
+    if (p.conf_first) {
+        if (!fused_barrier(p, sy)) { leave(); return; }
+        for (int rs = gw; rs < n_rs; rs += n_gw)
+            first_token_prob_body<true>(rs, lane, p.ft, p.token, p.lse, p.conf, p.conf_first);
+    }
+    // the last barrier: nobody leaves (and CTA 0 does not publish the next base) before all have arrived
+    fused_barrier(p, sy);
+    leave();
+}
+
+static size_t fused_smem(int M, int K, int d)
+{
+    const size_t lm = ((((size_t)(K + 1) * M * (d + 1) + 3) & ~(size_t)3) + (((size_t)8 * kFusedEntries * d + 3) & ~(size_t)3)) * 4 +
+                      8 * 32 * sizeof(Partial);
+    return lm;      // (the head phases' [M, d] and [M, F] arrays are checked against it in fused_ok)
+}
+
+// Whether a call runs as the one-kernel pass: a few short rows, at least one head, no KL objective; not under
+// MRP_FLAG_NO_CHAIN (which asks for one kernel per step).
+static bool fused_ok(const Ctx *c, int M, int K)
+{
+    return M >= 1 && M <= kFusedMaxRows && c->cfg.d <= kFusedMaxD && K >= 1 && K <= kFusedMaxHeads &&
+           (K + 1) * M <= kFusedMaxRowSteps && !c->teacher && !(c->cfg.flags & MRP_FLAG_NO_CHAIN) &&
+           fused_smem(M, K, c->cfg.d) <= kFusedMaxSmem && (size_t)M * c->cfg.d_ff * 4 <= fused_smem(M, K, c->cfg.d);
+}
+
+template <typename T>
+static cudaError_t simt_fused_t(Ctx *c, const void *hidden, const float *logits0, const int32_t *row_index, int M, int K,
+                                const mrp_draft_out &out, cudaStream_t st, bool *launched)
+{
+    *launched = false;
+    auto kern = simt_fused_kernel<T>;
+    // all CTAs wait for one another: they must be resident together (asked once per device)
+    static std::atomic<unsigned long long> asked{0}, fits{0};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    const unsigned long long bit = 1ull << (dev & 63);
+    if (!(asked.load() & bit)) {
+        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFusedMaxSmem);
+        if (e != cudaSuccess) return e;
+        int per_sm = 0;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, 256, kFusedMaxSmem);
+        if (e != cudaSuccess) return e;
+        if (per_sm >= 1) fits.fetch_or(bit);
+        asked.fetch_or(bit);
+    }
+    if (!(fits.load() & bit)) return cudaSuccess;
+    const int d = c->cfg.d, V = c->cfg.vocab;
+    FusedParams<T> p;
+    memset(&p, 0, sizeof(p));
+    p.hidden = (const T *)hidden; p.w_lm = (const T *)c->w_lm; p.final_gamma = (const T *)c->final_gamma;
+    for (int k = 0; k < K; ++k) {
+        p.gamma[k] = (const T *)c->heads[k].rms_gamma; p.w_gate[k] = (const T *)c->heads[k].w_gate;
+        p.w_up[k] = (const T *)c->heads[k].w_up; p.w_down[k] = (const T *)c->heads[k].w_down;
+    }
+    p.row_index = row_index; p.logits0 = logits0;
+    p.M = M; p.K = K; p.d = d; p.F = c->cfg.d_ff; p.V = V; p.n_rows_in = c->input_rows; p.l0_bf16 = c->l0_bf16 ? 1 : 0;
+    p.eps = c->cfg.rms_eps;
+    p.h0f = (float *)(c->ws + c->lay.h0f); p.hcur = (float *)(c->ws + c->lay.hcur);
+    p.act = (float *)(c->ws + c->lay.act); p.xt = (float *)(c->ws + c->lay.xt);
+    p.xt0 = c->from_hidden ? p.xt + (size_t)K * M * d : nullptr;
+    p.partials = (Partial *)(c->ws + c->lay.partials);
+    p.conf = out.conf; p.lse = out.lse; p.margin = out.margin; p.logits_out = out.logits_out; p.hidden_out = out.hidden_out;
+    p.conf_first = out.conf_first; p.token = out.token;
+    p.status = (int32_t *)(c->ws + c->lay.status); p.user_status = out.status;
+    p.bar = (unsigned int *)(c->ws + c->lay.status) + 16;
+    p.ft.w = c->w_lm; p.ft.w_bf16 = c->cfg.dtype == MRP_BF16; p.ft.logits0 = logits0; p.ft.row_index = row_index;
+    p.ft.l0_bf16 = p.l0_bf16; p.ft.n_rows_in = c->input_rows; p.ft.x = p.xt; p.ft.x_bf16 = 0;
+    p.ft.M = M; p.ft.K = K; p.ft.d = d; p.ft.V = V;
+    int grid = c->sm_count;
+    if (grid > c->lay.n_slices_max) grid = c->lay.n_slices_max;
+    prof_mark(c, 0, st);
+    e = note_err(c, wait_logits0(c, st), "wait for the base logits");
+    if (e != cudaSuccess) return e;
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(256);
+    cfg.dynamicSmemBytes = fused_smem(M, K, d);
+    cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeCooperative;
+    at[0].val.cooperative = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    e = note_err(c, cudaLaunchKernelEx(&cfg, kern, p), "one-kernel CUDA-core pass");
+    c->launches++;
+    *launched = true;
+    // the phases of the pass are not separate launches: the profile books the whole kernel under the heads
+    prof_mark(c, 1, st);
+    prof_mark(c, 2, st);
+    prof_mark(c, 3, st);
+    return e;
+}
+
 cudaError_t simt_draft(Ctx *c, const void *hidden, const float *logits0, const int32_t *row_index,
                        int M, int K, const mrp_draft_out &out, cudaStream_t st)
 {
     if (M == 0) return cudaSuccess;
+    if (fused_ok(c, M, K)) {
+        bool launched = false;
+        const cudaError_t e = c->cfg.dtype == MRP_F32
+                                  ? simt_fused_t<float>(c, hidden, logits0, row_index, M, K, out, st, &launched)
+                                  : simt_fused_t<__nv_bfloat16>(c, hidden, logits0, row_index, M, K, out, st, &launched);
+        if (launched || e != cudaSuccess) return e;
+    }
     if (c->cfg.dtype == MRP_F32)
         return simt_draft_t<float>(c, hidden, logits0, row_index, M, K, out, st);
     return simt_draft_t<__nv_bfloat16>(c, hidden, logits0, row_index, M, K, out, st);

@@ -114,6 +114,70 @@ def test_ragged_shapes_on_cuda_cores(dtype, flags):
         check_stats(o, r, "f32")
 
 
+@pytest.mark.parametrize("dtype,flags", [("f32", 0), ("bf16", binding.MRP_FLAG_FORCE_SIMT)])
+@pytest.mark.parametrize("d,F,V,B,L", [(72, 136, 1000, 2, 3), (256, 512, 4096, 1, 4), (512, 264, 20000, 2, 4)])
+def test_one_kernel_pass_for_a_few_short_rows(dtype, flags, d, F, V, B, L):
+    """Up to 8 rows of up to 512 features run the whole drafting pass as one cooperative kernel on the CUDA
+    cores: one launch, same results as one kernel per step (MRP_FLAG_NO_CHAIN) up to the merge order of the slices, oracle parity
+    with every optional output, repeated calls (the grid barrier's counter carries over from call to call),
+    the base logits computed in the pass, a row subset and an out-of-range row."""
+    K = 3
+    # (the fp32 tolerance is absolute, 1e-5: residuals that keep the logits near 10, where that is 10 ulp)
+    w = synth.make_weights(d, F, V, K, dtype, 47, head_std=0.1 if d < 512 else 0.03)
+    inp = synth.make_inputs(w, B, L, 47, 1.0, 4.0)
+    M = len(inp.row_index)
+    assert 1 <= M <= 8
+    heads, w_lm = harness.upload_weights(w, DEV)
+    ctx = binding.mrp_create(d, F, V, heads, w_lm, max_rows=B * L, max_seqs=B, block_len=L, flags=flags)
+    ctx1 = binding.mrp_create(d, F, V, heads, w_lm, max_rows=B * L, max_seqs=B, block_len=L,
+                              flags=flags | binding.MRP_FLAG_NO_CHAIN)
+    assert ctx.family == "simt"
+    hid = harness.to_device(inp.hidden, w.dtype, DEV)
+    l0 = torch.from_numpy(inp.logits0).to(DEV)
+    ri = torch.from_numpy(inp.row_index).to(DEV)
+    ref = oracle.draft(inp.hidden, inp.logits0, w.heads, w.w_lm, K=K, row_index=inp.row_index, want_logits=True,
+                       want_hidden=True)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    for rep in range(3):
+        out = harness.alloc_draft_out(M, K, V, d, DEV, margin=True, logits=True, hidden=True, conf_first=True)
+        out.status = status
+        harness.draft(ctx, hid, l0, ri, M, K, out)
+        torch.cuda.synchronize()
+        assert ctx.last_launch_count == 1
+        check_stats(out, ref, "f32")
+        assert np.abs(out.logits.cpu().numpy() - ref.logits).max() <= 1e-4
+        assert np.abs(out.hidden.cpu().numpy() - ref.hidden).max() <= 1e-4
+        clear0 = ref.margin[0] > 1e-2
+        assert np.abs(out.conf_first.cpu().numpy() - ref.conf_first)[:, clear0].max() <= 1e-5
+    assert int(status.item()) == 0
+    sep = harness.alloc_draft_out(M, K, V, d, DEV, margin=True)
+    harness.draft(ctx1, hid, l0, ri, M, K, sep)
+    torch.cuda.synchronize()
+    assert ctx1.last_launch_count > 1
+    assert torch.equal(sep.token, out.token)
+    assert float((sep.conf - out.conf).abs().max()) <= 1e-5 and float((sep.lse - out.lse).abs().max()) <= 1e-5
+    # shorter chain, row subset, base logits computed in the pass
+    sub = inp.row_index[::2]
+    o2 = harness.alloc_draft_out(len(sub), 2, V, d, DEV)
+    harness.draft_from_hidden(ctx, hid, None, torch.from_numpy(sub).to(DEV), len(sub), 2, o2)
+    torch.cuda.synchronize()
+    assert ctx.last_launch_count == 1
+    check_stats(o2, oracle.draft(inp.hidden, None, w.heads, w.w_lm, K=2, row_index=sub), "f32")
+    # an out-of-range row reads as zeros and raises the status bit; the other rows are untouched by it
+    bad = inp.row_index.copy()
+    bad[-1] = B * L + 5
+    o3 = harness.alloc_draft_out(M, K, V, d, DEV)
+    o3.status = status
+    harness.draft(ctx, hid, l0, torch.from_numpy(bad).to(DEV), M, K, o3)
+    torch.cuda.synchronize()
+    assert int(status.item()) & binding.MRP_DEV_BAD_INDEX
+    if M > 1:
+        assert torch.equal(o3.token[:, :M - 1], out.token[:, :M - 1])
+        assert float((o3.conf[:, :M - 1] - out.conf[:, :M - 1]).abs().max()) <= 1e-5
+    binding.mrp_destroy(ctx)
+    binding.mrp_destroy(ctx1)
+
+
 def test_empty_call_and_argument_errors():
     cfg = synth.CONFIGS[0]
     w, inp = synth.make_config(cfg)
