@@ -718,8 +718,8 @@ struct FusedSync {
 };
 
 // All threads of all CTAs.  False: the wait ran out (the caller returns; the owed arrivals are already paid).
-template <typename T>
-__device__ __forceinline__ bool fused_barrier(const FusedParams<T> &p, FusedSync &sy)
+template <typename P>
+__device__ __forceinline__ bool fused_barrier(const P &p, FusedSync &sy)
 {
     __syncthreads();
     int ok = 1;
@@ -935,7 +935,7 @@ simt_fused_kernel(const FusedParams<T> p)
             for (; j < d; ++j) {
                 const float x0 = xr[j];
 #pragma unroll
-                for (int e = 0; e < kFusedEntries; ++e) a[e][j & 1] = fmaf(wrow[e * d + j], x0, a[e][j & 1]);
+                for (int e = 0; e < kFusedEntries; ++e) a[e][0] = fmaf(wrow[e * d + j], x0, a[e][0]);
             }
             __syncwarp();
             if (mine) {
@@ -1231,6 +1231,454 @@ __global__ void mod_operand_kernel(const float *__restrict__ h_state, const T *_
     }
 }
 
+// ---- the module step as ONE kernel, for a handful of positions -----------------------------------
+// With n = B * L <= 4 positions every matrix of the module is a matrix-vector product bound by its own weight
+// stream (269 MB per step at d = 2048, F = 4096, D = 3), and a kernel per product leaves the stream idle
+// between 33 launches.  Here the step is one cooperative kernel of 5 D + 2 phases between grid barriers (the
+// barrier of the one-kernel drafting pass above):
+//   [h ; emb[x]] -> z = W_proj .   | per layer: RMSNorm -> q, k, v | attention, a warp per (position, head)
+//   | z += W_o o | RMSNorm -> silu(gate) * up | z += W_down a | h += z, LM-head operand of the masked rows.
+// A product phase stages its input rows in shared memory (what other CTAs wrote: through L2) and every warp
+// walks groups of four weight rows at once: each 16-byte read of an input row from shared memory then feeds four
+// rows' products (one weight row at a time would need 128 bytes of shared memory per 16 bytes of weights), and
+// four independent 16-byte weight loads are in flight per lane and iteration.  Where a product has fewer groups
+// than the grid has warps its contraction is cut across the warps of a CTA, which add their parts in a fixed
+// order.
+constexpr int kModThreads = 512;
+constexpr int kModRows = 4;            // positions (rows of every product)
+constexpr int kModGroup = 4;           // weight rows a warp works on at a time
+constexpr int kModMaxLayers = 8;
+constexpr size_t kModMaxSmem = 200 * 1024;
+
+template <typename T>
+struct ModParams {
+    const int32_t *tokens;
+    const T *hidden0, *emb, *w_proj;
+    float *h_state;
+    const T *g_attn[kModMaxLayers], *w_q[kModMaxLayers], *w_k[kModMaxLayers], *w_v[kModMaxLayers], *w_o[kModMaxLayers];
+    const T *g_mlp[kModMaxLayers], *w_gate[kModMaxLayers], *w_up[kModMaxLayers], *w_down[kModMaxLayers];
+    int first_step, mask_token, emb_rows, n_layers;
+    int n, B, L, d, F, H;
+    float eps;
+    float *z, *q, *k, *v, *act;            // module workspace, [n, d] each, act [n, F]
+    const int32_t *row_index;
+    int M;
+    float *xt_f32;                         // LM-head operand rows h - h_0 of the masked rows: fp32 [M, d], or ...
+    __nv_bfloat16 *xt_bf16;                // ... bf16 hi + lo rows behind the zero rows of step 0
+    int lo_rows;
+    __half *xt16;
+    float *hidden_out;
+    int32_t *status, *user_status;
+    unsigned int *bar;
+};
+
+// Lane-partial products of kModGroup weight rows (nullptr: none), `len` columns each, with `rows` <= kModRows input
+// rows in shared memory (fp32, row pitch `pitch`), then added over the lanes: every lane returns with all the
+// sums.  bf16 rows of a multiple of 256 columns are read 16 bytes per lane.
+template <typename T>
+__device__ __forceinline__ void group_dots(const T *const (&wr)[kModGroup], const float *xs, int rows, int pitch, int len,
+                                           int lane, float (&acc)[kModGroup][kModRows])
+{
+#pragma unroll
+    for (int f = 0; f < kModGroup; ++f)
+#pragma unroll
+        for (int r = 0; r < kModRows; ++r) acc[f][r] = 0.f;
+    if (std::is_same<T, __nv_bfloat16>::value && (len & 255) == 0) {
+#pragma unroll 2
+        for (int c = lane * 8; c < len; c += 256) {
+            uint4 q[kModGroup];
+#pragma unroll
+            for (int f = 0; f < kModGroup; ++f)
+                q[f] = wr[f] ? __ldg(reinterpret_cast<const uint4 *>(reinterpret_cast<const __nv_bfloat16 *>(wr[f]) + c))
+                             : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+            for (int r = 0; r < kModRows; ++r) {
+                if (r < rows) {
+                    const float4 a = *reinterpret_cast<const float4 *>(xs + (size_t)r * pitch + c);
+                    const float4 b = *reinterpret_cast<const float4 *>(xs + (size_t)r * pitch + c + 4);
+#pragma unroll
+                    for (int f = 0; f < kModGroup; ++f) {
+                        float t = acc[f][r];
+                        t = fmaf(__uint_as_float(q[f].x << 16), a.x, t); t = fmaf(__uint_as_float(q[f].x & 0xFFFF0000u), a.y, t);
+                        t = fmaf(__uint_as_float(q[f].y << 16), a.z, t); t = fmaf(__uint_as_float(q[f].y & 0xFFFF0000u), a.w, t);
+                        t = fmaf(__uint_as_float(q[f].z << 16), b.x, t); t = fmaf(__uint_as_float(q[f].z & 0xFFFF0000u), b.y, t);
+                        t = fmaf(__uint_as_float(q[f].w << 16), b.z, t); t = fmaf(__uint_as_float(q[f].w & 0xFFFF0000u), b.w, t);
+                        acc[f][r] = t;
+                    }
+                }
+            }
+        }
+    } else {
+#pragma unroll 4
+        for (int c = lane; c < len; c += 32) {
+            float wv[kModGroup];
+#pragma unroll
+            for (int f = 0; f < kModGroup; ++f) wv[f] = wr[f] ? ld_f(wr[f], c) : 0.f;
+#pragma unroll
+            for (int r = 0; r < kModRows; ++r) {
+                if (r < rows) {
+                    const float x = xs[(size_t)r * pitch + c];
+#pragma unroll
+                    for (int f = 0; f < kModGroup; ++f) acc[f][r] = fmaf(wv[f], x, acc[f][r]);
+                }
+            }
+        }
+    }
+#pragma unroll
+    for (int f = 0; f < kModGroup; ++f)
+#pragma unroll
+        for (int r = 0; r < kModRows; ++r) acc[f][r] = warp_sum(acc[f][r]);
+}
+
+// How the groups of a product are dealt out: the contraction is cut into S pieces (a power of two) when there
+// are fewer groups than warps in the grid, so that all of them stream; the S warps of a group sit in one CTA
+// and their partial sums are added there in a fixed order.
+__device__ __forceinline__ int split_for(int n_groups, int n_in, int n_gw, bool wide)
+{
+    int S = 1;
+    const int unit = wide ? 256 : 32;
+    while (S < kModThreads / 32 && n_groups * (2 * S) <= n_gw && (n_in % (2 * S)) == 0 && ((n_in / (2 * S)) % unit) == 0) S *= 2;
+    return S;
+}
+
+// One product of the step: y(g, f, r) for every group g of kModGroup weight rows (row(g, f): the row, or nullptr)
+// and input row r, handed to epi(g, f, r, value) by one lane each.  xs: the input rows in shared memory (pitch
+// n_in); red: kModThreads / 32 * 16 floats of shared memory.  Every thread of the CTA calls it.
+template <typename T, typename RowFn, typename Epi>
+__device__ __forceinline__ void gemv_phase(RowFn row, Epi epi, const float *xs, int rows, int n_in, int n_groups, int S,
+                                           float *red)
+{
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, n_warps = kModThreads / 32;
+    const int G = gridDim.x, cta = blockIdx.x;
+    const int per_round = n_warps / S, team = warp / S, split = warp % S, chunk = n_in / S;
+    const int rounds = (n_groups + G * per_round - 1) / (G * per_round);
+    for (int rd = 0; rd < rounds; ++rd) {
+        const int g = (rd * G + cta) * per_round + team;
+        const T *wr[kModGroup];
+        float acc[kModGroup][kModRows];
+#pragma unroll
+        for (int f = 0; f < kModGroup; ++f) {
+            const T *w = g < n_groups ? row(g, f) : nullptr;
+            wr[f] = w ? w + (size_t)split * chunk : nullptr;
+        }
+        group_dots<T>(wr, xs + (size_t)split * chunk, rows, n_in, chunk, lane, acc);
+        // lane f * kModRows + r takes sum (f, r)
+        float mine = 0.f;
+#pragma unroll
+        for (int f = 0; f < kModGroup; ++f)
+#pragma unroll
+            for (int r = 0; r < kModRows; ++r)
+                if (lane == f * kModRows + r) mine = acc[f][r];
+        if (S > 1) {
+            if (lane < kModGroup * kModRows) red[warp * 16 + lane] = mine;
+            __syncthreads();
+            if (split == 0 && lane < kModGroup * kModRows) {
+                mine = red[warp * 16 + lane];
+                for (int s2 = 1; s2 < S; ++s2) mine += red[(warp + s2) * 16 + lane];
+            }
+        }
+        if (split == 0 && lane < kModGroup * kModRows && g < n_groups) epi(g, lane / kModRows, lane % kModRows, mine);
+        if (S > 1) __syncthreads();
+    }
+}
+
+// Rows [n, width] of a buffer another phase wrote, into shared memory (through L2).
+__device__ __forceinline__ void stage_rows(float *dst, const float *src, int count)
+{
+    if ((count & 3) == 0) {
+#pragma unroll 8
+        for (int i = threadIdx.x * 4; i < count; i += blockDim.x * 4)
+            *reinterpret_cast<float4 *>(dst + i) = __ldcg(reinterpret_cast<const float4 *>(src + i));
+    } else {
+        for (int i = threadIdx.x; i < count; i += blockDim.x) dst[i] = __ldcg(src + i);
+    }
+}
+
+// RMSNorm of the n rows in shared memory, in place (warp per row).
+template <typename T>
+__device__ __forceinline__ void norm_rows(float *xs, int n, int d, const T *gamma, float eps)
+{
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int r = warp; r < n; r += (int)(blockDim.x >> 5)) {
+        float ss = 0.f;
+        for (int j = lane; j < d; j += 32) ss = fmaf(xs[(size_t)r * d + j], xs[(size_t)r * d + j], ss);
+        ss = warp_sum(ss);
+        const float rstd = rsqrtf(ss / (float)d + eps);
+        for (int j = lane; j < d; j += 32) xs[(size_t)r * d + j] = xs[(size_t)r * d + j] * rstd * ld_f(gamma, j);
+    }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kModThreads)
+module_fused_kernel(const ModParams<T> p)
+{
+    extern __shared__ __align__(16) float sh[];
+    __shared__ float red[kModThreads / 32 * 16];
+    __shared__ int inv[kModRows];            // dense position -> masked row, or -1
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n_warps = kModThreads / 32;
+    const int G = gridDim.x, cta = blockIdx.x;
+    const int gw = cta * n_warps + warp, n_gw = G * n_warps;
+    const int n = p.n, d = p.d, F = p.F, L = p.L;
+    const bool wide = std::is_same<T, __nv_bfloat16>::value;
+    FusedSync sy;
+    sy.base = *reinterpret_cast<volatile unsigned int *>(p.bar + 1);
+    sy.done = 0;
+    sy.total = 5 * p.n_layers + 2;
+    auto leave = [&]() {
+        if (cta == 0 && threadIdx.x == 0) {
+            *reinterpret_cast<volatile unsigned int *>(p.bar + 1) = sy.base + (unsigned int)sy.total * G;
+            __threadfence();
+        }
+    };
+    // the products of the step: groups of kModGroup weight rows and how their contraction is split
+    const int ng_d = (d + kModGroup - 1) / kModGroup, ng_qkv = 3 * d / kModGroup, ng_gu = (F + 1) / 2;
+    const int s_proj = split_for(ng_d, 2 * d, n_gw, wide), s_qkv = split_for(ng_qkv, d, n_gw, wide);
+    const int s_o = split_for(ng_d, d, n_gw, wide), s_gu = split_for(ng_gu, d, n_gw, wide), s_dn = split_for(ng_d, F, n_gw, wide);
+    auto row_proj = [&](int g, int f) { const int j = g * kModGroup + f; return j < d ? p.w_proj + (size_t)j * 2 * d : (const T *)nullptr; };
+    auto rows_of = [&](const T *w, int n_in) {
+        return [=](int g, int f) { const int j = g * kModGroup + f; return j < d ? w + (size_t)j * n_in : (const T *)nullptr; };
+    };
+    auto row_qkv = [&](int l) {
+        const T *wq = p.w_q[l], *wk = p.w_k[l], *wv = p.w_v[l];
+        return [=](int g, int f) {                      // (kModGroup divides d: a group stays within one matrix)
+            const int j = g * kModGroup + f, which = j / d;
+            return (which == 0 ? wq : which == 1 ? wk : wv) + (size_t)(j - which * d) * d;
+        };
+    };
+    auto row_gu = [&](int l) {
+        const T *wg = p.w_gate[l], *wu = p.w_up[l];
+        return [=](int g, int f) {                      // rows 0, 1: gate and up of feature 2 g; rows 2, 3: of feature 2 g + 1
+            const int ft = 2 * g + (f >> 1);
+            return ft < F ? ((f & 1) ? wu : wg) + (size_t)ft * d : (const T *)nullptr;
+        };
+    };
+    auto add_to_z = [&](int g, int f, int r, float v) {
+        const int j = g * kModGroup + f;
+        if (j < d && r < n) { float *dst = p.z + (size_t)r * d + j; *dst = __ldcg(dst) + v; }
+    };
+
+    // ---- z = W_proj [h ; emb[x]] ----
+    for (int i = 0; i < n; ++i) {
+        int tok = p.tokens[i];
+        if (tok >= p.emb_rows || tok < -1) {          // outside the table: reads as masked, raises the bit
+            if (cta == 0 && threadIdx.x == 0) {
+                atomicOr(p.status, MRP_DEV_BAD_INDEX);
+                if (p.user_status) atomicOr(p.user_status, MRP_DEV_BAD_INDEX);
+            }
+            tok = -1;
+        }
+        if (tok < 0) tok = p.mask_token;
+        for (int j = threadIdx.x; j < d; j += blockDim.x) {
+            const float h = p.first_step ? ld_f(p.hidden0, (size_t)i * d + j) : __ldcg(p.h_state + (size_t)i * d + j);
+            if (p.first_step && i % G == cta) p.h_state[(size_t)i * d + j] = h;
+            sh[(size_t)i * 2 * d + j] = h;
+            sh[(size_t)i * 2 * d + d + j] = ld_f(p.emb, (size_t)tok * d + j);
+        }
+    }
+    __syncthreads();
+    gemv_phase<T>(row_proj, [&](int g, int f, int r, float v) {
+        const int j = g * kModGroup + f;
+        if (j < d && r < n) p.z[(size_t)r * d + j] = v;
+    }, sh, n, 2 * d, ng_d, s_proj, red);
+    if (!fused_barrier(p, sy)) { leave(); return; }
+
+    for (int l = 0; l < p.n_layers; ++l) {
+        // ---- q, k, v of RMSNorm(z) g_attn: one product over 3 d output features ----
+        stage_rows(sh, p.z, n * d);
+        __syncthreads();
+        norm_rows<T>(sh, n, d, p.g_attn[l], p.eps);
+        __syncthreads();
+        gemv_phase<T>(row_qkv(l), [&](int g, int f, int r, float v) {
+            const int j = g * kModGroup + f, which = j / d;
+            if (r < n) (which == 0 ? p.q : which == 1 ? p.k : p.v)[(size_t)r * d + (j - which * d)] = v;
+        }, sh, n, d, ng_qkv, s_qkv, red);
+        if (!fused_barrier(p, sy)) { leave(); return; }
+
+        // ---- block-local bidirectional attention: a warp per (position, attention head) ----
+        {
+            const int dh = d / p.H;
+            const float scale = rsqrtf((float)dh);
+            for (int item = gw; item < n * p.H; item += n_gw) {
+                const int i = item / p.H, hd = item - i * p.H, b = i / L;
+                const float *qi = p.q + (size_t)i * d + (size_t)hd * dh;
+                float sc[kModRows], mx = -INFINITY;
+#pragma unroll
+                for (int j = 0; j < kModRows; ++j) {
+                    sc[j] = -INFINITY;
+                    if (j < L) {
+                        const float *kj = p.k + ((size_t)b * L + j) * d + (size_t)hd * dh;
+                        float t = 0.f;
+                        for (int c = lane; c < dh; c += 32) t = fmaf(__ldcg(qi + c), __ldcg(kj + c), t);
+                        sc[j] = warp_sum(t) * scale;
+                        mx = fmaxf(mx, sc[j]);
+                    }
+                }
+                float sum = 0.f;
+#pragma unroll
+                for (int j = 0; j < kModRows; ++j) {
+                    sc[j] = j < L ? expf(sc[j] - mx) : 0.f;
+                    sum += sc[j];
+                }
+                for (int c = lane; c < dh; c += 32) {
+                    float a = 0.f;
+#pragma unroll
+                    for (int j = 0; j < kModRows; ++j)
+                        if (j < L) a = fmaf(sc[j], __ldcg(p.v + ((size_t)b * L + j) * d + (size_t)hd * dh + c), a);
+                    p.act[(size_t)i * d + (size_t)hd * dh + c] = a / sum;       // (the activation buffer is free here)
+                }
+            }
+        }
+        if (!fused_barrier(p, sy)) { leave(); return; }
+
+        // ---- z += W_o o ----
+        stage_rows(sh, p.act, n * d);
+        __syncthreads();
+        gemv_phase<T>(rows_of(p.w_o[l], d), add_to_z, sh, n, d, ng_d, s_o, red);
+        if (!fused_barrier(p, sy)) { leave(); return; }
+
+        // ---- a = silu(W_gate n) * (W_up n), n = RMSNorm(z) g_mlp: two features (four weight rows) per group ----
+        stage_rows(sh, p.z, n * d);
+        __syncthreads();
+        norm_rows<T>(sh, n, d, p.g_mlp[l], p.eps);
+        __syncthreads();
+        {
+            // gate and up of a feature land in neighbouring lanes: lane f * kModRows + r holds row f of the group
+            gemv_phase<T>(row_gu(l), [&](int g, int f, int r, float v) {
+                // (every lane below 16 is here together: the up sum sits kModRows lanes above the gate sum)
+                const float us = __shfl_down_sync(0x0000ffffu, v, kModRows);
+                const int ft = 2 * g + (f >> 1);
+                if (!(f & 1) && ft < F && r < n) p.act[(size_t)r * F + ft] = v / (1.f + expf(-v)) * us;
+            }, sh, n, d, ng_gu, s_gu, red);
+        }
+        if (!fused_barrier(p, sy)) { leave(); return; }
+
+        // ---- z += W_down a ----
+        stage_rows(sh, p.act, n * F);
+        __syncthreads();
+        gemv_phase<T>(rows_of(p.w_down[l], F), add_to_z, sh, n, F, ng_d, s_dn, red);
+        if (!fused_barrier(p, sy)) { leave(); return; }
+    }
+
+    // ---- h <- h + Delta at every position; the LM-head operand h - h_0 of the masked rows ----
+    if (threadIdx.x < kModRows) inv[threadIdx.x] = -1;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int m = 0; m < p.M; ++m) {
+            const int idx = p.row_index ? p.row_index[m] : m;
+            if (row_ok(idx, n)) inv[idx] = m;
+            else if (cta == 0) {
+                atomicOr(p.status, MRP_DEV_BAD_INDEX);
+                if (p.user_status) atomicOr(p.user_status, MRP_DEV_BAD_INDEX);
+            }
+        }
+    }
+    __syncthreads();
+    auto put_operand = [&](int m, int j, float h, float r) {
+        if (p.hidden_out) p.hidden_out[(size_t)m * d + j] = h;
+        if (p.xt_f32) p.xt_f32[(size_t)m * d + j] = r;
+        if (p.xt_bf16) {
+            const __nv_bfloat16 hi = __float2bfloat16_rn(r);
+            p.xt_bf16[(size_t)m * d + j] = __float2bfloat16(0.f);                          // step 0 has no residual
+            p.xt_bf16[((size_t)p.lo_rows + m) * d + j] = __float2bfloat16(0.f);
+            p.xt_bf16[((size_t)p.M + m) * d + j] = hi;
+            p.xt_bf16[((size_t)p.lo_rows + p.M + m) * d + j] = __float2bfloat16_rn(r - __bfloat162float(hi));
+            if (p.xt16) p.xt16[(size_t)m * d + j] = __float2half_rn(r);
+        }
+    };
+    for (int e = cta * kModThreads + threadIdx.x; e < n * d; e += G * kModThreads) {
+        const int i = e / d, j = e - i * d;
+        const float h = __ldcg(p.h_state + e) + __ldcg(p.z + e);
+        p.h_state[e] = h;
+        if (inv[i] >= 0) put_operand(inv[i], j, h, h - ld_f(p.hidden0, (size_t)e));
+    }
+    // rows whose index was out of range read as zeros
+    for (int m = 0; m < p.M; ++m) {
+        const int idx = p.row_index ? p.row_index[m] : m;
+        if (!row_ok(idx, n) || inv[idx] != m)
+            for (int j = cta * kModThreads + threadIdx.x; j < d; j += G * kModThreads) put_operand(m, j, 0.f, 0.f);
+    }
+    fused_barrier(p, sy);
+    leave();
+}
+
+static size_t module_fused_smem(int n, int d, int F)
+{
+    size_t fl = (size_t)n * 2 * d;
+    if ((size_t)n * F > fl) fl = (size_t)n * F;
+    return fl * 4;
+}
+
+// Launches the one-kernel module step if the shape fits it (*launched tells).
+template <typename T>
+static cudaError_t module_fused_t(Ctx *c, const int32_t *tokens, const void *hidden0, float *h_state, const int32_t *row_index,
+                                  int M, int B, int L, bool first_step, const mrp_draft_out &out, cudaStream_t st,
+                                  float *xt_f32, __nv_bfloat16 *xt_bf16, int lo_rows, __half *xt16, bool *launched)
+{
+    *launched = false;
+    const mrp_module_weights &w = c->module;
+    const int d = c->cfg.d, F = c->cfg.d_ff, n = B * L;
+    if (n > kModRows || L > kModRows || w.n_layers > kModMaxLayers || (c->cfg.flags & MRP_FLAG_NO_CHAIN) || (d & 3) || (F & 3) || F < d ||
+        module_fused_smem(n, d, F) > kModMaxSmem)
+        return cudaSuccess;
+    auto kern = module_fused_kernel<T>;
+    static std::atomic<unsigned long long> asked{0}, fits{0};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    const unsigned long long bit = 1ull << (dev & 63);
+    if (!(asked.load() & bit)) {
+        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kModMaxSmem);
+        if (e != cudaSuccess) return e;
+        int per_sm = 0;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kModThreads, kModMaxSmem);
+        if (e != cudaSuccess) return e;
+        if (per_sm >= 1) fits.fetch_or(bit);
+        asked.fetch_or(bit);
+    }
+    if (!(fits.load() & bit)) return cudaSuccess;
+    ModParams<T> p;
+    memset(&p, 0, sizeof(p));
+    p.tokens = tokens; p.hidden0 = (const T *)hidden0; p.emb = (const T *)w.emb; p.w_proj = (const T *)w.w_proj;
+    p.h_state = h_state;
+    for (int l = 0; l < w.n_layers; ++l) {
+        const mrp_module_layer &y = w.layers[l];
+        p.g_attn[l] = (const T *)y.g_attn; p.w_q[l] = (const T *)y.w_q; p.w_k[l] = (const T *)y.w_k; p.w_v[l] = (const T *)y.w_v;
+        p.w_o[l] = (const T *)y.w_o; p.g_mlp[l] = (const T *)y.g_mlp; p.w_gate[l] = (const T *)y.w_gate;
+        p.w_up[l] = (const T *)y.w_up; p.w_down[l] = (const T *)y.w_down;
+    }
+    p.first_step = first_step ? 1 : 0; p.mask_token = w.mask_token; p.emb_rows = w.emb_rows; p.n_layers = w.n_layers;
+    p.n = n; p.B = B; p.L = L; p.d = d; p.F = F; p.H = w.n_attn_heads; p.eps = c->cfg.rms_eps;
+    const size_t cap = (size_t)c->cfg.max_seqs * c->cfg.block_len;
+    char *ws = c->module_ws;
+    auto take = [&](size_t bytes) { char *p0 = ws; ws += align_up(bytes, 256); return (float *)p0; };
+    take(cap * 2 * d * 4);                 // (the concatenated rows of the separate kernels)
+    p.z = take(cap * d * 4);
+    take(cap * d * 4);
+    p.q = take(cap * d * 4); p.k = take(cap * d * 4); p.v = take(cap * d * 4);
+    take(cap * d * 4);
+    p.act = take(cap * F * 4);
+    p.row_index = row_index; p.M = M;
+    p.xt_f32 = xt_f32; p.xt_bf16 = xt_bf16; p.lo_rows = lo_rows; p.xt16 = xt16; p.hidden_out = out.hidden_out;
+    p.status = (int32_t *)(c->ws + c->lay.status); p.user_status = out.status;
+    p.bar = (unsigned int *)(c->ws + c->lay.status) + 16;
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3(c->sm_count);
+    cfg.blockDim = dim3(kModThreads);
+    cfg.dynamicSmemBytes = module_fused_smem(n, d, F);
+    cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeCooperative;
+    at[0].val.cooperative = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    e = note_err(c, cudaLaunchKernelEx(&cfg, kern, p), "one-kernel module step");
+    c->launches++;
+    *launched = true;
+    return e;
+}
+
 size_t module_workspace_bytes(const mrp_config &cfg, int n_layers)
 {
     (void)n_layers;
@@ -1257,6 +1705,22 @@ static cudaError_t module_step_t(Ctx *c, const int32_t *tokens, const void *hidd
         return launch_k(linear_kernel<T>, dim3((n_out + 7) / 8), dim3(256), 0, st, pdl, (const T *)wm, x, n, n_in, n_out, y, acc);
     };
     prof_mark(c, 0, st);
+    {
+        // a handful of positions: the whole module step as one kernel, then the LM-head kernels
+        bool launched = false;
+        TcPlan pl;
+        if (c->use_tc && M > 0) pl = tc_plan(c, M, 1, out, st, false);
+        __nv_bfloat16 *xtb = c->use_tc ? (__nv_bfloat16 *)(c->ws + c->lay.xt) : nullptr;
+        const cudaError_t ef = module_fused_t<T>(c, tokens, hidden0, h_state, row_index, M, B, L, first_step, out, st,
+                                                 c->use_tc ? (float *)nullptr : (float *)(c->ws + c->lay.xt), xtb, c->lo_xt,
+                                                 (c->use_tc && M > 0 && pl.f16_lm) ? (__half *)(c->ws + c->lay.xt16) : (__half *)nullptr,
+                                                 &launched);
+        if (ef != cudaSuccess) return ef;
+        if (launched) {
+            if (M == 0) return cudaSuccess;
+            return c->use_tc ? tc_lm_tail(c, pl, logits0, row_index, M, 1, out, st) : simt_lm_tail(c, logits0, row_index, M, 1, out, st);
+        }
+    }
     cudaError_t e = launch_k(mod_concat_kernel<T>, dim3(n), dim3(256), 0, st, pdl, (const float *)h_state, (const T *)hidden0,
                              first_step ? 1 : 0, tokens, (const T *)w.emb, w.mask_token, w.emb_rows, d, h_state, cat, status,
                              out.status);

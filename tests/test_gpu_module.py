@@ -24,6 +24,11 @@ def upload_module(mw, dtype):
     ("bf16", 0, 256, 512, 4096, 3, 4, 1, 4, 3),                             # the paper's depth; few-row tcgen05 LM head
     ("bf16", 0, 128, 256, 2048, 2, 4, 10, 4, 2),                            # 80 row-steps: row-major LM head, fp16 operand
     ("bf16", 0, 256, 512, 4096, 0, 4, 2, 4, 1),                             # the fusion projection alone
+    # four positions or fewer: the module step is one cooperative kernel
+    ("f32", 0, 64, 96, 512, 2, 4, 1, 4, 3),                                 # fp32 weights, ragged widths
+    ("bf16", binding.MRP_FLAG_FORCE_SIMT, 256, 512, 1024, 2, 2, 1, 3, 2),   # 16-byte weight loads, block of three
+    ("bf16", 0, 256, 512, 4096, 0, 4, 1, 4, 2),                             # no layers
+    ("bf16", binding.MRP_FLAG_NO_CHAIN, 256, 512, 4096, 3, 4, 1, 4, 3),     # the same shape as one kernel per product
 ])
 def test_module_steps_follow_the_oracle_through_direct_decoding(dtype, flags, d, F, V, D, heads, B, L, steps):
     w = synth.make_weights(d, F, V, 1, dtype, 41)
@@ -83,31 +88,33 @@ def test_module_steps_follow_the_oracle_through_direct_decoding(dtype, flags, d,
     binding.mrp_destroy(ctx)
 
 
-def test_module_step_checks_tokens_and_needs_an_attached_module():
+@pytest.mark.parametrize("B,L", [(2, 4), (1, 4)])          # one kernel per product / one kernel for the step
+def test_module_step_checks_tokens_and_needs_an_attached_module(B, L):
     d, F, V = 64, 96, 512
+    n = B * L
     w = synth.make_weights(d, F, V, 1, "f32", 43)
     mw = synth.make_module_weights(d, F, V, 1, 2, "f32", 43, std=0.05)
-    inp = synth.make_inputs(w, 2, 4, 43, 1.0, 3.0)
+    inp = synth.make_inputs(w, B, L, 43, 1.0, 3.0)
     heads_dev, w_lm = harness.upload_weights(w, DEV)
-    ctx = binding.mrp_create(d, F, V, heads_dev, w_lm, max_rows=8, max_seqs=2, block_len=4)
+    ctx = binding.mrp_create(d, F, V, heads_dev, w_lm, max_rows=n, max_seqs=B, block_len=L)
     hid0 = harness.to_device(inp.hidden, "f32", DEV)
     l0 = torch.from_numpy(inp.logits0).to(DEV)
-    h_state = torch.empty((8, d), device=DEV)
-    out = harness.alloc_draft_out(8, 1, V, d, DEV)
-    tok = torch.full((8,), -1, device=DEV, dtype=torch.int32)
+    h_state = torch.empty((n, d), device=DEV)
+    out = harness.alloc_draft_out(n, 1, V, d, DEV)
+    tok = torch.full((n,), -1, device=DEV, dtype=torch.int32)
     with pytest.raises(binding.MrpError) as ei:
-        binding.mrp_module_step(ctx, tok, hid0, h_state, l0, None, 8, 2, 4, True, out.conf, out.lse, out.token)
+        binding.mrp_module_step(ctx, tok, hid0, h_state, l0, None, n, B, L, True, out.conf, out.lse, out.token)
     assert ei.value.status == 2
     emb, w_proj, layers = upload_module(mw, "f32")
     binding.mrp_module_attach(ctx, emb, w_proj, layers, 2, mw.mask_token)
     # a token id outside the embedding table is read as masked and raises the bit
     bad = tok.clone()
     bad[3] = V + 5
-    binding.mrp_module_step(ctx, bad, hid0, h_state, l0, None, 8, 2, 4, True, out.conf, out.lse, out.token, status=out.status)
+    binding.mrp_module_step(ctx, bad, hid0, h_state, l0, None, n, B, L, True, out.conf, out.lse, out.token, status=out.status)
     torch.cuda.synchronize()
     assert int(out.status.item()) == binding.MRP_DEV_BAD_INDEX
-    ref = harness.alloc_draft_out(8, 1, V, d, DEV)
-    binding.mrp_module_step(ctx, tok, hid0, h_state, l0, None, 8, 2, 4, True, ref.conf, ref.lse, ref.token, status=ref.status)
+    ref = harness.alloc_draft_out(n, 1, V, d, DEV)
+    binding.mrp_module_step(ctx, tok, hid0, h_state, l0, None, n, B, L, True, ref.conf, ref.lse, ref.token, status=ref.status)
     torch.cuda.synchronize()
     assert int(ref.status.item()) == 0 and torch.equal(ref.conf, out.conf) and torch.equal(ref.token, out.token)
     binding.mrp_destroy(ctx)
