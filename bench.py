@@ -634,43 +634,49 @@ class Bench:
                 "steps": n_e2e, "ms_per_step": dt / n_e2e * 1e3, "mode": e2e_mode}
 
 
-def run_module_workload(bench, cpu_budget_s):
-    """The token-conditioned module at the decode shape (configuration 1's d, V, block): a step is the K = 3
-    MRP steps that follow one backbone forward in direct decoding (Algorithm 2), each = mrp_module_step
-    (module forward + one LM-head pass) + mrp_reveal_remask + mrp_commit, the reveals of a step
-    conditioning the next.  Drafted tokens per step: K (one reveal per MRP step)."""
+def run_module_workload(bench, cpu_budget_s, which=1):
+    """The token-conditioned module at the shape of configuration `which` (1: the decode shape, one block of 4
+    positions; 2: 32 blocks of 4, d = 4096): a step is the K = 3 MRP steps that follow one backbone forward in
+    direct decoding (Algorithm 2), each = mrp_module_step (module forward + one LM-head pass) +
+    mrp_reveal_remask + mrp_commit, the reveals of a step conditioning the next.  Drafted tokens per step:
+    K * B (one reveal per block and MRP step)."""
     import numpy as np
     import torch
     import oracle
     from paper_2605_18817_b200 import binding, harness, synth
     args, dev, dist = bench.args, bench.dev, bench.dist
-    cfg = dict(synth.CONFIGS[1], name="module_decode_1p7b")
-    w, heads, w_lm = bench.weights_for(synth.CONFIGS[1], "1")
-    _, inp = synth.make_config(synth.CONFIGS[1], w)
+    base = synth.CONFIGS[which]
+    cfg = dict(base, name="module_" + base["name"])
+    w, heads, w_lm = bench.weights_for(base, str(which))
+    big = base["d"] >= 4096
+    _, inp = synth.make_config(base, w, logits_fn=harness.device_logits_fn(w_lm) if big else None)
     K, B, L, d, V, F = cfg["K"], cfg["B"], cfg["L"], cfg["d"], cfg["V"], cfg["F"]
     n = B * L
-    mw = synth.make_module_weights(d, F, V, MODULE_LAYERS, MODULE_ATTN_HEADS, "bf16", 11, std=0.02)
+    n_attn = d // 128                                  # 128 features per attention head
+    # (layer weights scaled so that the residual stays inside the accuracy range of the tensor-core LM head:
+    # d * rms(h - h_0) <= MRP_RANGE_LIMIT, checked by the device status word below)
+    mw = synth.make_module_weights(d, F, V, MODULE_LAYERS, n_attn, "bf16", 11, std=0.02 if d < 4096 else 0.01)
     ctx = binding.mrp_create(d, F, V, heads[:1], w_lm, max_rows=n, max_seqs=B, block_len=L, flags=args.flags)
     up = lambda a: harness.to_device(a, "bf16", dev)
     binding.mrp_module_attach(ctx, up(mw.emb), up(mw.w_proj), [{k: up(v) for k, v in lay.items()} for lay in mw.layers],
-                              MODULE_ATTN_HEADS, mw.mask_token)
+                              n_attn, mw.mask_token)
     hid0 = harness.to_device(inp.hidden, "bf16", dev)
     l0 = torch.from_numpy(inp.logits0).to(dev)
     h_state = torch.empty((n, d), device=dev)
     # block state after the backbone's own reveal of one token (position 0 here: any would do for timing)
     tokens0 = np.full(n, -1, np.int32)
-    tokens0[0] = 17
+    tokens0[::L] = 17
     state = harness.alloc_block_state(B, L, dev)
     tok_init = torch.from_numpy(tokens0).to(dev)
     out = harness.alloc_draft_out(n, 1, V, d, dev, margin=False)
     sel = harness.alloc_select_out(B, L, 0, dev)
     launches = [0]
     conf_flat, token_flat = out.conf.view(-1), out.token.view(-1)
+    ri = torch.from_numpy(np.flatnonzero(tokens0 < 0).astype(np.int32)).to(dev)
 
     def step():
         state.tokens.copy_(tok_init)
-        m = n - 1                                   # rows still masked: one fewer after every MRP step
-        ri = torch.arange(1, n, device=dev, dtype=torch.int32)
+        m = n - B                                   # rows still masked: one fewer per block after every MRP step
         cnt = 1                                     # the tensor fill above
         for k in range(K):
             rows = ri[:m] if k == 0 else state.row_index[:m]
@@ -682,12 +688,12 @@ def run_module_workload(bench, cpu_budget_s):
             cnt += ctx.last_launch_count
             harness.commit(ctx, sel, state, B, L, 0)
             cnt += ctx.last_launch_count
-            m -= 1
+            m -= B
         launches[0] = cnt
 
     step()
     torch.cuda.synchronize()
-    res = bench.time_step(step, K, launches, ctx, cfg, n - 1)
+    res = bench.time_step(step, K * B, launches, ctx, cfg, n - B)
     res.pop("steps_per_batch")
     # roofline of the dominant kernel: the LM-head kernel, launched once per MRP step (K weight streams)
     binding.mrp_profile_enable(ctx, True)
@@ -697,13 +703,15 @@ def run_module_workload(bench, cpu_budget_s):
     (ms_mod, ms_lm, ms_comb), n_calls = binding.mrp_profile_read(ctx)
     binding.mrp_profile_enable(ctx, False)
     one = dict(cfg, K=1)
-    roofline = lm_head_roofline(one, n - 2, ms_lm / max(n_calls, 1), bench.peaks, bench.peaks_kind)
+    roofline = lm_head_roofline(one, n - 2 * B, ms_lm / max(n_calls, 1), bench.peaks, bench.peaks_kind)
     roofline["kernel"] = "fused LM head, one launch per MRP step (K = %d weight streams per backbone forward)" % K
     roofline["units_per_launch"] = 1
     res["roofline"] = roofline
     res["phases"] = {"module_ms_per_mrp_step": ms_mod / max(n_calls, 1), "lm_head_ms_per_mrp_step": ms_lm / max(n_calls, 1),
                      "combine_ms_per_mrp_step": ms_comb / max(n_calls, 1), "family": ctx.family,
-                     "module": "D = %d layers, %d attention heads, CUDA-core kernels" % (MODULE_LAYERS, MODULE_ATTN_HEADS)}
+                     "module": "D = %d layers, %d attention heads, %s" % (
+                         MODULE_LAYERS, n_attn, "one CUDA-core kernel per step" if n <= 4 else
+                         "products on the row-major tcgen05 kernel")}
     # end to end with host buffers: hidden states, base logits and the block's tokens in, the block state out
     e2e = None
     if not args.no_e2e:
@@ -726,22 +734,26 @@ def run_module_workload(bench, cpu_budget_s):
             e2e_step()
         bench.barrier()
         dt = time.perf_counter() - t0
-        v, dt = replica_throughput(dist, dev, K * n_e2e, dt)
+        v, dt = replica_throughput(dist, dev, K * B * n_e2e, dt)
         e2e = {"value": v, "unit": UNIT, "h2d_bytes_per_step": h_hid.numel() * 2 + h_l0.numel() * 4 + h_tok.numel() * 4,
                "d2h_bytes_per_step": h_out.numel() * 4, "steps": n_e2e, "ms_per_step": dt / n_e2e * 1e3, "mode": "eager calls"}
     res["e2e"] = e2e
     cpu = None
     if bench.rank == 0 and bench.world == 1 and not args.no_cpu_baseline:
-        ri = np.arange(1, n, dtype=np.int32)
+        # a bounded sample: the first blocks only (blocks are independent), one application when the shape is large
+        Bs = B if not big else 2
+        ns = Bs * L
+        ri_h = np.flatnonzero(tokens0[:ns] < 0).astype(np.int32)
+        Ks = K if not big else 1
         t0 = time.perf_counter()
         reps = 0
         while time.perf_counter() - t0 < min(cpu_budget_s, 6.0) or reps == 0:
-            for k in range(K):
-                oracle.module(inp.hidden, tokens0, B, L, mw.emb, mw.w_proj, mw.layers, w.w_lm, MODULE_ATTN_HEADS,
-                              mw.mask_token, row_index=ri[:n - 1 - k])
+            for k in range(Ks):
+                oracle.module(inp.hidden[:ns], tokens0[:ns], Bs, L, mw.emb, mw.w_proj, mw.layers, w.w_lm, n_attn,
+                              mw.mask_token, row_index=ri_h[:len(ri_h) - Bs * k])
             reps += 1
-        cpu = {"value": K * reps / (time.perf_counter() - t0), "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
-               "sample": "the module oracle, K = %d applications on the whole block, %d repetitions" % (K, reps)}
+        cpu = {"value": Ks * Bs * reps / (time.perf_counter() - t0), "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+               "sample": "the module oracle, %d application(s) on %d of %d blocks, %d repetitions" % (Ks, Bs, B, reps)}
     res["cpu_baseline"] = cpu
     res["device_status_word"] = binding.mrp_fetch_status(ctx)
     binding.mrp_destroy(ctx)
@@ -782,8 +794,8 @@ def main():
     head_name = HEADLINE if args.config == "all" else args.config
     results = {}
     for name in names:
-        if name == "module":
-            results[name] = run_module_workload(bench, 5.0)
+        if name in ("module", "module:1", "module:2"):
+            results[name] = run_module_workload(bench, 5.0, 2 if name == "module:2" else 1)
         else:
             results[name] = bench.run_workload(name, 12.0 if name == head_name else 5.0)
     if bench.rank == 0:

@@ -261,8 +261,9 @@ int mrp_draft_kl(mrp_ctx *ctx, const void *hidden, const float *logits0, const f
  * head above, this module reads the embeddings of the tokens revealed so far, so step k + 1 depends on
  * the reveals of step k and the LM head runs once per step.
  * The paper fixes the parts and leaves the details open; the form implemented (first slice: CUDA-core
- * kernels for the module itself -- one cooperative kernel for the whole step when B * L <= 4, one kernel per
- * matrix product above that -- and the context's own LM-head kernels behind it):
+ * kernels for the module itself -- one cooperative kernel for the whole step when B * L <= 4; above that one
+ * kernel per matrix product, on the tensor cores for tensor-core contexts whose module matrices are 16-byte
+ * aligned -- and the context's own LM-head kernels behind it):
  *     e_i = emb[x_i]  (emb[mask_token] where x_i = -1);   z_i = W_proj [h_i ; e_i]
  *     n_layers times:  z += W_o Attn(RMSNorm(z) g_attn),  attention over the positions of the same block,
  *                      bidirectional, n_attn_heads heads, no positional term;

@@ -1679,6 +1679,133 @@ static cudaError_t module_fused_t(Ctx *c, const int32_t *tokens, const void *hid
     return e;
 }
 
+// ---- the module's products on the tensor cores (more than a handful of positions) ----------------------
+// The matrix products of the step run on the row-major tcgen05 kernel (tc_linear / tc_gate_up: bf16 hi + lo
+// operand rows, fp32 accumulation, RMSNorm folded in as gamma on the operand and 1 / rms on the result); what is
+// between them (embedding fusion, operand splitting, attention, the residual sums) stays on the CUDA cores.
+// bf16 hi + lo rows of [h_i ; emb[x_i]]: the hi rows [n, 2 d], the lo rows n rows further on.
+__global__ void mod_cat_split_kernel(const float *h_state, const __nv_bfloat16 *__restrict__ hidden0, int first_step,
+                                     const int32_t *__restrict__ tokens, const __nv_bfloat16 *__restrict__ emb, int mask_token,
+                                     int emb_rows, int n, int d, float *h_out /* = h_state */, __nv_bfloat16 *__restrict__ cat,
+                                     int32_t *__restrict__ status, int32_t *__restrict__ user_status)
+{
+    pdl_trigger();
+    pdl_wait();
+    const int i = blockIdx.x;
+    int tok = tokens[i];
+    if (tok >= emb_rows || tok < -1) {
+        if (threadIdx.x == 0) {
+            atomicOr(status, MRP_DEV_BAD_INDEX);
+            if (user_status) atomicOr(user_status, MRP_DEV_BAD_INDEX);
+        }
+        tok = -1;
+    }
+    if (tok < 0) tok = mask_token;
+    __nv_bfloat16 *hi = cat + (size_t)i * 2 * d, *lo = cat + ((size_t)n + i) * 2 * d;
+    for (int j = threadIdx.x; j < d; j += blockDim.x) {
+        const float h = first_step ? __bfloat162float(hidden0[(size_t)i * d + j]) : h_state[(size_t)i * d + j];
+        if (first_step) h_out[(size_t)i * d + j] = h;
+        const __nv_bfloat16 hh = __float2bfloat16_rn(h);
+        hi[j] = hh;
+        lo[j] = __float2bfloat16_rn(h - __bfloat162float(hh));
+        hi[d + j] = emb[(size_t)tok * d + j];            // a bf16 value: no remainder
+        lo[d + j] = __float2bfloat16(0.f);
+    }
+}
+
+// bf16 hi + lo rows of x[i, :] * gamma (gamma == nullptr: of x itself), and the row's sum of squares of x.
+__global__ void mod_split_kernel(const float *__restrict__ x, const __nv_bfloat16 *__restrict__ gamma, int n, int width,
+                                 __nv_bfloat16 *__restrict__ out, float *__restrict__ sumsq)
+{
+    pdl_trigger();
+    pdl_wait();
+    __shared__ float red[32];
+    const int i = blockIdx.x;
+    __nv_bfloat16 *hi = out + (size_t)i * width, *lo = out + ((size_t)n + i) * width;
+    float ss = 0.f;
+    for (int j = threadIdx.x; j < width; j += blockDim.x) {
+        const float v = x[(size_t)i * width + j];
+        ss = fmaf(v, v, ss);
+        const float y = gamma ? v * __bfloat162float(gamma[j]) : v;
+        const __nv_bfloat16 hh = __float2bfloat16_rn(y);
+        hi[j] = hh;
+        lo[j] = __float2bfloat16_rn(y - __bfloat162float(hh));
+    }
+    if (!sumsq) return;
+    ss = warp_sum(ss);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float t = 0.f;
+        for (int w = 0; w < (int)(blockDim.x >> 5); ++w) t += red[w];
+        sumsq[i] = t;
+    }
+}
+
+// Whether the module's products of a call over n positions can run on the tensor cores.
+static bool module_tc_ok(const Ctx *c, int n)
+{
+    if (!c->use_tc || c->cfg.dtype != MRP_BF16 || (c->cfg.flags & MRP_FLAG_FORCE_SIMT)) return false;
+    if (c->cfg.d % 64 || c->cfg.d_ff % 64 || n > c->cfg.max_rows * kSumsqSlices) return false;
+    const mrp_module_weights &w = c->module;
+    auto al = [](const void *p) { return ((uintptr_t)p & 15u) == 0; };
+    if (!al(w.emb) || !al(w.w_proj)) return false;
+    for (int l = 0; l < w.n_layers; ++l) {
+        const mrp_module_layer &y = w.layers[l];
+        if (!al(y.w_q) || !al(y.w_k) || !al(y.w_v) || !al(y.w_o) || !al(y.w_gate) || !al(y.w_up) || !al(y.w_down)) return false;
+    }
+    return true;
+}
+
+// The module itself (everything in front of `h <- h + Delta`) with its products on the tensor cores.
+static cudaError_t module_body_tc(Ctx *c, const int32_t *tokens, const void *hidden0, float *h_state, int B, int L,
+                                  bool first_step, const mrp_draft_out &out, cudaStream_t st, float *z)
+{
+    const mrp_module_weights &w = c->module;
+    const int d = c->cfg.d, F = c->cfg.d_ff, n = B * L, dh = d / w.n_attn_heads;
+    const size_t cap = (size_t)c->cfg.max_seqs * c->cfg.block_len;
+    char *ws = c->module_ws;
+    auto take = [&](size_t bytes) { char *p0 = ws; ws += align_up(bytes, 256); return p0; };
+    // the regions of the fp32 path hold the bf16 hi + lo operands here (same bytes: two halves of two bytes)
+    __nv_bfloat16 *cat16 = (__nv_bfloat16 *)take(cap * 2 * d * 4);
+    float *zz = (float *)take(cap * d * 4);
+    __nv_bfloat16 *x16 = (__nv_bfloat16 *)take(cap * d * 4);
+    float *q = (float *)take(cap * d * 4), *k = (float *)take(cap * d * 4), *v = (float *)take(cap * d * 4);
+    float *o = (float *)take(cap * d * 4);
+    __nv_bfloat16 *act16 = (__nv_bfloat16 *)take(cap * F * 4);
+    (void)zz;
+    float *sumsq = (float *)(c->ws + c->lay.sumsq);
+    int32_t *status = (int32_t *)(c->ws + c->lay.status);
+    const bool pdl = !(c->cfg.flags & MRP_FLAG_NO_PDL);
+    cudaError_t e = launch_k(mod_cat_split_kernel, dim3(n), dim3(256), 0, st, pdl, (const float *)h_state,
+                             (const __nv_bfloat16 *)hidden0, first_step ? 1 : 0, tokens, (const __nv_bfloat16 *)w.emb, w.mask_token,
+                             w.emb_rows, n, d, h_state, cat16, status, out.status);
+    c->launches++;
+    if (e == cudaSuccess) e = tc_linear(c, cat16, n, 2 * d, w.w_proj, d, nullptr, z, false, out.status, st);
+    auto split = [&](const float *x, const void *gamma, int width, __nv_bfloat16 *dst, float *ss) {
+        c->launches++;
+        return launch_k(mod_split_kernel, dim3(n), dim3(256), 0, st, pdl, x, (const __nv_bfloat16 *)gamma, n, width, dst, ss);
+    };
+    for (int l = 0; l < w.n_layers && e == cudaSuccess; ++l) {
+        const mrp_module_layer &y = w.layers[l];
+        e = split(z, y.g_attn, d, x16, sumsq);
+        if (e == cudaSuccess) e = tc_linear(c, x16, n, d, y.w_q, d, sumsq, q, false, out.status, st);
+        if (e == cudaSuccess) e = tc_linear(c, x16, n, d, y.w_k, d, sumsq, k, false, out.status, st);
+        if (e == cudaSuccess) e = tc_linear(c, x16, n, d, y.w_v, d, sumsq, v, false, out.status, st);
+        if (e == cudaSuccess) {
+            e = launch_k(mod_attention_kernel, dim3(B, w.n_attn_heads), dim3(128), (size_t)4 * L * 4, st, pdl, (const float *)q,
+                         (const float *)k, (const float *)v, L, d, dh, o);
+            c->launches++;
+        }
+        if (e == cudaSuccess) e = split(o, nullptr, d, x16, nullptr);
+        if (e == cudaSuccess) e = tc_linear(c, x16, n, d, y.w_o, d, nullptr, z, true, out.status, st);
+        if (e == cudaSuccess) e = split(z, y.g_mlp, d, x16, sumsq);
+        if (e == cudaSuccess) e = tc_gate_up(c, x16, n, d, y.w_gate, y.w_up, F, sumsq, act16, out.status, st);
+        if (e == cudaSuccess) e = tc_linear(c, act16, n, F, y.w_down, d, nullptr, z, true, out.status, st);
+    }
+    return e;
+}
+
 size_t module_workspace_bytes(const mrp_config &cfg, int n_layers)
 {
     (void)n_layers;
@@ -1721,12 +1848,17 @@ static cudaError_t module_step_t(Ctx *c, const int32_t *tokens, const void *hidd
             return c->use_tc ? tc_lm_tail(c, pl, logits0, row_index, M, 1, out, st) : simt_lm_tail(c, logits0, row_index, M, 1, out, st);
         }
     }
-    cudaError_t e = launch_k(mod_concat_kernel<T>, dim3(n), dim3(256), 0, st, pdl, (const float *)h_state, (const T *)hidden0,
-                             first_step ? 1 : 0, tokens, (const T *)w.emb, w.mask_token, w.emb_rows, d, h_state, cat, status,
-                             out.status);
-    c->launches++;
-    if (e == cudaSuccess) e = lin(w.w_proj, cat, 2 * d, d, z, 0);
-    for (int l = 0; l < w.n_layers && e == cudaSuccess; ++l) {
+    const bool on_tc = module_tc_ok(c, n);
+    cudaError_t e = cudaSuccess;
+    if (on_tc) {
+        e = module_body_tc(c, tokens, hidden0, h_state, B, L, first_step, out, st, z);
+    } else {
+        e = launch_k(mod_concat_kernel<T>, dim3(n), dim3(256), 0, st, pdl, (const float *)h_state, (const T *)hidden0,
+                     first_step ? 1 : 0, tokens, (const T *)w.emb, w.mask_token, w.emb_rows, d, h_state, cat, status, out.status);
+        c->launches++;
+        if (e == cudaSuccess) e = lin(w.w_proj, cat, 2 * d, d, z, 0);
+    }
+    for (int l = 0; l < (on_tc ? 0 : w.n_layers) && e == cudaSuccess; ++l) {
         const mrp_module_layer &y = w.layers[l];
         e = launch_k(rmsnorm_kernel<T>, dim3(n), dim3(256), 0, st, pdl, (const float *)z, (const T *)y.g_attn, d, c->cfg.rms_eps, nn);
         c->launches++;

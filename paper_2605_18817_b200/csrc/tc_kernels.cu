@@ -34,7 +34,7 @@ constexpr int kThreads = 192;
 constexpr int kATile = 128 * 128;          // bytes of a 128-row A tile
 constexpr int kAccCols = 256;              // TMEM columns per accumulator buffer (two buffers)
 
-enum { KIND_GU = 0, KIND_DN = 1, KIND_LM = 2 };
+enum { KIND_GU = 0, KIND_DN = 1, KIND_LM = 2, KIND_LIN = 3 };
 
 struct TcParams {
     // decomposition of the weight rows (MMA N)
@@ -78,6 +78,10 @@ struct TcParams {
     __half *xt16_k;      // optional: the same rows rounded once to fp16
     float *sumsq_out;
     float *hidden_out;
+    // LIN: a plain product, out[row, j] (+)= rstd(row) * acc (rstd from `sumsq` as in GU, 1 without it)
+    float *lin_out;
+    int lin_n_out;
+    int lin_accumulate;
     int32_t *status;
     int32_t *user_status;
 };
@@ -310,7 +314,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         tp = p.teacher + ((size_t)(k_of_row - 1) * p.M + m_of_row) * (size_t)p.V;   // step_base is 1 here
                     }
                 }
-            } else if (KIND == KIND_GU && valid) {
+            } else if ((KIND == KIND_GU || (KIND == KIND_LIN && p.sumsq)) && valid) {
                 float s = 0.f;
                 for (int i = 0; i < p.n_ss; ++i) s += p.sumsq[(size_t)i * p.M + m_of_row];
                 rstd = rsqrtf(s / (float)p.d + p.eps);
@@ -366,6 +370,26 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                                 av[j] = gj / (1.f + __expf(-gj)) * (u[j] * rstd);
                             }
                             store_split<8>(p.act + (size_t)m_of_row * p.F + f_tile + c * 8, (size_t)p.M * p.F, av);
+                        }
+                    }
+                } else if (KIND == KIND_LIN) {
+                    const int j_tile = ut * 16;
+                    for (int c = 0; c < units_here; ++c) {
+                        float a[16];
+                        tmem_ld16(tacc + c * 16, a);
+                        if (valid) {
+                            const size_t o = (size_t)m_of_row * p.lin_n_out + j_tile + c * 16;
+                            if (p.sumsq) {
+#pragma unroll
+                                for (int j = 0; j < 16; ++j) a[j] *= rstd;
+                            }
+                            if (p.lin_accumulate) {
+                                float z[16];
+                                load16_rw(p.lin_out + o, z);
+#pragma unroll
+                                for (int j = 0; j < 16; ++j) a[j] += z[j];
+                            }
+                            store16(p.lin_out + o, a);
                         }
                     }
                 } else {
@@ -825,6 +849,54 @@ cudaError_t tc_lm_tail(Ctx *c, const TcPlan &pl, const float *logits0, const int
     ft.x = xt; ft.x_bf16 = 1; ft.lo_rows = c->lo_xt; ft.M = M; ft.K = K; ft.d = d; ft.V = V;
     return launch_first_token_prob(c, ft, out, st);
 }
+// out[n, n_out] (+)= rstd(row) * (A W^T): A = bf16 hi rows [n, n_in] with the lo rows n rows further on, W bf16
+// [n_out, n_in]; rstd(row) = rsqrt(sumsq[row] / n_in + eps) where sumsq is given, else 1.  n_in % 64 == 0,
+// n_out % 16 == 0, 16-byte aligned pointers.
+cudaError_t tc_linear(Ctx *c, const __nv_bfloat16 *a, int n, int n_in, const void *w, int n_out, const float *sumsq,
+                      float *out, bool accumulate, int32_t *user_status, cudaStream_t st)
+{
+    const TcState *s = (const TcState *)c->tc_state;
+    const int G = c->sm_count, n_mb = (n + 127) / 128;
+    CUtensorMap mA, mB;
+    TcParams p;
+    memset(&p, 0, sizeof(p));
+    p.units_total = n_out / 16; p.unit_rows = 16; p.n_boxes = 1; p.k_chunks = n_in / kBK;
+    p.n_groups = choose_groups(n_mb, p.units_total, G); p.n_rb = n_mb; p.rows = n; p.a_row_base = 0; p.a_part_rows = n;
+    p.M = n; p.d = n_in; p.sumsq = sumsq; p.n_ss = 1; p.eps = c->cfg.rms_eps;
+    p.lin_out = out; p.lin_n_out = n_out; p.lin_accumulate = accumulate ? 1 : 0;
+    p.status = (int32_t *)(c->ws + c->lay.status); p.user_status = user_status;
+    finish_shape(p, G / p.n_groups);
+    if (!make_map(s, &mA, a, n_in, 2 * (uint64_t)n, 128) || !make_map(s, &mB, w, n_in, n_out, p.bn))
+        return note_err(c, cudaErrorInvalidValue, "tensor map (module product)");
+    c->launches++;
+    return note_err(c, launch_tc<KIND_LIN, false>(mA, mB, mB, p, p.n_groups * p.n_vr, st, !(c->cfg.flags & MRP_FLAG_NO_PDL)),
+                    "module product kernel");
+}
+
+// act[n, F] (bf16 hi rows, lo rows n * F elements further on) = silu(rstd * A Wg^T) * (rstd * A Wu^T): the head
+// chain's gate/up kernel on other operands.
+cudaError_t tc_gate_up(Ctx *c, const __nv_bfloat16 *a, int n, int n_in, const void *w_gate, const void *w_up, int F,
+                       const float *sumsq, __nv_bfloat16 *act, int32_t *user_status, cudaStream_t st)
+{
+    const TcState *s = (const TcState *)c->tc_state;
+    const int G = c->sm_count, n_mb = (n + 127) / 128;
+    CUtensorMap mA, mB0, mB1;
+    TcParams p;
+    memset(&p, 0, sizeof(p));
+    p.units_total = F / 8; p.unit_rows = 8; p.n_boxes = 2; p.k_chunks = n_in / kBK;
+    p.n_groups = choose_groups(n_mb, p.units_total, G); p.n_rb = n_mb; p.rows = n; p.a_row_base = 0; p.a_part_rows = n;
+    p.M = n; p.d = n_in; p.F = F;
+    p.sumsq = sumsq; p.n_ss = 1; p.eps = c->cfg.rms_eps; p.act = act;
+    p.status = (int32_t *)(c->ws + c->lay.status); p.user_status = user_status;
+    finish_shape(p, G / p.n_groups);
+    if (!make_map(s, &mA, a, n_in, 2 * (uint64_t)n, 128) || !make_map(s, &mB0, w_gate, n_in, F, p.bn / 2) ||
+        !make_map(s, &mB1, w_up, n_in, F, p.bn / 2))
+        return note_err(c, cudaErrorInvalidValue, "tensor map (module gate/up)");
+    c->launches++;
+    return note_err(c, launch_tc<KIND_GU, false>(mA, mB0, mB1, p, p.n_groups * p.n_vr, st, !(c->cfg.flags & MRP_FLAG_NO_PDL)),
+                    "module gate/up kernel");
+}
+
 cudaError_t tc_draft(Ctx *c, const void *hidden, const float *logits0, const int32_t *row_index, int M,
                      int K, const mrp_draft_out &out, cudaStream_t st)
 {
