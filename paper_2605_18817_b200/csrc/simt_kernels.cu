@@ -1160,16 +1160,29 @@ __global__ void mod_attention_kernel(const float *__restrict__ q, const float *_
     for (int i = warp; i < L; i += n_warps) {
         const float *qi = q + ((size_t)b * L + i) * d + (size_t)hd * dh;
         float mx = -INFINITY;
-        for (int j = lane; j < L; j += 32) {
-            const float *kj = k + ((size_t)b * L + j) * d + (size_t)hd * dh;
-            float sdot = 0.f;
-            for (int c = 0; c < dh; ++c) sdot = fmaf(qi[c], kj[c], sdot);
-            sdot *= scale;
-            p[j] = sdot;
-            mx = fmaxf(mx, sdot);
-        }
+        if (L < 32) {
+            // short blocks: lanes over the head's features (coalesced rows), one warp sum per key
+            for (int j = 0; j < L; ++j) {
+                const float *kj = k + ((size_t)b * L + j) * d + (size_t)hd * dh;
+                float sdot = 0.f;
+                for (int c = lane; c < dh; c += 32) sdot = fmaf(qi[c], kj[c], sdot);
+                sdot = warp_sum(sdot) * scale;
+                if (lane == 0) p[j] = sdot;
+                mx = fmaxf(mx, sdot);
+            }
+        } else {
+            for (int j = lane; j < L; j += 32) {
+                const float *kj = k + ((size_t)b * L + j) * d + (size_t)hd * dh;
+                float sdot = 0.f;
+                for (int c = 0; c < dh; ++c) sdot = fmaf(qi[c], kj[c], sdot);
+                sdot *= scale;
+                p[j] = sdot;
+                mx = fmaxf(mx, sdot);
+            }
 #pragma unroll
-        for (int w = 16; w > 0; w >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, w));
+            for (int w = 16; w > 0; w >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, w));
+        }
+        __syncwarp();
         float sum = 0.f;
         for (int j = lane; j < L; j += 32) {
             const float e = expf(p[j] - mx);
@@ -1723,13 +1736,35 @@ __global__ void mod_split_kernel(const float *__restrict__ x, const __nv_bfloat1
     const int i = blockIdx.x;
     __nv_bfloat16 *hi = out + (size_t)i * width, *lo = out + ((size_t)n + i) * width;
     float ss = 0.f;
-    for (int j = threadIdx.x; j < width; j += blockDim.x) {
-        const float v = x[(size_t)i * width + j];
-        ss = fmaf(v, v, ss);
-        const float y = gamma ? v * __bfloat162float(gamma[j]) : v;
-        const __nv_bfloat16 hh = __float2bfloat16_rn(y);
-        hi[j] = hh;
-        lo[j] = __float2bfloat16_rn(y - __bfloat162float(hh));
+    if ((width & 7) == 0) {
+        // eight elements per thread: 32-byte reads, 16-byte writes of each half
+        for (int j = threadIdx.x * 8; j < width; j += blockDim.x * 8) {
+            const float4 a = *reinterpret_cast<const float4 *>(x + (size_t)i * width + j);
+            const float4 b = *reinterpret_cast<const float4 *>(x + (size_t)i * width + j + 4);
+            const float v[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+            __nv_bfloat162 h2[4], l2[4];
+#pragma unroll
+            for (int e = 0; e < 8; e += 2) {
+                ss = fmaf(v[e], v[e], fmaf(v[e + 1], v[e + 1], ss));
+                const float y0 = gamma ? v[e] * __bfloat162float(gamma[j + e]) : v[e];
+                const float y1 = gamma ? v[e + 1] * __bfloat162float(gamma[j + e + 1]) : v[e + 1];
+                const __nv_bfloat16 h0 = __float2bfloat16_rn(y0), h1 = __float2bfloat16_rn(y1);
+                h2[e >> 1] = __halves2bfloat162(h0, h1);
+                l2[e >> 1] = __halves2bfloat162(__float2bfloat16_rn(y0 - __bfloat162float(h0)),
+                                                __float2bfloat16_rn(y1 - __bfloat162float(h1)));
+            }
+            *reinterpret_cast<uint4 *>(hi + j) = *reinterpret_cast<const uint4 *>(h2);
+            *reinterpret_cast<uint4 *>(lo + j) = *reinterpret_cast<const uint4 *>(l2);
+        }
+    } else {
+        for (int j = threadIdx.x; j < width; j += blockDim.x) {
+            const float v = x[(size_t)i * width + j];
+            ss = fmaf(v, v, ss);
+            const float y = gamma ? v * __bfloat162float(gamma[j]) : v;
+            const __nv_bfloat16 hh = __float2bfloat16_rn(y);
+            hi[j] = hh;
+            lo[j] = __float2bfloat16_rn(y - __bfloat162float(hh));
+        }
     }
     if (!sumsq) return;
     ss = warp_sum(ss);
