@@ -396,7 +396,9 @@ class Bench:
         evs = [torch.cuda.Event(enable_timing=True) for _ in range(n_batches + 1)]
         sampler = ClockSampler(self.local)
         sampler.start()
-        time.sleep(0.12)                       # the sampler's first line
+        t_w = time.time()                      # the sampler's first line (nvidia-smi can take a second to come up)
+        while not sampler.samples and sampler.proc is not None and time.time() - t_w < 3.0:
+            time.sleep(0.02)
         self.barrier()
         t_wall0 = time.time()
         evs[0].record()
