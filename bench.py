@@ -45,12 +45,12 @@ MODULE_LAYERS, MODULE_ATTN_HEADS = 3, 16      # the paper's depth D = 3 (Sec. 4.
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the fused LM-head kernel, from
 # the ncu captures summarised under profiles/ (bytes per launch, and the summary they come from).
 NCU_TRAFFIC = {
-    "decode_1p7b": (627908096, "profiles/lm_head_dram_traffic.md"),
-    "spec_8b": (1366403328, "profiles/lm_head_dram_traffic.md"),
-    "remask_8b": (2794008320, "profiles/lm_head_dram_traffic.md"),
-    "sweep_M64_K4": (1368513792, "profiles/lm_head_dram_traffic.md"),
-    "sweep_M256_K1": (1486397184, "profiles/lm_head_dram_traffic.md"),
-    "sweep_M4096_K4": (35227708160, "profiles/lm_head_dram_traffic.md"),
+    "decode_1p7b": (628348416, "profiles/lm_head_dram_traffic.md"),
+    "spec_8b": (1372888320, "profiles/lm_head_dram_traffic.md"),
+    "remask_8b": (2900311296, "profiles/lm_head_dram_traffic.md"),
+    "sweep_M64_K4": (1368602368, "profiles/lm_head_dram_traffic.md"),
+    "sweep_M256_K1": (1486869504, "profiles/lm_head_dram_traffic.md"),
+    "sweep_M4096_K4": (43686557440, "profiles/lm_head_dram_traffic.md"),
 }
 
 
