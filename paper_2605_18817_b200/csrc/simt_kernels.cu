@@ -422,18 +422,40 @@ __device__ __forceinline__ void combine_body(int rs, int lane, const Partial *pa
         const bool have = fix.logits0 && (!fix.row_index || row_ok(idx, fix.n_rows_in));
         const __nv_bfloat16 *wr = fix.w + (size_t)tok * fix.d;
         const __nv_bfloat16 *xh = fix.xt + (size_t)rs * fix.d, *xl = xh + (size_t)fix.n_rs * fix.d;
+        // (the base logit of the top token is asked for before the dot product, not after it)
+        const float l0_top = have ? ld_l0(fix.logits0, fix.l0_bf16, (size_t)idx * (size_t)fix.V + tok) : 0.f;
         float dot = 0.f;
+        if ((fix.d & 255) == 0) {
+            // 16 bytes per lane and load: the three rows of a step of 256 elements are in flight together
 #pragma unroll 8
-        for (int j = lane * 2; j < fix.d; j += 64) {
-            const float2 w2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(wr + j));
-            const float2 h2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(xh + j));
-            const float2 l2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(xl + j));
-            dot = fmaf(w2.x, h2.x + l2.x, dot);
-            dot = fmaf(w2.y, h2.y + l2.y, dot);
-            ssq = fmaf(h2.x, h2.x, fmaf(h2.y, h2.y, ssq));
+            for (int j = lane * 8; j < fix.d; j += 256) {
+                const uint4 wq = __ldg(reinterpret_cast<const uint4 *>(wr + j));
+                const uint4 hq = *reinterpret_cast<const uint4 *>(xh + j);
+                const uint4 lq = *reinterpret_cast<const uint4 *>(xl + j);
+                const uint32_t w4[4] = {wq.x, wq.y, wq.z, wq.w}, h4[4] = {hq.x, hq.y, hq.z, hq.w}, l4[4] = {lq.x, lq.y, lq.z, lq.w};
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const float2 w2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&w4[i]));
+                    const float2 h2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&h4[i]));
+                    const float2 l2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&l4[i]));
+                    dot = fmaf(w2.x, h2.x + l2.x, dot);
+                    dot = fmaf(w2.y, h2.y + l2.y, dot);
+                    ssq = fmaf(h2.x, h2.x, fmaf(h2.y, h2.y, ssq));
+                }
+            }
+        } else {
+#pragma unroll 8
+            for (int j = lane * 2; j < fix.d; j += 64) {
+                const float2 w2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(wr + j));
+                const float2 h2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(xh + j));
+                const float2 l2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(xl + j));
+                dot = fmaf(w2.x, h2.x + l2.x, dot);
+                dot = fmaf(w2.y, h2.y + l2.y, dot);
+                ssq = fmaf(h2.x, h2.x, fmaf(h2.y, h2.y, ssq));
+            }
         }
         dot = warp_sum(dot);
-        top = (have ? ld_l0(fix.logits0, fix.l0_bf16, (size_t)idx * (size_t)fix.V + tok) : 0.f) + dot;
+        top = l0_top + dot;
     } else if (fix.range_limit > 0.f && has_operand) {
         // only the size of the operand row is needed: 16-byte loads of its hi part (d % 64 == 0)
         const uint4 *xh = reinterpret_cast<const uint4 *>(fix.xt + (size_t)rs * fix.d);
@@ -1060,7 +1082,13 @@ static cudaError_t simt_fused_t(Ctx *c, const void *hidden, const float *logits0
     at[0].val.cooperative = 1;
     cfg.attrs = at;
     cfg.numAttrs = 1;
-    e = note_err(c, cudaLaunchKernelEx(&cfg, kern, p), "one-kernel CUDA-core pass");
+    e = cudaLaunchKernelEx(&cfg, kern, p);
+    if (e == cudaErrorCooperativeLaunchTooLarge) {
+        // the context may use fewer SMs than the device has (MPS share, partition): one kernel per step instead
+        (void)cudaGetLastError();
+        return cudaSuccess;
+    }
+    e = note_err(c, e, "one-kernel CUDA-core pass");
     c->launches++;
     *launched = true;
     // the phases of the pass are not separate launches: the profile books the whole kernel under the heads
@@ -1686,7 +1714,13 @@ static cudaError_t module_fused_t(Ctx *c, const int32_t *tokens, const void *hid
     at[0].val.cooperative = 1;
     cfg.attrs = at;
     cfg.numAttrs = 1;
-    e = note_err(c, cudaLaunchKernelEx(&cfg, kern, p), "one-kernel module step");
+    e = cudaLaunchKernelEx(&cfg, kern, p);
+    if (e == cudaErrorCooperativeLaunchTooLarge) {
+        // the context may use fewer SMs than the device has (MPS share, partition): one kernel per product instead
+        (void)cudaGetLastError();
+        return cudaSuccess;
+    }
+    e = note_err(c, e, "one-kernel module step");
     c->launches++;
     *launched = true;
     return e;
