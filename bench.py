@@ -47,10 +47,10 @@ MODULE_LAYERS, MODULE_ATTN_HEADS = 3, 16      # the paper's depth D = 3 (Sec. 4.
 NCU_TRAFFIC = {
     "decode_1p7b": (628348416, "profiles/lm_head_dram_traffic.md"),
     "spec_8b": (1372888320, "profiles/lm_head_dram_traffic.md"),
-    "remask_8b": (2900311296, "profiles/lm_head_dram_traffic.md"),
-    "sweep_M64_K4": (1368602368, "profiles/lm_head_dram_traffic.md"),
-    "sweep_M256_K1": (1486869504, "profiles/lm_head_dram_traffic.md"),
-    "sweep_M4096_K4": (43686557440, "profiles/lm_head_dram_traffic.md"),
+    "remask_8b": (2638083328, "profiles/lm_head_dram_traffic.md"),
+    "sweep_M64_K4": (1365900032, "profiles/lm_head_dram_traffic.md"),
+    "sweep_M256_K1": (1486500096, "profiles/lm_head_dram_traffic.md"),
+    "sweep_M4096_K4": (36579955712, "profiles/lm_head_dram_traffic.md"),
 }
 
 

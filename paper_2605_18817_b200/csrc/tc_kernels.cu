@@ -92,7 +92,9 @@ struct TcParams {
 // F16: one fp16 A tile per stage against fp16 weights (LM head only); otherwise the bf16 hi and lo
 // A tiles of a k-chunk against bf16 weights.
 // PAIR: the grid is launched in clusters of two CTAs that share every MMA (cta_group::2, M = 256): CTA r of
-// a pair owns row block 2 pb + r and loads its own A tiles plus HALF of the B tile (rows r * bn / 2 ...),
+// a pair owns row block pb + r * (number of pairs of blocks) -- with an even number K of steps stacked these are
+// the same masked rows at steps k and k + K / 2, so that the pair reads each tile of their base logits from
+// DRAM once -- and loads its own A tiles plus HALF of the B tile (rows r * bn / 2 ...),
 // which halves the weight bytes a CTA pulls from L2 per MMA cycle and so deepens the ring.  The leader
 // (rank 0) issues the MMAs; both CTAs' loads complete on the leader's full barrier; the MMA commits
 // arrive on both CTAs' empty / accumulator-full barriers; both CTAs' epilogue warps arrive on the
@@ -121,7 +123,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     // PAIR: `cta` numbers the pair, `rank` the CTA in it; a pair walks PAIRS of row blocks (p.n_rb counts pairs,
-    // row block of this CTA = 2 * pair-block + rank)
+    // row block of this CTA = pair-block + rank * p.n_rb)
     const int rank = PAIR ? (int)cluster_ctarank() : 0;
     const int cta = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
     const int vr = cta % p.n_vr, grp = cta / p.n_vr;
@@ -184,7 +186,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             };
             auto load_a = [&](int mb_, int kk_, int s_) {
                 const uint32_t sa = base + (uint32_t)s_ * stage_bytes;
-                const int row0 = p.a_row_base + (PAIR ? 2 * mb_ + rank : mb_) * 128;
+                const int row0 = p.a_row_base + (PAIR ? mb_ + rank * p.n_rb : mb_) * 128;
                 if (PAIR) {
                     tma_load_2d_pair(sa, &tmA, kk_ * kBK, row0, full_bar(s_));
                     if (!F16) tma_load_2d_pair(sa + kATile, &tmA, kk_ * kBK, p.a_part_rows + row0, full_bar(s_));
@@ -287,7 +289,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         bool ok = true;
         for (int mb = grp; mb < p.n_rb && ok; mb += p.n_groups) {
             // ---- per-block state: this thread's activation row ----
-            const int r = (PAIR ? 2 * mb + rank : mb) * 128 + rl;
+            const int r = (PAIR ? mb + rank * p.n_rb : mb) * 128 + rl;
             const bool valid = r < p.rows;
             RowStat st, st0;       // LM: statistics of the row's own step, and of step 0 (rows of step 1 only)
             KlStat kst;            // LM, KL variant: the row-step's share of the training objective
