@@ -1858,9 +1858,7 @@ static cudaError_t module_body_tc(Ctx *c, const int32_t *tokens, const void *hid
     for (int l = 0; l < w.n_layers && e == cudaSuccess; ++l) {
         const mrp_module_layer &y = w.layers[l];
         e = split(z, y.g_attn, d, x16, sumsq);
-        if (e == cudaSuccess) e = tc_linear(c, x16, n, d, y.w_q, d, sumsq, q, false, out.status, st);
-        if (e == cudaSuccess) e = tc_linear(c, x16, n, d, y.w_k, d, sumsq, k, false, out.status, st);
-        if (e == cudaSuccess) e = tc_linear(c, x16, n, d, y.w_v, d, sumsq, v, false, out.status, st);
+        if (e == cudaSuccess) e = tc_linear3(c, x16, n, d, y.w_q, y.w_k, y.w_v, d, sumsq, q, k, v, out.status, st);
         if (e == cudaSuccess) {
             e = launch_k(mod_attention_kernel, dim3(B, w.n_attn_heads), dim3(128), (size_t)4 * L * 4, st, pdl, (const float *)q,
                          (const float *)k, (const float *)v, L, d, dh, o);

@@ -82,6 +82,10 @@ struct TcParams {
     float *lin_out;
     int lin_n_out;
     int lin_accumulate;
+    // LIN over lin_nw = 3 weight matrices of the same shape sharing the activation rows (q, k, v of the module):
+    // the weight-row ranges are dealt out per matrix (n_vr / 3 each), results to lin_out, lin_out1, lin_out2
+    int lin_nw;
+    float *lin_out1, *lin_out2;
     int32_t *status;
     int32_t *user_status;
 };
@@ -102,7 +106,7 @@ struct TcParams {
 template <int KIND, bool MARGIN, bool F16, bool KL, bool PAIR = false>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
-               const __grid_constant__ CUtensorMap tmB1, const TcParams p)
+               const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmB2, const TcParams p)
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -127,8 +131,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int rank = PAIR ? (int)cluster_ctarank() : 0;
     const int cta = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
     const int vr = cta % p.n_vr, grp = cta / p.n_vr;
-    const int u0 = (int)((long long)vr * p.units_total / p.n_vr);
-    const int u1 = (int)((long long)(vr + 1) * p.units_total / p.n_vr);
+    // (LIN over three matrices: `which` of them this CTA works on, and its range among that matrix's n_vr / 3)
+    const int n_vr_w = (KIND == KIND_LIN && p.lin_nw == 3) ? p.n_vr / 3 : p.n_vr;
+    const int which = (KIND == KIND_LIN && p.lin_nw == 3) ? vr / n_vr_w : 0;
+    const int vr_w = vr - which * n_vr_w;
+    const CUtensorMap *tmB = which == 0 ? &tmB0 : which == 1 ? &tmB1 : &tmB2;
+    float *lin_dst = which == 0 ? p.lin_out : which == 1 ? p.lin_out1 : p.lin_out2;
+    const int u0 = (int)((long long)vr_w * p.units_total / n_vr_w);
+    const int u1 = (int)((long long)(vr_w + 1) * p.units_total / n_vr_w);
     const int n_t = (u1 - u0 + p.w_units - 1) / p.w_units;
 
     if (threadIdx.x == 0) {
@@ -137,7 +147,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         prefetch_tmap(&tmA);
-        prefetch_tmap(&tmB0);
+        prefetch_tmap(KIND == KIND_LIN ? tmB : &tmB0);
         if (KIND == KIND_GU) prefetch_tmap(&tmB1);
     }
     if (warp == 1) {
@@ -178,9 +188,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     // this CTA's half of the B tile: rows [rank * bn / 2, ...) of a one-box tile; of a gate/up tile
                     // the gate rows (leader) or the up rows (peer), so that the columns stay [gate | up]
                     if (KIND == KIND_GU) tma_load_2d_pair(sb, rank ? &tmB1 : &tmB0, kk_ * kBK, n0, full_bar(s_));
-                    else tma_load_2d_pair(sb, &tmB0, kk_ * kBK, n0 + rank * bn_own, full_bar(s_));
+                    else tma_load_2d_pair(sb, KIND == KIND_LIN ? tmB : &tmB0, kk_ * kBK, n0 + rank * bn_own, full_bar(s_));
                 } else {
-                    tma_load_2d(sb, &tmB0, kk_ * kBK, n0, full_bar(s_));
+                    tma_load_2d(sb, KIND == KIND_LIN ? tmB : &tmB0, kk_ * kBK, n0, full_bar(s_));
                     if (KIND == KIND_GU) tma_load_2d(sb + box_rows * 128, &tmB1, kk_ * kBK, n0, full_bar(s_));
                 }
             };
@@ -387,11 +397,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                             }
                             if (p.lin_accumulate) {
                                 float z[16];
-                                load16_rw(p.lin_out + o, z);
+                                load16_rw(lin_dst + o, z);
 #pragma unroll
                                 for (int j = 0; j < 16; ++j) a[j] += z[j];
                             }
-                            store16(p.lin_out + o, a);
+                            store16(lin_dst + o, a);
                         }
                     }
                 } else {
@@ -643,8 +653,9 @@ size_t smem_bytes(const TcParams &p, int parts, bool pair)
 // PAIR: `grid` counts CTAs (two per pair); the launch carries the cluster shape (2, 1, 1).
 template <int KIND, bool MARGIN, bool F16 = false, bool KL = false, bool PAIR = false>
 cudaError_t launch_tc(const CUtensorMap &a, const CUtensorMap &b0, const CUtensorMap &b1, const TcParams &p,
-                      int grid, cudaStream_t st, bool pdl)
+                      int grid, cudaStream_t st, bool pdl, const CUtensorMap *b2_opt = nullptr)
 {
+    const CUtensorMap &b2 = b2_opt ? *b2_opt : b1;
     auto kern = tc_gemm_kernel<KIND, MARGIN, F16, KL, PAIR>;
     const size_t smem = smem_bytes(p, F16 ? 1 : 2, PAIR);
     // the shared-memory limit of a kernel is set once per device (the attribute is per device)
@@ -671,9 +682,9 @@ cudaError_t launch_tc(const CUtensorMap &a, const CUtensorMap &b0, const CUtenso
         at[1].val.programmaticStreamSerializationAllowed = 1;
         cfg.attrs = at;
         cfg.numAttrs = pdl ? 2 : 1;
-        return cudaLaunchKernelEx(&cfg, kern, a, b0, b1, p);
+        return cudaLaunchKernelEx(&cfg, kern, a, b0, b1, b2, p);
     }
-    return launch_k(kern, dim3(grid), dim3(kThreads), smem, st, pdl, a, b0, b1, p);
+    return launch_k(kern, dim3(grid), dim3(kThreads), smem, st, pdl, a, b0, b1, b2, p);
 }
 
 }  // namespace
@@ -873,6 +884,35 @@ cudaError_t tc_linear(Ctx *c, const __nv_bfloat16 *a, int n, int n_in, const voi
     c->launches++;
     return note_err(c, launch_tc<KIND_LIN, false>(mA, mB, mB, p, p.n_groups * p.n_vr, st, !(c->cfg.flags & MRP_FLAG_NO_PDL)),
                     "module product kernel");
+}
+
+// Three products over the same operand rows in one launch: out_i[n, n_out] = rstd(row) * (A W_i^T), i = 0, 1, 2
+// (q, k, v of a module layer).  The weight-row ranges are dealt out per matrix, so a CTA's tile is three times as
+// wide as with a launch per matrix, and the activation tiles are loaded a third as often per weight byte.
+cudaError_t tc_linear3(Ctx *c, const __nv_bfloat16 *a, int n, int n_in, const void *w0, const void *w1, const void *w2,
+                       int n_out, const float *sumsq, float *out0, float *out1, float *out2, int32_t *user_status,
+                       cudaStream_t st)
+{
+    const TcState *s = (const TcState *)c->tc_state;
+    const int G = c->sm_count, n_mb = (n + 127) / 128;
+    CUtensorMap mA, mB0, mB1, mB2;
+    TcParams p;
+    memset(&p, 0, sizeof(p));
+    p.units_total = n_out / 16; p.unit_rows = 16; p.n_boxes = 1; p.k_chunks = n_in / kBK;
+    p.n_groups = choose_groups(n_mb, 3 * p.units_total, G); p.n_rb = n_mb; p.rows = n; p.a_row_base = 0; p.a_part_rows = n;
+    p.M = n; p.d = n_in; p.sumsq = sumsq; p.n_ss = 1; p.eps = c->cfg.rms_eps;
+    p.lin_out = out0; p.lin_out1 = out1; p.lin_out2 = out2; p.lin_n_out = n_out; p.lin_nw = 3;
+    p.status = (int32_t *)(c->ws + c->lay.status); p.user_status = user_status;
+    int per_w = (G / p.n_groups) / 3;                    // weight-row ranges per matrix
+    if (per_w < 1) per_w = 1;
+    finish_shape(p, per_w);
+    p.n_vr = 3 * per_w;
+    if (!make_map(s, &mA, a, n_in, 2 * (uint64_t)n, 128) || !make_map(s, &mB0, w0, n_in, n_out, p.bn) ||
+        !make_map(s, &mB1, w1, n_in, n_out, p.bn) || !make_map(s, &mB2, w2, n_in, n_out, p.bn))
+        return note_err(c, cudaErrorInvalidValue, "tensor map (module q, k, v)");
+    c->launches++;
+    return note_err(c, launch_tc<KIND_LIN, false>(mA, mB0, mB1, p, p.n_groups * p.n_vr, st, !(c->cfg.flags & MRP_FLAG_NO_PDL), &mB2),
+                    "module q, k, v kernel");
 }
 
 // act[n, F] (bf16 hi rows, lo rows n * F elements further on) = silu(rstd * A Wg^T) * (rstd * A Wu^T): the head
