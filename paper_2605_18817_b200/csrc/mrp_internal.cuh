@@ -237,12 +237,13 @@ cudaError_t tc_lm_tail(Ctx *c, const TcPlan &pl, const float *logits0, const int
                        const mrp_draft_out &out, cudaStream_t st);
 // Row-major tensor-core products on operands of the caller's own (the module): see tc_kernels.cu.
 cudaError_t tc_linear(Ctx *c, const __nv_bfloat16 *a, int n, int n_in, const void *w, int n_out, const float *sumsq,
-                      float *out, bool accumulate, int32_t *user_status, cudaStream_t st);
+                      int n_ss, float *out, bool accumulate, int32_t *user_status, cudaStream_t st, const void *gamma_next,
+                      __nv_bfloat16 *xg_next, float *sumsq_out, int *n_ss_out);
 cudaError_t tc_linear3(Ctx *c, const __nv_bfloat16 *a, int n, int n_in, const void *w0, const void *w1, const void *w2,
-                       int n_out, const float *sumsq, float *out0, float *out1, float *out2, int32_t *user_status,
+                       int n_out, const float *sumsq, int n_ss, float *out0, float *out1, float *out2, int32_t *user_status,
                        cudaStream_t st);
 cudaError_t tc_gate_up(Ctx *c, const __nv_bfloat16 *a, int n, int n_in, const void *w_gate, const void *w_up, int F,
-                       const float *sumsq, __nv_bfloat16 *act, int32_t *user_status, cudaStream_t st);
+                       const float *sumsq, int n_ss, __nv_bfloat16 *act, int32_t *user_status, cudaStream_t st);
 // The same for the CUDA-core family (operand rows: fp32 xt).
 cudaError_t simt_lm_tail(Ctx *c, const float *logits0, const int32_t *row_index, int M, int K,
                          const mrp_draft_out &out, cudaStream_t st);

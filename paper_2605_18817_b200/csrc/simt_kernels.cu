@@ -1175,8 +1175,10 @@ __global__ void linear_kernel(const T *__restrict__ w, const float *__restrict__
 
 // Block-local bidirectional attention: CTA = (block b, attention head); a warp per query position, lanes
 // over the key positions for the scores and over the head's features for the output.
+// (o16: the output as bf16 hi rows [n_rows, d] with the lo rows n_rows rows further on instead of fp32 rows in o)
 __global__ void mod_attention_kernel(const float *__restrict__ q, const float *__restrict__ k,
-                                     const float *__restrict__ v, int L, int d, int dh, float *__restrict__ o)
+                                     const float *__restrict__ v, int L, int d, int dh, float *__restrict__ o,
+                                     __nv_bfloat16 *__restrict__ o16, int n_rows)
 {
     pdl_trigger();
     pdl_wait();
@@ -1222,7 +1224,15 @@ __global__ void mod_attention_kernel(const float *__restrict__ q, const float *_
         for (int c = lane; c < dh; c += 32) {
             float acc = 0.f;
             for (int j = 0; j < L; ++j) acc = fmaf(p[j], v[((size_t)b * L + j) * d + (size_t)hd * dh + c], acc);
-            o[((size_t)b * L + i) * d + (size_t)hd * dh + c] = acc / sum;
+            const float val = acc / sum;
+            const size_t at = ((size_t)b * L + i) * d + (size_t)hd * dh + c;
+            if (o16) {
+                const __nv_bfloat16 hh = __float2bfloat16_rn(val);
+                o16[at] = hh;
+                o16[(size_t)n_rows * d + at] = __float2bfloat16_rn(val - __bfloat162float(hh));
+            } else {
+                o[at] = val;
+            }
         }
         __syncwarp();
     }
@@ -1728,8 +1738,9 @@ static cudaError_t module_fused_t(Ctx *c, const int32_t *tokens, const void *hid
 
 // ---- the module's products on the tensor cores (more than a handful of positions) ----------------------
 // The matrix products of the step run on the row-major tcgen05 kernel (tc_linear / tc_gate_up: bf16 hi + lo
-// operand rows, fp32 accumulation, RMSNorm folded in as gamma on the operand and 1 / rms on the result); what is
-// between them (embedding fusion, operand splitting, attention, the residual sums) stays on the CUDA cores.
+// operand rows, fp32 accumulation, RMSNorm folded in as gamma on the operand and 1 / rms on the result; a product
+// that completes z writes the next product's operand and its partial sums of squares itself); the embedding
+// fusion in front and the attention stay on the CUDA cores.
 // bf16 hi + lo rows of [h_i ; emb[x_i]]: the hi rows [n, 2 d], the lo rows n rows further on.
 __global__ void mod_cat_split_kernel(const float *h_state, const __nv_bfloat16 *__restrict__ hidden0, int first_step,
                                      const int32_t *__restrict__ tokens, const __nv_bfloat16 *__restrict__ emb, int mask_token,
@@ -1760,62 +1771,12 @@ __global__ void mod_cat_split_kernel(const float *h_state, const __nv_bfloat16 *
     }
 }
 
-// bf16 hi + lo rows of x[i, :] * gamma (gamma == nullptr: of x itself), and the row's sum of squares of x.
-__global__ void mod_split_kernel(const float *__restrict__ x, const __nv_bfloat16 *__restrict__ gamma, int n, int width,
-                                 __nv_bfloat16 *__restrict__ out, float *__restrict__ sumsq)
-{
-    pdl_trigger();
-    pdl_wait();
-    __shared__ float red[32];
-    const int i = blockIdx.x;
-    __nv_bfloat16 *hi = out + (size_t)i * width, *lo = out + ((size_t)n + i) * width;
-    float ss = 0.f;
-    if ((width & 7) == 0) {
-        // eight elements per thread: 32-byte reads, 16-byte writes of each half
-        for (int j = threadIdx.x * 8; j < width; j += blockDim.x * 8) {
-            const float4 a = *reinterpret_cast<const float4 *>(x + (size_t)i * width + j);
-            const float4 b = *reinterpret_cast<const float4 *>(x + (size_t)i * width + j + 4);
-            const float v[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
-            __nv_bfloat162 h2[4], l2[4];
-#pragma unroll
-            for (int e = 0; e < 8; e += 2) {
-                ss = fmaf(v[e], v[e], fmaf(v[e + 1], v[e + 1], ss));
-                const float y0 = gamma ? v[e] * __bfloat162float(gamma[j + e]) : v[e];
-                const float y1 = gamma ? v[e + 1] * __bfloat162float(gamma[j + e + 1]) : v[e + 1];
-                const __nv_bfloat16 h0 = __float2bfloat16_rn(y0), h1 = __float2bfloat16_rn(y1);
-                h2[e >> 1] = __halves2bfloat162(h0, h1);
-                l2[e >> 1] = __halves2bfloat162(__float2bfloat16_rn(y0 - __bfloat162float(h0)),
-                                                __float2bfloat16_rn(y1 - __bfloat162float(h1)));
-            }
-            *reinterpret_cast<uint4 *>(hi + j) = *reinterpret_cast<const uint4 *>(h2);
-            *reinterpret_cast<uint4 *>(lo + j) = *reinterpret_cast<const uint4 *>(l2);
-        }
-    } else {
-        for (int j = threadIdx.x; j < width; j += blockDim.x) {
-            const float v = x[(size_t)i * width + j];
-            ss = fmaf(v, v, ss);
-            const float y = gamma ? v * __bfloat162float(gamma[j]) : v;
-            const __nv_bfloat16 hh = __float2bfloat16_rn(y);
-            hi[j] = hh;
-            lo[j] = __float2bfloat16_rn(y - __bfloat162float(hh));
-        }
-    }
-    if (!sumsq) return;
-    ss = warp_sum(ss);
-    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        float t = 0.f;
-        for (int w = 0; w < (int)(blockDim.x >> 5); ++w) t += red[w];
-        sumsq[i] = t;
-    }
-}
-
 // Whether the module's products of a call over n positions can run on the tensor cores.
 static bool module_tc_ok(const Ctx *c, int n)
 {
     if (!c->use_tc || c->cfg.dtype != MRP_BF16 || (c->cfg.flags & MRP_FLAG_FORCE_SIMT)) return false;
-    if (c->cfg.d % 64 || c->cfg.d_ff % 64 || n > c->cfg.max_rows * kSumsqSlices) return false;
+    // (the partial sums of squares of the module's norms use the context's [kSumsqSlices, max_rows] array)
+    if (c->cfg.d % 64 || c->cfg.d_ff % 64 || (long long)c->sm_count * n > (long long)c->cfg.max_rows * kSumsqSlices) return false;
     const mrp_module_weights &w = c->module;
     auto al = [](const void *p) { return ((uintptr_t)p & 15u) == 0; };
     if (!al(w.emb) || !al(w.w_proj)) return false;
@@ -1838,9 +1799,9 @@ static cudaError_t module_body_tc(Ctx *c, const int32_t *tokens, const void *hid
     // the regions of the fp32 path hold the bf16 hi + lo operands here (same bytes: two halves of two bytes)
     __nv_bfloat16 *cat16 = (__nv_bfloat16 *)take(cap * 2 * d * 4);
     float *zz = (float *)take(cap * d * 4);
-    __nv_bfloat16 *x16 = (__nv_bfloat16 *)take(cap * d * 4);
+    __nv_bfloat16 *xa = (__nv_bfloat16 *)take(cap * d * 4);          // operand of q/k/v and of gate/up
     float *q = (float *)take(cap * d * 4), *k = (float *)take(cap * d * 4), *v = (float *)take(cap * d * 4);
-    float *o = (float *)take(cap * d * 4);
+    __nv_bfloat16 *xb = (__nv_bfloat16 *)take(cap * d * 4);          // operand of the output projection
     __nv_bfloat16 *act16 = (__nv_bfloat16 *)take(cap * F * 4);
     (void)zz;
     float *sumsq = (float *)(c->ws + c->lay.sumsq);
@@ -1850,25 +1811,28 @@ static cudaError_t module_body_tc(Ctx *c, const int32_t *tokens, const void *hid
                              (const __nv_bfloat16 *)hidden0, first_step ? 1 : 0, tokens, (const __nv_bfloat16 *)w.emb, w.mask_token,
                              w.emb_rows, n, d, h_state, cat16, status, out.status);
     c->launches++;
-    if (e == cudaSuccess) e = tc_linear(c, cat16, n, 2 * d, w.w_proj, d, nullptr, z, false, out.status, st);
-    auto split = [&](const float *x, const void *gamma, int width, __nv_bfloat16 *dst, float *ss) {
-        c->launches++;
-        return launch_k(mod_split_kernel, dim3(n), dim3(256), 0, st, pdl, x, (const __nv_bfloat16 *)gamma, n, width, dst, ss);
-    };
+    // Every product that completes z also writes the next product's operand (z * next norm weight, hi + lo) and
+    // its partial sums of squares: no kernel between them.
+    int n_ss = 1;
+    const void *g_first = w.n_layers > 0 ? w.layers[0].g_attn : nullptr;
+    if (e == cudaSuccess)
+        e = tc_linear(c, cat16, n, 2 * d, w.w_proj, d, nullptr, 1, z, false, out.status, st, g_first, g_first ? xa : nullptr,
+                      sumsq, &n_ss);
     for (int l = 0; l < w.n_layers && e == cudaSuccess; ++l) {
         const mrp_module_layer &y = w.layers[l];
-        e = split(z, y.g_attn, d, x16, sumsq);
-        if (e == cudaSuccess) e = tc_linear3(c, x16, n, d, y.w_q, y.w_k, y.w_v, d, sumsq, q, k, v, out.status, st);
+        e = tc_linear3(c, xa, n, d, y.w_q, y.w_k, y.w_v, d, sumsq, n_ss, q, k, v, out.status, st);
         if (e == cudaSuccess) {
             e = launch_k(mod_attention_kernel, dim3(B, w.n_attn_heads), dim3(128), (size_t)4 * L * 4, st, pdl, (const float *)q,
-                         (const float *)k, (const float *)v, L, d, dh, o);
+                         (const float *)k, (const float *)v, L, d, dh, (float *)nullptr, xb, n);
             c->launches++;
         }
-        if (e == cudaSuccess) e = split(o, nullptr, d, x16, nullptr);
-        if (e == cudaSuccess) e = tc_linear(c, x16, n, d, y.w_o, d, nullptr, z, true, out.status, st);
-        if (e == cudaSuccess) e = split(z, y.g_mlp, d, x16, sumsq);
-        if (e == cudaSuccess) e = tc_gate_up(c, x16, n, d, y.w_gate, y.w_up, F, sumsq, act16, out.status, st);
-        if (e == cudaSuccess) e = tc_linear(c, act16, n, F, y.w_down, d, nullptr, z, true, out.status, st);
+        if (e == cudaSuccess)
+            e = tc_linear(c, xb, n, d, y.w_o, d, nullptr, 1, z, true, out.status, st, y.g_mlp, xa, sumsq, &n_ss);
+        if (e == cudaSuccess) e = tc_gate_up(c, xa, n, d, y.w_gate, y.w_up, F, sumsq, n_ss, act16, out.status, st);
+        const void *g_next = l + 1 < w.n_layers ? w.layers[l + 1].g_attn : nullptr;
+        if (e == cudaSuccess)
+            e = tc_linear(c, act16, n, F, y.w_down, d, nullptr, 1, z, true, out.status, st, g_next, g_next ? xa : nullptr, sumsq,
+                          &n_ss);
     }
     return e;
 }
@@ -1934,7 +1898,7 @@ static cudaError_t module_step_t(Ctx *c, const int32_t *tokens, const void *hidd
         if (e == cudaSuccess) e = lin(y.w_v, nn, d, d, v, 0);
         if (e == cudaSuccess) {
             e = launch_k(mod_attention_kernel, dim3(B, w.n_attn_heads), dim3(128), (size_t)4 * L * 4, st, pdl, (const float *)q,
-                         (const float *)k, (const float *)v, L, d, dh, o);
+                         (const float *)k, (const float *)v, L, d, dh, o, (__nv_bfloat16 *)nullptr, n);
             c->launches++;
         }
         if (e == cudaSuccess) e = lin(y.w_o, o, d, d, z, 1);

@@ -402,6 +402,18 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                                 for (int j = 0; j < 16; ++j) a[j] += z[j];
                             }
                             store16(lin_dst + o, a);
+                            if (p.xg_next) {
+                                // the next product's operand rows, out * gamma_next as bf16 hi + lo, and this CTA's
+                                // share of the row's sum of squares (its RMSNorm)
+                                const __nv_bfloat16 *gm = p.gamma_next + j_tile + c * 16;
+                                float x[16];
+#pragma unroll
+                                for (int j = 0; j < 16; ++j) {
+                                    ssq = fmaf(a[j], a[j], ssq);
+                                    x[j] = a[j] * __bfloat162float(gm[j]);
+                                }
+                                store_split<16>(p.xg_next + o, (size_t)p.M * p.lin_n_out, x);
+                            }
                         }
                     }
                 } else {
@@ -455,6 +467,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     if (KL)
                         p.kl_partials[(size_t)vr * ((size_t)p.K * p.M) + (size_t)(k_of_row - 1) * p.M + m_of_row] = kst.partial();
                 } else if (KIND == KIND_DN) {
+                    p.sumsq_out[(size_t)vr * p.M + m_of_row] = ssq;
+                } else if (KIND == KIND_LIN && p.xg_next) {
                     p.sumsq_out[(size_t)vr * p.M + m_of_row] = ssq;
                 }
             }
@@ -865,8 +879,11 @@ cudaError_t tc_lm_tail(Ctx *c, const TcPlan &pl, const float *logits0, const int
 // out[n, n_out] (+)= rstd(row) * (A W^T): A = bf16 hi rows [n, n_in] with the lo rows n rows further on, W bf16
 // [n_out, n_in]; rstd(row) = rsqrt(sumsq[row] / n_in + eps) where sumsq is given, else 1.  n_in % 64 == 0,
 // n_out % 16 == 0, 16-byte aligned pointers.
+// With xg_next: also writes the rows of out * gamma_next as the next product's bf16 hi + lo operand (lo rows n rows
+// further on) and per-CTA partial sums of squares of out to sumsq_out[*n_ss_out, n] (the next RMSNorm).
 cudaError_t tc_linear(Ctx *c, const __nv_bfloat16 *a, int n, int n_in, const void *w, int n_out, const float *sumsq,
-                      float *out, bool accumulate, int32_t *user_status, cudaStream_t st)
+                      int n_ss, float *out, bool accumulate, int32_t *user_status, cudaStream_t st, const void *gamma_next,
+                      __nv_bfloat16 *xg_next, float *sumsq_out, int *n_ss_out)
 {
     const TcState *s = (const TcState *)c->tc_state;
     const int G = c->sm_count, n_mb = (n + 127) / 128;
@@ -875,10 +892,12 @@ cudaError_t tc_linear(Ctx *c, const __nv_bfloat16 *a, int n, int n_in, const voi
     memset(&p, 0, sizeof(p));
     p.units_total = n_out / 16; p.unit_rows = 16; p.n_boxes = 1; p.k_chunks = n_in / kBK;
     p.n_groups = choose_groups(n_mb, p.units_total, G); p.n_rb = n_mb; p.rows = n; p.a_row_base = 0; p.a_part_rows = n;
-    p.M = n; p.d = n_in; p.sumsq = sumsq; p.n_ss = 1; p.eps = c->cfg.rms_eps;
+    p.M = n; p.d = n_in; p.sumsq = sumsq; p.n_ss = n_ss; p.eps = c->cfg.rms_eps;
     p.lin_out = out; p.lin_n_out = n_out; p.lin_accumulate = accumulate ? 1 : 0;
+    p.gamma_next = (const __nv_bfloat16 *)gamma_next; p.xg_next = xg_next; p.sumsq_out = sumsq_out;
     p.status = (int32_t *)(c->ws + c->lay.status); p.user_status = user_status;
     finish_shape(p, G / p.n_groups);
+    if (n_ss_out) *n_ss_out = p.n_vr;
     if (!make_map(s, &mA, a, n_in, 2 * (uint64_t)n, 128) || !make_map(s, &mB, w, n_in, n_out, p.bn))
         return note_err(c, cudaErrorInvalidValue, "tensor map (module product)");
     c->launches++;
@@ -890,7 +909,7 @@ cudaError_t tc_linear(Ctx *c, const __nv_bfloat16 *a, int n, int n_in, const voi
 // (q, k, v of a module layer).  The weight-row ranges are dealt out per matrix, so a CTA's tile is three times as
 // wide as with a launch per matrix, and the activation tiles are loaded a third as often per weight byte.
 cudaError_t tc_linear3(Ctx *c, const __nv_bfloat16 *a, int n, int n_in, const void *w0, const void *w1, const void *w2,
-                       int n_out, const float *sumsq, float *out0, float *out1, float *out2, int32_t *user_status,
+                       int n_out, const float *sumsq, int n_ss, float *out0, float *out1, float *out2, int32_t *user_status,
                        cudaStream_t st)
 {
     const TcState *s = (const TcState *)c->tc_state;
@@ -900,7 +919,7 @@ cudaError_t tc_linear3(Ctx *c, const __nv_bfloat16 *a, int n, int n_in, const vo
     memset(&p, 0, sizeof(p));
     p.units_total = n_out / 16; p.unit_rows = 16; p.n_boxes = 1; p.k_chunks = n_in / kBK;
     p.n_groups = choose_groups(n_mb, 3 * p.units_total, G); p.n_rb = n_mb; p.rows = n; p.a_row_base = 0; p.a_part_rows = n;
-    p.M = n; p.d = n_in; p.sumsq = sumsq; p.n_ss = 1; p.eps = c->cfg.rms_eps;
+    p.M = n; p.d = n_in; p.sumsq = sumsq; p.n_ss = n_ss; p.eps = c->cfg.rms_eps;
     p.lin_out = out0; p.lin_out1 = out1; p.lin_out2 = out2; p.lin_n_out = n_out; p.lin_nw = 3;
     p.status = (int32_t *)(c->ws + c->lay.status); p.user_status = user_status;
     int per_w = (G / p.n_groups) / 3;                    // weight-row ranges per matrix
@@ -918,7 +937,7 @@ cudaError_t tc_linear3(Ctx *c, const __nv_bfloat16 *a, int n, int n_in, const vo
 // act[n, F] (bf16 hi rows, lo rows n * F elements further on) = silu(rstd * A Wg^T) * (rstd * A Wu^T): the head
 // chain's gate/up kernel on other operands.
 cudaError_t tc_gate_up(Ctx *c, const __nv_bfloat16 *a, int n, int n_in, const void *w_gate, const void *w_up, int F,
-                       const float *sumsq, __nv_bfloat16 *act, int32_t *user_status, cudaStream_t st)
+                       const float *sumsq, int n_ss, __nv_bfloat16 *act, int32_t *user_status, cudaStream_t st)
 {
     const TcState *s = (const TcState *)c->tc_state;
     const int G = c->sm_count, n_mb = (n + 127) / 128;
@@ -928,7 +947,7 @@ cudaError_t tc_gate_up(Ctx *c, const __nv_bfloat16 *a, int n, int n_in, const vo
     p.units_total = F / 8; p.unit_rows = 8; p.n_boxes = 2; p.k_chunks = n_in / kBK;
     p.n_groups = choose_groups(n_mb, p.units_total, G); p.n_rb = n_mb; p.rows = n; p.a_row_base = 0; p.a_part_rows = n;
     p.M = n; p.d = n_in; p.F = F;
-    p.sumsq = sumsq; p.n_ss = 1; p.eps = c->cfg.rms_eps; p.act = act;
+    p.sumsq = sumsq; p.n_ss = n_ss; p.eps = c->cfg.rms_eps; p.act = act;
     p.status = (int32_t *)(c->ws + c->lay.status); p.user_status = user_status;
     finish_shape(p, G / p.n_groups);
     if (!make_map(s, &mA, a, n_in, 2 * (uint64_t)n, 128) || !make_map(s, &mB0, w_gate, n_in, F, p.bn / 2) ||
