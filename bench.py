@@ -636,7 +636,7 @@ class Bench:
                 "steps": n_e2e, "ms_per_step": dt / n_e2e * 1e3, "mode": e2e_mode}
 
 
-def run_module_workload(bench, cpu_budget_s, which=1):
+def run_module_workload(bench, cpu_budget_s, which=1, block_len=None):
     """The token-conditioned module at the shape of configuration `which` (1: the decode shape, one block of 4
     positions; 2: 32 blocks of 4, d = 4096): a step is the K = 3 MRP steps that follow one backbone forward in
     direct decoding (Algorithm 2), each = mrp_module_step (module forward + one LM-head pass) +
@@ -648,6 +648,8 @@ def run_module_workload(bench, cpu_budget_s, which=1):
     from paper_2605_18817_b200 import binding, harness, synth
     args, dev, dist = bench.args, bench.dev, bench.dist
     base = synth.CONFIGS[which]
+    if block_len:                                      # the paper's block length (Sec. 4.1) instead of the configuration's
+        base = dict(base, L=block_len, name="%s_L%d" % (base["name"], block_len))
     cfg = dict(base, name="module_" + base["name"])
     w, heads, w_lm = bench.weights_for(base, str(which))
     big = base["d"] >= 4096
@@ -796,8 +798,8 @@ def main():
     head_name = HEADLINE if args.config == "all" else args.config
     results = {}
     for name in names:
-        if name in ("module", "module:1", "module:2"):
-            results[name] = run_module_workload(bench, 5.0, 2 if name == "module:2" else 1)
+        if name in ("module", "module:1", "module:2", "module:L16"):
+            results[name] = run_module_workload(bench, 5.0, 2 if name == "module:2" else 1, 16 if name == "module:L16" else None)
         else:
             results[name] = bench.run_workload(name, 12.0 if name == head_name else 5.0)
     if bench.rank == 0:

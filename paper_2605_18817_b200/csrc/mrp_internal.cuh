@@ -244,6 +244,13 @@ cudaError_t tc_linear3(Ctx *c, const __nv_bfloat16 *a, int n, int n_in, const vo
                        cudaStream_t st);
 cudaError_t tc_gate_up(Ctx *c, const __nv_bfloat16 *a, int n, int n_in, const void *w_gate, const void *w_up, int F,
                        const float *sumsq, int n_ss, __nv_bfloat16 *act, int32_t *user_status, cudaStream_t st);
+// Few-row tensor-core products on the caller's own operands (n <= 64 rows; lo rows sk_head_pad(n) rows behind the
+// hi rows): see tc_skinny.cu.
+cudaError_t sk_linear(Ctx *c, const __nv_bfloat16 *a, int n, int n_in, const void *w, int n_out, const float *sumsq,
+                      int n_ss, float *out, bool accumulate, const void *gamma_next, __nv_bfloat16 *xg_next,
+                      float *sumsq_out, int *n_ss_out, int32_t *user_status, cudaStream_t st);
+cudaError_t sk_gate_up(Ctx *c, const __nv_bfloat16 *a, int n, int n_in, const void *w_gate, const void *w_up, int F,
+                       const float *sumsq, int n_ss, __nv_bfloat16 *act, int32_t *user_status, cudaStream_t st);
 // The same for the CUDA-core family (operand rows: fp32 xt).
 cudaError_t simt_lm_tail(Ctx *c, const float *logits0, const int32_t *row_index, int M, int K,
                          const mrp_draft_out &out, cudaStream_t st);

@@ -1282,6 +1282,14 @@ __global__ void mod_operand_kernel(const float *__restrict__ h_state, const T *_
     }
 }
 
+// Rows every region of the module workspace is sized for: the positions of a call (max_seqs * block_len), rounded up
+// to the row padding of the few-row tensor-core kernels where those may serve the call.
+static size_t module_cap_rows(const mrp_config &cfg)
+{
+    const size_t cap = (size_t)cfg.max_seqs * cfg.block_len;
+    return cap <= 64 ? (size_t)sk_head_pad((int)cap) : cap;
+}
+
 // ---- the module step as ONE kernel, for a handful of positions -----------------------------------
 // With n = B * L <= 4 positions every matrix of the module is a matrix-vector product bound by its own weight
 // stream (269 MB per step at d = 2048, F = 4096, D = 3), and a kernel per product leaves the stream idle
@@ -1700,7 +1708,7 @@ static cudaError_t module_fused_t(Ctx *c, const int32_t *tokens, const void *hid
     }
     p.first_step = first_step ? 1 : 0; p.mask_token = w.mask_token; p.emb_rows = w.emb_rows; p.n_layers = w.n_layers;
     p.n = n; p.B = B; p.L = L; p.d = d; p.F = F; p.H = w.n_attn_heads; p.eps = c->cfg.rms_eps;
-    const size_t cap = (size_t)c->cfg.max_seqs * c->cfg.block_len;
+    const size_t cap = module_cap_rows(c->cfg);
     char *ws = c->module_ws;
     auto take = [&](size_t bytes) { char *p0 = ws; ws += align_up(bytes, 256); return (float *)p0; };
     take(cap * 2 * d * 4);                 // (the concatenated rows of the separate kernels)
@@ -1741,10 +1749,10 @@ static cudaError_t module_fused_t(Ctx *c, const int32_t *tokens, const void *hid
 // operand rows, fp32 accumulation, RMSNorm folded in as gamma on the operand and 1 / rms on the result; a product
 // that completes z writes the next product's operand and its partial sums of squares itself); the embedding
 // fusion in front and the attention stay on the CUDA cores.
-// bf16 hi + lo rows of [h_i ; emb[x_i]]: the hi rows [n, 2 d], the lo rows n rows further on.
+// bf16 hi + lo rows of [h_i ; emb[x_i]]: the hi rows [n, 2 d], the lo rows lo_rows rows further on.
 __global__ void mod_cat_split_kernel(const float *h_state, const __nv_bfloat16 *__restrict__ hidden0, int first_step,
                                      const int32_t *__restrict__ tokens, const __nv_bfloat16 *__restrict__ emb, int mask_token,
-                                     int emb_rows, int n, int d, float *h_out /* = h_state */, __nv_bfloat16 *__restrict__ cat,
+                                     int emb_rows, int lo_rows, int d, float *h_out /* = h_state */, __nv_bfloat16 *__restrict__ cat,
                                      int32_t *__restrict__ status, int32_t *__restrict__ user_status)
 {
     pdl_trigger();
@@ -1759,7 +1767,7 @@ __global__ void mod_cat_split_kernel(const float *h_state, const __nv_bfloat16 *
         tok = -1;
     }
     if (tok < 0) tok = mask_token;
-    __nv_bfloat16 *hi = cat + (size_t)i * 2 * d, *lo = cat + ((size_t)n + i) * 2 * d;
+    __nv_bfloat16 *hi = cat + (size_t)i * 2 * d, *lo = cat + ((size_t)lo_rows + i) * 2 * d;
     for (int j = threadIdx.x; j < d; j += blockDim.x) {
         const float h = first_step ? __bfloat162float(hidden0[(size_t)i * d + j]) : h_state[(size_t)i * d + j];
         if (first_step) h_out[(size_t)i * d + j] = h;
@@ -1793,7 +1801,7 @@ static cudaError_t module_body_tc(Ctx *c, const int32_t *tokens, const void *hid
 {
     const mrp_module_weights &w = c->module;
     const int d = c->cfg.d, F = c->cfg.d_ff, n = B * L, dh = d / w.n_attn_heads;
-    const size_t cap = (size_t)c->cfg.max_seqs * c->cfg.block_len;
+    const size_t cap = module_cap_rows(c->cfg);
     char *ws = c->module_ws;
     auto take = [&](size_t bytes) { char *p0 = ws; ws += align_up(bytes, 256); return p0; };
     // the regions of the fp32 path hold the bf16 hi + lo operands here (same bytes: two halves of two bytes)
@@ -1807,14 +1815,48 @@ static cudaError_t module_body_tc(Ctx *c, const int32_t *tokens, const void *hid
     float *sumsq = (float *)(c->ws + c->lay.sumsq);
     int32_t *status = (int32_t *)(c->ws + c->lay.status);
     const bool pdl = !(c->cfg.flags & MRP_FLAG_NO_PDL);
+    // where the lo rows of an operand sit behind its hi rows: the few-row kernels fetch both with one TMA box
+    const bool few = sk_head_rows_ok(n) && sk_heads_ok(c->cfg) && (size_t)sk_head_pad(n) <= cap &&
+                     !(c->cfg.flags & MRP_FLAG_ROW_MAJOR_ONLY);
+    const int lo_rows = few ? sk_head_pad(n) : n;
     cudaError_t e = launch_k(mod_cat_split_kernel, dim3(n), dim3(256), 0, st, pdl, (const float *)h_state,
                              (const __nv_bfloat16 *)hidden0, first_step ? 1 : 0, tokens, (const __nv_bfloat16 *)w.emb, w.mask_token,
-                             w.emb_rows, n, d, h_state, cat16, status, out.status);
+                             w.emb_rows, lo_rows, d, h_state, cat16, status, out.status);
     c->launches++;
     // Every product that completes z also writes the next product's operand (z * next norm weight, hi + lo) and
     // its partial sums of squares: no kernel between them.
     int n_ss = 1;
     const void *g_first = w.n_layers > 0 ? w.layers[0].g_attn : nullptr;
+    if (few) {
+        // up to 64 positions: the few-row kernels (weight rows on the MMA M axis, contraction split over CTAs), whose
+        // tiles stream the weights once whatever the number of positions.  Their per-tile arrival counters must be
+        // zero at the first launch (every launch leaves them at zero again).
+        if (e == cudaSuccess) e = cudaMemsetAsync(c->ws + c->lay.sk_counters, 0, (size_t)kSkMaxTiles * 4, st);
+        if (e == cudaSuccess)
+            e = sk_linear(c, cat16, n, 2 * d, w.w_proj, d, nullptr, 1, z, false, g_first, g_first ? xa : nullptr, sumsq, &n_ss,
+                          out.status, st);
+        for (int l = 0; l < w.n_layers && e == cudaSuccess; ++l) {
+            const mrp_module_layer &y = w.layers[l];
+            e = sk_linear(c, xa, n, d, y.w_q, d, sumsq, n_ss, q, false, nullptr, nullptr, nullptr, nullptr, out.status, st);
+            if (e == cudaSuccess)
+                e = sk_linear(c, xa, n, d, y.w_k, d, sumsq, n_ss, k, false, nullptr, nullptr, nullptr, nullptr, out.status, st);
+            if (e == cudaSuccess)
+                e = sk_linear(c, xa, n, d, y.w_v, d, sumsq, n_ss, v, false, nullptr, nullptr, nullptr, nullptr, out.status, st);
+            if (e == cudaSuccess) {
+                e = launch_k(mod_attention_kernel, dim3(B, w.n_attn_heads), dim3(128), (size_t)4 * L * 4, st, pdl, (const float *)q,
+                             (const float *)k, (const float *)v, L, d, dh, (float *)nullptr, xb, lo_rows);
+                c->launches++;
+            }
+            if (e == cudaSuccess)
+                e = sk_linear(c, xb, n, d, y.w_o, d, nullptr, 1, z, true, y.g_mlp, xa, sumsq, &n_ss, out.status, st);
+            if (e == cudaSuccess) e = sk_gate_up(c, xa, n, d, y.w_gate, y.w_up, F, sumsq, n_ss, act16, out.status, st);
+            const void *g_next = l + 1 < w.n_layers ? w.layers[l + 1].g_attn : nullptr;
+            if (e == cudaSuccess)
+                e = sk_linear(c, act16, n, F, y.w_down, d, nullptr, 1, z, true, g_next, g_next ? xa : nullptr, sumsq, &n_ss,
+                              out.status, st);
+        }
+        return e;
+    }
     if (e == cudaSuccess)
         e = tc_linear(c, cat16, n, 2 * d, w.w_proj, d, nullptr, 1, z, false, out.status, st, g_first, g_first ? xa : nullptr,
                       sumsq, &n_ss);
@@ -1840,7 +1882,7 @@ static cudaError_t module_body_tc(Ctx *c, const int32_t *tokens, const void *hid
 size_t module_workspace_bytes(const mrp_config &cfg, int n_layers)
 {
     (void)n_layers;
-    const size_t n = (size_t)cfg.max_seqs * cfg.block_len, d = (size_t)cfg.d, F = (size_t)cfg.d_ff;
+    const size_t n = module_cap_rows(cfg), d = (size_t)cfg.d, F = (size_t)cfg.d_ff;
     return align_up(n * 2 * d * 4, 256) + 6 * align_up(n * d * 4, 256) + align_up(n * F * 4, 256);
 }
 
@@ -1851,7 +1893,7 @@ static cudaError_t module_step_t(Ctx *c, const int32_t *tokens, const void *hidd
 {
     const mrp_module_weights &w = c->module;
     const int d = c->cfg.d, F = c->cfg.d_ff, n = B * L, dh = d / w.n_attn_heads;
-    const size_t cap = (size_t)c->cfg.max_seqs * c->cfg.block_len;
+    const size_t cap = module_cap_rows(c->cfg);
     char *ws = c->module_ws;
     auto take = [&](size_t bytes) { char *p0 = ws; ws += align_up(bytes, 256); return (float *)p0; };
     float *cat = take(cap * 2 * d * 4), *z = take(cap * d * 4), *nn = take(cap * d * 4), *q = take(cap * d * 4);

@@ -35,7 +35,7 @@ constexpr int kAuxVote = 768;              // int: epilogue warps' common decisi
 constexpr int kAuxSsq = 1024;              // float[4][128]
 constexpr int kAuxExch = 4096;             // float[16][64]
 
-enum { SK_GU = 0, SK_DN = 1, SK_LM = 2 };
+enum { SK_GU = 0, SK_DN = 1, SK_LM = 2, SK_LIN = 3 };
 
 struct SkMaps {
     CUtensorMap x;      // activation operand, box = r_pad rows
@@ -79,6 +79,11 @@ struct SkParams {
     __half *xt16_k;      // optional: the same rows rounded once to fp16 (fp16 LM-head mode)
     float *sumsq_out;
     float *hidden_out;
+    // LIN: a plain product on operands of the caller's own (the module): out[m, j] (+)= rstd(m) * sum, rstd from
+    // `sumsq` (as GU) or 1; with xg_next also out * gamma_next as the next operand and partial sums of squares of out
+    float *lin_out;
+    int lin_n_out;       // row pitch of lin_out and of xg_next
+    int lin_accumulate;
     int32_t *status;
     int32_t *user_status;
     // LM with 8-bit weights: per-vocabulary-row scales of the e4m3 copy of W_lm, per-row-step scales of
@@ -286,11 +291,12 @@ sk_gemm_kernel(const __grid_constant__ SkMaps maps, const SkParams p)
                 // -1: no base logits for this row-step (none given, or the caller's index is out of range)
                 rowoff_s[t] = (p.logits0 && (!p.row_index || row_ok(idx, p.n_rows_in))) ? (long long)idx * p.V : -1ll;
             }
-        } else if (KIND == SK_GU) {
+        } else if (KIND == SK_GU || KIND == SK_LIN) {
             if (t < p.M) {
                 float s = 0.f;
-                for (int i = 0; i < p.n_ss; ++i) s += p.sumsq[(size_t)i * p.M + t];
-                rstd_s[t] = rsqrtf(s / (float)p.d + p.eps);
+                if (KIND == SK_GU || p.sumsq)
+                    for (int i = 0; i < p.n_ss; ++i) s += p.sumsq[(size_t)i * p.M + t];
+                rstd_s[t] = (KIND == SK_GU || p.sumsq) ? rsqrtf(s / (float)p.d + p.eps) : 1.f;
             }
         }
         epi_sync();
@@ -446,7 +452,7 @@ sk_gemm_kernel(const __grid_constant__ SkMaps maps, const SkParams p)
             }
             if (finisher) {
                 const float *first = p.scratch + ((size_t)tile * p.n_split * RP) * 128;
-                const float gm = (KIND == SK_DN && valid && p.xg_next) ? __bfloat162float(p.gamma_next[wrow]) : 0.f;
+                const float gm = ((KIND == SK_DN || KIND == SK_LIN) && valid && p.xg_next) ? __bfloat162float(p.gamma_next[wrow]) : 0.f;
 #pragma unroll 1
                 for (int ch = 0; ch < n_ch; ++ch) {
                     const int c0 = ch * 16;
@@ -497,6 +503,32 @@ sk_gemm_kernel(const __grid_constant__ SkMaps maps, const SkParams p)
                             }
                         }
                         epi_sync();
+                    } else if (KIND == SK_LIN) {
+                        float sq[16];
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) sq[j] = 0.f;
+                        if (valid) {
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) {
+                                if (c0 + j < p.M) {
+                                    const size_t o = (size_t)(c0 + j) * p.lin_n_out + wrow;
+                                    float h = v[j] * rstd_s[c0 + j];
+                                    if (p.lin_accumulate) h += p.lin_out[o];
+                                    p.lin_out[o] = h;
+                                    sq[j] = h * h;
+                                    if (p.xg_next) store_hi_lo(p.xg_next + o, (size_t)p.lo_x * p.lin_n_out, h * gm);
+                                }
+                            }
+                        }
+                        if (p.xg_next) {
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) {
+                                float s = sq[j];
+#pragma unroll
+                                for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+                                if (lane == 0) ssq_s[q * 128 + c0 + j] = s;
+                            }
+                        }
                     } else {
                         float sq[16];
 #pragma unroll
@@ -526,7 +558,7 @@ sk_gemm_kernel(const __grid_constant__ SkMaps maps, const SkParams p)
                     }
                 }
             }
-            if (KIND == SK_DN) {
+            if (KIND == SK_DN || (KIND == SK_LIN && p.xg_next)) {
                 epi_sync();
                 // one slice of sums of squares per weight tile, written by the CTA that finished it
                 if (finisher) {
@@ -804,6 +836,61 @@ cudaError_t sk_down(Ctx *c, int k, int M, int K, const mrp_draft_out &out, cudaS
         return note_err(c, cudaErrorInvalidValue, "tensor map (down, few rows)");
     c->launches++;
     return note_err(c, sk_launch_rp<SK_DN>(maps, p, grid, st, pdl, false), "down kernel (few rows)");
+}
+
+// Few-row products on operands of the caller's own (the module; n <= 64 rows).  Operand a: bf16 hi rows [n, n_in]
+// with the lo rows sk_head_pad(n) rows further on.
+// out[n, n_out] (+)= rstd(row) * (A W^T), rstd from sumsq[n_ss, n] (nullptr: 1); with xg_next also out * gamma_next
+// in operand form and partial sums of squares of out to sumsq_out[*n_ss_out, n].
+cudaError_t sk_linear(Ctx *c, const __nv_bfloat16 *a, int n, int n_in, const void *w, int n_out, const float *sumsq,
+                      int n_ss, float *out, bool accumulate, const void *gamma_next, __nv_bfloat16 *xg_next,
+                      float *sumsq_out, int *n_ss_out, int32_t *user_status, cudaStream_t st)
+{
+    const TcState *s = (const TcState *)c->tc_state;
+    SkParams p;
+    memset(&p, 0, sizeof(p));
+    p.M = n; p.d = n_in; p.F = n_in;
+    p.status = (int32_t *)(c->ws + c->lay.status); p.user_status = user_status;
+    p.units_total = n_out / 16; p.k_chunks = n_in / kBK; p.r_pad = sk_head_pad(n); p.w_rows = n_out;
+    p.lo_x = p.r_pad; p.lo_xt = p.r_pad;
+    p.sumsq = sumsq; p.n_ss = n_ss; p.eps = c->cfg.rms_eps;
+    p.lin_out = out; p.lin_n_out = n_out; p.lin_accumulate = accumulate ? 1 : 0;
+    p.gamma_next = (const __nv_bfloat16 *)gamma_next; p.xg_next = xg_next; p.sumsq_out = sumsq_out;
+    sk_finish_shape(p, 0);
+    const int n_tiles = (n_out + 127) / 128;
+    const int grid = sk_split(c, p, n_tiles);
+    if (n_ss_out) *n_ss_out = n_tiles;
+    SkMaps maps;
+    memset(&maps, 0, sizeof(maps));
+    if (!make_map(s, &maps.x, a, n_in, 2 * (uint64_t)p.r_pad, 2 * p.r_pad) || !sk_weight_maps(s, maps, 0, w, n_in, n_out, 16, p))
+        return note_err(c, cudaErrorInvalidValue, "tensor map (module product, few rows)");
+    c->launches++;
+    return note_err(c, sk_launch_rp<SK_LIN>(maps, p, grid, st, !(c->cfg.flags & MRP_FLAG_NO_PDL), false),
+                    "module product kernel (few rows)");
+}
+
+// act[n, F] = silu(rstd * A Wg^T) * (rstd * A Wu^T) in operand form (lo rows sk_head_pad(n) rows further on).
+cudaError_t sk_gate_up(Ctx *c, const __nv_bfloat16 *a, int n, int n_in, const void *w_gate, const void *w_up, int F,
+                       const float *sumsq, int n_ss, __nv_bfloat16 *act, int32_t *user_status, cudaStream_t st)
+{
+    const TcState *s = (const TcState *)c->tc_state;
+    SkParams p;
+    memset(&p, 0, sizeof(p));
+    p.M = n; p.d = n_in; p.F = F;
+    p.status = (int32_t *)(c->ws + c->lay.status); p.user_status = user_status;
+    p.units_total = F / 8; p.k_chunks = n_in / kBK; p.r_pad = sk_head_pad(n); p.w_rows = F;
+    p.lo_x = p.r_pad; p.lo_xt = p.r_pad;
+    p.sumsq = sumsq; p.n_ss = n_ss; p.eps = c->cfg.rms_eps; p.act = act;
+    sk_finish_shape(p, 0);
+    const int grid = sk_split(c, p, F / 64);
+    SkMaps maps;
+    memset(&maps, 0, sizeof(maps));
+    if (!make_map(s, &maps.x, a, n_in, 2 * (uint64_t)p.r_pad, 2 * p.r_pad) ||
+        !sk_weight_maps(s, maps, 0, w_gate, n_in, F, 8, p) || !sk_weight_maps(s, maps, 1, w_up, n_in, F, 8, p))
+        return note_err(c, cudaErrorInvalidValue, "tensor map (module gate/up, few rows)");
+    c->launches++;
+    return note_err(c, sk_launch_rp<SK_GU>(maps, p, grid, st, !(c->cfg.flags & MRP_FLAG_NO_PDL), false),
+                    "module gate/up kernel (few rows)");
 }
 
 cudaError_t sk_lm(Ctx *c, const float *logits0, const int32_t *row_index, int M, int K,
