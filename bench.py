@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of the MRP drafting step on B200.
 
-    python bench.py [--gpus N] [--steps S] [--warmup W] [--config all|0..3|sweep:M:K|sweep]
+    python bench.py [--gpus N] [--steps S] [--warmup W] [--config all|0..3|module|module:2|module:L16|sweep:M:K|sweep]
                     [--impl ours|reference]
 
 A step is one pass of the whole hot path over one batch of synthetic input: mrp_draft (row
@@ -62,6 +62,8 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="all",
                     help="all = the five configurations in one line (default); 0..3 = one configuration; "
+                         "module / module:2 / module:L16 = the token-conditioned module at the decode shape, at "
+                         "spec_8b's shape, at the decode shape with one block of 16 positions; "
                          "sweep:M:K = one roofline-sweep point; sweep = all 21 points, one line each")
     ap.add_argument("--min-seconds", type=float, default=1.0,
                     help="GPU time per workload spent in timed batches of --steps steps")
