@@ -249,6 +249,9 @@ cudaError_t tc_gate_up(Ctx *c, const __nv_bfloat16 *a, int n, int n_in, const vo
 cudaError_t sk_linear(Ctx *c, const __nv_bfloat16 *a, int n, int n_in, const void *w, int n_out, const float *sumsq,
                       int n_ss, float *out, bool accumulate, const void *gamma_next, __nv_bfloat16 *xg_next,
                       float *sumsq_out, int *n_ss_out, int32_t *user_status, cudaStream_t st);
+cudaError_t sk_linear3(Ctx *c, const __nv_bfloat16 *a, int n, int n_in, const void *w0, const void *w1, const void *w2,
+                       int n_out, const float *sumsq, int n_ss, float *out0, float *out1, float *out2, int32_t *user_status,
+                       cudaStream_t st);
 cudaError_t sk_gate_up(Ctx *c, const __nv_bfloat16 *a, int n, int n_in, const void *w_gate, const void *w_up, int F,
                        const float *sumsq, int n_ss, __nv_bfloat16 *act, int32_t *user_status, cudaStream_t st);
 // The same for the CUDA-core family (operand rows: fp32 xt).

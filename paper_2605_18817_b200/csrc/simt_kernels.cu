@@ -1837,11 +1837,7 @@ static cudaError_t module_body_tc(Ctx *c, const int32_t *tokens, const void *hid
                           out.status, st);
         for (int l = 0; l < w.n_layers && e == cudaSuccess; ++l) {
             const mrp_module_layer &y = w.layers[l];
-            e = sk_linear(c, xa, n, d, y.w_q, d, sumsq, n_ss, q, false, nullptr, nullptr, nullptr, nullptr, out.status, st);
-            if (e == cudaSuccess)
-                e = sk_linear(c, xa, n, d, y.w_k, d, sumsq, n_ss, k, false, nullptr, nullptr, nullptr, nullptr, out.status, st);
-            if (e == cudaSuccess)
-                e = sk_linear(c, xa, n, d, y.w_v, d, sumsq, n_ss, v, false, nullptr, nullptr, nullptr, nullptr, out.status, st);
+            e = sk_linear3(c, xa, n, d, y.w_q, y.w_k, y.w_v, d, sumsq, n_ss, q, k, v, out.status, st);
             if (e == cudaSuccess) {
                 e = launch_k(mod_attention_kernel, dim3(B, w.n_attn_heads), dim3(128), (size_t)4 * L * 4, st, pdl, (const float *)q,
                              (const float *)k, (const float *)v, L, d, dh, (float *)nullptr, xb, lo_rows);

@@ -84,6 +84,10 @@ struct SkParams {
     float *lin_out;
     int lin_n_out;       // row pitch of lin_out and of xg_next
     int lin_accumulate;
+    // LIN over lin_nw = 3 matrices of one shape sharing the operand rows (q, k, v): lin_tiles_w tiles each, through
+    // maps w[0], w[1], w[2], results to lin_out, lin_out1, lin_out2
+    int lin_nw, lin_tiles_w;
+    float *lin_out1, *lin_out2;
     int32_t *status;
     int32_t *user_status;
     // LM with 8-bit weights: per-vocabulary-row scales of the e4m3 copy of W_lm, per-row-step scales of
@@ -143,6 +147,7 @@ sk_gemm_kernel(const __grid_constant__ SkMaps maps, const SkParams p)
         const int cps = (p.k_chunks + p.n_split - 1) / p.n_split;
         units = 8;
         u0 = (cta / p.n_split) * 8;
+        if (KIND == SK_LIN && p.lin_nw == 3) u0 = ((cta / p.n_split) % p.lin_tiles_w) * 8;
         kc0 = (cta % p.n_split) * cps;
         kc1 = min(p.k_chunks, kc0 + cps);
     }
@@ -197,7 +202,8 @@ sk_gemm_kernel(const __grid_constant__ SkMaps maps, const SkParams p)
                         tma_load_2d_hint(sw + b * sub_bytes, &maps.w[0], kx, ut * 8, full_bar(s), pol_w);
                         tma_load_2d_hint(sw + b * sub_bytes + 64 * 128, &maps.w[3], kx, ut * 8, full_bar(s), pol_w);
                     } else {
-                        tma_load_2d_hint(sw + b * sub_bytes, &maps.w[tile_map(h)], kx, ut * 16, full_bar(s), pol_w);
+                        const int mi = (KIND == SK_LIN && p.lin_nw == 3) ? (cta / p.n_split) / p.lin_tiles_w : tile_map(h);
+                        tma_load_2d_hint(sw + b * sub_bytes, &maps.w[mi], kx, ut * 16, full_bar(s), pol_w);
                     }
                 }
             };
@@ -418,6 +424,8 @@ sk_gemm_kernel(const __grid_constant__ SkMaps maps, const SkParams p)
             const bool valid = KIND == SK_GU ? (t < 64 && wrow < p.w_rows) : (wrow < p.w_rows);
             const int n_ch = (p.M + 15) >> 4;
             const int tile = cta / p.n_split;
+            const int which = (KIND == SK_LIN && p.lin_nw == 3) ? tile / p.lin_tiles_w : 0;
+            float *lin_dst = which == 0 ? p.lin_out : which == 1 ? p.lin_out1 : p.lin_out2;
             bool ok = __all_sync(0xffffffffu, mbar_wait(tfull_bar(0), 0u, abort_flag, p));
             // the four warps meet at barriers below: they must agree on going on
             if (!ok && lane == 0) *vote_s = 1;
@@ -513,8 +521,8 @@ sk_gemm_kernel(const __grid_constant__ SkMaps maps, const SkParams p)
                                 if (c0 + j < p.M) {
                                     const size_t o = (size_t)(c0 + j) * p.lin_n_out + wrow;
                                     float h = v[j] * rstd_s[c0 + j];
-                                    if (p.lin_accumulate) h += p.lin_out[o];
-                                    p.lin_out[o] = h;
+                                    if (p.lin_accumulate) h += lin_dst[o];
+                                    lin_dst[o] = h;
                                     sq[j] = h * h;
                                     if (p.xg_next) store_hi_lo(p.xg_next + o, (size_t)p.lo_x * p.lin_n_out, h * gm);
                                 }
@@ -867,6 +875,34 @@ cudaError_t sk_linear(Ctx *c, const __nv_bfloat16 *a, int n, int n_in, const voi
     c->launches++;
     return note_err(c, sk_launch_rp<SK_LIN>(maps, p, grid, st, !(c->cfg.flags & MRP_FLAG_NO_PDL), false),
                     "module product kernel (few rows)");
+}
+
+// Three such products over the same operand rows in one launch (q, k, v): out_i = rstd(row) * (A W_i^T).
+cudaError_t sk_linear3(Ctx *c, const __nv_bfloat16 *a, int n, int n_in, const void *w0, const void *w1, const void *w2,
+                       int n_out, const float *sumsq, int n_ss, float *out0, float *out1, float *out2, int32_t *user_status,
+                       cudaStream_t st)
+{
+    const TcState *s = (const TcState *)c->tc_state;
+    SkParams p;
+    memset(&p, 0, sizeof(p));
+    p.M = n; p.d = n_in; p.F = n_in;
+    p.status = (int32_t *)(c->ws + c->lay.status); p.user_status = user_status;
+    p.units_total = n_out / 16; p.k_chunks = n_in / kBK; p.r_pad = sk_head_pad(n); p.w_rows = n_out;
+    p.lo_x = p.r_pad; p.lo_xt = p.r_pad;
+    p.sumsq = sumsq; p.n_ss = n_ss; p.eps = c->cfg.rms_eps;
+    p.lin_out = out0; p.lin_out1 = out1; p.lin_out2 = out2; p.lin_n_out = n_out;
+    sk_finish_shape(p, 0);
+    const int n_tiles = (n_out + 127) / 128;
+    p.lin_nw = 3; p.lin_tiles_w = n_tiles;
+    const int grid = sk_split(c, p, 3 * n_tiles);
+    SkMaps maps;
+    memset(&maps, 0, sizeof(maps));
+    if (!make_map(s, &maps.x, a, n_in, 2 * (uint64_t)p.r_pad, 2 * p.r_pad) || !make_map(s, &maps.w[0], w0, n_in, n_out, 128) ||
+        !make_map(s, &maps.w[1], w1, n_in, n_out, 128) || !make_map(s, &maps.w[2], w2, n_in, n_out, 128))
+        return note_err(c, cudaErrorInvalidValue, "tensor map (module q, k, v, few rows)");
+    c->launches++;
+    return note_err(c, sk_launch_rp<SK_LIN>(maps, p, grid, st, !(c->cfg.flags & MRP_FLAG_NO_PDL), false),
+                    "module q, k, v kernel (few rows)");
 }
 
 // act[n, F] = silu(rstd * A Wg^T) * (rstd * A Wu^T) in operand form (lo rows sk_head_pad(n) rows further on).
