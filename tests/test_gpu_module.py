@@ -123,3 +123,54 @@ def test_module_step_checks_tokens_and_needs_an_attached_module(B, L):
     torch.cuda.synchronize()
     assert int(ref.status.item()) == 0 and torch.equal(ref.conf, out.conf) and torch.equal(ref.token, out.token)
     binding.mrp_destroy(ctx)
+
+
+@pytest.mark.parametrize("which,L,blocks_checked", [
+    (1, 4, 1),      # the decode shape, one block of 4: the step as one cooperative CUDA-core kernel
+    (1, 16, 1),     # the same with the paper's block of 16: products on the few-row tensor-core kernels
+    (2, 4, 2),      # 32 blocks of 4 at d = 4096: products on the row-major tensor-core kernel; oracle on two blocks
+])
+def test_module_step_at_the_benchmark_shapes(which, L, blocks_checked):
+    """One module step at the shapes bench.py times (D = 3, 128 features per attention head), in the launch
+    configuration it times, against the oracle on the first blocks (blocks do not see one another: Sec. 3.2,
+    block-local attention): h <- h + Delta at every position of those blocks, statistics of their masked rows."""
+    cfg = dict(synth.CONFIGS[which], L=L)
+    d, F, V, B = cfg["d"], cfg["F"], cfg["V"], cfg["B"]
+    n, n_attn, D = B * L, d // 128, 3
+    w = synth.make_weights(d, F, V, 1, "bf16", cfg["seed"])
+    heads_dev, w_lm = harness.upload_weights(w, DEV)
+    _, inp = synth.make_config(cfg, w, logits_fn=harness.device_logits_fn(w_lm))
+    mw = synth.make_module_weights(d, F, V, D, n_attn, "bf16", 11, std=0.02 if d < 4096 else 0.01)
+    ctx = binding.mrp_create(d, F, V, heads_dev, w_lm, max_rows=n, max_seqs=B, block_len=L)
+    up = lambda a: harness.to_device(a, "bf16", DEV)
+    binding.mrp_module_attach(ctx, up(mw.emb), up(mw.w_proj), [{k: up(v) for k, v in lay.items()} for lay in mw.layers],
+                              n_attn, mw.mask_token)
+    tokens = np.full(n, -1, np.int32)
+    tokens[::L] = 17                                   # one position of every block already revealed
+    ri = np.flatnonzero(tokens < 0).astype(np.int32)
+    M = ri.size
+    hid0 = harness.to_device(inp.hidden, "bf16", DEV)
+    l0 = torch.from_numpy(inp.logits0).to(DEV)
+    h_state = torch.empty((n, d), device=DEV, dtype=torch.float32)
+    out = harness.alloc_draft_out(M, 1, V, d, DEV, hidden=True)
+    binding.mrp_module_step(ctx, torch.from_numpy(tokens).to(DEV), hid0, h_state, l0, torch.from_numpy(ri).to(DEV), M, B, L,
+                            True, out.conf, out.lse, out.token, margin=out.margin, hidden_out=out.hidden, status=out.status)
+    torch.cuda.synchronize()
+    assert int(out.status.item()) == 0
+    ns = blocks_checked * L
+    ri_s = np.flatnonzero(tokens[:ns] < 0).astype(np.int32)
+    dh, dl = oracle.module(inp.hidden[:ns], tokens[:ns], blocks_checked, L, mw.emb, mw.w_proj, mw.layers, w.w_lm, n_attn,
+                           mw.mask_token, row_index=ri_s)
+    assert np.abs(dh).max() > 1e-2
+    h_ref = inp.hidden[:ns].astype(np.float64) + dh
+    assert np.abs(h_state[:ns].cpu().numpy() - h_ref).max() <= 1e-3 * max(1.0, np.abs(h_ref).max())
+    conf, lse, tok, margin = oracle.stats(inp.logits0[ri_s].astype(np.float64) + dl)
+    m_s = ri_s.size                                     # the checked blocks' masked rows come first in ri
+    g_conf, g_lse, g_tok = (t.cpu().numpy() for t in (out.conf, out.lse, out.token))
+    assert np.abs(g_conf[1, :m_s] - conf).max() <= TOL["bf16"] and np.abs(g_lse[1, :m_s] - lse).max() <= TOL["bf16"]
+    clear = margin > 1e-2
+    assert np.array_equal(g_tok[1, :m_s][clear], tok[clear])
+    assert np.abs(out.hidden[:m_s].cpu().numpy() - h_ref[ri_s]).max() <= 1e-3 * max(1.0, np.abs(h_ref).max())
+    binding.mrp_destroy(ctx)
+    del ctx, w_lm, heads_dev, hid0, l0
+    torch.cuda.empty_cache()
