@@ -800,8 +800,12 @@ def main():
     head_name = HEADLINE if args.config == "all" else args.config
     results = {}
     for name in names:
-        if name in ("module", "module:1", "module:2", "module:L16"):
-            results[name] = run_module_workload(bench, 5.0, 2 if name == "module:2" else 1, 16 if name == "module:L16" else None)
+        if name == "module" or name.startswith("module:"):
+            # module[:1|:2][:L<block length>], e.g. module:L16 (decode shape, one block of 16), module:2:L2
+            parts = name.split(":")[1:]
+            which = 2 if "2" in parts else 1
+            blen = [int(x[1:]) for x in parts if x.startswith("L")]
+            results[name] = run_module_workload(bench, 5.0, which, blen[0] if blen else None)
         else:
             results[name] = bench.run_workload(name, 12.0 if name == head_name else 5.0)
     if bench.rank == 0:

@@ -73,7 +73,8 @@ typedef enum { MRP_F32 = 0, MRP_BF16 = 1 } mrp_dtype;
 #define MRP_FLAG_ROW_MAJOR_ONLY 4   /* tensor-core family: never use the few-row kernels  */
 #define MRP_FLAG_NO_CHAIN 16    /* run every step as a kernel of its own: the tensor-core family's head
                                   chain of a few-row call as one kernel per GEMM instead of one
-                                  persistent kernel; the CUDA-core family's pass over a few short rows
+                                  persistent kernel (likewise a layer of the token-conditioned module);
+                                  the CUDA-core family's pass over a few short rows
                                   (at most 8 rows, d <= 512, (K + 1) * M <= 32) as one kernel per step
                                   instead of one cooperative kernel for the whole mrp_draft call      */
 #define MRP_FLAG_REQUIRE_TENSOR_CORES 32   /* bf16 context: mrp_create fails with MRP_ERR_UNSUPPORTED

@@ -1190,8 +1190,8 @@ __global__ void mod_attention_kernel(const float *__restrict__ q, const float *_
     for (int i = warp; i < L; i += n_warps) {
         const float *qi = q + ((size_t)b * L + i) * d + (size_t)hd * dh;
         float mx = -INFINITY;
-        if (L < 32) {
-            // short blocks: lanes over the head's features (coalesced rows), one warp sum per key
+        if (L <= 64) {
+            // blocks of up to 64 positions: lanes over the head's features (coalesced rows), one warp sum per key
             for (int j = 0; j < L; ++j) {
                 const float *kj = k + ((size_t)b * L + j) * d + (size_t)hd * dh;
                 float sdot = 0.f;
@@ -1287,7 +1287,7 @@ __global__ void mod_operand_kernel(const float *__restrict__ h_state, const T *_
 static size_t module_cap_rows(const mrp_config &cfg)
 {
     const size_t cap = (size_t)cfg.max_seqs * cfg.block_len;
-    return cap <= 64 ? (size_t)sk_head_pad((int)cap) : cap;
+    return cap <= 128 ? (size_t)sk_head_pad((int)cap) : cap;
 }
 
 // ---- the module step as ONE kernel, for a handful of positions -----------------------------------
@@ -1818,7 +1818,13 @@ static cudaError_t module_body_tc(Ctx *c, const int32_t *tokens, const void *hid
     // where the lo rows of an operand sit behind its hi rows: the few-row kernels fetch both with one TMA box
     const bool few = sk_head_rows_ok(n) && sk_heads_ok(c->cfg) && (size_t)sk_head_pad(n) <= cap &&
                      !(c->cfg.flags & MRP_FLAG_ROW_MAJOR_ONLY);
-    const int lo_rows = few ? sk_head_pad(n) : n;
+    // up to 64 positions: a layer (the first with the fusion projection) as one cooperative kernel, if the shape fits
+    // (at 128 positions and d = 4096 the row-major kernels are ahead: 0.52 against 0.76 ms per step of the module)
+    const bool chain = w.n_layers > 0 && n <= 64 && (size_t)sk_head_pad(n) <= cap && sk_heads_ok(c->cfg) &&
+                       !(c->cfg.flags & (MRP_FLAG_ROW_MAJOR_ONLY | MRP_FLAG_NO_CHAIN)) &&
+                       sk_module_layer(c, n, L, w.n_attn_heads, w.layers[0], w.w_proj, nullptr, nullptr, nullptr, nullptr, nullptr,
+                                       nullptr, nullptr, nullptr, 0, 1, nullptr, out.status, st, true) == cudaSuccess;
+    const int lo_rows = (few || chain) ? sk_head_pad(n) : n;
     cudaError_t e = launch_k(mod_cat_split_kernel, dim3(n), dim3(256), 0, st, pdl, (const float *)h_state,
                              (const __nv_bfloat16 *)hidden0, first_step ? 1 : 0, tokens, (const __nv_bfloat16 *)w.emb, w.mask_token,
                              w.emb_rows, lo_rows, d, h_state, cat16, status, out.status);
@@ -1827,6 +1833,16 @@ static cudaError_t module_body_tc(Ctx *c, const int32_t *tokens, const void *hid
     // its partial sums of squares: no kernel between them.
     int n_ss = 1;
     const void *g_first = w.n_layers > 0 ? w.layers[0].g_attn : nullptr;
+    if (chain) {
+        // the norms' sums of squares live in slots of the fixed-point array; the slot the first launch adds to is cleared here
+        if (e == cudaSuccess) e = cudaMemsetAsync(c->ws + c->lay.ssq_fix, 0, (size_t)5 * 128 * 8, st);
+        for (int l = 0; l < w.n_layers && e == cudaSuccess; ++l) {
+            const void *g_next = l + 1 < w.n_layers ? w.layers[l + 1].g_attn : nullptr;
+            e = sk_module_layer(c, n, L, w.n_attn_heads, w.layers[l], l == 0 ? w.w_proj : nullptr, cat16, xa, xb, act16, q, k, v, z,
+                                l & 1, 1 - (l & 1), g_next, out.status, st, false);
+        }
+        return e;
+    }
     if (few) {
         // up to 64 positions: the few-row kernels (weight rows on the MMA M axis, contraction split over CTAs), whose
         // tiles stream the weights once whatever the number of positions.  Their per-tile arrival counters must be

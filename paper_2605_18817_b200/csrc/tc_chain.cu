@@ -42,10 +42,11 @@ constexpr int kChTilesPerPhase = 448;      // arrival counters per phase
 constexpr int kChMaxPhases = 8;
 constexpr long long kBarrierCycles = 1000000000LL;   // bound on a grid-barrier wait (about 0.5 s)
 
-enum { CH_GU = 0, CH_DN = 1 };
+enum { CH_GU = 0, CH_DN = 1, CH_LIN = 2, CH_ATT = 3 };      // LIN, ATT: the module's phases (MOD instantiations)
 
 struct ChainMaps {
     CUtensorMap m[2 + 3 * 4];   // 0: head input (xg), 1: SwiGLU output (act), 2+3h: gate, 3+3h: up, 4+3h: down of head h
+                                // (a module layer: 0 xa, 1 act, 2 xb, 3-5 q k v, 6 o, 7 gate, 8 up, 9 down)
 };
 
 struct ChainPhase {
@@ -61,6 +62,16 @@ struct ChainPhase {
     __nv_bfloat16 *xt_k;
     __half *xt16_k;
     float *hidden_out;
+    // LIN (a plain product of the module): out[m, j] (+)= rstd(m) * sum, rstd from slot ssq_in of ssq_fix (< 0: 1);
+    // with xg_next also out * gamma_next in operand form and the sums of squares of out added to slot ssq_idx.
+    // lin3_tiles > 0: three matrices of lin3_tiles tiles each (maps map_w0, +1, +2; results lin_out, lin_out1, lin_out2)
+    float *lin_out, *lin_out1, *lin_out2;
+    int lin_acc, ssq_in, lin3_tiles;
+    // ATT (no product): block-local attention over q, k, v [M, d] (fp32) into att_out in operand form
+    const float *att_q, *att_k, *att_v;
+    __nv_bfloat16 *att_out;
+    int att_L, att_H;
+    int zero_slot0, zero_slot1;      // ssq_fix slots this phase clears for later phases of the launch (< 0: none)
 };
 
 struct ChainParams {
@@ -122,7 +133,9 @@ __device__ __forceinline__ bool grid_bar_wait(const unsigned int *bar, unsigned 
     return true;
 }
 
-template <int RP, int KC>
+// MOD: the instantiation that also knows the module's phase kinds (LIN, ATT); the head chain's own instantiations
+// compile none of that code.
+template <int RP, int KC, bool MOD = false>
 __global__ void __launch_bounds__(kChThreads, 1)
 sk_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainParams p)
 {
@@ -203,6 +216,10 @@ sk_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant__ 
                         if (ph.kind == CH_GU) {
                             tma_load_2d_hint(sw, &maps.m[ph.map_w0], col, tile * 64, full_bar(stage_of(n)), pol_w);
                             tma_load_2d_hint(sw + 64 * 128, &maps.m[ph.map_w1], col, tile * 64, full_bar(stage_of(n)), pol_w);
+                        } else if (MOD && ph.kind == CH_LIN && ph.lin3_tiles > 0) {
+                            const int which = tile / ph.lin3_tiles;
+                            tma_load_2d_hint(sw, &maps.m[ph.map_w0 + which], col, (tile - which * ph.lin3_tiles) * 128,
+                                             full_bar(stage_of(n)), pol_w);
                         } else {
                             tma_load_2d_hint(sw, &maps.m[ph.map_w0], col, tile * 128, full_bar(stage_of(n)), pol_w);
                         }
@@ -336,6 +353,16 @@ sk_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant__ 
                         const unsigned long long v = __ldcg(p.ssq_fix + ph.ssq_idx * 128 + t);
                         const float s = (float)((double)v * (1.0 / 16777216.0));
                         rstd_s[t] = rsqrtf(s / (float)p.d + p.eps);
+                    }
+                }
+                if (MOD && ph.kind == CH_LIN) {
+                    if (t < p.M) {
+                        float r = 1.f;
+                        if (ph.ssq_in >= 0) {
+                            const unsigned long long v = __ldcg(p.ssq_fix + ph.ssq_in * 128 + t);
+                            r = rsqrtf((float)((double)v * (1.0 / 16777216.0)) / (float)p.d + p.eps);
+                        }
+                        rstd_s[t] = r;
                     }
                 }
                 const int acc = n_acc & 1, use = n_acc >> 1;
@@ -478,6 +505,43 @@ sk_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant__ 
                                 }
                             }
                         }
+                    } else if (MOD && ph.kind == CH_LIN) {
+                        // a plain product: this CTA's rows of the tile, one output at a time from the parked slices
+                        const int which = ph.lin3_tiles > 0 ? tile / ph.lin3_tiles : 0;
+                        const int tile_w = ph.lin3_tiles > 0 ? tile - which * ph.lin3_tiles : tile;
+                        float *dst = which == 0 ? ph.lin_out : which == 1 ? ph.lin_out1 : ph.lin_out2;
+#pragma unroll 2
+                        for (int e = t; e < n_items; e += 128) {
+                            const int m = e / n_r, row = r0 + (e - m * n_r);
+                            const int j = tile_w * 128 + row;
+                            float sq = 0.f;
+                            if (j < ph.w_rows) {
+                                const size_t o = (size_t)m * ph.w_rows + j;
+                                float a = 0.f;
+                                for (int s0 = 0; s0 < ph.n_split; s0 += 8) {      // slice order; 8 slices' loads in flight
+                                    float as[8];
+#pragma unroll
+                                    for (int k = 0; k < 8; ++k)
+                                        as[k] = (s0 + k < ph.n_split) ? __ldcg(first + ((size_t)(s0 + k) * RP + m) * 128 + row) : 0.f;
+#pragma unroll
+                                    for (int k = 0; k < 8; ++k) a += as[k];
+                                }
+                                float h = a * rstd_s[m];
+                                if (ph.lin_acc) h += __ldcg(dst + o);
+                                dst[o] = h;
+                                sq = h * h;
+                                if (ph.xg_next) ch_store_hi_lo(ph.xg_next + o, (size_t)p.lo_x * ph.w_rows, h * __bfloat162float(ph.gamma_next[j]));
+                            }
+                            if (ph.xg_next) sq_s[e] = sq;        // (a share without a norm behind it may exceed the buffer)
+                        }
+                        if (ph.xg_next) {
+                            ch_epi_sync();
+                            for (int m = t; m < p.M; m += 128) {
+                                float s2 = 0.f;
+                                for (int r = 0; r < n_r; ++r) s2 += sq_s[m * n_r + r];
+                                atomicAdd(p.ssq_fix + ph.ssq_idx * 128 + m, (unsigned long long)__double2ll_rn((double)s2 * 16777216.0));
+                            }
+                        }
                     } else {
                         int n_sq = n_r;                      // entries of the buffer of squares per batch row
                         bool done = false;
@@ -570,6 +634,50 @@ sk_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant__ 
                     }
                 }
             }
+            if (MOD) {
+                if (cta == 0 && t < p.M) {          // sums of squares later phases of this launch add to start at zero
+                    if (ph.zero_slot0 >= 0) p.ssq_fix[ph.zero_slot0 * 128 + t] = 0ull;
+                    if (ph.zero_slot1 >= 0) p.ssq_fix[ph.zero_slot1 * 128 + t] = 0ull;
+                }
+                if (ph.kind == CH_ATT) {
+                    // block-local bidirectional attention, a warp per (position, attention head) over the whole grid;
+                    // lanes over the head's features, one warp sum per key; output in operand form (hi + lo)
+                    const int L = ph.att_L, H = ph.att_H, dh = p.d / H;
+                    const float scale = rsqrtf((float)dh);
+                    for (int item = cta * 4 + q; item < p.M * H; item += G * 4) {
+                        const int pos = item / H, hd = item - pos * H, b0 = (pos / L) * L;
+                        const float *qi = ph.att_q + (size_t)pos * p.d + (size_t)hd * dh;
+                        // online softmax over the keys of the block: running maximum, sum and output
+                        float mx = -INFINITY, sum = 0.f;
+                        float oacc[8];                   // dh <= 256: eight features per lane at most
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) oacc[u] = 0.f;
+                        for (int j = 0; j < L; ++j) {
+                            const float *kj = ph.att_k + (size_t)(b0 + j) * p.d + (size_t)hd * dh;
+                            const float *vj = ph.att_v + (size_t)(b0 + j) * p.d + (size_t)hd * dh;
+                            float sd = 0.f;
+                            for (int cidx = lane; cidx < dh; cidx += 32) sd = fmaf(__ldcg(qi + cidx), __ldcg(kj + cidx), sd);
+#pragma unroll
+                            for (int o2 = 16; o2 > 0; o2 >>= 1) sd += __shfl_xor_sync(0xffffffffu, sd, o2);
+                            sd *= scale;
+                            const float nm = fmaxf(mx, sd), corr = __expf(mx - nm), e2 = __expf(sd - nm);
+                            sum = sum * corr + e2;
+#pragma unroll
+                            for (int u = 0; u < 8; ++u) {
+                                const int cidx = lane + 32 * u;
+                                oacc[u] = oacc[u] * corr + (cidx < dh ? e2 * __ldcg(vj + cidx) : 0.f);
+                            }
+                            mx = nm;
+                        }
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) {
+                            const int cidx = lane + 32 * u;
+                            if (cidx < dh)
+                                ch_store_hi_lo(ph.att_out + (size_t)pos * p.d + (size_t)hd * dh + cidx, (size_t)p.lo_x * p.d, oacc[u] / sum);
+                        }
+                    }
+                }
+            }
             // this CTA's part of the phase is in memory: arrive at the grid barrier
             ch_epi_sync();
             if (t == 0) {
@@ -599,10 +707,10 @@ sk_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant__ 
 // whether `grid` CTAs of it can be resident together, which the phase barriers need: on a
 // context that may use only part of the SMs (MPS with a thread percentage, a partitioned
 // device) they cannot, and the caller then runs the chain as one kernel per GEMM.
-template <int RP, int KC>
+template <int RP, int KC, bool MOD = false>
 cudaError_t chain_prepare(int grid, size_t smem, int sm_count, bool *fits)
 {
-    auto kern = sk_chain_kernel<RP, KC>;
+    auto kern = sk_chain_kernel<RP, KC, MOD>;
     static std::atomic<unsigned long long> attr_devices{0}, fit_devices{0}, nofit_devices{0};
     int dev = 0;
     cudaError_t ea = cudaGetDevice(&dev);
@@ -623,10 +731,10 @@ cudaError_t chain_prepare(int grid, size_t smem, int sm_count, bool *fits)
     return cudaSuccess;
 }
 
-template <int RP, int KC>
+template <int RP, int KC, bool MOD = false>
 cudaError_t chain_launch(const ChainMaps &maps, const ChainParams &p, int grid, size_t smem, cudaStream_t st)
 {
-    auto kern = sk_chain_kernel<RP, KC>;
+    auto kern = sk_chain_kernel<RP, KC, MOD>;
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));
     cfg.gridDim = dim3(grid);
@@ -755,6 +863,130 @@ cudaError_t sk_chain(Ctx *c, int M, int K, const mrp_draft_out &out, cudaStream_
     }
     c->launches++;
     return note_err(c, e, "head-chain kernel");
+}
+
+// One layer of the token-conditioned module (Sec. 3.2) over n <= 128 positions as ONE cooperative kernel: the
+// phases q/k/v (three matrices, one product) -> attention -> output projection -> gate/up -> down projection of the
+// head-chain kernel's machinery (split contraction, slices finished by all CTAs, weights of the next phase
+// prefetched before the grid barrier); with `w_proj` the fusion projection runs as a phase in front.  Operands in
+// the few-row form (lo rows sk_head_pad(n) rows behind the hi rows); the sums of squares of the norms live in
+// slots of the fixed-point array (s_in: the slot the q/k/v norm reads, written by the previous launch or, with
+// w_proj, by this one).  cudaErrorNotSupported (nothing launched): the shape does not fit; the caller runs the
+// products as separate kernels.
+cudaError_t sk_module_layer(Ctx *c, int n, int L, int n_attn_heads, const mrp_module_layer &y, const void *w_proj,
+                            const __nv_bfloat16 *cat16, __nv_bfloat16 *xa, __nv_bfloat16 *xb, __nv_bfloat16 *act16, float *q,
+                            float *k, float *v, float *z, int s_in, int s_next, const void *gamma_next, int32_t *user_status,
+                            cudaStream_t st, bool check_only)
+{
+    const TcState *s = (const TcState *)c->tc_state;
+    const int d = c->cfg.d, F = c->cfg.d_ff, G = c->sm_count;
+    const int s_mlp = 3;
+    if (n < 1 || n > 128 || d % 128 || F % 64 || d / n_attn_heads > 256 || (d / n_attn_heads) % 32) return cudaErrorNotSupported;
+    const int r_pad = sk_head_pad(n);
+    const int d_tiles = d / 128, gu_tiles = F / 64;
+    if (3 * d_tiles > G || gu_tiles > G || 3 * d_tiles > kChTilesPerPhase || gu_tiles > kChTilesPerPhase ||
+        kChMaxPhases * kChTilesPerPhase >= kSkMaxTiles || (size_t)G * r_pad * 128 * 4 > (size_t)kSkScratchBytes)
+        return cudaErrorNotSupported;
+    auto split = [&](int n_tiles, int k_chunks) {
+        int S = G / n_tiles;
+        if (S < 1) S = 1;
+        if (S > k_chunks) S = k_chunks;
+        const int cps = (k_chunks + S - 1) / S;
+        return (k_chunks + cps - 1) / cps;          // no empty slice
+    };
+    const int sp_proj = split(d_tiles, 2 * d / kBK), sp_qkv = split(3 * d_tiles, d / kBK), sp_o = split(d_tiles, d / kBK);
+    const int sp_gu = split(gu_tiles, d / kBK), sp_dn = split(d_tiles, F / kBK);
+    auto share_fits = [&](int sp) { return n * ((128 + sp - 1) / sp) <= kChMaxShare; };
+    // (the products with a norm behind them keep a share's squares in shared memory)
+    if (!share_fits(sp_o) || !share_fits(sp_dn) || (w_proj && !share_fits(sp_proj))) return cudaErrorNotSupported;
+    const int stage = kChWTile + 2 * r_pad * 128;           // one k-chunk per ring stage
+    int ns = (kSmemBudget - 1024 - 256 - 16 - kChAuxBytes) / stage;
+    if (ns > 12) ns = 12;
+    const size_t smem = (size_t)ns * stage + 1024 + 8 * (2 * ns + 4) + 16 + kChAuxBytes;
+    {
+        bool fits = false;
+        cudaError_t eq;
+        switch (r_pad) {
+        case 16: eq = chain_prepare<16, 1, true>(G, smem, G, &fits); break;
+        case 32: eq = chain_prepare<32, 1, true>(G, smem, G, &fits); break;
+        case 64: eq = chain_prepare<64, 1, true>(G, smem, G, &fits); break;
+        default: eq = chain_prepare<128, 1, true>(G, smem, G, &fits); break;
+        }
+        if (eq != cudaSuccess || !fits) return cudaErrorNotSupported;
+    }
+    if (check_only) return cudaSuccess;
+
+    ChainParams p;
+    memset(&p, 0, sizeof(p));
+    ChainMaps maps;
+    memset(&maps, 0, sizeof(maps));
+    p.M = n; p.d = d; p.F = F; p.eps = c->cfg.rms_eps; p.lo_x = r_pad; p.lo_xt = r_pad;
+    p.act = act16;
+    p.ssq_fix = (unsigned long long *)(c->ws + c->lay.ssq_fix);
+    p.scratch = (float *)(c->ws + c->lay.sk_scratch);
+    p.counters = (int32_t *)(c->ws + c->lay.sk_counters);
+    p.grid_bar = (unsigned int *)(c->ws + c->lay.sk_counters) + (kSkMaxTiles - 1);
+    p.status = (int32_t *)(c->ws + c->lay.status); p.user_status = user_status;
+    p.n_stages = ns;
+    int cols = 32;
+    while (cols < 2 * 2 * r_pad) cols <<= 1;
+    p.tmem_cols = cols;
+    if (!make_map(s, &maps.m[0], xa, d, 2 * (uint64_t)r_pad, 2 * r_pad) || !make_map(s, &maps.m[1], act16, F, 2 * (uint64_t)r_pad, 2 * r_pad) ||
+        !make_map(s, &maps.m[2], xb, d, 2 * (uint64_t)r_pad, 2 * r_pad) || !make_map(s, &maps.m[3], y.w_q, d, d, 128) ||
+        !make_map(s, &maps.m[4], y.w_k, d, d, 128) || !make_map(s, &maps.m[5], y.w_v, d, d, 128) ||
+        !make_map(s, &maps.m[6], y.w_o, d, d, 128) || !make_map(s, &maps.m[7], y.w_gate, d, F, 64) ||
+        !make_map(s, &maps.m[8], y.w_up, d, F, 64) || !make_map(s, &maps.m[9], y.w_down, F, d, 128))
+        return note_err(c, cudaErrorInvalidValue, "tensor map (module layer)");
+    if (w_proj && (!make_map(s, &maps.m[10], cat16, 2 * d, 2 * (uint64_t)r_pad, 2 * r_pad) ||
+                   !make_map(s, &maps.m[11], w_proj, 2 * d, d, 128)))
+        return note_err(c, cudaErrorInvalidValue, "tensor map (module fusion projection)");
+    int i = 0;
+    auto lin = [&](int k_chunks, int n_tiles, int n_split, int map_x, int map_w) -> ChainPhase & {
+        ChainPhase &ph = p.ph[i++];
+        ph.kind = CH_LIN; ph.k_chunks = k_chunks; ph.n_tiles = n_tiles; ph.n_split = n_split; ph.w_rows = d;
+        ph.map_x = map_x; ph.map_w0 = map_w; ph.map_w1 = map_w; ph.ssq_in = -1; ph.zero_slot0 = -1; ph.zero_slot1 = -1;
+        return ph;
+    };
+    if (w_proj) {
+        ChainPhase &ph = lin(2 * d / kBK, d_tiles, sp_proj, 10, 11);
+        ph.lin_out = z; ph.gamma_next = (const __nv_bfloat16 *)y.g_attn; ph.xg_next = xa; ph.ssq_idx = s_in;
+    }
+    {
+        ChainPhase &ph = lin(d / kBK, 3 * d_tiles, sp_qkv, 0, 3);
+        ph.lin_out = q; ph.lin_out1 = k; ph.lin_out2 = v; ph.lin3_tiles = d_tiles; ph.ssq_in = s_in;
+    }
+    p.ph[0].zero_slot0 = s_mlp; p.ph[0].zero_slot1 = s_next;      // (with w_proj: s_in was cleared before the launch)
+    {
+        ChainPhase &ph = p.ph[i++];
+        ph.kind = CH_ATT; ph.n_tiles = 0; ph.n_split = 1; ph.k_chunks = 1; ph.zero_slot0 = -1; ph.zero_slot1 = -1;
+        ph.att_q = q; ph.att_k = k; ph.att_v = v; ph.att_out = xb; ph.att_L = L; ph.att_H = n_attn_heads;
+    }
+    {
+        ChainPhase &ph = lin(d / kBK, d_tiles, sp_o, 2, 6);
+        ph.lin_out = z; ph.lin_acc = 1; ph.gamma_next = (const __nv_bfloat16 *)y.g_mlp; ph.xg_next = xa; ph.ssq_idx = s_mlp;
+    }
+    {
+        ChainPhase &ph = p.ph[i++];
+        ph.kind = CH_GU; ph.k_chunks = d / kBK; ph.n_tiles = gu_tiles; ph.n_split = sp_gu; ph.w_rows = F;
+        ph.map_x = 0; ph.map_w0 = 7; ph.map_w1 = 8; ph.ssq_idx = s_mlp; ph.zero_slot0 = -1; ph.zero_slot1 = -1;
+    }
+    {
+        ChainPhase &ph = lin(F / kBK, d_tiles, sp_dn, 1, 9);
+        ph.lin_out = z; ph.lin_acc = 1;
+        ph.gamma_next = (const __nv_bfloat16 *)gamma_next; ph.xg_next = gamma_next ? xa : nullptr; ph.ssq_idx = s_next;
+    }
+    p.n_phases = i;
+    // arrival counters and the grid barrier start at zero
+    cudaError_t e = cudaMemsetAsync(c->ws + c->lay.sk_counters, 0, (size_t)kSkMaxTiles * 4, st);
+    if (e != cudaSuccess) return note_err(c, e, "module layer, counters");
+    switch (r_pad) {
+    case 16: e = chain_launch<16, 1, true>(maps, p, G, smem, st); break;
+    case 32: e = chain_launch<32, 1, true>(maps, p, G, smem, st); break;
+    case 64: e = chain_launch<64, 1, true>(maps, p, G, smem, st); break;
+    default: e = chain_launch<128, 1, true>(maps, p, G, smem, st); break;
+    }
+    c->launches++;
+    return note_err(c, e, "module layer kernel");
 }
 
 }  // namespace mrp

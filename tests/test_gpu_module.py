@@ -29,6 +29,9 @@ def upload_module(mw, dtype):
     ("bf16", 0, 192, 320, 2064, 3, 3, 3, 5, 2),                             # 15 positions, ragged tiles, three layers
     ("bf16", 0, 256, 512, 4096, 2, 4, 3, 4, 2),                             # 12 positions, three units per CTA
     ("bf16", 0, 512, 1024, 4096, 1, 4, 40, 4, 2),                           # 160 positions, two row blocks, wider model
+    ("bf16", binding.MRP_FLAG_NO_CHAIN, 256, 512, 4096, 2, 4, 3, 4, 2),     # the few-row kernels, one launch per product
+    ("bf16", 0, 256, 512, 4096, 3, 2, 2, 32, 2),                            # two blocks of 32: a layer as one kernel, 64 rows
+    ("bf16", binding.MRP_FLAG_NO_CHAIN, 128, 256, 2048, 1, 4, 1, 48, 2),    # a block of 48 through the separate attention kernel
     # four positions or fewer: the module step is one cooperative kernel
     ("f32", 0, 64, 96, 512, 2, 4, 1, 4, 3),                                 # fp32 weights, ragged widths
     ("bf16", binding.MRP_FLAG_FORCE_SIMT, 256, 512, 1024, 2, 2, 1, 3, 2),   # 16-byte weight loads, block of three
