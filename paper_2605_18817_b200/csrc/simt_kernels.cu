@@ -1795,6 +1795,16 @@ static bool module_tc_ok(const Ctx *c, int n)
     return true;
 }
 
+// Whether a call over n positions runs its layers as one cooperative tensor-core kernel each.
+static bool module_chain_ok(Ctx *c, int n, int L, cudaStream_t st)
+{
+    const mrp_module_weights &w = c->module;
+    return module_tc_ok(c, n) && w.n_layers > 0 && n <= 64 && (size_t)sk_head_pad(n) <= module_cap_rows(c->cfg) &&
+           sk_heads_ok(c->cfg) && !(c->cfg.flags & (MRP_FLAG_ROW_MAJOR_ONLY | MRP_FLAG_NO_CHAIN)) &&
+           sk_module_layer(c, n, L, w.n_attn_heads, w.layers[0], w.w_proj, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr,
+                           nullptr, nullptr, 0, 1, nullptr, nullptr, st, true) == cudaSuccess;
+}
+
 // The module itself (everything in front of `h <- h + Delta`) with its products on the tensor cores.
 static cudaError_t module_body_tc(Ctx *c, const int32_t *tokens, const void *hidden0, float *h_state, int B, int L,
                                   bool first_step, const mrp_draft_out &out, cudaStream_t st, float *z)
@@ -1820,10 +1830,7 @@ static cudaError_t module_body_tc(Ctx *c, const int32_t *tokens, const void *hid
                      !(c->cfg.flags & MRP_FLAG_ROW_MAJOR_ONLY);
     // up to 64 positions: a layer (the first with the fusion projection) as one cooperative kernel, if the shape fits
     // (at 128 positions and d = 4096 the row-major kernels are ahead: 0.52 against 0.76 ms per step of the module)
-    const bool chain = w.n_layers > 0 && n <= 64 && (size_t)sk_head_pad(n) <= cap && sk_heads_ok(c->cfg) &&
-                       !(c->cfg.flags & (MRP_FLAG_ROW_MAJOR_ONLY | MRP_FLAG_NO_CHAIN)) &&
-                       sk_module_layer(c, n, L, w.n_attn_heads, w.layers[0], w.w_proj, nullptr, nullptr, nullptr, nullptr, nullptr,
-                                       nullptr, nullptr, nullptr, 0, 1, nullptr, out.status, st, true) == cudaSuccess;
+    const bool chain = module_chain_ok(c, n, L, st);
     const int lo_rows = (few || chain) ? sk_head_pad(n) : n;
     cudaError_t e = launch_k(mod_cat_split_kernel, dim3(n), dim3(256), 0, st, pdl, (const float *)h_state,
                              (const __nv_bfloat16 *)hidden0, first_step ? 1 : 0, tokens, (const __nv_bfloat16 *)w.emb, w.mask_token,
@@ -1917,7 +1924,9 @@ static cudaError_t module_step_t(Ctx *c, const int32_t *tokens, const void *hidd
         return launch_k(linear_kernel<T>, dim3((n_out + 7) / 8), dim3(256), 0, st, pdl, (const T *)wm, x, n, n_in, n_out, y, acc);
     };
     prof_mark(c, 0, st);
-    {
+    // (measured at four positions, decode shape: 0.166 ms per step on the tensor-core chain, 0.225 ms as the one
+    // CUDA-core kernel below, which therefore serves the contexts and shapes the chain does not)
+    if (!module_chain_ok(c, n, L, st)) {
         // a handful of positions: the whole module step as one kernel, then the LM-head kernels
         bool launched = false;
         TcPlan pl;
