@@ -1795,14 +1795,14 @@ static bool module_tc_ok(const Ctx *c, int n)
     return true;
 }
 
-// Whether a call over n positions runs its layers as one cooperative tensor-core kernel each.
+// Whether a call over n positions runs as one cooperative tensor-core kernel.
 static bool module_chain_ok(Ctx *c, int n, int L, cudaStream_t st)
 {
     const mrp_module_weights &w = c->module;
     return module_tc_ok(c, n) && w.n_layers > 0 && n <= 64 && (size_t)sk_head_pad(n) <= module_cap_rows(c->cfg) &&
            sk_heads_ok(c->cfg) && !(c->cfg.flags & (MRP_FLAG_ROW_MAJOR_ONLY | MRP_FLAG_NO_CHAIN)) &&
-           sk_module_layer(c, n, L, w.n_attn_heads, w.layers[0], w.w_proj, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr,
-                           nullptr, nullptr, 0, 1, nullptr, nullptr, st, true) == cudaSuccess;
+           sk_module_step(c, n, L, nullptr, nullptr, nullptr, false, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr,
+                          nullptr, nullptr, nullptr, 0, 0, false, nullptr, nullptr, st, true) == cudaSuccess;
 }
 
 // The module itself (everything in front of `h <- h + Delta`) with its products on the tensor cores.
@@ -1828,10 +1828,7 @@ static cudaError_t module_body_tc(Ctx *c, const int32_t *tokens, const void *hid
     // where the lo rows of an operand sit behind its hi rows: the few-row kernels fetch both with one TMA box
     const bool few = sk_head_rows_ok(n) && sk_heads_ok(c->cfg) && (size_t)sk_head_pad(n) <= cap &&
                      !(c->cfg.flags & MRP_FLAG_ROW_MAJOR_ONLY);
-    // up to 64 positions: a layer (the first with the fusion projection) as one cooperative kernel, if the shape fits
-    // (at 128 positions and d = 4096 the row-major kernels are ahead: 0.52 against 0.76 ms per step of the module)
-    const bool chain = module_chain_ok(c, n, L, st);
-    const int lo_rows = (few || chain) ? sk_head_pad(n) : n;
+    const int lo_rows = few ? sk_head_pad(n) : n;
     cudaError_t e = launch_k(mod_cat_split_kernel, dim3(n), dim3(256), 0, st, pdl, (const float *)h_state,
                              (const __nv_bfloat16 *)hidden0, first_step ? 1 : 0, tokens, (const __nv_bfloat16 *)w.emb, w.mask_token,
                              w.emb_rows, lo_rows, d, h_state, cat16, status, out.status);
@@ -1840,16 +1837,6 @@ static cudaError_t module_body_tc(Ctx *c, const int32_t *tokens, const void *hid
     // its partial sums of squares: no kernel between them.
     int n_ss = 1;
     const void *g_first = w.n_layers > 0 ? w.layers[0].g_attn : nullptr;
-    if (chain) {
-        // the norms' sums of squares live in slots of the fixed-point array; the slot the first launch adds to is cleared here
-        if (e == cudaSuccess) e = cudaMemsetAsync(c->ws + c->lay.ssq_fix, 0, (size_t)5 * 128 * 8, st);
-        for (int l = 0; l < w.n_layers && e == cudaSuccess; ++l) {
-            const void *g_next = l + 1 < w.n_layers ? w.layers[l + 1].g_attn : nullptr;
-            e = sk_module_layer(c, n, L, w.n_attn_heads, w.layers[l], l == 0 ? w.w_proj : nullptr, cat16, xa, xb, act16, q, k, v, z,
-                                l & 1, 1 - (l & 1), g_next, out.status, st, false);
-        }
-        return e;
-    }
     if (few) {
         // up to 64 positions: the few-row kernels (weight rows on the MMA M axis, contraction split over CTAs), whose
         // tiles stream the weights once whatever the number of positions.  Their per-tile arrival counters must be
@@ -1902,7 +1889,9 @@ size_t module_workspace_bytes(const mrp_config &cfg, int n_layers)
 {
     (void)n_layers;
     const size_t n = module_cap_rows(cfg), d = (size_t)cfg.d, F = (size_t)cfg.d_ff;
-    return align_up(n * 2 * d * 4, 256) + 6 * align_up(n * d * 4, 256) + align_up(n * F * 4, 256);
+    // (the last term: the arrival counters of the one-launch tensor-core step)
+    return align_up(n * 2 * d * 4, 256) + 6 * align_up(n * d * 4, 256) + align_up(n * F * 4, 256) +
+           align_up((size_t)kModChainBarInts * 4, 256);
 }
 
 template <typename T>
@@ -1924,9 +1913,28 @@ static cudaError_t module_step_t(Ctx *c, const int32_t *tokens, const void *hidd
         return launch_k(linear_kernel<T>, dim3((n_out + 7) / 8), dim3(256), 0, st, pdl, (const T *)wm, x, n, n_in, n_out, y, acc);
     };
     prof_mark(c, 0, st);
-    // (measured at four positions, decode shape: 0.166 ms per step on the tensor-core chain, 0.225 ms as the one
-    // CUDA-core kernel below, which therefore serves the contexts and shapes the chain does not)
-    if (!module_chain_ok(c, n, L, st)) {
+    if (module_chain_ok(c, n, L, st)) {
+        // up to 64 positions on a tensor-core context: the whole step (fusion, the layers, h <- h + Delta, the LM-head
+        // operand) as one cooperative tcgen05 kernel, then the LM-head kernels.  (At four positions, decode shape:
+        // 0.14 ms against 0.225 ms for the one CUDA-core kernel below, which serves the contexts and shapes this
+        // one does not.)
+        TcPlan pl;
+        if (M > 0) pl = tc_plan(c, M, 1, out, st, false);
+        char *wp = c->module_ws;
+        auto tk = [&](size_t bytes) { char *p0 = wp; wp += align_up(bytes, 256); return p0; };
+        __nv_bfloat16 *cat16 = (__nv_bfloat16 *)tk(cap * 2 * d * 4);
+        float *zc = (float *)tk(cap * d * 4);
+        __nv_bfloat16 *xa = (__nv_bfloat16 *)tk(cap * d * 4);
+        float *qc = (float *)tk(cap * d * 4), *kc2 = (float *)tk(cap * d * 4), *vc = (float *)tk(cap * d * 4);
+        __nv_bfloat16 *xb = (__nv_bfloat16 *)tk(cap * d * 4);
+        __nv_bfloat16 *act16 = (__nv_bfloat16 *)tk(cap * F * 4);
+        int32_t *bar_mem = (int32_t *)wp;
+        const cudaError_t ec = sk_module_step(c, n, L, tokens, hidden0, h_state, first_step, cat16, xa, xb, act16, qc, kc2, vc, zc,
+                                              bar_mem, row_index, M, c->lo_xt, M > 0 && pl.f16_lm, out.hidden_out, out.status, st,
+                                              false);
+        if (ec != cudaSuccess || M == 0) return ec;
+        return tc_lm_tail(c, pl, logits0, row_index, M, 1, out, st);
+    } else {
         // a handful of positions: the whole module step as one kernel, then the LM-head kernels
         bool launched = false;
         TcPlan pl;

@@ -42,12 +42,18 @@ constexpr int kChTilesPerPhase = 448;      // arrival counters per phase
 constexpr int kChMaxPhases = 8;
 constexpr long long kBarrierCycles = 1000000000LL;   // bound on a grid-barrier wait (about 0.5 s)
 
-enum { CH_GU = 0, CH_DN = 1, CH_LIN = 2, CH_ATT = 3 };      // LIN, ATT: the module's phases (MOD instantiations)
+enum { CH_GU = 0, CH_DN = 1, CH_LIN = 2, CH_ATT = 3, CH_CAT = 4, CH_FIN = 5 };   // from LIN on: the module's phases (MOD instantiations)
 
-struct ChainMaps {
-    CUtensorMap m[2 + 3 * 4];   // 0: head input (xg), 1: SwiGLU output (act), 2+3h: gate, 3+3h: up, 4+3h: down of head h
-                                // (a module layer: 0 xa, 1 act, 2 xb, 3-5 q k v, 6 o, 7 gate, 8 up, 9 down)
+constexpr int kModChainLayers = 4;     // module layers one launch can hold
+constexpr int kModChainPhases = 3 + 5 * kModChainLayers;   // fusion + projection, five per layer, the closing phase
+template <int NM>
+struct ChainMapsT {
+    CUtensorMap m[NM];
 };
+// head chain: 0: head input (xg), 1: SwiGLU output (act), 2+3h: gate, 3+3h: up, 4+3h: down of head h
+using ChainMaps = ChainMapsT<2 + 3 * 4>;
+// module step: 0 xa, 1 act, 2 xb, 3 [h ; emb] rows, 4 fusion projection, 5 + 7 l ...: q k v o gate up down of layer l
+using ModChainMaps = ChainMapsT<5 + 7 * kModChainLayers>;
 
 struct ChainPhase {
     int kind;
@@ -74,12 +80,29 @@ struct ChainPhase {
     int zero_slot0, zero_slot1;      // ssq_fix slots this phase clears for later phases of the launch (< 0: none)
 };
 
-struct ChainParams {
+// What the module's first (CAT: the rows [h ; emb[x]] in operand form) and last phase (FIN: h <- h + Delta and the
+// LM-head operand of the masked rows) need.
+struct ModEnds {
+    const int32_t *tokens;
+    const __nv_bfloat16 *hidden0, *emb;
+    float *h_state, *z;
+    __nv_bfloat16 *cat;
+    int first_step, mask_token, emb_rows;
+    const int32_t *row_index;
+    int n_masked;
+    __nv_bfloat16 *xt;       // LM-head operand rows (step 0 zero rows, then h - h_0), lo rows lo_xt rows further on
+    __half *xt16;
+    float *hidden_out;
+};
+
+template <int NP>
+struct ChainParamsT {
     int n_phases, n_stages, tmem_cols;
     int M, d, F, n_rs;
     int lo_x, lo_xt;         // row offset of the lo block in the head operands / the LM-head operand
     float eps;
-    ChainPhase ph[kChMaxPhases];
+    ChainPhase ph[NP];
+    ModEnds mod;
     __nv_bfloat16 *act;
     float *hcur;
     const float *h0f;
@@ -91,6 +114,11 @@ struct ChainParams {
     int32_t *status;
     int32_t *user_status;
 };
+static_assert(kModChainBarInts == kModChainPhases * kChTilesPerPhase + 1, "counter array of the one-launch module step");
+using ChainParams = ChainParamsT<kChMaxPhases>;
+using ModChainParams = ChainParamsT<kModChainPhases>;
+template <bool MOD> struct ChainTypes { using Maps = ChainMaps; using Params = ChainParams; };
+template <> struct ChainTypes<true> { using Maps = ModChainMaps; using Params = ModChainParams; };
 
 __device__ __forceinline__ void ch_epi_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 __device__ __forceinline__ void ch_store_hi_lo(__nv_bfloat16 *dst, size_t lo_off, float v)
@@ -115,8 +143,9 @@ __device__ __forceinline__ unsigned int ld_acquire_u32(const unsigned int *p)
     return v;
 }
 // Waits until `target` arrivals have been counted; false if the wait ran out or another role gave up.
+template <typename P>
 __device__ __forceinline__ bool grid_bar_wait(const unsigned int *bar, unsigned int target, volatile int *abort_flag,
-                                              const ChainParams &p)
+                                              const P &p)
 {
     if ((int)(ld_acquire_u32(bar) - target) >= 0) return true;
     const long long t0 = clock64();
@@ -137,7 +166,8 @@ __device__ __forceinline__ bool grid_bar_wait(const unsigned int *bar, unsigned 
 // compile none of that code.
 template <int RP, int KC, bool MOD = false>
 __global__ void __launch_bounds__(kChThreads, 1)
-sk_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainParams p)
+sk_chain_kernel(const __grid_constant__ typename ChainTypes<MOD>::Maps maps,
+                const __grid_constant__ typename ChainTypes<MOD>::Params p)
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -639,6 +669,67 @@ sk_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant__ 
                     if (ph.zero_slot0 >= 0) p.ssq_fix[ph.zero_slot0 * 128 + t] = 0ull;
                     if (ph.zero_slot1 >= 0) p.ssq_fix[ph.zero_slot1 * 128 + t] = 0ull;
                 }
+                if (ph.kind == CH_CAT) {
+                    // the rows [h_i ; emb[x_i]] in operand form; on the first step of a backbone forward h is the
+                    // backbone's hidden state, which also starts the running state
+                    const ModEnds &e = p.mod;
+                    const int d2 = 2 * p.d;
+                    for (int idx = cta * 128 + t; idx < p.M * p.d; idx += G * 128) {
+                        const int pos = idx / p.d, j = idx - pos * p.d;
+                        int tok = e.tokens[pos];
+                        if (tok >= e.emb_rows || tok < -1) {          // outside the table: reads as masked, raises the bit
+                            if (j == 0) {
+                                atomicOr(p.status, MRP_DEV_BAD_INDEX);
+                                if (p.user_status) atomicOr(p.user_status, MRP_DEV_BAD_INDEX);
+                            }
+                            tok = -1;
+                        }
+                        if (tok < 0) tok = e.mask_token;
+                        const float h = e.first_step ? __bfloat162float(e.hidden0[idx]) : __ldcg(e.h_state + idx);
+                        if (e.first_step) e.h_state[idx] = h;
+                        ch_store_hi_lo(e.cat + (size_t)pos * d2 + j, (size_t)p.lo_x * d2, h);
+                        e.cat[(size_t)pos * d2 + p.d + j] = e.emb[(size_t)tok * p.d + j];       // a bf16 value: no remainder
+                        e.cat[((size_t)p.lo_x + pos) * d2 + p.d + j] = __float2bfloat16(0.f);
+                    }
+                }
+                if (ph.kind == CH_FIN) {
+                    // h <- h + Delta at every position; the LM-head operand h - h_0 of the masked rows behind the zero
+                    // rows of step 0 (a row index out of range: zero rows, and the bit)
+                    const ModEnds &e = p.mod;
+                    int *inv = reinterpret_cast<int *>(sq_s);          // dense position -> masked row, or -1
+                    for (int i2 = t; i2 < p.M; i2 += 128) inv[i2] = -1;
+                    ch_epi_sync();
+                    if (t == 0) {
+                        for (int m = 0; m < e.n_masked; ++m) {
+                            const int idx = e.row_index ? e.row_index[m] : m;
+                            if (row_ok(idx, p.M)) inv[idx] = m;
+                            else if (cta == 0) {
+                                atomicOr(p.status, MRP_DEV_BAD_INDEX);
+                                if (p.user_status) atomicOr(p.user_status, MRP_DEV_BAD_INDEX);
+                            }
+                        }
+                    }
+                    ch_epi_sync();
+                    auto put = [&](int m, int j, float h, float r) {
+                        const size_t o = (size_t)m * p.d + j;
+                        if (e.hidden_out) e.hidden_out[o] = h;
+                        e.xt[o] = __float2bfloat16(0.f);
+                        e.xt[(size_t)p.lo_xt * p.d + o] = __float2bfloat16(0.f);
+                        ch_store_hi_lo(e.xt + (size_t)e.n_masked * p.d + o, (size_t)p.lo_xt * p.d, r);
+                        if (e.xt16) e.xt16[o] = __float2half_rn(r);
+                    };
+                    for (int idx = cta * 128 + t; idx < p.M * p.d; idx += G * 128) {
+                        const int pos = idx / p.d, j = idx - pos * p.d;
+                        const float h = __ldcg(e.h_state + idx) + __ldcg(e.z + idx);
+                        e.h_state[idx] = h;
+                        if (inv[pos] >= 0) put(inv[pos], j, h, h - __bfloat162float(e.hidden0[idx]));
+                    }
+                    for (int m = 0; m < e.n_masked; ++m) {
+                        const int idx = e.row_index ? e.row_index[m] : m;
+                        if (!row_ok(idx, p.M) || inv[idx] != m)
+                            for (int j = cta * 128 + t; j < p.d; j += G * 128) put(m, j, 0.f, 0.f);
+                    }
+                }
                 if (ph.kind == CH_ATT) {
                     // block-local bidirectional attention, a warp per (position, attention head) over the whole grid;
                     // lanes over the head's features, one warp sum per key; output in operand form (hi + lo)
@@ -732,7 +823,8 @@ cudaError_t chain_prepare(int grid, size_t smem, int sm_count, bool *fits)
 }
 
 template <int RP, int KC, bool MOD = false>
-cudaError_t chain_launch(const ChainMaps &maps, const ChainParams &p, int grid, size_t smem, cudaStream_t st)
+cudaError_t chain_launch(const typename ChainTypes<MOD>::Maps &maps, const typename ChainTypes<MOD>::Params &p, int grid,
+                         size_t smem, cudaStream_t st)
 {
     auto kern = sk_chain_kernel<RP, KC, MOD>;
     cudaLaunchConfig_t cfg;
@@ -865,27 +957,28 @@ cudaError_t sk_chain(Ctx *c, int M, int K, const mrp_draft_out &out, cudaStream_
     return note_err(c, e, "head-chain kernel");
 }
 
-// One layer of the token-conditioned module (Sec. 3.2) over n <= 128 positions as ONE cooperative kernel: the
-// phases q/k/v (three matrices, one product) -> attention -> output projection -> gate/up -> down projection of the
-// head-chain kernel's machinery (split contraction, slices finished by all CTAs, weights of the next phase
-// prefetched before the grid barrier); with `w_proj` the fusion projection runs as a phase in front.  Operands in
-// the few-row form (lo rows sk_head_pad(n) rows behind the hi rows); the sums of squares of the norms live in
-// slots of the fixed-point array (s_in: the slot the q/k/v norm reads, written by the previous launch or, with
-// w_proj, by this one).  cudaErrorNotSupported (nothing launched): the shape does not fit; the caller runs the
-// products as separate kernels.
-cudaError_t sk_module_layer(Ctx *c, int n, int L, int n_attn_heads, const mrp_module_layer &y, const void *w_proj,
-                            const __nv_bfloat16 *cat16, __nv_bfloat16 *xa, __nv_bfloat16 *xb, __nv_bfloat16 *act16, float *q,
-                            float *k, float *v, float *z, int s_in, int s_next, const void *gamma_next, int32_t *user_status,
-                            cudaStream_t st, bool check_only)
+// One step of the token-conditioned module (Sec. 3.2) over n <= 128 positions as ONE cooperative kernel: the rows
+// [h ; emb[x]] -> fusion projection -> per layer q/k/v (three matrices, one product) -> attention -> output projection
+// -> gate/up -> down projection -> h <- h + Delta and the LM-head operand of the masked rows, as phases of the
+// head-chain kernel's machinery (split contraction, slices finished by all CTAs, weights of the next phase prefetched
+// before the grid barrier).  Operands in the few-row form (lo rows sk_head_pad(n) rows behind the hi rows); the sums
+// of squares of the norms live in slots of the fixed-point array.  `bar_mem`: kModChainPhases * kChTilesPerPhase + 1
+// zero-able counters of the caller's (module workspace).  cudaErrorNotSupported (nothing launched): the shape does
+// not fit; the caller runs the products as separate kernels.
+cudaError_t sk_module_step(Ctx *c, int n, int L, const int32_t *tokens, const void *hidden0, float *h_state, bool first_step,
+                           __nv_bfloat16 *cat16, __nv_bfloat16 *xa, __nv_bfloat16 *xb, __nv_bfloat16 *act16, float *q, float *k,
+                           float *v, float *z, int32_t *bar_mem, const int32_t *row_index, int n_masked, int lo_xt, bool f16_lm,
+                           float *hidden_out, int32_t *user_status, cudaStream_t st, bool check_only)
 {
     const TcState *s = (const TcState *)c->tc_state;
-    const int d = c->cfg.d, F = c->cfg.d_ff, G = c->sm_count;
-    const int s_mlp = 3;
-    if (n < 1 || n > 128 || d % 128 || F % 64 || d / n_attn_heads > 256 || (d / n_attn_heads) % 32) return cudaErrorNotSupported;
+    const mrp_module_weights &w = c->module;
+    const int d = c->cfg.d, F = c->cfg.d_ff, G = c->sm_count, D = w.n_layers, H = w.n_attn_heads;
+    if (D < 1 || D > kModChainLayers || n < 1 || n > 128 || d % 128 || F % 64 || d / H > 256 || (d / H) % 32)
+        return cudaErrorNotSupported;
     const int r_pad = sk_head_pad(n);
     const int d_tiles = d / 128, gu_tiles = F / 64;
     if (3 * d_tiles > G || gu_tiles > G || 3 * d_tiles > kChTilesPerPhase || gu_tiles > kChTilesPerPhase ||
-        kChMaxPhases * kChTilesPerPhase >= kSkMaxTiles || (size_t)G * r_pad * 128 * 4 > (size_t)kSkScratchBytes)
+        (size_t)G * r_pad * 128 * 4 > (size_t)kSkScratchBytes)
         return cudaErrorNotSupported;
     auto split = [&](int n_tiles, int k_chunks) {
         int S = G / n_tiles;
@@ -896,9 +989,9 @@ cudaError_t sk_module_layer(Ctx *c, int n, int L, int n_attn_heads, const mrp_mo
     };
     const int sp_proj = split(d_tiles, 2 * d / kBK), sp_qkv = split(3 * d_tiles, d / kBK), sp_o = split(d_tiles, d / kBK);
     const int sp_gu = split(gu_tiles, d / kBK), sp_dn = split(d_tiles, F / kBK);
-    auto share_fits = [&](int sp) { return n * ((128 + sp - 1) / sp) <= kChMaxShare; };
     // (the products with a norm behind them keep a share's squares in shared memory)
-    if (!share_fits(sp_o) || !share_fits(sp_dn) || (w_proj && !share_fits(sp_proj))) return cudaErrorNotSupported;
+    auto share_fits = [&](int sp) { return n * ((128 + sp - 1) / sp) <= kChMaxShare; };
+    if (!share_fits(sp_o) || !share_fits(sp_dn) || !share_fits(sp_proj)) return cudaErrorNotSupported;
     const int stage = kChWTile + 2 * r_pad * 128;           // one k-chunk per ring stage
     int ns = (kSmemBudget - 1024 - 256 - 16 - kChAuxBytes) / stage;
     if (ns > 12) ns = 12;
@@ -916,69 +1009,95 @@ cudaError_t sk_module_layer(Ctx *c, int n, int L, int n_attn_heads, const mrp_mo
     }
     if (check_only) return cudaSuccess;
 
-    ChainParams p;
+    ModChainParams p;
     memset(&p, 0, sizeof(p));
-    ChainMaps maps;
+    ModChainMaps maps;
     memset(&maps, 0, sizeof(maps));
-    p.M = n; p.d = d; p.F = F; p.eps = c->cfg.rms_eps; p.lo_x = r_pad; p.lo_xt = r_pad;
+    p.M = n; p.d = d; p.F = F; p.eps = c->cfg.rms_eps; p.lo_x = r_pad; p.lo_xt = lo_xt;
     p.act = act16;
     p.ssq_fix = (unsigned long long *)(c->ws + c->lay.ssq_fix);
     p.scratch = (float *)(c->ws + c->lay.sk_scratch);
-    p.counters = (int32_t *)(c->ws + c->lay.sk_counters);
-    p.grid_bar = (unsigned int *)(c->ws + c->lay.sk_counters) + (kSkMaxTiles - 1);
+    p.counters = bar_mem;
+    p.grid_bar = (unsigned int *)bar_mem + kModChainPhases * kChTilesPerPhase;
     p.status = (int32_t *)(c->ws + c->lay.status); p.user_status = user_status;
     p.n_stages = ns;
     int cols = 32;
     while (cols < 2 * 2 * r_pad) cols <<= 1;
     p.tmem_cols = cols;
-    if (!make_map(s, &maps.m[0], xa, d, 2 * (uint64_t)r_pad, 2 * r_pad) || !make_map(s, &maps.m[1], act16, F, 2 * (uint64_t)r_pad, 2 * r_pad) ||
-        !make_map(s, &maps.m[2], xb, d, 2 * (uint64_t)r_pad, 2 * r_pad) || !make_map(s, &maps.m[3], y.w_q, d, d, 128) ||
-        !make_map(s, &maps.m[4], y.w_k, d, d, 128) || !make_map(s, &maps.m[5], y.w_v, d, d, 128) ||
-        !make_map(s, &maps.m[6], y.w_o, d, d, 128) || !make_map(s, &maps.m[7], y.w_gate, d, F, 64) ||
-        !make_map(s, &maps.m[8], y.w_up, d, F, 64) || !make_map(s, &maps.m[9], y.w_down, F, d, 128))
-        return note_err(c, cudaErrorInvalidValue, "tensor map (module layer)");
-    if (w_proj && (!make_map(s, &maps.m[10], cat16, 2 * d, 2 * (uint64_t)r_pad, 2 * r_pad) ||
-                   !make_map(s, &maps.m[11], w_proj, 2 * d, d, 128)))
-        return note_err(c, cudaErrorInvalidValue, "tensor map (module fusion projection)");
+    p.mod.tokens = tokens; p.mod.hidden0 = (const __nv_bfloat16 *)hidden0; p.mod.emb = (const __nv_bfloat16 *)w.emb;
+    p.mod.h_state = h_state; p.mod.z = z; p.mod.cat = cat16; p.mod.first_step = first_step ? 1 : 0;
+    p.mod.mask_token = w.mask_token; p.mod.emb_rows = w.emb_rows; p.mod.row_index = row_index; p.mod.n_masked = n_masked;
+    p.mod.xt = (__nv_bfloat16 *)(c->ws + c->lay.xt); p.mod.xt16 = f16_lm ? (__half *)(c->ws + c->lay.xt16) : nullptr;
+    p.mod.hidden_out = hidden_out;
+    bool ok = make_map(s, &maps.m[0], xa, d, 2 * (uint64_t)r_pad, 2 * r_pad) && make_map(s, &maps.m[1], act16, F, 2 * (uint64_t)r_pad, 2 * r_pad) &&
+              make_map(s, &maps.m[2], xb, d, 2 * (uint64_t)r_pad, 2 * r_pad) &&
+              make_map(s, &maps.m[3], cat16, 2 * d, 2 * (uint64_t)r_pad, 2 * r_pad) && make_map(s, &maps.m[4], w.w_proj, 2 * d, d, 128);
+    for (int l = 0; l < D && ok; ++l) {
+        const mrp_module_layer &y = w.layers[l];
+        const int b = 5 + 7 * l;
+        ok = make_map(s, &maps.m[b], y.w_q, d, d, 128) && make_map(s, &maps.m[b + 1], y.w_k, d, d, 128) &&
+             make_map(s, &maps.m[b + 2], y.w_v, d, d, 128) && make_map(s, &maps.m[b + 3], y.w_o, d, d, 128) &&
+             make_map(s, &maps.m[b + 4], y.w_gate, d, F, 64) && make_map(s, &maps.m[b + 5], y.w_up, d, F, 64) &&
+             make_map(s, &maps.m[b + 6], y.w_down, F, d, 128);
+    }
+    if (!ok) return note_err(c, cudaErrorInvalidValue, "tensor map (module step)");
     int i = 0;
+    auto plain = [&](int kind) -> ChainPhase & {           // a phase without a product
+        ChainPhase &ph = p.ph[i++];
+        ph.kind = kind; ph.n_tiles = 0; ph.n_split = 1; ph.k_chunks = 1; ph.ssq_in = -1; ph.zero_slot0 = -1; ph.zero_slot1 = -1;
+        return ph;
+    };
     auto lin = [&](int k_chunks, int n_tiles, int n_split, int map_x, int map_w) -> ChainPhase & {
         ChainPhase &ph = p.ph[i++];
         ph.kind = CH_LIN; ph.k_chunks = k_chunks; ph.n_tiles = n_tiles; ph.n_split = n_split; ph.w_rows = d;
         ph.map_x = map_x; ph.map_w0 = map_w; ph.map_w1 = map_w; ph.ssq_in = -1; ph.zero_slot0 = -1; ph.zero_slot1 = -1;
         return ph;
     };
-    if (w_proj) {
-        ChainPhase &ph = lin(2 * d / kBK, d_tiles, sp_proj, 10, 11);
-        ph.lin_out = z; ph.gamma_next = (const __nv_bfloat16 *)y.g_attn; ph.xg_next = xa; ph.ssq_idx = s_in;
+    // slots of the fixed-point sums of squares: 0 / 1 alternate as the attention norm of layer l / l + 1, 3 is the MLP norm;
+    // slot 0 is cleared before the launch, the others by the first phase
+    const int s_mlp = 3;
+    {
+        ChainPhase &ph = plain(CH_CAT);
+        ph.zero_slot0 = 1; ph.zero_slot1 = s_mlp;
     }
     {
-        ChainPhase &ph = lin(d / kBK, 3 * d_tiles, sp_qkv, 0, 3);
-        ph.lin_out = q; ph.lin_out1 = k; ph.lin_out2 = v; ph.lin3_tiles = d_tiles; ph.ssq_in = s_in;
+        ChainPhase &ph = lin(2 * d / kBK, d_tiles, sp_proj, 3, 4);
+        ph.lin_out = z; ph.gamma_next = (const __nv_bfloat16 *)w.layers[0].g_attn; ph.xg_next = xa; ph.ssq_idx = 0;
     }
-    p.ph[0].zero_slot0 = s_mlp; p.ph[0].zero_slot1 = s_next;      // (with w_proj: s_in was cleared before the launch)
-    {
-        ChainPhase &ph = p.ph[i++];
-        ph.kind = CH_ATT; ph.n_tiles = 0; ph.n_split = 1; ph.k_chunks = 1; ph.zero_slot0 = -1; ph.zero_slot1 = -1;
-        ph.att_q = q; ph.att_k = k; ph.att_v = v; ph.att_out = xb; ph.att_L = L; ph.att_H = n_attn_heads;
+    for (int l = 0; l < D; ++l) {
+        const mrp_module_layer &y = w.layers[l];
+        const int b = 5 + 7 * l, s_in = l & 1, s_next = 1 - s_in;
+        {
+            ChainPhase &ph = lin(d / kBK, 3 * d_tiles, sp_qkv, 0, b);
+            ph.lin_out = q; ph.lin_out1 = k; ph.lin_out2 = v; ph.lin3_tiles = d_tiles; ph.ssq_in = s_in;
+            if (l > 0) { ph.zero_slot0 = s_next; ph.zero_slot1 = s_mlp; }     // (their readers are behind us, their writers ahead)
+        }
+        {
+            ChainPhase &ph = plain(CH_ATT);
+            ph.att_q = q; ph.att_k = k; ph.att_v = v; ph.att_out = xb; ph.att_L = L; ph.att_H = H;
+        }
+        {
+            ChainPhase &ph = lin(d / kBK, d_tiles, sp_o, 2, b + 3);
+            ph.lin_out = z; ph.lin_acc = 1; ph.gamma_next = (const __nv_bfloat16 *)y.g_mlp; ph.xg_next = xa; ph.ssq_idx = s_mlp;
+        }
+        {
+            ChainPhase &ph = p.ph[i++];
+            ph.kind = CH_GU; ph.k_chunks = d / kBK; ph.n_tiles = gu_tiles; ph.n_split = sp_gu; ph.w_rows = F;
+            ph.map_x = 0; ph.map_w0 = b + 4; ph.map_w1 = b + 5; ph.ssq_idx = s_mlp; ph.ssq_in = -1; ph.zero_slot0 = -1; ph.zero_slot1 = -1;
+        }
+        {
+            ChainPhase &ph = lin(F / kBK, d_tiles, sp_dn, 1, b + 6);
+            const void *g_next = l + 1 < D ? w.layers[l + 1].g_attn : nullptr;
+            ph.lin_out = z; ph.lin_acc = 1;
+            ph.gamma_next = (const __nv_bfloat16 *)g_next; ph.xg_next = g_next ? xa : nullptr; ph.ssq_idx = s_next;
+        }
     }
-    {
-        ChainPhase &ph = lin(d / kBK, d_tiles, sp_o, 2, 6);
-        ph.lin_out = z; ph.lin_acc = 1; ph.gamma_next = (const __nv_bfloat16 *)y.g_mlp; ph.xg_next = xa; ph.ssq_idx = s_mlp;
-    }
-    {
-        ChainPhase &ph = p.ph[i++];
-        ph.kind = CH_GU; ph.k_chunks = d / kBK; ph.n_tiles = gu_tiles; ph.n_split = sp_gu; ph.w_rows = F;
-        ph.map_x = 0; ph.map_w0 = 7; ph.map_w1 = 8; ph.ssq_idx = s_mlp; ph.zero_slot0 = -1; ph.zero_slot1 = -1;
-    }
-    {
-        ChainPhase &ph = lin(F / kBK, d_tiles, sp_dn, 1, 9);
-        ph.lin_out = z; ph.lin_acc = 1;
-        ph.gamma_next = (const __nv_bfloat16 *)gamma_next; ph.xg_next = gamma_next ? xa : nullptr; ph.ssq_idx = s_next;
-    }
+    plain(CH_FIN);
     p.n_phases = i;
-    // arrival counters and the grid barrier start at zero
-    cudaError_t e = cudaMemsetAsync(c->ws + c->lay.sk_counters, 0, (size_t)kSkMaxTiles * 4, st);
-    if (e != cudaSuccess) return note_err(c, e, "module layer, counters");
+    // arrival counters, the grid barrier and the first slot of the sums of squares start at zero
+    cudaError_t e = cudaMemsetAsync(bar_mem, 0, ((size_t)kModChainPhases * kChTilesPerPhase + 1) * 4, st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(c->ws + c->lay.ssq_fix, 0, (size_t)128 * 8, st);
+    if (e != cudaSuccess) return note_err(c, e, "module step, counters");
     switch (r_pad) {
     case 16: e = chain_launch<16, 1, true>(maps, p, G, smem, st); break;
     case 32: e = chain_launch<32, 1, true>(maps, p, G, smem, st); break;
@@ -986,7 +1105,7 @@ cudaError_t sk_module_layer(Ctx *c, int n, int L, int n_attn_heads, const mrp_mo
     default: e = chain_launch<128, 1, true>(maps, p, G, smem, st); break;
     }
     c->launches++;
-    return note_err(c, e, "module layer kernel");
+    return note_err(c, e, "module step kernel");
 }
 
 }  // namespace mrp
