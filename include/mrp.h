@@ -261,10 +261,11 @@ int mrp_draft_kl(mrp_ctx *ctx, const void *hidden, const float *logits0, const f
  * one application per call so that the caller can reveal tokens between MRP steps: unlike the reduced
  * head above, this module reads the embeddings of the tokens revealed so far, so step k + 1 depends on
  * the reveals of step k and the LM head runs once per step.
- * The paper fixes the parts and leaves the details open; the form implemented (first slice: CUDA-core
- * kernels for the module itself -- one cooperative kernel for the whole step when B * L <= 4; above that one
- * kernel per matrix product, on the tensor cores for tensor-core contexts whose module matrices are 16-byte
- * aligned -- and the context's own LM-head kernels behind it):
+ * The paper fixes the parts and leaves the details open; the form implemented (one MRP step per call:
+ * the module itself as one cooperative tensor-core kernel per step for up to 64 positions on tensor-core
+ * contexts (d % 128 == 0, at most 4 layers, 16-byte aligned matrices), one tensor-core kernel per matrix product
+ * above that; on other contexts one cooperative CUDA-core kernel per step when B * L <= 4, else one CUDA-core kernel
+ * per product; the context's own LM-head kernels behind it):
  *     e_i = emb[x_i]  (emb[mask_token] where x_i = -1);   z_i = W_proj [h_i ; e_i]
  *     n_layers times:  z += W_o Attn(RMSNorm(z) g_attn),  attention over the positions of the same block,
  *                      bidirectional, n_attn_heads heads, no positional term;
