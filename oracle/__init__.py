@@ -47,6 +47,7 @@ def _load():
         _lib.mrp_oracle_draft_from_hidden.restype = ctypes.c_int
         _lib.mrp_oracle_draft_kl.restype = ctypes.c_int
         _lib.mrp_oracle_module.restype = ctypes.c_int
+        _lib.mrp_oracle_module_prefix.restype = ctypes.c_int
         _lib.mrp_oracle_select.restype = ctypes.c_int
         _lib.mrp_oracle_verify.restype = ctypes.c_int
     return _lib
@@ -193,10 +194,15 @@ def draft_kl(hidden, logits0, teacher, heads, w_lm, K=None, row_index=None, eps=
 MODULE_LAYER_KEYS = ("g_attn", "w_q", "w_k", "w_v", "w_o", "g_mlp", "w_gate", "w_up", "w_down")
 
 
-def module(hidden, tokens, B, L, emb, w_proj, layers, w_lm, n_attn_heads, mask_token, row_index=None, eps=1e-6):
+def module(hidden, tokens, B, L, emb, w_proj, layers, w_lm, n_attn_heads, mask_token, row_index=None, eps=1e-6,
+           prefix=None, want_kv=False):
     """One application of the token-conditioned MRP module g(x_t, h) (Sec. 3.2; Algorithm 2) to the L
     positions of each of B blocks: returns (delta_h [B*L, d], delta_l [M, V]) in float64.  ``layers`` is a
-    sequence of dicts with the arrays named in MODULE_LAYER_KEYS; ``tokens`` [B*L] with -1 = masked."""
+    sequence of dicts with the arrays named in MODULE_LAYER_KEYS; ``tokens`` [B*L] with -1 = masked.
+    ``prefix`` = (k, v, length) gives the clean prefix of Fig. 1(c): k, v are sequences of D arrays
+    [B, cap, d] (the keys and values of the prefix positions per layer), length [B] the rows in use per
+    sequence.  With ``want_kv`` the result gains (k, v): per layer the [B*L, d] float64 keys and values of
+    the block's own positions."""
     lib = _load()
     hidden, emb, w_proj, w_lm = _f32(hidden), _f32(emb), _f32(w_proj), _f32(w_lm)
     tokens = _i32(tokens)
@@ -223,14 +229,41 @@ def module(hidden, tokens, B, L, emb, w_proj, layers, w_lm, n_attn_heads, mask_t
         M = ri.shape[0]
     delta_h = np.zeros((n, d), np.float64)
     delta_l = np.zeros((M, V), np.float64)
-    rc = lib.mrp_oracle_module(
+    pk = pv = plen = None
+    cap = 0
+    if prefix is not None:
+        ks, vs, length = prefix
+        assert len(ks) == D and len(vs) == D
+        plen = _i32(length)
+        assert plen.shape == (B,)
+        lk, lv = [], []
+        for a, b in zip(ks, vs):
+            a, b = _f32(a), _f32(b)
+            assert a.ndim == 3 and a.shape == b.shape and a.shape[0] == B and a.shape[2] == d
+            cap = a.shape[1]
+            keep += [a, b]
+            lk.append(_p(a, ctypes.c_float))
+            lv.append(_p(b, ctypes.c_float))
+        pk, pv = PtrArr(*lk), PtrArr(*lv)
+    ko = vo = None
+    k_out = v_out = None
+    if want_kv:
+        DArr = ctypes.POINTER(ctypes.c_double) * max(D, 1)
+        k_out = [np.zeros((n, d), np.float64) for _ in range(D)]
+        v_out = [np.zeros((n, d), np.float64) for _ in range(D)]
+        ko = DArr(*[_p(a, ctypes.c_double) for a in k_out])
+        vo = DArr(*[_p(a, ctypes.c_double) for a in v_out])
+    rc = lib.mrp_oracle_module_prefix(
         ctypes.c_int(d), ctypes.c_int(F), ctypes.c_int(V), ctypes.c_int(D), ctypes.c_int(n_attn_heads), ctypes.c_int(B),
         ctypes.c_int(L), ctypes.c_int(mask_token), ctypes.c_double(eps), _p(hidden, ctypes.c_float),
         _p(tokens, ctypes.c_int32), _p(emb, ctypes.c_float), _p(w_proj, ctypes.c_float),
         *[arrs[k] for k in MODULE_LAYER_KEYS], _p(w_lm, ctypes.c_float), _p(ri, ctypes.c_int32), ctypes.c_int(M),
-        _p(delta_h, ctypes.c_double), _p(delta_l, ctypes.c_double))
+        _p(delta_h, ctypes.c_double), _p(delta_l, ctypes.c_double), pk, pv, _p(plen, ctypes.c_int32), ctypes.c_int(cap),
+        ko, vo)
     if rc != 0:
-        raise RuntimeError("mrp_oracle_module failed (%d)" % rc)
+        raise RuntimeError("mrp_oracle_module_prefix failed (%d)" % rc)
+    if want_kv:
+        return delta_h, delta_l, k_out, v_out
     return delta_h, delta_l
 
 

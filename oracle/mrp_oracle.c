@@ -474,21 +474,38 @@ int mrp_oracle_verify(const int32_t *draft_tok, const int32_t *verify_tok,
  * Outputs: delta_h [B*L, d] double for every position; delta_l [M, V] double for the masked rows
  * listed in row_index (may be NULL with M = 0).  tokens [B*L] int32, -1 = masked.
  * Layer weights: arrays of D pointers each.  Returns 0, or -1 on bad arguments.
+ *
+ * The clean prefix (Fig. 1(c): the new block is decoded given the committed clean prefix, under the
+ * same attention pattern as in training, where a block attends to itself and to the clean blocks in
+ * front of it).  Reading: what a block sees of its prefix are the keys and values the module's own
+ * layers produced for the prefix positions when those were committed; they are inputs here,
+ * prefix_k / prefix_v = D pointers to [B, prefix_cap, d] arrays of which sequence b uses the first
+ * prefix_len[b] rows (NULL = no prefix), and position i of block b attends to those rows and to the L
+ * positions of its block in one softmax.  k_out / v_out (optional, D pointers to [B*L, d] doubles)
+ * receive the keys and values of the block's own positions per layer: what a caller appends to the
+ * prefix once the block is committed.
  */
-int mrp_oracle_module(int d, int F, int V, int D, int n_attn_heads, int B, int L, int mask_token, double eps,
-                      const float *hidden, const int32_t *tokens, const float *emb, const float *w_proj,
-                      const float *const *g_attn, const float *const *w_q, const float *const *w_k,
-                      const float *const *w_v, const float *const *w_o, const float *const *g_mlp,
-                      const float *const *w_gate, const float *const *w_up, const float *const *w_down,
-                      const float *w_lm, const int32_t *row_index, int M, double *delta_h, double *delta_l)
+int mrp_oracle_module_prefix(int d, int F, int V, int D, int n_attn_heads, int B, int L, int mask_token, double eps,
+                             const float *hidden, const int32_t *tokens, const float *emb, const float *w_proj,
+                             const float *const *g_attn, const float *const *w_q, const float *const *w_k,
+                             const float *const *w_v, const float *const *w_o, const float *const *g_mlp,
+                             const float *const *w_gate, const float *const *w_up, const float *const *w_down,
+                             const float *w_lm, const int32_t *row_index, int M, double *delta_h, double *delta_l,
+                             const float *const *prefix_k, const float *const *prefix_v, const int32_t *prefix_len,
+                             int prefix_cap, double *const *k_out, double *const *v_out)
 {
     if (d <= 0 || F <= 0 || V <= 0 || D < 0 || n_attn_heads <= 0 || d % n_attn_heads || B <= 0 || L <= 0) return -1;
+    if (prefix_k && (!prefix_v || !prefix_len || prefix_cap < 0)) return -1;
+    if (prefix_k)
+        for (int b = 0; b < B; ++b)
+            if (prefix_len[b] < 0 || prefix_len[b] > prefix_cap) return -1;
     const int dh = d / n_attn_heads;
     const size_t n = (size_t)B * L;
+    const int max_keys = L + (prefix_k ? prefix_cap : 0);
     double *z = (double *)malloc(sizeof(double) * n * d), *nn = (double *)malloc(sizeof(double) * n * d);
     double *q = (double *)malloc(sizeof(double) * n * d), *k = (double *)malloc(sizeof(double) * n * d);
     double *v = (double *)malloc(sizeof(double) * n * d), *o = (double *)malloc(sizeof(double) * n * d);
-    double *a = (double *)malloc(sizeof(double) * (size_t)F), *p = (double *)malloc(sizeof(double) * (size_t)L);
+    double *a = (double *)malloc(sizeof(double) * (size_t)F), *p = (double *)malloc(sizeof(double) * (size_t)max_keys);
     if (!z || !nn || !q || !k || !v || !o || !a || !p) { free(z); free(nn); free(q); free(k); free(v); free(o); free(a); free(p); return -1; }
 
     /* fusion of hidden state and token embedding */
@@ -522,26 +539,39 @@ int mrp_oracle_module(int d, int F, int V, int D, int n_attn_heads, int B, int L
                 }
                 q[i * d + j] = sq; k[i * d + j] = sk; v[i * d + j] = sv;
             }
-        for (int b = 0; b < B; ++b)
+        if (k_out) memcpy(k_out[layer], k, sizeof(double) * n * d);
+        if (v_out) memcpy(v_out[layer], v, sizeof(double) * n * d);
+        for (int b = 0; b < B; ++b) {
+            /* the keys of a position: the P_b rows of its sequence's clean prefix (Fig. 1(c)), then its block */
+            const int P = prefix_k ? prefix_len[b] : 0;
+            const float *pk = prefix_k ? prefix_k[layer] + (size_t)b * prefix_cap * d : NULL;
+            const float *pv = prefix_k ? prefix_v[layer] + (size_t)b * prefix_cap * d : NULL;
             for (int hd = 0; hd < n_attn_heads; ++hd)
                 for (int i = 0; i < L; ++i) {
                     const size_t ri = ((size_t)b * L + i) * d + (size_t)hd * dh;
                     double mx = -INFINITY;
-                    for (int j = 0; j < L; ++j) {
-                        const size_t rj = ((size_t)b * L + j) * d + (size_t)hd * dh;
+                    for (int j = 0; j < P + L; ++j) {
                         double s = 0.0;
-                        for (int c = 0; c < dh; ++c) s += q[ri + c] * k[rj + c];
+                        if (j < P) {
+                            const float *kr = pk + (size_t)j * d + (size_t)hd * dh;
+                            for (int c = 0; c < dh; ++c) s += q[ri + c] * (double)kr[c];
+                        } else {
+                            const size_t rj = ((size_t)b * L + (j - P)) * d + (size_t)hd * dh;
+                            for (int c = 0; c < dh; ++c) s += q[ri + c] * k[rj + c];
+                        }
                         p[j] = s / sqrt((double)dh);
                         if (p[j] > mx) mx = p[j];
                     }
                     double sum = 0.0;
-                    for (int j = 0; j < L; ++j) { p[j] = exp(p[j] - mx); sum += p[j]; }
+                    for (int j = 0; j < P + L; ++j) { p[j] = exp(p[j] - mx); sum += p[j]; }
                     for (int c = 0; c < dh; ++c) {
                         double s = 0.0;
-                        for (int j = 0; j < L; ++j) s += p[j] * v[((size_t)b * L + j) * d + (size_t)hd * dh + c];
+                        for (int j = 0; j < P; ++j) s += p[j] * (double)pv[(size_t)j * d + (size_t)hd * dh + c];
+                        for (int j = 0; j < L; ++j) s += p[P + j] * v[((size_t)b * L + j) * d + (size_t)hd * dh + c];
                         o[ri + c] = s / sum;
                     }
                 }
+        }
         for (size_t i = 0; i < n; ++i)
             for (int j = 0; j < d; ++j) {
                 double s = 0.0;
@@ -585,4 +615,17 @@ int mrp_oracle_module(int d, int F, int V, int D, int n_attn_heads, int B, int L
     }
     free(z); free(nn); free(q); free(k); free(v); free(o); free(a); free(p);
     return 0;
+}
+
+/* The module without a clean prefix: attention over the positions of the block alone. */
+int mrp_oracle_module(int d, int F, int V, int D, int n_attn_heads, int B, int L, int mask_token, double eps,
+                      const float *hidden, const int32_t *tokens, const float *emb, const float *w_proj,
+                      const float *const *g_attn, const float *const *w_q, const float *const *w_k,
+                      const float *const *w_v, const float *const *w_o, const float *const *g_mlp,
+                      const float *const *w_gate, const float *const *w_up, const float *const *w_down,
+                      const float *w_lm, const int32_t *row_index, int M, double *delta_h, double *delta_l)
+{
+    return mrp_oracle_module_prefix(d, F, V, D, n_attn_heads, B, L, mask_token, eps, hidden, tokens, emb, w_proj, g_attn, w_q,
+                                    w_k, w_v, w_o, g_mlp, w_gate, w_up, w_down, w_lm, row_index, M, delta_h, delta_l, NULL, NULL,
+                                    NULL, 0, NULL, NULL);
 }

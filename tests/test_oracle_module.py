@@ -135,3 +135,104 @@ def test_numpy_statistics_agree_with_the_c_statistics():
     assert np.allclose(conf, r.conf[0], atol=1e-15) and np.allclose(lse, r.lse[0], atol=1e-13)
     assert np.array_equal(tok, r.token[0]) and np.allclose(margin, r.margin[0], atol=1e-13)
     assert tok[2] == 3 and margin[2] == 0
+
+
+# ---- the clean prefix of Fig. 1(c): keys and values of committed positions as inputs ----
+
+def _tail_problem(seed=5, B=2, P=4, L=3, D=2):
+    mw, hidden, tokens, w_lm = problem(seed=seed, D=D, B=B, L=P + L)
+    long_h, _, k_long, v_long = oracle.module(hidden, tokens, B, P + L, mw.emb, mw.w_proj, mw.layers, w_lm, mw.n_attn_heads,
+                                              mw.mask_token, want_kv=True)
+    d = hidden.shape[1]
+    tail = (np.arange(B * (P + L)) % (P + L)) >= P
+    cap = P + 2                                                         # rows beyond the length: never read
+    ks = [np.full((B, cap, d), np.nan, np.float32) for _ in range(D)]
+    vs = [np.full((B, cap, d), np.nan, np.float32) for _ in range(D)]
+    for l in range(D):
+        ks[l][:, :P] = k_long[l].reshape(B, P + L, d)[:, :P]
+        vs[l][:, :P] = v_long[l].reshape(B, P + L, d)[:, :P]
+    return mw, hidden, tokens, w_lm, long_h, tail, ks, vs, k_long, v_long
+
+
+def test_block_behind_a_prefix_equals_the_tail_of_the_longer_block():
+    # Given the per-layer keys and values of the first P positions, the last L positions of a block of P + L
+    # compute exactly what a block of L behind that prefix computes: the prefix enters through nothing else.
+    B, P, L, D = 2, 4, 3, 2
+    mw, hidden, tokens, w_lm, long_h, tail, ks, vs, k_long, v_long = _tail_problem(B=B, P=P, L=L, D=D)
+    rows = np.array([0, 4, 5], np.int32)
+    dh, dl, k_out, v_out = oracle.module(hidden[tail], tokens[tail], B, L, mw.emb, mw.w_proj, mw.layers, w_lm, mw.n_attn_heads,
+                                         mw.mask_token, row_index=rows, prefix=(ks, vs, np.full(B, P, np.int32)), want_kv=True)
+    assert np.abs(long_h[tail]).max() > 0.1
+    assert np.allclose(dh, long_h[tail], rtol=0, atol=2e-6)             # (the prefix rows were rounded to fp32)
+    assert np.allclose(dl, dh[rows] @ w_lm.astype(np.float64).T, rtol=0, atol=1e-11)
+    for l in range(D):
+        assert np.allclose(k_out[l], k_long[l][tail], rtol=0, atol=2e-6) and np.allclose(v_out[l], v_long[l][tail], rtol=0, atol=2e-6)
+    # ... and the prefix matters: without it the block computes something else
+    alone, _ = run(mw, hidden[tail], tokens[tail], w_lm, B, L)
+    assert np.abs(alone - long_h[tail]).max() > 1e-3
+
+
+def test_prefix_lengths_are_per_sequence():
+    B, P, L, D = 2, 4, 3, 2
+    mw, hidden, tokens, w_lm, long_h, tail, ks, vs, _, _ = _tail_problem(B=B, P=P, L=L, D=D)
+    alone, _ = run(mw, hidden[tail], tokens[tail], w_lm, B, L)
+    dh, _ = oracle.module(hidden[tail], tokens[tail], B, L, mw.emb, mw.w_proj, mw.layers, w_lm, mw.n_attn_heads, mw.mask_token,
+                          prefix=(ks, vs, np.array([P, 0], np.int32)))
+    assert np.allclose(dh[:L], long_h[tail][:L], rtol=0, atol=2e-6)     # sequence 0: behind its prefix
+    assert np.array_equal(dh[L:], alone[L:])                            # sequence 1: no prefix rows in use
+    # a shorter prefix is another function
+    dh2, _ = oracle.module(hidden[tail], tokens[tail], B, L, mw.emb, mw.w_proj, mw.layers, w_lm, mw.n_attn_heads, mw.mask_token,
+                           prefix=(ks, vs, np.array([P - 1, 0], np.int32)))
+    assert np.abs(dh2[:L] - dh[:L]).max() > 1e-4 and np.array_equal(dh2[L:], dh[L:])
+
+
+def test_zero_keys_average_the_values_of_prefix_and_block():
+    # W_k = 0 and zero prefix keys: every score is 0, the softmax is uniform over the P_b + L keys and the
+    # attention output is the plain mean of the prefix's and the block's values (one layer, W_o = I, no MLP)
+    B, L, D = 2, 3, 1
+    mw, hidden, tokens, w_lm = problem(seed=8, D=D, B=B, L=L)
+    d = hidden.shape[1]
+    lay = dict(mw.layers[0], w_k=np.zeros((d, d), np.float32), w_o=np.eye(d, dtype=np.float32),
+               w_down=np.zeros_like(mw.layers[0]["w_down"]))
+    rng = np.random.default_rng(1)
+    cap, plen = 5, np.array([5, 2], np.int32)
+    pv = rng.standard_normal((B, cap, d)).astype(np.float32)
+    z0, _, _, v_blk = oracle.module(hidden, tokens, B, L, mw.emb, mw.w_proj, [dict(lay, w_o=np.zeros((d, d), np.float32))], w_lm,
+                                    mw.n_attn_heads, mw.mask_token, want_kv=True)
+    dh, _ = oracle.module(hidden, tokens, B, L, mw.emb, mw.w_proj, [lay], w_lm, mw.n_attn_heads, mw.mask_token,
+                          prefix=([np.zeros((B, cap, d), np.float32)], [pv], plen))
+    for b in range(B):
+        mean = (pv[b, :plen[b]].astype(np.float64).sum(axis=0) + v_blk[0][b * L:(b + 1) * L].sum(axis=0)) / (plen[b] + L)
+        assert np.allclose(dh[b * L:(b + 1) * L], z0[b * L:(b + 1) * L] + mean, rtol=0, atol=1e-12)
+
+
+def test_prefix_matches_library_implementation():
+    # second implementation on library routines: softmax over the concatenated keys, one sequence at a time
+    B, L, D = 2, 3, 2
+    mw, hidden, tokens, w_lm = problem(seed=9, D=D, B=B, L=L)
+    d, H = hidden.shape[1], mw.n_attn_heads
+    dh_ = d // H
+    rng = np.random.default_rng(2)
+    cap, plen = 6, np.array([6, 3], np.int32)
+    ks = [rng.standard_normal((B, cap, d)).astype(np.float32) for _ in range(D)]
+    vs = [rng.standard_normal((B, cap, d)).astype(np.float32) for _ in range(D)]
+    got, _ = oracle.module(hidden, tokens, B, L, mw.emb, mw.w_proj, mw.layers, w_lm, H, mw.mask_token, prefix=(ks, vs, plen))
+    tok = np.where(tokens >= 0, tokens, mw.mask_token)
+    z = np.concatenate([hidden.astype(np.float64), mw.emb[tok].astype(np.float64)], axis=1) @ mw.w_proj.astype(np.float64).T
+    rms = lambda x, g: x / np.sqrt((x * x).mean(axis=1, keepdims=True) + 1e-6) * g.astype(np.float64)
+    for l, lay in enumerate(mw.layers):
+        n = rms(z, lay["g_attn"])
+        q, k, v = (n @ lay[w].astype(np.float64).T for w in ("w_q", "w_k", "w_v"))
+        o = np.zeros_like(z)
+        for b in range(B):
+            kk = np.concatenate([ks[l][b, :plen[b]].astype(np.float64), k[b * L:(b + 1) * L]])
+            vv = np.concatenate([vs[l][b, :plen[b]].astype(np.float64), v[b * L:(b + 1) * L]])
+            for h in range(H):
+                c = slice(h * dh_, (h + 1) * dh_)
+                p = softmax(q[b * L:(b + 1) * L, c] @ kk[:, c].T / np.sqrt(dh_), axis=-1)
+                o[b * L:(b + 1) * L, c] = p @ vv[:, c]
+        z = z + o @ lay["w_o"].astype(np.float64).T
+        n = rms(z, lay["g_mlp"])
+        g = n @ lay["w_gate"].astype(np.float64).T
+        z = z + (g * expit(g) * (n @ lay["w_up"].astype(np.float64).T)) @ lay["w_down"].astype(np.float64).T
+    assert np.allclose(got, z, rtol=0, atol=1e-11)
