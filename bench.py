@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of the MRP drafting step on B200.
 
-    python bench.py [--gpus N] [--steps S] [--warmup W] [--config all|0..3|module|module:2|module:L16|sweep:M:K|sweep]
+    python bench.py [--gpus N] [--steps S] [--warmup W] [--config all|0..3|module|module:2|module:L16|module:P1024|sweep:M:K|sweep]
                     [--impl ours|reference]
 
 A step is one pass of the whole hot path over one batch of synthetic input: mrp_draft (row
@@ -63,7 +63,8 @@ def parse_args():
     ap.add_argument("--config", default="all",
                     help="all = the five configurations in one line (default); 0..3 = one configuration; "
                          "module / module:2 / module:L16 = the token-conditioned module at the decode shape, at "
-                         "spec_8b's shape, at the decode shape with one block of 16 positions; "
+                         "spec_8b's shape, at the decode shape with one block of 16 positions (:P<n> adds a clean prefix of n "
+                         "positions to the module's attention); "
                          "sweep:M:K = one roofline-sweep point; sweep = all 21 points, one line each")
     ap.add_argument("--min-seconds", type=float, default=1.0,
                     help="GPU time per workload spent in timed batches of --steps steps")
@@ -638,12 +639,13 @@ class Bench:
                 "steps": n_e2e, "ms_per_step": dt / n_e2e * 1e3, "mode": e2e_mode}
 
 
-def run_module_workload(bench, cpu_budget_s, which=1, block_len=None):
+def run_module_workload(bench, cpu_budget_s, which=1, block_len=None, prefix=0):
     """The token-conditioned module at the shape of configuration `which` (1: the decode shape, one block of 4
     positions; 2: 32 blocks of 4, d = 4096): a step is the K = 3 MRP steps that follow one backbone forward in
     direct decoding (Algorithm 2), each = mrp_module_step (module forward + one LM-head pass) +
     mrp_reveal_remask + mrp_commit, the reveals of a step conditioning the next.  Drafted tokens per step:
-    K * B (one reveal per block and MRP step)."""
+    K * B (one reveal per block and MRP step).  prefix > 0: every sequence has a clean prefix of that many positions
+    in the module's key / value cache (Fig. 1(c)), random values."""
     import numpy as np
     import torch
     import oracle
@@ -652,7 +654,7 @@ def run_module_workload(bench, cpu_budget_s, which=1, block_len=None):
     base = synth.CONFIGS[which]
     if block_len:                                      # the paper's block length (Sec. 4.1) instead of the configuration's
         base = dict(base, L=block_len, name="%s_L%d" % (base["name"], block_len))
-    cfg = dict(base, name="module_" + base["name"])
+    cfg = dict(base, name="module_" + base["name"] + ("_P%d" % prefix if prefix else ""))
     w, heads, w_lm = bench.weights_for(base, str(which))
     big = base["d"] >= 4096
     _, inp = synth.make_config(base, w, logits_fn=harness.device_logits_fn(w_lm) if big else None)
@@ -666,6 +668,14 @@ def run_module_workload(bench, cpu_budget_s, which=1, block_len=None):
     up = lambda a: harness.to_device(a, "bf16", dev)
     binding.mrp_module_attach(ctx, up(mw.emb), up(mw.w_proj), [{k: up(v) for k, v in lay.items()} for lay in mw.layers],
                               n_attn, mw.mask_token)
+    caches = None
+    if prefix:
+        g = torch.Generator().manual_seed(13)
+        host_kv = [(torch.randn((B, prefix, d), generator=g).bfloat16(), torch.randn((B, prefix, d), generator=g).bfloat16())
+                   for _ in range(MODULE_LAYERS)]
+        caches = [(k.to(dev), v.to(dev)) for k, v in host_kv]
+        plen = torch.full((B,), prefix, dtype=torch.int32, device=dev)
+        binding.mrp_module_set_prefix(ctx, caches, plen)
     hid0 = harness.to_device(inp.hidden, "bf16", dev)
     l0 = torch.from_numpy(inp.logits0).to(dev)
     h_state = torch.empty((n, d), device=dev)
@@ -716,8 +726,9 @@ def run_module_workload(bench, cpu_budget_s, which=1, block_len=None):
     res["phases"] = {"module_ms_per_mrp_step": ms_mod / max(n_calls, 1), "lm_head_ms_per_mrp_step": ms_lm / max(n_calls, 1),
                      "combine_ms_per_mrp_step": ms_comb / max(n_calls, 1), "family": ctx.family,
                      "module": "D = %d layers, %d attention heads, %s" % (
-                         MODULE_LAYERS, n_attn, "one CUDA-core kernel per step" if n <= 4 else
-                         "products on the row-major tcgen05 kernel")}
+                         MODULE_LAYERS, n_attn, "one cooperative tcgen05 kernel per step" if n <= 64 else
+                         "products on the row-major tcgen05 kernel"),
+                     "prefix_positions": prefix}
     # end to end with host buffers: hidden states, base logits and the block's tokens in, the block state out
     e2e = None
     if not args.no_e2e:
@@ -751,12 +762,16 @@ def run_module_workload(bench, cpu_budget_s, which=1, block_len=None):
         ns = Bs * L
         ri_h = np.flatnonzero(tokens0[:ns] < 0).astype(np.int32)
         Ks = K if not big else 1
+        pre = None
+        if prefix:
+            pre = ([k[:Bs].float().numpy() for k, _ in host_kv], [v[:Bs].float().numpy() for _, v in host_kv],
+                   np.full(Bs, prefix, np.int32))
         t0 = time.perf_counter()
         reps = 0
         while time.perf_counter() - t0 < min(cpu_budget_s, 6.0) or reps == 0:
             for k in range(Ks):
                 oracle.module(inp.hidden[:ns], tokens0[:ns], Bs, L, mw.emb, mw.w_proj, mw.layers, w.w_lm, n_attn,
-                              mw.mask_token, row_index=ri_h[:len(ri_h) - Bs * k])
+                              mw.mask_token, row_index=ri_h[:len(ri_h) - Bs * k], prefix=pre)
             reps += 1
         cpu = {"value": Ks * Bs * reps / (time.perf_counter() - t0), "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
                "sample": "the module oracle, %d application(s) on %d of %d blocks, %d repetitions" % (Ks, Bs, B, reps)}
@@ -801,11 +816,12 @@ def main():
     results = {}
     for name in names:
         if name == "module" or name.startswith("module:"):
-            # module[:1|:2][:L<block length>], e.g. module:L16 (decode shape, one block of 16), module:2:L2
+            # module[:1|:2][:L<block length>][:P<prefix positions>], e.g. module:L16 (decode shape, one block of 16), module:P1024
             parts = name.split(":")[1:]
             which = 2 if "2" in parts else 1
             blen = [int(x[1:]) for x in parts if x.startswith("L")]
-            results[name] = run_module_workload(bench, 5.0, which, blen[0] if blen else None)
+            pre = [int(x[1:]) for x in parts if x.startswith("P")]
+            results[name] = run_module_workload(bench, 5.0, which, blen[0] if blen else None, pre[0] if pre else 0)
         else:
             results[name] = bench.run_workload(name, 12.0 if name == head_name else 5.0)
     if bench.rank == 0:

@@ -315,6 +315,34 @@ int mrp_module_step(mrp_ctx *ctx, const int32_t *tokens, const void *hidden0, fl
                     const float *logits0, const int32_t *row_index, int32_t M, int32_t B, int32_t L,
                     int32_t first_step, const mrp_draft_out *out, void *cuda_stream);
 
+/*
+ * The clean prefix of the module's attention (Fig. 1(c): a new block is decoded given the committed clean
+ * prefix, under the attention pattern of training, where a block attends to itself and to the clean blocks in
+ * front of it).  What a block sees of its prefix are the keys and values the module's own layers produced for
+ * the prefix positions; the caller keeps them, per module layer, in a cache
+ *     k, v   DEVICE [max_seqs, prefix_cap, d], context dtype, 16-byte aligned
+ * of which sequence b (the b-th block of an mrp_module_step call) uses the first prefix_len[b] rows:
+ * position i of block b then attends to those rows and to the L positions of its block in one softmax.
+ *   layers      HOST array [n_layers] of the caches' DEVICE pointers (copied); NULL detaches the prefix
+ *   prefix_len  DEVICE [max_seqs] int32, read by every following mrp_module_step (the caller may change the
+ *               values between calls); an entry outside [0, prefix_cap] raises MRP_DEV_BAD_INDEX and is
+ *               clamped
+ *   append      != 0: every following mrp_module_step also stores the keys and values of its own L positions,
+ *               rounded to the context dtype, in rows prefix_len[b] .. prefix_len[b] + L - 1 of sequence b's
+ *               slab (what the caller does once a block is committed, with all its tokens revealed, before it
+ *               raises prefix_len[b] by L); a block that does not fit raises MRP_DEV_BAD_INDEX and stores
+ *               nothing.  The rows stored by a call are not among the rows it reads.
+ * Needs d / n_attn_heads <= 256.  With a prefix attached the module step runs as one cooperative tensor-core
+ * kernel where it does without (up to 64 positions), else as one kernel per matrix product.
+ * Errors: INVALID_ARG, UNSUPPORTED (no module attached, or heads wider than 256), NOMEM.
+ */
+typedef struct {
+    void *k, *v;
+} mrp_module_kv;
+
+int mrp_module_set_prefix(mrp_ctx *ctx, const mrp_module_kv *layers, const int32_t *prefix_len, int32_t prefix_cap,
+                          int32_t append);
+
 typedef enum { MRP_SELECT_STATIC = 0, MRP_SELECT_DYNAMIC_REMASK = 1 } mrp_select_mode;
 
 typedef struct {

@@ -37,7 +37,7 @@ EXPORTS = ("mrp_workspace_bytes", "mrp_create", "mrp_destroy", "mrp_draft", "mrp
            "mrp_profile_enable", "mrp_profile_read", "mrp_last_error",
            "mrp_reveal_remask_noalloc", "mrp_selftest_wait_timeout", "mrp_draft_from_hidden", "mrp_commit",
            "mrp_set_logits0_event", "mrp_set_input_rows", "mrp_fetch_status", "mrp_draft_kl", "mrp_draft_bf16_logits", "mrp_quantised_lm_head",
-           "mrp_module_workspace_bytes", "mrp_module_attach", "mrp_module_step")
+           "mrp_module_workspace_bytes", "mrp_module_attach", "mrp_module_step", "mrp_module_set_prefix")
 MRP_NOALLOC_MAX_POSITIONS = 65536
 MRP_ERR_CAPACITY = 7
 
@@ -86,6 +86,10 @@ class mrp_module_weights(ctypes.Structure):
                 ("layers", ctypes.POINTER(mrp_module_layer))]
 
 
+class mrp_module_kv(ctypes.Structure):
+    _fields_ = [("k", ctypes.c_void_p), ("v", ctypes.c_void_p)]
+
+
 class mrp_block_state(ctypes.Structure):
     _fields_ = [("tokens", ctypes.c_void_p), ("row_index", ctypes.c_void_p),
                 ("n_masked", ctypes.c_void_p), ("block_masked", ctypes.c_void_p)]
@@ -119,6 +123,9 @@ def _load():
     lib.mrp_module_workspace_bytes.argtypes = [ctypes.POINTER(mrp_config), ctypes.POINTER(mrp_module_weights)]
     lib.mrp_module_attach.restype = ctypes.c_int
     lib.mrp_module_attach.argtypes = [ctypes.c_void_p, ctypes.POINTER(mrp_module_weights), ctypes.c_void_p, ctypes.c_size_t]
+    lib.mrp_module_set_prefix.restype = ctypes.c_int
+    lib.mrp_module_set_prefix.argtypes = [ctypes.c_void_p, ctypes.POINTER(mrp_module_kv), ctypes.c_void_p, ctypes.c_int32,
+                                          ctypes.c_int32]
     lib.mrp_module_step.restype = ctypes.c_int
     lib.mrp_module_step.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
                                     ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
@@ -327,6 +334,33 @@ def mrp_module_step(ctx: Context, tokens, hidden0, h_state, logits0, row_index, 
                              int(M), int(B), int(L), int(bool(first_step)), ctypes.byref(out), _stream(stream))
     if rc != 0:
         raise MrpError("mrp_module_step", rc, lib.mrp_last_error(ctx.handle).decode())
+
+
+def mrp_module_set_prefix(ctx: Context, caches, prefix_len, append=False) -> None:
+    """Attach the clean prefix of the module's attention: ``caches`` a list (one entry per module layer) of
+    (k, v) CUDA tensors [max_seqs, prefix_cap, d] in the context dtype, ``prefix_len`` [max_seqs] int32 on the
+    device; ``caches`` None detaches.  With ``append`` the following steps also store their own keys and values
+    behind the prefix rows."""
+    if caches is None:
+        rc = lib.mrp_module_set_prefix(ctx.handle, None, None, 0, 0)
+        if rc != 0:
+            raise MrpError("mrp_module_set_prefix", rc)
+        return
+    tdtype = torch.float32 if ctx.cfg.dtype == MRP_F32 else torch.bfloat16
+    _check(prefix_len, torch.int32, "prefix_len")
+    arr = (mrp_module_kv * max(len(caches), 1))()
+    cap = 0
+    for i, (k, v) in enumerate(caches):
+        _check(k, tdtype, "prefix k")
+        _check(v, tdtype, "prefix v")
+        if k.dim() != 3 or k.shape != v.shape or k.shape[2] != ctx.cfg.d:
+            raise ValueError("prefix caches are [max_seqs, prefix_cap, d]")
+        cap = int(k.shape[1])
+        arr[i] = mrp_module_kv(k.data_ptr(), v.data_ptr())
+    rc = lib.mrp_module_set_prefix(ctx.handle, arr, _ptr(prefix_len), cap, int(bool(append)))
+    if rc != 0:
+        raise MrpError("mrp_module_set_prefix", rc)
+    ctx.prefix_keep = (caches, prefix_len)
 
 
 def mrp_set_input_rows(ctx: Context, n_rows: int) -> None:

@@ -218,6 +218,7 @@ void mrp_destroy(mrp_ctx *ctx)
     prof_release(ctx->c);
     if (ctx->c.use_tc) tc_destroy(&ctx->c);
     free(ctx->c.module_layers);
+    free(ctx->c.prefix_layers);
     free(ctx->c.heads);
     delete ctx;
 }
@@ -362,6 +363,39 @@ int mrp_module_attach(mrp_ctx *ctx, const mrp_module_weights *w, void *workspace
     c.module.layers = copy;
     c.module_ws = (char *)workspace;
     c.has_module = true;
+    free(c.prefix_layers);                     // a prefix belongs to the module it was attached for
+    c.prefix_layers = nullptr;
+    c.has_prefix = false;
+    return MRP_OK;
+}
+
+int mrp_module_set_prefix(mrp_ctx *ctx, const mrp_module_kv *layers, const int32_t *prefix_len, int32_t prefix_cap,
+                          int32_t append)
+{
+    if (!ctx) return MRP_ERR_INVALID_ARG;
+    Ctx &c = ctx->c;
+    if (!c.has_module) return MRP_ERR_UNSUPPORTED;
+    if (!layers) {
+        free(c.prefix_layers);
+        c.prefix_layers = nullptr;
+        c.has_prefix = false;
+        return MRP_OK;
+    }
+    const int D = c.module.n_layers;
+    if (!prefix_len || prefix_cap < 0 || (long long)prefix_cap + c.cfg.block_len > 0x7fffffffLL / 2) return MRP_ERR_INVALID_ARG;
+    for (int l = 0; l < D; ++l)
+        if (!layers[l].k || !layers[l].v || ((uintptr_t)layers[l].k & 15u) || ((uintptr_t)layers[l].v & 15u))
+            return MRP_ERR_INVALID_ARG;
+    if (c.cfg.d / c.module.n_attn_heads > kAttMaxDh) return MRP_ERR_UNSUPPORTED;
+    mrp_module_kv *copy = (mrp_module_kv *)malloc(sizeof(mrp_module_kv) * (size_t)(D > 0 ? D : 1));
+    if (!copy) return MRP_ERR_NOMEM;
+    if (D > 0) memcpy(copy, layers, sizeof(mrp_module_kv) * (size_t)D);
+    free(c.prefix_layers);
+    c.prefix_layers = copy;
+    c.prefix_len = prefix_len;
+    c.prefix_cap = prefix_cap;
+    c.prefix_append = append != 0;
+    c.has_prefix = true;
     return MRP_OK;
 }
 

@@ -93,6 +93,13 @@ struct Ctx {
     mrp_module_weights module;
     mrp_module_layer *module_layers;   // host copy [n_layers]
     char *module_ws;
+    // the clean prefix of the module's attention (mrp_module_set_prefix): per layer the device pointers of the
+    // key / value cache [max_seqs][prefix_cap][d] (context dtype), host copy; lengths per sequence on the device
+    bool has_prefix;
+    mrp_module_kv *prefix_layers;
+    const int32_t *prefix_len;
+    int prefix_cap;
+    bool prefix_append;
     char err[192];             // detail of the last failure ("" if none)
     bool prof_enabled;
     cudaEvent_t *prof_events;  // [kProfSlots][kProfMarks]
@@ -317,5 +324,178 @@ __device__ inline Partial merge_partial(const Partial &a, const Partial &b)
     r.sum = ea + eb;
     return r;
 }
+
+// ---- the module's attention behind a clean prefix (Fig. 1(c)) ------------------------------------------------
+// One (query position, attention head) by the four warps of a CTA (or of its epilogue warpgroup).  Keys and values:
+// the first P rows of the sequence's slab of the prefix cache (type T, written by earlier calls, read through the
+// read-only path), then the L rows of the block (fp32, possibly written earlier in this same kernel: read from L2).
+// Every warp takes each fourth group of 32 keys: a lane per key for the scores, lanes over the head's features for
+// the weighted values, with a running maximum and sum; the four partial results meet in shared memory.
+//   sh      kAttShFloats floats of shared memory;  sync(): a barrier over exactly these 128 threads
+//   out(c, value) is called once per feature c of the head
+// All pointers already point at the head's slice of their row; d is the row stride of all of them.
+constexpr int kAttMaxDh = 256;
+constexpr int kAttShFloats = kAttMaxDh + 4 * (kAttMaxDh + 2);
+
+__device__ __forceinline__ float att_f(float x) { return x; }
+__device__ __forceinline__ float att_f(__nv_bfloat16 x) { return __bfloat162float(x); }
+
+// q_s . row over dh features; vec: rows 16-byte aligned and dh % 8 == 0
+__device__ __forceinline__ float att_dot8(const float *q8, const uint4 &u, float s)
+{
+    const float4 a = *reinterpret_cast<const float4 *>(q8), b = *reinterpret_cast<const float4 *>(q8 + 4);
+    const __nv_bfloat162 *h = reinterpret_cast<const __nv_bfloat162 *>(&u);
+    const float2 f0 = __bfloat1622float2(h[0]), f1 = __bfloat1622float2(h[1]), f2 = __bfloat1622float2(h[2]), f3 = __bfloat1622float2(h[3]);
+    s = fmaf(a.x, f0.x, s); s = fmaf(a.y, f0.y, s); s = fmaf(a.z, f1.x, s); s = fmaf(a.w, f1.y, s);
+    s = fmaf(b.x, f2.x, s); s = fmaf(b.y, f2.y, s); s = fmaf(b.z, f3.x, s); s = fmaf(b.w, f3.y, s);
+    return s;
+}
+__device__ __forceinline__ float att_dot_ro(const float *q_s, const __nv_bfloat16 *row, int dh, bool vec)
+{
+    float s = 0.f;
+    if (vec && (dh & 31) == 0) {
+        // 64 bytes of the row per step, the loads of several steps in flight together
+        float s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll 4
+        for (int c = 0; c < dh; c += 32) {
+            const uint4 *r4 = reinterpret_cast<const uint4 *>(row + c);
+            const uint4 u0 = __ldg(r4), u1 = __ldg(r4 + 1), u2 = __ldg(r4 + 2), u3 = __ldg(r4 + 3);
+            s = att_dot8(q_s + c, u0, s);
+            s1 = att_dot8(q_s + c + 8, u1, s1);
+            s2 = att_dot8(q_s + c + 16, u2, s2);
+            s3 = att_dot8(q_s + c + 24, u3, s3);
+        }
+        s = (s + s1) + (s2 + s3);
+    } else if (vec) {
+        for (int c = 0; c < dh; c += 8) s = att_dot8(q_s + c, __ldg(reinterpret_cast<const uint4 *>(row + c)), s);
+    } else {
+        for (int c = 0; c < dh; ++c) s = fmaf(q_s[c], __bfloat162float(__ldg(row + c)), s);
+    }
+    return s;
+}
+__device__ __forceinline__ float att_dot_ro(const float *q_s, const float *row, int dh, bool vec)
+{
+    float s = 0.f;
+    if (vec) {
+#pragma unroll 8
+        for (int c = 0; c < dh; c += 4) {
+            const float4 u = __ldg(reinterpret_cast<const float4 *>(row + c)), a = *reinterpret_cast<const float4 *>(q_s + c);
+            s = fmaf(a.x, u.x, s); s = fmaf(a.y, u.y, s); s = fmaf(a.z, u.z, s); s = fmaf(a.w, u.w, s);
+        }
+    } else {
+        for (int c = 0; c < dh; ++c) s = fmaf(q_s[c], __ldg(row + c), s);
+    }
+    return s;
+}
+__device__ __forceinline__ float att_dot_cg(const float *q_s, const float *row, int dh, bool vec)
+{
+    float s = 0.f;
+    if (vec) {
+        for (int c = 0; c < dh; c += 4) {
+            const float4 u = __ldcg(reinterpret_cast<const float4 *>(row + c)), a = *reinterpret_cast<const float4 *>(q_s + c);
+            s = fmaf(a.x, u.x, s); s = fmaf(a.y, u.y, s); s = fmaf(a.z, u.z, s); s = fmaf(a.w, u.w, s);
+        }
+    } else {
+        for (int c = 0; c < dh; ++c) s = fmaf(q_s[c], __ldcg(row + c), s);
+    }
+    return s;
+}
+
+template <typename T, typename Sync, typename Out>
+__device__ __forceinline__ void att_prefix_item(const float *qi, const T *pk, const T *pv, int P, const float *kb,
+                                                const float *vb, int L, int d, int dh, float *sh, int warp, int lane, Sync sync,
+                                                Out out)
+{
+    float *q_s = sh, *part = sh + kAttMaxDh;              // part[w]: maximum, sum, o[dh]
+    const int t = warp * 32 + lane;
+    for (int c = t; c < dh; c += 128) q_s[c] = __ldcg(qi + c);
+    sync();
+    const float scale = rsqrtf((float)dh);
+    const bool vec = (dh % 8) == 0 && (d % 8) == 0;
+    float mx = -INFINITY, sum = 0.f, oacc[kAttMaxDh / 32];
+#pragma unroll
+    for (int u = 0; u < kAttMaxDh / 32; ++u) oacc[u] = 0.f;
+    const int gp = (P + 31) / 32, gb = (L + 31) / 32;
+    for (int g = warp; g < gp + gb; g += 4) {
+        const bool pre = g < gp;
+        const int j0 = pre ? g * 32 : (g - gp) * 32;
+        const int left = (pre ? P : L) - j0, cnt = left < 32 ? left : 32;
+        float s = -INFINITY;
+        if (lane < cnt)
+            s = (pre ? att_dot_ro(q_s, pk + (size_t)(j0 + lane) * d, dh, vec) : att_dot_cg(q_s, kb + (size_t)(j0 + lane) * d, dh, vec)) *
+                scale;
+        float gm = s;
+#pragma unroll
+        for (int w = 16; w > 0; w >>= 1) gm = fmaxf(gm, __shfl_xor_sync(0xffffffffu, gm, w));
+        const float nm = fmaxf(mx, gm), corr = expf(mx - nm);            // (mx = -inf at first: corr = 0)
+        const float pj = lane < cnt ? expf(s - nm) : 0.f;
+        sum = sum * corr + pj;                                           // per-lane share; corr is the same in every lane
+#pragma unroll
+        for (int u = 0; u < kAttMaxDh / 32; ++u) oacc[u] *= corr;
+        if (pre && cnt == 32) {
+            // a full group of prefix rows: the value loads of eight keys in flight together
+#pragma unroll 8
+            for (int jj = 0; jj < 32; ++jj) {
+                const float w = __shfl_sync(0xffffffffu, pj, jj);
+                const T *vr = pv + (size_t)(j0 + jj) * d;
+#pragma unroll
+                for (int u = 0; u < kAttMaxDh / 32; ++u) {
+                    const int c = lane + 32 * u;
+                    if (c < dh) oacc[u] = fmaf(w, att_f(__ldg(vr + c)), oacc[u]);
+                }
+            }
+        } else {
+            for (int jj = 0; jj < cnt; ++jj) {
+                const float w = __shfl_sync(0xffffffffu, pj, jj);
+                if (pre) {
+                    const T *vr = pv + (size_t)(j0 + jj) * d;
+#pragma unroll
+                    for (int u = 0; u < kAttMaxDh / 32; ++u) {
+                        const int c = lane + 32 * u;
+                        if (c < dh) oacc[u] = fmaf(w, att_f(__ldg(vr + c)), oacc[u]);
+                    }
+                } else {
+                    const float *vr = vb + (size_t)(j0 + jj) * d;
+#pragma unroll
+                    for (int u = 0; u < kAttMaxDh / 32; ++u) {
+                        const int c = lane + 32 * u;
+                        if (c < dh) oacc[u] = fmaf(w, __ldcg(vr + c), oacc[u]);
+                    }
+                }
+            }
+        }
+        mx = nm;
+    }
+#pragma unroll
+    for (int w = 16; w > 0; w >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, w);
+    float *mine = part + warp * (kAttMaxDh + 2);
+    if (lane == 0) {
+        mine[0] = mx;
+        mine[1] = sum;
+    }
+#pragma unroll
+    for (int u = 0; u < kAttMaxDh / 32; ++u) {
+        const int c = lane + 32 * u;
+        if (c < dh) mine[2 + c] = oacc[u];
+    }
+    sync();
+    // the block has at least one key, so the overall maximum is finite; a warp that had no keys weighs 0
+    float top = -INFINITY, e[4], tot = 0.f;
+#pragma unroll
+    for (int w = 0; w < 4; ++w) top = fmaxf(top, part[w * (kAttMaxDh + 2)]);
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+        e[w] = expf(part[w * (kAttMaxDh + 2)] - top);
+        tot = fmaf(part[w * (kAttMaxDh + 2) + 1], e[w], tot);
+    }
+    for (int c = t; c < dh; c += 128) {
+        float o = 0.f;
+#pragma unroll
+        for (int w = 0; w < 4; ++w) o = fmaf(part[w * (kAttMaxDh + 2) + 2 + c], e[w], o);
+        out(c, o / tot);
+    }
+    sync();                                                              // sh is free again
+}
+
 
 }  // namespace mrp

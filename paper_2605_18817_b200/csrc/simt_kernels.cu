@@ -1238,6 +1238,51 @@ __global__ void mod_attention_kernel(const float *__restrict__ q, const float *_
     }
 }
 
+// The same behind a clean prefix (Fig. 1(c)): CTA = (query position, attention head); keys and values are the first
+// prefix_len[b] rows of sequence b's slab of the cache [*, cap, d], then the block's own rows.  With `append` the
+// block's keys and values are also stored behind the prefix rows (rows the call itself never reads).
+template <typename T>
+__global__ void __launch_bounds__(128) mod_attention_prefix_kernel(const float *__restrict__ q, const float *k, const float *v, int L,
+                                                                   int d, int dh, int H, float *__restrict__ o,
+                                                                   __nv_bfloat16 *__restrict__ o16, int n_rows, T *pk, T *pv,
+                                                                   const int32_t *__restrict__ plen, int cap, int append,
+                                                                   int32_t *__restrict__ status, int32_t *__restrict__ user_status)
+{
+    pdl_trigger();
+    pdl_wait();
+    __shared__ __align__(16) float sh[kAttShFloats];
+    const int item = blockIdx.x, pos = item / H, hd = item - pos * H, b = pos / L, i = pos - b * L;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    int P = plen[b];
+    bool bad = P < 0 || P > cap;
+    P = P < 0 ? 0 : (P > cap ? cap : P);
+    const bool store = append && !bad && P + L <= cap;
+    bad = bad || (append && !store);
+    if (bad && threadIdx.x == 0 && hd == 0 && i == 0) {
+        atomicOr(status, MRP_DEV_BAD_INDEX);
+        if (user_status) atomicOr(user_status, MRP_DEV_BAD_INDEX);
+    }
+    const size_t head = (size_t)hd * dh, slab = (size_t)b * cap * d + head, own = (size_t)pos * d + head;
+    if (store) {
+        T *dk = pk + slab + (size_t)(P + i) * d, *dv = pv + slab + (size_t)(P + i) * d;
+        for (int c = threadIdx.x; c < dh; c += 128) {
+            dk[c] = (T)k[own + c];
+            dv[c] = (T)v[own + c];
+        }
+    }
+    att_prefix_item<T>(q + own, pk + slab, pv + slab, P, k + (size_t)b * L * d + head, v + (size_t)b * L * d + head, L, d, dh, sh,
+                       warp, lane, [] { __syncthreads(); }, [&](int c, float val) {
+                           const size_t at = own + c;
+                           if (o16) {
+                               const __nv_bfloat16 hh = __float2bfloat16_rn(val);
+                               o16[at] = hh;
+                               o16[(size_t)n_rows * d + at] = __float2bfloat16_rn(val - __bfloat162float(hh));
+                           } else {
+                               o[at] = val;
+                           }
+                       });
+}
+
 // h <- h + Delta for every dense position.
 __global__ void mod_add_kernel(float *__restrict__ h_state, const float *__restrict__ z, size_t n)
 {
@@ -1677,7 +1722,8 @@ static cudaError_t module_fused_t(Ctx *c, const int32_t *tokens, const void *hid
     *launched = false;
     const mrp_module_weights &w = c->module;
     const int d = c->cfg.d, F = c->cfg.d_ff, n = B * L;
-    if (n > kModRows || L > kModRows || w.n_layers > kModMaxLayers || (c->cfg.flags & MRP_FLAG_NO_CHAIN) || (d & 3) || (F & 3) || F < d ||
+    // (with a clean prefix attached the attention runs in the per-product form or in the tensor-core step)
+    if (c->has_prefix || n > kModRows || L > kModRows || w.n_layers > kModMaxLayers || (c->cfg.flags & MRP_FLAG_NO_CHAIN) || (d & 3) || (F & 3) || F < d ||
         module_fused_smem(n, d, F) > kModMaxSmem)
         return cudaSuccess;
     auto kern = module_fused_kernel<T>;
@@ -1805,6 +1851,23 @@ static bool module_chain_ok(Ctx *c, int n, int L, cudaStream_t st)
                           nullptr, nullptr, nullptr, 0, 0, false, nullptr, nullptr, st, true) == cudaSuccess;
 }
 
+// The attention of layer l over B blocks of L positions: block-local, or behind the context's clean prefix.
+template <typename T>
+static cudaError_t module_attention(Ctx *c, int layer, int B, int L, const float *q, const float *k, const float *v, float *o,
+                                    __nv_bfloat16 *o16, int n_rows, const mrp_draft_out &out, cudaStream_t st)
+{
+    const mrp_module_weights &w = c->module;
+    const int d = c->cfg.d, dh = d / w.n_attn_heads;
+    const bool pdl = !(c->cfg.flags & MRP_FLAG_NO_PDL);
+    c->launches++;
+    if (!c->has_prefix)
+        return launch_k(mod_attention_kernel, dim3(B, w.n_attn_heads), dim3(128), (size_t)4 * L * 4, st, pdl, q, k, v, L, d, dh, o, o16,
+                        n_rows);
+    return launch_k(mod_attention_prefix_kernel<T>, dim3((unsigned)(B * L * w.n_attn_heads)), dim3(128), 0, st, pdl, q, k, v, L, d, dh,
+                    w.n_attn_heads, o, o16, n_rows, (T *)c->prefix_layers[layer].k, (T *)c->prefix_layers[layer].v, c->prefix_len,
+                    c->prefix_cap, c->prefix_append ? 1 : 0, (int32_t *)(c->ws + c->lay.status), out.status);
+}
+
 // The module itself (everything in front of `h <- h + Delta`) with its products on the tensor cores.
 static cudaError_t module_body_tc(Ctx *c, const int32_t *tokens, const void *hidden0, float *h_state, int B, int L,
                                   bool first_step, const mrp_draft_out &out, cudaStream_t st, float *z)
@@ -1848,11 +1911,7 @@ static cudaError_t module_body_tc(Ctx *c, const int32_t *tokens, const void *hid
         for (int l = 0; l < w.n_layers && e == cudaSuccess; ++l) {
             const mrp_module_layer &y = w.layers[l];
             e = sk_linear3(c, xa, n, d, y.w_q, y.w_k, y.w_v, d, sumsq, n_ss, q, k, v, out.status, st);
-            if (e == cudaSuccess) {
-                e = launch_k(mod_attention_kernel, dim3(B, w.n_attn_heads), dim3(128), (size_t)4 * L * 4, st, pdl, (const float *)q,
-                             (const float *)k, (const float *)v, L, d, dh, (float *)nullptr, xb, lo_rows);
-                c->launches++;
-            }
+            if (e == cudaSuccess) e = module_attention<__nv_bfloat16>(c, l, B, L, q, k, v, nullptr, xb, lo_rows, out, st);
             if (e == cudaSuccess)
                 e = sk_linear(c, xb, n, d, y.w_o, d, nullptr, 1, z, true, y.g_mlp, xa, sumsq, &n_ss, out.status, st);
             if (e == cudaSuccess) e = sk_gate_up(c, xa, n, d, y.w_gate, y.w_up, F, sumsq, n_ss, act16, out.status, st);
@@ -1869,11 +1928,7 @@ static cudaError_t module_body_tc(Ctx *c, const int32_t *tokens, const void *hid
     for (int l = 0; l < w.n_layers && e == cudaSuccess; ++l) {
         const mrp_module_layer &y = w.layers[l];
         e = tc_linear3(c, xa, n, d, y.w_q, y.w_k, y.w_v, d, sumsq, n_ss, q, k, v, out.status, st);
-        if (e == cudaSuccess) {
-            e = launch_k(mod_attention_kernel, dim3(B, w.n_attn_heads), dim3(128), (size_t)4 * L * 4, st, pdl, (const float *)q,
-                         (const float *)k, (const float *)v, L, d, dh, (float *)nullptr, xb, n);
-            c->launches++;
-        }
+        if (e == cudaSuccess) e = module_attention<__nv_bfloat16>(c, l, B, L, q, k, v, nullptr, xb, n, out, st);
         if (e == cudaSuccess)
             e = tc_linear(c, xb, n, d, y.w_o, d, nullptr, 1, z, true, out.status, st, y.g_mlp, xa, sumsq, &n_ss);
         if (e == cudaSuccess) e = tc_gate_up(c, xa, n, d, y.w_gate, y.w_up, F, sumsq, n_ss, act16, out.status, st);
@@ -1967,11 +2022,7 @@ static cudaError_t module_step_t(Ctx *c, const int32_t *tokens, const void *hidd
         if (e == cudaSuccess) e = lin(y.w_q, nn, d, d, q, 0);
         if (e == cudaSuccess) e = lin(y.w_k, nn, d, d, k, 0);
         if (e == cudaSuccess) e = lin(y.w_v, nn, d, d, v, 0);
-        if (e == cudaSuccess) {
-            e = launch_k(mod_attention_kernel, dim3(B, w.n_attn_heads), dim3(128), (size_t)4 * L * 4, st, pdl, (const float *)q,
-                         (const float *)k, (const float *)v, L, d, dh, o, (__nv_bfloat16 *)nullptr, n);
-            c->launches++;
-        }
+        if (e == cudaSuccess) e = module_attention<T>(c, l, B, L, q, k, v, o, nullptr, n, out, st);
         if (e == cudaSuccess) e = lin(y.w_o, o, d, d, z, 1);
         if (e == cudaSuccess) {
             e = launch_k(rmsnorm_kernel<T>, dim3(n), dim3(256), 0, st, pdl, (const float *)z, (const T *)y.g_mlp, d, c->cfg.rms_eps, nn);

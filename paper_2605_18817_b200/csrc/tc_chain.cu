@@ -77,6 +77,7 @@ struct ChainPhase {
     const float *att_q, *att_k, *att_v;
     __nv_bfloat16 *att_out;
     int att_L, att_H;
+    __nv_bfloat16 *att_pk, *att_pv;  // the layer's clean-prefix cache [*, pcap, d] (nullptr: block-local attention)
     int zero_slot0, zero_slot1;      // ssq_fix slots this phase clears for later phases of the launch (< 0: none)
 };
 
@@ -93,6 +94,8 @@ struct ModEnds {
     __nv_bfloat16 *xt;       // LM-head operand rows (step 0 zero rows, then h - h_0), lo rows lo_xt rows further on
     __half *xt16;
     float *hidden_out;
+    const int32_t *plen;     // clean prefix: rows in use per sequence, rows per slab, whether the block's own keys and
+    int pcap, append;        // values are stored behind them
 };
 
 template <int NP>
@@ -730,7 +733,36 @@ sk_chain_kernel(const __grid_constant__ typename ChainTypes<MOD>::Maps maps,
                             for (int j = cta * 128 + t; j < p.d; j += G * 128) put(m, j, 0.f, 0.f);
                     }
                 }
-                if (ph.kind == CH_ATT) {
+                if (ph.kind == CH_ATT && ph.att_pk) {
+                    // attention behind a clean prefix: the four warps on one (position, attention head) at a time
+                    const ModEnds &e = p.mod;
+                    const int L = ph.att_L, H = ph.att_H, dh = p.d / H;
+                    for (int item = cta; item < p.M * H; item += G) {
+                        const int pos = item / H, hd = item - pos * H, b = pos / L, i2 = pos - b * L;
+                        int P = e.plen[b];
+                        bool bad = P < 0 || P > e.pcap;
+                        P = P < 0 ? 0 : (P > e.pcap ? e.pcap : P);
+                        const bool store = e.append && !bad && P + L <= e.pcap;
+                        bad = bad || (e.append && !store);
+                        if (bad && t == 0 && hd == 0 && i2 == 0) {
+                            atomicOr(p.status, MRP_DEV_BAD_INDEX);
+                            if (p.user_status) atomicOr(p.user_status, MRP_DEV_BAD_INDEX);
+                        }
+                        const size_t head = (size_t)hd * dh, slab = (size_t)b * e.pcap * p.d + head, own = (size_t)pos * p.d + head;
+                        if (store) {                  // rows this call never reads
+                            __nv_bfloat16 *dk = ph.att_pk + slab + (size_t)(P + i2) * p.d, *dv = ph.att_pv + slab + (size_t)(P + i2) * p.d;
+                            for (int cidx = t; cidx < dh; cidx += 128) {
+                                dk[cidx] = __float2bfloat16_rn(__ldcg(ph.att_k + own + cidx));
+                                dv[cidx] = __float2bfloat16_rn(__ldcg(ph.att_v + own + cidx));
+                            }
+                        }
+                        att_prefix_item<__nv_bfloat16>(ph.att_q + own, ph.att_pk + slab, ph.att_pv + slab, P,
+                                                       ph.att_k + (size_t)b * L * p.d + head, ph.att_v + (size_t)b * L * p.d + head, L, p.d,
+                                                       dh, sq_s, q, lane, [&] { ch_epi_sync(); }, [&](int cidx, float val) {
+                                                           ch_store_hi_lo(ph.att_out + own + cidx, (size_t)p.lo_x * p.d, val);
+                                                       });
+                    }
+                } else if (ph.kind == CH_ATT) {
                     // block-local bidirectional attention, a warp per (position, attention head) over the whole grid;
                     // lanes over the head's features, one warp sum per key; output in operand form (hi + lo)
                     const int L = ph.att_L, H = ph.att_H, dh = p.d / H;
@@ -1029,6 +1061,7 @@ cudaError_t sk_module_step(Ctx *c, int n, int L, const int32_t *tokens, const vo
     p.mod.mask_token = w.mask_token; p.mod.emb_rows = w.emb_rows; p.mod.row_index = row_index; p.mod.n_masked = n_masked;
     p.mod.xt = (__nv_bfloat16 *)(c->ws + c->lay.xt); p.mod.xt16 = f16_lm ? (__half *)(c->ws + c->lay.xt16) : nullptr;
     p.mod.hidden_out = hidden_out;
+    if (c->has_prefix) { p.mod.plen = c->prefix_len; p.mod.pcap = c->prefix_cap; p.mod.append = c->prefix_append ? 1 : 0; }
     bool ok = make_map(s, &maps.m[0], xa, d, 2 * (uint64_t)r_pad, 2 * r_pad) && make_map(s, &maps.m[1], act16, F, 2 * (uint64_t)r_pad, 2 * r_pad) &&
               make_map(s, &maps.m[2], xb, d, 2 * (uint64_t)r_pad, 2 * r_pad) &&
               make_map(s, &maps.m[3], cat16, 2 * d, 2 * (uint64_t)r_pad, 2 * r_pad) && make_map(s, &maps.m[4], w.w_proj, 2 * d, d, 128);
@@ -1075,6 +1108,10 @@ cudaError_t sk_module_step(Ctx *c, int n, int L, const int32_t *tokens, const vo
         {
             ChainPhase &ph = plain(CH_ATT);
             ph.att_q = q; ph.att_k = k; ph.att_v = v; ph.att_out = xb; ph.att_L = L; ph.att_H = H;
+            if (c->has_prefix) {
+                ph.att_pk = (__nv_bfloat16 *)c->prefix_layers[l].k;
+                ph.att_pv = (__nv_bfloat16 *)c->prefix_layers[l].v;
+            }
         }
         {
             ChainPhase &ph = lin(d / kBK, d_tiles, sp_o, 2, b + 3);
