@@ -266,7 +266,8 @@ constexpr int kModChainBarInts = 23 * 448 + 1;
 cudaError_t sk_module_step(Ctx *c, int n, int L, const int32_t *tokens, const void *hidden0, float *h_state, bool first_step,
                            __nv_bfloat16 *cat16, __nv_bfloat16 *xa, __nv_bfloat16 *xb, __nv_bfloat16 *act16, float *q, float *k,
                            float *v, float *z, int32_t *bar_mem, const int32_t *row_index, int n_masked, int lo_xt, bool f16_lm,
-                           float *hidden_out, int32_t *user_status, cudaStream_t st, bool check_only);
+                           float *hidden_out, int32_t *user_status, cudaStream_t st, bool check_only, float *att_part = nullptr,
+                           int *att_counters = nullptr);
 // The same for the CUDA-core family (operand rows: fp32 xt).
 cudaError_t simt_lm_tail(Ctx *c, const float *logits0, const int32_t *row_index, int M, int K,
                          const mrp_draft_out &out, cudaStream_t st);
@@ -277,6 +278,7 @@ cudaError_t module_step(Ctx *c, const int32_t *tokens, const void *hidden0, floa
                         const int32_t *row_index, int M, int B, int L, bool first_step, const mrp_draft_out &out,
                         cudaStream_t st);
 size_t module_workspace_bytes(const mrp_config &cfg, int n_layers);
+size_t module_att_offset(const mrp_config &cfg);   // the clean-prefix attention's area of the module workspace
 
 // Few-row variants (tc_skinny.cu): weight rows on the MMA M axis; rows <= 32.
 bool sk_rows_ok(int rows);          // LM head: row-steps incl. step 0
@@ -326,176 +328,343 @@ __device__ inline Partial merge_partial(const Partial &a, const Partial &b)
 }
 
 // ---- the module's attention behind a clean prefix (Fig. 1(c)) ------------------------------------------------
-// One (query position, attention head) by the four warps of a CTA (or of its epilogue warpgroup).  Keys and values:
-// the first P rows of the sequence's slab of the prefix cache (type T, written by earlier calls, read through the
-// read-only path), then the L rows of the block (fp32, possibly written earlier in this same kernel: read from L2).
-// Every warp takes each fourth group of 32 keys: a lane per key for the scores, lanes over the head's features for
-// the weighted values, with a running maximum and sum; the four partial results meet in shared memory.
-//   sh      kAttShFloats floats of shared memory;  sync(): a barrier over exactly these 128 threads
-//   out(c, value) is called once per feature c of the head
-// All pointers already point at the head's slice of their row; d is the row stride of all of them.
+// Work unit = (block b, attention head, chunk of the key range), run by the four warps of a CTA (or of its epilogue
+// warpgroup).  Keys and values: the first P rows of the sequence's slab of the prefix cache (type T, written by
+// earlier calls, read through the read-only path), then the L rows of the block (fp32, possibly written earlier in
+// this same kernel: read from L2).  The keys go in groups of 32 (prefix groups, then block groups); chunk ch covers
+// groups [ch * gpc, (ch + 1) * gpc) and its warps take them round-robin: a lane per key for the scores of kAttQT
+// queries at a time (a key row is loaded once for all of them), then lanes over the head's features for the weighted
+// values, with a running maximum and sum per query.  The four warps' partial results meet in shared memory; with
+// more than one chunk the chunk's partial results go to `part` and the CTA that arrives last at the (block, head)
+// counter merges them -- no CTA waits for another.
+//   q, kb, vb   the block's first row of q / k / v at the head's columns; pk, pv the slab's first row there;
+//               d = row stride of all of them
+//   part        [n_ch][L][dh + 2] floats of this (block, head); counter: its arrival counter, zero before and after
+//   sh          att_sh_floats(dh) floats of shared memory, 16-byte aligned;  sync(): a barrier over exactly these
+//               128 threads;  out(i, c, value) is called once per query i of the block and feature c of the head
 constexpr int kAttMaxDh = 256;
-constexpr int kAttShFloats = kAttMaxDh + 4 * (kAttMaxDh + 2);
+constexpr int kAttQT = 4;
+constexpr int kAttMaxChunks = 16;
+constexpr int kAttCounters = 4096;                    // (block, head) pairs that can split their keys over CTAs
+constexpr size_t kAttPartFloats = (size_t)1 << 20;    // partial results of split units
+__host__ __device__ constexpr int att_sh_floats(int dh) { return kAttQT * dh + 4 * kAttQT * (dh + 2); }
+
+// How a call splits the keys: groups per chunk and chunks, for sequences of up to `cap` prefix rows and blocks of L,
+// aiming at `target` units in all.
+struct AttSplit { int gpc, n_ch; };
+inline AttSplit att_split(int cap, int L, int BH, int dh, int target)
+{
+    const int groups = (cap + 31) / 32 + (L + 31) / 32;
+    int want = BH > 0 ? target / BH : 1;
+    if (want > kAttMaxChunks) want = kAttMaxChunks;
+    if (want > groups) want = groups;
+    const size_t per_chunk = (size_t)BH * L * (dh + 2);
+    if (BH > kAttCounters || per_chunk > kAttPartFloats) want = 1;
+    else if ((size_t)want * per_chunk > kAttPartFloats) want = (int)(kAttPartFloats / per_chunk);
+    if (want < 1) want = 1;
+    AttSplit sp;
+    sp.gpc = (groups + want - 1) / want;
+    sp.n_ch = (groups + sp.gpc - 1) / sp.gpc;
+    return sp;
+}
 
 __device__ __forceinline__ float att_f(float x) { return x; }
 __device__ __forceinline__ float att_f(__nv_bfloat16 x) { return __bfloat162float(x); }
 
-// q_s . row over dh features; vec: rows 16-byte aligned and dh % 8 == 0
-__device__ __forceinline__ float att_dot8(const float *q8, const uint4 &u, float s)
+// eight consecutive elements of a row as floats (16-byte aligned); CG: through L2 (data written in this kernel)
+template <bool CG>
+__device__ __forceinline__ void att_ld8(const __nv_bfloat16 *p, float f[8])
 {
-    const float4 a = *reinterpret_cast<const float4 *>(q8), b = *reinterpret_cast<const float4 *>(q8 + 4);
+    const uint4 u = __ldg(reinterpret_cast<const uint4 *>(p));
     const __nv_bfloat162 *h = reinterpret_cast<const __nv_bfloat162 *>(&u);
-    const float2 f0 = __bfloat1622float2(h[0]), f1 = __bfloat1622float2(h[1]), f2 = __bfloat1622float2(h[2]), f3 = __bfloat1622float2(h[3]);
-    s = fmaf(a.x, f0.x, s); s = fmaf(a.y, f0.y, s); s = fmaf(a.z, f1.x, s); s = fmaf(a.w, f1.y, s);
-    s = fmaf(b.x, f2.x, s); s = fmaf(b.y, f2.y, s); s = fmaf(b.z, f3.x, s); s = fmaf(b.w, f3.y, s);
-    return s;
+#pragma unroll
+    for (int x = 0; x < 4; ++x) {
+        const float2 t = __bfloat1622float2(h[x]);
+        f[2 * x] = t.x;
+        f[2 * x + 1] = t.y;
+    }
 }
-__device__ __forceinline__ float att_dot_ro(const float *q_s, const __nv_bfloat16 *row, int dh, bool vec)
+template <bool CG>
+__device__ __forceinline__ void att_ld8(const float *p, float f[8])
 {
-    float s = 0.f;
+    const float4 *p4 = reinterpret_cast<const float4 *>(p);
+    const float4 a = CG ? __ldcg(p4) : __ldg(p4), b = CG ? __ldcg(p4 + 1) : __ldg(p4 + 1);
+    f[0] = a.x; f[1] = a.y; f[2] = a.z; f[3] = a.w; f[4] = b.x; f[5] = b.y; f[6] = b.z; f[7] = b.w;
+}
+template <bool CG, typename T>
+__device__ __forceinline__ float att_ld1(const T *p)
+{
+    if (CG) return att_f(__ldcg(p));
+    return att_f(__ldg(p));
+}
+
+// scores of one key row against the kAttQT staged queries (q_s: [kAttQT][dh])
+template <bool CG, typename T>
+__device__ __forceinline__ void att_scores(const float *q_s, const T *row, int dh, bool vec, float s[kAttQT])
+{
+#pragma unroll
+    for (int qi = 0; qi < kAttQT; ++qi) s[qi] = 0.f;
     if (vec && (dh & 31) == 0) {
-        // 64 bytes of the row per step, the loads of several steps in flight together
-        float s1 = 0.f, s2 = 0.f, s3 = 0.f;
+        // 32 elements of the row per step: four loads in flight together, several steps overlapping
 #pragma unroll 4
         for (int c = 0; c < dh; c += 32) {
-            const uint4 *r4 = reinterpret_cast<const uint4 *>(row + c);
-            const uint4 u0 = __ldg(r4), u1 = __ldg(r4 + 1), u2 = __ldg(r4 + 2), u3 = __ldg(r4 + 3);
-            s = att_dot8(q_s + c, u0, s);
-            s1 = att_dot8(q_s + c + 8, u1, s1);
-            s2 = att_dot8(q_s + c + 16, u2, s2);
-            s3 = att_dot8(q_s + c + 24, u3, s3);
+            float f[4][8];
+#pragma unroll
+            for (int x = 0; x < 4; ++x) att_ld8<CG>(row + c + 8 * x, f[x]);
+#pragma unroll
+            for (int qi = 0; qi < kAttQT; ++qi) {
+                const float *qq = q_s + qi * dh + c;
+#pragma unroll
+                for (int x = 0; x < 4; ++x) {
+                    const float4 a = *reinterpret_cast<const float4 *>(qq + 8 * x), b = *reinterpret_cast<const float4 *>(qq + 8 * x + 4);
+                    s[qi] = fmaf(a.x, f[x][0], s[qi]); s[qi] = fmaf(a.y, f[x][1], s[qi]);
+                    s[qi] = fmaf(a.z, f[x][2], s[qi]); s[qi] = fmaf(a.w, f[x][3], s[qi]);
+                    s[qi] = fmaf(b.x, f[x][4], s[qi]); s[qi] = fmaf(b.y, f[x][5], s[qi]);
+                    s[qi] = fmaf(b.z, f[x][6], s[qi]); s[qi] = fmaf(b.w, f[x][7], s[qi]);
+                }
+            }
         }
-        s = (s + s1) + (s2 + s3);
     } else if (vec) {
-        for (int c = 0; c < dh; c += 8) s = att_dot8(q_s + c, __ldg(reinterpret_cast<const uint4 *>(row + c)), s);
-    } else {
-        for (int c = 0; c < dh; ++c) s = fmaf(q_s[c], __bfloat162float(__ldg(row + c)), s);
-    }
-    return s;
-}
-__device__ __forceinline__ float att_dot_ro(const float *q_s, const float *row, int dh, bool vec)
-{
-    float s = 0.f;
-    if (vec) {
-#pragma unroll 8
-        for (int c = 0; c < dh; c += 4) {
-            const float4 u = __ldg(reinterpret_cast<const float4 *>(row + c)), a = *reinterpret_cast<const float4 *>(q_s + c);
-            s = fmaf(a.x, u.x, s); s = fmaf(a.y, u.y, s); s = fmaf(a.z, u.z, s); s = fmaf(a.w, u.w, s);
+        for (int c = 0; c < dh; c += 8) {
+            float f[8];
+            att_ld8<CG>(row + c, f);
+#pragma unroll
+            for (int qi = 0; qi < kAttQT; ++qi)
+#pragma unroll
+                for (int x = 0; x < 8; ++x) s[qi] = fmaf(q_s[qi * dh + c + x], f[x], s[qi]);
         }
     } else {
-        for (int c = 0; c < dh; ++c) s = fmaf(q_s[c], __ldg(row + c), s);
-    }
-    return s;
-}
-__device__ __forceinline__ float att_dot_cg(const float *q_s, const float *row, int dh, bool vec)
-{
-    float s = 0.f;
-    if (vec) {
-        for (int c = 0; c < dh; c += 4) {
-            const float4 u = __ldcg(reinterpret_cast<const float4 *>(row + c)), a = *reinterpret_cast<const float4 *>(q_s + c);
-            s = fmaf(a.x, u.x, s); s = fmaf(a.y, u.y, s); s = fmaf(a.z, u.z, s); s = fmaf(a.w, u.w, s);
+        for (int c = 0; c < dh; ++c) {
+            const float f = att_ld1<CG>(row + c);
+#pragma unroll
+            for (int qi = 0; qi < kAttQT; ++qi) s[qi] = fmaf(q_s[qi * dh + c], f, s[qi]);
         }
-    } else {
-        for (int c = 0; c < dh; ++c) s = fmaf(q_s[c], __ldcg(row + c), s);
     }
-    return s;
+}
+
+// the lane's features of a value row: PER consecutive ones from lane * PER (PER > 0), or lane + 32 u, u < 8 (PER == 0)
+template <int PER, bool CG, typename T>
+__device__ __forceinline__ void att_ldv(const T *row, int lane, int dh, float v[8])
+{
+    if (PER == 8) {
+        att_ld8<CG>(row + lane * 8, v);
+    } else if (PER == 4 && sizeof(T) == 2) {
+        const uint2 u = __ldg(reinterpret_cast<const uint2 *>(row + lane * 4));
+        const __nv_bfloat162 *h = reinterpret_cast<const __nv_bfloat162 *>(&u);
+        const float2 a = __bfloat1622float2(h[0]), b = __bfloat1622float2(h[1]);
+        v[0] = a.x; v[1] = a.y; v[2] = b.x; v[3] = b.y;
+    } else if (PER == 4) {
+        const float4 *p4 = reinterpret_cast<const float4 *>(row + lane * 4);
+        const float4 a = CG ? __ldcg(p4) : __ldg(p4);
+        v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
+    } else if (PER > 0) {
+#pragma unroll
+        for (int u = 0; u < PER; ++u) v[u] = att_ld1<CG>(row + lane * PER + u);
+    } else {
+#pragma unroll
+        for (int u = 0; u < 8; ++u) v[u] = lane + 32 * u < dh ? att_ld1<CG>(row + lane + 32 * u) : 0.f;
+    }
+}
+
+// one group of up to 32 keys (rows krow0 + j * d, vrow0 + j * d, j < cnt) folded into the warp's running state
+template <int PER, bool CG, typename T>
+__device__ __forceinline__ void att_group(const float *q_s, const T *krow0, const T *vrow0, int cnt, int d, int dh, bool vec, float scale,
+                                          int lane, float mx[kAttQT], float sum[kAttQT], float (&oacc)[kAttQT][8])
+{
+    constexpr int NU = PER > 0 ? PER : 8;
+    float s[kAttQT], pj[kAttQT];
+    if (lane < cnt) {
+        att_scores<CG>(q_s, krow0 + (size_t)lane * d, dh, vec, s);
+    } else {
+#pragma unroll
+        for (int qi = 0; qi < kAttQT; ++qi) s[qi] = -INFINITY;
+    }
+#pragma unroll
+    for (int qi = 0; qi < kAttQT; ++qi) {
+        s[qi] *= scale;
+        float gm = s[qi];
+#pragma unroll
+        for (int w = 16; w > 0; w >>= 1) gm = fmaxf(gm, __shfl_xor_sync(0xffffffffu, gm, w));
+        const float nm = fmaxf(mx[qi], gm), corr = expf(mx[qi] - nm);       // (first group: mx = -inf, corr = 0)
+        pj[qi] = lane < cnt ? expf(s[qi] - nm) : 0.f;
+        sum[qi] = sum[qi] * corr + pj[qi];                                   // per-lane share; corr is the same in every lane
+#pragma unroll
+        for (int u = 0; u < NU; ++u) oacc[qi][u] *= corr;
+        mx[qi] = nm;
+    }
+    // weighted values: eight or sixteen keys' rows in flight together; a key index beyond the group reads the group's last row
+    // with weight 0 (the lanes beyond cnt hold pj = 0)
+    constexpr int VB = NU <= 4 ? 16 : 8;
+    for (int j0 = 0; j0 < cnt; j0 += VB) {
+        float v[VB][8];
+#pragma unroll
+        for (int x = 0; x < VB; ++x) {
+            const int j = j0 + x < cnt ? j0 + x : cnt - 1;
+            att_ldv<PER, CG>(vrow0 + (size_t)j * d, lane, dh, v[x]);
+        }
+#pragma unroll
+        for (int x = 0; x < VB; ++x)
+#pragma unroll
+            for (int qi = 0; qi < kAttQT; ++qi) {
+                const float w = __shfl_sync(0xffffffffu, pj[qi], (j0 + x) & 31);
+#pragma unroll
+                for (int u = 0; u < NU; ++u) oacc[qi][u] = fmaf(w, v[x][u], oacc[qi][u]);
+            }
+    }
+}
+
+template <int PER, typename T, typename Sync, typename Out>
+__device__ __forceinline__ void att_unit_per(const float *q, const T *pk, const T *pv, int P, const float *kb, const float *vb, int L,
+                                             int d, int dh, int ch, int n_ch, int gpc, float *part, int *counter, float *sh, int warp,
+                                             int lane, Sync sync, Out out)
+{
+    constexpr int NU = PER > 0 ? PER : 8;
+    float *q_s = sh, *part_s = sh + kAttQT * dh;              // part_s[w][qi]: maximum, sum, o[dh]
+    const int t = warp * 32 + lane, stride = dh + 2;
+    const float scale = rsqrtf((float)dh);
+    const bool vec = (dh % 8) == 0 && (d % 8) == 0;
+    const int gp = (P + 31) / 32, gb = (L + 31) / 32;
+    const int g_end = (ch + 1) * gpc < gp + gb ? (ch + 1) * gpc : gp + gb;
+    auto feat = [&](int u) { return PER > 0 ? lane * PER + u : lane + 32 * u; };
+    // The prefix rows this warp will read, asked into L2 up front: each lane reads whole rows of its own in the score
+    // loops, a handful of loads at a time, and would otherwise pay the DRAM latency once per handful.
+    for (int g = ch * gpc + warp; g < g_end && g < gp; g += 4) {
+        const int j = g * 32 + lane;
+        if (j < P) {
+            const char *rk = reinterpret_cast<const char *>(pk + (size_t)j * d), *rv = reinterpret_cast<const char *>(pv + (size_t)j * d);
+            for (int off = 0; off < dh * (int)sizeof(T); off += 128) {
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(rk + off));
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(rv + off));
+            }
+        }
+    }
+    for (int q0 = 0; q0 < L; q0 += kAttQT) {
+        // the tile's queries (zero rows beyond the block)
+        for (int x = t; x < kAttQT * dh; x += 128) {
+            const int qi = x / dh, c = x - qi * dh;
+            q_s[x] = q0 + qi < L ? __ldcg(q + (size_t)(q0 + qi) * d + c) : 0.f;
+        }
+        sync();
+        float mx[kAttQT], sum[kAttQT], oacc[kAttQT][8];
+#pragma unroll
+        for (int qi = 0; qi < kAttQT; ++qi) {
+            mx[qi] = -INFINITY;
+            sum[qi] = 0.f;
+#pragma unroll
+            for (int u = 0; u < 8; ++u) oacc[qi][u] = 0.f;
+        }
+        for (int g = ch * gpc + warp; g < g_end; g += 4) {
+            if (g < gp) {
+                const int j0 = g * 32, left = P - j0;
+                att_group<PER, false>(q_s, pk + (size_t)j0 * d, pv + (size_t)j0 * d, left < 32 ? left : 32, d, dh, vec, scale, lane, mx, sum,
+                                      oacc);
+            } else {
+                const int j0 = (g - gp) * 32, left = L - j0;
+                att_group<PER, true>(q_s, kb + (size_t)j0 * d, vb + (size_t)j0 * d, left < 32 ? left : 32, d, dh, vec, scale, lane, mx, sum,
+                                     oacc);
+            }
+        }
+#pragma unroll
+        for (int qi = 0; qi < kAttQT; ++qi) {
+            float sm = sum[qi];
+#pragma unroll
+            for (int w = 16; w > 0; w >>= 1) sm += __shfl_xor_sync(0xffffffffu, sm, w);
+            float *mine = part_s + (size_t)(warp * kAttQT + qi) * stride;
+            if (lane == 0) {
+                mine[0] = mx[qi];
+                mine[1] = sm;
+            }
+#pragma unroll
+            for (int u = 0; u < NU; ++u)
+                if (feat(u) < dh) mine[2 + feat(u)] = oacc[qi][u];
+        }
+        sync();
+        // the four warps' results of each query of the tile: merged, and either final or this chunk's partial result
+        for (int qi = 0; qi < kAttQT && q0 + qi < L; ++qi) {
+            float top = -INFINITY, e[4], tot = 0.f;
+#pragma unroll
+            for (int w = 0; w < 4; ++w) top = fmaxf(top, part_s[(size_t)(w * kAttQT + qi) * stride]);
+#pragma unroll
+            for (int w = 0; w < 4; ++w) {
+                const float m = part_s[(size_t)(w * kAttQT + qi) * stride];
+                e[w] = m == -INFINITY ? 0.f : expf(m - top);          // (a warp, or a whole chunk, without keys)
+                tot = fmaf(part_s[(size_t)(w * kAttQT + qi) * stride + 1], e[w], tot);
+            }
+            float *dst = part + ((size_t)ch * L + q0 + qi) * stride;
+            if (n_ch > 1 && t == 0) {
+                dst[0] = top;
+                dst[1] = tot;
+            }
+            for (int c = t; c < dh; c += 128) {
+                float o = 0.f;
+#pragma unroll
+                for (int w = 0; w < 4; ++w) o = fmaf(part_s[(size_t)(w * kAttQT + qi) * stride + 2 + c], e[w], o);
+                if (n_ch > 1) dst[2 + c] = o;
+                else out(q0 + qi, c, o / tot);
+            }
+        }
+        sync();                                               // sh is free again
+    }
+    if (n_ch > 1) {
+        // arrive at the (block, head) counter; the CTA that arrives last merges the chunks and leaves the counter at zero
+        int *flag = reinterpret_cast<int *>(sh);
+        __threadfence();
+        sync();
+        if (t == 0) {
+            const int old = atomicAdd(counter, 1);
+            *flag = old == n_ch - 1;
+            if (old == n_ch - 1) {
+                __threadfence();
+                *counter = 0;
+            }
+        }
+        sync();
+        const bool last = *flag != 0;
+        sync();
+        if (last) {
+            // a warp per query: lanes over the chunks for the weights, then over the features, the partial results of
+            // all chunks in flight together
+            for (int i = warp; i < L; i += 4) {
+                const float m = lane < n_ch ? __ldcg(part + ((size_t)lane * L + i) * stride) : -INFINITY;
+                const float sm = lane < n_ch ? __ldcg(part + ((size_t)lane * L + i) * stride + 1) : 0.f;
+                float top = m;
+#pragma unroll
+                for (int w = 16; w > 0; w >>= 1) top = fmaxf(top, __shfl_xor_sync(0xffffffffu, top, w));
+                const float e = m == -INFINITY ? 0.f : expf(m - top);
+                float tot = sm * e;
+#pragma unroll
+                for (int w = 16; w > 0; w >>= 1) tot += __shfl_xor_sync(0xffffffffu, tot, w);
+                float o[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) o[u] = 0.f;
+#pragma unroll 4
+                for (int x = 0; x < n_ch; ++x) {
+                    const float ex = __shfl_sync(0xffffffffu, e, x);
+                    const float *src = part + ((size_t)x * L + i) * stride + 2;
+#pragma unroll
+                    for (int u = 0; u < 8; ++u)
+                        if (lane + 32 * u < dh) o[u] = fmaf(__ldcg(src + lane + 32 * u), ex, o[u]);
+                }
+#pragma unroll
+                for (int u = 0; u < 8; ++u)
+                    if (lane + 32 * u < dh) out(i, lane + 32 * u, o[u] / tot);
+            }
+        }
+    }
 }
 
 template <typename T, typename Sync, typename Out>
-__device__ __forceinline__ void att_prefix_item(const float *qi, const T *pk, const T *pv, int P, const float *kb,
-                                                const float *vb, int L, int d, int dh, float *sh, int warp, int lane, Sync sync,
-                                                Out out)
+__device__ __forceinline__ void att_unit(const float *q, const T *pk, const T *pv, int P, const float *kb, const float *vb, int L, int d,
+                                         int dh, int ch, int n_ch, int gpc, float *part, int *counter, float *sh, int warp, int lane,
+                                         Sync sync, Out out)
 {
-    float *q_s = sh, *part = sh + kAttMaxDh;              // part[w]: maximum, sum, o[dh]
-    const int t = warp * 32 + lane;
-    for (int c = t; c < dh; c += 128) q_s[c] = __ldcg(qi + c);
-    sync();
-    const float scale = rsqrtf((float)dh);
-    const bool vec = (dh % 8) == 0 && (d % 8) == 0;
-    float mx = -INFINITY, sum = 0.f, oacc[kAttMaxDh / 32];
-#pragma unroll
-    for (int u = 0; u < kAttMaxDh / 32; ++u) oacc[u] = 0.f;
-    const int gp = (P + 31) / 32, gb = (L + 31) / 32;
-    for (int g = warp; g < gp + gb; g += 4) {
-        const bool pre = g < gp;
-        const int j0 = pre ? g * 32 : (g - gp) * 32;
-        const int left = (pre ? P : L) - j0, cnt = left < 32 ? left : 32;
-        float s = -INFINITY;
-        if (lane < cnt)
-            s = (pre ? att_dot_ro(q_s, pk + (size_t)(j0 + lane) * d, dh, vec) : att_dot_cg(q_s, kb + (size_t)(j0 + lane) * d, dh, vec)) *
-                scale;
-        float gm = s;
-#pragma unroll
-        for (int w = 16; w > 0; w >>= 1) gm = fmaxf(gm, __shfl_xor_sync(0xffffffffu, gm, w));
-        const float nm = fmaxf(mx, gm), corr = expf(mx - nm);            // (mx = -inf at first: corr = 0)
-        const float pj = lane < cnt ? expf(s - nm) : 0.f;
-        sum = sum * corr + pj;                                           // per-lane share; corr is the same in every lane
-#pragma unroll
-        for (int u = 0; u < kAttMaxDh / 32; ++u) oacc[u] *= corr;
-        if (pre && cnt == 32) {
-            // a full group of prefix rows: the value loads of eight keys in flight together
-#pragma unroll 8
-            for (int jj = 0; jj < 32; ++jj) {
-                const float w = __shfl_sync(0xffffffffu, pj, jj);
-                const T *vr = pv + (size_t)(j0 + jj) * d;
-#pragma unroll
-                for (int u = 0; u < kAttMaxDh / 32; ++u) {
-                    const int c = lane + 32 * u;
-                    if (c < dh) oacc[u] = fmaf(w, att_f(__ldg(vr + c)), oacc[u]);
-                }
-            }
-        } else {
-            for (int jj = 0; jj < cnt; ++jj) {
-                const float w = __shfl_sync(0xffffffffu, pj, jj);
-                if (pre) {
-                    const T *vr = pv + (size_t)(j0 + jj) * d;
-#pragma unroll
-                    for (int u = 0; u < kAttMaxDh / 32; ++u) {
-                        const int c = lane + 32 * u;
-                        if (c < dh) oacc[u] = fmaf(w, att_f(__ldg(vr + c)), oacc[u]);
-                    }
-                } else {
-                    const float *vr = vb + (size_t)(j0 + jj) * d;
-#pragma unroll
-                    for (int u = 0; u < kAttMaxDh / 32; ++u) {
-                        const int c = lane + 32 * u;
-                        if (c < dh) oacc[u] = fmaf(w, __ldcg(vr + c), oacc[u]);
-                    }
-                }
-            }
-        }
-        mx = nm;
-    }
-#pragma unroll
-    for (int w = 16; w > 0; w >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, w);
-    float *mine = part + warp * (kAttMaxDh + 2);
-    if (lane == 0) {
-        mine[0] = mx;
-        mine[1] = sum;
-    }
-#pragma unroll
-    for (int u = 0; u < kAttMaxDh / 32; ++u) {
-        const int c = lane + 32 * u;
-        if (c < dh) mine[2 + c] = oacc[u];
-    }
-    sync();
-    // the block has at least one key, so the overall maximum is finite; a warp that had no keys weighs 0
-    float top = -INFINITY, e[4], tot = 0.f;
-#pragma unroll
-    for (int w = 0; w < 4; ++w) top = fmaxf(top, part[w * (kAttMaxDh + 2)]);
-#pragma unroll
-    for (int w = 0; w < 4; ++w) {
-        e[w] = expf(part[w * (kAttMaxDh + 2)] - top);
-        tot = fmaf(part[w * (kAttMaxDh + 2) + 1], e[w], tot);
-    }
-    for (int c = t; c < dh; c += 128) {
-        float o = 0.f;
-#pragma unroll
-        for (int w = 0; w < 4; ++w) o = fmaf(part[w * (kAttMaxDh + 2) + 2 + c], e[w], o);
-        out(c, o / tot);
-    }
-    sync();                                                              // sh is free again
+    // heads of 64 or 128 features, rows 16-byte aligned: the lane's features are consecutive and load as one vector
+    if (dh == 128 && (d % 8) == 0)
+        att_unit_per<4>(q, pk, pv, P, kb, vb, L, d, dh, ch, n_ch, gpc, part, counter, sh, warp, lane, sync, out);
+    else if (dh == 64 && (d % 8) == 0)
+        att_unit_per<2>(q, pk, pv, P, kb, vb, L, d, dh, ch, n_ch, gpc, part, counter, sh, warp, lane, sync, out);
+    else
+        att_unit_per<0>(q, pk, pv, P, kb, vb, L, d, dh, ch, n_ch, gpc, part, counter, sh, warp, lane, sync, out);
 }
-
 
 }  // namespace mrp

@@ -1238,49 +1238,51 @@ __global__ void mod_attention_kernel(const float *__restrict__ q, const float *_
     }
 }
 
-// The same behind a clean prefix (Fig. 1(c)): CTA = (query position, attention head); keys and values are the first
-// prefix_len[b] rows of sequence b's slab of the cache [*, cap, d], then the block's own rows.  With `append` the
-// block's keys and values are also stored behind the prefix rows (rows the call itself never reads).
+// The same behind a clean prefix (Fig. 1(c)): CTA = (block, attention head, chunk of the keys); keys and values are
+// the first prefix_len[b] rows of sequence b's slab of the cache [*, cap, d], then the block's own rows.  With `append`
+// the block's keys and values are also stored behind the prefix rows (rows the call itself never reads).
 template <typename T>
 __global__ void __launch_bounds__(128) mod_attention_prefix_kernel(const float *__restrict__ q, const float *k, const float *v, int L,
                                                                    int d, int dh, int H, float *__restrict__ o,
                                                                    __nv_bfloat16 *__restrict__ o16, int n_rows, T *pk, T *pv,
-                                                                   const int32_t *__restrict__ plen, int cap, int append,
+                                                                   const int32_t *__restrict__ plen, int cap, int append, int n_ch,
+                                                                   int gpc, float *part, int *counters,
                                                                    int32_t *__restrict__ status, int32_t *__restrict__ user_status)
 {
     pdl_trigger();
     pdl_wait();
-    __shared__ __align__(16) float sh[kAttShFloats];
-    const int item = blockIdx.x, pos = item / H, hd = item - pos * H, b = pos / L, i = pos - b * L;
+    extern __shared__ __align__(16) float att_sh[];
+    const int unit = blockIdx.x, ch = unit % n_ch, bh = unit / n_ch, b = bh / H, hd = bh - b * H;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     int P = plen[b];
     bool bad = P < 0 || P > cap;
     P = P < 0 ? 0 : (P > cap ? cap : P);
     const bool store = append && !bad && P + L <= cap;
     bad = bad || (append && !store);
-    if (bad && threadIdx.x == 0 && hd == 0 && i == 0) {
+    if (bad && threadIdx.x == 0 && hd == 0 && ch == 0) {
         atomicOr(status, MRP_DEV_BAD_INDEX);
         if (user_status) atomicOr(user_status, MRP_DEV_BAD_INDEX);
     }
-    const size_t head = (size_t)hd * dh, slab = (size_t)b * cap * d + head, own = (size_t)pos * d + head;
-    if (store) {
-        T *dk = pk + slab + (size_t)(P + i) * d, *dv = pv + slab + (size_t)(P + i) * d;
-        for (int c = threadIdx.x; c < dh; c += 128) {
-            dk[c] = (T)k[own + c];
-            dv[c] = (T)v[own + c];
+    const size_t head = (size_t)hd * dh, slab = (size_t)b * cap * d + head, blk = (size_t)b * L * d + head;
+    if (store && ch == 0) {
+        for (int x = threadIdx.x; x < L * dh; x += 128) {
+            const int i = x / dh, c = x - i * dh;
+            pk[slab + (size_t)(P + i) * d + c] = (T)k[blk + (size_t)i * d + c];
+            pv[slab + (size_t)(P + i) * d + c] = (T)v[blk + (size_t)i * d + c];
         }
     }
-    att_prefix_item<T>(q + own, pk + slab, pv + slab, P, k + (size_t)b * L * d + head, v + (size_t)b * L * d + head, L, d, dh, sh,
-                       warp, lane, [] { __syncthreads(); }, [&](int c, float val) {
-                           const size_t at = own + c;
-                           if (o16) {
-                               const __nv_bfloat16 hh = __float2bfloat16_rn(val);
-                               o16[at] = hh;
-                               o16[(size_t)n_rows * d + at] = __float2bfloat16_rn(val - __bfloat162float(hh));
-                           } else {
-                               o[at] = val;
-                           }
-                       });
+    att_unit<T>(q + blk, pk + slab, pv + slab, P, k + blk, v + blk, L, d, dh, ch, n_ch, gpc,
+                part + (size_t)bh * n_ch * L * (dh + 2), counters + bh, att_sh, warp, lane, [] { __syncthreads(); },
+                [&](int i, int c, float val) {
+                    const size_t at = blk + (size_t)i * d + c;
+                    if (o16) {
+                        const __nv_bfloat16 hh = __float2bfloat16_rn(val);
+                        o16[at] = hh;
+                        o16[(size_t)n_rows * d + at] = __float2bfloat16_rn(val - __bfloat162float(hh));
+                    } else {
+                        o[at] = val;
+                    }
+                });
 }
 
 // h <- h + Delta for every dense position.
@@ -1863,9 +1865,15 @@ static cudaError_t module_attention(Ctx *c, int layer, int B, int L, const float
     if (!c->has_prefix)
         return launch_k(mod_attention_kernel, dim3(B, w.n_attn_heads), dim3(128), (size_t)4 * L * 4, st, pdl, q, k, v, L, d, dh, o, o16,
                         n_rows);
-    return launch_k(mod_attention_prefix_kernel<T>, dim3((unsigned)(B * L * w.n_attn_heads)), dim3(128), 0, st, pdl, q, k, v, L, d, dh,
-                    w.n_attn_heads, o, o16, n_rows, (T *)c->prefix_layers[layer].k, (T *)c->prefix_layers[layer].v, c->prefix_len,
-                    c->prefix_cap, c->prefix_append ? 1 : 0, (int32_t *)(c->ws + c->lay.status), out.status);
+    // the keys of a (block, head) split over CTAs where there are few of those; the partial results and the arrival
+    // counters (zero before and after every launch) sit behind the module's other workspace
+    const AttSplit sp = att_split(c->prefix_cap, L, B * w.n_attn_heads, dh, 4 * c->sm_count);
+    float *part = (float *)(c->module_ws + module_att_offset(c->cfg));
+    int *counters = (int *)(part + kAttPartFloats);
+    return launch_k(mod_attention_prefix_kernel<T>, dim3((unsigned)(B * w.n_attn_heads * sp.n_ch)), dim3(128),
+                    (size_t)att_sh_floats(dh) * 4, st, pdl, q, k, v, L, d, dh, w.n_attn_heads, o, o16, n_rows,
+                    (T *)c->prefix_layers[layer].k, (T *)c->prefix_layers[layer].v, c->prefix_len, c->prefix_cap,
+                    c->prefix_append ? 1 : 0, sp.n_ch, sp.gpc, part, counters, (int32_t *)(c->ws + c->lay.status), out.status);
 }
 
 // The module itself (everything in front of `h <- h + Delta`) with its products on the tensor cores.
@@ -1940,13 +1948,20 @@ static cudaError_t module_body_tc(Ctx *c, const int32_t *tokens, const void *hid
     return e;
 }
 
-size_t module_workspace_bytes(const mrp_config &cfg, int n_layers)
+// Where the clean-prefix attention's area starts: the partial results of split units, then their arrival counters
+// (zeroed at the start of every step that uses them).
+size_t module_att_offset(const mrp_config &cfg)
 {
-    (void)n_layers;
     const size_t n = module_cap_rows(cfg), d = (size_t)cfg.d, F = (size_t)cfg.d_ff;
     // (the last term: the arrival counters of the one-launch tensor-core step)
     return align_up(n * 2 * d * 4, 256) + 6 * align_up(n * d * 4, 256) + align_up(n * F * 4, 256) +
            align_up((size_t)kModChainBarInts * 4, 256);
+}
+
+size_t module_workspace_bytes(const mrp_config &cfg, int n_layers)
+{
+    (void)n_layers;
+    return module_att_offset(cfg) + align_up(kAttPartFloats * 4, 256) + align_up((size_t)kAttCounters * 4, 256);
 }
 
 template <typename T>
@@ -1968,6 +1983,12 @@ static cudaError_t module_step_t(Ctx *c, const int32_t *tokens, const void *hidd
         return launch_k(linear_kernel<T>, dim3((n_out + 7) / 8), dim3(256), 0, st, pdl, (const T *)wm, x, n, n_in, n_out, y, acc);
     };
     prof_mark(c, 0, st);
+    float *att_part = (float *)(c->module_ws + module_att_offset(c->cfg));
+    if (c->has_prefix) {
+        // the arrival counters of the clean-prefix attention's split units start at zero (every launch leaves them so)
+        const cudaError_t ez = cudaMemsetAsync(att_part + kAttPartFloats, 0, (size_t)kAttCounters * 4, st);
+        if (ez != cudaSuccess) return ez;
+    }
     if (module_chain_ok(c, n, L, st)) {
         // up to 64 positions on a tensor-core context: the whole step (fusion, the layers, h <- h + Delta, the LM-head
         // operand) as one cooperative tcgen05 kernel, then the LM-head kernels.  (At four positions, decode shape:
@@ -1986,7 +2007,7 @@ static cudaError_t module_step_t(Ctx *c, const int32_t *tokens, const void *hidd
         int32_t *bar_mem = (int32_t *)wp;
         const cudaError_t ec = sk_module_step(c, n, L, tokens, hidden0, h_state, first_step, cat16, xa, xb, act16, qc, kc2, vc, zc,
                                               bar_mem, row_index, M, c->lo_xt, M > 0 && pl.f16_lm, out.hidden_out, out.status, st,
-                                              false);
+                                              false, att_part, (int *)(att_part + kAttPartFloats));
         if (ec != cudaSuccess || M == 0) return ec;
         return tc_lm_tail(c, pl, logits0, row_index, M, 1, out, st);
     } else {

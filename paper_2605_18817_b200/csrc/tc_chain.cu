@@ -96,6 +96,9 @@ struct ModEnds {
     float *hidden_out;
     const int32_t *plen;     // clean prefix: rows in use per sequence, rows per slab, whether the block's own keys and
     int pcap, append;        // values are stored behind them
+    int att_nch, att_gpc;    // ... chunks of the key range per (block, head), groups of 32 keys per chunk
+    float *att_part;         // partial results of the chunks
+    int *att_counters;       // arrivals per (block, head): zero before and after the launch
 };
 
 template <int NP>
@@ -734,33 +737,34 @@ sk_chain_kernel(const __grid_constant__ typename ChainTypes<MOD>::Maps maps,
                     }
                 }
                 if (ph.kind == CH_ATT && ph.att_pk) {
-                    // attention behind a clean prefix: the four warps on one (position, attention head) at a time
+                    // attention behind a clean prefix: the four warps on one (block, attention head, chunk of the keys)
+                    // at a time; the CTA that arrives last at a (block, head) merges its chunks
                     const ModEnds &e = p.mod;
-                    const int L = ph.att_L, H = ph.att_H, dh = p.d / H;
-                    for (int item = cta; item < p.M * H; item += G) {
-                        const int pos = item / H, hd = item - pos * H, b = pos / L, i2 = pos - b * L;
+                    const int L = ph.att_L, H = ph.att_H, dh = p.d / H, n_ch = e.att_nch;
+                    for (int unit = cta; unit < (p.M / L) * H * n_ch; unit += G) {
+                        const int ch = unit % n_ch, bh = unit / n_ch, b = bh / H, hd = bh - b * H;
                         int P = e.plen[b];
                         bool bad = P < 0 || P > e.pcap;
                         P = P < 0 ? 0 : (P > e.pcap ? e.pcap : P);
                         const bool store = e.append && !bad && P + L <= e.pcap;
                         bad = bad || (e.append && !store);
-                        if (bad && t == 0 && hd == 0 && i2 == 0) {
+                        if (bad && t == 0 && hd == 0 && ch == 0) {
                             atomicOr(p.status, MRP_DEV_BAD_INDEX);
                             if (p.user_status) atomicOr(p.user_status, MRP_DEV_BAD_INDEX);
                         }
-                        const size_t head = (size_t)hd * dh, slab = (size_t)b * e.pcap * p.d + head, own = (size_t)pos * p.d + head;
-                        if (store) {                  // rows this call never reads
-                            __nv_bfloat16 *dk = ph.att_pk + slab + (size_t)(P + i2) * p.d, *dv = ph.att_pv + slab + (size_t)(P + i2) * p.d;
-                            for (int cidx = t; cidx < dh; cidx += 128) {
-                                dk[cidx] = __float2bfloat16_rn(__ldcg(ph.att_k + own + cidx));
-                                dv[cidx] = __float2bfloat16_rn(__ldcg(ph.att_v + own + cidx));
+                        const size_t head = (size_t)hd * dh, slab = (size_t)b * e.pcap * p.d + head, blk = (size_t)b * L * p.d + head;
+                        if (store && ch == 0) {       // rows this call never reads
+                            for (int x = t; x < L * dh; x += 128) {
+                                const int i2 = x / dh, cidx = x - i2 * dh;
+                                ph.att_pk[slab + (size_t)(P + i2) * p.d + cidx] = __float2bfloat16_rn(__ldcg(ph.att_k + blk + (size_t)i2 * p.d + cidx));
+                                ph.att_pv[slab + (size_t)(P + i2) * p.d + cidx] = __float2bfloat16_rn(__ldcg(ph.att_v + blk + (size_t)i2 * p.d + cidx));
                             }
                         }
-                        att_prefix_item<__nv_bfloat16>(ph.att_q + own, ph.att_pk + slab, ph.att_pv + slab, P,
-                                                       ph.att_k + (size_t)b * L * p.d + head, ph.att_v + (size_t)b * L * p.d + head, L, p.d,
-                                                       dh, sq_s, q, lane, [&] { ch_epi_sync(); }, [&](int cidx, float val) {
-                                                           ch_store_hi_lo(ph.att_out + own + cidx, (size_t)p.lo_x * p.d, val);
-                                                       });
+                        att_unit<__nv_bfloat16>(ph.att_q + blk, ph.att_pk + slab, ph.att_pv + slab, P, ph.att_k + blk, ph.att_v + blk, L, p.d,
+                                                dh, ch, n_ch, e.att_gpc, e.att_part + (size_t)bh * n_ch * L * (dh + 2), e.att_counters + bh,
+                                                sq_s, q, lane, [&] { ch_epi_sync(); }, [&](int i2, int cidx, float val) {
+                                                    ch_store_hi_lo(ph.att_out + blk + (size_t)i2 * p.d + cidx, (size_t)p.lo_x * p.d, val);
+                                                });
                     }
                 } else if (ph.kind == CH_ATT) {
                     // block-local bidirectional attention, a warp per (position, attention head) over the whole grid;
@@ -1000,13 +1004,17 @@ cudaError_t sk_chain(Ctx *c, int M, int K, const mrp_draft_out &out, cudaStream_
 cudaError_t sk_module_step(Ctx *c, int n, int L, const int32_t *tokens, const void *hidden0, float *h_state, bool first_step,
                            __nv_bfloat16 *cat16, __nv_bfloat16 *xa, __nv_bfloat16 *xb, __nv_bfloat16 *act16, float *q, float *k,
                            float *v, float *z, int32_t *bar_mem, const int32_t *row_index, int n_masked, int lo_xt, bool f16_lm,
-                           float *hidden_out, int32_t *user_status, cudaStream_t st, bool check_only)
+                           float *hidden_out, int32_t *user_status, cudaStream_t st, bool check_only, float *att_part,
+                           int *att_counters)
 {
     const TcState *s = (const TcState *)c->tc_state;
     const mrp_module_weights &w = c->module;
     const int d = c->cfg.d, F = c->cfg.d_ff, G = c->sm_count, D = w.n_layers, H = w.n_attn_heads;
     if (D < 1 || D > kModChainLayers || n < 1 || n > 128 || d % 128 || F % 64 || d / H > 256 || (d / H) % 32)
         return cudaErrorNotSupported;
+    // (the clean-prefix attention stages a tile of queries and the four warps' partial results in the 16 KB of
+    // shared memory the phases share)
+    if (c->has_prefix && att_sh_floats(d / H) > 4096) return cudaErrorNotSupported;
     const int r_pad = sk_head_pad(n);
     const int d_tiles = d / 128, gu_tiles = F / 64;
     if (3 * d_tiles > G || gu_tiles > G || 3 * d_tiles > kChTilesPerPhase || gu_tiles > kChTilesPerPhase ||
@@ -1061,7 +1069,11 @@ cudaError_t sk_module_step(Ctx *c, int n, int L, const int32_t *tokens, const vo
     p.mod.mask_token = w.mask_token; p.mod.emb_rows = w.emb_rows; p.mod.row_index = row_index; p.mod.n_masked = n_masked;
     p.mod.xt = (__nv_bfloat16 *)(c->ws + c->lay.xt); p.mod.xt16 = f16_lm ? (__half *)(c->ws + c->lay.xt16) : nullptr;
     p.mod.hidden_out = hidden_out;
-    if (c->has_prefix) { p.mod.plen = c->prefix_len; p.mod.pcap = c->prefix_cap; p.mod.append = c->prefix_append ? 1 : 0; }
+    if (c->has_prefix) {
+        const AttSplit sp = att_split(c->prefix_cap, L, (n / L) * H, d / H, G);
+        p.mod.plen = c->prefix_len; p.mod.pcap = c->prefix_cap; p.mod.append = c->prefix_append ? 1 : 0;
+        p.mod.att_nch = sp.n_ch; p.mod.att_gpc = sp.gpc; p.mod.att_part = att_part; p.mod.att_counters = att_counters;
+    }
     bool ok = make_map(s, &maps.m[0], xa, d, 2 * (uint64_t)r_pad, 2 * r_pad) && make_map(s, &maps.m[1], act16, F, 2 * (uint64_t)r_pad, 2 * r_pad) &&
               make_map(s, &maps.m[2], xb, d, 2 * (uint64_t)r_pad, 2 * r_pad) &&
               make_map(s, &maps.m[3], cat16, 2 * d, 2 * (uint64_t)r_pad, 2 * r_pad) && make_map(s, &maps.m[4], w.w_proj, 2 * d, d, 128);
