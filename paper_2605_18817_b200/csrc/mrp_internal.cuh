@@ -344,7 +344,7 @@ __device__ inline Partial merge_partial(const Partial &a, const Partial &b)
 //               128 threads;  out(i, c, value) is called once per query i of the block and feature c of the head
 constexpr int kAttMaxDh = 256;
 constexpr int kAttQT = 4;
-constexpr int kAttMaxChunks = 16;
+constexpr int kAttMaxChunks = 32;                      // (the merge puts a lane on every chunk)
 constexpr int kAttCounters = 4096;                    // (block, head) pairs that can split their keys over CTAs
 constexpr size_t kAttPartFloats = (size_t)1 << 20;    // partial results of split units
 __host__ __device__ constexpr int att_sh_floats(int dh) { return kAttQT * dh + 4 * kAttQT * (dh + 2); }

@@ -1867,7 +1867,7 @@ static cudaError_t module_attention(Ctx *c, int layer, int B, int L, const float
                         n_rows);
     // the keys of a (block, head) split over CTAs where there are few of those; the partial results and the arrival
     // counters (zero before and after every launch) sit behind the module's other workspace
-    const AttSplit sp = att_split(c->prefix_cap, L, B * w.n_attn_heads, dh, 4 * c->sm_count);
+    const AttSplit sp = att_split(c->prefix_cap, L, B * w.n_attn_heads, dh, 8 * c->sm_count);
     float *part = (float *)(c->module_ws + module_att_offset(c->cfg));
     int *counters = (int *)(part + kAttPartFloats);
     return launch_k(mod_attention_prefix_kernel<T>, dim3((unsigned)(B * w.n_attn_heads * sp.n_ch)), dim3(128),
