@@ -280,3 +280,57 @@ def test_random_shapes_behind_random_prefixes(seed):
         clear = margin > 1e-2
         assert np.array_equal(out.token[1].cpu().numpy()[clear], tok[clear]), what
         binding.mrp_destroy(ctx)
+
+
+@pytest.mark.parametrize("which,L,P,blocks_checked", [
+    (1, 4, 1024, 1),     # decode shape, one block of 4 behind 1024 prefix positions: 9 key chunks per (block, head)
+    (1, 16, 1024, 1),    # ... one block of 16: four query tiles per unit
+    (2, 4, 300, 2),      # 32 blocks of 4 at d = 4096: the separate kernel, one unit per (block, head); oracle on two blocks
+])
+def test_prefix_at_the_benchmark_shapes(which, L, P, blocks_checked):
+    """One module step behind a prefix at the shapes bench.py's module:P<n> workloads time (D = 3, 128 features per
+    attention head, random caches), against the oracle on the first blocks."""
+    cfg = dict(synth.CONFIGS[which], L=L)
+    d, F, V, B = cfg["d"], cfg["F"], cfg["V"], cfg["B"]
+    n, n_attn, D = B * L, d // 128, 3
+    w = synth.make_weights(d, F, V, 1, "bf16", cfg["seed"])
+    heads_dev, w_lm = harness.upload_weights(w, DEV)
+    _, inp = synth.make_config(cfg, w, logits_fn=harness.device_logits_fn(w_lm))
+    mw = synth.make_module_weights(d, F, V, D, n_attn, "bf16", 11, std=0.02 if d < 4096 else 0.01)
+    ctx = binding.mrp_create(d, F, V, heads_dev, w_lm, max_rows=n, max_seqs=B, block_len=L)
+    up = lambda a: harness.to_device(a, "bf16", DEV)
+    binding.mrp_module_attach(ctx, up(mw.emb), up(mw.w_proj), [{k: up(v) for k, v in lay.items()} for lay in mw.layers],
+                              n_attn, mw.mask_token)
+    plen = [P - (b % 3) for b in range(B)]
+    host = make_prefix(D, B, P, d, plen, "bf16", 13)
+    dev = [(k.to(DEV), v.to(DEV)) for k, v in host]
+    binding.mrp_module_set_prefix(ctx, dev, torch.tensor(plen, dtype=torch.int32, device=DEV))
+    tokens = np.full(n, -1, np.int32)
+    tokens[::L] = 17
+    ri = np.flatnonzero(tokens < 0).astype(np.int32)
+    M = ri.size
+    h_state = torch.empty((n, d), device=DEV, dtype=torch.float32)
+    out = harness.alloc_draft_out(M, 1, V, d, DEV)
+    binding.mrp_module_step(ctx, torch.from_numpy(tokens).to(DEV), harness.to_device(inp.hidden, "bf16", DEV), h_state,
+                            torch.from_numpy(inp.logits0).to(DEV), torch.from_numpy(ri).to(DEV), M, B, L, True, out.conf, out.lse,
+                            out.token, status=out.status)
+    torch.cuda.synchronize()
+    assert int(out.status.item()) == 0
+    ns, Bs = blocks_checked * L, blocks_checked
+    ri_s = np.flatnonzero(tokens[:ns] < 0).astype(np.int32)
+    ks, vs, pl = as_oracle_prefix(host, plen)
+    dh, dl = oracle.module(inp.hidden[:ns], tokens[:ns], Bs, L, mw.emb, mw.w_proj, mw.layers, w.w_lm, n_attn, mw.mask_token,
+                           row_index=ri_s, prefix=([k[:Bs] for k in ks], [v[:Bs] for v in vs], pl[:Bs]))
+    alone, _ = oracle.module(inp.hidden[:ns], tokens[:ns], Bs, L, mw.emb, mw.w_proj, mw.layers, w.w_lm, n_attn, mw.mask_token)
+    assert np.abs(dh - alone).max() > 1e-3
+    h_ref = inp.hidden[:ns].astype(np.float64) + dh
+    assert np.abs(h_state[:ns].cpu().numpy() - h_ref).max() <= 1e-3 * max(1.0, np.abs(h_ref).max())
+    conf, lse, tok, margin = oracle.stats(inp.logits0[ri_s].astype(np.float64) + dl)
+    m_s = ri_s.size
+    assert np.abs(out.conf[1, :m_s].cpu().numpy() - conf).max() <= TOL["bf16"]
+    assert np.abs(out.lse[1, :m_s].cpu().numpy() - lse).max() <= TOL["bf16"]
+    clear = margin > 1e-2
+    assert np.array_equal(out.token[1, :m_s].cpu().numpy()[clear], tok[clear])
+    binding.mrp_destroy(ctx)
+    del ctx, w_lm, heads_dev, dev
+    torch.cuda.empty_cache()
