@@ -654,7 +654,7 @@ def run_module_workload(bench, cpu_budget_s, which=1, block_len=None, prefix=0):
     base = synth.CONFIGS[which]
     if block_len:                                      # the paper's block length (Sec. 4.1) instead of the configuration's
         base = dict(base, L=block_len, name="%s_L%d" % (base["name"], block_len))
-    cfg = dict(base, name="module_" + base["name"] + ("_P%d" % prefix if prefix else ""))
+    cfg = dict(base, name="module_" + base["name"] + ("_P%d" % prefix if prefix else "") + ("_fp8lm" if args.fp8_lm else ""))
     w, heads, w_lm = bench.weights_for(base, str(which))
     big = base["d"] >= 4096
     _, inp = synth.make_config(base, w, logits_fn=harness.device_logits_fn(w_lm) if big else None)
@@ -664,7 +664,8 @@ def run_module_workload(bench, cpu_budget_s, which=1, block_len=None, prefix=0):
     # (layer weights scaled so that the residual stays inside the accuracy range of the tensor-core LM head:
     # d * rms(h - h_0) <= MRP_RANGE_LIMIT, checked by the device status word below)
     mw = synth.make_module_weights(d, F, V, MODULE_LAYERS, n_attn, "bf16", 11, std=0.02 if d < 4096 else 0.01)
-    ctx = binding.mrp_create(d, F, V, heads[:1], w_lm, max_rows=n, max_seqs=B, block_len=L, flags=args.flags)
+    ctx = binding.mrp_create(d, F, V, heads[:1], w_lm, max_rows=n, max_seqs=B, block_len=L,
+                             flags=args.flags | (binding.MRP_FLAG_FP8_LM if args.fp8_lm else 0))
     up = lambda a: harness.to_device(a, "bf16", dev)
     binding.mrp_module_attach(ctx, up(mw.emb), up(mw.w_proj), [{k: up(v) for k, v in lay.items()} for lay in mw.layers],
                               n_attn, mw.mask_token)
@@ -719,7 +720,7 @@ def run_module_workload(bench, cpu_budget_s, which=1, block_len=None, prefix=0):
     (ms_mod, ms_lm, ms_comb), n_calls = binding.mrp_profile_read(ctx)
     binding.mrp_profile_enable(ctx, False)
     one = dict(cfg, K=1)
-    roofline = lm_head_roofline(one, n - 2 * B, ms_lm / max(n_calls, 1), bench.peaks, bench.peaks_kind)
+    roofline = lm_head_roofline(one, n - 2 * B, ms_lm / max(n_calls, 1), bench.peaks, bench.peaks_kind, fp8=args.fp8_lm)
     roofline["kernel"] = "fused LM head, one launch per MRP step (K = %d weight streams per backbone forward)" % K
     roofline["units_per_launch"] = 1
     res["roofline"] = roofline

@@ -309,7 +309,10 @@ int mrp_module_attach(mrp_ctx *ctx, const mrp_module_weights *w, void *workspace
  *            logits, entry 1 the logits after this step, l_0 + W_lm (h - h_0), which by linearity is the
  *            running sum l <- l + delta of Algorithm 2; hidden_out optional [M, d]; logits_out [1, M, V]
  * The caller reveals from entry 1 (mrp_reveal_remask with K = 0 on it, mrp_commit), updates tokens and
- * calls again.  Errors: INVALID_ARG, UNSUPPORTED (no module attached), CUDA.
+ * calls again.  On a context created with MRP_FLAG_FP8_LM the step's LM-head pass runs on the 8-bit copy of
+ * W_lm, like mrp_draft's (the module's own matrices stay in the context dtype): with one LM-head pass per MRP
+ * step instead of one per backbone forward, that stream weighs K times as much here.
+ * Errors: INVALID_ARG, UNSUPPORTED (no module attached), CUDA.
  */
 int mrp_module_step(mrp_ctx *ctx, const int32_t *tokens, const void *hidden0, float *h_state,
                     const float *logits0, const int32_t *row_index, int32_t M, int32_t B, int32_t L,

@@ -405,7 +405,7 @@ int mrp_module_step(mrp_ctx *ctx, const int32_t *tokens, const void *hidden0, fl
 {
     if (!ctx || !out) return MRP_ERR_INVALID_ARG;
     Ctx &c = ctx->c;
-    if (!c.has_module || c.use_fp8_lm) return MRP_ERR_UNSUPPORTED;
+    if (!c.has_module) return MRP_ERR_UNSUPPORTED;
     if (B < 1 || B > c.cfg.max_seqs || L < 1 || L > c.cfg.block_len) return MRP_ERR_INVALID_ARG;
     if (M < 0 || M > c.cfg.max_rows || (long long)M > (long long)B * L) return MRP_ERR_INVALID_ARG;
     if (!tokens || !hidden0 || !h_state || ((uintptr_t)hidden0 & 15u) || ((uintptr_t)h_state & 15u)) return MRP_ERR_INVALID_ARG;

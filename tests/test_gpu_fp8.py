@@ -82,3 +82,60 @@ def test_8_bit_lm_head_is_refused_outside_the_decode_regime():
     with pytest.raises(binding.MrpError):
         binding.mrp_quantised_lm_head(ctx)                                       # no 8-bit copy in this context
     binding.mrp_destroy(ctx)
+
+
+@pytest.mark.parametrize("d,F,V,D,heads,B,L", [
+    (256, 512, 4096, 2, 2, 2, 4),        # 16 row-steps, the step as one cooperative kernel
+    (512, 1024, 2064, 1, 4, 1, 5),       # ragged vocabulary, a block of five
+    (2048, 4096, 151936, 3, 16, 1, 4),   # the decode configuration at full size, the paper's depth
+])
+def test_module_step_on_the_8_bit_lm_head(d, F, V, D, heads, B, L):
+    """The token-conditioned module's step on an MRP_FLAG_FP8_LM context: its LM-head pass runs on the 8-bit copy,
+    so its results are the oracle's module with the dequantised matrix as the LM head."""
+    from test_gpu_module import upload_module
+    big = d == 2048
+    w = synth.make_weights(d, F, V, 1, "bf16", 1 if big else 95)
+    mw = synth.make_module_weights(d, F, V, D, heads, "bf16", 11 if big else 95, std=0.02 if big else 0.06,
+                                   proj_std=None if big else 0.3 / np.sqrt(2 * d))
+    inp = synth.make_inputs(w, B, L, 95, 1.0, 4.0)
+    _, _, w8 = fp8.quantise_rows(w.w_lm)
+    n = B * L
+    ctx = _ctx(w, n, B, L)
+    emb, w_proj, layers = upload_module(mw, "bf16")
+    binding.mrp_module_attach(ctx, emb, w_proj, layers, heads, mw.mask_token)
+    tokens = np.full(n, -1, np.int32)
+    tokens[::L] = 17
+    hid0 = harness.to_device(inp.hidden, "bf16", DEV)
+    l0 = torch.from_numpy(inp.logits0).to(DEV)
+    h_state = torch.empty((n, d), device=DEV, dtype=torch.float32)
+    h_run = inp.hidden.astype(np.float64)
+    l_run = inp.logits0.astype(np.float64)
+    for s in range(2):
+        ri = np.flatnonzero(tokens < 0).astype(np.int32)
+        M = ri.size
+        out = harness.alloc_draft_out(M, 1, V, d, DEV, hidden=True)
+        binding.mrp_module_step(ctx, torch.from_numpy(tokens).to(DEV), hid0, h_state, l0, torch.from_numpy(ri).to(DEV), M, B, L,
+                                s == 0, out.conf, out.lse, out.token, margin=out.margin, hidden_out=out.hidden, status=out.status)
+        torch.cuda.synchronize()
+        assert int(out.status.item()) == 0
+        dh, dl = oracle.module(h_run.astype(np.float32), tokens, B, L, mw.emb, mw.w_proj, mw.layers, w8, heads, mw.mask_token,
+                               row_index=ri)
+        h_run = h_run.astype(np.float32).astype(np.float64) + dh
+        l_run[ri] += dl
+        conf, lse, tok, margin = oracle.stats(l_run[ri])
+        assert np.abs(h_state.cpu().numpy() - h_run).max() <= 1e-3 * max(1.0, np.abs(h_run).max())
+        assert np.abs(out.conf[1].cpu().numpy() - conf).max() <= 2e-3 and np.abs(out.lse[1].cpu().numpy() - lse).max() <= 2e-3
+        clear = margin > 1e-2
+        assert np.array_equal(out.token[1].cpu().numpy()[clear], tok[clear])
+        # the quantisation is visible against the unquantised head
+        if s == 0:
+            _, dl_full = oracle.module(inp.hidden, tokens, B, L, mw.emb, mw.w_proj, mw.layers, w.w_lm, heads, mw.mask_token,
+                                       row_index=ri)
+            assert np.abs(dl_full - dl).max() > 1e-4
+        # reveal the most confident masked position of every block for the next step
+        for b in range(B):
+            rows = [m for m in range(M) if ri[m] // L == b]
+            if rows:
+                best = max(rows, key=lambda m: conf[m])
+                tokens[ri[best]] = tok[best]
+    binding.mrp_destroy(ctx)
