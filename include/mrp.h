@@ -319,6 +319,20 @@ int mrp_module_step(mrp_ctx *ctx, const int32_t *tokens, const void *hidden0, fl
                     int32_t first_step, const mrp_draft_out *out, void *cuda_stream);
 
 /*
+ * mrp_module_step with the training objective of that step fused into its LM-head pass (Algorithm 1: the
+ * module g is what the objective trains; Eq. (3); Sec. 4.1):
+ *     kl[m] = KL( softmax(teacher[m, :]) || softmax(l[m, :]) ),   l = l_0 + W_lm (h - h_0) after this step,
+ * teacher the frozen backbone's logits on the sequence with this step's ground-truth tokens revealed, accumulated
+ * online next to the softmax statistics as in mrp_draft_kl.
+ *   teacher [M, V] fp32 DEVICE, rows compacted like the outputs;   kl [M] fp32 DEVICE
+ * The other arguments are those of mrp_module_step.  Needs a context created with MRP_FLAG_TRAINING_KL (and
+ * without MRP_FLAG_FP8_LM).  Errors: INVALID_ARG, UNSUPPORTED, CUDA.  (The backward pass is outside this library.)
+ */
+int mrp_module_step_kl(mrp_ctx *ctx, const int32_t *tokens, const void *hidden0, float *h_state,
+                       const float *logits0, const float *teacher, const int32_t *row_index, int32_t M, int32_t B,
+                       int32_t L, int32_t first_step, const mrp_draft_out *out, float *kl, void *cuda_stream);
+
+/*
  * The clean prefix of the module's attention (Fig. 1(c): a new block is decoded given the committed clean
  * prefix, under the attention pattern of training, where a block attends to itself and to the clean blocks in
  * front of it).  What a block sees of its prefix are the keys and values the module's own layers produced for

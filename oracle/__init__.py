@@ -267,6 +267,14 @@ def module(hidden, tokens, B, L, emb, w_proj, layers, w_lm, n_attn_heads, mask_t
     return delta_h, delta_l
 
 
+def kl_rows(teacher, logits):
+    """KL(softmax(teacher[m]) || softmax(logits[m])) per row, by the definition of Eq. (3), in float64."""
+    t, l = np.asarray(teacher, np.float64), np.asarray(logits, np.float64)
+    lt = t - (t.max(axis=1, keepdims=True) + np.log(np.exp(t - t.max(axis=1, keepdims=True)).sum(axis=1, keepdims=True)))
+    ll = l - (l.max(axis=1, keepdims=True) + np.log(np.exp(l - l.max(axis=1, keepdims=True)).sum(axis=1, keepdims=True)))
+    return (np.exp(lt) * (lt - ll)).sum(axis=1)
+
+
 def stats(logits):
     """(conf, lse, token, margin) of logit rows [M, V] by the definitions of Sec. 2, in float64."""
     l = np.asarray(logits, np.float64)

@@ -37,7 +37,7 @@ EXPORTS = ("mrp_workspace_bytes", "mrp_create", "mrp_destroy", "mrp_draft", "mrp
            "mrp_profile_enable", "mrp_profile_read", "mrp_last_error",
            "mrp_reveal_remask_noalloc", "mrp_selftest_wait_timeout", "mrp_draft_from_hidden", "mrp_commit",
            "mrp_set_logits0_event", "mrp_set_input_rows", "mrp_fetch_status", "mrp_draft_kl", "mrp_draft_bf16_logits", "mrp_quantised_lm_head",
-           "mrp_module_workspace_bytes", "mrp_module_attach", "mrp_module_step", "mrp_module_set_prefix")
+           "mrp_module_workspace_bytes", "mrp_module_attach", "mrp_module_step", "mrp_module_set_prefix", "mrp_module_step_kl")
 MRP_NOALLOC_MAX_POSITIONS = 65536
 MRP_ERR_CAPACITY = 7
 
@@ -123,6 +123,10 @@ def _load():
     lib.mrp_module_workspace_bytes.argtypes = [ctypes.POINTER(mrp_config), ctypes.POINTER(mrp_module_weights)]
     lib.mrp_module_attach.restype = ctypes.c_int
     lib.mrp_module_attach.argtypes = [ctypes.c_void_p, ctypes.POINTER(mrp_module_weights), ctypes.c_void_p, ctypes.c_size_t]
+    lib.mrp_module_step_kl.restype = ctypes.c_int
+    lib.mrp_module_step_kl.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                                       ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
+                                       ctypes.c_int32, ctypes.POINTER(mrp_draft_out), ctypes.c_void_p, ctypes.c_void_p]
     lib.mrp_module_set_prefix.restype = ctypes.c_int
     lib.mrp_module_set_prefix.argtypes = [ctypes.c_void_p, ctypes.POINTER(mrp_module_kv), ctypes.c_void_p, ctypes.c_int32,
                                           ctypes.c_int32]
@@ -334,6 +338,24 @@ def mrp_module_step(ctx: Context, tokens, hidden0, h_state, logits0, row_index, 
                              int(M), int(B), int(L), int(bool(first_step)), ctypes.byref(out), _stream(stream))
     if rc != 0:
         raise MrpError("mrp_module_step", rc, lib.mrp_last_error(ctx.handle).decode())
+
+
+def mrp_module_step_kl(ctx: Context, tokens, hidden0, h_state, logits0, teacher, row_index, M, B, L, first_step, conf, lse,
+                       token, kl, margin=None, hidden_out=None, status=None, stream=None) -> None:
+    """mrp_module_step with kl[m] = KL(softmax(teacher[m]) || softmax(l[m])) of the step fused into its LM-head pass:
+    ``teacher`` [M, V] fp32, ``kl`` [M] fp32 (context created with MRP_FLAG_TRAINING_KL)."""
+    tdtype = torch.float32 if ctx.cfg.dtype == MRP_F32 else torch.bfloat16
+    for t, dt, nm in ((tokens, torch.int32, "tokens"), (hidden0, tdtype, "hidden0"), (h_state, torch.float32, "h_state"),
+                      (logits0, torch.float32, "logits0"), (teacher, torch.float32, "teacher"), (row_index, torch.int32, "row_index"),
+                      (conf, torch.float32, "conf"), (lse, torch.float32, "lse"), (token, torch.int32, "token"),
+                      (kl, torch.float32, "kl"), (margin, torch.float32, "margin"), (hidden_out, torch.float32, "hidden_out"),
+                      (status, torch.int32, "status")):
+        _check(t, dt, nm)
+    out = mrp_draft_out(_ptr(conf), _ptr(lse), _ptr(token), _ptr(margin), None, _ptr(hidden_out), _ptr(status), None)
+    rc = lib.mrp_module_step_kl(ctx.handle, _ptr(tokens), _ptr(hidden0), _ptr(h_state), _ptr(logits0), _ptr(teacher), _ptr(row_index),
+                                int(M), int(B), int(L), int(bool(first_step)), ctypes.byref(out), _ptr(kl), _stream(stream))
+    if rc != 0:
+        raise MrpError("mrp_module_step_kl", rc, lib.mrp_last_error(ctx.handle).decode())
 
 
 def mrp_module_set_prefix(ctx: Context, caches, prefix_len, append=False) -> None:

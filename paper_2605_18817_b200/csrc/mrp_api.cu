@@ -399,9 +399,9 @@ int mrp_module_set_prefix(mrp_ctx *ctx, const mrp_module_kv *layers, const int32
     return MRP_OK;
 }
 
-int mrp_module_step(mrp_ctx *ctx, const int32_t *tokens, const void *hidden0, float *h_state, const float *logits0,
-                    const int32_t *row_index, int32_t M, int32_t B, int32_t L, int32_t first_step,
-                    const mrp_draft_out *out, void *cuda_stream)
+static int module_call(mrp_ctx *ctx, const int32_t *tokens, const void *hidden0, float *h_state, const float *logits0,
+                       const int32_t *row_index, int32_t M, int32_t B, int32_t L, int32_t first_step,
+                       const mrp_draft_out *out, void *cuda_stream, const float *teacher, float *kl)
 {
     if (!ctx || !out) return MRP_ERR_INVALID_ARG;
     Ctx &c = ctx->c;
@@ -414,14 +414,33 @@ int mrp_module_step(mrp_ctx *ctx, const int32_t *tokens, const void *hidden0, fl
     DeviceGuard guard(c.cfg.device);
     if (guard.err != cudaSuccess) return MRP_ERR_CUDA;
     c.err[0] = 0;
-    c.from_hidden = false; c.final_gamma = nullptr; c.teacher = nullptr; c.kl_out = nullptr; c.l0_bf16 = false;
+    c.from_hidden = false; c.final_gamma = nullptr; c.l0_bf16 = false;
+    c.teacher = M > 0 ? teacher : nullptr; c.kl_out = M > 0 ? kl : nullptr;
     const int saved_rows = c.input_rows;
     c.input_rows = B * L;                       // the dense arrays of this call have B * L rows
     cudaError_t e = module_step(&c, tokens, hidden0, h_state, logits0, row_index, M, B, L, first_step != 0, *out,
                                 (cudaStream_t)cuda_stream);
     c.input_rows = saved_rows;
+    c.teacher = nullptr; c.kl_out = nullptr;
     if (e != cudaSuccess && !c.err[0]) note_err(&c, e, "mrp_module_step");
     return e == cudaSuccess ? MRP_OK : MRP_ERR_CUDA;
+}
+
+int mrp_module_step(mrp_ctx *ctx, const int32_t *tokens, const void *hidden0, float *h_state, const float *logits0,
+                    const int32_t *row_index, int32_t M, int32_t B, int32_t L, int32_t first_step,
+                    const mrp_draft_out *out, void *cuda_stream)
+{
+    return module_call(ctx, tokens, hidden0, h_state, logits0, row_index, M, B, L, first_step, out, cuda_stream, nullptr, nullptr);
+}
+
+int mrp_module_step_kl(mrp_ctx *ctx, const int32_t *tokens, const void *hidden0, float *h_state, const float *logits0,
+                       const float *teacher, const int32_t *row_index, int32_t M, int32_t B, int32_t L, int32_t first_step,
+                       const mrp_draft_out *out, float *kl, void *cuda_stream)
+{
+    if (!ctx) return MRP_ERR_INVALID_ARG;
+    if (!(ctx->c.cfg.flags & MRP_FLAG_TRAINING_KL) || ctx->c.use_fp8_lm) return MRP_ERR_UNSUPPORTED;
+    if ((M > 0 && (!teacher || !kl)) || ((uintptr_t)teacher & 15u)) return MRP_ERR_INVALID_ARG;
+    return module_call(ctx, tokens, hidden0, h_state, logits0, row_index, M, B, L, first_step, out, cuda_stream, teacher, kl);
 }
 
 int mrp_quantised_lm_head(mrp_ctx *ctx, const uint8_t **codes, const float **scales)

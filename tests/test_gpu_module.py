@@ -177,3 +177,81 @@ def test_module_step_at_the_benchmark_shapes(which, L, blocks_checked):
     binding.mrp_destroy(ctx)
     del ctx, w_lm, heads_dev, hid0, l0
     torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("dtype,flags,d,F,V,D,heads,B,L", [
+    ("f32", 0, 64, 96, 512, 2, 4, 2, 4),                                 # CUDA-core kernels
+    ("bf16", binding.MRP_FLAG_FORCE_SIMT, 64, 96, 512, 1, 2, 1, 4),     # ... the step as one cooperative kernel
+    ("bf16", 0, 256, 512, 4096, 3, 4, 1, 4),                            # one tensor-core kernel per step, row-major KL LM head
+    ("bf16", 0, 256, 512, 4096, 2, 4, 3, 16),                           # 48 positions
+    ("bf16", 0, 128, 256, 2048, 2, 4, 5, 32),                           # 160 positions: row-major products
+])
+def test_module_step_with_the_training_objective(dtype, flags, d, F, V, D, heads, B, L):
+    """mrp_module_step_kl: kl[m] = KL(softmax(teacher[m]) || softmax(l[m])) of the step (Eq. (3); Algorithm 1 trains the
+    module with it) against the definition on the oracle's logits, over two unrolled steps; the ordinary outputs stay
+    those of mrp_module_step."""
+    w = synth.make_weights(d, F, V, 1, dtype, 61)
+    mw = synth.make_module_weights(d, F, V, D, heads, dtype, 61, std=0.06, proj_std=0.3 / np.sqrt(2 * d))
+    inp = synth.make_inputs(w, B, L, 61, 1.0, 3.0)
+    n = B * L
+    heads_dev, w_lm = harness.upload_weights(w, DEV)
+    ctx = binding.mrp_create(d, F, V, heads_dev, w_lm, max_rows=n, max_seqs=B, block_len=L,
+                             flags=flags | binding.MRP_FLAG_TRAINING_KL)
+    emb, w_proj, layers = upload_module(mw, dtype)
+    binding.mrp_module_attach(ctx, emb, w_proj, layers, heads, mw.mask_token)
+    hid0 = harness.to_device(inp.hidden, dtype, DEV)
+    l0 = torch.from_numpy(inp.logits0).to(DEV)
+    h_state = torch.empty((n, d), device=DEV, dtype=torch.float32)
+    rng = np.random.default_rng(5)
+    tokens = np.full(n, -1, np.int32)
+    tokens[::L] = rng.integers(0, V - 1, B)
+    h_run = inp.hidden.astype(np.float64)
+    l_run = inp.logits0.astype(np.float64)
+    tol = TOL[dtype] if dtype == "bf16" else 5e-5
+    for s in range(2):
+        ri = np.flatnonzero(tokens < 0).astype(np.int32)
+        M = ri.size
+        dh, dl = oracle.module(h_run.astype(np.float32), tokens, B, L, mw.emb, mw.w_proj, mw.layers, w.w_lm, heads, mw.mask_token,
+                               row_index=ri)
+        h_run = h_run.astype(np.float32).astype(np.float64) + dh
+        l_run[ri] += dl
+        scale = rng.uniform(0.02, 0.6, size=(M, 1))
+        teacher = (l_run[ri] + scale * rng.standard_normal((M, V))).astype(np.float32)
+        kl_ref = oracle.kl_rows(teacher, l_run[ri])
+        out = harness.alloc_draft_out(M, 1, V, d, DEV, hidden=True)
+        kl = torch.full((M,), -1.0, device=DEV)
+        binding.mrp_module_step_kl(ctx, torch.from_numpy(tokens).to(DEV), hid0, h_state, l0, torch.from_numpy(teacher).to(DEV),
+                                   torch.from_numpy(ri).to(DEV), M, B, L, s == 0, out.conf, out.lse, out.token, kl,
+                                   margin=out.margin, hidden_out=out.hidden, status=out.status)
+        torch.cuda.synchronize()
+        assert int(out.status.item()) == 0
+        conf, lse, tok, margin = oracle.stats(l_run[ri])
+        assert np.abs(h_state.cpu().numpy() - h_run).max() <= 1e-3 * max(1.0, np.abs(h_run).max())
+        assert np.abs(out.conf[1].cpu().numpy() - conf).max() <= tol and np.abs(out.lse[1].cpu().numpy() - lse).max() <= tol
+        clear = margin > 1e-2
+        assert np.array_equal(out.token[1].cpu().numpy()[clear], tok[clear])
+        got = kl.cpu().numpy().astype(np.float64)
+        assert kl_ref.min() > 0 and kl_ref.max() > 1e-2
+        assert np.all(np.abs(got - kl_ref) <= tol + 2e-3 * kl_ref), np.abs(got - kl_ref).max()
+        for b in range(B):                                   # reveal a position per block for the next unrolled step
+            rows = [m for m in range(M) if ri[m] // L == b]
+            if rows:
+                tokens[ri[rows[0]]] = int(rng.integers(0, V - 1))
+    # nothing of the KL call lingers: the plain step runs on the same context afterwards
+    h2 = torch.empty_like(h_state)
+    ri_d = torch.from_numpy(np.flatnonzero(tokens < 0).astype(np.int32)).to(DEV)
+    M2 = int(ri_d.numel())
+    out3 = harness.alloc_draft_out(M2, 1, V, d, DEV)
+    binding.mrp_module_step(ctx, torch.from_numpy(tokens).to(DEV), hid0, h2, l0, ri_d, M2, B, L, True, out3.conf, out3.lse,
+                            out3.token, status=out3.status)
+    torch.cuda.synchronize()
+    assert int(out3.status.item()) == 0
+    binding.mrp_destroy(ctx)
+    # a context without the flag has no room for the partial sums
+    ctx = binding.mrp_create(d, F, V, heads_dev, w_lm, max_rows=n, max_seqs=B, block_len=L, flags=flags)
+    binding.mrp_module_attach(ctx, emb, w_proj, layers, heads, mw.mask_token)
+    with pytest.raises(binding.MrpError) as ei:
+        binding.mrp_module_step_kl(ctx, torch.from_numpy(tokens).to(DEV), hid0, h2, l0, torch.from_numpy(teacher).to(DEV), ri_d, M2,
+                                   B, L, True, out3.conf, out3.lse, out3.token, kl)
+    assert ei.value.status == 2
+    binding.mrp_destroy(ctx)

@@ -236,3 +236,27 @@ def test_prefix_matches_library_implementation():
         g = n @ lay["w_gate"].astype(np.float64).T
         z = z + (g * expit(g) * (n @ lay["w_up"].astype(np.float64).T)) @ lay["w_down"].astype(np.float64).T
     assert np.allclose(got, z, rtol=0, atol=1e-11)
+
+
+def test_kl_rows_agrees_with_the_chain_objective_and_closed_forms():
+    # the numpy objective used for the module against the C objective of the head chain (itself pinned against a
+    # library relative entropy and a closed form): with a zero down projection l_1 = l_0, so both see the same rows
+    from scipy.special import rel_entr
+    rng = np.random.default_rng(6)
+    d, F, V, M = 8, 12, 30, 5
+    w = synth.make_weights(d, F, V, 1, "f32", 3)
+    w.heads[0]["w_down"][:] = 0
+    hidden = rng.standard_normal((M, d)).astype(np.float32)
+    l0 = (rng.standard_normal((M, V)) * 2).astype(np.float32)
+    teacher = (l0 + rng.standard_normal((M, V))).astype(np.float32)
+    _, kl_c = oracle.draft_kl(hidden, l0, teacher[None], w.heads, w.w_lm)
+    got = oracle.kl_rows(teacher, l0)
+    assert np.all(got > 0) and np.allclose(got, kl_c[0], rtol=1e-12, atol=1e-14)
+    assert np.allclose(got, rel_entr(softmax(teacher.astype(np.float64), axis=1), softmax(l0.astype(np.float64), axis=1)).sum(axis=1),
+                       rtol=1e-10, atol=1e-13)
+    assert np.abs(oracle.kl_rows(l0, l0 + 3.5)).max() < 1e-12           # shift invariance, equal distributions
+    # two tokens: p = sigmoid(a), q = sigmoid(b)
+    a, b = 0.7, -0.4
+    p, q = expit(a), expit(b)
+    want = p * np.log(p / q) + (1 - p) * np.log((1 - p) / (1 - q))
+    assert abs(oracle.kl_rows([[a, 0.0]], [[b, 0.0]])[0] - want) < 1e-14
