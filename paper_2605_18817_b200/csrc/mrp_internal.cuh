@@ -262,7 +262,7 @@ cudaError_t sk_linear3(Ctx *c, const __nv_bfloat16 *a, int n, int n_in, const vo
 cudaError_t sk_gate_up(Ctx *c, const __nv_bfloat16 *a, int n, int n_in, const void *w_gate, const void *w_up, int F,
                        const float *sumsq, int n_ss, __nv_bfloat16 *act, int32_t *user_status, cudaStream_t st);
 // One module step as one cooperative kernel (see tc_chain.cu); bar_mem: kModChainBarInts zero-able ints.
-constexpr int kModChainBarInts = 23 * 448 + 1;
+constexpr int kModChainBarInts = 22 * 448 + 1;
 cudaError_t sk_module_step(Ctx *c, int n, int L, const int32_t *tokens, const void *hidden0, float *h_state, bool first_step,
                            __nv_bfloat16 *cat16, __nv_bfloat16 *xa, __nv_bfloat16 *xb, __nv_bfloat16 *act16, float *q, float *k,
                            float *v, float *z, int32_t *bar_mem, const int32_t *row_index, int n_masked, int lo_xt, bool f16_lm,

@@ -42,10 +42,10 @@ constexpr int kChTilesPerPhase = 448;      // arrival counters per phase
 constexpr int kChMaxPhases = 8;
 constexpr long long kBarrierCycles = 1000000000LL;   // bound on a grid-barrier wait (about 0.5 s)
 
-enum { CH_GU = 0, CH_DN = 1, CH_LIN = 2, CH_ATT = 3, CH_CAT = 4, CH_FIN = 5 };   // from LIN on: the module's phases (MOD instantiations)
+enum { CH_GU = 0, CH_DN = 1, CH_LIN = 2, CH_ATT = 3, CH_CAT = 4 };   // from LIN on: the module's phases (MOD instantiations)
 
 constexpr int kModChainLayers = 4;     // module layers one launch can hold
-constexpr int kModChainPhases = 3 + 5 * kModChainLayers;   // fusion + projection, five per layer, the closing phase
+constexpr int kModChainPhases = 2 + 5 * kModChainLayers;   // fusion rows + projection, five per layer
 template <int NM>
 struct ChainMapsT {
     CUtensorMap m[NM];
@@ -79,10 +79,11 @@ struct ChainPhase {
     int att_L, att_H;
     __nv_bfloat16 *att_pk, *att_pv;  // the layer's clean-prefix cache [*, pcap, d] (nullptr: block-local attention)
     int zero_slot0, zero_slot1;      // ssq_fix slots this phase clears for later phases of the launch (< 0: none)
+    int fin;                         // LIN that completes Delta: its finish also does h <- h + Delta and the LM-head operand
 };
 
-// What the module's first (CAT: the rows [h ; emb[x]] in operand form) and last phase (FIN: h <- h + Delta and the
-// LM-head operand of the masked rows) need.
+// What the module's first phase (CAT: the rows [h ; emb[x]] in operand form) and the finish of its last product
+// (h <- h + Delta and the LM-head operand of the masked rows) need.
 struct ModEnds {
     const int32_t *tokens;
     const __nv_bfloat16 *hidden0, *emb;
@@ -369,6 +370,16 @@ sk_chain_kernel(const __grid_constant__ typename ChainTypes<MOD>::Maps maps,
         const int n_ch = (p.M + 15) >> 4;
         int n_acc = 0;
         bool alive = true;
+        // row m of the LM-head operand: zero rows of step 0, then h - h_0 (hi + lo; fp16 copy where that LM head runs)
+        auto fin_put = [&](int m, int j, float h, float r) {
+            const ModEnds &e = p.mod;
+            const size_t o = (size_t)m * p.d + j;
+            if (e.hidden_out) e.hidden_out[o] = h;
+            e.xt[o] = __float2bfloat16(0.f);
+            e.xt[(size_t)p.lo_xt * p.d + o] = __float2bfloat16(0.f);
+            ch_store_hi_lo(e.xt + (size_t)e.n_masked * p.d + o, (size_t)p.lo_xt * p.d, r);
+            if (e.xt16) e.xt16[o] = __float2half_rn(r);
+        };
         pdl_wait();
         for (int i = 0; i < p.n_phases && alive; ++i) {
             const ChainPhase &ph = p.ph[i];
@@ -380,6 +391,25 @@ sk_chain_kernel(const __grid_constant__ typename ChainTypes<MOD>::Maps maps,
             }
             ch_epi_sync();
             if (*vote_s == 1) { alive = false; break; }
+            if (MOD && ph.fin) {
+                // the product that completes Delta: dense position -> masked row (or -1), for its finish below
+                // (the buffer of squares is free: no norm follows this product)
+                const ModEnds &e = p.mod;
+                int *inv = reinterpret_cast<int *>(sq_s);
+                for (int i2 = t; i2 < p.M; i2 += 128) inv[i2] = -1;
+                ch_epi_sync();
+                if (t == 0) {
+                    for (int m = 0; m < e.n_masked; ++m) {
+                        const int idx = e.row_index ? e.row_index[m] : m;
+                        if (row_ok(idx, p.M)) inv[idx] = m;
+                        else if (cta == 0) {
+                            atomicOr(p.status, MRP_DEV_BAD_INDEX);
+                            if (p.user_status) atomicOr(p.user_status, MRP_DEV_BAD_INDEX);
+                        }
+                    }
+                }
+                ch_epi_sync();
+            }
             int tile, kc0, nk;
             const bool active = share(i, tile, kc0, nk);
             if (active) {
@@ -566,6 +596,14 @@ sk_chain_kernel(const __grid_constant__ typename ChainTypes<MOD>::Maps maps,
                                 if (ph.lin_acc) h += __ldcg(dst + o);
                                 dst[o] = h;
                                 sq = h * h;
+                                if (ph.fin) {
+                                    // Delta is complete here: h <- h + Delta, and the LM-head operand of a masked position
+                                    const ModEnds &en = p.mod;
+                                    const int *inv = reinterpret_cast<const int *>(sq_s);
+                                    const float hs = __ldcg(en.h_state + o) + h;
+                                    en.h_state[o] = hs;
+                                    if (inv[m] >= 0) fin_put(inv[m], j, hs, hs - __bfloat162float(en.hidden0[o]));
+                                }
                                 if (ph.xg_next) ch_store_hi_lo(ph.xg_next + o, (size_t)p.lo_x * ph.w_rows, h * __bfloat162float(ph.gamma_next[j]));
                             }
                             if (ph.xg_next) sq_s[e] = sq;        // (a share without a norm behind it may exceed the buffer)
@@ -698,42 +736,14 @@ sk_chain_kernel(const __grid_constant__ typename ChainTypes<MOD>::Maps maps,
                         e.cat[((size_t)p.lo_x + pos) * d2 + p.d + j] = __float2bfloat16(0.f);
                     }
                 }
-                if (ph.kind == CH_FIN) {
-                    // h <- h + Delta at every position; the LM-head operand h - h_0 of the masked rows behind the zero
-                    // rows of step 0 (a row index out of range: zero rows, and the bit)
+                if (ph.kind == CH_LIN && ph.fin) {
+                    // masked rows whose index is out of range, or names a position that a later row names too: zero rows
                     const ModEnds &e = p.mod;
-                    int *inv = reinterpret_cast<int *>(sq_s);          // dense position -> masked row, or -1
-                    for (int i2 = t; i2 < p.M; i2 += 128) inv[i2] = -1;
-                    ch_epi_sync();
-                    if (t == 0) {
-                        for (int m = 0; m < e.n_masked; ++m) {
-                            const int idx = e.row_index ? e.row_index[m] : m;
-                            if (row_ok(idx, p.M)) inv[idx] = m;
-                            else if (cta == 0) {
-                                atomicOr(p.status, MRP_DEV_BAD_INDEX);
-                                if (p.user_status) atomicOr(p.user_status, MRP_DEV_BAD_INDEX);
-                            }
-                        }
-                    }
-                    ch_epi_sync();
-                    auto put = [&](int m, int j, float h, float r) {
-                        const size_t o = (size_t)m * p.d + j;
-                        if (e.hidden_out) e.hidden_out[o] = h;
-                        e.xt[o] = __float2bfloat16(0.f);
-                        e.xt[(size_t)p.lo_xt * p.d + o] = __float2bfloat16(0.f);
-                        ch_store_hi_lo(e.xt + (size_t)e.n_masked * p.d + o, (size_t)p.lo_xt * p.d, r);
-                        if (e.xt16) e.xt16[o] = __float2half_rn(r);
-                    };
-                    for (int idx = cta * 128 + t; idx < p.M * p.d; idx += G * 128) {
-                        const int pos = idx / p.d, j = idx - pos * p.d;
-                        const float h = __ldcg(e.h_state + idx) + __ldcg(e.z + idx);
-                        e.h_state[idx] = h;
-                        if (inv[pos] >= 0) put(inv[pos], j, h, h - __bfloat162float(e.hidden0[idx]));
-                    }
+                    const int *inv = reinterpret_cast<const int *>(sq_s);
                     for (int m = 0; m < e.n_masked; ++m) {
                         const int idx = e.row_index ? e.row_index[m] : m;
                         if (!row_ok(idx, p.M) || inv[idx] != m)
-                            for (int j = cta * 128 + t; j < p.d; j += G * 128) put(m, j, 0.f, 0.f);
+                            for (int j = cta * 128 + t; j < p.d; j += G * 128) fin_put(m, j, 0.f, 0.f);
                     }
                 }
                 if (ph.kind == CH_ATT && ph.att_pk) {
@@ -1139,9 +1149,9 @@ cudaError_t sk_module_step(Ctx *c, int n, int L, const int32_t *tokens, const vo
             const void *g_next = l + 1 < D ? w.layers[l + 1].g_attn : nullptr;
             ph.lin_out = z; ph.lin_acc = 1;
             ph.gamma_next = (const __nv_bfloat16 *)g_next; ph.xg_next = g_next ? xa : nullptr; ph.ssq_idx = s_next;
+            ph.fin = l + 1 == D ? 1 : 0;       // Delta complete: h <- h + Delta and the LM-head operand in the same finish
         }
     }
-    plain(CH_FIN);
     p.n_phases = i;
     // arrival counters, the grid barrier and the first slot of the sums of squares start at zero
     cudaError_t e = cudaMemsetAsync(bar_mem, 0, ((size_t)kModChainPhases * kChTilesPerPhase + 1) * 4, st);
