@@ -513,22 +513,78 @@ __device__ __forceinline__ void att_group(const float *q_s, const T *krow0, cons
     }
 }
 
+// The chunks of a (block, head) meet: every CTA arrives at the pair's counter once its partial results are written;
+// the CTA that arrives last merges them (a warp per query) and leaves the counter at zero.  No CTA waits.
+template <typename Sync, typename Out>
+__device__ __forceinline__ void att_arrive_merge(int n_ch, int L, int dh, float *part, int *counter, float *sh, int warp, int lane,
+                                                 Sync sync, Out out)
+{
+    const int t = warp * 32 + lane, stride = dh + 2;
+    {
+        // arrive at the (block, head) counter; the CTA that arrives last merges the chunks and leaves the counter at zero
+        int *flag = reinterpret_cast<int *>(sh);
+        __threadfence();
+        sync();
+        if (t == 0) {
+            const int old = atomicAdd(counter, 1);
+            *flag = old == n_ch - 1;
+            if (old == n_ch - 1) {
+                __threadfence();
+                *counter = 0;
+            }
+        }
+        sync();
+        const bool last = *flag != 0;
+        sync();
+        if (last) {
+            // a warp per query: lanes over the chunks for the weights, then over the features, the partial results of
+            // all chunks in flight together
+            for (int i = warp; i < L; i += 4) {
+                const float m = lane < n_ch ? __ldcg(part + ((size_t)lane * L + i) * stride) : -INFINITY;
+                const float sm = lane < n_ch ? __ldcg(part + ((size_t)lane * L + i) * stride + 1) : 0.f;
+                float top = m;
+#pragma unroll
+                for (int w = 16; w > 0; w >>= 1) top = fmaxf(top, __shfl_xor_sync(0xffffffffu, top, w));
+                const float e = m == -INFINITY ? 0.f : expf(m - top);
+                float tot = sm * e;
+#pragma unroll
+                for (int w = 16; w > 0; w >>= 1) tot += __shfl_xor_sync(0xffffffffu, tot, w);
+                float o[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) o[u] = 0.f;
+#pragma unroll 4
+                for (int x = 0; x < n_ch; ++x) {
+                    const float ex = __shfl_sync(0xffffffffu, e, x);
+                    const float *src = part + ((size_t)x * L + i) * stride + 2;
+#pragma unroll
+                    for (int u = 0; u < 8; ++u)
+                        if (lane + 32 * u < dh) o[u] = fmaf(__ldcg(src + lane + 32 * u), ex, o[u]);
+                }
+#pragma unroll
+                for (int u = 0; u < 8; ++u)
+                    if (lane + 32 * u < dh) out(i, lane + 32 * u, o[u] / tot);
+            }
+        }
+    }
+}
+
 template <int PER, typename T, typename Sync, typename Out>
 __device__ __forceinline__ void att_unit_per(const float *q, const T *pk, const T *pv, int P, const float *kb, const float *vb, int L,
-                                             int d, int dh, int ch, int n_ch, int gpc, float *part, int *counter, float *sh, int warp,
-                                             int lane, Sync sync, Out out)
+                                             int d, int dh, int g_lo, int g_hi, int ch, int n_ch, float *part, int *counter, float *sh,
+                                             int warp, int lane, Sync sync, Out out)
 {
+    // (groups [g_lo, g_hi) of the sequence's prefix groups followed by its block groups; ch: the slot of the partial results)
     constexpr int NU = PER > 0 ? PER : 8;
     float *q_s = sh, *part_s = sh + kAttQT * dh;              // part_s[w][qi]: maximum, sum, o[dh]
     const int t = warp * 32 + lane, stride = dh + 2;
     const float scale = rsqrtf((float)dh);
     const bool vec = (dh % 8) == 0 && (d % 8) == 0;
     const int gp = (P + 31) / 32, gb = (L + 31) / 32;
-    const int g_end = (ch + 1) * gpc < gp + gb ? (ch + 1) * gpc : gp + gb;
+    const int g_end = g_hi < gp + gb ? g_hi : gp + gb;
     auto feat = [&](int u) { return PER > 0 ? lane * PER + u : lane + 32 * u; };
     // The prefix rows this warp will read, asked into L2 up front: each lane reads whole rows of its own in the score
     // loops, a handful of loads at a time, and would otherwise pay the DRAM latency once per handful.
-    for (int g = ch * gpc + warp; g < g_end && g < gp; g += 4) {
+    for (int g = g_lo + warp; g < g_end && g < gp; g += 4) {
         const int j = g * 32 + lane;
         if (j < P) {
             const char *rk = reinterpret_cast<const char *>(pk + (size_t)j * d), *rv = reinterpret_cast<const char *>(pv + (size_t)j * d);
@@ -553,7 +609,7 @@ __device__ __forceinline__ void att_unit_per(const float *q, const T *pk, const 
 #pragma unroll
             for (int u = 0; u < 8; ++u) oacc[qi][u] = 0.f;
         }
-        for (int g = ch * gpc + warp; g < g_end; g += 4) {
+        for (int g = g_lo + warp; g < g_end; g += 4) {
             if (g < gp) {
                 const int j0 = g * 32, left = P - j0;
                 att_group<PER, false>(q_s, pk + (size_t)j0 * d, pv + (size_t)j0 * d, left < 32 ? left : 32, d, dh, vec, scale, lane, mx, sum,
@@ -605,66 +661,276 @@ __device__ __forceinline__ void att_unit_per(const float *q, const T *pk, const 
         }
         sync();                                               // sh is free again
     }
-    if (n_ch > 1) {
-        // arrive at the (block, head) counter; the CTA that arrives last merges the chunks and leaves the counter at zero
-        int *flag = reinterpret_cast<int *>(sh);
-        __threadfence();
-        sync();
-        if (t == 0) {
-            const int old = atomicAdd(counter, 1);
-            *flag = old == n_ch - 1;
-            if (old == n_ch - 1) {
-                __threadfence();
-                *counter = 0;
-            }
+    if (n_ch > 1) att_arrive_merge(n_ch, L, dh, part, counter, sh, warp, lane, sync, out);
+}
+
+// ---- the prefix part on tensor cores ------------------------------------------------------------------------
+// For bf16 caches and heads of 64 or 128 features the prefix groups of a chunk run as small matrix products
+// (mma.sync m16n8k16, bf16 operands, fp32 accumulation): S = Q K^T over 16 queries x 32 keys per group, online softmax on
+// the accumulator fragments, O += P V.  Queries and probabilities enter as bf16 hi + lo pairs (two products each), keys
+// and values are the cache's own bf16.  The contraction index of S runs over features in an order that lets every
+// lane fetch 16 bytes of a key row at once (A and B use the same order, so the sum is the same); the value rows are
+// fetched the same way and turned with movmatrix, which leaves each lane with eight consecutive features of two
+// queries.  Only cache rows pass through here: the block's own fp32 keys and values are a chunk of their own on the
+// CUDA-core routine above, and the chunks always meet through att_arrive_merge.
+__device__ __forceinline__ void att_mma16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1)
+{
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t att_movm(uint32_t a)
+{
+    uint32_t d;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+    return d;
+}
+// (x, y) as a bf16 pair, x in the low half; and the pair of what that rounding left over
+__device__ __forceinline__ void att_split2(float x, float y, uint32_t &hi, uint32_t &lo)
+{
+    const __nv_bfloat162 h = __floats2bfloat162_rn(x, y);
+    const float2 hf = __bfloat1622float2(h);
+    const __nv_bfloat162 l = __floats2bfloat162_rn(x - hf.x, y - hf.y);
+    hi = *reinterpret_cast<const uint32_t *>(&h);
+    lo = *reinterpret_cast<const uint32_t *>(&l);
+}
+__device__ __forceinline__ uint32_t att_comp(const uint4 &v, int i) { return i == 0 ? v.x : i == 1 ? v.y : i == 2 ? v.z : v.w; }
+
+// shared floats the tensor-core unit needs: 16 staged queries as bf16 hi + lo rows (padded), or the merge area
+__host__ __device__ constexpr int att_mma_sh_floats(int dh)
+{
+    return (2 * 16 * (dh + 8)) / 2 > 4 * 4 * (dh + 2) ? (2 * 16 * (dh + 8)) / 2 : 4 * 4 * (dh + 2);
+}
+
+template <int NG, typename Sync>
+__device__ __forceinline__ void att_unit_mma(const float *q, const __nv_bfloat16 *pk, const __nv_bfloat16 *pv, int P, int L, int d, int g_lo,
+                                             int g_hi, float *part_slot, float *sh, int warp, int lane, Sync sync)
+{
+    constexpr int DH = 32 * NG, QS = DH + 8, stride = DH + 2;
+    __nv_bfloat16 *q_hi = reinterpret_cast<__nv_bfloat16 *>(sh), *q_lo = q_hi + 16 * QS;
+    float *part_s = sh;                                   // [4 warps][4 queries][DH + 2], once the queries are done with
+    const int t = warp * 32 + lane, r = lane >> 2, j = lane & 3;
+    const float scale = rsqrtf((float)DH);
+    const int gp = (P + 31) / 32;
+    if (g_hi > gp) g_hi = gp;
+    for (int q0 = 0; q0 < L; q0 += 16) {
+        const int nq = L - q0 < 16 ? L - q0 : 16;
+        for (int x = t; x < 16 * DH; x += 128) {
+            const int qi = x / DH, c = x - qi * DH;
+            const float v = qi < nq ? __ldcg(q + (size_t)(q0 + qi) * d + c) : 0.f;
+            const __nv_bfloat16 h = __float2bfloat16_rn(v);
+            q_hi[qi * QS + c] = h;
+            q_lo[qi * QS + c] = __float2bfloat16_rn(v - __bfloat162float(h));
         }
         sync();
-        const bool last = *flag != 0;
-        sync();
-        if (last) {
-            // a warp per query: lanes over the chunks for the weights, then over the features, the partial results of
-            // all chunks in flight together
-            for (int i = warp; i < L; i += 4) {
-                const float m = lane < n_ch ? __ldcg(part + ((size_t)lane * L + i) * stride) : -INFINITY;
-                const float sm = lane < n_ch ? __ldcg(part + ((size_t)lane * L + i) * stride + 1) : 0.f;
-                float top = m;
+        float o[NG][4][4];
 #pragma unroll
-                for (int w = 16; w > 0; w >>= 1) top = fmaxf(top, __shfl_xor_sync(0xffffffffu, top, w));
-                const float e = m == -INFINITY ? 0.f : expf(m - top);
-                float tot = sm * e;
+        for (int a = 0; a < NG; ++a)
 #pragma unroll
-                for (int w = 16; w > 0; w >>= 1) tot += __shfl_xor_sync(0xffffffffu, tot, w);
-                float o[8];
+            for (int b = 0; b < 4; ++b)
 #pragma unroll
-                for (int u = 0; u < 8; ++u) o[u] = 0.f;
-#pragma unroll 4
-                for (int x = 0; x < n_ch; ++x) {
-                    const float ex = __shfl_sync(0xffffffffu, e, x);
-                    const float *src = part + ((size_t)x * L + i) * stride + 2;
+                for (int c = 0; c < 4; ++c) o[a][b][c] = 0.f;
+        float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;      // rows r and r + 8 of the tile
+        for (int g = g_lo + warp; g < g_hi; g += 4) {
+            const int j0 = g * 32, left = P - j0, cnt = left < 32 ? left : 32;
+            // ---- S = Q K^T: four tiles of 8 keys; a key index beyond the group reads the group's last row (masked below)
+            float sacc[4][4];
 #pragma unroll
-                    for (int u = 0; u < 8; ++u)
-                        if (lane + 32 * u < dh) o[u] = fmaf(__ldcg(src + lane + 32 * u), ex, o[u]);
+            for (int a = 0; a < 4; ++a)
+#pragma unroll
+                for (int b = 0; b < 4; ++b) sacc[a][b] = 0.f;
+#pragma unroll
+            for (int s = 0; s < NG; ++s) {
+                uint4 kk[4];
+#pragma unroll
+                for (int tt = 0; tt < 4; ++tt) {
+                    const int key = 8 * tt + r < cnt ? 8 * tt + r : cnt - 1;
+                    kk[tt] = __ldg(reinterpret_cast<const uint4 *>(pk + (size_t)(j0 + key) * d + 32 * s + 8 * j));
+                }
+                const uint4 ah0 = *reinterpret_cast<const uint4 *>(q_hi + r * QS + 32 * s + 8 * j);
+                const uint4 ah1 = *reinterpret_cast<const uint4 *>(q_hi + (r + 8) * QS + 32 * s + 8 * j);
+                const uint4 al0 = *reinterpret_cast<const uint4 *>(q_lo + r * QS + 32 * s + 8 * j);
+                const uint4 al1 = *reinterpret_cast<const uint4 *>(q_lo + (r + 8) * QS + 32 * s + 8 * j);
+#pragma unroll
+                for (int tt = 0; tt < 4; ++tt) {
+                    att_mma16816(sacc[tt], ah0.x, ah1.x, ah0.y, ah1.y, kk[tt].x, kk[tt].y);
+                    att_mma16816(sacc[tt], al0.x, al1.x, al0.y, al1.y, kk[tt].x, kk[tt].y);
+                    att_mma16816(sacc[tt], ah0.z, ah1.z, ah0.w, ah1.w, kk[tt].z, kk[tt].w);
+                    att_mma16816(sacc[tt], al0.z, al1.z, al0.w, al1.w, kk[tt].z, kk[tt].w);
+                }
+            }
+            // ---- online softmax on the fragments: [0], [1] belong to row r, [2], [3] to row r + 8; columns = keys 8 tt + 2 j + e
+            float g0 = -INFINITY, g1 = -INFINITY;
+#pragma unroll
+            for (int tt = 0; tt < 4; ++tt)
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    const bool in = 8 * tt + 2 * j + e < cnt;
+                    sacc[tt][e] = in ? sacc[tt][e] * scale : -INFINITY;
+                    sacc[tt][2 + e] = in ? sacc[tt][2 + e] * scale : -INFINITY;
+                    g0 = fmaxf(g0, sacc[tt][e]);
+                    g1 = fmaxf(g1, sacc[tt][2 + e]);
+                }
+            g0 = fmaxf(g0, __shfl_xor_sync(0xffffffffu, g0, 1));
+            g0 = fmaxf(g0, __shfl_xor_sync(0xffffffffu, g0, 2));
+            g1 = fmaxf(g1, __shfl_xor_sync(0xffffffffu, g1, 1));
+            g1 = fmaxf(g1, __shfl_xor_sync(0xffffffffu, g1, 2));
+            const float n0 = fmaxf(m0, g0), n1 = fmaxf(m1, g1);          // finite: the group has a key
+            const float c0 = expf(m0 - n0), c1 = expf(m1 - n1);          // (first group: exp(-inf) = 0)
+            float ps0 = 0.f, ps1 = 0.f;
+#pragma unroll
+            for (int tt = 0; tt < 4; ++tt)
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    sacc[tt][e] = expf(sacc[tt][e] - n0);                // a masked key: exp(-inf) = 0
+                    sacc[tt][2 + e] = expf(sacc[tt][2 + e] - n1);
+                    ps0 += sacc[tt][e];
+                    ps1 += sacc[tt][2 + e];
+                }
+            l0 = l0 * c0 + ps0;                                          // (the lane's share of the row sums)
+            l1 = l1 * c1 + ps1;
+            m0 = n0;
+            m1 = n1;
+#pragma unroll
+            for (int a = 0; a < NG; ++a)
+#pragma unroll
+                for (int b = 0; b < 4; ++b) {
+                    o[a][b][0] *= c0; o[a][b][1] *= c0;
+                    o[a][b][2] *= c1; o[a][b][3] *= c1;
+                }
+            // ---- O += P V: two steps of 16 keys; the probabilities as A fragments (hi + lo), the values turned by movmatrix
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+                uint32_t ph[4], pl[4];
+                att_split2(sacc[2 * u][0], sacc[2 * u][1], ph[0], pl[0]);
+                att_split2(sacc[2 * u][2], sacc[2 * u][3], ph[1], pl[1]);
+                att_split2(sacc[2 * u + 1][0], sacc[2 * u + 1][1], ph[2], pl[2]);
+                att_split2(sacc[2 * u + 1][2], sacc[2 * u + 1][3], ph[3], pl[3]);
+                const int k0 = 16 * u + r < cnt ? 16 * u + r : cnt - 1, k1 = 16 * u + 8 + r < cnt ? 16 * u + 8 + r : cnt - 1;
+                uint4 va[NG], vb[NG];
+#pragma unroll
+                for (int a = 0; a < NG; ++a) {
+                    va[a] = __ldg(reinterpret_cast<const uint4 *>(pv + (size_t)(j0 + k0) * d + 32 * a + 8 * j));
+                    vb[a] = __ldg(reinterpret_cast<const uint4 *>(pv + (size_t)(j0 + k1) * d + 32 * a + 8 * j));
                 }
 #pragma unroll
-                for (int u = 0; u < 8; ++u)
-                    if (lane + 32 * u < dh) out(i, lane + 32 * u, o[u] / tot);
+                for (int a = 0; a < NG; ++a)
+#pragma unroll
+                    for (int b = 0; b < 4; ++b) {
+                        const uint32_t b0 = att_movm(att_comp(va[a], b)), b1 = att_movm(att_comp(vb[a], b));
+                        att_mma16816(o[a][b], ph[0], ph[1], ph[2], ph[3], b0, b1);
+                        att_mma16816(o[a][b], pl[0], pl[1], pl[2], pl[3], b0, b1);
+                    }
+            }
+        }
+        l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
+        l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
+        l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
+        l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
+        sync();                                              // the staged queries are done with: the merge area takes their place
+        // the four warps' results, four queries at a time: rows 4 sub .. 4 sub + 3 sit in the lanes with r in
+        // [4 (sub & 1), + 4), in fragment entries [0], [1] (sub < 2) or [2], [3]
+#pragma unroll
+        for (int sub = 0; sub < 4; ++sub) {
+            if (4 * sub < nq) {
+                const int rr = r - 4 * (sub & 1);
+                if (rr >= 0 && rr < 4) {
+                    float *mine = part_s + (size_t)(warp * 4 + rr) * stride;
+                    if (j == 0) {
+                        mine[0] = sub < 2 ? m0 : m1;
+                        mine[1] = sub < 2 ? l0 : l1;
+                    }
+#pragma unroll
+                    for (int a = 0; a < NG; ++a)
+#pragma unroll
+                        for (int b = 0; b < 4; ++b) {
+                            mine[2 + 32 * a + 8 * j + 2 * b] = o[a][b][sub < 2 ? 0 : 2];
+                            mine[2 + 32 * a + 8 * j + 2 * b + 1] = o[a][b][sub < 2 ? 1 : 3];
+                        }
+                }
+                sync();
+                for (int qi = 0; qi < 4 && 4 * sub + qi < nq; ++qi) {
+                    float top = -INFINITY, e[4], tot = 0.f;
+#pragma unroll
+                    for (int w = 0; w < 4; ++w) top = fmaxf(top, part_s[(size_t)(w * 4 + qi) * stride]);
+#pragma unroll
+                    for (int w = 0; w < 4; ++w) {
+                        const float m = part_s[(size_t)(w * 4 + qi) * stride];
+                        e[w] = m == -INFINITY ? 0.f : expf(m - top);
+                        tot = fmaf(part_s[(size_t)(w * 4 + qi) * stride + 1], e[w], tot);
+                    }
+                    float *dst = part_slot + (size_t)(q0 + 4 * sub + qi) * stride;
+                    if (t == 0) {
+                        dst[0] = top;
+                        dst[1] = tot;
+                    }
+                    for (int c = t; c < DH; c += 128) {
+                        float acc = 0.f;
+#pragma unroll
+                        for (int w = 0; w < 4; ++w) acc = fmaf(part_s[(size_t)(w * 4 + qi) * stride + 2 + c], e[w], acc);
+                        dst[2 + c] = acc;
+                    }
+                }
+                sync();
             }
         }
     }
 }
 
+// How a call on the tensor-core routine splits its keys: n_pre chunks of gpc prefix groups each, then the block's chunk.
+inline AttSplit att_split_mma(int cap, int L, int BH, int dh, int target)
+{
+    const int groups = (cap + 31) / 32;
+    int want = BH > 0 ? target / BH - 1 : 1;
+    if (want > kAttMaxChunks - 1) want = kAttMaxChunks - 1;
+    if (want > groups) want = groups;
+    if (want < 1) want = 1;
+    const size_t per_chunk = (size_t)BH * L * (dh + 2);
+    while (want > 1 && (size_t)(want + 1) * per_chunk > kAttPartFloats) --want;
+    AttSplit sp;
+    sp.gpc = (groups + want - 1) / want;
+    sp.n_ch = (groups + sp.gpc - 1) / sp.gpc + 1;
+    return sp;
+}
+// Whether a call can use it (the caches are bf16: a tensor-core context).
+inline bool att_mma_ok(int cap, int L, int BH, int d, int dh, const void *const *ptrs, int n_ptrs)
+{
+    if (cap < 1 || (dh != 64 && dh != 128) || (d % 8) || BH > kAttCounters) return false;
+    if ((size_t)2 * BH * L * (dh + 2) > kAttPartFloats) return false;
+    for (int i = 0; i < n_ptrs; ++i)
+        if (reinterpret_cast<uintptr_t>(ptrs[i]) & 15u) return false;
+    return true;
+}
+
 template <typename T, typename Sync, typename Out>
 __device__ __forceinline__ void att_unit(const float *q, const T *pk, const T *pv, int P, const float *kb, const float *vb, int L, int d,
-                                         int dh, int ch, int n_ch, int gpc, float *part, int *counter, float *sh, int warp, int lane,
-                                         Sync sync, Out out)
+                                         int dh, int ch, int n_ch, int gpc, int mma, float *part, int *counter, float *sh, int warp,
+                                         int lane, Sync sync, Out out)
 {
+    if constexpr (sizeof(T) == 2) {
+        if (mma) {
+            // chunks 0 .. n_ch - 2: prefix groups on tensor cores; the last chunk: the block's own keys
+            const int stride = dh + 2;
+            if (ch < n_ch - 1) {
+                float *slot = part + (size_t)ch * L * stride;
+                if (dh == 128) att_unit_mma<4>(q, pk, pv, P, L, d, ch * gpc, (ch + 1) * gpc, slot, sh, warp, lane, sync);
+                else att_unit_mma<2>(q, pk, pv, P, L, d, ch * gpc, (ch + 1) * gpc, slot, sh, warp, lane, sync);
+                att_arrive_merge(n_ch, L, dh, part, counter, sh, warp, lane, sync, out);
+            } else if (dh == 128) {
+                att_unit_per<4>(q, pk, pv, 0, kb, vb, L, d, dh, 0, 1 << 30, ch, n_ch, part, counter, sh, warp, lane, sync, out);
+            } else {
+                att_unit_per<2>(q, pk, pv, 0, kb, vb, L, d, dh, 0, 1 << 30, ch, n_ch, part, counter, sh, warp, lane, sync, out);
+            }
+            return;
+        }
+    }
     // heads of 64 or 128 features, rows 16-byte aligned: the lane's features are consecutive and load as one vector
     if (dh == 128 && (d % 8) == 0)
-        att_unit_per<4>(q, pk, pv, P, kb, vb, L, d, dh, ch, n_ch, gpc, part, counter, sh, warp, lane, sync, out);
+        att_unit_per<4>(q, pk, pv, P, kb, vb, L, d, dh, ch * gpc, (ch + 1) * gpc, ch, n_ch, part, counter, sh, warp, lane, sync, out);
     else if (dh == 64 && (d % 8) == 0)
-        att_unit_per<2>(q, pk, pv, P, kb, vb, L, d, dh, ch, n_ch, gpc, part, counter, sh, warp, lane, sync, out);
+        att_unit_per<2>(q, pk, pv, P, kb, vb, L, d, dh, ch * gpc, (ch + 1) * gpc, ch, n_ch, part, counter, sh, warp, lane, sync, out);
     else
-        att_unit_per<0>(q, pk, pv, P, kb, vb, L, d, dh, ch, n_ch, gpc, part, counter, sh, warp, lane, sync, out);
+        att_unit_per<0>(q, pk, pv, P, kb, vb, L, d, dh, ch * gpc, (ch + 1) * gpc, ch, n_ch, part, counter, sh, warp, lane, sync, out);
 }
 
 }  // namespace mrp

@@ -1246,7 +1246,7 @@ __global__ void __launch_bounds__(128) mod_attention_prefix_kernel(const float *
                                                                    int d, int dh, int H, float *__restrict__ o,
                                                                    __nv_bfloat16 *__restrict__ o16, int n_rows, T *pk, T *pv,
                                                                    const int32_t *__restrict__ plen, int cap, int append, int n_ch,
-                                                                   int gpc, float *part, int *counters,
+                                                                   int gpc, int mma, float *part, int *counters,
                                                                    int32_t *__restrict__ status, int32_t *__restrict__ user_status)
 {
     pdl_trigger();
@@ -1271,7 +1271,7 @@ __global__ void __launch_bounds__(128) mod_attention_prefix_kernel(const float *
             pv[slab + (size_t)(P + i) * d + c] = (T)v[blk + (size_t)i * d + c];
         }
     }
-    att_unit<T>(q + blk, pk + slab, pv + slab, P, k + blk, v + blk, L, d, dh, ch, n_ch, gpc,
+    att_unit<T>(q + blk, pk + slab, pv + slab, P, k + blk, v + blk, L, d, dh, ch, n_ch, gpc, mma,
                 part + (size_t)bh * n_ch * L * (dh + 2), counters + bh, att_sh, warp, lane, [] { __syncthreads(); },
                 [&](int i, int c, float val) {
                     const size_t at = blk + (size_t)i * d + c;
@@ -1867,13 +1867,20 @@ static cudaError_t module_attention(Ctx *c, int layer, int B, int L, const float
                         n_rows);
     // the keys of a (block, head) split over CTAs where there are few of those; the partial results and the arrival
     // counters (zero before and after every launch) sit behind the module's other workspace
-    const AttSplit sp = att_split(c->prefix_cap, L, B * w.n_attn_heads, dh, 8 * c->sm_count);
+    // (bf16 caches, heads of 64 or 128 features: the prefix part as small tensor-core products, the block's keys a chunk
+    // of their own)
+    const void *ptrs[2] = {c->prefix_layers[layer].k, c->prefix_layers[layer].v};
+    const bool mma = sizeof(T) == 2 && !(c->cfg.flags & MRP_FLAG_FORCE_SIMT) &&
+                     att_mma_ok(c->prefix_cap, L, B * w.n_attn_heads, d, dh, ptrs, 2);
+    const AttSplit sp = mma ? att_split_mma(c->prefix_cap, L, B * w.n_attn_heads, dh, 8 * c->sm_count)
+                            : att_split(c->prefix_cap, L, B * w.n_attn_heads, dh, 8 * c->sm_count);
     float *part = (float *)(c->module_ws + module_att_offset(c->cfg));
     int *counters = (int *)(part + kAttPartFloats);
     return launch_k(mod_attention_prefix_kernel<T>, dim3((unsigned)(B * w.n_attn_heads * sp.n_ch)), dim3(128),
                     (size_t)att_sh_floats(dh) * 4, st, pdl, q, k, v, L, d, dh, w.n_attn_heads, o, o16, n_rows,
                     (T *)c->prefix_layers[layer].k, (T *)c->prefix_layers[layer].v, c->prefix_len, c->prefix_cap,
-                    c->prefix_append ? 1 : 0, sp.n_ch, sp.gpc, part, counters, (int32_t *)(c->ws + c->lay.status), out.status);
+                    c->prefix_append ? 1 : 0, sp.n_ch, sp.gpc, mma ? 1 : 0, part, counters, (int32_t *)(c->ws + c->lay.status),
+                    out.status);
 }
 
 // The module itself (everything in front of `h <- h + Delta`) with its products on the tensor cores.

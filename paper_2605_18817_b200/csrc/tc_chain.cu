@@ -98,6 +98,7 @@ struct ModEnds {
     const int32_t *plen;     // clean prefix: rows in use per sequence, rows per slab, whether the block's own keys and
     int pcap, append;        // values are stored behind them
     int att_nch, att_gpc;    // ... chunks of the key range per (block, head), groups of 32 keys per chunk
+    int att_mma;             // ... the prefix chunks as tensor-core products, the block's keys a chunk of their own
     float *att_part;         // partial results of the chunks
     int *att_counters;       // arrivals per (block, head): zero before and after the launch
 };
@@ -771,7 +772,7 @@ sk_chain_kernel(const __grid_constant__ typename ChainTypes<MOD>::Maps maps,
                             }
                         }
                         att_unit<__nv_bfloat16>(ph.att_q + blk, ph.att_pk + slab, ph.att_pv + slab, P, ph.att_k + blk, ph.att_v + blk, L, p.d,
-                                                dh, ch, n_ch, e.att_gpc, e.att_part + (size_t)bh * n_ch * L * (dh + 2), e.att_counters + bh,
+                                                dh, ch, n_ch, e.att_gpc, e.att_mma, e.att_part + (size_t)bh * n_ch * L * (dh + 2), e.att_counters + bh,
                                                 sq_s, q, lane, [&] { ch_epi_sync(); }, [&](int i2, int cidx, float val) {
                                                     ch_store_hi_lo(ph.att_out + blk + (size_t)i2 * p.d + cidx, (size_t)p.lo_x * p.d, val);
                                                 });
@@ -1080,9 +1081,13 @@ cudaError_t sk_module_step(Ctx *c, int n, int L, const int32_t *tokens, const vo
     p.mod.xt = (__nv_bfloat16 *)(c->ws + c->lay.xt); p.mod.xt16 = f16_lm ? (__half *)(c->ws + c->lay.xt16) : nullptr;
     p.mod.hidden_out = hidden_out;
     if (c->has_prefix) {
-        const AttSplit sp = att_split(c->prefix_cap, L, (n / L) * H, d / H, G);
+        const void *ptrs[2 * kModChainLayers];
+        for (int l = 0; l < D; ++l) { ptrs[2 * l] = c->prefix_layers[l].k; ptrs[2 * l + 1] = c->prefix_layers[l].v; }
+        const bool mma = att_mma_ok(c->prefix_cap, L, (n / L) * H, d, d / H, ptrs, 2 * D);
+        const AttSplit sp = mma ? att_split_mma(c->prefix_cap, L, (n / L) * H, d / H, G) : att_split(c->prefix_cap, L, (n / L) * H, d / H, G);
         p.mod.plen = c->prefix_len; p.mod.pcap = c->prefix_cap; p.mod.append = c->prefix_append ? 1 : 0;
-        p.mod.att_nch = sp.n_ch; p.mod.att_gpc = sp.gpc; p.mod.att_part = att_part; p.mod.att_counters = att_counters;
+        p.mod.att_nch = sp.n_ch; p.mod.att_gpc = sp.gpc; p.mod.att_mma = mma ? 1 : 0;
+        p.mod.att_part = att_part; p.mod.att_counters = att_counters;
     }
     bool ok = make_map(s, &maps.m[0], xa, d, 2 * (uint64_t)r_pad, 2 * r_pad) && make_map(s, &maps.m[1], act16, F, 2 * (uint64_t)r_pad, 2 * r_pad) &&
               make_map(s, &maps.m[2], xb, d, 2 * (uint64_t)r_pad, 2 * r_pad) &&
