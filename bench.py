@@ -674,7 +674,8 @@ def run_module_workload(bench, cpu_budget_s, which=1, block_len=None, prefix=0):
         g = torch.Generator().manual_seed(13)
         host_kv = [(torch.randn((B, prefix, d), generator=g).bfloat16(), torch.randn((B, prefix, d), generator=g).bfloat16())
                    for _ in range(MODULE_LAYERS)]
-        caches = [(k.to(dev), v.to(dev)) for k, v in host_kv]
+        caches = [(binding.prefix_to_head_major(k, n_attn).to(dev), binding.prefix_to_head_major(v, n_attn).to(dev))
+                  for k, v in host_kv]
         plen = torch.full((B,), prefix, dtype=torch.int32, device=dev)
         binding.mrp_module_set_prefix(ctx, caches, plen)
     hid0 = harness.to_device(inp.hidden, "bf16", dev)

@@ -337,8 +337,9 @@ int mrp_module_step_kl(mrp_ctx *ctx, const int32_t *tokens, const void *hidden0,
  * prefix, under the attention pattern of training, where a block attends to itself and to the clean blocks in
  * front of it).  What a block sees of its prefix are the keys and values the module's own layers produced for
  * the prefix positions; the caller keeps them, per module layer, in a cache
- *     k, v   DEVICE [max_seqs, prefix_cap, d], context dtype, 16-byte aligned
- * of which sequence b (the b-th block of an mrp_module_step call) uses the first prefix_len[b] rows:
+ *     k, v   DEVICE [max_seqs, n_attn_heads, prefix_cap, d / n_attn_heads], context dtype, 16-byte aligned
+ *            (head-major: the rows an attention head reads are one contiguous run)
+ * of which sequence b (the b-th block of an mrp_module_step call) uses the first prefix_len[b] rows per head:
  * position i of block b then attends to those rows and to the L positions of its block in one softmax.
  *   layers      HOST array [n_layers] of the caches' DEVICE pointers (copied); NULL detaches the prefix
  *   prefix_len  DEVICE [max_seqs] int32, read by every following mrp_module_step (the caller may change the
@@ -346,7 +347,7 @@ int mrp_module_step_kl(mrp_ctx *ctx, const int32_t *tokens, const void *hidden0,
  *               clamped
  *   append      != 0: every following mrp_module_step also stores the keys and values of its own L positions,
  *               rounded to the context dtype, in rows prefix_len[b] .. prefix_len[b] + L - 1 of sequence b's
- *               slab (what the caller does once a block is committed, with all its tokens revealed, before it
+ *               slabs (what the caller does once a block is committed, with all its tokens revealed, before it
  *               raises prefix_len[b] by L); a block that does not fit raises MRP_DEV_BAD_INDEX and stores
  *               nothing.  The rows stored by a call are not among the rows it reads.
  * Needs d / n_attn_heads <= 256.  With a prefix attached the module step runs as one cooperative tensor-core

@@ -358,11 +358,23 @@ def mrp_module_step_kl(ctx: Context, tokens, hidden0, h_state, logits0, teacher,
         raise MrpError("mrp_module_step_kl", rc, lib.mrp_last_error(ctx.handle).decode())
 
 
+def prefix_to_head_major(x, n_attn_heads: int):
+    """[sequences, positions, d] -> the cache layout [sequences, heads, positions, d / heads] (a contiguous copy)."""
+    B, cap, d = x.shape
+    return x.view(B, cap, n_attn_heads, d // n_attn_heads).permute(0, 2, 1, 3).contiguous()
+
+
+def prefix_from_head_major(x):
+    """The inverse of prefix_to_head_major."""
+    B, H, cap, dh = x.shape
+    return x.permute(0, 2, 1, 3).reshape(B, cap, H * dh)
+
+
 def mrp_module_set_prefix(ctx: Context, caches, prefix_len, append=False) -> None:
     """Attach the clean prefix of the module's attention: ``caches`` a list (one entry per module layer) of
-    (k, v) CUDA tensors [max_seqs, prefix_cap, d] in the context dtype, ``prefix_len`` [max_seqs] int32 on the
-    device; ``caches`` None detaches.  With ``append`` the following steps also store their own keys and values
-    behind the prefix rows."""
+    (k, v) CUDA tensors [max_seqs, n_attn_heads, prefix_cap, d / n_attn_heads] (head-major) in the context dtype,
+    ``prefix_len`` [max_seqs] int32 on the device; ``caches`` None detaches.  With ``append`` the following steps also
+    store their own keys and values behind the prefix rows."""
     if caches is None:
         rc = lib.mrp_module_set_prefix(ctx.handle, None, None, 0, 0)
         if rc != 0:
@@ -375,9 +387,9 @@ def mrp_module_set_prefix(ctx: Context, caches, prefix_len, append=False) -> Non
     for i, (k, v) in enumerate(caches):
         _check(k, tdtype, "prefix k")
         _check(v, tdtype, "prefix v")
-        if k.dim() != 3 or k.shape != v.shape or k.shape[2] != ctx.cfg.d:
-            raise ValueError("prefix caches are [max_seqs, prefix_cap, d]")
-        cap = int(k.shape[1])
+        if k.dim() != 4 or k.shape != v.shape or k.shape[1] * k.shape[3] != ctx.cfg.d:
+            raise ValueError("prefix caches are [max_seqs, n_attn_heads, prefix_cap, d / n_attn_heads]")
+        cap = int(k.shape[2])
         arr[i] = mrp_module_kv(k.data_ptr(), v.data_ptr())
     rc = lib.mrp_module_set_prefix(ctx.handle, arr, _ptr(prefix_len), cap, int(bool(append)))
     if rc != 0:

@@ -94,7 +94,8 @@ struct Ctx {
     mrp_module_layer *module_layers;   // host copy [n_layers]
     char *module_ws;
     // the clean prefix of the module's attention (mrp_module_set_prefix): per layer the device pointers of the
-    // key / value cache [max_seqs][prefix_cap][d] (context dtype), host copy; lengths per sequence on the device
+    // key / value cache [max_seqs][n_attn_heads][prefix_cap][d / n_attn_heads] (context dtype), host copy; lengths per
+    // sequence on the device
     bool has_prefix;
     mrp_module_kv *prefix_layers;
     const int32_t *prefix_len;
@@ -329,7 +330,7 @@ __device__ inline Partial merge_partial(const Partial &a, const Partial &b)
 
 // ---- the module's attention behind a clean prefix (Fig. 1(c)) ------------------------------------------------
 // Work unit = (block b, attention head, chunk of the key range), run by the four warps of a CTA (or of its epilogue
-// warpgroup).  Keys and values: the first P rows of the sequence's slab of the prefix cache (type T, written by
+// warpgroup).  Keys and values: the first P rows of the (sequence, head) slab of the prefix cache (type T, written by
 // earlier calls, read through the read-only path), then the L rows of the block (fp32, possibly written earlier in
 // this same kernel: read from L2).  The keys go in groups of 32 (prefix groups, then block groups); chunk ch covers
 // groups [ch * gpc, (ch + 1) * gpc) and its warps take them round-robin: a lane per key for the scores of kAttQT
@@ -337,8 +338,8 @@ __device__ inline Partial merge_partial(const Partial &a, const Partial &b)
 // values, with a running maximum and sum per query.  The four warps' partial results meet in shared memory; with
 // more than one chunk the chunk's partial results go to `part` and the CTA that arrives last at the (block, head)
 // counter merges them -- no CTA waits for another.
-//   q, kb, vb   the block's first row of q / k / v at the head's columns; pk, pv the slab's first row there;
-//               d = row stride of all of them
+//   q, kb, vb   the block's first row of q / k / v at the head's columns, row stride d; pk, pv the first row of the
+//               (sequence, head) slab of the cache, whose rows are the head's dh features, one after the other
 //   part        [n_ch][L][dh + 2] floats of this (block, head); counter: its arrival counter, zero before and after
 //   sh          att_sh_floats(dh) floats of shared memory, 16-byte aligned;  sync(): a barrier over exactly these
 //               128 threads;  out(i, c, value) is called once per query i of the block and feature c of the head
@@ -587,7 +588,7 @@ __device__ __forceinline__ void att_unit_per(const float *q, const T *pk, const 
     for (int g = g_lo + warp; g < g_end && g < gp; g += 4) {
         const int j = g * 32 + lane;
         if (j < P) {
-            const char *rk = reinterpret_cast<const char *>(pk + (size_t)j * d), *rv = reinterpret_cast<const char *>(pv + (size_t)j * d);
+            const char *rk = reinterpret_cast<const char *>(pk + (size_t)j * dh), *rv = reinterpret_cast<const char *>(pv + (size_t)j * dh);
             for (int off = 0; off < dh * (int)sizeof(T); off += 128) {
                 asm volatile("prefetch.global.L2 [%0];" ::"l"(rk + off));
                 asm volatile("prefetch.global.L2 [%0];" ::"l"(rv + off));
@@ -612,7 +613,7 @@ __device__ __forceinline__ void att_unit_per(const float *q, const T *pk, const 
         for (int g = g_lo + warp; g < g_end; g += 4) {
             if (g < gp) {
                 const int j0 = g * 32, left = P - j0;
-                att_group<PER, false>(q_s, pk + (size_t)j0 * d, pv + (size_t)j0 * d, left < 32 ? left : 32, d, dh, vec, scale, lane, mx, sum,
+                att_group<PER, false>(q_s, pk + (size_t)j0 * dh, pv + (size_t)j0 * dh, left < 32 ? left : 32, dh, dh, vec, scale, lane, mx, sum,
                                       oacc);
             } else {
                 const int j0 = (g - gp) * 32, left = L - j0;
@@ -713,6 +714,17 @@ __device__ __forceinline__ void att_unit_mma(const float *q, const __nv_bfloat16
     const float scale = rsqrtf((float)DH);
     const int gp = (P + 31) / 32;
     if (g_hi > gp) g_hi = gp;
+    if (g_lo < g_hi) {
+        // the chunk's rows (one contiguous run per tensor in the head-major cache) asked into L2 up front: a group then
+        // pays the L2 latency three times (keys, two halves of the values), not the DRAM latency
+        const int row_hi = g_hi * 32 < P ? g_hi * 32 : P;
+        const char *k0 = reinterpret_cast<const char *>(pk + (size_t)g_lo * 32 * DH), *v0 = reinterpret_cast<const char *>(pv + (size_t)g_lo * 32 * DH);
+        const size_t bytes = (size_t)(row_hi - g_lo * 32) * DH * 2;
+        for (size_t off = (size_t)t * 128; off < bytes; off += 128 * 128) {
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(k0 + off));
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(v0 + off));
+        }
+    }
     for (int q0 = 0; q0 < L; q0 += 16) {
         const int nq = L - q0 < 16 ? L - q0 : 16;
         for (int x = t; x < 16 * DH; x += 128) {
@@ -745,7 +757,7 @@ __device__ __forceinline__ void att_unit_mma(const float *q, const __nv_bfloat16
 #pragma unroll
                 for (int tt = 0; tt < 4; ++tt) {
                     const int key = 8 * tt + r < cnt ? 8 * tt + r : cnt - 1;
-                    kk[tt] = __ldg(reinterpret_cast<const uint4 *>(pk + (size_t)(j0 + key) * d + 32 * s + 8 * j));
+                    kk[tt] = __ldg(reinterpret_cast<const uint4 *>(pk + (size_t)(j0 + key) * DH + 32 * s + 8 * j));
                 }
                 const uint4 ah0 = *reinterpret_cast<const uint4 *>(q_hi + r * QS + 32 * s + 8 * j);
                 const uint4 ah1 = *reinterpret_cast<const uint4 *>(q_hi + (r + 8) * QS + 32 * s + 8 * j);
@@ -810,8 +822,8 @@ __device__ __forceinline__ void att_unit_mma(const float *q, const __nv_bfloat16
                 uint4 va[NG], vb[NG];
 #pragma unroll
                 for (int a = 0; a < NG; ++a) {
-                    va[a] = __ldg(reinterpret_cast<const uint4 *>(pv + (size_t)(j0 + k0) * d + 32 * a + 8 * j));
-                    vb[a] = __ldg(reinterpret_cast<const uint4 *>(pv + (size_t)(j0 + k1) * d + 32 * a + 8 * j));
+                    va[a] = __ldg(reinterpret_cast<const uint4 *>(pv + (size_t)(j0 + k0) * DH + 32 * a + 8 * j));
+                    vb[a] = __ldg(reinterpret_cast<const uint4 *>(pv + (size_t)(j0 + k1) * DH + 32 * a + 8 * j));
                 }
 #pragma unroll
                 for (int a = 0; a < NG; ++a)
@@ -902,12 +914,13 @@ inline bool att_mma_ok(int cap, int L, int BH, int d, int dh, const void *const 
     return true;
 }
 
-template <typename T, typename Sync, typename Out>
+// (MMA: whether the kernel carries the tensor-core routine at all: it costs registers)
+template <typename T, bool MMA, typename Sync, typename Out>
 __device__ __forceinline__ void att_unit(const float *q, const T *pk, const T *pv, int P, const float *kb, const float *vb, int L, int d,
                                          int dh, int ch, int n_ch, int gpc, int mma, float *part, int *counter, float *sh, int warp,
                                          int lane, Sync sync, Out out)
 {
-    if constexpr (sizeof(T) == 2) {
+    if constexpr (MMA && sizeof(T) == 2) {
         if (mma) {
             // chunks 0 .. n_ch - 2: prefix groups on tensor cores; the last chunk: the block's own keys
             const int stride = dh + 2;

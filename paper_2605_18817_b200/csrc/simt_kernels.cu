@@ -1239,7 +1239,7 @@ __global__ void mod_attention_kernel(const float *__restrict__ q, const float *_
 }
 
 // The same behind a clean prefix (Fig. 1(c)): CTA = (block, attention head, chunk of the keys); keys and values are
-// the first prefix_len[b] rows of sequence b's slab of the cache [*, cap, d], then the block's own rows.  With `append`
+// the first prefix_len[b] rows of the (sequence b, head) slab of the cache [*, H, cap, dh], then the block's own rows.  With `append`
 // the block's keys and values are also stored behind the prefix rows (rows the call itself never reads).
 template <typename T>
 __global__ void __launch_bounds__(128) mod_attention_prefix_kernel(const float *__restrict__ q, const float *k, const float *v, int L,
@@ -1263,15 +1263,15 @@ __global__ void __launch_bounds__(128) mod_attention_prefix_kernel(const float *
         atomicOr(status, MRP_DEV_BAD_INDEX);
         if (user_status) atomicOr(user_status, MRP_DEV_BAD_INDEX);
     }
-    const size_t head = (size_t)hd * dh, slab = (size_t)b * cap * d + head, blk = (size_t)b * L * d + head;
+    const size_t head = (size_t)hd * dh, slab = ((size_t)b * H + hd) * cap * dh, blk = (size_t)b * L * d + head;
     if (store && ch == 0) {
         for (int x = threadIdx.x; x < L * dh; x += 128) {
             const int i = x / dh, c = x - i * dh;
-            pk[slab + (size_t)(P + i) * d + c] = (T)k[blk + (size_t)i * d + c];
-            pv[slab + (size_t)(P + i) * d + c] = (T)v[blk + (size_t)i * d + c];
+            pk[slab + (size_t)(P + i) * dh + c] = (T)k[blk + (size_t)i * d + c];
+            pv[slab + (size_t)(P + i) * dh + c] = (T)v[blk + (size_t)i * d + c];
         }
     }
-    att_unit<T>(q + blk, pk + slab, pv + slab, P, k + blk, v + blk, L, d, dh, ch, n_ch, gpc, mma,
+    att_unit<T, false>(q + blk, pk + slab, pv + slab, P, k + blk, v + blk, L, d, dh, ch, n_ch, gpc, mma,
                 part + (size_t)bh * n_ch * L * (dh + 2), counters + bh, att_sh, warp, lane, [] { __syncthreads(); },
                 [&](int i, int c, float val) {
                     const size_t at = blk + (size_t)i * d + c;
@@ -1867,13 +1867,10 @@ static cudaError_t module_attention(Ctx *c, int layer, int B, int L, const float
                         n_rows);
     // the keys of a (block, head) split over CTAs where there are few of those; the partial results and the arrival
     // counters (zero before and after every launch) sit behind the module's other workspace
-    // (bf16 caches, heads of 64 or 128 features: the prefix part as small tensor-core products, the block's keys a chunk
-    // of their own)
-    const void *ptrs[2] = {c->prefix_layers[layer].k, c->prefix_layers[layer].v};
-    const bool mma = sizeof(T) == 2 && !(c->cfg.flags & MRP_FLAG_FORCE_SIMT) &&
-                     att_mma_ok(c->prefix_cap, L, B * w.n_attn_heads, d, dh, ptrs, 2);
-    const AttSplit sp = mma ? att_split_mma(c->prefix_cap, L, B * w.n_attn_heads, dh, 8 * c->sm_count)
-                            : att_split(c->prefix_cap, L, B * w.n_attn_heads, dh, 8 * c->sm_count);
+    // (this kernel keeps the CUDA-core routine: with three CTAs per SM it is as fast here as the tensor-core routine of
+    // the one-kernel step, which takes 248 registers)
+    const bool mma = false;
+    const AttSplit sp = att_split(c->prefix_cap, L, B * w.n_attn_heads, dh, 8 * c->sm_count);
     float *part = (float *)(c->module_ws + module_att_offset(c->cfg));
     int *counters = (int *)(part + kAttPartFloats);
     return launch_k(mod_attention_prefix_kernel<T>, dim3((unsigned)(B * w.n_attn_heads * sp.n_ch)), dim3(128),

@@ -77,7 +77,7 @@ struct ChainPhase {
     const float *att_q, *att_k, *att_v;
     __nv_bfloat16 *att_out;
     int att_L, att_H;
-    __nv_bfloat16 *att_pk, *att_pv;  // the layer's clean-prefix cache [*, pcap, d] (nullptr: block-local attention)
+    __nv_bfloat16 *att_pk, *att_pv;  // the layer's clean-prefix cache [*, H, pcap, dh] (nullptr: block-local attention)
     int zero_slot0, zero_slot1;      // ssq_fix slots this phase clears for later phases of the launch (< 0: none)
     int fin;                         // LIN that completes Delta: its finish also does h <- h + Delta and the LM-head operand
 };
@@ -763,15 +763,15 @@ sk_chain_kernel(const __grid_constant__ typename ChainTypes<MOD>::Maps maps,
                             atomicOr(p.status, MRP_DEV_BAD_INDEX);
                             if (p.user_status) atomicOr(p.user_status, MRP_DEV_BAD_INDEX);
                         }
-                        const size_t head = (size_t)hd * dh, slab = (size_t)b * e.pcap * p.d + head, blk = (size_t)b * L * p.d + head;
+                        const size_t head = (size_t)hd * dh, slab = ((size_t)b * H + hd) * e.pcap * dh, blk = (size_t)b * L * p.d + head;
                         if (store && ch == 0) {       // rows this call never reads
                             for (int x = t; x < L * dh; x += 128) {
                                 const int i2 = x / dh, cidx = x - i2 * dh;
-                                ph.att_pk[slab + (size_t)(P + i2) * p.d + cidx] = __float2bfloat16_rn(__ldcg(ph.att_k + blk + (size_t)i2 * p.d + cidx));
-                                ph.att_pv[slab + (size_t)(P + i2) * p.d + cidx] = __float2bfloat16_rn(__ldcg(ph.att_v + blk + (size_t)i2 * p.d + cidx));
+                                ph.att_pk[slab + (size_t)(P + i2) * dh + cidx] = __float2bfloat16_rn(__ldcg(ph.att_k + blk + (size_t)i2 * p.d + cidx));
+                                ph.att_pv[slab + (size_t)(P + i2) * dh + cidx] = __float2bfloat16_rn(__ldcg(ph.att_v + blk + (size_t)i2 * p.d + cidx));
                             }
                         }
-                        att_unit<__nv_bfloat16>(ph.att_q + blk, ph.att_pk + slab, ph.att_pv + slab, P, ph.att_k + blk, ph.att_v + blk, L, p.d,
+                        att_unit<__nv_bfloat16, true>(ph.att_q + blk, ph.att_pk + slab, ph.att_pv + slab, P, ph.att_k + blk, ph.att_v + blk, L, p.d,
                                                 dh, ch, n_ch, e.att_gpc, e.att_mma, e.att_part + (size_t)bh * n_ch * L * (dh + 2), e.att_counters + bh,
                                                 sq_s, q, lane, [&] { ch_epi_sync(); }, [&](int i2, int cidx, float val) {
                                                     ch_store_hi_lo(ph.att_out + blk + (size_t)i2 * p.d + cidx, (size_t)p.lo_x * p.d, val);

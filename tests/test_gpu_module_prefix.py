@@ -32,6 +32,16 @@ def make_prefix(D, B, cap, d, plen, dtype, seed, poison=True):
     return caches
 
 
+def to_dev(host, heads):
+    """The caches in the library's head-major layout, on the device."""
+    return [(binding.prefix_to_head_major(k, heads).to(DEV), binding.prefix_to_head_major(v, heads).to(DEV)) for k, v in host]
+
+
+def from_dev(t):
+    """A device cache back in [sequences, positions, d] on the host."""
+    return binding.prefix_from_head_major(t.cpu())
+
+
 def as_oracle_prefix(caches, plen):
     ks = [np.nan_to_num(k.float().numpy(), nan=0.0) for k, _ in caches]
     vs = [np.nan_to_num(v.float().numpy(), nan=0.0) for _, v in caches]
@@ -66,7 +76,7 @@ def test_module_step_behind_a_prefix_follows_the_oracle(dtype, flags, d, F, V, D
     emb, w_proj, layers = upload_module(mw, dtype)
     binding.mrp_module_attach(ctx, emb, w_proj, layers, heads, mw.mask_token)
     host = make_prefix(D, B, cap, d, plen, dtype, 5)
-    dev = [(k.to(DEV), v.to(DEV)) for k, v in host]
+    dev = to_dev(host, heads)
     plen_d = torch.tensor(plen, dtype=torch.int32, device=DEV)
     binding.mrp_module_set_prefix(ctx, dev, plen_d)
     hid0 = harness.to_device(inp.hidden, dtype, DEV)
@@ -103,7 +113,8 @@ def test_module_step_behind_a_prefix_follows_the_oracle(dtype, flags, d, F, V, D
     assert np.array_equal(g_tok[1][clear], tok[clear])
     # the caches were only read
     for (k, v), (hk, hv) in zip(dev, host):
-        assert torch.equal(k.cpu().view(torch.uint8), hk.view(torch.uint8)) and torch.equal(v.cpu().view(torch.uint8), hv.view(torch.uint8))
+        assert torch.equal(from_dev(k).contiguous().view(torch.uint8), hk.view(torch.uint8))
+        assert torch.equal(from_dev(v).contiguous().view(torch.uint8), hv.view(torch.uint8))
     # detached again, the step is the block-local one
     binding.mrp_module_set_prefix(ctx, None, None)
     binding.mrp_module_step(ctx, torch.from_numpy(tokens).to(DEV), hid0, h_state, l0, torch.from_numpy(ri).to(DEV), M, B, L, True,
@@ -134,7 +145,7 @@ def test_committed_block_is_appended_and_serves_the_next_block(dtype, flags, d, 
     emb, w_proj, layers = upload_module(mw, dtype)
     binding.mrp_module_attach(ctx, emb, w_proj, layers, heads, mw.mask_token)
     host = make_prefix(D, B, cap, d, plen, dtype, 6, poison=False)
-    dev = [(k.to(DEV), v.to(DEV)) for k, v in host]
+    dev = to_dev(host, heads)
     plen_d = torch.tensor(plen, dtype=torch.int32, device=DEV)
     binding.mrp_module_set_prefix(ctx, dev, plen_d, append=True)
     rng = np.random.default_rng(4)
@@ -151,7 +162,7 @@ def test_committed_block_is_appended_and_serves_the_next_block(dtype, flags, d, 
     rel = 2.0 ** -8 if dtype == "bf16" else 1e-5
     grown = []
     for l, ((k, v), (hk, hv)) in enumerate(zip(dev, host)):
-        gk, gv = k.cpu().float().numpy(), v.cpu().float().numpy()
+        gk, gv = from_dev(k).float().numpy(), from_dev(v).float().numpy()
         wk, wv = hk.float().numpy().copy(), hv.float().numpy().copy()
         mask = np.zeros((B, cap), bool)
         for b in range(B):
@@ -199,7 +210,7 @@ def test_prefix_lengths_are_checked_on_the_device(dtype, B, L, d, heads):
     emb, w_proj, layers = upload_module(mw, dtype)
     binding.mrp_module_attach(ctx, emb, w_proj, layers, heads, mw.mask_token)
     host = make_prefix(D, B, cap, d, [cap, cap], dtype, 7, poison=False)
-    dev = [(k.to(DEV), v.to(DEV)) for k, v in host]
+    dev = to_dev(host, heads)
     hid0 = harness.to_device(inp.hidden, dtype, DEV)
     l0 = torch.from_numpy(inp.logits0).to(DEV)
     tok = torch.full((n,), -1, device=DEV, dtype=torch.int32)
@@ -227,6 +238,7 @@ def test_prefix_lengths_are_checked_on_the_device(dtype, B, L, d, heads):
     assert st == binding.MRP_DEV_BAD_INDEX
     for (k, v), (bk, bv) in zip(dev, before):
         assert torch.equal(k[0], bk[0]) and torch.equal(v[0], bv[0])
+        k, bk = from_dev(k), from_dev(bk)
         assert not torch.equal(k[1, 3:3 + L], bk[1, 3:3 + L]) and torch.equal(k[1, 3 + L:], bk[1, 3 + L:]) and torch.equal(k[1, :3], bk[1, :3])
     binding.mrp_destroy(ctx)
 
@@ -256,7 +268,7 @@ def test_random_shapes_behind_random_prefixes(seed):
         emb, w_proj, layers = upload_module(mw, dtype)
         binding.mrp_module_attach(ctx, emb, w_proj, layers, heads, mw.mask_token)
         host = make_prefix(D, B, cap, d, plen, dtype, 300 + case)
-        dev = [(k.to(DEV), v.to(DEV)) for k, v in host]
+        dev = to_dev(host, heads)
         binding.mrp_module_set_prefix(ctx, dev, torch.tensor(plen, dtype=torch.int32, device=DEV))
         tokens = np.where(rng.random(n) < 0.5, rng.integers(0, V - 1, n), -1).astype(np.int32)
         tokens[int(rng.integers(0, n))] = -1
@@ -303,7 +315,7 @@ def test_prefix_at_the_benchmark_shapes(which, L, P, blocks_checked):
                               n_attn, mw.mask_token)
     plen = [P - (b % 3) for b in range(B)]
     host = make_prefix(D, B, P, d, plen, "bf16", 13)
-    dev = [(k.to(DEV), v.to(DEV)) for k, v in host]
+    dev = to_dev(host, n_attn)
     binding.mrp_module_set_prefix(ctx, dev, torch.tensor(plen, dtype=torch.int32, device=DEV))
     tokens = np.full(n, -1, np.int32)
     tokens[::L] = 17
