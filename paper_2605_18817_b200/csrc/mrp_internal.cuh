@@ -751,6 +751,16 @@ __device__ __forceinline__ void att_unit_mma(const float *q, const __nv_bfloat16
             for (int a = 0; a < 4; ++a)
 #pragma unroll
                 for (int b = 0; b < 4; ++b) sacc[a][b] = 0.f;
+            // the value rows of the first 16 keys are asked for together with the keys: one round of loads less
+            uint4 va0[NG], vb0[NG];
+            {
+                const int k0 = r < cnt ? r : cnt - 1, k1 = 8 + r < cnt ? 8 + r : cnt - 1;
+#pragma unroll
+                for (int a = 0; a < NG; ++a) {
+                    va0[a] = __ldg(reinterpret_cast<const uint4 *>(pv + (size_t)(j0 + k0) * DH + 32 * a + 8 * j));
+                    vb0[a] = __ldg(reinterpret_cast<const uint4 *>(pv + (size_t)(j0 + k1) * DH + 32 * a + 8 * j));
+                }
+            }
 #pragma unroll
             for (int s = 0; s < NG; ++s) {
                 uint4 kk[4];
@@ -822,8 +832,13 @@ __device__ __forceinline__ void att_unit_mma(const float *q, const __nv_bfloat16
                 uint4 va[NG], vb[NG];
 #pragma unroll
                 for (int a = 0; a < NG; ++a) {
-                    va[a] = __ldg(reinterpret_cast<const uint4 *>(pv + (size_t)(j0 + k0) * DH + 32 * a + 8 * j));
-                    vb[a] = __ldg(reinterpret_cast<const uint4 *>(pv + (size_t)(j0 + k1) * DH + 32 * a + 8 * j));
+                    if (u == 0) {
+                        va[a] = va0[a];
+                        vb[a] = vb0[a];
+                    } else {
+                        va[a] = __ldg(reinterpret_cast<const uint4 *>(pv + (size_t)(j0 + k0) * DH + 32 * a + 8 * j));
+                        vb[a] = __ldg(reinterpret_cast<const uint4 *>(pv + (size_t)(j0 + k1) * DH + 32 * a + 8 * j));
+                    }
                 }
 #pragma unroll
                 for (int a = 0; a < NG; ++a)
