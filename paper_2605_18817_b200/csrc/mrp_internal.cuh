@@ -761,14 +761,19 @@ __device__ __forceinline__ void att_unit_mma(const float *q, const __nv_bfloat16
                     vb0[a] = __ldg(reinterpret_cast<const uint4 *>(pv + (size_t)(j0 + k1) * DH + 32 * a + 8 * j));
                 }
             }
+            // every key row piece of the group in flight at once (the products below would otherwise wait for them
+            // one 32-feature step at a time)
+            uint4 kall[NG][4];
+#pragma unroll
+            for (int tt = 0; tt < 4; ++tt) {
+                const int key = 8 * tt + r < cnt ? 8 * tt + r : cnt - 1;
+#pragma unroll
+                for (int s = 0; s < NG; ++s)
+                    kall[s][tt] = __ldg(reinterpret_cast<const uint4 *>(pk + (size_t)(j0 + key) * DH + 32 * s + 8 * j));
+            }
 #pragma unroll
             for (int s = 0; s < NG; ++s) {
-                uint4 kk[4];
-#pragma unroll
-                for (int tt = 0; tt < 4; ++tt) {
-                    const int key = 8 * tt + r < cnt ? 8 * tt + r : cnt - 1;
-                    kk[tt] = __ldg(reinterpret_cast<const uint4 *>(pk + (size_t)(j0 + key) * DH + 32 * s + 8 * j));
-                }
+                const uint4 *kk = kall[s];
                 const uint4 ah0 = *reinterpret_cast<const uint4 *>(q_hi + r * QS + 32 * s + 8 * j);
                 const uint4 ah1 = *reinterpret_cast<const uint4 *>(q_hi + (r + 8) * QS + 32 * s + 8 * j);
                 const uint4 al0 = *reinterpret_cast<const uint4 *>(q_lo + r * QS + 32 * s + 8 * j);
